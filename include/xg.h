@@ -1,0 +1,208 @@
+/*
+ * xg.h -- C ABI of the token-mask library (byte-level Earley, CUDA sm_100a).
+ *
+ * The library implements the data-parallel part of grammar-constrained decoding as described in
+ * "XGrammar-2" (arXiv 2601.04426): checking every vocabulary token against a byte-level Earley
+ * grammar state.  That happens in two places:
+ *   - at compile time, filling the adaptive token mask cache: every (scannable grammar state,
+ *     token) pair is classified accepted / rejected / uncertain (Section 3.4; appendix
+ *     "XGrammar's Adaptive Token Mask cache Generation Algorithm");
+ *   - at every decode step, merging the cached sets of the current scannable states with a full
+ *     Earley check of the uncertain tokens (same appendix, run-time paragraph), and setting the
+ *     logits of disallowed tokens to -inf (Section 2.1).
+ *
+ * Conventions
+ *   - Every function returns an xg_status_t (0 = XG_OK, negative = error) and never throws,
+ *     aborts or traps the device.  xg_last_error() returns a thread-local message for the last
+ *     failing call on the calling thread.
+ *   - Handles are opaque; the library creates them and the caller destroys them with the
+ *     matching *_destroy.  Destroy matchers before their grammar, grammars before their
+ *     tokenizer and cache pool.
+ *   - "device" pointers are CUDA device memory of the current device, owned by the caller and
+ *     never freed or retained past the call's stream order.  "host" pointers are ordinary memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls that take a
+ *     stream only enqueue work on it unless stated otherwise.
+ *   - Bitmask layout: row-major int32 words, bit j (LSB first) of word w of a row is token id
+ *     32*w + j; 1 = allowed.  Bits of ids >= vocab_size are 0.
+ */
+#ifndef XG_H_
+#define XG_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t xg_status_t;
+enum {
+  XG_OK = 0,
+  XG_ERR_INVALID_ARG = -1,
+  XG_ERR_PARSE = -2,          /* grammar / schema text is malformed */
+  XG_ERR_UNSUPPORTED = -3,    /* schema keyword or construct outside the supported subset */
+  XG_ERR_OOM = -4,
+  XG_ERR_CUDA = -5,           /* a CUDA runtime call failed, or no usable device */
+  XG_ERR_CAPACITY = -6,       /* a fixed-capacity structure (item sets, history) overflowed */
+  XG_ERR_TOKEN_REJECTED = -7, /* xg_accept_token: the token is not allowed in this state */
+  XG_ERR_TERMINATED = -8,     /* the matcher already accepted EOS */
+  XG_ERR_TIMEOUT = -9
+};
+
+typedef enum { XG_EBNF = 0, XG_JSON_SCHEMA = 1, XG_TAG_DISPATCH_JSON = 2 } xg_grammar_kind_t;
+typedef enum { XG_F32 = 0, XG_BF16 = 1 } xg_dtype_t;
+/* how the accepted/rejected split of one cache entry is stored (the smallest of the three) */
+typedef enum { XG_STORE_ACCEPT_LIST = 0, XG_STORE_REJECT_LIST = 1, XG_STORE_BITSET = 2 } xg_store_kind_t;
+
+typedef struct xg_tokenizer xg_tokenizer_t;
+typedef struct xg_cache_pool xg_cache_pool_t;
+typedef struct xg_grammar xg_grammar_t;
+typedef struct xg_matcher xg_matcher_t;
+
+/* Message of the last failing call on this thread ("" if none).  Valid until the next call. */
+const char* xg_last_error(void);
+
+/* ---- vocabulary ---------------------------------------------------------------------------
+ * The token set V of the tokenizer (appendix "Formal Definitions": V is the vocabulary).
+ * bytes/offsets (host): token i is bytes[offsets[i] .. offsets[i+1]).  eos_token_id = -1 for none.
+ * special_ids (host, may be NULL): tokens that are never allowed.  Zero-length tokens are never
+ * allowed either (EOS is decided separately).  Tokens longer than 255 bytes are refused
+ * (XG_ERR_UNSUPPORTED).  The library copies everything; it stores the tokens on the device
+ * sorted by their bytes (trie order) with the permutation back to ids.  Synchronous. */
+xg_status_t xg_tokenizer_create(const uint8_t* bytes, const int64_t* offsets, int32_t vocab_size,
+                                int32_t eos_token_id, const int32_t* special_ids, int32_t n_special,
+                                void* stream, xg_tokenizer_t** out);
+void xg_tokenizer_destroy(xg_tokenizer_t* tok);
+
+/* ---- cross-grammar cache pool (Section 3.3) -----------------------------------------------
+ * Cache entries are keyed by the structural hash of the rule automaton they belong to
+ * (Algorithm 1; Algorithm 2 for cycles) and verified against the canonical serialisation, so
+ * identical sub-structures in different grammars, or inside one grammar, are built once.
+ * A pool belongs to one tokenizer and must outlive the grammars compiled with it. */
+xg_status_t xg_cache_pool_create(const xg_tokenizer_t* tok, xg_cache_pool_t** out);
+void xg_cache_pool_destroy(xg_cache_pool_t* pool);
+
+typedef struct {
+  uint32_t struct_size;       /* sizeof(xg_compile_options_t), for versioning */
+  int32_t inline_max_states;  /* inline non-recursive rules whose automaton has at most this many
+                                 states into their users; 0 = never; negative = default (12). */
+  int32_t max_rule_states;    /* XG_ERR_CAPACITY if one rule's automaton grows past this.  <= 0 = default (1<<20). */
+  int32_t build_cache;        /* 0 = front end only (tables, no device work).  Otherwise build. */
+} xg_compile_options_t;
+
+/* ---- grammar compilation (Section 3.5 "compilation stage"; Sections 3.2, 3.3, 3.4) ---------
+ * Parses `text` (EBNF with the TagDispatch intrinsic, a JSON schema, or a TagDispatch spec in
+ * JSON), lowers it to one byte-level automaton per rule with byte-class and rule-reference edges
+ * (Section 3.3), and fills the adaptive token mask cache on the GPU: for every scannable state
+ * and every token, accepted / rejected / uncertain, stored as the smallest of accepted list,
+ * rejected list or bitset, plus the uncertain list (Section 3.4).
+ * tok == NULL (or opt->build_cache == 0): front end only; the result can be inspected with
+ * xg_grammar_get_tables but cannot make matchers, and no CUDA call is made.
+ * pool may be NULL (a private pool is used).  root_rule: EBNF only, NULL = "root".
+ * Synchronous: the cache is complete when the call returns.
+ * Errors: XG_ERR_PARSE, XG_ERR_UNSUPPORTED, XG_ERR_CAPACITY, XG_ERR_CUDA, XG_ERR_OOM. */
+xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool, xg_grammar_kind_t kind,
+                               const char* text, size_t len, const char* root_rule,
+                               const xg_compile_options_t* opt, void* stream, xg_grammar_t** out);
+void xg_grammar_destroy(xg_grammar_t* g);
+
+/* Flattened rule and byte-class tables (host copies, valid until the grammar is destroyed).
+ * Rule r is an automaton over states; state s belongs to rule state_rule[s]; rule_start[r] is
+ * its start state; state_final[s] != 0 marks accepting states.  Byte-class edges of s are
+ * cedge_class/cedge_target[cedge_begin[s] .. cedge_begin[s+1]); rule-reference edges are
+ * redge_rule/redge_target[redge_begin[s] .. redge_begin[s+1]).  Class c contains byte b iff bit
+ * (b & 31) of class_bits[8*c + (b >> 5)] is set.  No rule accepts the empty string (references
+ * to such rules have been bypassed); root_nullable says whether the root rule originally did.
+ * A state is scannable iff it has at least one byte-class edge. */
+typedef struct {
+  int32_t n_rules, n_states, n_classes, n_class_edges, n_ref_edges;
+  int32_t root_rule, root_nullable;
+  const int32_t* rule_start;
+  const int32_t* state_rule;
+  const uint8_t* state_final;
+  const int32_t* cedge_begin;
+  const int32_t* cedge_class;
+  const int32_t* cedge_target;
+  const int32_t* redge_begin;
+  const int32_t* redge_rule;
+  const int32_t* redge_target;
+  const uint32_t* class_bits;
+} xg_grammar_tables_t;
+xg_status_t xg_grammar_get_tables(const xg_grammar_t* g, xg_grammar_tables_t* host_view);
+
+/* One cache entry, copied to the host (valid until the next call on this grammar or its
+ * destruction).  list = accepted ids (XG_STORE_ACCEPT_LIST) or rejected ids
+ * (XG_STORE_REJECT_LIST), ascending; bitset = accepted bits (XG_STORE_BITSET), ceil(V/32) words;
+ * uncertain = ascending ids.  Returns XG_ERR_INVALID_ARG if `state` is not scannable.
+ * Synchronises the device. */
+typedef struct {
+  int32_t state, kind;
+  int32_t n_accepted, n_rejected, n_uncertain;
+  int32_t n_list;
+  const int32_t* list;
+  const uint32_t* bitset;
+  const int32_t* uncertain;
+} xg_cache_entry_view_t;
+xg_status_t xg_grammar_get_cache_entry(const xg_grammar_t* g, int32_t state, xg_cache_entry_view_t* host_view);
+
+typedef struct {
+  int32_t n_rules, n_states, n_scannable, n_classes;
+  int32_t n_entries_built;      /* scannable states classified on the GPU by this compile */
+  int32_t n_entries_reused;     /* scannable states served by the pool (Section 3.3) */
+  int64_t pairs_classified;     /* n_entries_built * vocab_size */
+  int64_t total_accepted, total_rejected, total_uncertain;   /* over this grammar's entries */
+  int32_t kind_count[3];        /* entries per xg_store_kind_t */
+  int32_t pad;
+  int64_t cache_bytes;          /* device bytes of this grammar's entries (shared ones included) */
+  double frontend_ms, cache_build_ms;   /* host front end; GPU classification + packing */
+} xg_grammar_stats_t;
+xg_status_t xg_grammar_stats(const xg_grammar_t* g, xg_grammar_stats_t* out);
+
+/* ---- matcher: one request's Earley state (Section 3.4) ------------------------------------ */
+typedef struct {
+  uint32_t struct_size;
+  int32_t max_sets;    /* history capacity in Earley sets (one per accepted byte).  <= 0 = default (16384). */
+  int32_t max_items;   /* history capacity in items.  <= 0 = default (4 * max_sets). */
+} xg_matcher_options_t;
+xg_status_t xg_matcher_create(const xg_grammar_t* g, const xg_matcher_options_t* opt, void* stream, xg_matcher_t** out);
+xg_status_t xg_matcher_reset(xg_matcher_t* m, void* stream);
+void xg_matcher_destroy(xg_matcher_t* m);
+/* *out = 1 iff EOS has been accepted.  Synchronises `stream`. */
+xg_status_t xg_matcher_is_terminated(const xg_matcher_t* m, void* stream, int32_t* out);
+
+/* ---- per decode step ----------------------------------------------------------------------
+ * xg_fill_next_token_bitmask: for each of `batch` matchers (host array of handles, all on one
+ * tokenizer, grammars may differ) write its next-token bitmask into
+ * bitmask_dev[i*row_stride_words .. +ceil(V/32)) (device).  Merge rule of the appendix on
+ * XGrammar's cache: a token accepted by the cache of at least one current scannable state is
+ * allowed; otherwise, if some cache calls it uncertain, it is checked against the matcher's full
+ * Earley state; otherwise it is rejected.  EOS is allowed iff the root rule is complete.
+ * status_dev (device, [batch], may be NULL) receives XG_OK, XG_ERR_TERMINATED or XG_ERR_CAPACITY
+ * per matcher; rows of matchers whose status is not XG_OK are all zero. */
+xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t batch,
+                                       int32_t* bitmask_dev, int64_t row_stride_words,
+                                       int32_t* status_dev, void* stream);
+
+/* xg_apply_token_bitmask: logits[r][v] = -inf where bit v of mask row r is 0 (Section 2.1), in
+ * place, one pass.  logits_dev: device, [rows][logits_row_stride_elems] of dtype; every row must
+ * start on a 16-byte boundary (XG_ERR_INVALID_ARG otherwise).  row_indices_dev (device, may be
+ * NULL): the n_rows rows to touch (logits row = mask row = row_indices[i]); NULL = rows
+ * 0..batch-1.  Elements whose bit is 1 are not modified in any way (NaN payloads and -0
+ * survive); masked elements become the -inf bit pattern (0xFF800000 / 0xFF80) whatever they held. */
+xg_status_t xg_apply_token_bitmask(void* logits_dev, xg_dtype_t dtype, int32_t batch, int32_t vocab_size,
+                                   int64_t logits_row_stride_elems, const int32_t* bitmask_dev,
+                                   int64_t mask_row_stride_words, const int32_t* row_indices_dev,
+                                   int32_t n_rows, void* stream);
+
+/* xg_accept_token: advance each matcher by its sampled token (Section 2.2 "trace the output";
+ * scan / complete / predict of the appendix on Earley's algorithm).  token_ids_dev: device,
+ * [batch].  status_dev (device, [batch], may be NULL): XG_OK; XG_ERR_TOKEN_REJECTED (state
+ * unchanged); XG_ERR_TERMINATED; XG_ERR_CAPACITY (state unchanged).  Accepting EOS when the
+ * root is complete terminates the matcher. */
+xg_status_t xg_accept_token(xg_matcher_t* const* matchers, int32_t batch, const int32_t* token_ids_dev,
+                            int32_t* status_dev, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* XG_H_ */
