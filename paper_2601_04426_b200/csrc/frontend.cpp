@@ -1,0 +1,1231 @@
+// Host front end (see frontend.h).  Pipeline:
+//   text --lex/parse--> expression trees --Thompson--> NFAs with epsilon and rule-reference edges
+//   --bypass nullable references, drop epsilon--> NFAs --subset construction + partition
+//   refinement--> one DFA per rule --inline small rules--> --trim--> flat tables + closure lists.
+#include "frontend.h"
+
+#include <algorithm>
+#include <array>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <functional>
+#include <map>
+#include <memory>
+#include <set>
+
+#include "xg.h"
+
+namespace xg {
+namespace {
+
+[[noreturn]] void fail(int status, const std::string& msg) { throw FrontendError{status, msg}; }
+
+// ------------------------------------------------------------------------------------------
+// byte sets
+// ------------------------------------------------------------------------------------------
+struct ByteSet {
+  std::array<uint32_t, 8> w{};
+  void set(int b) { w[b >> 5] |= 1u << (b & 31); }
+  void set_range(int lo, int hi) { for (int b = lo; b <= hi; ++b) set(b); }
+  bool has(int b) const { return (w[b >> 5] >> (b & 31)) & 1u; }
+  bool empty() const { for (uint32_t x : w) if (x) return false; return true; }
+  void merge(const ByteSet& o) { for (int i = 0; i < 8; ++i) w[i] |= o.w[i]; }
+  bool operator==(const ByteSet& o) const { return w == o.w; }
+  bool operator<(const ByteSet& o) const { return w < o.w; }
+};
+
+// ------------------------------------------------------------------------------------------
+// expression trees
+// ------------------------------------------------------------------------------------------
+struct TagSpec {
+  std::vector<std::string> tags;
+  std::vector<std::string> tag_rules;
+  std::vector<std::string> stops;
+};
+struct Expr;
+typedef std::shared_ptr<Expr> ExprP;
+struct Expr {
+  enum Kind { kBytes, kClass, kRef, kSeq, kAlt, kRepeat, kTagDispatch } kind;
+  std::string bytes;                                  // kBytes
+  std::vector<std::pair<uint32_t, uint32_t>> ranges;  // kClass: code-point ranges (sorted, disjoint)
+  std::string name;                                   // kRef
+  std::vector<ExprP> kids;                            // kSeq, kAlt, kRepeat (one child)
+  int lo = 0, hi = 0;                                 // kRepeat: hi < 0 means unbounded
+  TagSpec tag;                                        // kTagDispatch
+};
+ExprP make(Expr::Kind k) { auto e = std::make_shared<Expr>(); e->kind = k; return e; }
+
+void put_utf8(std::string& out, uint32_t cp) {
+  if (cp <= 0x7F) { out += (char)cp; return; }
+  if (cp <= 0x7FF) { out += (char)(0xC0 | (cp >> 6)); out += (char)(0x80 | (cp & 63)); return; }
+  if (cp <= 0xFFFF) { out += (char)(0xE0 | (cp >> 12)); out += (char)(0x80 | ((cp >> 6) & 63)); out += (char)(0x80 | (cp & 63)); return; }
+  out += (char)(0xF0 | (cp >> 18)); out += (char)(0x80 | ((cp >> 12) & 63)); out += (char)(0x80 | ((cp >> 6) & 63)); out += (char)(0x80 | (cp & 63));
+}
+
+// ------------------------------------------------------------------------------------------
+// lexer + parser for the grammar text
+// ------------------------------------------------------------------------------------------
+struct Token {
+  enum Type { kEnd, kIdent, kDefine, kString, kClass, kBar, kLParen, kRParen, kStar, kPlus, kQuestion, kLBrace, kRBrace, kComma, kInt, kEquals } type = kEnd;
+  std::string text;                                   // identifier / decoded string bytes
+  std::vector<std::pair<uint32_t, uint32_t>> ranges;  // class
+  int value = 0;
+  size_t offset = 0;
+};
+
+class Lexer {
+ public:
+  explicit Lexer(const std::string& src) : src_(src) {}
+  std::vector<Token> run() {
+    std::vector<Token> out;
+    while (true) {
+      skip_space();
+      Token t;
+      t.offset = i_;
+      if (i_ >= src_.size()) { t.type = Token::kEnd; out.push_back(t); break; }
+      unsigned char c = src_[i_];
+      if (isalpha(c) || c == '_') {
+        size_t j = i_;
+        while (j < src_.size() && (isalnum((unsigned char)src_[j]) || src_[j] == '_')) ++j;
+        t.type = Token::kIdent; t.text = src_.substr(i_, j - i_); i_ = j;
+      } else if (isdigit(c)) {
+        long v = 0;
+        while (i_ < src_.size() && isdigit((unsigned char)src_[i_])) { v = v * 10 + (src_[i_++] - '0'); if (v > 1000000) err("number too large"); }
+        t.type = Token::kInt; t.value = (int)v;
+      } else if (c == ':' && src_.compare(i_, 3, "::=") == 0) { t.type = Token::kDefine; i_ += 3; }
+      else if (c == '"') { t.type = Token::kString; t.text = read_string(); }
+      else if (c == '[') { t.type = Token::kClass; t.ranges = read_class(); }
+      else {
+        ++i_;
+        switch (c) {
+          case '|': t.type = Token::kBar; break;
+          case '(': t.type = Token::kLParen; break;
+          case ')': t.type = Token::kRParen; break;
+          case '*': t.type = Token::kStar; break;
+          case '+': t.type = Token::kPlus; break;
+          case '?': t.type = Token::kQuestion; break;
+          case '{': t.type = Token::kLBrace; break;
+          case '}': t.type = Token::kRBrace; break;
+          case ',': t.type = Token::kComma; break;
+          case '=': t.type = Token::kEquals; break;
+          default: --i_; err(std::string("unexpected character '") + (char)c + "'");
+        }
+      }
+      out.push_back(t);
+    }
+    return out;
+  }
+
+ private:
+  const std::string& src_;
+  size_t i_ = 0;
+  [[noreturn]] void err(const std::string& m) { fail(XG_ERR_PARSE, "grammar text: " + m + " at offset " + std::to_string(i_)); }
+  void skip_space() {
+    while (i_ < src_.size()) {
+      char c = src_[i_];
+      if (c == '#') { while (i_ < src_.size() && src_[i_] != '\n') ++i_; }
+      else if (c == ' ' || c == '\t' || c == '\r' || c == '\n') ++i_;
+      else break;
+    }
+  }
+  uint32_t read_hex(int digits) {
+    uint32_t v = 0;
+    for (int k = 0; k < digits; ++k) {
+      if (i_ >= src_.size() || !isxdigit((unsigned char)src_[i_])) err("bad hexadecimal escape");
+      char c = src_[i_++];
+      v = v * 16 + (uint32_t)(isdigit((unsigned char)c) ? c - '0' : (tolower(c) - 'a' + 10));
+    }
+    return v;
+  }
+  // one (possibly escaped) unit; sets *raw_byte when it is \xHH outside a class
+  uint32_t read_unit(bool in_class, bool* raw_byte) {
+    *raw_byte = false;
+    unsigned char c = src_[i_];
+    if (c != '\\') {
+      ++i_;
+      if (c < 0x80) return c;
+      int extra = c >= 0xF0 ? 3 : c >= 0xE0 ? 2 : c >= 0xC0 ? 1 : -1;
+      if (extra < 0) err("invalid UTF-8 in grammar text");
+      uint32_t cp = c & (0xFF >> (extra + 2));
+      for (int k = 0; k < extra; ++k) {
+        if (i_ >= src_.size() || ((unsigned char)src_[i_] & 0xC0) != 0x80) err("invalid UTF-8 in grammar text");
+        cp = (cp << 6) | ((unsigned char)src_[i_++] & 63);
+      }
+      return cp;
+    }
+    ++i_;
+    if (i_ >= src_.size()) err("dangling backslash");
+    char e = src_[i_++];
+    switch (e) {
+      case 'n': return 10; case 't': return 9; case 'r': return 13;
+      case '\\': case '"': case '\'': case '/': return (uint32_t)e;
+      case 'x': *raw_byte = !in_class; return read_hex(2);
+      case 'u': return read_hex(4);
+      case 'U': return read_hex(8);
+      default:
+        if (in_class && (e == ']' || e == '-' || e == '^')) return (uint32_t)e;
+        err(std::string("unknown escape \\") + e);
+    }
+  }
+  std::string read_string() {
+    ++i_;
+    std::string out;
+    while (true) {
+      if (i_ >= src_.size()) err("unterminated string literal");
+      if (src_[i_] == '"') { ++i_; return out; }
+      bool raw;
+      uint32_t u = read_unit(false, &raw);
+      if (raw) out += (char)u;
+      else { if (u > 0x10FFFF || (u >= 0xD800 && u <= 0xDFFF)) err("escape is not a scalar value"); put_utf8(out, u); }
+    }
+  }
+  std::vector<std::pair<uint32_t, uint32_t>> read_class() {
+    ++i_;
+    bool negate = false;
+    if (i_ < src_.size() && src_[i_] == '^') { negate = true; ++i_; }
+    std::vector<std::pair<uint32_t, uint32_t>> rs;
+    while (true) {
+      if (i_ >= src_.size()) err("unterminated character class");
+      if (src_[i_] == ']') { ++i_; break; }
+      bool raw;
+      uint32_t a = read_unit(true, &raw), b = a;
+      if (i_ + 1 < src_.size() && src_[i_] == '-' && src_[i_ + 1] != ']') {
+        ++i_;
+        b = read_unit(true, &raw);
+        if (b < a) err("character class range is reversed");
+      }
+      rs.emplace_back(a, b);
+    }
+    std::sort(rs.begin(), rs.end());
+    std::vector<std::pair<uint32_t, uint32_t>> norm;
+    for (auto& r : rs) {
+      if (!norm.empty() && r.first <= norm.back().second + 1) norm.back().second = std::max(norm.back().second, r.second);
+      else norm.push_back(r);
+    }
+    if (!negate) return norm;
+    std::vector<std::pair<uint32_t, uint32_t>> comp;
+    uint32_t from = 0;
+    for (auto& r : norm) { if (r.first > from) comp.emplace_back(from, r.first - 1); from = r.second + 1; }
+    if (from <= 0x10FFFF) comp.emplace_back(from, 0x10FFFFu);
+    return comp;
+  }
+};
+
+class GrammarParser {
+ public:
+  explicit GrammarParser(std::vector<Token> toks) : t_(std::move(toks)) {}
+  std::vector<std::pair<std::string, ExprP>> run() {
+    std::vector<std::pair<std::string, ExprP>> rules;
+    while (peek().type != Token::kEnd) {
+      if (!starts_rule()) err("expected `name ::=`");
+      std::string name = t_[p_].text;
+      p_ += 2;
+      rules.emplace_back(name, alternatives());
+    }
+    if (rules.empty()) fail(XG_ERR_PARSE, "grammar text: no rules");
+    return rules;
+  }
+
+ private:
+  std::vector<Token> t_;
+  size_t p_ = 0;
+  const Token& peek() const { return t_[p_]; }
+  const Token& peek2() const { return t_[std::min(p_ + 1, t_.size() - 1)]; }
+  [[noreturn]] void err(const std::string& m) { fail(XG_ERR_PARSE, "grammar text: " + m + " at offset " + std::to_string(peek().offset)); }
+  void want(Token::Type ty, const char* what) { if (peek().type != ty) err(std::string("expected ") + what); ++p_; }
+  bool starts_rule() const { return peek().type == Token::kIdent && peek2().type == Token::kDefine; }
+
+  ExprP alternatives() {
+    auto alt = make(Expr::kAlt);
+    alt->kids.push_back(sequence());
+    while (peek().type == Token::kBar) { ++p_; alt->kids.push_back(sequence()); }
+    return alt->kids.size() == 1 ? alt->kids[0] : alt;
+  }
+  ExprP sequence() {
+    auto seq = make(Expr::kSeq);
+    while (true) {
+      Token::Type ty = peek().type;
+      if (ty == Token::kEnd || ty == Token::kBar || ty == Token::kRParen || starts_rule()) break;
+      seq->kids.push_back(postfix(primary()));
+    }
+    return seq;
+  }
+  ExprP primary() {
+    const Token& tk = peek();
+    if (tk.type == Token::kString) { auto e = make(Expr::kBytes); e->bytes = tk.text; ++p_; return e; }
+    if (tk.type == Token::kClass) { auto e = make(Expr::kClass); e->ranges = tk.ranges; ++p_; return e; }
+    if (tk.type == Token::kLParen) { ++p_; auto e = alternatives(); want(Token::kRParen, "')'"); return e; }
+    if (tk.type == Token::kIdent) {
+      if (tk.text == "TagDispatch" && peek2().type == Token::kLParen) { p_ += 2; return tag_dispatch(); }
+      auto e = make(Expr::kRef); e->name = tk.text; ++p_; return e;
+    }
+    err("expected a literal, class, rule name or '('");
+  }
+  ExprP postfix(ExprP e) {
+    while (true) {
+      Token::Type ty = peek().type;
+      int lo, hi;
+      if (ty == Token::kStar) { lo = 0; hi = -1; ++p_; }
+      else if (ty == Token::kPlus) { lo = 1; hi = -1; ++p_; }
+      else if (ty == Token::kQuestion) { lo = 0; hi = 1; ++p_; }
+      else if (ty == Token::kLBrace) {
+        ++p_;
+        if (peek().type != Token::kInt) err("expected a repetition count");
+        lo = hi = peek().value; ++p_;
+        if (peek().type == Token::kComma) {
+          ++p_;
+          if (peek().type == Token::kInt) { hi = peek().value; ++p_; } else hi = -1;
+        }
+        want(Token::kRBrace, "'}'");
+        if (hi >= 0 && hi < lo) err("repetition bounds are reversed");
+      } else break;
+      auto rep = make(Expr::kRepeat);
+      rep->lo = lo; rep->hi = hi; rep->kids.push_back(e);
+      e = rep;
+    }
+    return e;
+  }
+  std::vector<std::string> string_list() {
+    std::vector<std::string> out;
+    want(Token::kLParen, "'('");
+    while (peek().type != Token::kRParen) {
+      if (peek().type != Token::kString) err("expected a string");
+      out.push_back(peek().text); ++p_;
+      if (peek().type == Token::kComma) ++p_;
+    }
+    ++p_;
+    return out;
+  }
+  ExprP tag_dispatch() {       // after `TagDispatch(`
+    auto e = make(Expr::kTagDispatch);
+    while (peek().type != Token::kRParen) {
+      if (peek().type == Token::kLParen) {
+        ++p_;
+        if (peek().type != Token::kString || peek().text.empty()) err("expected a non-empty tag string");
+        e->tag.tags.push_back(peek().text); ++p_;
+        want(Token::kComma, "','");
+        if (peek().type != Token::kIdent) err("expected a rule name");
+        e->tag.tag_rules.push_back(peek().text); ++p_;
+        want(Token::kRParen, "')'");
+      } else if (peek().type == Token::kIdent && peek().text == "stop_strs") {
+        ++p_;
+        want(Token::kEquals, "'='");
+        e->tag.stops = string_list();
+        for (auto& s : e->tag.stops) if (s.empty()) err("empty stop string");
+      } else err("expected (\"tag\", rule) or stop_strs=(...)");
+      if (peek().type == Token::kComma) ++p_;
+    }
+    ++p_;
+    if (e->tag.tags.empty()) err("TagDispatch needs at least one tag");
+    return e;
+  }
+};
+
+// ------------------------------------------------------------------------------------------
+// automata
+// ------------------------------------------------------------------------------------------
+struct Edge {
+  enum Kind : uint8_t { kEps, kBytes, kRef } kind;
+  int rule;        // kRef
+  int to;
+  ByteSet set;     // kBytes
+};
+struct Fsm {
+  std::vector<std::vector<Edge>> out;
+  std::vector<char> fin;
+  int start = 0;
+  bool has_tag_dispatch = false;
+  int add() { out.emplace_back(); fin.push_back(0); return (int)out.size() - 1; }
+  int size() const { return (int)out.size(); }
+  void eps(int a, int b) { out[a].push_back({Edge::kEps, -1, b, {}}); }
+  void bytes(int a, const ByteSet& s, int b) { out[a].push_back({Edge::kBytes, -1, b, s}); }
+  void ref(int a, int rule, int b) { out[a].push_back({Edge::kRef, rule, b, {}}); }
+};
+
+// well-formed UTF-8 encodings of a code-point range as sequences of byte ranges
+typedef std::vector<std::pair<int, int>> ByteRangeSeq;
+void utf8_sequences(uint32_t lo, uint32_t hi, std::vector<ByteRangeSeq>& out) {
+  if (lo > hi) return;
+  static const uint32_t limits[4] = {0x7F, 0x7FF, 0xFFFF, 0x10FFFF};
+  // keep surrogates out
+  if (lo <= 0xDFFF && hi >= 0xD800) {
+    if (lo < 0xD800) utf8_sequences(lo, 0xD7FF, out);
+    if (hi > 0xDFFF) utf8_sequences(0xE000, hi, out);
+    return;
+  }
+  // one encoded length per piece
+  for (int k = 0; k < 3; ++k)
+    if (lo <= limits[k] && hi > limits[k]) { utf8_sequences(lo, limits[k], out); utf8_sequences(limits[k] + 1, hi, out); return; }
+  if (hi <= 0x7F) { out.push_back({{(int)lo, (int)hi}}); return; }
+  int n = hi <= 0x7FF ? 2 : hi <= 0xFFFF ? 3 : 4;
+  // split until the low 6*k bits span a full block wherever the higher bits differ
+  for (int k = 1; k < n; ++k) {
+    uint32_t m = (1u << (6 * k)) - 1;
+    if ((lo & ~m) != (hi & ~m)) {
+      if ((lo & m) != 0) { utf8_sequences(lo, lo | m, out); utf8_sequences((lo | m) + 1, hi, out); return; }
+      if ((hi & m) != m) { utf8_sequences(lo, (hi & ~m) - 1, out); utf8_sequences(hi & ~m, hi, out); return; }
+    }
+  }
+  std::string a, b;
+  put_utf8(a, lo); put_utf8(b, hi);
+  ByteRangeSeq seq;
+  for (int k = 0; k < n; ++k) seq.emplace_back((unsigned char)a[k], (unsigned char)b[k]);
+  out.push_back(seq);
+}
+
+// Aho-Corasick automaton over tags and stop strings (Section 3.2)
+struct AhoCorasick {
+  std::vector<std::array<int, 256>> next;   // goto function completed with failure links
+  std::vector<std::vector<int>> ends;       // patterns ending at the node (own or via suffix links)
+  explicit AhoCorasick(const std::vector<std::string>& patterns) {
+    std::vector<std::array<int, 256>> child;
+    std::vector<int> link;
+    auto node = [&]() { std::array<int, 256> a; a.fill(-1); child.push_back(a); ends.emplace_back(); link.push_back(0); return (int)child.size() - 1; };
+    node();
+    for (size_t p = 0; p < patterns.size(); ++p) {
+      int u = 0;
+      for (unsigned char c : patterns[p]) { if (child[u][c] < 0) { int v = node(); child[u][c] = v; } u = child[u][c]; }
+      ends[u].push_back((int)p);
+    }
+    next.assign(child.size(), {});
+    std::vector<int> queue;
+    for (int c = 0; c < 256; ++c) {
+      int v = child[0][c];
+      if (v < 0) next[0][c] = 0; else { next[0][c] = v; link[v] = 0; queue.push_back(v); }
+    }
+    for (size_t q = 0; q < queue.size(); ++q) {
+      int u = queue[q];
+      for (int p : ends[link[u]]) ends[u].push_back(p);
+      for (int c = 0; c < 256; ++c) {
+        int v = child[u][c];
+        if (v < 0) next[u][c] = next[link[u]][c];
+        else { next[u][c] = v; link[v] = next[link[u]][c]; queue.push_back(v); }
+      }
+    }
+  }
+};
+
+struct Builder {
+  std::vector<std::string> names;
+  std::map<std::string, int> ids;
+  std::vector<Fsm> rules;
+
+  int lookup(const std::string& n) const {
+    auto it = ids.find(n);
+    if (it == ids.end()) fail(XG_ERR_PARSE, "grammar text: undefined rule " + n);
+    return it->second;
+  }
+  // Thompson construction: returns (entry, exit) of a fragment inside f
+  std::pair<int, int> frag(Fsm& f, const Expr& e) {
+    switch (e.kind) {
+      case Expr::kBytes: {
+        int s = f.add(), cur = s;
+        for (unsigned char c : e.bytes) { int n = f.add(); ByteSet bs; bs.set(c); f.bytes(cur, bs, n); cur = n; }
+        return {s, cur};
+      }
+      case Expr::kClass: {
+        int s = f.add(), t = f.add();
+        std::vector<ByteRangeSeq> seqs;
+        for (auto& r : e.ranges) utf8_sequences(r.first, std::min<uint32_t>(r.second, 0x10FFFF), seqs);
+        for (auto& seq : seqs) {
+          int cur = s;
+          for (size_t k = 0; k < seq.size(); ++k) {
+            int n = k + 1 == seq.size() ? t : f.add();
+            ByteSet bs; bs.set_range(seq[k].first, seq[k].second);
+            f.bytes(cur, bs, n);
+            cur = n;
+          }
+        }
+        return {s, t};
+      }
+      case Expr::kRef: { int s = f.add(), t = f.add(); f.ref(s, lookup(e.name), t); return {s, t}; }
+      case Expr::kSeq: {
+        int s = f.add(), cur = s;
+        for (auto& k : e.kids) { auto p = frag(f, *k); f.eps(cur, p.first); cur = p.second; }
+        return {s, cur};
+      }
+      case Expr::kAlt: {
+        int s = f.add(), t = f.add();
+        for (auto& k : e.kids) { auto p = frag(f, *k); f.eps(s, p.first); f.eps(p.second, t); }
+        return {s, t};
+      }
+      case Expr::kRepeat: {
+        int s = f.add(), cur = s;
+        for (int i = 0; i < e.lo; ++i) { auto p = frag(f, *e.kids[0]); f.eps(cur, p.first); cur = p.second; }
+        int t = f.add();
+        if (e.hi < 0) {
+          int loop = f.add();
+          f.eps(cur, loop);
+          auto p = frag(f, *e.kids[0]);
+          f.eps(loop, p.first); f.eps(p.second, loop); f.eps(loop, t);
+        } else {
+          for (int i = e.lo; i < e.hi; ++i) { f.eps(cur, t); auto p = frag(f, *e.kids[0]); f.eps(cur, p.first); cur = p.second; }
+          f.eps(cur, t);
+        }
+        return {s, t};
+      }
+      case Expr::kTagDispatch: return tag_fragment(f, e.tag);
+    }
+    fail(XG_ERR_INVALID_ARG, "internal: unknown expression kind");
+  }
+  std::pair<int, int> tag_fragment(Fsm& f, const TagSpec& spec) {
+    f.has_tag_dispatch = true;
+    std::vector<std::string> patterns = spec.tags;
+    patterns.insert(patterns.end(), spec.stops.begin(), spec.stops.end());
+    int n_tags = (int)spec.tags.size();
+    AhoCorasick ac(patterns);
+    int n_nodes = (int)ac.next.size();
+    std::vector<int> node_state(n_nodes, -1);
+    for (int u = 0; u < n_nodes; ++u) if (ac.ends[u].empty()) node_state[u] = f.add();
+    int exit = f.add();
+    std::vector<int> dispatch(n_tags, -1);       // state holding the reference edge of tag j
+    for (int j = 0; j < n_tags; ++j) { dispatch[j] = f.add(); f.ref(dispatch[j], lookup(spec.tag_rules[j]), node_state[0]); }
+    for (int u = 0; u < n_nodes; ++u) {
+      if (node_state[u] < 0) continue;
+      std::map<int, ByteSet> by_target;          // target state -> bytes
+      for (int c = 0; c < 256; ++c) {
+        int v = ac.next[u][c];
+        if (ac.ends[v].empty()) { by_target[node_state[v]].set(c); continue; }
+        bool any_tag = false;
+        for (int p : ac.ends[v]) if (p < n_tags) { any_tag = true; by_target[dispatch[p]].set(c); }
+        if (!any_tag) by_target[exit].set(c);    // a stop string ends the construct
+      }
+      for (auto& kv : by_target) f.bytes(node_state[u], kv.second, kv.first);
+      if (spec.stops.empty()) f.eps(node_state[u], exit);   // may end anywhere while dispatching
+    }
+    return {node_state[0], exit};
+  }
+};
+
+// epsilon closure of every state
+std::vector<std::vector<int>> eps_closures(const Fsm& f) {
+  int n = f.size();
+  std::vector<std::vector<int>> cl(n);
+  std::vector<int> mark(n, -1), stack;
+  for (int s = 0; s < n; ++s) {
+    stack.assign(1, s); mark[s] = s;
+    while (!stack.empty()) {
+      int u = stack.back(); stack.pop_back();
+      cl[s].push_back(u);
+      for (const Edge& e : f.out[u]) if (e.kind == Edge::kEps && mark[e.to] != s) { mark[e.to] = s; stack.push_back(e.to); }
+    }
+  }
+  return cl;
+}
+
+Fsm drop_epsilon(const Fsm& f) {
+  auto cl = eps_closures(f);
+  Fsm g;
+  g.has_tag_dispatch = f.has_tag_dispatch;
+  for (int s = 0; s < f.size(); ++s) g.add();
+  g.start = f.start;
+  for (int s = 0; s < f.size(); ++s)
+    for (int u : cl[s]) {
+      if (f.fin[u]) g.fin[s] = 1;
+      for (const Edge& e : f.out[u]) if (e.kind != Edge::kEps) g.out[s].push_back(e);
+    }
+  return g;
+}
+
+// subset construction over the alphabet {bytes} + {rule references}; the input has no epsilon edges
+Fsm determinize(const Fsm& f, int max_states) {
+  Fsm d;
+  d.has_tag_dispatch = f.has_tag_dispatch;
+  std::map<std::vector<int>, int> index;
+  std::vector<std::vector<int>> subsets;
+  auto state_of = [&](std::vector<int>& set) {
+    std::sort(set.begin(), set.end());
+    set.erase(std::unique(set.begin(), set.end()), set.end());
+    auto it = index.find(set);
+    if (it != index.end()) return it->second;
+    int id = d.add();
+    if (id >= max_states) fail(XG_ERR_CAPACITY, "a rule automaton exceeds max_rule_states");
+    index[set] = id;
+    subsets.push_back(set);
+    for (int s : set) if (f.fin[s]) d.fin[id] = 1;
+    return id;
+  };
+  std::vector<int> init{f.start};
+  d.start = state_of(init);
+  for (int cur = 0; cur < (int)subsets.size(); ++cur) {
+    std::vector<int> members = subsets[cur];
+    std::map<int, std::vector<int>> by_rule;
+    std::vector<const Edge*> byte_edges;
+    for (int s : members)
+      for (const Edge& e : f.out[s]) {
+        if (e.kind == Edge::kRef) by_rule[e.rule].push_back(e.to);
+        else if (e.kind == Edge::kBytes) byte_edges.push_back(&e);
+      }
+    for (auto& kv : by_rule) { int t = state_of(kv.second); d.ref(cur, kv.first, t); }
+    if (byte_edges.empty()) continue;
+    std::map<std::vector<int>, ByteSet> groups;      // target subset -> bytes
+    std::vector<int> targets;
+    for (int b = 0; b < 256; ++b) {
+      targets.clear();
+      for (const Edge* e : byte_edges) if (e->set.has(b)) targets.push_back(e->to);
+      if (targets.empty()) continue;
+      std::sort(targets.begin(), targets.end());
+      targets.erase(std::unique(targets.begin(), targets.end()), targets.end());
+      groups[targets].set(b);
+    }
+    for (auto& kv : groups) { std::vector<int> tg = kv.first; int t = state_of(tg); d.bytes(cur, kv.second, t); }
+  }
+  return d;
+}
+
+// merge equivalent states of a deterministic automaton (partition refinement on sparse signatures)
+Fsm minimize(const Fsm& f) {
+  int n = f.size();
+  std::vector<int> block(n);
+  for (int s = 0; s < n; ++s) block[s] = f.fin[s] ? 1 : 0;
+  int n_blocks = 0;
+  typedef std::pair<std::vector<std::pair<int, ByteSet>>, std::vector<std::pair<int, int>>> Sig;
+  while (true) {
+    std::map<std::pair<int, Sig>, int> sig_id;
+    std::vector<int> nb(n);
+    for (int s = 0; s < n; ++s) {
+      std::map<int, ByteSet> by_block;
+      std::vector<std::pair<int, int>> refs;
+      for (const Edge& e : f.out[s]) {
+        if (e.kind == Edge::kBytes) by_block[block[e.to]].merge(e.set);
+        else refs.emplace_back(e.rule, block[e.to]);
+      }
+      std::sort(refs.begin(), refs.end());
+      Sig sig{std::vector<std::pair<int, ByteSet>>(by_block.begin(), by_block.end()), refs};
+      auto key = std::make_pair(block[s], sig);
+      auto it = sig_id.find(key);
+      if (it == sig_id.end()) it = sig_id.emplace(key, (int)sig_id.size()).first;
+      nb[s] = it->second;
+    }
+    int count = (int)sig_id.size();
+    block = nb;
+    if (count == n_blocks) break;
+    n_blocks = count;
+  }
+  Fsm m;
+  m.has_tag_dispatch = f.has_tag_dispatch;
+  for (int b = 0; b < n_blocks; ++b) m.add();
+  std::vector<char> done(n_blocks, 0);
+  m.start = block[f.start];
+  for (int s = 0; s < n; ++s) {
+    int b = block[s];
+    if (f.fin[s]) m.fin[b] = 1;
+    if (done[b]) continue;
+    done[b] = 1;
+    std::map<int, ByteSet> by_block;
+    for (const Edge& e : f.out[s]) {
+      if (e.kind == Edge::kBytes) by_block[block[e.to]].merge(e.set);
+      else m.ref(b, e.rule, block[e.to]);
+    }
+    for (auto& kv : by_block) m.bytes(b, kv.second, kv.first);
+  }
+  return m;
+}
+
+// breadth-first renumbering from the start state with edges in a fixed order; drops unreachable
+// states
+Fsm canonical_order(const Fsm& f) {
+  std::vector<int> order, id(f.size(), -1);
+  order.push_back(f.start); id[f.start] = 0;
+  auto sorted_edges = [&](int s) {
+    std::vector<const Edge*> es;
+    for (const Edge& e : f.out[s]) es.push_back(&e);
+    std::stable_sort(es.begin(), es.end(), [](const Edge* a, const Edge* b) {
+      if (a->kind != b->kind) return a->kind < b->kind;
+      if (a->kind == Edge::kBytes) return a->set < b->set;
+      return a->rule < b->rule;
+    });
+    return es;
+  };
+  for (size_t q = 0; q < order.size(); ++q)
+    for (const Edge* e : sorted_edges(order[q])) if (id[e->to] < 0) { id[e->to] = (int)order.size(); order.push_back(e->to); }
+  Fsm g;
+  g.has_tag_dispatch = f.has_tag_dispatch;
+  for (size_t k = 0; k < order.size(); ++k) g.add();
+  g.start = 0;
+  for (size_t k = 0; k < order.size(); ++k) {
+    int s = order[k];
+    g.fin[k] = f.fin[s];
+    for (const Edge* e : sorted_edges(s)) { Edge c = *e; c.to = id[e->to]; g.out[k].push_back(c); }
+  }
+  return g;
+}
+
+Fsm normalize(const Fsm& f, int max_states) { return canonical_order(minimize(determinize(drop_epsilon(f), max_states))); }
+
+struct Compiler {
+  Builder b;
+  FrontendOptions opt;
+  int root = 0;
+  bool root_nullable = false;
+
+  int n_rules() const { return (int)b.rules.size(); }
+
+  // rules that derive the empty string: fixpoint over "an accepting state is reachable from the
+  // start through epsilon edges and references to nullable rules"
+  std::vector<char> nullable_rules() {
+    std::vector<char> nullable(n_rules(), 0);
+    bool changed = true;
+    while (changed) {
+      changed = false;
+      for (int r = 0; r < n_rules(); ++r) {
+        if (nullable[r]) continue;
+        const Fsm& f = b.rules[r];
+        std::vector<char> seen(f.size(), 0);
+        std::vector<int> stack{f.start};
+        seen[f.start] = 1;
+        bool hit = false;
+        while (!stack.empty()) {
+          int u = stack.back(); stack.pop_back();
+          if (f.fin[u]) { hit = true; break; }
+          for (const Edge& e : f.out[u])
+            if ((e.kind == Edge::kEps || (e.kind == Edge::kRef && nullable[e.rule])) && !seen[e.to]) { seen[e.to] = 1; stack.push_back(e.to); }
+        }
+        if (hit) { nullable[r] = 1; changed = true; }
+      }
+    }
+    return nullable;
+  }
+
+  void remove_nullability() {
+    std::vector<char> nullable = nullable_rules();
+    root_nullable = nullable[root];
+    for (Fsm& f : b.rules)
+      for (int s = 0; s < f.size(); ++s) {
+        size_t n = f.out[s].size();
+        for (size_t k = 0; k < n; ++k)
+          if (f.out[s][k].kind == Edge::kRef && nullable[f.out[s][k].rule]) { int to = f.out[s][k].to; f.eps(s, to); }
+      }
+    for (int r = 0; r < n_rules(); ++r) {
+      Fsm g = drop_epsilon(b.rules[r]);
+      if (g.fin[g.start]) {          // take the empty string out: a fresh, non-accepting start
+        int s = g.add();
+        g.out[s] = g.out[g.start];
+        g.start = s;
+      }
+      b.rules[r] = g;
+    }
+  }
+
+  // Rules that derive at least one string; then: drop references to the others, and every state
+  // that cannot reach an accepting state.
+  void trim() {
+    int R = n_rules();
+    std::vector<char> productive(R, 0);
+    auto live_states = [&](const Fsm& f) {
+      int n = f.size();
+      std::vector<std::vector<int>> rev(n);
+      for (int s = 0; s < n; ++s)
+        for (const Edge& e : f.out[s]) {
+          bool usable = e.kind == Edge::kEps || (e.kind == Edge::kBytes && !e.set.empty()) || (e.kind == Edge::kRef && productive[e.rule]);
+          if (usable) rev[e.to].push_back(s);
+        }
+      std::vector<char> live(n, 0);
+      std::vector<int> stack;
+      for (int s = 0; s < n; ++s) if (f.fin[s]) { live[s] = 1; stack.push_back(s); }
+      while (!stack.empty()) { int u = stack.back(); stack.pop_back(); for (int p : rev[u]) if (!live[p]) { live[p] = 1; stack.push_back(p); } }
+      return live;
+    };
+    bool changed = true;
+    while (changed) {
+      changed = false;
+      for (int r = 0; r < R; ++r) if (!productive[r] && live_states(b.rules[r])[b.rules[r].start]) { productive[r] = 1; changed = true; }
+    }
+    for (int r = 0; r < R; ++r) {
+      Fsm& f = b.rules[r];
+      std::vector<char> live = live_states(f);
+      live[f.start] = 1;           // the start state stays even if the rule derives nothing
+      std::vector<int> id(f.size(), -1);
+      Fsm g;
+      g.has_tag_dispatch = f.has_tag_dispatch;
+      for (int s = 0; s < f.size(); ++s) if (live[s]) id[s] = g.add();
+      g.start = id[f.start];
+      for (int s = 0; s < f.size(); ++s) {
+        if (!live[s]) continue;
+        g.fin[id[s]] = f.fin[s];
+        for (const Edge& e : f.out[s]) {
+          if (!live[e.to]) continue;
+          if (e.kind == Edge::kRef && !productive[e.rule]) continue;
+          if (e.kind == Edge::kBytes && e.set.empty()) continue;
+          Edge c = e; c.to = id[e.to];
+          g.out[id[s]].push_back(c);
+        }
+      }
+      f = g;
+    }
+  }
+
+  // for each rule, whether it can reach itself through references
+  std::vector<char> recursive_rules() {
+    int R = n_rules();
+    std::vector<std::set<int>> adj(R);
+    for (int r = 0; r < R; ++r) for (auto& es : b.rules[r].out) for (const Edge& e : es) if (e.kind == Edge::kRef) adj[r].insert(e.rule);
+    std::vector<char> rec(R, 0);
+    for (int r = 0; r < R; ++r) {
+      std::vector<char> seen(R, 0);
+      std::vector<int> stack(adj[r].begin(), adj[r].end());
+      while (!stack.empty()) {
+        int u = stack.back(); stack.pop_back();
+        if (u == r) { rec[r] = 1; break; }
+        if (seen[u]) continue;
+        seen[u] = 1;
+        for (int v : adj[u]) stack.push_back(v);
+      }
+    }
+    return rec;
+  }
+
+  // Replace references to small non-recursive rules by a copy of their automaton.
+  void inline_small_rules() {
+    if (opt.inline_max_states <= 0) return;
+    int R = n_rules();
+    std::vector<char> rec = recursive_rules();
+    std::vector<char> inlinable(R, 0), done(R, 0);
+    std::function<void(int)> process = [&](int r) {       // callees first
+      if (done[r]) return;
+      done[r] = 1;          // also guards recursion through cycles
+      std::set<int> callees;
+      for (auto& es : b.rules[r].out) for (const Edge& e : es) if (e.kind == Edge::kRef) callees.insert(e.rule);
+      for (int c : callees) if (c != r) process(c);
+      const Fsm& f = b.rules[r];
+      bool changed = false;
+      Fsm g = f;
+      for (int s = 0; s < f.size(); ++s) {
+        std::vector<Edge> keep;
+        const std::vector<Edge> edges = g.out[s];     // g.out may reallocate while copies are appended
+        for (const Edge& e : edges) {
+          if (e.kind == Edge::kRef && e.rule != r && inlinable[e.rule] && g.size() + b.rules[e.rule].size() <= opt.max_rule_states) {
+            const Fsm& c = b.rules[e.rule];
+            int base = g.size();
+            for (int k = 0; k < c.size(); ++k) g.add();
+            for (int k = 0; k < c.size(); ++k) {
+              for (Edge ce : c.out[k]) { ce.to += base; g.out[base + k].push_back(ce); }
+              if (c.fin[k]) g.eps(base + k, e.to);
+            }
+            keep.push_back({Edge::kEps, -1, base + c.start, {}});
+            g.has_tag_dispatch = g.has_tag_dispatch || c.has_tag_dispatch;
+            changed = true;
+          } else keep.push_back(e);
+        }
+        g.out[s] = keep;
+      }
+      if (changed) b.rules[r] = normalize(g, opt.max_rule_states);
+      inlinable[r] = !rec[r] && r != root && b.rules[r].size() <= opt.inline_max_states;
+    };
+    for (int r = 0; r < R; ++r) process(r);
+  }
+
+  FlatGrammar flatten() {
+    int R = n_rules();
+    // keep only rules reachable from the root
+    std::vector<int> new_id(R, -1), order;
+    order.push_back(root); new_id[root] = 0;
+    for (size_t q = 0; q < order.size(); ++q)
+      for (auto& es : b.rules[order[q]].out)
+        for (const Edge& e : es) if (e.kind == Edge::kRef && new_id[e.rule] < 0) { new_id[e.rule] = (int)order.size(); order.push_back(e.rule); }
+    FlatGrammar g;
+    g.n_rules = (int)order.size();
+    g.root_rule = 0;
+    g.root_nullable = root_nullable ? 1 : 0;
+    std::map<ByteSet, int> class_id;
+    std::vector<int> base(g.n_rules);
+    for (int k = 0; k < g.n_rules; ++k) { base[k] = g.n_states; g.n_states += b.rules[order[k]].size(); }
+    g.cedge_begin.push_back(0); g.redge_begin.push_back(0);
+    for (int k = 0; k < g.n_rules; ++k) {
+      const Fsm& f = b.rules[order[k]];
+      g.rule_names.push_back(b.names[order[k]]);
+      g.rule_start.push_back(base[k] + f.start);
+      g.rule_kind.push_back(f.has_tag_dispatch ? 1 : 0);
+      for (int s = 0; s < f.size(); ++s) {
+        g.state_rule.push_back(k);
+        g.state_final.push_back(f.fin[s] ? 1 : 0);
+        for (const Edge& e : f.out[s]) {
+          if (e.kind == Edge::kBytes) {
+            auto it = class_id.find(e.set);
+            if (it == class_id.end()) {
+              it = class_id.emplace(e.set, (int)class_id.size()).first;
+              g.class_bits.insert(g.class_bits.end(), e.set.w.begin(), e.set.w.end());
+            }
+            g.cedge_class.push_back(it->second);
+            g.cedge_target.push_back(base[k] + e.to);
+          } else if (e.kind == Edge::kRef) {
+            g.redge_rule.push_back(new_id[e.rule]);
+            g.redge_target.push_back(base[k] + e.to);
+          }
+        }
+        g.cedge_begin.push_back((int)g.cedge_class.size());
+        g.redge_begin.push_back((int)g.redge_rule.size());
+      }
+    }
+    g.n_classes = (int)class_id.size();
+    build_closure_lists(g);
+    return g;
+  }
+
+  static void build_closure_lists(FlatGrammar& g) {
+    int R = g.n_rules, S = g.n_states;
+    // rules predicted transitively when rule r is predicted (r itself included)
+    std::vector<std::vector<int>> closure(R);
+    for (int r = 0; r < R; ++r) {
+      std::vector<char> seen(R, 0);
+      std::vector<int> stack{r};
+      seen[r] = 1;
+      while (!stack.empty()) {
+        int u = stack.back(); stack.pop_back();
+        closure[r].push_back(u);
+        int s0 = g.rule_start[u];
+        for (int e = g.redge_begin[s0]; e < g.redge_begin[s0 + 1]; ++e) if (!seen[g.redge_rule[e]]) { seen[g.redge_rule[e]] = 1; stack.push_back(g.redge_rule[e]); }
+      }
+    }
+    g.scan_begin.assign(1, 0); g.wait_begin.assign(1, 0); g.gather_begin.assign(1, 0);
+    g.scan_own_end.clear();
+    std::vector<int> predicted;
+    std::vector<char> mark(R, 0);
+    for (int s = 0; s < S; ++s) {
+      predicted.clear();
+      for (int e = g.redge_begin[s]; e < g.redge_begin[s + 1]; ++e)
+        for (int r : closure[g.redge_rule[e]]) if (!mark[r]) { mark[r] = 1; predicted.push_back(r); }
+      std::sort(predicted.begin(), predicted.end());
+      for (int r : predicted) mark[r] = 0;
+      for (int e = g.cedge_begin[s]; e < g.cedge_begin[s + 1]; ++e) { g.scan_class.push_back(g.cedge_class[e]); g.scan_target.push_back(g.cedge_target[e]); }
+      g.scan_own_end.push_back((int)g.scan_class.size());
+      for (int e = g.redge_begin[s]; e < g.redge_begin[s + 1]; ++e) { g.wait_rule.push_back(g.redge_rule[e]); g.wait_target.push_back(g.redge_target[e]); }
+      if (g.cedge_begin[s + 1] > g.cedge_begin[s]) g.gather_state.push_back(s);
+      for (int r : predicted) {
+        int s0 = g.rule_start[r];
+        for (int e = g.cedge_begin[s0]; e < g.cedge_begin[s0 + 1]; ++e) { g.scan_class.push_back(g.cedge_class[e]); g.scan_target.push_back((uint32_t)g.cedge_target[e] | kSelfBit); }
+        for (int e = g.redge_begin[s0]; e < g.redge_begin[s0 + 1]; ++e) { g.wait_rule.push_back(g.redge_rule[e]); g.wait_target.push_back((uint32_t)g.redge_target[e] | kSelfBit); }
+        if (g.cedge_begin[s0 + 1] > g.cedge_begin[s0] && s0 != s) g.gather_state.push_back(s0);
+      }
+      g.scan_begin.push_back((int)g.scan_class.size());
+      g.wait_begin.push_back((int)g.wait_rule.size());
+      g.gather_begin.push_back((int)g.gather_state.size());
+    }
+  }
+};
+
+// ------------------------------------------------------------------------------------------
+// a small JSON reader (for schemas and TagDispatch specs)
+// ------------------------------------------------------------------------------------------
+struct Json {
+  enum Type { kNull, kBool, kNumber, kString, kArray, kObject } type = kNull;
+  bool boolean = false;
+  std::string text;                                   // string value, or the number's source text
+  std::vector<Json> items;
+  std::vector<std::pair<std::string, Json>> members;  // declaration order kept
+  const Json* get(const std::string& key) const {
+    for (auto& m : members) if (m.first == key) return &m.second;
+    return nullptr;
+  }
+};
+class JsonReader {
+ public:
+  explicit JsonReader(const std::string& s) : s_(s) {}
+  Json run() { Json v = value(0); ws(); if (i_ != s_.size()) err("trailing characters"); return v; }
+
+ private:
+  const std::string& s_;
+  size_t i_ = 0;
+  [[noreturn]] void err(const std::string& m) { fail(XG_ERR_PARSE, "JSON: " + m + " at offset " + std::to_string(i_)); }
+  void ws() { while (i_ < s_.size() && (s_[i_] == ' ' || s_[i_] == '\t' || s_[i_] == '\n' || s_[i_] == '\r')) ++i_; }
+  bool eat(char c) { ws(); if (i_ < s_.size() && s_[i_] == c) { ++i_; return true; } return false; }
+  uint32_t hex4() {
+    uint32_t v = 0;
+    for (int k = 0; k < 4; ++k) {
+      if (i_ >= s_.size() || !isxdigit((unsigned char)s_[i_])) err("bad \\u escape");
+      char h = s_[i_++];
+      v = v * 16 + (uint32_t)(isdigit((unsigned char)h) ? h - '0' : tolower(h) - 'a' + 10);
+    }
+    return v;
+  }
+  std::string string() {
+    if (!eat('"')) err("expected a string");
+    std::string out;
+    while (true) {
+      if (i_ >= s_.size()) err("unterminated string");
+      unsigned char c = s_[i_++];
+      if (c == '"') return out;
+      if (c < 0x20) err("control character in string");
+      if (c != '\\') { out += (char)c; continue; }
+      if (i_ >= s_.size()) err("dangling backslash");
+      char e = s_[i_++];
+      switch (e) {
+        case '"': case '\\': case '/': out += e; break;
+        case 'b': out += '\b'; break; case 'f': out += '\f'; break; case 'n': out += '\n'; break;
+        case 'r': out += '\r'; break; case 't': out += '\t'; break;
+        case 'u': {
+          uint32_t cp = hex4();
+          if (cp >= 0xD800 && cp <= 0xDBFF && s_.compare(i_, 2, "\\u") == 0) { i_ += 2; uint32_t lo = hex4(); cp = 0x10000 + ((cp - 0xD800) << 10) + (lo - 0xDC00); }
+          put_utf8(out, cp);
+          break;
+        }
+        default: err("unknown escape");
+      }
+    }
+  }
+  Json value(int depth) {
+    if (depth > 64) err("nesting too deep");
+    ws();
+    if (i_ >= s_.size()) err("unexpected end");
+    Json v;
+    char c = s_[i_];
+    if (c == '{') {
+      ++i_; v.type = Json::kObject;
+      if (eat('}')) return v;
+      do { std::string k = string(); if (!eat(':')) err("expected ':'"); v.members.emplace_back(k, value(depth + 1)); } while (eat(','));
+      if (!eat('}')) err("expected '}'");
+    } else if (c == '[') {
+      ++i_; v.type = Json::kArray;
+      if (eat(']')) return v;
+      do v.items.push_back(value(depth + 1)); while (eat(','));
+      if (!eat(']')) err("expected ']'");
+    } else if (c == '"') { v.type = Json::kString; v.text = string(); }
+    else if (s_.compare(i_, 4, "true") == 0) { v.type = Json::kBool; v.boolean = true; i_ += 4; }
+    else if (s_.compare(i_, 5, "false") == 0) { v.type = Json::kBool; i_ += 5; }
+    else if (s_.compare(i_, 4, "null") == 0) { i_ += 4; }
+    else {
+      size_t j = i_;
+      while (j < s_.size() && (isdigit((unsigned char)s_[j]) || strchr("+-.eE", s_[j]))) ++j;
+      if (j == i_) err("unexpected character");
+      v.type = Json::kNumber; v.text = s_.substr(i_, j - i_); i_ = j;
+    }
+    return v;
+  }
+};
+
+// JSON text of a string value as it must appear in generated output: short escapes for the
+// usual controls, \u00XX for the rest, everything else verbatim
+std::string json_string_text(const std::string& s) {
+  std::string out = "\"";
+  for (unsigned char c : s) {
+    switch (c) {
+      case '"': out += "\\\""; break; case '\\': out += "\\\\"; break;
+      case '\n': out += "\\n"; break; case '\r': out += "\\r"; break; case '\t': out += "\\t"; break;
+      case '\b': out += "\\b"; break; case '\f': out += "\\f"; break;
+      default:
+        if (c < 0x20) { char buf[8]; snprintf(buf, sizeof buf, "\\u%04x", c); out += buf; }
+        else out += (char)c;
+    }
+  }
+  return out + "\"";
+}
+// a grammar-text literal for exact bytes
+std::string literal(const std::string& bytes) {
+  std::string out = "\"";
+  for (unsigned char c : bytes) {
+    if (c == '"' || c == '\\') { out += '\\'; out += (char)c; }
+    else if (c < 0x20 || c == 0x7F) { char buf[8]; snprintf(buf, sizeof buf, "\\x%02x", c); out += buf; }
+    else out += (char)c;
+  }
+  return out + "\"";
+}
+
+// JSON schema subset -> grammar text.  Objects list all their properties, in order, separated by
+// ", " with ": " after the key; strings, numbers, arrays as in JSON; bounds become repetitions
+// (Section 3.6: minLength / maxLength / minItems / maxItems generate repetition structures).
+class SchemaLowering {
+ public:
+  SchemaLowering(const Json* defs, std::string prefix) : defs_(defs), prefix_(std::move(prefix)) {}
+  std::vector<std::string> rules;
+
+  std::string lower(const Json& s) {
+    if (s.type != Json::kObject) fail(XG_ERR_UNSUPPORTED, "schema: expected an object");
+    if (const Json* ref = s.get("$ref")) {
+      const std::string pre = "#/$defs/";
+      if (ref->type != Json::kString || ref->text.compare(0, pre.size(), pre) != 0) fail(XG_ERR_UNSUPPORTED, "schema: only #/$defs/ references are supported");
+      std::string name = ref->text.substr(pre.size());
+      const Json* target = defs_ ? defs_->get(name) : nullptr;
+      if (!target) fail(XG_ERR_PARSE, "schema: unknown reference " + ref->text);
+      auto it = def_rule_.find(name);
+      if (it != def_rule_.end()) return it->second;
+      std::string rule = fresh("ref");
+      def_rule_[name] = rule;
+      std::string body = lower(*target);
+      rules.push_back(rule + " ::= " + body);
+      return rule;
+    }
+    if (const Json* en = s.get("enum")) {
+      if (en->type != Json::kArray || en->items.empty()) fail(XG_ERR_UNSUPPORTED, "schema: enum must be a non-empty array");
+      std::string out = "(";
+      for (size_t k = 0; k < en->items.size(); ++k) {
+        const Json& v = en->items[k];
+        std::string text;
+        if (v.type == Json::kString) text = json_string_text(v.text);
+        else if (v.type == Json::kNumber) text = v.text;
+        else if (v.type == Json::kBool) text = v.boolean ? "true" : "false";
+        else if (v.type == Json::kNull) text = "null";
+        else fail(XG_ERR_UNSUPPORTED, "schema: enum values must be scalars");
+        out += (k ? " | " : " ") + literal(text);
+      }
+      return out + " )";
+    }
+    static const char* known[] = {"type", "properties", "required", "items", "minItems", "maxItems", "minLength", "maxLength", "$defs", "additionalProperties", "description", "title"};
+    for (auto& m : s.members) {
+      bool ok = false;
+      for (const char* k : known) ok = ok || m.first == k;
+      if (!ok) fail(XG_ERR_UNSUPPORTED, "schema: unsupported keyword " + m.first);
+    }
+    const Json* type = s.get("type");
+    if (!type || type->type != Json::kString) fail(XG_ERR_UNSUPPORTED, "schema: missing type");
+    const std::string& t = type->text;
+    if (t == "object") return object(s);
+    if (t == "array") return array(s);
+    if (t == "string") {
+      int lo = bound(s, "minLength", 0), hi = bound(s, "maxLength", -1);
+      if (hi >= 0 && hi < lo) fail(XG_ERR_PARSE, "schema: maxLength < minLength");
+      std::string key = "string_" + std::to_string(lo) + "_" + (hi < 0 ? std::string("inf") : std::to_string(hi));
+      return shared(key, "\"\\\"\" " + char_rule() + repetition(lo, hi) + " \"\\\"\"");
+    }
+    if (t == "integer") return shared("integer", "\"-\"? ( \"0\" | [1-9] [0-9]* )");
+    if (t == "number") return shared("number", "\"-\"? ( \"0\" | [1-9] [0-9]* ) ( \".\" [0-9]+ )? ( [eE] [+\\-]? [0-9]+ )?");
+    if (t == "boolean") return shared("boolean", "\"true\" | \"false\"");
+    if (t == "null") return shared("null", "\"null\"");
+    fail(XG_ERR_UNSUPPORTED, "schema: unsupported type " + t);
+  }
+
+ private:
+  const Json* defs_;
+  std::string prefix_;
+  std::map<std::string, std::string> def_rule_, shared_rule_;
+  int counter_ = 0;
+  std::string fresh(const std::string& hint) { return prefix_ + hint + "_" + std::to_string(++counter_); }
+  std::string shared(const std::string& hint, const std::string& body) {
+    auto it = shared_rule_.find(hint);
+    if (it != shared_rule_.end()) return it->second;
+    std::string rule = prefix_ + "json_" + hint;
+    shared_rule_[hint] = rule;
+    rules.push_back(rule + " ::= " + body);
+    return rule;
+  }
+  std::string char_rule() { return shared("char", "[^\"\\\\\\x00-\\x1f] | \"\\\\\" ( [\"\\\\/bfnrt] | \"u\" [0-9a-fA-F]{4} )"); }
+  static int bound(const Json& s, const char* key, int dflt) {
+    const Json* v = s.get(key);
+    if (!v) return dflt;
+    if (v->type != Json::kNumber) fail(XG_ERR_PARSE, std::string("schema: ") + key + " must be a number");
+    int n = atoi(v->text.c_str());
+    if (n < 0 || n > 100000) fail(XG_ERR_UNSUPPORTED, std::string("schema: ") + key + " out of range");
+    return n;
+  }
+  static std::string repetition(int lo, int hi) {
+    if (hi < 0) return lo == 0 ? "*" : "{" + std::to_string(lo) + ",}";
+    return "{" + std::to_string(lo) + "," + std::to_string(hi) + "}";
+  }
+  std::string object(const Json& s) {
+    const Json* props = s.get("properties");
+    const Json* req = s.get("required");
+    if (const Json* ap = s.get("additionalProperties")) if (ap->type != Json::kBool || ap->boolean) fail(XG_ERR_UNSUPPORTED, "schema: additionalProperties must be false");
+    if (props && props->type != Json::kObject) fail(XG_ERR_PARSE, "schema: properties must be an object");
+    size_t n = props ? props->members.size() : 0;
+    if (req) {
+      if (req->type != Json::kArray || req->items.size() != n) fail(XG_ERR_UNSUPPORTED, "schema: every property must be required, in declared order");
+      for (size_t k = 0; k < n; ++k) if (req->items[k].type != Json::kString || req->items[k].text != props->members[k].first) fail(XG_ERR_UNSUPPORTED, "schema: every property must be required, in declared order");
+    }
+    if (n == 0) return "\"{}\"";
+    std::string body;
+    for (size_t k = 0; k < n; ++k) {
+      std::string lead = (k ? ", " : "{") + json_string_text(props->members[k].first) + ": ";
+      body += literal(lead) + " " + lower(props->members[k].second) + " ";
+    }
+    body += "\"}\"";
+    std::string rule = fresh("object");
+    rules.push_back(rule + " ::= " + body);
+    return rule;
+  }
+  std::string array(const Json& s) {
+    const Json* items = s.get("items");
+    if (!items) fail(XG_ERR_UNSUPPORTED, "schema: array without items");
+    int lo = bound(s, "minItems", 0), hi = bound(s, "maxItems", -1);
+    if (hi >= 0 && hi < lo) fail(XG_ERR_PARSE, "schema: maxItems < minItems");
+    if (hi == 0) return "\"[]\"";
+    std::string item = lower(*items);
+    std::string more = "( \", \" " + item + " )" + repetition(std::max(lo - 1, 0), hi < 0 ? -1 : hi - 1);
+    std::string rule = fresh("array");
+    if (lo == 0) rules.push_back(rule + " ::= \"[\" ( " + item + " " + more + " )? \"]\"");
+    else rules.push_back(rule + " ::= \"[\" " + item + " " + more + " \"]\"");
+    return rule;
+  }
+};
+
+}  // namespace
+
+std::string json_schema_to_ebnf(const std::string& schema_json, const std::string& root_name, const std::string& prefix) {
+  Json schema = JsonReader(schema_json).run();
+  SchemaLowering low(schema.get("$defs"), prefix);
+  std::string body = low.lower(schema);
+  std::string out = root_name + " ::= " + body + "\n";
+  for (auto& r : low.rules) out += r + "\n";
+  return out;
+}
+
+std::string tag_dispatch_to_ebnf(const std::string& spec_json) {
+  Json spec = JsonReader(spec_json).run();
+  const Json* tags = spec.get("tags");
+  if (!tags || tags->type != Json::kArray || tags->items.empty()) fail(XG_ERR_PARSE, "TagDispatch spec: \"tags\" must be a non-empty array");
+  std::string rules, pairs;
+  for (size_t ti = 0; ti < tags->items.size(); ++ti) {
+    const Json& tag = tags->items[ti];
+    const Json* text = tag.get("tag");
+    const Json* tools = tag.get("tools");
+    const Json* end = tag.get("end");
+    if (!text || text->type != Json::kString || text->text.empty()) fail(XG_ERR_PARSE, "TagDispatch spec: missing tag string");
+    if (!tools || tools->type != Json::kArray || tools->items.empty()) fail(XG_ERR_PARSE, "TagDispatch spec: \"tools\" must be a non-empty array");
+    std::string calls;
+    for (size_t k = 0; k < tools->items.size(); ++k) {
+      const Json* name = tools->items[k].get("name");
+      const Json* schema = tools->items[k].get("schema");
+      if (!name || name->type != Json::kString || !schema) fail(XG_ERR_PARSE, "TagDispatch spec: a tool needs \"name\" and \"schema\"");
+      std::string prefix = "tool" + std::to_string(ti) + "_" + std::to_string(k) + "_";
+      SchemaLowering low(schema->get("$defs"), prefix);
+      std::string args = low.lower(*schema);
+      for (auto& r : low.rules) rules += r + "\n";
+      rules += prefix + "call ::= " + literal("{\"name\": " + json_string_text(name->text) + ", \"arguments\": ") + " " + args + " \"}\"\n";
+      calls += (k ? " | " : "") + prefix + "call";
+    }
+    std::string rule = "dispatch_" + std::to_string(ti);
+    rules += rule + " ::= ( " + calls + " ) " + literal(end && end->type == Json::kString ? end->text : "") + "\n";
+    pairs += (ti ? ", " : "") + std::string("(") + literal(text->text) + ", " + rule + ")";
+  }
+  std::string stops;
+  if (const Json* ss = spec.get("stop_strs")) {
+    if (ss->type != Json::kArray) fail(XG_ERR_PARSE, "TagDispatch spec: stop_strs must be an array");
+    for (size_t k = 0; k < ss->items.size(); ++k) stops += (k ? ", " : "") + literal(ss->items[k].text);
+  }
+  return "root ::= TagDispatch(" + pairs + ", stop_strs=(" + stops + "))\n" + rules;
+}
+
+FlatGrammar compile_frontend(int kind, const std::string& text, const std::string& root, const FrontendOptions& opt) {
+  std::string ebnf;
+  if (kind == kEbnf) ebnf = text;
+  else if (kind == kJsonSchema) ebnf = json_schema_to_ebnf(text, "root", "");
+  else if (kind == kTagDispatchJson) ebnf = tag_dispatch_to_ebnf(text);
+  else fail(XG_ERR_INVALID_ARG, "unknown grammar kind");
+
+  auto parsed = GrammarParser(Lexer(ebnf).run()).run();
+  Compiler c;
+  c.opt = opt;
+  for (auto& r : parsed) {
+    if (c.b.ids.count(r.first)) fail(XG_ERR_PARSE, "grammar text: rule defined twice: " + r.first);
+    c.b.ids[r.first] = (int)c.b.names.size();
+    c.b.names.push_back(r.first);
+  }
+  std::string root_name = (kind == kEbnf && !root.empty()) ? root : "root";
+  c.root = c.b.lookup(root_name);
+  for (auto& r : parsed) {
+    Fsm f;
+    auto p = c.b.frag(f, *r.second);
+    f.start = p.first;
+    f.fin[p.second] = 1;
+    if (f.size() > opt.max_rule_states) fail(XG_ERR_CAPACITY, "rule " + r.first + " exceeds max_rule_states");
+    c.b.rules.push_back(std::move(f));
+  }
+  c.remove_nullability();
+  for (Fsm& f : c.b.rules) f = normalize(f, opt.max_rule_states);
+  c.trim();
+  c.inline_small_rules();
+  c.trim();
+  for (Fsm& f : c.b.rules) f = canonical_order(minimize(f));
+  return c.flatten();
+}
+
+}  // namespace xg
