@@ -1,0 +1,66 @@
+// Plain structs shared by host code and kernels (all pointers are device pointers).
+#pragma once
+#include <cstdint>
+
+namespace xg {
+
+// Vocabulary, sorted by token bytes (trie order): tokens that share a prefix are adjacent, so
+// neighbouring lanes of a warp walk the same automaton path for the shared prefix.
+struct VocabDev {
+  int32_t vocab_size;        // V
+  int32_t n_words;           // ceil(V / 32)
+  int32_t eos_id;            // -1 if none
+  int32_t max_len;           // longest token in bytes
+  const uint8_t* bytes;      // arena in rank order
+  const uint32_t* offset;    // [V+1] by rank
+  const int32_t* rank_to_id; // [V]
+  const int32_t* id_to_rank; // [V]
+  const uint8_t* never;      // [V] by rank: 1 = EOS, special or zero-length (never classified)
+};
+
+// One adaptive cache entry (Section 3.4): the accepted/rejected split in its smallest form plus
+// the uncertain tokens, the latter twice: by ascending id (set algebra) and by ascending rank
+// (the order they are walked in).
+struct EntryDev {
+  const uint32_t* data;      // accepted ids | rejected ids | accepted bitset (n_words words)
+  const uint32_t* unc_id;    // [n_unc] ascending token ids
+  const uint32_t* unc_rank;  // [n_unc] ascending ranks
+  int32_t kind;              // xg_store_kind_t
+  int32_t n_list;            // list length (0 for bitset)
+  int32_t n_unc;
+  int32_t n_acc;
+};
+
+struct GrammarDev {
+  int32_t n_states, n_rules, n_classes;
+  int32_t root_rule, root_nullable, root_start;
+  const uint32_t* state_info;     // [S] rule id | (accepting << 31)
+  const int32_t* scan_begin;      // [S+1]
+  const int32_t* scan_own_end;    // [S]   own edges are [scan_begin, scan_own_end)
+  const uint32_t* scan_class;
+  const uint32_t* scan_target;    // bit 31: origin = the set being scanned
+  const int32_t* wait_begin;      // [S+1]
+  const uint32_t* wait_rule;
+  const uint32_t* wait_target;    // bit 31: origin = the set the completed rule started in
+  const int32_t* gather_begin;    // [S+1]
+  const int32_t* gather_state;
+  const uint32_t* class_bits;     // [C][8]
+  const EntryDev* entries;        // [S]; meaningful for scannable states
+};
+
+// One request's Earley chart.  Only "kernel" items (made by scan or complete) are stored; the
+// predicted items of a set are implied by the grammar's per-state lists.
+struct MatcherDev {
+  const GrammarDev* grammar;
+  uint32_t* item_state;
+  int32_t* item_origin;
+  int32_t* set_begin;        // [cap_sets + 1]
+  int32_t n_sets, n_items;
+  int32_t cap_sets, cap_items;
+  int32_t terminated;
+  int32_t pad;
+};
+
+constexpr uint32_t kSelf = 0x80000000u;
+
+}  // namespace xg

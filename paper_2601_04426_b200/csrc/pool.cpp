@@ -1,0 +1,239 @@
+#include "pool.h"
+
+#include <algorithm>
+#include <functional>
+
+namespace xg {
+
+// tags of Algorithm 1 (any distinct constants) and the placeholder of Algorithm 2
+static const uint64_t kNodeTag = 0x4E4F44455F544147ull, kRangeTag = 0x52414E47455F5447ull, kRefTag = 0x5245465F5F544147ull,
+                      kPlaceholder = 0x58585F484F4C4445ull, kSccRefTag = 0x5343435F5F524546ull, kRuleTag = 0x52554C455F544147ull;
+
+uint64_t hash_fold(uint64_t h, uint64_t x) {
+  uint64_t z = (h ^ x) + 0x9E3779B97F4A7C15ull + (h << 6) + (h >> 2);
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+CachePool::~CachePool() {
+  for (void* p : chunks_) cudaFree(p);
+}
+
+void* CachePool::allocate_device(size_t bytes) {
+  void* p = nullptr;
+  if (cudaMalloc(&p, bytes) != cudaSuccess) return nullptr;
+  chunks_.push_back(p);
+  return p;
+}
+
+int CachePool::find_or_add(uint64_t hash, std::vector<uint64_t>&& serial) {
+  auto& bucket = by_hash_[hash];
+  for (int id : bucket) if (rules_[id].serial == serial) return id;     // equal hash is not trusted on its own
+  PoolRule r;
+  r.hash = hash;
+  r.serial = std::move(serial);
+  rules_.push_back(std::move(r));
+  bucket.push_back((int)rules_.size() - 1);
+  return (int)rules_.size() - 1;
+}
+
+namespace {
+
+struct OutEdge {
+  bool is_ref;
+  int lo, hi;       // byte range (a class edge is split into its maximal ranges)
+  int rule;         // referenced rule
+  int target;       // state offset inside the rule
+};
+
+struct RuleShape {
+  int first = 0, n = 0;                       // states [first, first + n)
+  std::vector<std::vector<OutEdge>> out;      // by state offset
+  std::vector<char> fin;
+  int start = 0;
+};
+
+RuleShape shape_of(const FlatGrammar& g, int r, int first, int n) {
+  RuleShape sh;
+  sh.first = first; sh.n = n; sh.start = g.rule_start[r] - first;
+  sh.out.resize(n); sh.fin.resize(n);
+  for (int k = 0; k < n; ++k) {
+    const int s = first + k;
+    sh.fin[k] = g.state_final[s];
+    for (int e = g.cedge_begin[s]; e < g.cedge_begin[s + 1]; ++e) {
+      const uint32_t* bits = &g.class_bits[(size_t)g.cedge_class[e] * 8];
+      int b = 0;
+      while (b < 256) {
+        if (!((bits[b >> 5] >> (b & 31)) & 1u)) { ++b; continue; }
+        int lo = b;
+        while (b < 256 && ((bits[b >> 5] >> (b & 31)) & 1u)) ++b;
+        sh.out[k].push_back({false, lo, b - 1, -1, g.cedge_target[e] - first});
+      }
+    }
+    for (int e = g.redge_begin[s]; e < g.redge_begin[s + 1]; ++e) sh.out[k].push_back({true, 0, 0, g.redge_rule[e], g.redge_target[e] - first});
+  }
+  return sh;
+}
+
+// Phase 1 of Algorithm 1: sort the out-edges (ranges by (min, max), references by the hash of
+// the referenced rule), breadth-first search from the start state, canonical ids in discovery
+// order.  Returns canonical index -> state offset.
+std::vector<int> canonical_states(RuleShape& sh, const std::vector<uint64_t>& ref_hash) {
+  for (auto& es : sh.out)
+    std::stable_sort(es.begin(), es.end(), [&](const OutEdge& a, const OutEdge& b) {
+      if (a.is_ref != b.is_ref) return !a.is_ref;
+      if (!a.is_ref) return a.lo != b.lo ? a.lo < b.lo : a.hi < b.hi;
+      if (ref_hash[a.rule] != ref_hash[b.rule]) return ref_hash[a.rule] < ref_hash[b.rule];
+      return a.rule < b.rule;
+    });
+  std::vector<int> order{sh.start}, id(sh.n, -1);
+  id[sh.start] = 0;
+  for (size_t q = 0; q < order.size(); ++q)
+    for (const OutEdge& e : sh.out[order[q]]) if (id[e.target] < 0) { id[e.target] = (int)order.size(); order.push_back(e.target); }
+  return order;
+}
+
+// Phase 2 of Algorithm 1
+uint64_t hash_rule(const RuleShape& sh, const std::vector<int>& order, const std::vector<uint64_t>& ref_hash) {
+  std::vector<int> id(sh.n, -1);
+  for (size_t k = 0; k < order.size(); ++k) id[order[k]] = (int)k;
+  uint64_t h = 0;
+  for (int s : order) {
+    h = hash_fold(hash_fold(h, kNodeTag), sh.fin[s] ? 1 : 0);
+    for (const OutEdge& e : sh.out[s]) {
+      if (!e.is_ref) h = hash_fold(hash_fold(hash_fold(hash_fold(h, kRangeTag), (uint64_t)e.lo), (uint64_t)e.hi), (uint64_t)id[e.target]);
+      else h = hash_fold(hash_fold(hash_fold(h, kRefTag), ref_hash[e.rule]), (uint64_t)id[e.target]);
+    }
+  }
+  return h;
+}
+
+struct Analysis {
+  std::vector<RuleShape> shapes;
+  std::vector<std::vector<int>> adj, comps;     // comps: strongly connected components, callees first
+  std::vector<int> comp;
+  RuleInterning out;
+  bool cyclic(const std::vector<int>& members) const {
+    return members.size() > 1 || std::binary_search(adj[members[0]].begin(), adj[members[0]].end(), members[0]);
+  }
+};
+
+Analysis analyse(const FlatGrammar& g) {
+  const int R = g.n_rules;
+  Analysis a;
+  RuleInterning& out = a.out;
+  out.pool_id.assign(R, -1);
+  out.canon.resize(R);
+  out.hash.assign(R, 0);
+  std::vector<int> first(R + 1, g.n_states);
+  for (int s = g.n_states - 1; s >= 0; --s) first[g.state_rule[s]] = s;
+  a.shapes.resize(R);
+  for (int r = 0; r < R; ++r) a.shapes[r] = shape_of(g, r, first[r], first[r + 1] - first[r]);
+  a.adj.resize(R);
+  for (int r = 0; r < R; ++r) {
+    for (auto& es : a.shapes[r].out) for (const OutEdge& e : es) if (e.is_ref) a.adj[r].push_back(e.rule);
+    std::sort(a.adj[r].begin(), a.adj[r].end());
+    a.adj[r].erase(std::unique(a.adj[r].begin(), a.adj[r].end()), a.adj[r].end());
+  }
+  // strongly connected components (Tarjan); components come out callees first
+  std::vector<int> index(R, -1), low(R, 0), stack;
+  a.comp.assign(R, -1);
+  std::vector<char> on_stack(R, 0);
+  int counter = 0;
+  std::function<void(int)> dfs = [&](int u) {
+    index[u] = low[u] = counter++;
+    stack.push_back(u); on_stack[u] = 1;
+    for (int w : a.adj[u]) {
+      if (index[w] < 0) { dfs(w); low[u] = std::min(low[u], low[w]); }
+      else if (on_stack[w]) low[u] = std::min(low[u], index[w]);
+    }
+    if (low[u] == index[u]) {
+      a.comps.emplace_back();
+      while (true) { int w = stack.back(); stack.pop_back(); on_stack[w] = 0; a.comp[w] = (int)a.comps.size() - 1; a.comps.back().push_back(w); if (w == u) break; }
+    }
+  };
+  for (int r = 0; r < R; ++r) if (index[r] < 0) dfs(r);
+
+  std::vector<uint64_t> ref_hash(R, kPlaceholder);     // unresolved references hash as the placeholder
+  for (auto& members : a.comps) {
+    if (!a.cyclic(members)) {
+      const int r = members[0];
+      out.canon[r] = canonical_states(a.shapes[r], ref_hash);
+      out.hash[r] = hash_rule(a.shapes[r], out.canon[r], ref_hash);
+      ref_hash[r] = out.hash[r];
+      continue;
+    }
+    // Local hashes with the placeholder on in-cycle references, then the refinement of
+    // Algorithm 2: fold the local hashes starting from each member.  For a simple cycle the
+    // members are visited in cycle order (the rotation of Algorithm 2); for a denser component,
+    // in breadth-first order of the reference edges.
+    std::vector<uint64_t> local(R, 0);
+    for (int r : members) {
+      out.canon[r] = canonical_states(a.shapes[r], ref_hash);
+      local[r] = hash_rule(a.shapes[r], out.canon[r], ref_hash);
+    }
+    for (int r : members) {
+      std::vector<int> seq{r};
+      std::vector<char> seen(R, 0);
+      seen[r] = 1;
+      for (size_t q = 0; q < seq.size(); ++q) {
+        const RuleShape& sh = a.shapes[seq[q]];
+        for (int s : out.canon[seq[q]])
+          for (const OutEdge& e : sh.out[s]) if (e.is_ref && a.comp[e.rule] == a.comp[r] && !seen[e.rule]) { seen[e.rule] = 1; seq.push_back(e.rule); }
+      }
+      uint64_t h = 0;
+      for (int m : seq) h = hash_fold(h, local[m]);
+      out.hash[r] = h;
+    }
+    for (int r : members) ref_hash[r] = out.hash[r];
+    // the hashes of in-cycle references changed the sort keys: fix the canonical orders again
+    for (int r : members) out.canon[r] = canonical_states(a.shapes[r], ref_hash);
+  }
+  return a;
+}
+
+}  // namespace
+
+RuleInterning structural_hashes(const FlatGrammar& g) { return analyse(g).out; }
+
+RuleInterning CachePool::intern(const FlatGrammar& g) {
+  Analysis a = analyse(g);
+  RuleInterning& out = a.out;
+  const int R = g.n_rules;
+  // exact identities: serialise each rule with its callees named by pool id; members of a
+  // cycle are serialised jointly, named by discovery order from the rule being keyed
+  for (auto& members : a.comps) {
+    const bool cyclic = a.cyclic(members);
+    for (int r : members) {
+      std::vector<int> seq{r};
+      std::vector<int> local_id(R, -1);
+      local_id[r] = 0;
+      std::vector<uint64_t> serial;
+      for (size_t q = 0; q < seq.size(); ++q) {
+        const int m = seq[q];
+        const RuleShape& sh = a.shapes[m];
+        std::vector<int> id(sh.n, -1);
+        for (size_t k = 0; k < out.canon[m].size(); ++k) id[out.canon[m][k]] = (int)k;
+        serial.push_back(kRuleTag);
+        serial.push_back((uint64_t)out.canon[m].size());
+        for (int s : out.canon[m]) {
+          serial.push_back(kNodeTag); serial.push_back(sh.fin[s] ? 1 : 0);
+          for (const OutEdge& e : sh.out[s]) {
+            if (!e.is_ref) { serial.push_back(kRangeTag); serial.push_back(((uint64_t)e.lo << 8) | (uint64_t)e.hi); serial.push_back((uint64_t)id[e.target]); }
+            else if (cyclic && a.comp[e.rule] == a.comp[r]) {
+              if (local_id[e.rule] < 0) { local_id[e.rule] = (int)seq.size(); seq.push_back(e.rule); }
+              serial.push_back(kSccRefTag); serial.push_back((uint64_t)local_id[e.rule]); serial.push_back((uint64_t)id[e.target]);
+            } else { serial.push_back(kRefTag); serial.push_back((uint64_t)out.pool_id[e.rule]); serial.push_back((uint64_t)id[e.target]); }
+          }
+        }
+      }
+      // pool ids of cycle members are only read by rules outside the cycle, so they can be
+      // assigned one by one
+      out.pool_id[r] = find_or_add(out.hash[r], std::move(serial));
+    }
+  }
+  return out;
+}
+
+}  // namespace xg

@@ -1,0 +1,61 @@
+// Cross-grammar cache pool (Section 3.3): rule automata are keyed by a structural hash
+// (Algorithm 1; cycles as in Algorithm 2) and verified against their canonical serialisation,
+// so identical sub-structures are classified once and shared between grammars.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <mutex>
+#include <unordered_map>
+#include <vector>
+
+#include "device_types.h"
+#include "frontend.h"
+
+namespace xg {
+
+struct PoolRule {
+  std::vector<uint64_t> serial;      // canonical serialisation (the exact identity of the rule)
+  uint64_t hash = 0;
+  bool built = false;
+  std::vector<EntryDev> entries;     // by canonical state index
+  std::vector<int2> counts;          // (accepted, uncertain) by canonical state index
+};
+
+// How one grammar's rules map onto the pool.
+struct RuleInterning {
+  std::vector<int> pool_id;                 // rule -> pool rule
+  std::vector<std::vector<int>> canon;      // rule -> canonical index -> state offset inside the rule
+  std::vector<uint64_t> hash;               // rule -> structural hash
+};
+
+// Hashes and canonical state orders only (no pool): Algorithm 1 bottom-up over the reference
+// graph, Algorithm 2's refinement on cycles.
+RuleInterning structural_hashes(const FlatGrammar& g);
+
+class CachePool {
+ public:
+  explicit CachePool(const void* owner) : owner_(owner) {}
+  ~CachePool();
+  const void* owner() const { return owner_; }
+  std::mutex mu;                            // one compile at a time per pool
+
+  // find-or-create pool rules for every rule of `g`, callees first (call with `mu` held)
+  RuleInterning intern(const FlatGrammar& g);
+  PoolRule& rule(int id) { return rules_[id]; }
+  size_t n_rules() const { return rules_.size(); }
+  void* allocate_device(size_t bytes);      // lives as long as the pool
+
+ private:
+  const void* owner_;
+  std::vector<PoolRule> rules_;
+  std::unordered_map<uint64_t, std::vector<int>> by_hash_;
+  std::vector<void*> chunks_;
+  int find_or_add(uint64_t hash, std::vector<uint64_t>&& serial);
+};
+
+// The order-sensitive hash of Algorithm 1 (the paper leaves it open; this is a 64-bit
+// multiply-xorshift fold).
+uint64_t hash_fold(uint64_t h, uint64_t x);
+
+}  // namespace xg
