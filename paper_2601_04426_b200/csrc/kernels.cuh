@@ -1,0 +1,558 @@
+// CUDA kernels of the token-mask path (sm_100a).  Integer / bit work only: nothing here is a
+// dense contraction, so no tensor cores; the rules that matter are coalesced streaming, work
+// that follows the trie order of the vocabulary, and grids sized to fill 148 SMs.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "device_types.h"
+
+namespace xg {
+
+enum : int { kWalkUncertain = 1, kWalkOverflow = 2 };
+
+constexpr int kFastCap = 48;     // items a token walk may create before it falls back
+constexpr int kFastMaxBytes = 32;
+constexpr int kSlowCap = 2048;
+constexpr int kSlowMaxBytes = 255;
+
+// ------------------------------------------------------------------------------------------
+// The token walk: Earley scan / complete over the bytes of one token (appendix "Earley's
+// Parsing Algorithm"), on kernel items only.
+//
+// Base chart: sets 0..n given by (h_st, h_org, h_sb); the walk starts from set n.  New sets are
+// appended to (st, org) with boundaries lsb[j] .. lsb[j+1] for the set reached after byte j
+// (1-based), and carry chart indices n+j.  Origin -1 stands for the unknown context of a cache
+// entry (Section 3.4): completing such an item cannot advance anything that is known here.
+//
+// Returns the number of bytes after which the set was still non-empty (len = token survives).
+// ------------------------------------------------------------------------------------------
+template <typename LsbT>
+__device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* h_st, const int32_t* h_org, const int32_t* h_sb, int n,
+                                          const uint8_t* __restrict__ bytes, int len, bool own_edges_first,
+                                          uint32_t* st, int32_t* org, int cap, LsbT* lsb, int* flags) {
+  int cnt = 0;
+  int cur_b = h_sb[n], cur_e = h_sb[n + 1];
+  bool cur_hist = true;
+  lsb[0] = 0;
+  lsb[1] = 0;
+  for (int k = 0; k < len; ++k) {
+    const uint32_t byte = bytes[k];
+    const uint32_t word = byte >> 5, bit = 1u << (byte & 31);
+    const int start = cnt;
+    const int self_idx = n + k;
+    // scan
+    for (int i = cur_b; i < cur_e; ++i) {
+      const uint32_t s = cur_hist ? h_st[i] : st[i];
+      const int32_t o = cur_hist ? h_org[i] : org[i];
+      const int e0 = g.scan_begin[s];
+      const int e1 = (k == 0 && own_edges_first) ? g.scan_own_end[s] : g.scan_begin[s + 1];
+      for (int e = e0; e < e1; ++e) {
+        if (g.class_bits[g.scan_class[e] * 8 + word] & bit) {
+          const uint32_t t = g.scan_target[e];
+          const uint32_t ns = t & ~kSelf;
+          const int32_t no = (t & kSelf) ? self_idx : o;
+          bool dup = false;
+          for (int q = start; q < cnt; ++q) dup = dup || (st[q] == ns && org[q] == no);
+          if (!dup) {
+            if (cnt >= cap) { *flags |= kWalkOverflow; return k; }
+            st[cnt] = ns; org[cnt] = no; ++cnt;
+          }
+        }
+      }
+    }
+    if (cnt == start) return k;
+    // complete (cascades through the growing set)
+    for (int q = start; q < cnt; ++q) {
+      const uint32_t info = g.state_info[st[q]];
+      if (!(info >> 31)) continue;
+      const uint32_t rule = info & 0x7FFFFFFFu;
+      const int32_t o = org[q];
+      if (o < 0) { if (k + 1 < len) *flags |= kWalkUncertain; continue; }
+      int b, e;
+      const bool hist = o <= n;
+      if (hist) { b = h_sb[o]; e = h_sb[o + 1]; } else { b = lsb[o - n]; e = lsb[o - n + 1]; }
+      for (int i = b; i < e; ++i) {
+        const uint32_t s2 = hist ? h_st[i] : st[i];
+        const int32_t o2 = hist ? h_org[i] : org[i];
+        for (int w = g.wait_begin[s2]; w < g.wait_begin[s2 + 1]; ++w) {
+          if (g.wait_rule[w] != rule) continue;
+          const uint32_t t = g.wait_target[w];
+          const uint32_t ns = t & ~kSelf;
+          const int32_t no = (t & kSelf) ? o : o2;
+          bool dup = false;
+          for (int z = start; z < cnt; ++z) dup = dup || (st[z] == ns && org[z] == no);
+          if (!dup) {
+            if (cnt >= cap) { *flags |= kWalkOverflow; return k; }
+            st[cnt] = ns; org[cnt] = no; ++cnt;
+          }
+        }
+      }
+    }
+    cur_b = start; cur_e = cnt; cur_hist = false;
+    lsb[k + 2] = (LsbT)cnt;
+  }
+  return len;
+}
+
+// ------------------------------------------------------------------------------------------
+// Cache build (Section 3.4; appendix on the adaptive token mask cache): classify every
+// (scannable state, token) pair.  grid.y = position, grid.x * block = token rank (trie order).
+// Accepted and uncertain bits are scattered into id-ordered rows; the uncertain bits are also
+// ballot-packed in rank order (the order later walks use).
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
+                uint32_t* __restrict__ acc_id, uint32_t* __restrict__ unc_id, uint32_t* __restrict__ unc_rank,
+                int2* __restrict__ overflow, int* __restrict__ overflow_count, int overflow_cap) {
+  __shared__ uint32_t sh_st[1];
+  __shared__ int32_t sh_org[1];
+  __shared__ int32_t sh_sb[2];
+  const int pos = blockIdx.y;
+  if (threadIdx.x == 0) { sh_st[0] = (uint32_t)positions[pos]; sh_org[0] = -1; sh_sb[0] = 0; sh_sb[1] = 1; }
+  __syncthreads();
+  const int rank = blockIdx.x * blockDim.x + threadIdx.x;
+  int cls = 0;
+  if (rank < v.vocab_size && !v.never[rank]) {
+    const uint32_t off = v.offset[rank];
+    const int len = (int)(v.offset[rank + 1] - off);
+    int flags = 0;
+    int consumed = 0;
+    if (len > kFastMaxBytes) flags = kWalkOverflow;
+    else {
+      uint32_t st[kFastCap];
+      int32_t org[kFastCap];
+      int16_t lsb[kFastMaxBytes + 2];
+      consumed = token_walk<int16_t>(g, sh_st, sh_org, sh_sb, 0, v.bytes + off, len, true, st, org, kFastCap, lsb, &flags);
+    }
+    if (flags & kWalkOverflow) {
+      int slot = atomicAdd(overflow_count, 1);
+      if (slot < overflow_cap) overflow[slot] = make_int2(pos, rank);
+    } else if (consumed == len) cls = 1;
+    else if (flags & kWalkUncertain) cls = 2;
+    if (cls) {
+      const int id = v.rank_to_id[rank];
+      uint32_t* row = (cls == 1 ? acc_id : unc_id) + (size_t)pos * v.n_words;
+      atomicOr(&row[id >> 5], 1u << (id & 31));
+    }
+  }
+  const uint32_t ballot = __ballot_sync(0xFFFFFFFFu, cls == 2);
+  if ((threadIdx.x & 31) == 0 && rank < v.vocab_size) unc_rank[(size_t)pos * v.n_words + (rank >> 5)] = ballot;
+}
+
+// exact fallback for the pairs whose walk did not fit the fast path's fixed arrays
+__global__ void classify_slow_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
+                                     const int2* __restrict__ pairs, int n_pairs, uint32_t* scratch_st, int32_t* scratch_org,
+                                     int32_t* scratch_lsb, uint32_t* acc_id, uint32_t* unc_id, uint32_t* unc_rank,
+                                     int* __restrict__ failed) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_pairs) return;
+  const int pos = pairs[i].x, rank = pairs[i].y;
+  uint32_t h_st = (uint32_t)positions[pos];
+  int32_t h_org = -1;
+  int32_t h_sb[2] = {0, 1};
+  const uint32_t off = v.offset[rank];
+  const int len = (int)(v.offset[rank + 1] - off);
+  if (len > kSlowMaxBytes) { atomicExch(failed, 1); return; }
+  int flags = 0;
+  int consumed = token_walk<int32_t>(g, &h_st, &h_org, h_sb, 0, v.bytes + off, len, true, scratch_st + (size_t)i * kSlowCap,
+                                     scratch_org + (size_t)i * kSlowCap, kSlowCap, scratch_lsb + (size_t)i * (kSlowMaxBytes + 2), &flags);
+  if (flags & kWalkOverflow) { atomicExch(failed, 1); return; }
+  int cls = consumed == len ? 1 : ((flags & kWalkUncertain) ? 2 : 0);
+  if (!cls) return;
+  const int id = v.rank_to_id[rank];
+  uint32_t* row = (cls == 1 ? acc_id : unc_id) + (size_t)pos * v.n_words;
+  atomicOr(&row[id >> 5], 1u << (id & 31));
+  if (cls == 2) atomicOr(&unc_rank[(size_t)pos * v.n_words + (rank >> 5)], 1u << (rank & 31));
+}
+
+// ------------------------------------------------------------------------------------------
+// Adaptive pack (Section 3.3 "adaptive storage"): per position count, choose the smallest of
+// accepted list / rejected list / bitset, exclusive-scan the sizes, compact.
+// ------------------------------------------------------------------------------------------
+struct PackPlan {
+  long long offset_words;   // into the arena
+  int32_t kind, n_list, n_acc, n_unc;
+};
+
+__device__ __forceinline__ int block_reduce_sum(int x, int* sh) {
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_down_sync(0xFFFFFFFFu, x, o);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = x;
+  __syncthreads();
+  int total = 0;
+  const int nw = (blockDim.x + 31) >> 5;
+  for (int i = 0; i < nw; ++i) total += sh[i];
+  __syncthreads();
+  return total;
+}
+
+__global__ void __launch_bounds__(256)
+count_kernel(const uint32_t* __restrict__ acc_id, const uint32_t* __restrict__ unc_id, int n_words, int2* __restrict__ counts) {
+  __shared__ int sh[8];
+  const size_t base = (size_t)blockIdx.x * n_words;
+  int a = 0, u = 0;
+  for (int w = threadIdx.x; w < n_words; w += blockDim.x) { a += __popc(acc_id[base + w]); u += __popc(unc_id[base + w]); }
+  a = block_reduce_sum(a, sh);
+  u = block_reduce_sum(u, sh);
+  if (threadIdx.x == 0) counts[blockIdx.x] = make_int2(a, u);
+}
+
+// one block: kinds, sizes and arena offsets for all positions of the batch
+__global__ void __launch_bounds__(1024)
+plan_kernel(const int2* __restrict__ counts, int n_pos, int vocab_size, int n_words, PackPlan* __restrict__ plan, long long* __restrict__ total_words) {
+  __shared__ long long sums[1024];
+  const int per = (n_pos + blockDim.x - 1) / blockDim.x;
+  const int lo = min(n_pos, (int)threadIdx.x * per), hi = min(n_pos, lo + per);
+  long long local = 0;
+  for (int p = lo; p < hi; ++p) {
+    const int na = counts[p].x, nu = counts[p].y, nr = vocab_size - na - nu;
+    int kind = 0, n_list = na;                       // ties: accepted list < rejected list < bitset
+    if (nr < n_list) { kind = 1; n_list = nr; }
+    if (n_words < n_list) { kind = 2; n_list = 0; }
+    plan[p].kind = kind; plan[p].n_list = n_list; plan[p].n_acc = na; plan[p].n_unc = nu;
+    local += (kind == 2 ? n_words : n_list) + 2LL * nu;
+  }
+  sums[threadIdx.x] = local;
+  __syncthreads();
+  for (int off = 1; off < (int)blockDim.x; off <<= 1) {
+    long long add = (int)threadIdx.x >= off ? sums[threadIdx.x - off] : 0;
+    __syncthreads();
+    sums[threadIdx.x] += add;
+    __syncthreads();
+  }
+  long long run = sums[threadIdx.x] - local;
+  for (int p = lo; p < hi; ++p) {
+    plan[p].offset_words = run;
+    run += (plan[p].kind == 2 ? n_words : plan[p].n_list) + 2LL * plan[p].n_unc;
+  }
+  if (threadIdx.x == blockDim.x - 1) *total_words = sums[threadIdx.x];
+}
+
+// ascending positions of the set bits of word_fn(w), w in [0, n_words), written to out
+template <typename F>
+__device__ __forceinline__ void compact_bits(F word_fn, int n_words, uint32_t* __restrict__ out, int* sh_scan) {
+  const int per = (n_words + blockDim.x - 1) / blockDim.x;
+  const int lo = min(n_words, (int)threadIdx.x * per), hi = min(n_words, lo + per);
+  int mine = 0;
+  for (int w = lo; w < hi; ++w) mine += __popc(word_fn(w));
+  sh_scan[threadIdx.x] = mine;
+  __syncthreads();
+  for (int off = 1; off < (int)blockDim.x; off <<= 1) {
+    int add = (int)threadIdx.x >= off ? sh_scan[threadIdx.x - off] : 0;
+    __syncthreads();
+    sh_scan[threadIdx.x] += add;
+    __syncthreads();
+  }
+  int at = sh_scan[threadIdx.x] - mine;
+  for (int w = lo; w < hi; ++w) {
+    uint32_t bits = word_fn(w);
+    while (bits) { int j = __ffs(bits) - 1; bits &= bits - 1; out[at++] = (uint32_t)(w * 32 + j); }
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(256)
+pack_kernel(const uint32_t* __restrict__ acc_id, const uint32_t* __restrict__ unc_id, const uint32_t* __restrict__ unc_rank,
+            const PackPlan* __restrict__ plan, int vocab_size, int n_words, uint32_t* __restrict__ arena, EntryDev* __restrict__ entries) {
+  __shared__ int sh_scan[256];
+  const int p = blockIdx.x;
+  const PackPlan pl = plan[p];
+  const uint32_t* a = acc_id + (size_t)p * n_words;
+  const uint32_t* u = unc_id + (size_t)p * n_words;
+  const uint32_t* ur = unc_rank + (size_t)p * n_words;
+  uint32_t* data = arena + pl.offset_words;
+  const int n_data = pl.kind == 2 ? n_words : pl.n_list;
+  uint32_t* out_uid = data + n_data;
+  uint32_t* out_urank = out_uid + pl.n_unc;
+  if (pl.kind == 2) {
+    for (int w = threadIdx.x; w < n_words; w += blockDim.x) data[w] = a[w];
+  } else if (pl.kind == 0) {
+    compact_bits([&](int w) { return a[w]; }, n_words, data, sh_scan);
+  } else {
+    const uint32_t tail = (vocab_size & 31) ? ((1u << (vocab_size & 31)) - 1) : 0xFFFFFFFFu;
+    compact_bits([&](int w) { uint32_t x = ~(a[w] | u[w]); return w == n_words - 1 ? (x & tail) : x; }, n_words, data, sh_scan);
+  }
+  compact_bits([&](int w) { return u[w]; }, n_words, out_uid, sh_scan);
+  compact_bits([&](int w) { return ur[w]; }, n_words, out_urank, sh_scan);
+  if (threadIdx.x == 0) {
+    EntryDev e;
+    e.data = data; e.unc_id = out_uid; e.unc_rank = out_urank;
+    e.kind = pl.kind; e.n_list = pl.n_list; e.n_unc = pl.n_unc; e.n_acc = pl.n_acc;
+    entries[p] = e;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// matcher state
+// ------------------------------------------------------------------------------------------
+__global__ void matcher_reset_kernel(MatcherDev* m) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    m->item_state[0] = (uint32_t)m->grammar->root_start;
+    m->item_origin[0] = 0;
+    m->set_begin[0] = 0;
+    m->set_begin[1] = 1;
+    m->n_sets = 1;
+    m->n_items = 1;
+    m->terminated = 0;
+  }
+}
+
+// is the root rule complete in the current set (EOS allowed)?
+__device__ __forceinline__ bool root_complete(const MatcherDev& m, const GrammarDev& g) {
+  if (m.n_sets == 1 && g.root_nullable) return true;
+  const int n = m.n_sets - 1;
+  for (int i = m.set_begin[n]; i < m.set_begin[n + 1]; ++i) {
+    if (m.item_origin[i] != 0) continue;
+    const uint32_t info = g.state_info[m.item_state[i]];
+    if ((info >> 31) && (info & 0x7FFFFFFFu) == (uint32_t)g.root_rule) return true;
+  }
+  return false;
+}
+
+// Accept one sampled token per request (Section 2.2 "trace the output"): the walk writes its
+// sets straight behind the request's history; they are committed only if every byte survived.
+__global__ void accept_kernel(MatcherDev* const* __restrict__ matchers, int batch, VocabDev v,
+                              const int32_t* __restrict__ token_ids, int32_t* __restrict__ status) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= batch) return;
+  MatcherDev& m = *matchers[b];
+  const GrammarDev& g = *m.grammar;
+  int st = 0;   // XG_OK
+  const int tok = token_ids[b];
+  if (m.terminated) st = -8;
+  else if (tok < 0 || tok >= v.vocab_size) st = -7;
+  else if (tok == v.eos_id) {
+    if (root_complete(m, g)) m.terminated = 1; else st = -7;
+  } else {
+    const int rank = v.id_to_rank[tok];
+    const uint32_t off = v.offset[rank];
+    const int len = (int)(v.offset[rank + 1] - off);
+    if (v.never[rank] || len == 0) st = -7;
+    else {
+      int n_sets = m.n_sets, n_items = m.n_items;
+      int done = 0;
+      while (done < len && st == 0) {            // long tokens go through in pieces
+        const int piece = min(len - done, kFastMaxBytes);
+        if (n_sets + piece > m.cap_sets) { st = -6; break; }
+        int16_t lsb[kFastMaxBytes + 2];
+        int flags = 0;
+        const int room = min(m.cap_items - n_items, 32000);
+        const int consumed = token_walk<int16_t>(g, m.item_state, m.item_origin, m.set_begin, n_sets - 1, v.bytes + off + done, piece,
+                                                 false, m.item_state + n_items, m.item_origin + n_items, room, lsb, &flags);
+        if (flags & kWalkOverflow) { st = -6; break; }
+        if (consumed < piece) { st = -7; break; }
+        // origins written by the walk are already chart indices (its base is set n_sets - 1);
+        // publish the boundaries of the new sets
+        for (int j = 1; j <= piece; ++j) m.set_begin[n_sets + j] = n_items + lsb[j + 1];
+        n_items += lsb[piece + 1];
+        n_sets += piece;
+        done += piece;
+      }
+      if (st == 0) { m.n_sets = n_sets; m.n_items = n_items; }
+    }
+  }
+  if (status) status[b] = st;
+}
+
+// ------------------------------------------------------------------------------------------
+// Per-step mask, part 1: merge the accepted sets of the current scannable states (run-time
+// paragraph of the appendix on the adaptive token mask cache).  grid = (chunks, batch): each
+// block owns a slice of one request's row in shared memory, ORs every entry's accepted tokens
+// into it (bitsets streamed with coalesced loads, sorted lists cut to the slice by binary
+// search) and writes the slice once.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ int lower_bound_u32(const uint32_t* __restrict__ a, int n, uint32_t key) {
+  int lo = 0, hi = n;
+  while (lo < hi) { int mid = (lo + hi) >> 1; if (a[mid] < key) lo = mid + 1; else hi = mid; }
+  return lo;
+}
+
+constexpr int kMergeMaxChunkWords = 2048;
+
+__global__ void __launch_bounds__(256)
+merge_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __restrict__ bitmask, long long row_stride,
+             int32_t* __restrict__ status_user, int32_t* __restrict__ status, int32_t* __restrict__ done_count) {
+  __shared__ uint32_t row[kMergeMaxChunkWords];
+  __shared__ uint32_t tmp[kMergeMaxChunkWords];
+  const int b = blockIdx.y;
+  const MatcherDev& m = *matchers[b];
+  const GrammarDev& g = *m.grammar;
+  const int chunk = (v.n_words + gridDim.x - 1) / gridDim.x;
+  const int w0 = blockIdx.x * chunk, w1 = min(v.n_words, w0 + chunk);
+  const int nw = max(0, w1 - w0);
+  for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] = 0;
+  const bool dead = m.terminated != 0;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    const int s = dead ? -8 : 0;
+    status[b] = s;
+    if (status_user) status_user[b] = s;
+    done_count[b] = 0;
+  }
+  __syncthreads();
+  if (!dead && nw > 0) {
+    const uint32_t id_lo = (uint32_t)w0 * 32u, id_hi = (uint32_t)w1 * 32u;
+    const int n = m.n_sets - 1;
+    for (int i = m.set_begin[n]; i < m.set_begin[n + 1]; ++i) {
+      const uint32_t s = m.item_state[i];
+      for (int gi = g.gather_begin[s]; gi < g.gather_begin[s + 1]; ++gi) {
+        const EntryDev e = g.entries[g.gather_state[gi]];
+        if (e.kind == 2) {
+          for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] |= e.data[w0 + w];
+        } else if (e.kind == 0) {
+          const int lo = lower_bound_u32(e.data, e.n_list, id_lo), hi = lower_bound_u32(e.data, e.n_list, id_hi);
+          for (int k = lo + threadIdx.x; k < hi; k += blockDim.x) { const uint32_t id = e.data[k]; atomicOr(&row[(id >> 5) - w0], 1u << (id & 31)); }
+        } else {
+          // accepted = everything except the rejected and the uncertain tokens
+          const uint32_t tail = (v.vocab_size & 31) ? ((1u << (v.vocab_size & 31)) - 1) : 0xFFFFFFFFu;
+          for (int w = threadIdx.x; w < nw; w += blockDim.x) tmp[w] = (w0 + w == v.n_words - 1) ? tail : 0xFFFFFFFFu;
+          __syncthreads();
+          int lo = lower_bound_u32(e.data, e.n_list, id_lo), hi = lower_bound_u32(e.data, e.n_list, id_hi);
+          for (int k = lo + threadIdx.x; k < hi; k += blockDim.x) { const uint32_t id = e.data[k]; atomicAnd(&tmp[(id >> 5) - w0], ~(1u << (id & 31))); }
+          lo = lower_bound_u32(e.unc_id, e.n_unc, id_lo); hi = lower_bound_u32(e.unc_id, e.n_unc, id_hi);
+          for (int k = lo + threadIdx.x; k < hi; k += blockDim.x) { const uint32_t id = e.unc_id[k]; atomicAnd(&tmp[(id >> 5) - w0], ~(1u << (id & 31))); }
+          __syncthreads();
+          for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] |= tmp[w];
+        }
+        __syncthreads();
+      }
+    }
+    if (threadIdx.x == 0 && v.eos_id >= 0 && (uint32_t)v.eos_id >= id_lo && (uint32_t)v.eos_id < id_hi && root_complete(m, g))
+      row[(v.eos_id >> 5) - w0] |= 1u << (v.eos_id & 31);
+    __syncthreads();
+  }
+  for (int w = threadIdx.x; w < nw; w += blockDim.x) bitmask[(long long)b * row_stride + w0 + w] = (int32_t)row[w];
+}
+
+// ------------------------------------------------------------------------------------------
+// Per-step mask, part 2: check the uncertain tokens of the current scannable states against
+// the request's full Earley state (Section 3.4).  grid = (slices, batch).  The uncertain lists
+// are walked in trie order, one token per lane, so neighbouring lanes share prefixes.
+// The last block of a request to finish clears the row if any of its walks overflowed.
+// ------------------------------------------------------------------------------------------
+constexpr int kMaxStepEntries = 64;
+
+__global__ void __launch_bounds__(256)
+check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __restrict__ bitmask, long long row_stride,
+             int32_t* __restrict__ status_user, int32_t* __restrict__ status, int32_t* __restrict__ done_count) {
+  __shared__ const uint32_t* ent_list[kMaxStepEntries];
+  __shared__ int ent_cum[kMaxStepEntries + 1];
+  __shared__ int ent_state[kMaxStepEntries];
+  __shared__ int n_ent;
+  __shared__ int sh_fail;
+  __shared__ int sh_last;
+  const int b = blockIdx.y;
+  const MatcherDev& m = *matchers[b];
+  const GrammarDev& g = *m.grammar;
+  const int n = m.n_sets - 1;
+  if (threadIdx.x == 0) {
+    int ne = 0, fail = 0;
+    ent_cum[0] = 0;
+    if (!m.terminated) {
+      for (int i = m.set_begin[n]; i < m.set_begin[n + 1] && !fail; ++i) {
+        const uint32_t s = m.item_state[i];
+        for (int gi = g.gather_begin[s]; gi < g.gather_begin[s + 1]; ++gi) {
+          const int q = g.gather_state[gi];
+          bool seen = false;
+          for (int z = 0; z < ne; ++z) seen = seen || ent_state[z] == q;
+          if (seen) continue;
+          const EntryDev& e = g.entries[q];
+          if (e.n_unc == 0) continue;
+          if (ne == kMaxStepEntries) { fail = 1; break; }
+          ent_state[ne] = q; ent_list[ne] = e.unc_rank; ent_cum[ne + 1] = ent_cum[ne] + e.n_unc; ++ne;
+        }
+      }
+    }
+    n_ent = ne;
+    sh_fail = fail;
+  }
+  __syncthreads();
+  const int total = ent_cum[n_ent];
+  uint32_t* row = (uint32_t*)bitmask + (long long)b * row_stride;
+  for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < total; j += gridDim.x * blockDim.x) {
+    int e = 0;
+    while (j >= ent_cum[e + 1]) ++e;
+    const int rank = (int)ent_list[e][j - ent_cum[e]];
+    const int id = v.rank_to_id[rank];
+    if ((row[id >> 5] >> (id & 31)) & 1u) continue;         // already allowed by some cache
+    const uint32_t off = v.offset[rank];
+    const int len = (int)(v.offset[rank + 1] - off);
+    int flags = 0, consumed = 0;
+    if (len > kFastMaxBytes) flags = kWalkOverflow;
+    else {
+      uint32_t st[kFastCap];
+      int32_t org[kFastCap];
+      int16_t lsb[kFastMaxBytes + 2];
+      consumed = token_walk<int16_t>(g, m.item_state, m.item_origin, m.set_begin, n, v.bytes + off, len, false, st, org, kFastCap, lsb, &flags);
+    }
+    if (flags & kWalkOverflow) sh_fail = 1;
+    else if (consumed == len) atomicOr(&row[id >> 5], 1u << (id & 31));
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (sh_fail) atomicExch(&status[b], -6);
+    __threadfence();
+    sh_last = atomicAdd(&done_count[b], 1) == (int)gridDim.x - 1;
+  }
+  __syncthreads();
+  if (sh_last) {
+    __threadfence();
+    const int s = *(volatile int32_t*)&status[b];
+    if (s == -6) {
+      for (int w = threadIdx.x; w < v.n_words; w += blockDim.x) row[w] = 0;
+      if (threadIdx.x == 0 && status_user) status_user[b] = -6;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Mask apply (Section 2.1): logits of disallowed tokens become -inf, in place, one pass.
+// One 16-byte vector per thread and step.  A vector whose tokens are all allowed is skipped
+// (neither read nor written); one whose tokens are all disallowed is overwritten without being
+// read; only mixed vectors are read, blended and written back.
+// ------------------------------------------------------------------------------------------
+template <int ELEMS>   // elements per 16-byte vector: 8 (bf16) or 4 (fp32)
+__global__ void __launch_bounds__(256)
+apply_kernel(void* __restrict__ logits, int vocab_size, long long row_stride_elems, const uint32_t* __restrict__ bitmask,
+             long long mask_stride, const int32_t* __restrict__ row_indices) {
+  const int r = row_indices ? row_indices[blockIdx.y] : blockIdx.y;
+  const uint32_t* mrow = bitmask + (long long)r * mask_stride;
+  const int n_vec = vocab_size / ELEMS;
+  constexpr uint32_t kAll = (1u << ELEMS) - 1;
+  const uint4 ninf = ELEMS == 8 ? make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u)
+                                : make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
+  uint4* base = ELEMS == 8 ? (uint4*)((uint16_t*)logits + (long long)r * row_stride_elems)
+                           : (uint4*)((uint32_t*)logits + (long long)r * row_stride_elems);
+  for (int vi = blockIdx.x * blockDim.x + threadIdx.x; vi < n_vec; vi += gridDim.x * blockDim.x) {
+    const int first = vi * ELEMS;
+    const uint32_t bits = (__ldg(&mrow[first >> 5]) >> (first & 31)) & kAll;
+    if (bits == kAll) continue;
+    if (bits == 0) { base[vi] = ninf; continue; }
+    uint4 x = base[vi];
+    if (ELEMS == 8) {
+      uint32_t p[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (!((bits >> (2 * k)) & 1u)) p[k] = (p[k] & 0xFFFF0000u) | 0xFF80u;
+        if (!((bits >> (2 * k + 1)) & 1u)) p[k] = (p[k] & 0x0000FFFFu) | 0xFF800000u;
+      }
+      x = make_uint4(p[0], p[1], p[2], p[3]);
+    } else {
+      if (!(bits & 1u)) x.x = 0xFF800000u;
+      if (!(bits & 2u)) x.y = 0xFF800000u;
+      if (!(bits & 4u)) x.z = 0xFF800000u;
+      if (!(bits & 8u)) x.w = 0xFF800000u;
+    }
+    base[vi] = x;
+  }
+  // ragged tail (vocab_size not a multiple of the vector width)
+  if (blockIdx.x == 0) {
+    for (int c = n_vec * ELEMS + threadIdx.x; c < vocab_size; c += blockDim.x) {
+      if ((mrow[c >> 5] >> (c & 31)) & 1u) continue;
+      if (ELEMS == 8) ((uint16_t*)logits)[(long long)r * row_stride_elems + c] = 0xFF80u;
+      else ((uint32_t*)logits)[(long long)r * row_stride_elems + c] = 0xFF800000u;
+    }
+  }
+}
+
+}  // namespace xg
