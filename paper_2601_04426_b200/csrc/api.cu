@@ -1,0 +1,627 @@
+// C ABI of the token-mask library: argument checking, device memory, launches.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <chrono>
+#include <cstring>
+#include <map>
+#include <memory>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "device_types.h"
+#include "frontend.h"
+#include "kernels.cuh"
+#include "pool.h"
+#include "xg.h"
+
+using namespace xg;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+xg_status_t set_error(xg_status_t st, const std::string& msg) {
+  g_last_error = msg;
+  return st;
+}
+
+#define XG_CUDA(expr)                                                                               \
+  do {                                                                                              \
+    cudaError_t err__ = (expr);                                                                     \
+    if (err__ != cudaSuccess)                                                                       \
+      return set_error(XG_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(err__));         \
+  } while (0)
+
+template <typename T>
+T* device_copy(const std::vector<T>& v, cudaError_t* err) {
+  T* p = nullptr;
+  size_t bytes = std::max<size_t>(v.size(), 1) * sizeof(T);
+  *err = cudaMalloc(&p, bytes);
+  if (*err != cudaSuccess) return nullptr;
+  if (!v.empty()) *err = cudaMemcpy(p, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice);
+  return p;
+}
+
+double now_ms() {
+  return std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now().time_since_epoch()).count();
+}
+
+}  // namespace
+
+// the device array of matcher pointers (and the per-request scratch words) of one batch
+struct BatchSlot {
+  std::vector<xg_matcher_t*> key;
+  MatcherDev** dev_matchers = nullptr;
+  int32_t* status = nullptr;       // [batch]
+  int32_t* done_count = nullptr;   // [batch]
+  uint64_t last_use = 0;
+};
+
+struct xg_tokenizer {
+  VocabDev dev{};
+  std::vector<void*> allocations;
+  std::vector<int32_t> rank_to_id, id_to_rank;
+  int32_t vocab_size = 0, n_words = 0;
+  mutable std::mutex mu;
+  mutable std::vector<BatchSlot> batch_slots;
+  mutable uint64_t use_counter = 0;
+};
+
+struct xg_grammar {
+  const xg_tokenizer* tok = nullptr;
+  std::shared_ptr<CachePool> pool;
+  FlatGrammar flat;
+  std::vector<EntryDev> entries;        // [n_states], host copy of the device headers
+  std::vector<int2> entry_counts;       // [n_states] (accepted, uncertain)
+  GrammarDev host_view{};               // device pointers
+  GrammarDev* dev = nullptr;            // the same struct in device memory
+  void* blob = nullptr;
+  xg_grammar_stats_t stats{};
+  // buffers behind xg_grammar_get_cache_entry's view
+  mutable std::vector<int32_t> view_list, view_unc;
+  mutable std::vector<uint32_t> view_bits;
+};
+
+struct xg_cache_pool {
+  std::shared_ptr<CachePool> impl;
+};
+
+struct xg_matcher {
+  const xg_grammar* grammar = nullptr;
+  MatcherDev* dev = nullptr;
+  void* block = nullptr;
+};
+
+extern "C" {
+
+const char* xg_last_error(void) { return g_last_error.c_str(); }
+
+// ---------------------------------------------------------------------------------------------
+// vocabulary: sort by bytes (trie order), upload
+// ---------------------------------------------------------------------------------------------
+xg_status_t xg_tokenizer_create(const uint8_t* bytes, const int64_t* offsets, int32_t vocab_size, int32_t eos_token_id,
+                                const int32_t* special_ids, int32_t n_special, void* stream, xg_tokenizer_t** out) {
+  (void)stream;
+  if (!out) return set_error(XG_ERR_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  if (!offsets || vocab_size <= 0 || (!bytes && offsets[vocab_size] > 0)) return set_error(XG_ERR_INVALID_ARG, "bad vocabulary arrays");
+  if (eos_token_id >= vocab_size || eos_token_id < -1) return set_error(XG_ERR_INVALID_ARG, "eos_token_id out of range");
+  if (n_special < 0 || (n_special > 0 && !special_ids)) return set_error(XG_ERR_INVALID_ARG, "bad special_ids");
+  int max_len = 0;
+  for (int i = 0; i < vocab_size; ++i) {
+    int64_t len = offsets[i + 1] - offsets[i];
+    if (len < 0) return set_error(XG_ERR_INVALID_ARG, "offsets must be non-decreasing");
+    if (len > kSlowMaxBytes) return set_error(XG_ERR_UNSUPPORTED, "tokens longer than 255 bytes are not supported");
+    max_len = std::max<int>(max_len, (int)len);
+  }
+  std::vector<char> never(vocab_size, 0);
+  for (int i = 0; i < n_special; ++i) {
+    if (special_ids[i] < 0 || special_ids[i] >= vocab_size) return set_error(XG_ERR_INVALID_ARG, "special id out of range");
+    never[special_ids[i]] = 1;
+  }
+  if (eos_token_id >= 0) never[eos_token_id] = 1;
+  std::unique_ptr<xg_tokenizer> t(new xg_tokenizer());
+  t->vocab_size = vocab_size;
+  t->n_words = (vocab_size + 31) / 32;
+  std::vector<int32_t>& order = t->rank_to_id;
+  order.resize(vocab_size);
+  for (int i = 0; i < vocab_size; ++i) order[i] = i;
+  std::sort(order.begin(), order.end(), [&](int a, int b) {
+    size_t la = (size_t)(offsets[a + 1] - offsets[a]), lb = (size_t)(offsets[b + 1] - offsets[b]);
+    int c = std::min(la, lb) ? std::memcmp(bytes + offsets[a], bytes + offsets[b], std::min(la, lb)) : 0;
+    if (c != 0) return c < 0;
+    if (la != lb) return la < lb;
+    return a < b;
+  });
+  t->id_to_rank.resize(vocab_size);
+  std::vector<uint8_t> arena;
+  std::vector<uint32_t> off(vocab_size + 1, 0);
+  std::vector<uint8_t> never_rank(vocab_size, 0);
+  arena.reserve((size_t)offsets[vocab_size] + 16);
+  for (int r = 0; r < vocab_size; ++r) {
+    int id = order[r];
+    t->id_to_rank[id] = r;
+    if (offsets[id + 1] > offsets[id]) arena.insert(arena.end(), bytes + offsets[id], bytes + offsets[id + 1]);
+    off[r + 1] = (uint32_t)arena.size();
+    never_rank[r] = (never[id] || offsets[id + 1] == offsets[id]) ? 1 : 0;
+  }
+  arena.resize(arena.size() + 16, 0);
+  cudaError_t err = cudaSuccess;
+  auto keep = [&](auto* p) { if (p) t->allocations.push_back((void*)p); return p; };
+  t->dev.vocab_size = vocab_size;
+  t->dev.n_words = t->n_words;
+  t->dev.eos_id = eos_token_id;
+  t->dev.max_len = max_len;
+  t->dev.bytes = keep(device_copy(arena, &err));
+  if (err == cudaSuccess) t->dev.offset = keep(device_copy(off, &err));
+  if (err == cudaSuccess) t->dev.rank_to_id = keep(device_copy(t->rank_to_id, &err));
+  if (err == cudaSuccess) t->dev.id_to_rank = keep(device_copy(t->id_to_rank, &err));
+  if (err == cudaSuccess) t->dev.never = keep(device_copy(never_rank, &err));
+  if (err != cudaSuccess) {
+    for (void* p : t->allocations) cudaFree(p);
+    return set_error(XG_ERR_CUDA, std::string("vocabulary upload: ") + cudaGetErrorString(err));
+  }
+  *out = t.release();
+  return XG_OK;
+}
+
+void xg_tokenizer_destroy(xg_tokenizer_t* t) {
+  if (!t) return;
+  for (auto& s : t->batch_slots) { cudaFree(s.dev_matchers); cudaFree(s.status); cudaFree(s.done_count); }
+  for (void* p : t->allocations) cudaFree(p);
+  delete t;
+}
+
+xg_status_t xg_cache_pool_create(const xg_tokenizer_t* tok, xg_cache_pool_t** out) {
+  if (!tok || !out) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
+  *out = new xg_cache_pool{std::make_shared<CachePool>((const void*)tok)};
+  return XG_OK;
+}
+void xg_cache_pool_destroy(xg_cache_pool_t* pool) { delete pool; }
+
+// ---------------------------------------------------------------------------------------------
+// grammar compilation
+// ---------------------------------------------------------------------------------------------
+static xg_status_t upload_grammar(xg_grammar* g) {
+  const FlatGrammar& f = g->flat;
+  // one blob, sections 16-byte aligned
+  size_t total = 0;
+  auto reserve = [&](size_t bytes) { size_t at = total; total += (bytes + 15) & ~size_t(15); return at; };
+  std::vector<uint32_t> info(f.n_states);
+  for (int s = 0; s < f.n_states; ++s) info[s] = (uint32_t)f.state_rule[s] | (f.state_final[s] ? 0x80000000u : 0u);
+  size_t o_info = reserve(info.size() * 4), o_sb = reserve(f.scan_begin.size() * 4), o_so = reserve(f.scan_own_end.size() * 4),
+         o_sc = reserve(f.scan_class.size() * 4), o_st = reserve(f.scan_target.size() * 4), o_wb = reserve(f.wait_begin.size() * 4),
+         o_wr = reserve(f.wait_rule.size() * 4), o_wt = reserve(f.wait_target.size() * 4), o_gb = reserve(f.gather_begin.size() * 4),
+         o_gs = reserve(f.gather_state.size() * 4), o_cb = reserve(f.class_bits.size() * 4),
+         o_en = reserve((size_t)f.n_states * sizeof(EntryDev)), o_self = reserve(sizeof(GrammarDev));
+  std::vector<uint8_t> host(total, 0);
+  auto put = [&](size_t at, const void* src, size_t bytes) { if (bytes) std::memcpy(host.data() + at, src, bytes); };
+  put(o_info, info.data(), info.size() * 4);
+  put(o_sb, f.scan_begin.data(), f.scan_begin.size() * 4);
+  put(o_so, f.scan_own_end.data(), f.scan_own_end.size() * 4);
+  put(o_sc, f.scan_class.data(), f.scan_class.size() * 4);
+  put(o_st, f.scan_target.data(), f.scan_target.size() * 4);
+  put(o_wb, f.wait_begin.data(), f.wait_begin.size() * 4);
+  put(o_wr, f.wait_rule.data(), f.wait_rule.size() * 4);
+  put(o_wt, f.wait_target.data(), f.wait_target.size() * 4);
+  put(o_gb, f.gather_begin.data(), f.gather_begin.size() * 4);
+  put(o_gs, f.gather_state.data(), f.gather_state.size() * 4);
+  put(o_cb, f.class_bits.data(), f.class_bits.size() * 4);
+  put(o_en, g->entries.data(), g->entries.size() * sizeof(EntryDev));
+  if (!g->blob) XG_CUDA(cudaMalloc(&g->blob, total));
+  uint8_t* d = (uint8_t*)g->blob;
+  GrammarDev& v = g->host_view;
+  v.n_states = f.n_states; v.n_rules = f.n_rules; v.n_classes = f.n_classes;
+  v.root_rule = f.root_rule; v.root_nullable = f.root_nullable; v.root_start = f.rule_start[f.root_rule];
+  v.state_info = (const uint32_t*)(d + o_info);
+  v.scan_begin = (const int32_t*)(d + o_sb); v.scan_own_end = (const int32_t*)(d + o_so);
+  v.scan_class = (const uint32_t*)(d + o_sc); v.scan_target = (const uint32_t*)(d + o_st);
+  v.wait_begin = (const int32_t*)(d + o_wb); v.wait_rule = (const uint32_t*)(d + o_wr); v.wait_target = (const uint32_t*)(d + o_wt);
+  v.gather_begin = (const int32_t*)(d + o_gb); v.gather_state = (const int32_t*)(d + o_gs);
+  v.class_bits = (const uint32_t*)(d + o_cb);
+  v.entries = (const EntryDev*)(d + o_en);
+  put(o_self, &v, sizeof(GrammarDev));
+  g->dev = (GrammarDev*)(d + o_self);
+  XG_CUDA(cudaMemcpy(g->blob, host.data(), total, cudaMemcpyHostToDevice));
+  return XG_OK;
+}
+
+// classify + pack the given states (device work of the compile stage); fills entries / counts
+static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& states, cudaStream_t stream) {
+  if (states.empty()) return XG_OK;
+  const VocabDev& v = g->tok->dev;
+  const int W = v.n_words, V = v.vocab_size;
+  const size_t row_bytes = (size_t)W * 4;
+  const size_t budget = size_t(768) << 20;                         // scratch rows per batch
+  const int per_batch = (int)std::max<size_t>(1, std::min<size_t>(std::min<size_t>(states.size(), 65535), budget / (3 * row_bytes)));
+  int32_t* d_pos = nullptr;
+  uint32_t* d_rows = nullptr;
+  int2* d_counts = nullptr;
+  PackPlan* d_plan = nullptr;
+  long long* d_total = nullptr;
+  EntryDev* d_entries = nullptr;
+  int2* d_over = nullptr;
+  int* d_over_count = nullptr;
+  const int over_cap = 1 << 16;
+  auto cleanup = [&]() { cudaFree(d_pos); cudaFree(d_rows); cudaFree(d_counts); cudaFree(d_plan); cudaFree(d_total); cudaFree(d_entries); cudaFree(d_over); cudaFree(d_over_count); };
+#define XG_CUDA_C(expr) do { cudaError_t e__ = (expr); if (e__ != cudaSuccess) { cleanup(); return set_error(XG_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)); } } while (0)
+  XG_CUDA_C(cudaMalloc(&d_pos, per_batch * sizeof(int32_t)));
+  XG_CUDA_C(cudaMalloc(&d_rows, 3 * row_bytes * per_batch));
+  XG_CUDA_C(cudaMalloc(&d_counts, per_batch * sizeof(int2)));
+  XG_CUDA_C(cudaMalloc(&d_plan, per_batch * sizeof(PackPlan)));
+  XG_CUDA_C(cudaMalloc(&d_total, sizeof(long long)));
+  XG_CUDA_C(cudaMalloc(&d_entries, per_batch * sizeof(EntryDev)));
+  XG_CUDA_C(cudaMalloc(&d_over, over_cap * sizeof(int2)));
+  XG_CUDA_C(cudaMalloc(&d_over_count, 2 * sizeof(int)));
+  for (size_t begin = 0; begin < states.size(); begin += per_batch) {
+    const int n = (int)std::min<size_t>(per_batch, states.size() - begin);
+    uint32_t* acc = d_rows;
+    uint32_t* unc = d_rows + (size_t)per_batch * W;
+    uint32_t* unr = d_rows + 2 * (size_t)per_batch * W;
+    XG_CUDA_C(cudaMemcpyAsync(d_pos, states.data() + begin, n * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+    XG_CUDA_C(cudaMemsetAsync(d_rows, 0, 3 * row_bytes * per_batch, stream));
+    XG_CUDA_C(cudaMemsetAsync(d_over_count, 0, 2 * sizeof(int), stream));
+    dim3 grid((V + 255) / 256, n);
+    classify_kernel<<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, acc, unc, unr, d_over, d_over_count, over_cap);
+    XG_CUDA_C(cudaGetLastError());
+    int over[2] = {0, 0};
+    XG_CUDA_C(cudaMemcpyAsync(over, d_over_count, 2 * sizeof(int), cudaMemcpyDeviceToHost, stream));
+    XG_CUDA_C(cudaStreamSynchronize(stream));
+    if (over[0] > over_cap) { cleanup(); return set_error(XG_ERR_CAPACITY, "too many token walks exceeded the fast path"); }
+    for (int done = 0; done < over[0];) {          // exact fallback, a bounded number of pairs per round
+      const int round = std::min(over[0] - done, 4096);
+      uint32_t* s_st = nullptr; int32_t* s_org = nullptr; int32_t* s_lsb = nullptr;
+      cudaError_t e1 = cudaMalloc(&s_st, (size_t)round * kSlowCap * 4), e2 = cudaMalloc(&s_org, (size_t)round * kSlowCap * 4),
+                  e3 = cudaMalloc(&s_lsb, (size_t)round * (kSlowMaxBytes + 2) * 4);
+      if (e1 == cudaSuccess && e2 == cudaSuccess && e3 == cudaSuccess)
+        classify_slow_kernel<<<(round + 63) / 64, 64, 0, stream>>>(g->host_view, v, d_pos, d_over + done, round, s_st, s_org, s_lsb, acc, unc, unr, d_over_count + 1);
+      cudaError_t e4 = cudaStreamSynchronize(stream);
+      cudaFree(s_st); cudaFree(s_org); cudaFree(s_lsb);
+      if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) { cleanup(); return set_error(XG_ERR_CUDA, "slow classification failed"); }
+      done += round;
+    }
+    if (over[0] > 0) {
+      XG_CUDA_C(cudaMemcpy(over, d_over_count, 2 * sizeof(int), cudaMemcpyDeviceToHost));
+      if (over[1]) { cleanup(); return set_error(XG_ERR_CAPACITY, "an Earley item set exceeded the supported size during cache build"); }
+    }
+    count_kernel<<<n, 256, 0, stream>>>(acc, unc, W, d_counts);
+    plan_kernel<<<1, 1024, 0, stream>>>(d_counts, n, V, W, d_plan, d_total);
+    XG_CUDA_C(cudaGetLastError());
+    long long total_words = 0;
+    XG_CUDA_C(cudaMemcpyAsync(&total_words, d_total, sizeof(long long), cudaMemcpyDeviceToHost, stream));
+    XG_CUDA_C(cudaStreamSynchronize(stream));
+    uint32_t* arena = (uint32_t*)g->pool->allocate_device((size_t)std::max<long long>(total_words, 1) * 4);
+    if (!arena) { cleanup(); return set_error(XG_ERR_OOM, "cache arena allocation failed"); }
+    pack_kernel<<<n, 256, 0, stream>>>(acc, unc, unr, d_plan, V, W, arena, d_entries);
+    XG_CUDA_C(cudaGetLastError());
+    std::vector<EntryDev> built(n);
+    std::vector<int2> counts(n);
+    XG_CUDA_C(cudaMemcpyAsync(built.data(), d_entries, n * sizeof(EntryDev), cudaMemcpyDeviceToHost, stream));
+    XG_CUDA_C(cudaMemcpyAsync(counts.data(), d_counts, n * sizeof(int2), cudaMemcpyDeviceToHost, stream));
+    XG_CUDA_C(cudaStreamSynchronize(stream));
+    for (int k = 0; k < n; ++k) { g->entries[states[begin + k]] = built[k]; g->entry_counts[states[begin + k]] = counts[k]; }
+  }
+  cleanup();
+#undef XG_CUDA_C
+  return XG_OK;
+}
+
+xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool, xg_grammar_kind_t kind, const char* text, size_t len,
+                               const char* root_rule, const xg_compile_options_t* opt, void* stream, xg_grammar_t** out) {
+  if (!out) return set_error(XG_ERR_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  if (!text) return set_error(XG_ERR_INVALID_ARG, "text is NULL");
+  FrontendOptions fo;
+  bool build_cache = tok != nullptr;
+  if (opt) {
+    if (opt->struct_size < 8) return set_error(XG_ERR_INVALID_ARG, "bad options struct_size");
+    if (opt->inline_max_states >= 0) fo.inline_max_states = opt->inline_max_states;
+    if (opt->struct_size >= 12 && opt->max_rule_states > 0) fo.max_rule_states = opt->max_rule_states;
+    if (opt->struct_size >= 16 && opt->build_cache == 0) build_cache = false;
+  }
+  if (pool && pool->impl->owner() != (const void*)tok) return set_error(XG_ERR_INVALID_ARG, "the pool belongs to another tokenizer");
+  std::unique_ptr<xg_grammar> g(new xg_grammar());
+  const double t0 = now_ms();
+  try {
+    g->flat = compile_frontend((int)kind, std::string(text, len), root_rule ? root_rule : "root", fo);
+  } catch (const FrontendError& e) {
+    return set_error(e.status, e.message);
+  } catch (const std::bad_alloc&) {
+    return set_error(XG_ERR_OOM, "out of host memory in the grammar front end");
+  } catch (const std::exception& e) {
+    return set_error(XG_ERR_PARSE, e.what());
+  }
+  const FlatGrammar& f = g->flat;
+  g->stats.frontend_ms = now_ms() - t0;
+  g->stats.n_rules = f.n_rules; g->stats.n_states = f.n_states; g->stats.n_classes = f.n_classes;
+  std::vector<int32_t> scannable;
+  for (int s = 0; s < f.n_states; ++s) if (f.cedge_begin[s + 1] > f.cedge_begin[s]) scannable.push_back(s);
+  g->stats.n_scannable = (int)scannable.size();
+  if (!build_cache) { *out = g.release(); return XG_OK; }
+
+  g->tok = tok;
+  g->pool = pool ? pool->impl : std::make_shared<CachePool>((const void*)tok);
+  g->entries.assign(f.n_states, EntryDev{});
+  g->entry_counts.assign(f.n_states, make_int2(0, 0));
+  const double t1 = now_ms();
+  xg_status_t st = upload_grammar(g.get());
+  if (st != XG_OK) { xg_grammar_destroy(g.release()); return st; }
+  // cross-grammar cache (Section 3.3): rules whose canonical structure is already in the pool
+  // reuse its entries; the others are classified now and registered afterwards
+  std::lock_guard<std::mutex> pool_lock(g->pool->mu);
+  RuleInterning in;
+  try {
+    in = g->pool->intern(f);
+  } catch (const std::exception& e) {
+    xg_grammar_destroy(g.release());
+    return set_error(XG_ERR_OOM, e.what());
+  }
+  std::vector<int> rule_first(f.n_rules + 1, f.n_states);
+  for (int s = f.n_states - 1; s >= 0; --s) rule_first[f.state_rule[s]] = s;
+  std::vector<int> canon_of(f.n_states, -1);          // state -> canonical index inside its rule
+  for (int r = 0; r < f.n_rules; ++r)
+    for (size_t k = 0; k < in.canon[r].size(); ++k) canon_of[rule_first[r] + in.canon[r][k]] = (int)k;
+  std::map<int, int> builder_of;                      // pool rule -> the rule of this grammar that builds it
+  std::vector<int32_t> to_build;
+  for (int s : scannable) {
+    const int r = f.state_rule[s];
+    PoolRule& pr = g->pool->rule(in.pool_id[r]);
+    if (pr.built) {
+      g->entries[s] = pr.entries[canon_of[s]];
+      g->entry_counts[s] = pr.counts[canon_of[s]];
+      ++g->stats.n_entries_reused;
+    } else {
+      auto it = builder_of.find(in.pool_id[r]);
+      if (it == builder_of.end()) it = builder_of.emplace(in.pool_id[r], r).first;
+      if (it->second == r) to_build.push_back(s);
+    }
+  }
+  st = build_entries(g.get(), to_build, (cudaStream_t)stream);
+  if (st != XG_OK) { xg_grammar_destroy(g.release()); return st; }
+  for (auto& kv : builder_of) {
+    PoolRule& pr = g->pool->rule(kv.first);
+    const int r = kv.second;
+    const int n_local = (int)in.canon[r].size();
+    pr.entries.resize(n_local);
+    pr.counts.resize(n_local);
+    for (int k = 0; k < n_local; ++k) { pr.entries[k] = g->entries[rule_first[r] + in.canon[r][k]]; pr.counts[k] = g->entry_counts[rule_first[r] + in.canon[r][k]]; }
+    pr.built = true;
+  }
+  for (int s : scannable) {                           // duplicates of a rule inside this grammar
+    const int r = f.state_rule[s];
+    auto it = builder_of.find(in.pool_id[r]);
+    if (it == builder_of.end() || it->second == r) continue;
+    const PoolRule& pr = g->pool->rule(in.pool_id[r]);
+    g->entries[s] = pr.entries[canon_of[s]];
+    g->entry_counts[s] = pr.counts[canon_of[s]];
+    ++g->stats.n_entries_reused;
+  }
+  st = upload_grammar(g.get());       // now with the entry headers
+  if (st != XG_OK) { xg_grammar_destroy(g.release()); return st; }
+  g->stats.cache_build_ms = now_ms() - t1;
+  g->stats.n_entries_built = (int)to_build.size();
+  g->stats.pairs_classified = (int64_t)to_build.size() * tok->vocab_size;
+  for (int s : scannable) {
+    const EntryDev& e = g->entries[s];
+    const int2 c = g->entry_counts[s];
+    g->stats.total_accepted += c.x;
+    g->stats.total_uncertain += c.y;
+    g->stats.total_rejected += tok->vocab_size - c.x - c.y;
+    g->stats.kind_count[e.kind]++;
+    g->stats.cache_bytes += 4LL * ((e.kind == 2 ? tok->n_words : e.n_list) + 2LL * e.n_unc);
+  }
+  *out = g.release();
+  return XG_OK;
+}
+
+void xg_grammar_destroy(xg_grammar_t* g) {
+  if (!g) return;
+  cudaFree(g->blob);
+  delete g;
+}
+
+xg_status_t xg_grammar_get_tables(const xg_grammar_t* g, xg_grammar_tables_t* t) {
+  if (!g || !t) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
+  const FlatGrammar& f = g->flat;
+  t->n_rules = f.n_rules; t->n_states = f.n_states; t->n_classes = f.n_classes;
+  t->n_class_edges = (int32_t)f.cedge_class.size(); t->n_ref_edges = (int32_t)f.redge_rule.size();
+  t->root_rule = f.root_rule; t->root_nullable = f.root_nullable;
+  t->rule_start = f.rule_start.data(); t->state_rule = f.state_rule.data(); t->state_final = f.state_final.data();
+  t->cedge_begin = f.cedge_begin.data(); t->cedge_class = f.cedge_class.data(); t->cedge_target = f.cedge_target.data();
+  t->redge_begin = f.redge_begin.data(); t->redge_rule = f.redge_rule.data(); t->redge_target = f.redge_target.data();
+  t->class_bits = f.class_bits.data();
+  return XG_OK;
+}
+
+xg_status_t xg_grammar_get_cache_entry(const xg_grammar_t* g, int32_t state, xg_cache_entry_view_t* view) {
+  if (!g || !view) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
+  if (!g->tok) return set_error(XG_ERR_INVALID_ARG, "the grammar was compiled without a cache");
+  const FlatGrammar& f = g->flat;
+  if (state < 0 || state >= f.n_states || f.cedge_begin[state + 1] == f.cedge_begin[state]) return set_error(XG_ERR_INVALID_ARG, "state is not scannable");
+  const EntryDev& e = g->entries[state];
+  const int2 c = g->entry_counts[state];
+  XG_CUDA(cudaDeviceSynchronize());
+  view->state = state; view->kind = e.kind;
+  view->n_accepted = c.x; view->n_uncertain = c.y; view->n_rejected = g->tok->vocab_size - c.x - c.y;
+  view->n_list = e.n_list; view->list = nullptr; view->bitset = nullptr;
+  if (e.kind == XG_STORE_BITSET) {
+    g->view_bits.resize(g->tok->n_words);
+    XG_CUDA(cudaMemcpy(g->view_bits.data(), e.data, g->view_bits.size() * 4, cudaMemcpyDeviceToHost));
+    view->bitset = g->view_bits.data();
+  } else {
+    g->view_list.resize(std::max(e.n_list, 1));
+    if (e.n_list) XG_CUDA(cudaMemcpy(g->view_list.data(), e.data, (size_t)e.n_list * 4, cudaMemcpyDeviceToHost));
+    view->list = g->view_list.data();
+  }
+  g->view_unc.resize(std::max(e.n_unc, 1));
+  if (e.n_unc) XG_CUDA(cudaMemcpy(g->view_unc.data(), e.unc_id, (size_t)e.n_unc * 4, cudaMemcpyDeviceToHost));
+  view->uncertain = g->view_unc.data();
+  return XG_OK;
+}
+
+xg_status_t xg_grammar_stats(const xg_grammar_t* g, xg_grammar_stats_t* out) {
+  if (!g || !out) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
+  *out = g->stats;
+  return XG_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// matchers
+// ---------------------------------------------------------------------------------------------
+xg_status_t xg_matcher_create(const xg_grammar_t* g, const xg_matcher_options_t* opt, void* stream, xg_matcher_t** out) {
+  if (!out) return set_error(XG_ERR_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  if (!g || !g->tok || !g->dev) return set_error(XG_ERR_INVALID_ARG, "the grammar has no compiled cache");
+  int max_sets = 16384, max_items = 0;
+  if (opt) {
+    if (opt->struct_size >= 8 && opt->max_sets > 0) max_sets = opt->max_sets;
+    if (opt->struct_size >= 12 && opt->max_items > 0) max_items = opt->max_items;
+  }
+  if (max_sets < 2) return set_error(XG_ERR_INVALID_ARG, "max_sets must be at least 2");
+  if (max_items <= 0) max_items = 4 * max_sets;
+  std::unique_ptr<xg_matcher> m(new xg_matcher());
+  m->grammar = g;
+  const size_t o_items = 256, o_org = o_items + (size_t)max_items * 4, o_sb = o_org + (size_t)max_items * 4;
+  const size_t total = o_sb + ((size_t)max_sets + 1) * 4;
+  XG_CUDA(cudaMalloc(&m->block, total));
+  uint8_t* d = (uint8_t*)m->block;
+  MatcherDev h{};
+  h.grammar = g->dev;
+  h.item_state = (uint32_t*)(d + o_items);
+  h.item_origin = (int32_t*)(d + o_org);
+  h.set_begin = (int32_t*)(d + o_sb);
+  h.cap_sets = max_sets; h.cap_items = max_items;
+  m->dev = (MatcherDev*)d;
+  cudaError_t err = cudaMemcpyAsync(m->dev, &h, sizeof h, cudaMemcpyHostToDevice, (cudaStream_t)stream);
+  if (err == cudaSuccess) { matcher_reset_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(m->dev); err = cudaGetLastError(); }
+  if (err == cudaSuccess) err = cudaStreamSynchronize((cudaStream_t)stream);     // `h` is a stack object
+  if (err != cudaSuccess) { cudaFree(m->block); return set_error(XG_ERR_CUDA, std::string("matcher init: ") + cudaGetErrorString(err)); }
+  *out = m.release();
+  return XG_OK;
+}
+
+xg_status_t xg_matcher_reset(xg_matcher_t* m, void* stream) {
+  if (!m) return set_error(XG_ERR_INVALID_ARG, "NULL matcher");
+  matcher_reset_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(m->dev);
+  XG_CUDA(cudaGetLastError());
+  return XG_OK;
+}
+
+void xg_matcher_destroy(xg_matcher_t* m) {
+  if (!m) return;
+  if (m->grammar && m->grammar->tok) {       // forget cached batches that contain this matcher
+    const xg_tokenizer* t = m->grammar->tok;
+    std::lock_guard<std::mutex> lock(t->mu);
+    for (auto& s : t->batch_slots)
+      if (std::find(s.key.begin(), s.key.end(), m) != s.key.end()) s.key.clear();
+  }
+  cudaFree(m->block);
+  delete m;
+}
+
+xg_status_t xg_matcher_is_terminated(const xg_matcher_t* m, void* stream, int32_t* out) {
+  if (!m || !out) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
+  MatcherDev h;
+  XG_CUDA(cudaMemcpyAsync(&h, m->dev, sizeof h, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+  XG_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  *out = h.terminated ? 1 : 0;
+  return XG_OK;
+}
+
+// device-side array of matcher pointers for this exact batch (built once, then reused)
+static xg_status_t batch_slot(xg_matcher_t* const* matchers, int32_t batch, const xg_tokenizer** tok_out, BatchSlot** slot_out) {
+  if (!matchers || batch <= 0) return set_error(XG_ERR_INVALID_ARG, "empty batch");
+  if (batch > 65535) return set_error(XG_ERR_INVALID_ARG, "batch larger than 65535");
+  for (int i = 0; i < batch; ++i) if (!matchers[i]) return set_error(XG_ERR_INVALID_ARG, "NULL matcher in batch");
+  const xg_tokenizer* tok = matchers[0]->grammar->tok;
+  for (int i = 1; i < batch; ++i) if (matchers[i]->grammar->tok != tok) return set_error(XG_ERR_INVALID_ARG, "matchers of one batch must share a tokenizer");
+  std::lock_guard<std::mutex> lock(tok->mu);
+  BatchSlot* hit = nullptr;
+  for (auto& s : tok->batch_slots)
+    if ((int)s.key.size() == batch && std::memcmp(s.key.data(), matchers, sizeof(void*) * batch) == 0) { hit = &s; break; }
+  if (!hit) {
+    if (tok->batch_slots.size() < 16) tok->batch_slots.emplace_back();
+    BatchSlot* victim = &tok->batch_slots[0];
+    for (auto& s : tok->batch_slots) {
+      if (s.key.empty()) { victim = &s; break; }
+      if (s.last_use < victim->last_use) victim = &s;
+    }
+    XG_CUDA(cudaDeviceSynchronize());            // the victim's arrays may still be in use
+    cudaFree(victim->dev_matchers); cudaFree(victim->status); cudaFree(victim->done_count);
+    victim->dev_matchers = nullptr; victim->status = nullptr; victim->done_count = nullptr;
+    victim->key.clear();
+    std::vector<MatcherDev*> ptrs(batch);
+    for (int i = 0; i < batch; ++i) ptrs[i] = matchers[i]->dev;
+    XG_CUDA(cudaMalloc(&victim->dev_matchers, sizeof(void*) * batch));
+    XG_CUDA(cudaMalloc(&victim->status, sizeof(int32_t) * batch));
+    XG_CUDA(cudaMalloc(&victim->done_count, sizeof(int32_t) * batch));
+    XG_CUDA(cudaMemcpy(victim->dev_matchers, ptrs.data(), sizeof(void*) * batch, cudaMemcpyHostToDevice));
+    victim->key.assign(matchers, matchers + batch);
+    hit = victim;
+  }
+  hit->last_use = ++tok->use_counter;
+  *tok_out = tok;
+  *slot_out = hit;
+  return XG_OK;
+}
+
+xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t batch, int32_t* bitmask_dev, int64_t row_stride_words,
+                                       int32_t* status_dev, void* stream) {
+  const xg_tokenizer* tok = nullptr;
+  BatchSlot* slot = nullptr;
+  xg_status_t st = batch_slot(matchers, batch, &tok, &slot);
+  if (st != XG_OK) return st;
+  if (!bitmask_dev || row_stride_words < tok->n_words) return set_error(XG_ERR_INVALID_ARG, "bad bitmask buffer");
+  const int W = tok->n_words;
+  int chunks = std::max((W + kMergeMaxChunkWords - 1) / kMergeMaxChunkWords, std::min(8, (W + 127) / 128));
+  dim3 grid_merge(chunks, batch);
+  merge_kernel<<<grid_merge, 256, 0, (cudaStream_t)stream>>>(slot->dev_matchers, tok->dev, bitmask_dev, (long long)row_stride_words,
+                                                             status_dev, slot->status, slot->done_count);
+  dim3 grid_check(8, batch);
+  check_kernel<<<grid_check, 256, 0, (cudaStream_t)stream>>>(slot->dev_matchers, tok->dev, bitmask_dev, (long long)row_stride_words,
+                                                             status_dev, slot->status, slot->done_count);
+  XG_CUDA(cudaGetLastError());
+  return XG_OK;
+}
+
+xg_status_t xg_accept_token(xg_matcher_t* const* matchers, int32_t batch, const int32_t* token_ids_dev, int32_t* status_dev, void* stream) {
+  const xg_tokenizer* tok = nullptr;
+  BatchSlot* slot = nullptr;
+  xg_status_t st = batch_slot(matchers, batch, &tok, &slot);
+  if (st != XG_OK) return st;
+  if (!token_ids_dev) return set_error(XG_ERR_INVALID_ARG, "token_ids_dev is NULL");
+  accept_kernel<<<(batch + 31) / 32, 32, 0, (cudaStream_t)stream>>>(slot->dev_matchers, batch, tok->dev, token_ids_dev, status_dev);
+  XG_CUDA(cudaGetLastError());
+  return XG_OK;
+}
+
+xg_status_t xg_apply_token_bitmask(void* logits_dev, xg_dtype_t dtype, int32_t batch, int32_t vocab_size, int64_t logits_row_stride_elems,
+                                   const int32_t* bitmask_dev, int64_t mask_row_stride_words, const int32_t* row_indices_dev,
+                                   int32_t n_rows, void* stream) {
+  if (!logits_dev || !bitmask_dev) return set_error(XG_ERR_INVALID_ARG, "NULL buffer");
+  if (dtype != XG_F32 && dtype != XG_BF16) return set_error(XG_ERR_INVALID_ARG, "unknown dtype");
+  if (vocab_size <= 0 || logits_row_stride_elems < vocab_size || mask_row_stride_words < (vocab_size + 31) / 32)
+    return set_error(XG_ERR_INVALID_ARG, "bad shape or stride");
+  const int rows = row_indices_dev ? n_rows : batch;
+  if (rows == 0 && row_indices_dev) return XG_OK;
+  if (rows <= 0 || rows > 65535) return set_error(XG_ERR_INVALID_ARG, "row count must be in 1..65535");
+  const int elt = dtype == XG_BF16 ? 2 : 4;
+  if (((uintptr_t)logits_dev & 15) || ((logits_row_stride_elems * elt) & 15))
+    return set_error(XG_ERR_INVALID_ARG, "logits rows must start on 16-byte boundaries");
+  const int elems = 16 / elt;
+  const int n_vec = vocab_size / elems;
+  int bx = std::max(1, std::min((n_vec + 256 * 4 - 1) / (256 * 4), 65535));
+  dim3 grid(bx, rows);
+  if (dtype == XG_BF16)
+    apply_kernel<8><<<grid, 256, 0, (cudaStream_t)stream>>>(logits_dev, vocab_size, (long long)logits_row_stride_elems, (const uint32_t*)bitmask_dev,
+                                                            (long long)mask_row_stride_words, row_indices_dev);
+  else
+    apply_kernel<4><<<grid, 256, 0, (cudaStream_t)stream>>>(logits_dev, vocab_size, (long long)logits_row_stride_elems, (const uint32_t*)bitmask_dev,
+                                                            (long long)mask_row_stride_words, row_indices_dev);
+  XG_CUDA(cudaGetLastError());
+  return XG_OK;
+}
+
+}  // extern "C"
