@@ -130,6 +130,12 @@ typedef struct {
 } xg_grammar_tables_t;
 xg_status_t xg_grammar_get_tables(const xg_grammar_t* g, xg_grammar_tables_t* host_view);
 
+/* Structural hash of every rule (Section 3.3: Algorithm 1 bottom-up over the reference graph,
+ * cycles refined as in Algorithm 2), the keys of the cross-grammar cache.  out: host, [n_rules].
+ * Equal structures hash equally whatever the rule names and numbering; the pool additionally
+ * compares canonical serialisations, so a collision can never share an entry. */
+xg_status_t xg_grammar_get_rule_hashes(const xg_grammar_t* g, uint64_t* out);
+
 /* One cache entry, copied to the host (valid until the next call on this grammar or its
  * destruction).  list = accepted ids (XG_STORE_ACCEPT_LIST) or rejected ids
  * (XG_STORE_REJECT_LIST), ascending; bitset = accepted bits (XG_STORE_BITSET), ceil(V/32) words;

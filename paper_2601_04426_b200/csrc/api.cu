@@ -435,6 +435,17 @@ xg_status_t xg_grammar_get_tables(const xg_grammar_t* g, xg_grammar_tables_t* t)
   return XG_OK;
 }
 
+xg_status_t xg_grammar_get_rule_hashes(const xg_grammar_t* g, uint64_t* out) {
+  if (!g || !out) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
+  try {
+    RuleInterning in = structural_hashes(g->flat);
+    for (int r = 0; r < g->flat.n_rules; ++r) out[r] = in.hash[r];
+  } catch (const std::exception& e) {
+    return set_error(XG_ERR_OOM, e.what());
+  }
+  return XG_OK;
+}
+
 xg_status_t xg_grammar_get_cache_entry(const xg_grammar_t* g, int32_t state, xg_cache_entry_view_t* view) {
   if (!g || !view) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
   if (!g->tok) return set_error(XG_ERR_INVALID_ARG, "the grammar was compiled without a cache");

@@ -776,12 +776,17 @@ struct Compiler {
     return rec;
   }
 
-  // Replace references to small non-recursive rules by a copy of their automaton.
+  // Replace references to small non-recursive rules by a copy of their automaton.  A rule that
+  // is referenced from a single place may be larger (inlining it duplicates nothing); this also
+  // folds alternatives such as the tool calls of a TagDispatch into one deterministic automaton.
   void inline_small_rules() {
     if (opt.inline_max_states <= 0) return;
+    const int single_use_max = std::max(64, opt.inline_max_states);
     int R = n_rules();
     std::vector<char> rec = recursive_rules();
-    std::vector<char> inlinable(R, 0), done(R, 0);
+    std::vector<int> uses(R, 0);
+    for (const Fsm& f : b.rules) for (auto& es : f.out) for (const Edge& e : es) if (e.kind == Edge::kRef) ++uses[e.rule];
+    std::vector<char> candidate(R, 0), done(R, 0);
     std::function<void(int)> process = [&](int r) {       // callees first
       if (done[r]) return;
       done[r] = 1;          // also guards recursion through cycles
@@ -795,23 +800,27 @@ struct Compiler {
         std::vector<Edge> keep;
         const std::vector<Edge> edges = g.out[s];     // g.out may reallocate while copies are appended
         for (const Edge& e : edges) {
-          if (e.kind == Edge::kRef && e.rule != r && inlinable[e.rule] && g.size() + b.rules[e.rule].size() <= opt.max_rule_states) {
+          bool take = e.kind == Edge::kRef && e.rule != r && candidate[e.rule] &&
+                      (b.rules[e.rule].size() <= opt.inline_max_states || uses[e.rule] == 1) &&
+                      g.size() + b.rules[e.rule].size() <= opt.max_rule_states;
+          if (take) {
             const Fsm& c = b.rules[e.rule];
             int base = g.size();
             for (int k = 0; k < c.size(); ++k) g.add();
             for (int k = 0; k < c.size(); ++k) {
-              for (Edge ce : c.out[k]) { ce.to += base; g.out[base + k].push_back(ce); }
+              for (Edge ce : c.out[k]) { if (ce.kind == Edge::kRef) ++uses[ce.rule]; ce.to += base; g.out[base + k].push_back(ce); }
               if (c.fin[k]) g.eps(base + k, e.to);
             }
             keep.push_back({Edge::kEps, -1, base + c.start, {}});
             g.has_tag_dispatch = g.has_tag_dispatch || c.has_tag_dispatch;
+            --uses[e.rule];
             changed = true;
           } else keep.push_back(e);
         }
         g.out[s] = keep;
       }
       if (changed) b.rules[r] = normalize(g, opt.max_rule_states);
-      inlinable[r] = !rec[r] && r != root && b.rules[r].size() <= opt.inline_max_states;
+      candidate[r] = !rec[r] && r != root && b.rules[r].size() <= single_use_max;
     };
     for (int r = 0; r < R; ++r) process(r);
   }

@@ -1,0 +1,242 @@
+"""Host logic of the library (no GPU): the grammar front end's tables, checked against the oracle.
+
+The oracle reads the grammar text with its own parser and runs a textbook Earley recogniser; the
+library lowers the same text to per-rule automata.  The oracle's table interpreter runs those
+tables, so language and mask equality here means the two front ends agree.
+"""
+import ctypes
+import json
+import os
+
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from oracle import schema_ebnf as SE
+from paper_2601_04426_b200 import binding as B
+from paper_2601_04426_b200 import inputs
+from test_oracle_earley import CFG_CASES, REGEX_CASES, all_strings
+
+
+def tables_of(kind, text, **kw):
+    g = B.Grammar(None, kind, text, **kw)
+    t = g.tables()
+    scal = {k: t.pop(k) for k in ("n_rules", "n_states", "n_classes", "root_rule", "root_nullable")}
+    return O.Tables(scal["n_rules"], scal["n_states"], scal["n_classes"], scal["root_rule"], scal["root_nullable"], **t), g
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(B.lib_path()) if os.path.exists(B.lib_path()) else B.lib()
+    header = open(os.path.join(os.path.dirname(B.lib_path()), "..", "include", "xg.h")).read()
+    import re
+    declared = set(re.findall(r"\b(xg_[a-z_]+)\s*\(", header)) - {"xg_status_t"}
+    assert declared == set(B.EXPORTS), declared ^ set(B.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def _same_language(ebnf, alphabet, max_len, **kw):
+    og = O.Grammar(ebnf)
+    tb, _ = tables_of("ebnf", ebnf, **kw)
+    for s in all_strings(alphabet, max_len):
+        data = s.encode()
+        tm = O.TableMatcher(tb)
+        ok = tm.accept_bytes(data)
+        assert ok == O.is_prefix(og, data), (ebnf, s)
+        if ok:
+            assert tm.can_terminate() == O.accepts(og, data), (ebnf, s)
+
+
+@pytest.mark.parametrize("inline", [0, 12])
+def test_tables_same_language_as_oracle_on_small_grammars(inline):
+    for name, ebnf, _, alphabet, _ in CFG_CASES:
+        _same_language(ebnf, alphabet, 6, inline_max_states=inline)
+    for ebnf, _, alphabet in REGEX_CASES:
+        _same_language(ebnf, alphabet, 6, inline_max_states=inline)
+    _same_language('root ::= TagDispatch(("ab", g), stop_strs=("xb")) "!"\ng ::= "a"', "abx!", 6, inline_max_states=inline)
+    _same_language('root ::= TagDispatch(("ab", g))\ng ::= "x" "x"?', "abx", 7, inline_max_states=inline)
+    _same_language('root ::= "q"? TagDispatch(("<a>", r0), ("<<b", r1)) \nr0 ::= "0"\nr1 ::= "1" root?', "<>ab01q", 5, inline_max_states=inline)
+
+
+def test_tables_invariants():
+    for name in ("C1", "C3", "C4", "C5"):
+        w = inputs.make_workload(name, batch=1, steps=2)
+        g = B.Grammar(None, w.grammars[0].kind, w.grammars[0].text)
+        t = g.tables()
+        S, R = t["n_states"], t["n_rules"]
+        assert len(t["state_rule"]) == S and len(t["rule_start"]) == R
+        assert all(t["state_rule"][t["rule_start"][r]] == r for r in range(R))
+        # no rule accepts the empty string; every rule has an accepting state
+        assert not any(t["state_final"][t["rule_start"][r]] for r in range(R))
+        for r in range(R):
+            assert t["state_final"][t["state_rule"] == r].any()
+        # deterministic: byte classes leaving one state are pairwise disjoint, references distinct
+        bits = t["class_bits"].reshape(-1, 8)
+        for s in range(S):
+            acc = np.zeros(8, dtype=np.uint32)
+            for e in range(t["cedge_begin"][s], t["cedge_begin"][s + 1]):
+                c = bits[t["cedge_class"][e]]
+                assert c.any() and not (acc & c).any()
+                acc |= c
+            refs = t["redge_rule"][t["redge_begin"][s]:t["redge_begin"][s + 1]]
+            assert len(set(refs.tolist())) == len(refs)
+        assert (t["cedge_target"] < S).all() and (t["redge_target"] < S).all() and (t["redge_rule"] < R).all()
+
+
+def _mutate(rng, doc, alphabet):
+    pos = rng.below(len(doc))
+    b = bytes([alphabet[rng.below(len(alphabet))]])
+    kind = rng.below(3)
+    return doc[:pos] + b + doc[pos + 1:] if kind == 0 else (doc[:pos] + doc[pos + 1:] if kind == 1 else doc[:pos] + b + doc[pos:])
+
+
+@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4", "C5"])
+def test_workload_grammars_same_language_as_oracle(name):
+    w = inputs.make_workload(name, batch=3, steps=40)
+    rng = inputs.Rng(17)
+    alphabet = b'{}[]:,"\\ -.0123456789etrufalsn<>/_\xc3\xa9'
+    for gi in sorted(set(w.request_grammar)):
+        spec = w.grammars[gi]
+        og = O.Grammar(SE.grammar_text(spec.kind, spec.text))
+        tb, _ = tables_of(spec.kind, spec.text)
+        for b in [i for i, x in enumerate(w.request_grammar) if x == gi]:
+            for doc in w.documents[b][:2]:
+                tm = O.TableMatcher(tb)
+                assert tm.accept_bytes(doc), doc
+                if name != "C4" or True:
+                    assert tm.can_terminate() == O.accepts(og, doc)
+                for _ in range(25):
+                    mut = _mutate(rng, doc, alphabet)
+                    tm = O.TableMatcher(tb)
+                    ok = tm.accept_bytes(mut)
+                    assert ok == O.is_prefix(og, mut), mut
+                    if ok:
+                        assert tm.can_terminate() == O.accepts(og, mut), mut
+
+
+@pytest.mark.parametrize("name,vsize,steps", [("C1", 2048, 40), ("C4", 2048, 60), ("C5", 4096, 30)])
+def test_masks_plain_equals_merged_equals_oracle(name, vsize, steps):
+    """The cache classification plus the merge rule reproduces the plain definition, step by step."""
+    w = inputs.make_workload(name, batch=1, steps=steps, vocab_size=vsize)
+    spec = w.grammars[0]
+    ov = O.Vocab(w.vocab.tokens, w.vocab.eos_id, w.vocab.special_ids)
+    og = O.Grammar(SE.grammar_text(spec.kind, spec.text))
+    tb, _ = tables_of(spec.kind, spec.text)
+    om, tm = O.Matcher(og), O.TableMatcher(tb)
+    checked_total = 0
+    for step, tok in enumerate(w.trajectories[0]):
+        ref = om.mask(ov)
+        assert np.array_equal(tm.mask_plain(ov), ref), step
+        merged, n_checked = tm.mask_merged(ov)
+        assert np.array_equal(merged, ref), step
+        checked_total += n_checked
+        if tok == w.vocab.eos_id:
+            assert om.accept_token(ov, tok) == 2
+            om.reset(); tm.reset()
+        else:
+            assert om.accept_token(ov, tok) == 1
+            assert tm.accept_bytes(w.vocab.tokens[tok])
+    assert checked_total < steps * vsize          # the cache decides most tokens
+
+
+def test_classification_partition_and_soundness():
+    """Accepted / uncertain / rejected partition the vocabulary; accepted tokens are allowed in
+    every state that contains the position, rejected ones are allowed only through other items."""
+    w = inputs.make_workload("C5", batch=1, steps=25, vocab_size=2048)
+    ov = O.Vocab(w.vocab.tokens, w.vocab.eos_id, w.vocab.special_ids)
+    tb, _ = tables_of("ebnf", w.grammars[0].text)
+    tm = O.TableMatcher(tb)
+    cls_cache = {}
+    for tok in w.trajectories[0]:
+        if tok == w.vocab.eos_id:
+            tm.reset()
+            continue
+        bits = O.unpack_bits(tm.mask_plain(ov), ov.size)
+        states = sorted({s for s, _ in tm.get_set(tm.num_sets() - 1) if s in set(tb.scannable_states())})
+        union_acc = np.zeros(ov.size, bool)
+        union_unc = np.zeros(ov.size, bool)
+        for s in states:
+            if s not in cls_cache:
+                cls_cache[s] = tb.classify(ov, s)
+            c = cls_cache[s]
+            assert set(np.unique(c)) <= {0, 1, 2}
+            assert not bits[(c == 1) & ~bits].any() and bits[c == 1].all()
+            union_acc |= c == 1
+            union_unc |= c == 2
+        assert not (bits & ~union_acc & ~union_unc)[:ov.size].any()      # allowed => accepted or uncertain somewhere
+        tm.accept_bytes(w.vocab.tokens[tok])
+
+
+def test_front_end_errors():
+    cases = [("ebnf", 'root ::= "a', B.XG_ERR_PARSE), ("ebnf", "root ::= missing", B.XG_ERR_PARSE), ("ebnf", 'x ::= "a"', B.XG_ERR_PARSE),
+             ("ebnf", 'root ::= "a"{3,2}', B.XG_ERR_PARSE), ("json_schema", "{", B.XG_ERR_PARSE),
+             ("json_schema", json.dumps({"type": "string", "pattern": "a"}), B.XG_ERR_UNSUPPORTED),
+             ("json_schema", json.dumps({"type": "object", "properties": {"a": {"type": "null"}}, "required": []}), B.XG_ERR_UNSUPPORTED),
+             ("tag_dispatch", json.dumps({"tags": []}), B.XG_ERR_PARSE)]
+    for kind, text, status in cases:
+        with pytest.raises(B.XgError) as e:
+            B.Grammar(None, kind, text)
+        assert e.value.status == status, (text, e.value)
+        assert str(e.value)
+
+
+def test_schema_lowerings_agree():
+    """The library's schema -> grammar text and the oracle's, each read by the oracle's parser,
+    accept the same documents (the texts themselves differ)."""
+    rng = inputs.Rng(3)
+    for _ in range(6):
+        schema = inputs.make_object_schema(rng, rng.randint(2, 6), 2)
+        text = json.dumps(schema)
+        ga = O.Grammar(SE.schema_to_ebnf(text))
+        tb, _ = tables_of("json_schema", text)
+        for _ in range(5):
+            doc = inputs.sample_document(schema, rng, wide=True).encode()
+            assert O.accepts(ga, doc)
+            tm = O.TableMatcher(tb)
+            assert tm.accept_bytes(doc) and tm.can_terminate()
+
+
+# ---------------------------------------------------------------------------------------
+# structural hash (Section 3.3, Algorithms 1 and 2)
+# ---------------------------------------------------------------------------------------
+
+def _hashes(ebnf, root="root"):
+    g = B.Grammar(None, "ebnf", ebnf, root=root, inline_max_states=0)
+    return g.rule_hashes()
+
+
+def test_structural_hash_ignores_names_and_order():
+    a = _hashes('root ::= "x" item "y" | "z"\nitem ::= [0-9]+ "." [a-f]')
+    b = _hashes('digits ::= [0-9]+ "." [a-f]\nroot ::= "z" | "x" digits "y"')
+    assert a[0] == b[0] and a[1] == b[1]
+    # the same sub-rule inside a different grammar keeps its hash (cross-grammar reuse)
+    c = _hashes('root ::= "{" item "}" item\nitem ::= [0-9]+ "." [a-f]')
+    assert c[1] == a[1] and c[0] != a[0]
+
+
+def test_structural_hash_sees_single_edits():
+    base = 'root ::= "x" item "y"\nitem ::= [0-9]+ "." [a-f]'
+    h0 = _hashes(base)
+    for edit in ['root ::= "x" item "z"\nitem ::= [0-9]+ "." [a-f]',
+                 'root ::= "x" item "y"\nitem ::= [0-8]+ "." [a-f]',
+                 'root ::= "x" item "y"\nitem ::= [0-9]+ "." [a-f]?',
+                 'root ::= "x" item "y"\nitem ::= [0-9]* "." [a-f]']:
+        h = _hashes(edit)
+        assert h[0] != h0[0]
+    # an edit inside the referenced rule changes both hashes; an edit in the user only the user's
+    h = _hashes('root ::= "x" item "q"\nitem ::= [0-9]+ "." [a-f]')
+    assert h[1] == h0[1] and h[0] != h0[0]
+
+
+def test_structural_hash_on_cycles():
+    """Members of a reference cycle get distinct hashes, stable under renaming and under which
+    member is the root (Algorithm 2: the fold starts at the member being hashed)."""
+    ring = 'a ::= "1" b | "x"\nb ::= "2" c | "y"\nc ::= "3" a | "z"'
+    ha = _hashes(ring, root="a")
+    assert len(set(ha.tolist())) == 3
+    hb = _hashes(ring, root="b")
+    assert set(ha.tolist()) == set(hb.tolist())
+    renamed = 'p ::= "1" q | "x"\nq ::= "2" r | "y"\nr ::= "3" p | "z"'
+    assert set(_hashes(renamed, root="p").tolist()) == set(ha.tolist())
+    other = 'a ::= "1" b | "x"\nb ::= "2" c | "y"\nc ::= "4" a | "z"'
+    assert not set(_hashes(other, root="a").tolist()) & set(ha.tolist())
