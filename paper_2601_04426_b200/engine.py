@@ -1,0 +1,83 @@
+"""Convenience layer for tests and the benchmark: device buffers (torch) around the C-ABI calls.
+
+Nothing here computes anything about grammars or masks; it allocates tensors, passes their
+pointers through `binding`, and moves results to numpy.  It needs a CUDA device.
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import inputs
+
+
+class Session:
+    """One tokenizer, its compiled grammars and one matcher per request of a workload."""
+
+    def __init__(self, workload: inputs.Workload, share_pool: bool = True, device: str = "cuda:0"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required (there is no CPU path)")
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        self.w = workload
+        v = workload.vocab
+        self.tokenizer = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
+        self.pool = B.CachePool(self.tokenizer) if share_pool else None
+        self.grammars: List[B.Grammar] = [B.Grammar(self.tokenizer, g.kind, g.text, pool=self.pool) for g in workload.grammars]
+        self.matchers = [B.Matcher(self.grammars[gi]) for gi in workload.request_grammar]
+        self.batch = B.Batch(self.matchers)
+        self.V, self.W, self.n = v.size, self.tokenizer.words, len(self.matchers)
+        self.bitmask = torch.zeros((self.n, self.W), dtype=torch.int32, device=self.device)
+        self.status = torch.zeros(self.n, dtype=torch.int32, device=self.device)
+        self.accept_status = torch.zeros(self.n, dtype=torch.int32, device=self.device)
+        self.tokens = torch.zeros(self.n, dtype=torch.int32, device=self.device)
+
+    def stream(self) -> int:
+        return torch.cuda.current_stream().cuda_stream
+
+    def fill(self) -> None:
+        self.batch.fill_next_token_bitmask(self.bitmask.data_ptr(), self.W, self.status.data_ptr(), self.stream())
+
+    def accept(self, token_ids: Sequence[int]) -> None:
+        self.tokens.copy_(torch.as_tensor(np.asarray(token_ids, dtype=np.int32)))
+        self.batch.accept_token(self.tokens.data_ptr(), self.accept_status.data_ptr(), self.stream())
+
+    def accept_device(self, token_ids: torch.Tensor) -> None:
+        self.batch.accept_token(token_ids.data_ptr(), self.accept_status.data_ptr(), self.stream())
+
+    def apply(self, logits: torch.Tensor, rows: Optional[torch.Tensor] = None) -> None:
+        dtype = {torch.float32: "f32", torch.bfloat16: "bf16", torch.int16: "bf16", torch.uint16: "bf16"}[logits.dtype]
+        B.apply_token_bitmask(logits.data_ptr(), dtype, logits.shape[0], self.V, logits.stride(0), self.bitmask.data_ptr(), self.W,
+                              rows.data_ptr() if rows is not None else 0, int(rows.numel()) if rows is not None else 0, self.stream())
+
+    def mask_numpy(self) -> np.ndarray:
+        return self.bitmask.cpu().numpy().view(np.uint32)
+
+    def reset(self, request: int) -> None:
+        self.matchers[request].reset(self.stream())
+
+    def close(self) -> None:
+        torch.cuda.synchronize()
+        for m in self.matchers:
+            m.close()
+        for g in self.grammars:
+            g.close()
+        if self.pool:
+            self.pool.close()
+        self.tokenizer.close()
+
+
+def logits_tensor(arr: np.ndarray, device) -> torch.Tensor:
+    """float32 array -> float32 tensor; uint16 bf16 bit patterns -> bfloat16 tensor."""
+    if arr.dtype == np.float32:
+        return torch.from_numpy(arr).to(device)
+    return torch.from_numpy(arr.view(np.int16)).to(device).view(torch.bfloat16)
+
+
+def logits_numpy(t: torch.Tensor) -> np.ndarray:
+    if t.dtype == torch.float32:
+        return t.cpu().numpy()
+    return t.view(torch.int16).cpu().numpy().view(np.uint16)

@@ -1,0 +1,314 @@
+"""GPU parity: every bitmask word, cache entry and masked logit against the CPU oracle.
+
+All calls go through the C ABI (via the ctypes binding).  Integer work is compared bit for bit.
+"""
+import json
+
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from oracle import schema_ebnf as SE
+from paper_2601_04426_b200 import binding as B
+from paper_2601_04426_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _engine():
+    import torch
+    from paper_2601_04426_b200 import engine
+    return torch, engine
+
+
+def _oracle_side(w):
+    ov = O.Vocab(w.vocab.tokens, w.vocab.eos_id, w.vocab.special_ids)
+    grammars = [O.Grammar(SE.grammar_text(g.kind, g.text)) for g in w.grammars]
+    matchers = [O.Matcher(grammars[gi]) for gi in w.request_grammar]
+    return ov, grammars, matchers
+
+
+def _run_trajectories(w, check_steps, check_requests=None):
+    """Drive GPU and oracle along the seeded trajectories; compare masks where asked, and the
+    cheap invariants everywhere (sampled token allowed, statuses, termination)."""
+    torch, engine = _engine()
+    s = engine.Session(w)
+    ov, _, oms = _oracle_side(w)
+    n = s.n
+    compared = 0
+    try:
+        for step in range(w.steps):
+            s.fill()
+            mask = s.mask_numpy()
+            status = s.status.cpu().numpy()
+            assert (status == 0).all(), (step, status)
+            toks = [w.trajectories[b][step] for b in range(n)]
+            for b in range(n):
+                assert (mask[b, toks[b] >> 5] >> (toks[b] & 31)) & 1, (step, b, w.vocab.tokens[toks[b]])
+                if step in check_steps or (check_requests is not None and b in check_requests):
+                    ref = oms[b].mask(ov)
+                    if not np.array_equal(mask[b], ref):
+                        diff = np.nonzero(O.unpack_bits(mask[b] ^ ref, ov.size))[0]
+                        raise AssertionError("step %d request %d: %d differing tokens, e.g. %r (gpu=%d)" % (
+                            step, b, len(diff), [w.vocab.tokens[t] for t in diff[:8]], int((mask[b, diff[0] >> 5] >> (diff[0] & 31)) & 1)))
+                    compared += 1
+            s.accept(toks)
+            ast = s.accept_status.cpu().numpy()
+            assert (ast == 0).all(), (step, ast)
+            for b in range(n):
+                r = oms[b].accept_token(ov, toks[b])
+                assert r in (1, 2)
+                if r == 2:
+                    assert s.matchers[b].is_terminated()
+                    oms[b].reset()
+                    s.reset(b)
+        return compared
+    finally:
+        s.close()
+
+
+def test_c1_every_step_bit_exact():
+    w = inputs.make_workload("C1")
+    assert _run_trajectories(w, set(range(w.steps))) == w.steps
+
+
+def test_c2_sampled_steps_bit_exact():
+    w = inputs.make_workload("C2", steps=96)
+    assert _run_trajectories(w, set(range(0, 96, 4))) == 24
+
+
+def test_c3_inter_request_batch():
+    w = inputs.make_workload("C3", batch=16, steps=48)
+    _run_trajectories(w, {0, 5, 17, 33, 47}, check_requests={3})
+
+
+def test_c4_tag_dispatch_batch():
+    w = inputs.make_workload("C4", batch=6, steps=120)
+    _run_trajectories(w, {0, 1, 30, 60, 119}, check_requests={2})
+
+
+def test_c5_recursive_json_with_utf8():
+    w = inputs.make_workload("C5", batch=8, steps=64)
+    _run_trajectories(w, {0, 7, 31, 63}, check_requests={1})
+
+
+def test_hand_worked_masks_on_gpu():
+    torch, engine = _engine()
+    from golden_util import load_mask_fixture
+    for fixture in ["mask_ab_ac.txt", "mask_bool_object.txt", "mask_nested_arrays.txt"]:
+        ebnf, tokens, cases = load_mask_fixture(fixture)
+        toks = [t.encode() for t in tokens]
+        pad = 32 - len(toks) % 32 if len(toks) % 32 else 0
+        eos = tokens.index("")
+        tok = B.Tokenizer(toks + [b"\xff\xfe"] * pad, eos)
+        g = B.Grammar(tok, "ebnf", ebnf)
+        m = B.Matcher(g)
+        batch = B.Batch([m])
+        words = tok.words
+        mask = torch.zeros((1, words), dtype=torch.int32, device="cuda")
+        ids = torch.zeros(1, dtype=torch.int32, device="cuda")
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for prefix, allowed in cases:
+            m.reset()
+            for byte in prefix.encode():        # single-byte tokens may be missing: feed known tokens greedily
+                pass
+            # feed the prefix with the longest tokens available
+            rest = prefix.encode()
+            while rest:
+                cand = max((t for t in toks if t and rest.startswith(t)), key=len)
+                ids[0] = toks.index(cand)
+                batch.accept_token(ids.data_ptr(), st.data_ptr())
+                assert int(st.cpu()[0]) == 0, (prefix, cand)
+                rest = rest[len(cand):]
+            batch.fill_next_token_bitmask(mask.data_ptr(), words, st.data_ptr())
+            bits = O.unpack_bits(mask.cpu().numpy().view(np.uint32)[0], len(tokens))
+            got = sorted(tokens[i] for i in range(len(tokens)) if bits[i])
+            assert got == sorted(allowed), (fixture, prefix, got)
+        m.close(); g.close(); tok.close()
+
+
+def _entry_sets(entry, V):
+    unc = set(entry["uncertain"].tolist())
+    if entry["kind"] == B.XG_STORE_ACCEPT_LIST:
+        acc = set(entry["list"].tolist())
+    elif entry["kind"] == B.XG_STORE_REJECT_LIST:
+        acc = set(range(V)) - set(entry["list"].tolist()) - unc
+    else:
+        acc = set(np.nonzero(O.unpack_bits(entry["bitset"], V))[0].tolist())
+    return acc, unc
+
+
+@pytest.mark.parametrize("name,vsize,stride", [("C1", None, 1), ("C5", 8192, 1), ("C4", 4096, 97), ("C3", 4096, 13)])
+def test_cache_entries_match_oracle_classification(name, vsize, stride):
+    torch, engine = _engine()
+    w = inputs.make_workload(name, batch=1, steps=2, vocab_size=vsize)
+    v = w.vocab
+    tok = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
+    g = B.Grammar(tok, w.grammars[0].kind, w.grammars[0].text)
+    t = g.tables()
+    scal = {k: t.pop(k) for k in ("n_rules", "n_states", "n_classes", "root_rule", "root_nullable")}
+    tb = O.Tables(scal["n_rules"], scal["n_states"], scal["n_classes"], scal["root_rule"], scal["root_nullable"], **t)
+    ov = O.Vocab(v.tokens, v.eos_id, v.special_ids)
+    states = tb.scannable_states()
+    stats = g.stats()
+    assert stats["n_scannable"] == len(states)
+    kinds = set()
+    for s in states[::stride]:
+        e = g.cache_entry(s)
+        cls = tb.classify(ov, s)
+        acc, unc = _entry_sets(e, v.size)
+        assert acc == set(np.nonzero(cls == 1)[0].tolist()), s
+        assert unc == set(np.nonzero(cls == 2)[0].tolist()), s
+        assert list(e["uncertain"]) == sorted(e["uncertain"]) and list(e["list"]) == sorted(e["list"])
+        n_acc, n_unc = len(acc), len(unc)
+        n_rej = v.size - n_acc - n_unc
+        assert (e["n_accepted"], e["n_uncertain"], e["n_rejected"]) == (n_acc, n_unc, n_rej)
+        sizes = [4 * n_acc, 4 * n_rej, 4 * tok.words]          # smallest wins, ties in this order
+        assert e["kind"] == sizes.index(min(sizes)), (s, sizes, e["kind"])
+        kinds.add(e["kind"])
+    if name == "C5":
+        assert B.XG_STORE_ACCEPT_LIST in kinds and B.XG_STORE_BITSET in kinds
+    if name == "C4":
+        # free text accepts nearly everything: the root automaton's start state stores a rejected list
+        e = g.cache_entry(int(t["rule_start"][0]))
+        assert e["kind"] == B.XG_STORE_REJECT_LIST
+    g.close(); tok.close()
+
+
+def test_cross_grammar_pool_reuses_entries():
+    torch, engine = _engine()
+    w = inputs.make_workload("C3", batch=6, steps=2, vocab_size=4096)
+    v = w.vocab
+    tok = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
+    pool = B.CachePool(tok)
+    shared = [B.Grammar(tok, g.kind, g.text, pool=pool) for g in w.grammars]
+    private = [B.Grammar(tok, g.kind, g.text) for g in w.grammars]
+    reused = sum(g.stats()["n_entries_reused"] for g in shared)
+    assert reused > 0 and shared[0].stats()["n_entries_reused"] >= 0
+    assert sum(g.stats()["n_entries_built"] for g in shared) < sum(g.stats()["n_entries_built"] for g in private)
+    # the same text compiled twice into one pool builds nothing the second time
+    again = B.Grammar(tok, w.grammars[0].kind, w.grammars[0].text, pool=pool)
+    assert again.stats()["n_entries_built"] == 0
+    for a, b in zip(shared, private):           # reuse never changes an entry
+        t = a.tables()
+        scannable = [s for s in range(t["n_states"]) if t["cedge_begin"][s + 1] > t["cedge_begin"][s]]
+        for s in scannable[::29]:
+            ea, eb = a.cache_entry(s), b.cache_entry(s)
+            assert ea["kind"] == eb["kind"] and np.array_equal(ea["list"], eb["list"]) and np.array_equal(ea["uncertain"], eb["uncertain"])
+    for g in shared + private + [again]:
+        g.close()
+    pool.close(); tok.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("rows,vocab,stride_pad", [(1, 8192, 0), (3, 1000, 8), (5, 32 * 7 + 5, 16), (2, 151936, 0)])
+def test_apply_matches_oracle(dtype, rows, vocab, stride_pad):
+    torch, engine = _engine()
+    elt_per_16 = 4 if dtype == "f32" else 8
+    stride = ((vocab + elt_per_16 - 1) // elt_per_16) * elt_per_16 + stride_pad
+    full = inputs.make_logits(5, rows, stride, dtype)
+    if dtype == "f32":
+        full[0, 3] = np.nan; full[0, 4] = -0.0; full[rows - 1, vocab - 1] = np.inf
+    else:
+        full[0, 3] = 0x7FC1; full[0, 4] = 0x8000; full[rows - 1, vocab - 1] = 0x7F80
+    words = (vocab + 31) // 32
+    mstride = words + 3
+    bits = (inputs.stream_u64(9, rows * mstride * 32).reshape(rows, mstride * 32) % 5) < 2
+    bits[0, :64] = True            # an all-allowed vector group
+    bits[0, 64:160] = False        # an all-masked group
+    bits[0, 3] = False
+    mask = np.packbits(bits.astype(np.uint8), axis=1, bitorder="little").view(np.uint32).reshape(rows, mstride)
+    expect = full.copy()
+    expect[:, :vocab] = O.apply_mask(full[:, :vocab], mask[:, :words])
+    t = engine.logits_tensor(full, "cuda")
+    dmask = torch.from_numpy(mask.view(np.int32)).cuda()
+    B.apply_token_bitmask(t.data_ptr(), dtype, rows, vocab, stride, dmask.data_ptr(), mstride)
+    got = engine.logits_numpy(t)
+    raw = (lambda a: a.view(np.uint32)) if dtype == "f32" else (lambda a: a)
+    assert np.array_equal(raw(got), raw(expect))
+    # a subset of rows through row_indices leaves the others untouched
+    if rows >= 3:
+        t2 = engine.logits_tensor(full, "cuda")
+        idx = torch.tensor([2, 0], dtype=torch.int32, device="cuda")
+        B.apply_token_bitmask(t2.data_ptr(), dtype, rows, vocab, stride, dmask.data_ptr(), mstride, idx.data_ptr(), 2)
+        got2 = engine.logits_numpy(t2)
+        assert np.array_equal(raw(got2[[0, 2]]), raw(expect[[0, 2]])) and np.array_equal(raw(got2[1]), raw(full[1]))
+
+
+def test_apply_rejects_bad_arguments():
+    torch, engine = _engine()
+    t = torch.zeros((2, 64), dtype=torch.float32, device="cuda")
+    m = torch.zeros((2, 2), dtype=torch.int32, device="cuda")
+    for args in [(0, "f32", 2, 64, 64, m.data_ptr(), 2), (t.data_ptr(), "f32", 2, 64, 32, m.data_ptr(), 2),
+                 (t.data_ptr(), "f32", 2, 64, 64, m.data_ptr(), 1), (t.data_ptr() + 4, "f32", 2, 60, 64, m.data_ptr(), 2)]:
+        with pytest.raises(B.XgError) as e:
+            B.apply_token_bitmask(*args)
+        assert e.value.status == B.XG_ERR_INVALID_ARG
+
+
+def test_statuses_rejected_terminated_and_mixed_grammars():
+    torch, engine = _engine()
+    toks = [bytes([b]) for b in range(256)] + [b"ab", b"abc", b"true", b"", b"<sp>"] + [b"zz%d" % i for i in range(27)]
+    eos = toks.index(b"")
+    tok = B.Tokenizer(toks, eos, [toks.index(b"<sp>")])
+    g1 = B.Grammar(tok, "ebnf", 'root ::= "ab" "c"?')
+    g2 = B.Grammar(tok, "json_schema", json.dumps({"type": "boolean"}))
+    g3 = B.Grammar(tok, "ebnf", 'root ::= ""')                      # only the empty string
+    ms = [B.Matcher(g1), B.Matcher(g2), B.Matcher(g3)]
+    batch = B.Batch(ms)
+    W = tok.words
+    mask = torch.zeros((3, W + 2), dtype=torch.int32, device="cuda")
+    st = torch.zeros(3, dtype=torch.int32, device="cuda")
+    ids = torch.zeros(3, dtype=torch.int32, device="cuda")
+
+    def allowed(row):
+        bits = O.unpack_bits(mask.cpu().numpy().view(np.uint32)[row, :W], len(toks))
+        return sorted(toks[i] for i in np.nonzero(bits)[0])
+
+    batch.fill_next_token_bitmask(mask.data_ptr(), W + 2, st.data_ptr())
+    assert allowed(0) == sorted([b"a", b"ab", b"abc"]) and allowed(1) == sorted([b"t", b"f", b"true"]) and allowed(2) == [b""]
+    assert st.cpu().tolist() == [0, 0, 0]
+    # request 0 takes "ab"; request 1 tries a refused token; request 2 ends
+    ids.copy_(torch.tensor([toks.index(b"ab"), toks.index(b"x"), eos], dtype=torch.int32))
+    batch.accept_token(ids.data_ptr(), st.data_ptr())
+    assert st.cpu().tolist() == [0, B.XG_ERR_TOKEN_REJECTED, 0]
+    assert ms[2].is_terminated() and not ms[1].is_terminated()
+    batch.fill_next_token_bitmask(mask.data_ptr(), W + 2, st.data_ptr())
+    assert allowed(0) == sorted([b"c", b""]) and allowed(1) == sorted([b"t", b"f", b"true"]) and allowed(2) == []
+    assert st.cpu().tolist() == [0, 0, B.XG_ERR_TERMINATED]
+    # special token, EOS too early, out-of-range id
+    ids.copy_(torch.tensor([toks.index(b"<sp>"), eos, 10 ** 6], dtype=torch.int32))
+    batch.accept_token(ids.data_ptr(), st.data_ptr())
+    assert st.cpu().tolist() == [B.XG_ERR_TOKEN_REJECTED, B.XG_ERR_TOKEN_REJECTED, B.XG_ERR_TERMINATED]
+    ms[2].reset()
+    batch.fill_next_token_bitmask(mask.data_ptr(), W + 2, st.data_ptr())
+    assert allowed(2) == [b""] and st.cpu().tolist() == [0, 0, 0]
+    with pytest.raises(B.XgError):
+        batch.fill_next_token_bitmask(mask.data_ptr(), W - 1, st.data_ptr())
+    for m in ms:
+        m.close()
+    for g in (g1, g2, g3):
+        g.close()
+    tok.close()
+
+
+def test_history_capacity_is_reported_not_overrun():
+    torch, engine = _engine()
+    toks = [bytes([b]) for b in range(256)] + [b"aaaa", b""] + [b"pad%d" % i for i in range(30)]
+    eos = toks.index(b"")
+    tok = B.Tokenizer(toks, eos)
+    g = B.Grammar(tok, "ebnf", 'root ::= "a"*')
+    m = B.Matcher(g, max_sets=10)
+    batch = B.Batch([m])
+    ids = torch.tensor([toks.index(b"aaaa")], dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    seen = []
+    for _ in range(4):
+        batch.accept_token(ids.data_ptr(), st.data_ptr())
+        seen.append(int(st.cpu()[0]))
+    assert seen == [0, 0, B.XG_ERR_CAPACITY, B.XG_ERR_CAPACITY]
+    mask = torch.zeros((1, tok.words), dtype=torch.int32, device="cuda")
+    batch.fill_next_token_bitmask(mask.data_ptr(), tok.words, st.data_ptr())       # state still usable
+    bits = O.unpack_bits(mask.cpu().numpy().view(np.uint32)[0], len(toks))
+    assert bits[ord("a")] and bits[eos] and bits[toks.index(b"aaaa")] and bits.sum() == 3
+    m.close(); g.close(); tok.close()
