@@ -98,9 +98,10 @@ def test_hand_worked_masks_on_gpu():
     for fixture in ["mask_ab_ac.txt", "mask_bool_object.txt", "mask_nested_arrays.txt"]:
         ebnf, tokens, cases = load_mask_fixture(fixture)
         toks = [t.encode() for t in tokens]
-        pad = 32 - len(toks) % 32 if len(toks) % 32 else 0
         eos = tokens.index("")
-        tok = B.Tokenizer(toks + [b"\xff\xfe"] * pad, eos)
+        feed = toks + [bytes([b]) for b in range(256)]         # extra single bytes, only used to feed prefixes
+        feed += [b"\xff\xfe"] * (-len(feed) % 32)
+        tok = B.Tokenizer(feed, eos)
         g = B.Grammar(tok, "ebnf", ebnf)
         m = B.Matcher(g)
         batch = B.Batch([m])
@@ -110,13 +111,10 @@ def test_hand_worked_masks_on_gpu():
         st = torch.zeros(1, dtype=torch.int32, device="cuda")
         for prefix, allowed in cases:
             m.reset()
-            for byte in prefix.encode():        # single-byte tokens may be missing: feed known tokens greedily
-                pass
-            # feed the prefix with the longest tokens available
             rest = prefix.encode()
-            while rest:
-                cand = max((t for t in toks if t and rest.startswith(t)), key=len)
-                ids[0] = toks.index(cand)
+            while rest:                          # feed the prefix with the longest tokens available
+                cand = max((t for t in feed if t and rest.startswith(t)), key=len)
+                ids[0] = feed.index(cand)
                 batch.accept_token(ids.data_ptr(), st.data_ptr())
                 assert int(st.cpu()[0]) == 0, (prefix, cand)
                 rest = rest[len(cand):]
