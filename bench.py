@@ -1,0 +1,322 @@
+#!/usr/bin/env python
+"""Benchmark of the token-mask hot path.
+
+One step = one decode step of the whole batch: accept the previously sampled tokens, build every
+request's next-token bitmask (cached sets merged with the Earley check of the uncertain tokens),
+apply it to the batch's logits in place.  The workload is the seeded synthetic config C3
+(128 requests, each with its own JSON-schema grammar, vocabulary 151 936, bf16 logits) unless
+--workload says otherwise.  Grammar compilation (cache build) is timed once before the steps and
+reported beside them.
+
+Prints one JSON line.  `--impl reference` times the CPU oracle instead, as it stands, on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2601_04426_b200 import inputs  # noqa: E402
+
+SHAPES = {"C1": (1, 8192), "C2": (1, 128256), "C3": (128, 151936), "C4": (64, 128256), "C5": (256, 200064)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, index: int = 0):
+        super().__init__(daemon=True)
+        self.index = index
+        self.samples = []
+        self.reasons = set()
+        self.stop_flag = threading.Event()
+        self.proc = None
+
+    def run(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + q, "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            return
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.proc.stdout:
+            if self.stop_flag.is_set():
+                break
+            parts = [x.strip() for x in line.split(",")]
+            try:
+                self.samples.append((float(parts[0]), float(parts[1])))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    self.reasons.add(n)
+
+    def finish(self):
+        self.stop_flag.set()
+        if self.proc is not None:
+            self.proc.terminate()       # the exact child started above
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        sm = sorted(s[0] for s in self.samples)
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(s[1] for s in self.samples), "reasons": sorted(self.reasons), "samples": len(sm)}
+
+
+def oracle_leg(w, steps, warmup, sample_pairs=None):
+    """The CPU oracle, as it stands, on a bounded sample: a few (request, step) masks plus the
+    apply of one row each, scaled to a whole batch step."""
+    from oracle import oracle as O
+    from oracle import schema_ebnf as SE
+    threads = O.default_threads()
+    ov = O.Vocab(w.vocab.tokens, w.vocab.eos_id, w.vocab.special_ids)
+    n_req = min(w.batch, 4)
+    oms = [O.Matcher(O.Grammar(SE.grammar_text(w.grammars[w.request_grammar[b]].kind, w.grammars[w.request_grammar[b]].text))) for b in range(n_req)]
+    logits = inputs.make_logits(w.logits_seed, 1, w.vocab.size, w.dtype)
+    per_step = []
+    total_steps = warmup + steps
+    budget_s = 25.0
+    t_begin = time.perf_counter()
+    for step in range(min(total_steps, w.steps)):
+        t0 = time.perf_counter()
+        for b in range(n_req):
+            mask = oms[b].mask(ov, threads)
+            O.apply_mask(logits, mask[None, :])
+        dt = time.perf_counter() - t0
+        for b in range(n_req):
+            tok = w.trajectories[b][step]
+            if oms[b].accept_token(ov, tok) == 2:
+                oms[b].reset()
+        if step >= warmup:
+            per_step.append(dt / n_req * w.batch)
+        if time.perf_counter() - t_begin > budget_s and len(per_step) >= 1:
+            break
+    us = 1e6 * float(np.mean(per_step))
+    return us, threads, "%d steps x %d of %d requests (mask + apply of each), scaled to the batch" % (len(per_step), n_req, w.batch)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C3", choices=sorted(SHAPES))
+    ap.add_argument("--batch", type=int, default=None, help="shrink the batch (debugging only; the line then names it)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    B0, V = SHAPES[args.workload]
+    metric = "per-step token-mask us (accept + fill + apply) at batch %d x vocab %d" % (args.batch or B0, V)
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        w = inputs.make_workload(args.workload, batch=min(args.batch or B0, 4))
+        w_full_batch = args.batch or B0
+        us, threads, sample = oracle_leg(_with_batch(w, w_full_batch), args.steps, args.warmup)
+        line = {"impl": "reference", "metric": metric, "value": us, "unit": "us/step", "n_gpus": args.gpus, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+                "dtype": "int32", "data": "synthetic", "config": {"workload": args.workload, "batch": w_full_batch, "vocab": V},
+                "cpu_baseline": {"value": us, "unit": "us/step", "cores": threads, "kind": "oracle", "sample": sample},
+                "e2e": {"value": us, "unit": "us/step", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}
+        print(json.dumps(line))
+        return 0
+
+    import torch
+    from paper_2601_04426_b200 import binding as XB
+    from paper_2601_04426_b200 import dist_util, engine
+    torch.cuda.set_device(local_rank)
+    dist_util.init_from_env("nccl")
+    XB.lib()          # fails loudly if the CUDA library is missing
+
+    w = inputs.make_workload(args.workload, batch=args.batch)
+    if world > 1:     # weak scaling: every rank serves its own batch of requests (no data-path collective)
+        w = dist_util.rotate_requests(w, rank)
+    t0 = time.perf_counter()
+    s = engine.Session(w, device="cuda:%d" % local_rank)
+    torch.cuda.synchronize()
+    compile_s = time.perf_counter() - t0
+    stats = [g.stats() for g in s.grammars]
+    build_ms = sum(x["cache_build_ms"] for x in stats)
+    pairs = sum(x["pairs_classified"] for x in stats)
+    pairs_dense = sum(x["n_scannable"] for x in stats) * s.V
+
+    n, W = s.n, s.W
+    elt = 2 if w.dtype == "bf16" else 4
+    tdtype = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    # logits ring larger than twice the L2, so the apply kernel always works out of HBM
+    l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size
+    bytes_one = n * s.V * elt
+    ring_n = max(2, int(np.ceil(2.2 * l2 / bytes_one)) + 1)
+    base = engine.logits_tensor(inputs.make_logits(w.logits_seed, min(n, 8), s.V, w.dtype), s.device)
+    ring = [base.repeat((n + base.shape[0] - 1) // base.shape[0], 1)[:n].contiguous() for _ in range(ring_n)]
+    traj = torch.from_numpy(np.asarray([[w.trajectories[b][t] for b in range(n)] for t in range(w.steps)], dtype=np.int32)).to(s.device)
+    eos_at = {t: [b for b in range(n) if w.trajectories[b][t] == w.vocab.eos_id] for t in range(w.steps)}
+    total = warmup + args.steps
+    launches = {"accept": 0, "merge": 0, "check": 0, "apply": 0, "reset": 0}
+
+    def restart():
+        for b in range(n):
+            s.reset(b)
+
+    def one_step(i, events=None):
+        t = i % w.steps
+        if t == 0 and i > 0:
+            restart()
+        buf = ring[i % ring_n]
+        if events is not None:
+            events[0].record()
+        s.fill()
+        if events is not None:
+            events[1].record()
+        s.apply(buf)
+        if events is not None:
+            events[2].record()
+        s.accept_device(traj[t])
+        for b in eos_at[t]:
+            s.reset(b)
+            launches["reset"] += 1
+        if events is not None:
+            events[3].record()
+        launches["merge"] += 1; launches["check"] += 1; launches["apply"] += 1; launches["accept"] += 1
+
+    # ---- pass A: the headline number (events only around the timed region) --------------------
+    for i in range(warmup):
+        one_step(i)
+    for k in launches:
+        launches[k] = 0
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    dist_util.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(warmup, total):
+        one_step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    dist_util.barrier()
+    clocks = sampler.finish()
+    ms_total = dist_util.max_over_ranks(e0.elapsed_time(e1))
+    us_per_step = 1e3 * ms_total / args.steps
+    timed_launches = sum(launches.values())
+    # masked fraction of the last mask (context for the apply numbers)
+    zero_bits = n * s.V - int(np.unpackbits(s.mask_numpy().view(np.uint8)).sum())
+
+    # ---- pass B: per-kernel times, same steps, events between the calls ------------------------
+    restart()
+    for i in range(warmup):
+        one_step(i)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    for k, i in enumerate(range(warmup, total)):
+        one_step(i, evs[k])
+    torch.cuda.synchronize()
+    t_fill = float(np.mean([e[0].elapsed_time(e[1]) for e in evs])) * 1e3
+    t_apply = float(np.mean([e[1].elapsed_time(e[2]) for e in evs])) * 1e3
+    t_accept = float(np.mean([e[2].elapsed_time(e[3]) for e in evs])) * 1e3
+
+    # apply's algorithmic bytes: the mask words read plus the masked logits written (allowed
+    # logits are neither read nor written); and the conventional count (read + write everything)
+    masked_frac = zero_bits / float(n * s.V)
+    apply_alg_bytes = 4.0 * n * W + elt * zero_bits
+    apply_conv_bytes = 2.0 * elt * n * s.V + 4.0 * n * W
+    peak, peak_kind = measured_peaks()
+    apply_gbs = apply_alg_bytes / (t_apply * 1e-6) / 1e9
+    dominant = max((("fill (merge+check)", t_fill), ("apply", t_apply), ("accept", t_accept)), key=lambda x: x[1])[0]
+    roofline = {"kernel": "apply_kernel", "bound": "hbm", "achieved": apply_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": apply_gbs / peak, "traffic": None, "us_per_launch": t_apply, "masked_fraction": masked_frac,
+                "conventional_gbs": apply_conv_bytes / (t_apply * 1e-6) / 1e9, "dominant_by_time": dominant}
+
+    # ---- end to end through the C ABI with host buffers ---------------------------------------
+    e2e_steps = max(3, min(args.steps, 12))
+    host_in = torch.empty((n, s.V), dtype=tdtype).pin_memory()
+    host_in.copy_(ring[0].cpu())
+    host_out = torch.empty((n, s.V), dtype=tdtype).pin_memory()
+    host_traj = traj.cpu().pin_memory()
+    restart()
+    dev_buf = ring[0]
+    torch.cuda.synchronize()
+    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for phase in ("warm", "timed"):
+        restart()
+        if phase == "timed":
+            torch.cuda.synchronize()
+            h0.record()
+        for t in range(e2e_steps):
+            dev_buf.copy_(host_in, non_blocking=True)
+            s.fill()
+            s.apply(dev_buf)
+            host_out.copy_(dev_buf, non_blocking=True)
+            s.tokens.copy_(host_traj[t], non_blocking=True)
+            s.accept_device(s.tokens)
+            for b in eos_at[t]:
+                s.reset(b)
+        if phase == "timed":
+            h1.record()
+            torch.cuda.synchronize()
+    e2e_us = dist_util.max_over_ranks(h0.elapsed_time(h1)) * 1e3 / e2e_steps
+
+    line = {
+        "metric": metric, "value": us_per_step, "unit": "us/step", "n_gpus": world, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": us_per_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32", "data": "synthetic",
+        "config": {"workload": args.workload, "batch": n, "global_batch": n * world, "vocab": s.V, "logits_dtype": w.dtype,
+                   "grammars": len(w.grammars), "l2": "logits ring of %d buffers (%.0f MB) > 2 x L2" % (ring_n, ring_n * bytes_one / 1e6),
+                   "parallelism": "replicas x%d" % world},
+        "clocks": clocks,
+        "kernels_us": {"fill": t_fill, "apply": t_apply, "accept": t_accept},
+        "apply_gbs": apply_gbs,
+        "cache_build": {"seconds": build_ms / 1e3, "compile_wall_s": compile_s, "pairs_classified": pairs, "pairs_per_s": pairs / max(build_ms / 1e3, 1e-9),
+                        "pairs_dense": pairs_dense, "pairs_dense_per_s": pairs_dense / max(build_ms / 1e3, 1e-9),
+                        "entries_built": sum(x["n_entries_built"] for x in stats), "entries_reused": sum(x["n_entries_reused"] for x in stats),
+                        "cache_bytes_unique_upper": sum(x["cache_bytes"] for x in stats)},
+        "roofline": roofline,
+        "e2e": {"value": e2e_us, "unit": "us/step", "h2d_bytes_per_step": bytes_one + 4 * n, "d2h_bytes_per_step": bytes_one, "steps": e2e_steps},
+        "gpu_launches": timed_launches,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        us, threads, sample = oracle_leg(w, min(args.steps, 6), 0)
+        line["cpu_baseline"] = {"value": us, "unit": "us/step", "cores": threads, "kind": "oracle", "sample": sample}
+    s.close()
+    if rank == 0:
+        print(json.dumps(line))
+    dist_util.finish()
+    return 0
+
+
+def _with_batch(w, batch):
+    """A workload whose nominal batch is `batch` while only the first requests are materialised."""
+    class _View:
+        pass
+    v = _View()
+    v.__dict__.update(w.__dict__)
+    v.batch = batch
+    return v
+
+
+if __name__ == "__main__":
+    sys.exit(main())
