@@ -189,6 +189,29 @@ xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t ba
                                        int32_t* bitmask_dev, int64_t row_stride_words,
                                        int32_t* status_dev, void* stream);
 
+/* xg_fill_next_token_bitmask_static: the same result as xg_fill_next_token_bitmask, for callers
+ * that must not allocate device memory inside their decode loop.  (The paper has no counterpart;
+ * this is a deployment variant of the call above.)  A serving engine that has already handed all
+ * free device memory to its own allocator, or that must keep its step free of the device-wide
+ * synchronisation cudaMalloc / cudaFree imply, cannot use the call above for a batch it has not
+ * seen before, because that call creates the batch's device-side request table and status words
+ * on first use.  This variant keeps them in one fixed array that is part of the library image:
+ * XG_STATIC_FILL_MAX_BATCH requests, 16 KiB, resident on every GPU that loads the library until
+ * the process exits.  It never calls cudaMalloc, cudaFree or any allocating routine; the caller
+ * still passes the bitmask (and optional status) buffers.
+ *   - batch > XG_STATIC_FILL_MAX_BATCH returns XG_ERR_CAPACITY and does nothing.
+ *   - The first call on each device looks up the array's device address; make that first call
+ *     before any stream capture begins.
+ *   - Every call on a device uses the same array: the request table and the per-request words
+ *     are rewritten at the start of each call, so nothing is carried over from the previous one,
+ *     but two calls whose GPU work overlaps (different streams) race; keep them on one stream or
+ *     order them with events.
+ * Arguments, layout, statuses and errors are otherwise those of xg_fill_next_token_bitmask. */
+#define XG_STATIC_FILL_MAX_BATCH 1024
+xg_status_t xg_fill_next_token_bitmask_static(xg_matcher_t* const* matchers, int32_t batch,
+                                              int32_t* bitmask_dev, int64_t row_stride_words,
+                                              int32_t* status_dev, void* stream);
+
 /* xg_apply_token_bitmask: logits[r][v] = -inf where bit v of mask row r is 0 (Section 2.1), in
  * place, one pass.  logits_dev: device, [rows][logits_row_stride_elems] of dtype; every row must
  * start on a 16-byte boundary (XG_ERR_INVALID_ARG otherwise).  row_indices_dev (device, may be

@@ -28,8 +28,9 @@ EXPORTS = [
     "xg_last_error", "xg_tokenizer_create", "xg_tokenizer_destroy", "xg_cache_pool_create", "xg_cache_pool_destroy",
     "xg_compile_grammar", "xg_grammar_destroy", "xg_grammar_get_tables", "xg_grammar_get_rule_hashes", "xg_grammar_get_cache_entry", "xg_grammar_stats",
     "xg_matcher_create", "xg_matcher_reset", "xg_matcher_destroy", "xg_matcher_is_terminated",
-    "xg_fill_next_token_bitmask", "xg_apply_token_bitmask", "xg_accept_token",
+    "xg_fill_next_token_bitmask", "xg_fill_next_token_bitmask_static", "xg_apply_token_bitmask", "xg_accept_token",
 ]
+XG_STATIC_FILL_MAX_BATCH = 1024
 
 
 class XgError(RuntimeError):
@@ -97,6 +98,7 @@ def lib():
         L.xg_matcher_destroy.restype = None
         L.xg_matcher_is_terminated.argtypes = [vp, vp, C.POINTER(i32)]
         L.xg_fill_next_token_bitmask.argtypes = [vp, i32, vp, i64, vp, vp]
+        L.xg_fill_next_token_bitmask_static.argtypes = [vp, i32, vp, i64, vp, vp]
         L.xg_apply_token_bitmask.argtypes = [vp, C.c_int, i32, i32, i64, vp, i64, vp, i32, vp]
         L.xg_accept_token.argtypes = [vp, i32, vp, vp, vp]
         _lib = L
@@ -231,6 +233,11 @@ class Batch:
 
     def fill_next_token_bitmask(self, bitmask_ptr: int, row_stride_words: int, status_ptr: int = 0, stream: int = 0):
         _check(lib().xg_fill_next_token_bitmask(self.handles, self.n, bitmask_ptr, row_stride_words, status_ptr or None, stream))
+
+    def fill_next_token_bitmask_static(self, bitmask_ptr: int, row_stride_words: int, status_ptr: int = 0, stream: int = 0):
+        """Same masks as fill_next_token_bitmask, without any device allocation (at most
+        XG_STATIC_FILL_MAX_BATCH requests; calls must not overlap on the GPU)."""
+        _check(lib().xg_fill_next_token_bitmask_static(self.handles, self.n, bitmask_ptr, row_stride_words, status_ptr or None, stream))
 
     def accept_token(self, token_ids_ptr: int, status_ptr: int = 0, stream: int = 0):
         _check(lib().xg_accept_token(self.handles, self.n, token_ids_ptr, status_ptr or None, stream))

@@ -597,6 +597,65 @@ xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t ba
   return XG_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// the per-step fill for callers that must not allocate: request table, status words and
+// completion counters live in a fixed array inside the library image instead of cudaMalloc'ed
+// per-batch buffers
+// ---------------------------------------------------------------------------------------------
+struct StaticFillScratch {
+  MatcherDev* matchers[XG_STATIC_FILL_MAX_BATCH];
+  int32_t status[XG_STATIC_FILL_MAX_BATCH];
+  int32_t done_count[XG_STATIC_FILL_MAX_BATCH];
+};
+static __device__ __align__(256) unsigned char g_static_fill_scratch[sizeof(StaticFillScratch)];
+
+// The symbol above is only a host-side stand-in; kernels need its device address, which differs
+// per device.  Looked up once per device, with that device current.
+static xg_status_t static_fill_scratch(StaticFillScratch** out) {
+  static std::mutex mu;
+  static StaticFillScratch* by_device[64] = {};
+  int dev = 0;
+  XG_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return set_error(XG_ERR_UNSUPPORTED, "device ordinal above 63");
+  std::lock_guard<std::mutex> lock(mu);
+  if (!by_device[dev]) {
+    void* p = nullptr;
+    XG_CUDA(cudaGetSymbolAddress(&p, g_static_fill_scratch));
+    by_device[dev] = (StaticFillScratch*)p;
+  }
+  *out = by_device[dev];
+  return XG_OK;
+}
+
+xg_status_t xg_fill_next_token_bitmask_static(xg_matcher_t* const* matchers, int32_t batch, int32_t* bitmask_dev, int64_t row_stride_words,
+                                              int32_t* status_dev, void* stream) {
+  if (!matchers || batch <= 0) return set_error(XG_ERR_INVALID_ARG, "empty batch");
+  if (batch > XG_STATIC_FILL_MAX_BATCH)
+    return set_error(XG_ERR_CAPACITY, "batch of " + std::to_string(batch) + " requests exceeds the static scratch limit of " +
+                                          std::to_string(XG_STATIC_FILL_MAX_BATCH) + "; use xg_fill_next_token_bitmask or split the batch");
+  MatcherDev* ptrs[XG_STATIC_FILL_MAX_BATCH];
+  for (int i = 0; i < batch; ++i) {
+    if (!matchers[i]) return set_error(XG_ERR_INVALID_ARG, "NULL matcher in batch");
+    if (matchers[i]->grammar->tok != matchers[0]->grammar->tok) return set_error(XG_ERR_INVALID_ARG, "matchers of one batch must share a tokenizer");
+    ptrs[i] = matchers[i]->dev;
+  }
+  const xg_tokenizer* tok = matchers[0]->grammar->tok;
+  if (!bitmask_dev || row_stride_words < tok->n_words) return set_error(XG_ERR_INVALID_ARG, "bad bitmask buffer");
+  StaticFillScratch* sc = nullptr;
+  xg_status_t st = static_fill_scratch(&sc);
+  if (st != XG_OK) return st;
+  cudaStream_t cs = (cudaStream_t)stream;
+  // the array keeps the previous call's contents: rewrite the request table, clear the words
+  XG_CUDA(cudaMemcpyAsync(sc->matchers, ptrs, sizeof(MatcherDev*) * batch, cudaMemcpyHostToDevice, cs));
+  XG_CUDA(cudaMemsetAsync(sc->status, 0, 2 * sizeof(int32_t) * XG_STATIC_FILL_MAX_BATCH, cs));
+  const int W = tok->n_words;
+  int chunks = std::max((W + kMergeMaxChunkWords - 1) / kMergeMaxChunkWords, std::min(8, (W + 127) / 128));
+  merge_kernel<<<dim3(chunks, batch), 256, 0, cs>>>(sc->matchers, tok->dev, bitmask_dev, (long long)row_stride_words, status_dev, sc->status, sc->done_count);
+  check_kernel<<<dim3(8, batch), 256, 0, cs>>>(sc->matchers, tok->dev, bitmask_dev, (long long)row_stride_words, status_dev, sc->status, sc->done_count);
+  XG_CUDA(cudaGetLastError());
+  return XG_OK;
+}
+
 xg_status_t xg_accept_token(xg_matcher_t* const* matchers, int32_t batch, const int32_t* token_ids_dev, int32_t* status_dev, void* stream) {
   const xg_tokenizer* tok = nullptr;
   BatchSlot* slot = nullptr;
