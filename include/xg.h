@@ -85,7 +85,7 @@ void xg_cache_pool_destroy(xg_cache_pool_t* pool);
 typedef struct {
   uint32_t struct_size;       /* sizeof(xg_compile_options_t), for versioning */
   int32_t inline_max_states;  /* inline non-recursive rules whose automaton has at most this many
-                                 states into their users; 0 = never; negative = default (12). */
+                                 states into their users; 0 = never; negative = default (16). */
   int32_t max_rule_states;    /* XG_ERR_CAPACITY if one rule's automaton grows past this.  <= 0 = default (1<<20). */
   int32_t build_cache;        /* 0 = front end only (tables, no device work).  Otherwise build. */
 } xg_compile_options_t;

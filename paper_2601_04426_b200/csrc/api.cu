@@ -295,6 +295,7 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
     uint32_t* arena = (uint32_t*)g->pool->allocate_device((size_t)std::max<long long>(total_words, 1) * 4);
     if (!arena) { cleanup(); return set_error(XG_ERR_OOM, "cache arena allocation failed"); }
     pack_kernel<<<n, 256, 0, stream>>>(acc, unc, unr, d_plan, V, W, arena, d_entries);
+    exit_kernel<<<n, 256, 0, stream>>>(g->host_view, v, d_pos, d_entries);
     XG_CUDA_C(cudaGetLastError());
     std::vector<EntryDev> built(n);
     std::vector<int2> counts(n);
@@ -410,7 +411,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     g->stats.total_uncertain += c.y;
     g->stats.total_rejected += tok->vocab_size - c.x - c.y;
     g->stats.kind_count[e.kind]++;
-    g->stats.cache_bytes += 4LL * ((e.kind == 2 ? tok->n_words : e.n_list) + 2LL * e.n_unc);
+    g->stats.cache_bytes += 4LL * ((e.kind == 2 ? tok->n_words : e.n_list) + 3LL * e.n_unc);
   }
   *out = g.release();
   return XG_OK;

@@ -25,6 +25,7 @@ struct EntryDev {
   const uint32_t* data;      // accepted ids | rejected ids | accepted bitset (n_words words)
   const uint32_t* unc_id;    // [n_unc] ascending token ids
   const uint32_t* unc_rank;  // [n_unc] ascending ranks
+  const uint32_t* unc_exit;  // [n_unc] parallel to unc_rank: bit j = the token leaves the entry's rule after j bytes
   int32_t kind;              // xg_store_kind_t
   int32_t n_list;            // list length (0 for bitset)
   int32_t n_unc;
@@ -43,7 +44,7 @@ struct GrammarDev {
   const uint32_t* wait_rule;
   const uint32_t* wait_target;    // bit 31: origin = the set the completed rule started in
   const int32_t* gather_begin;    // [S+1]
-  const int32_t* gather_state;
+  const int32_t* gather_state;    // bit 31: a predicted start state (its items begin in the current set)
   const uint32_t* class_bits;     // [C][8]
   const EntryDev* entries;        // [S]; meaningful for scannable states
 };

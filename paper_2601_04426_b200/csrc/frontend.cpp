@@ -779,6 +779,9 @@ struct Compiler {
   // Replace references to small non-recursive rules by a copy of their automaton.  A rule that
   // is referenced from a single place may be larger (inlining it duplicates nothing); this also
   // folds alternatives such as the tool calls of a TagDispatch into one deterministic automaton.
+  // A rule used a few times may also be somewhat larger as long as size x uses stays bounded
+  // (a character rule repeated by a bounded string must not stay a rule of its own: every
+  // multi-byte token would leave it and become context-dependent).
   void inline_small_rules() {
     if (opt.inline_max_states <= 0) return;
     const int single_use_max = std::max(64, opt.inline_max_states);
@@ -801,7 +804,8 @@ struct Compiler {
         const std::vector<Edge> edges = g.out[s];     // g.out may reallocate while copies are appended
         for (const Edge& e : edges) {
           bool take = e.kind == Edge::kRef && e.rule != r && candidate[e.rule] &&
-                      (b.rules[e.rule].size() <= opt.inline_max_states || uses[e.rule] == 1) &&
+                      (b.rules[e.rule].size() <= opt.inline_max_states || uses[e.rule] == 1 ||
+                       b.rules[e.rule].size() * uses[e.rule] <= 16 * opt.inline_max_states) &&
                       g.size() + b.rules[e.rule].size() <= opt.max_rule_states;
           if (take) {
             const Fsm& c = b.rules[e.rule];
@@ -905,7 +909,7 @@ struct Compiler {
         int s0 = g.rule_start[r];
         for (int e = g.cedge_begin[s0]; e < g.cedge_begin[s0 + 1]; ++e) { g.scan_class.push_back(g.cedge_class[e]); g.scan_target.push_back((uint32_t)g.cedge_target[e] | kSelfBit); }
         for (int e = g.redge_begin[s0]; e < g.redge_begin[s0 + 1]; ++e) { g.wait_rule.push_back(g.redge_rule[e]); g.wait_target.push_back((uint32_t)g.redge_target[e] | kSelfBit); }
-        if (g.cedge_begin[s0 + 1] > g.cedge_begin[s0] && s0 != s) g.gather_state.push_back(s0);
+        if (g.cedge_begin[s0 + 1] > g.cedge_begin[s0]) g.gather_state.push_back((int32_t)((uint32_t)s0 | kSelfBit));
       }
       g.scan_begin.push_back((int)g.scan_class.size());
       g.wait_begin.push_back((int)g.wait_rule.size());

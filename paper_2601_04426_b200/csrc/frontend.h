@@ -27,7 +27,7 @@ struct FrontendError {
 };
 
 struct FrontendOptions {
-  int inline_max_states = 12;
+  int inline_max_states = 16;
   int max_rule_states = 1 << 20;
 };
 
@@ -52,8 +52,9 @@ struct FlatGrammar {
   //                     every rule predicted (transitively) from s, flagged kSelfBit;
   //   wait list of s  = own rule-reference edges, then those of the predicted start states
   //                     (kSelfBit): who advances when rule r completes back into this set;
-  //   gather list of s = the scannable states among s and its predicted start states: the
-  //                     cache entries a kernel item contributes to a step's mask.
+  //   gather list of s = the scannable states among s and its predicted start states (the
+  //                     latter flagged kSelfBit, even when equal to s): the cache entries a
+  //                     kernel item contributes to a step's mask.
   std::vector<int32_t> scan_begin, scan_own_end;
   std::vector<uint32_t> scan_class, scan_target;
   std::vector<int32_t> wait_begin;

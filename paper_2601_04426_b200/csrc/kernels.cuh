@@ -21,44 +21,87 @@ constexpr int kSlowMaxBytes = 255;
 // The token walk: Earley scan / complete over the bytes of one token (appendix "Earley's
 // Parsing Algorithm"), on kernel items only.
 //
-// Base chart: sets 0..n given by (h_st, h_org, h_sb); the walk starts from set n.  New sets are
-// appended to (st, org) with boundaries lsb[j] .. lsb[j+1] for the set reached after byte j
-// (1-based), and carry chart indices n+j.  Origin -1 stands for the unknown context of a cache
-// entry (Section 3.4): completing such an item cannot advance anything that is known here.
+// Chart: history sets 0..n given by (h_st, h_org, h_sb); an initial set (i_st, i_org, i_cnt)
+// with chart index i_idx >= n (it may simply be history set n); the walk appends new sets to
+// (st, org) with boundaries lsb[j] .. lsb[j+1] for the set reached after byte j (1-based), chart
+// index i_idx + j.  Origin -1 stands for the unknown context of a cache entry (Section 3.4):
+// completing such an item cannot advance anything known here; the byte offsets at which that
+// happens (with bytes left) are the token's exits from its rule.
 //
 // Returns the number of bytes after which the set was still non-empty (len = token survives).
 // ------------------------------------------------------------------------------------------
+struct Chart {
+  const uint32_t* h_st;
+  const int32_t* h_org;
+  const int32_t* h_sb;
+  int n;
+  const uint32_t* i_st;
+  const int32_t* i_org;
+  int i_cnt, i_idx;
+};
+
+__device__ __forceinline__ Chart chart_of_history(const uint32_t* h_st, const int32_t* h_org, const int32_t* h_sb, int n) {
+  Chart c;
+  c.h_st = h_st; c.h_org = h_org; c.h_sb = h_sb; c.n = n;
+  const int b = h_sb[n];
+  c.i_st = h_st + b; c.i_org = h_org + b; c.i_cnt = h_sb[n + 1] - b; c.i_idx = n;
+  return c;
+}
+
+// append (ns, no) to the set [start, cnt) unless present; false on overflow
+__device__ __forceinline__ bool add_item(uint32_t* st, int32_t* org, int start, int& cnt, int cap, uint32_t ns, int32_t no) {
+  for (int q = start; q < cnt; ++q) if (st[q] == ns && org[q] == no) return true;
+  if (cnt >= cap) return false;
+  st[cnt] = ns; org[cnt] = no; ++cnt;
+  return true;
+}
+
+// advance every item of chart set `o` that waits for `rule` into the set [start, cnt)
 template <typename LsbT>
-__device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* h_st, const int32_t* h_org, const int32_t* h_sb, int n,
-                                          const uint8_t* __restrict__ bytes, int len, bool own_edges_first,
-                                          uint32_t* st, int32_t* org, int cap, LsbT* lsb, int* flags) {
+__device__ __forceinline__ bool advance_waiters(const GrammarDev& g, const Chart& c, uint32_t rule, int32_t o, uint32_t* st, int32_t* org,
+                                                const LsbT* lsb, int start, int& cnt, int cap) {
+  const uint32_t* src_st;
+  const int32_t* src_org;
+  int b, e;
+  if (o < c.i_idx) { src_st = c.h_st; src_org = c.h_org; b = c.h_sb[o]; e = c.h_sb[o + 1]; }
+  else if (o == c.i_idx) { src_st = c.i_st; src_org = c.i_org; b = 0; e = c.i_cnt; }
+  else { src_st = st; src_org = org; b = lsb[o - c.i_idx]; e = lsb[o - c.i_idx + 1]; }
+  for (int i = b; i < e; ++i) {
+    const uint32_t s2 = src_st[i];
+    const int32_t o2 = src_org[i];
+    for (int w = g.wait_begin[s2]; w < g.wait_begin[s2 + 1]; ++w) {
+      if (g.wait_rule[w] != rule) continue;
+      const uint32_t t = g.wait_target[w];
+      if (!add_item(st, org, start, cnt, cap, t & ~kSelf, (t & kSelf) ? o : o2)) return false;
+    }
+  }
+  return true;
+}
+
+template <typename LsbT>
+__device__ __forceinline__ int token_walk(const GrammarDev& g, const Chart& c, const uint8_t* __restrict__ bytes, int len, bool own_edges_first,
+                                          uint32_t* st, int32_t* org, int cap, LsbT* lsb, int* flags, uint32_t* exit_mask) {
   int cnt = 0;
-  int cur_b = h_sb[n], cur_e = h_sb[n + 1];
-  bool cur_hist = true;
+  const uint32_t* cur_st = c.i_st;
+  const int32_t* cur_org = c.i_org;
+  int cur_b = 0, cur_e = c.i_cnt;
   lsb[0] = 0;
   lsb[1] = 0;
   for (int k = 0; k < len; ++k) {
     const uint32_t byte = bytes[k];
     const uint32_t word = byte >> 5, bit = 1u << (byte & 31);
     const int start = cnt;
-    const int self_idx = n + k;
+    const int self_idx = c.i_idx + k;
     // scan
     for (int i = cur_b; i < cur_e; ++i) {
-      const uint32_t s = cur_hist ? h_st[i] : st[i];
-      const int32_t o = cur_hist ? h_org[i] : org[i];
+      const uint32_t s = cur_st[i];
+      const int32_t o = cur_org[i];
       const int e0 = g.scan_begin[s];
       const int e1 = (k == 0 && own_edges_first) ? g.scan_own_end[s] : g.scan_begin[s + 1];
       for (int e = e0; e < e1; ++e) {
         if (g.class_bits[g.scan_class[e] * 8 + word] & bit) {
           const uint32_t t = g.scan_target[e];
-          const uint32_t ns = t & ~kSelf;
-          const int32_t no = (t & kSelf) ? self_idx : o;
-          bool dup = false;
-          for (int q = start; q < cnt; ++q) dup = dup || (st[q] == ns && org[q] == no);
-          if (!dup) {
-            if (cnt >= cap) { *flags |= kWalkOverflow; return k; }
-            st[cnt] = ns; org[cnt] = no; ++cnt;
-          }
+          if (!add_item(st, org, start, cnt, cap, t & ~kSelf, (t & kSelf) ? self_idx : o)) { *flags |= kWalkOverflow; return k; }
         }
       }
     }
@@ -67,30 +110,14 @@ __device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* h
     for (int q = start; q < cnt; ++q) {
       const uint32_t info = g.state_info[st[q]];
       if (!(info >> 31)) continue;
-      const uint32_t rule = info & 0x7FFFFFFFu;
       const int32_t o = org[q];
-      if (o < 0) { if (k + 1 < len) *flags |= kWalkUncertain; continue; }
-      int b, e;
-      const bool hist = o <= n;
-      if (hist) { b = h_sb[o]; e = h_sb[o + 1]; } else { b = lsb[o - n]; e = lsb[o - n + 1]; }
-      for (int i = b; i < e; ++i) {
-        const uint32_t s2 = hist ? h_st[i] : st[i];
-        const int32_t o2 = hist ? h_org[i] : org[i];
-        for (int w = g.wait_begin[s2]; w < g.wait_begin[s2 + 1]; ++w) {
-          if (g.wait_rule[w] != rule) continue;
-          const uint32_t t = g.wait_target[w];
-          const uint32_t ns = t & ~kSelf;
-          const int32_t no = (t & kSelf) ? o : o2;
-          bool dup = false;
-          for (int z = start; z < cnt; ++z) dup = dup || (st[z] == ns && org[z] == no);
-          if (!dup) {
-            if (cnt >= cap) { *flags |= kWalkOverflow; return k; }
-            st[cnt] = ns; org[cnt] = no; ++cnt;
-          }
-        }
+      if (o < 0) {
+        if (k + 1 < len) { *flags |= kWalkUncertain; if (exit_mask && k + 1 < 32) *exit_mask |= 1u << (k + 1); }
+        continue;
       }
+      if (!advance_waiters(g, c, info & 0x7FFFFFFFu, o, st, org, lsb, start, cnt, cap)) { *flags |= kWalkOverflow; return k; }
     }
-    cur_b = start; cur_e = cnt; cur_hist = false;
+    cur_st = st; cur_org = org; cur_b = start; cur_e = cnt;
     lsb[k + 2] = (LsbT)cnt;
   }
   return len;
@@ -108,9 +135,8 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
                 int2* __restrict__ overflow, int* __restrict__ overflow_count, int overflow_cap) {
   __shared__ uint32_t sh_st[1];
   __shared__ int32_t sh_org[1];
-  __shared__ int32_t sh_sb[2];
   const int pos = blockIdx.y;
-  if (threadIdx.x == 0) { sh_st[0] = (uint32_t)positions[pos]; sh_org[0] = -1; sh_sb[0] = 0; sh_sb[1] = 1; }
+  if (threadIdx.x == 0) { sh_st[0] = (uint32_t)positions[pos]; sh_org[0] = -1; }
   __syncthreads();
   const int rank = blockIdx.x * blockDim.x + threadIdx.x;
   int cls = 0;
@@ -124,7 +150,10 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
       uint32_t st[kFastCap];
       int32_t org[kFastCap];
       int16_t lsb[kFastMaxBytes + 2];
-      consumed = token_walk<int16_t>(g, sh_st, sh_org, sh_sb, 0, v.bytes + off, len, true, st, org, kFastCap, lsb, &flags);
+      Chart c;
+      c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1;
+      c.i_st = sh_st; c.i_org = sh_org; c.i_cnt = 1; c.i_idx = 0;
+      consumed = token_walk<int16_t>(g, c, v.bytes + off, len, true, st, org, kFastCap, lsb, &flags, nullptr);
     }
     if (flags & kWalkOverflow) {
       int slot = atomicAdd(overflow_count, 1);
@@ -151,13 +180,15 @@ __global__ void classify_slow_kernel(GrammarDev g, VocabDev v, const int32_t* __
   const int pos = pairs[i].x, rank = pairs[i].y;
   uint32_t h_st = (uint32_t)positions[pos];
   int32_t h_org = -1;
-  int32_t h_sb[2] = {0, 1};
+  Chart c;
+  c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1;
+  c.i_st = &h_st; c.i_org = &h_org; c.i_cnt = 1; c.i_idx = 0;
   const uint32_t off = v.offset[rank];
   const int len = (int)(v.offset[rank + 1] - off);
   if (len > kSlowMaxBytes) { atomicExch(failed, 1); return; }
   int flags = 0;
-  int consumed = token_walk<int32_t>(g, &h_st, &h_org, h_sb, 0, v.bytes + off, len, true, scratch_st + (size_t)i * kSlowCap,
-                                     scratch_org + (size_t)i * kSlowCap, kSlowCap, scratch_lsb + (size_t)i * (kSlowMaxBytes + 2), &flags);
+  int consumed = token_walk<int32_t>(g, c, v.bytes + off, len, true, scratch_st + (size_t)i * kSlowCap,
+                                     scratch_org + (size_t)i * kSlowCap, kSlowCap, scratch_lsb + (size_t)i * (kSlowMaxBytes + 2), &flags, nullptr);
   if (flags & kWalkOverflow) { atomicExch(failed, 1); return; }
   int cls = consumed == len ? 1 : ((flags & kWalkUncertain) ? 2 : 0);
   if (!cls) return;
@@ -211,7 +242,7 @@ plan_kernel(const int2* __restrict__ counts, int n_pos, int vocab_size, int n_wo
     if (nr < n_list) { kind = 1; n_list = nr; }
     if (n_words < n_list) { kind = 2; n_list = 0; }
     plan[p].kind = kind; plan[p].n_list = n_list; plan[p].n_acc = na; plan[p].n_unc = nu;
-    local += (kind == 2 ? n_words : n_list) + 2LL * nu;
+    local += (kind == 2 ? n_words : n_list) + 3LL * nu;
   }
   sums[threadIdx.x] = local;
   __syncthreads();
@@ -224,7 +255,7 @@ plan_kernel(const int2* __restrict__ counts, int n_pos, int vocab_size, int n_wo
   long long run = sums[threadIdx.x] - local;
   for (int p = lo; p < hi; ++p) {
     plan[p].offset_words = run;
-    run += (plan[p].kind == 2 ? n_words : plan[p].n_list) + 2LL * plan[p].n_unc;
+    run += (plan[p].kind == 2 ? n_words : plan[p].n_list) + 3LL * plan[p].n_unc;
   }
   if (threadIdx.x == blockDim.x - 1) *total_words = sums[threadIdx.x];
 }
@@ -277,9 +308,41 @@ pack_kernel(const uint32_t* __restrict__ acc_id, const uint32_t* __restrict__ un
   compact_bits([&](int w) { return ur[w]; }, n_words, out_urank, sh_scan);
   if (threadIdx.x == 0) {
     EntryDev e;
-    e.data = data; e.unc_id = out_uid; e.unc_rank = out_urank;
+    e.data = data; e.unc_id = out_uid; e.unc_rank = out_urank; e.unc_exit = out_urank + pl.n_unc;
     e.kind = pl.kind; e.n_list = pl.n_list; e.n_unc = pl.n_unc; e.n_acc = pl.n_acc;
     entries[p] = e;
+  }
+}
+
+// For every uncertain token of every packed entry: the byte offsets at which the token leaves
+// the entry's rule (bit j = after j bytes).  The run-time check restarts there instead of
+// re-walking the part of the token that the cache already decided.  0 = unknown (walk in full).
+__global__ void __launch_bounds__(256)
+exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, const EntryDev* __restrict__ entries) {
+  __shared__ uint32_t sh_st[1];
+  __shared__ int32_t sh_org[1];
+  const int p = blockIdx.x;
+  const EntryDev e = entries[p];
+  if (threadIdx.x == 0) { sh_st[0] = (uint32_t)positions[p]; sh_org[0] = -1; }
+  __syncthreads();
+  uint32_t* out = const_cast<uint32_t*>(e.unc_exit);
+  for (int k = threadIdx.x; k < e.n_unc; k += blockDim.x) {
+    const int rank = (int)e.unc_rank[k];
+    const uint32_t off = v.offset[rank];
+    const int len = (int)(v.offset[rank + 1] - off);
+    uint32_t mask = 0;
+    if (len <= kFastMaxBytes) {
+      uint32_t st[kFastCap];
+      int32_t org[kFastCap];
+      int16_t lsb[kFastMaxBytes + 2];
+      int flags = 0;
+      Chart c;
+      c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1;
+      c.i_st = sh_st; c.i_org = sh_org; c.i_cnt = 1; c.i_idx = 0;
+      token_walk<int16_t>(g, c, v.bytes + off, len, true, st, org, kFastCap, lsb, &flags, &mask);
+      if (flags & kWalkOverflow) mask = 0;
+    }
+    out[k] = mask;
   }
 }
 
@@ -338,8 +401,9 @@ __global__ void accept_kernel(MatcherDev* const* __restrict__ matchers, int batc
         int16_t lsb[kFastMaxBytes + 2];
         int flags = 0;
         const int room = min(m.cap_items - n_items, 32000);
-        const int consumed = token_walk<int16_t>(g, m.item_state, m.item_origin, m.set_begin, n_sets - 1, v.bytes + off + done, piece,
-                                                 false, m.item_state + n_items, m.item_origin + n_items, room, lsb, &flags);
+        const Chart c = chart_of_history(m.item_state, m.item_origin, m.set_begin, n_sets - 1);
+        const int consumed = token_walk<int16_t>(g, c, v.bytes + off + done, piece, false, m.item_state + n_items, m.item_origin + n_items,
+                                                 room, lsb, &flags, nullptr);
         if (flags & kWalkOverflow) { st = -6; break; }
         if (consumed < piece) { st = -7; break; }
         // origins written by the walk are already chart indices (its base is set n_sets - 1);
@@ -396,7 +460,7 @@ merge_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
     for (int i = m.set_begin[n]; i < m.set_begin[n + 1]; ++i) {
       const uint32_t s = m.item_state[i];
       for (int gi = g.gather_begin[s]; gi < g.gather_begin[s + 1]; ++gi) {
-        const EntryDev e = g.entries[g.gather_state[gi]];
+        const EntryDev e = g.entries[g.gather_state[gi] & 0x7FFFFFFF];
         if (e.kind == 2) {
           for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] |= e.data[w0 + w];
         } else if (e.kind == 0) {
@@ -426,18 +490,32 @@ merge_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
 
 // ------------------------------------------------------------------------------------------
 // Per-step mask, part 2: check the uncertain tokens of the current scannable states against
-// the request's full Earley state (Section 3.4).  grid = (slices, batch).  The uncertain lists
-// are walked in trie order, one token per lane, so neighbouring lanes share prefixes.
-// The last block of a request to finish clears the row if any of its walks overflowed.
+// the request's full Earley state (Section 3.4).  grid = (slices, batch).
+//
+// An uncertain token of entry (state q, origin o) fails inside q's rule; its only way to be
+// allowed is to leave the rule at one of its recorded exit offsets and continue in the context.
+// What the context looks like right after the rule completes does not depend on the token: it
+// is the set obtained by completing rule(q) started at o.  That continuation set is computed
+// once per entry, together with the set of bytes it can scan; each token then needs one bit
+// test per exit, and only the survivors walk their remaining bytes from the continuation set.
+// Tokens are taken in trie order, one per lane, so neighbouring lanes share prefixes.
+// The last block of a request to finish clears the row if anything overflowed.
 // ------------------------------------------------------------------------------------------
-constexpr int kMaxStepEntries = 64;
+constexpr int kMaxStepEntries = 48;
+constexpr int kContCap = 16;
 
 __global__ void __launch_bounds__(256)
 check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __restrict__ bitmask, long long row_stride,
              int32_t* __restrict__ status_user, int32_t* __restrict__ status, int32_t* __restrict__ done_count) {
-  __shared__ const uint32_t* ent_list[kMaxStepEntries];
+  __shared__ const uint32_t* ent_rank[kMaxStepEntries];
+  __shared__ const uint32_t* ent_exit[kMaxStepEntries];
   __shared__ int ent_cum[kMaxStepEntries + 1];
   __shared__ int ent_state[kMaxStepEntries];
+  __shared__ int ent_origin[kMaxStepEntries];
+  __shared__ uint32_t cont_st[kMaxStepEntries][kContCap];
+  __shared__ int32_t cont_org[kMaxStepEntries][kContCap];
+  __shared__ int cont_cnt[kMaxStepEntries];
+  __shared__ uint32_t cont_first[kMaxStepEntries][8];
   __shared__ int n_ent;
   __shared__ int sh_fail;
   __shared__ int sh_last;
@@ -445,21 +523,24 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
   const MatcherDev& m = *matchers[b];
   const GrammarDev& g = *m.grammar;
   const int n = m.n_sets - 1;
+  const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
   if (threadIdx.x == 0) {
     int ne = 0, fail = 0;
     ent_cum[0] = 0;
     if (!m.terminated) {
-      for (int i = m.set_begin[n]; i < m.set_begin[n + 1] && !fail; ++i) {
-        const uint32_t s = m.item_state[i];
+      for (int i = 0; i < hist.i_cnt && !fail; ++i) {
+        const uint32_t s = hist.i_st[i];
         for (int gi = g.gather_begin[s]; gi < g.gather_begin[s + 1]; ++gi) {
-          const int q = g.gather_state[gi];
+          const int q = g.gather_state[gi] & 0x7FFFFFFF;
+          const int origin = g.gather_state[gi] < 0 ? n : hist.i_org[i];     // predicted start states begin here
           bool seen = false;
-          for (int z = 0; z < ne; ++z) seen = seen || ent_state[z] == q;
+          for (int z = 0; z < ne; ++z) seen = seen || (ent_state[z] == q && ent_origin[z] == origin);
           if (seen) continue;
           const EntryDev& e = g.entries[q];
           if (e.n_unc == 0) continue;
           if (ne == kMaxStepEntries) { fail = 1; break; }
-          ent_state[ne] = q; ent_list[ne] = e.unc_rank; ent_cum[ne + 1] = ent_cum[ne] + e.n_unc; ++ne;
+          ent_state[ne] = q; ent_origin[ne] = origin; ent_rank[ne] = e.unc_rank; ent_exit[ne] = e.unc_exit;
+          ent_cum[ne + 1] = ent_cum[ne] + e.n_unc; ++ne;
         }
       }
     }
@@ -467,26 +548,71 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
     sh_fail = fail;
   }
   __syncthreads();
+  // continuation set of every entry: complete rule(q) started at its origin, with cascades
+  if ((int)threadIdx.x < n_ent) {
+    const int e = threadIdx.x;
+    uint32_t* st = cont_st[e];
+    int32_t* org = cont_org[e];
+    int cnt = 0;
+    int16_t no_local[2] = {0, 0};
+    bool ok = advance_waiters(g, hist, g.state_info[ent_state[e]] & 0x7FFFFFFFu, ent_origin[e], st, org, no_local, 0, cnt, kContCap);
+    for (int q = 0; ok && q < cnt; ++q) {
+      const uint32_t info = g.state_info[st[q]];
+      if (info >> 31) ok = advance_waiters(g, hist, info & 0x7FFFFFFFu, org[q], st, org, no_local, 0, cnt, kContCap);
+    }
+    if (!ok) sh_fail = 1;
+    cont_cnt[e] = ok ? cnt : 0;
+    uint32_t first[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int q = 0; q < cont_cnt[e]; ++q)
+      for (int x = g.scan_begin[st[q]]; x < g.scan_begin[st[q] + 1]; ++x) {
+        const uint32_t* cb = g.class_bits + g.scan_class[x] * 8;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) first[w] |= cb[w];
+      }
+#pragma unroll
+    for (int w = 0; w < 8; ++w) cont_first[e][w] = first[w];
+  }
+  __syncthreads();
   const int total = ent_cum[n_ent];
   uint32_t* row = (uint32_t*)bitmask + (long long)b * row_stride;
   for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < total; j += gridDim.x * blockDim.x) {
     int e = 0;
     while (j >= ent_cum[e + 1]) ++e;
-    const int rank = (int)ent_list[e][j - ent_cum[e]];
-    const int id = v.rank_to_id[rank];
-    if ((row[id >> 5] >> (id & 31)) & 1u) continue;         // already allowed by some cache
+    const int k = j - ent_cum[e];
+    const int rank = (int)ent_rank[e][k];
+    uint32_t exits = ent_exit[e][k];
     const uint32_t off = v.offset[rank];
     const int len = (int)(v.offset[rank + 1] - off);
-    int flags = 0, consumed = 0;
-    if (len > kFastMaxBytes) flags = kWalkOverflow;
-    else {
-      uint32_t st[kFastCap];
-      int32_t org[kFastCap];
-      int16_t lsb[kFastMaxBytes + 2];
-      consumed = token_walk<int16_t>(g, m.item_state, m.item_origin, m.set_begin, n, v.bytes + off, len, false, st, org, kFastCap, lsb, &flags);
+    bool pass = false, overflow = false;
+    if (exits == 0) {
+      // no exit record (very long token, or its walk overflowed at build time): walk in full
+      if (len > kFastMaxBytes) overflow = true;
+      else {
+        uint32_t st[kFastCap];
+        int32_t org[kFastCap];
+        int16_t lsb[kFastMaxBytes + 2];
+        int flags = 0;
+        pass = token_walk<int16_t>(g, hist, v.bytes + off, len, false, st, org, kFastCap, lsb, &flags, nullptr) == len;
+        overflow = (flags & kWalkOverflow) != 0;
+      }
+    } else {
+      while (exits && !pass && !overflow) {
+        const int at = __ffs(exits) - 1;
+        exits &= exits - 1;
+        const uint32_t byte = v.bytes[off + at];
+        if (!((cont_first[e][byte >> 5] >> (byte & 31)) & 1u)) continue;
+        uint32_t st[kFastCap];
+        int32_t org[kFastCap];
+        int16_t lsb[kFastMaxBytes + 2];
+        int flags = 0;
+        Chart c = hist;
+        c.i_st = cont_st[e]; c.i_org = cont_org[e]; c.i_cnt = cont_cnt[e]; c.i_idx = n + at;
+        pass = token_walk<int16_t>(g, c, v.bytes + off + at, len - at, false, st, org, kFastCap, lsb, &flags, nullptr) == len - at;
+        overflow = (flags & kWalkOverflow) != 0;
+      }
     }
-    if (flags & kWalkOverflow) sh_fail = 1;
-    else if (consumed == len) atomicOr(&row[id >> 5], 1u << (id & 31));
+    if (overflow) sh_fail = 1;
+    else if (pass) { const int id = v.rank_to_id[rank]; atomicOr(&row[id >> 5], 1u << (id & 31)); }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
