@@ -174,34 +174,52 @@ def main():
     ring_n = max(2, int(np.ceil(2.2 * l2 / bytes_one)) + 1)
     base = engine.logits_tensor(inputs.make_logits(w.logits_seed, min(n, 8), s.V, w.dtype), s.device)
     ring = [base.repeat((n + base.shape[0] - 1) // base.shape[0], 1)[:n].contiguous() for _ in range(ring_n)]
-    traj = torch.from_numpy(np.asarray([[w.trajectories[b][t] for b in range(n)] for t in range(w.steps)], dtype=np.int32)).to(s.device)
+    traj = torch.from_numpy(np.asarray([[w.trajectories[b][t] for b in range(n)] for t in range(w.steps)], dtype=np.int32)).to(s.device)      # [steps, n]
     eos_at = {t: [b for b in range(n) if w.trajectories[b][t] == w.vocab.eos_id] for t in range(w.steps)}
     total = warmup + args.steps
-    launches = {"accept": 0, "merge": 0, "check": 0, "apply": 0, "reset": 0}
+    launches = {"accept": 0, "merge": 0, "check": 0, "apply": 0, "reset": 0}      # this library's kernels only
 
     def restart():
         for b in range(n):
             s.reset(b)
+        step_idx.zero_()
 
-    def one_step(i, events=None):
+    # The decode loop is launch-bound (four short kernels per step), so the timed loop replays
+    # CUDA graphs, as a serving engine's decode loop does: one graph per ring buffer holding
+    # fill + apply + accept.  The tokens of step t are gathered on the device from the resident
+    # trajectory table by a step counter that the graph itself advances.
+    step_idx = torch.zeros(1, dtype=torch.int64, device=s.device)
+    n_steps_t = torch.tensor([w.steps], dtype=torch.int64, device=s.device)
+
+    def step_body(buf):
+        s.fill()
+        s.apply(buf)
+        torch.index_select(traj, 0, step_idx, out=s.tokens.view(1, n))
+        s.accept_device(s.tokens)
+        step_idx.add_(1)
+        step_idx.remainder_(n_steps_t)
+
+    for k in range(ring_n):              # eager warm-up of every call before capture (first-use set-up)
+        step_body(ring[k])
+    torch.cuda.synchronize()
+    restart()
+    graphs = []
+    for k in range(ring_n):
+        gph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gph):
+            step_body(ring[k])
+        graphs.append(gph)
+    torch.cuda.synchronize()
+    restart()
+
+    def one_step(i):
         t = i % w.steps
         if t == 0 and i > 0:
             restart()
-        buf = ring[i % ring_n]
-        if events is not None:
-            events[0].record()
-        s.fill()
-        if events is not None:
-            events[1].record()
-        s.apply(buf)
-        if events is not None:
-            events[2].record()
-        s.accept_device(traj[t])
+        graphs[i % ring_n].replay()
         for b in eos_at[t]:
             s.reset(b)
             launches["reset"] += 1
-        if events is not None:
-            events[3].record()
         launches["merge"] += 1; launches["check"] += 1; launches["apply"] += 1; launches["accept"] += 1
 
     # ---- pass A: the headline number (events only around the timed region) --------------------
@@ -224,20 +242,46 @@ def main():
     ms_total = dist_util.max_over_ranks(e0.elapsed_time(e1))
     us_per_step = 1e3 * ms_total / args.steps
     timed_launches = sum(launches.values())
-    # masked fraction of the last mask (context for the apply numbers)
-    zero_bits = n * s.V - int(np.unpackbits(s.mask_numpy().view(np.uint8)).sum())
 
-    # ---- pass B: per-kernel times, same steps, events between the calls ------------------------
+    # ---- pass B: per-kernel device times over the same steps -----------------------------------
+    # Eager calls with events between them.  A short spin kernel in front of every step lets the
+    # host queue the whole step before the GPU starts it, so the event intervals are device time
+    # (kernel + launch gap) rather than host issue time.
     restart()
-    for i in range(warmup):
-        one_step(i)
+    spin_cycles = int(2.0e5)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-    for k, i in enumerate(range(warmup, total)):
-        one_step(i, evs[k])
+    zero_bits_sum, mask_samples = 0, 0
+    for i in range(total):
+        t = i % w.steps
+        if t == 0 and i > 0:
+            restart()
+        buf = ring[i % ring_n]
+        ev = evs[i - warmup] if i >= warmup else None
+        torch.cuda._sleep(spin_cycles)
+        if ev:
+            ev[0].record()
+        s.fill()
+        if ev:
+            ev[1].record()
+        s.apply(buf)
+        if ev:
+            ev[2].record()
+        torch.index_select(traj, 0, step_idx, out=s.tokens.view(1, n))
+        s.accept_device(s.tokens)
+        if ev:
+            ev[3].record()
+        step_idx.add_(1)
+        step_idx.remainder_(n_steps_t)
+        for b in eos_at[t]:
+            s.reset(b)
+        if ev and (i - warmup) % 10 == 0:            # masked fraction, sampled (synchronises; outside the event intervals)
+            zero_bits_sum += n * s.V - int(np.unpackbits(s.mask_numpy().view(np.uint8)).sum())
+            mask_samples += 1
     torch.cuda.synchronize()
     t_fill = float(np.mean([e[0].elapsed_time(e[1]) for e in evs])) * 1e3
     t_apply = float(np.mean([e[1].elapsed_time(e[2]) for e in evs])) * 1e3
     t_accept = float(np.mean([e[2].elapsed_time(e[3]) for e in evs])) * 1e3
+    zero_bits = zero_bits_sum / max(mask_samples, 1)
 
     # apply's algorithmic bytes: the mask words read plus the masked logits written (allowed
     # logits are neither read nor written); and the conventional count (read + write everything)
@@ -284,7 +328,7 @@ def main():
         "metric": metric, "value": us_per_step, "unit": "us/step", "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": us_per_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "int32", "data": "synthetic",
-        "config": {"workload": args.workload, "batch": n, "global_batch": n * world, "vocab": s.V, "logits_dtype": w.dtype,
+        "config": {"workload": args.workload, "batch": n, "global_batch": n * world, "vocab": s.V, "logits_dtype": w.dtype, "launch": "CUDA graph per step (fill, apply, accept)",
                    "grammars": len(w.grammars), "l2": "logits ring of %d buffers (%.0f MB) > 2 x L2" % (ring_n, ring_n * bytes_one / 1e6),
                    "parallelism": "replicas x%d" % world},
         "clocks": clocks,

@@ -189,24 +189,25 @@ static xg_status_t upload_grammar(xg_grammar* g) {
   // one blob, sections 16-byte aligned
   size_t total = 0;
   auto reserve = [&](size_t bytes) { size_t at = total; total += (bytes + 15) & ~size_t(15); return at; };
-  std::vector<uint32_t> info(f.n_states);
-  for (int s = 0; s < f.n_states; ++s) info[s] = (uint32_t)f.state_rule[s] | (f.state_final[s] ? 0x80000000u : 0u);
-  size_t o_info = reserve(info.size() * 4), o_sb = reserve(f.scan_begin.size() * 4), o_so = reserve(f.scan_own_end.size() * 4),
-         o_sc = reserve(f.scan_class.size() * 4), o_st = reserve(f.scan_target.size() * 4), o_wb = reserve(f.wait_begin.size() * 4),
-         o_wr = reserve(f.wait_rule.size() * 4), o_wt = reserve(f.wait_target.size() * 4), o_gb = reserve(f.gather_begin.size() * 4),
+  std::vector<StateRec> recs(f.n_states);
+  for (int s = 0; s < f.n_states; ++s) {
+    StateRec& r = recs[s];
+    r.scan_begin = f.scan_begin[s]; r.scan_own_end = f.scan_own_end[s]; r.scan_end = f.scan_begin[s + 1];
+    r.wait_begin = f.wait_begin[s]; r.wait_end = f.wait_begin[s + 1];
+    r.gather_begin = f.gather_begin[s]; r.gather_end = f.gather_begin[s + 1];
+    r.info = (uint32_t)f.state_rule[s] | (f.state_final[s] ? 0x80000000u : 0u);
+  }
+  std::vector<uint2> scan(f.scan_class.size()), wait(f.wait_rule.size());
+  for (size_t e = 0; e < scan.size(); ++e) scan[e] = make_uint2(f.scan_class[e], f.scan_target[e]);
+  for (size_t e = 0; e < wait.size(); ++e) wait[e] = make_uint2(f.wait_rule[e], f.wait_target[e]);
+  size_t o_rec = reserve(recs.size() * sizeof(StateRec)), o_scan = reserve(scan.size() * sizeof(uint2)), o_wait = reserve(wait.size() * sizeof(uint2)),
          o_gs = reserve(f.gather_state.size() * 4), o_cb = reserve(f.class_bits.size() * 4),
          o_en = reserve((size_t)f.n_states * sizeof(EntryDev)), o_self = reserve(sizeof(GrammarDev));
   std::vector<uint8_t> host(total, 0);
   auto put = [&](size_t at, const void* src, size_t bytes) { if (bytes) std::memcpy(host.data() + at, src, bytes); };
-  put(o_info, info.data(), info.size() * 4);
-  put(o_sb, f.scan_begin.data(), f.scan_begin.size() * 4);
-  put(o_so, f.scan_own_end.data(), f.scan_own_end.size() * 4);
-  put(o_sc, f.scan_class.data(), f.scan_class.size() * 4);
-  put(o_st, f.scan_target.data(), f.scan_target.size() * 4);
-  put(o_wb, f.wait_begin.data(), f.wait_begin.size() * 4);
-  put(o_wr, f.wait_rule.data(), f.wait_rule.size() * 4);
-  put(o_wt, f.wait_target.data(), f.wait_target.size() * 4);
-  put(o_gb, f.gather_begin.data(), f.gather_begin.size() * 4);
+  put(o_rec, recs.data(), recs.size() * sizeof(StateRec));
+  put(o_scan, scan.data(), scan.size() * sizeof(uint2));
+  put(o_wait, wait.data(), wait.size() * sizeof(uint2));
   put(o_gs, f.gather_state.data(), f.gather_state.size() * 4);
   put(o_cb, f.class_bits.data(), f.class_bits.size() * 4);
   put(o_en, g->entries.data(), g->entries.size() * sizeof(EntryDev));
@@ -215,11 +216,10 @@ static xg_status_t upload_grammar(xg_grammar* g) {
   GrammarDev& v = g->host_view;
   v.n_states = f.n_states; v.n_rules = f.n_rules; v.n_classes = f.n_classes;
   v.root_rule = f.root_rule; v.root_nullable = f.root_nullable; v.root_start = f.rule_start[f.root_rule];
-  v.state_info = (const uint32_t*)(d + o_info);
-  v.scan_begin = (const int32_t*)(d + o_sb); v.scan_own_end = (const int32_t*)(d + o_so);
-  v.scan_class = (const uint32_t*)(d + o_sc); v.scan_target = (const uint32_t*)(d + o_st);
-  v.wait_begin = (const int32_t*)(d + o_wb); v.wait_rule = (const uint32_t*)(d + o_wr); v.wait_target = (const uint32_t*)(d + o_wt);
-  v.gather_begin = (const int32_t*)(d + o_gb); v.gather_state = (const int32_t*)(d + o_gs);
+  v.state = (const StateRec*)(d + o_rec);
+  v.scan_edge = (const uint2*)(d + o_scan);
+  v.wait_edge = (const uint2*)(d + o_wait);
+  v.gather_state = (const int32_t*)(d + o_gs);
   v.class_bits = (const uint32_t*)(d + o_cb);
   v.entries = (const EntryDev*)(d + o_en);
   put(o_self, &v, sizeof(GrammarDev));
@@ -677,13 +677,18 @@ xg_status_t xg_apply_token_bitmask(void* logits_dev, xg_dtype_t dtype, int32_t b
     return set_error(XG_ERR_INVALID_ARG, "bad shape or stride");
   const int rows = row_indices_dev ? n_rows : batch;
   if (rows == 0 && row_indices_dev) return XG_OK;
-  if (rows <= 0 || rows > 65535) return set_error(XG_ERR_INVALID_ARG, "row count must be in 1..65535");
+  if (rows <= 0) return set_error(XG_ERR_INVALID_ARG, "no rows");
   const int elt = dtype == XG_BF16 ? 2 : 4;
   if (((uintptr_t)logits_dev & 15) || ((logits_row_stride_elems * elt) & 15))
     return set_error(XG_ERR_INVALID_ARG, "logits rows must start on 16-byte boundaries");
   const int elems = 16 / elt;
   const int n_vec = vocab_size / elems;
-  int bx = std::max(1, std::min((n_vec + 256 * 4 - 1) / (256 * 4), 65535));
+  // about eight blocks of 256 threads per SM in total (one full wave), split evenly over the rows
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int per_row_max = std::max(1, (n_vec + 255) / 256);
+  const int bx = std::max(1, std::min(per_row_max, (sms * 8 + rows / 2) / rows));
+  if (rows > 65535) return set_error(XG_ERR_INVALID_ARG, "more than 65535 rows");
   dim3 grid(bx, rows);
   if (dtype == XG_BF16)
     apply_kernel<8><<<grid, 256, 0, (cudaStream_t)stream>>>(logits_dev, vocab_size, (long long)logits_row_stride_elems, (const uint32_t*)bitmask_dev,

@@ -32,18 +32,21 @@ struct EntryDev {
   int32_t n_acc;
 };
 
+// Everything a walk needs to know about one automaton state, in one 32-byte record (two 16-byte
+// loads): the scan list [scan_begin, scan_end) with the state's own edges first
+// [scan_begin, scan_own_end), the wait list, the gather list, and rule id | (accepting << 31).
+struct __align__(16) StateRec {
+  int32_t scan_begin, scan_own_end, scan_end, wait_begin;
+  int32_t wait_end, gather_begin, gather_end;
+  uint32_t info;
+};
+
 struct GrammarDev {
   int32_t n_states, n_rules, n_classes;
   int32_t root_rule, root_nullable, root_start;
-  const uint32_t* state_info;     // [S] rule id | (accepting << 31)
-  const int32_t* scan_begin;      // [S+1]
-  const int32_t* scan_own_end;    // [S]   own edges are [scan_begin, scan_own_end)
-  const uint32_t* scan_class;
-  const uint32_t* scan_target;    // bit 31: origin = the set being scanned
-  const int32_t* wait_begin;      // [S+1]
-  const uint32_t* wait_rule;
-  const uint32_t* wait_target;    // bit 31: origin = the set the completed rule started in
-  const int32_t* gather_begin;    // [S+1]
+  const StateRec* state;          // [S]
+  const uint2* scan_edge;         // (byte class, target); target bit 31: origin = the set being scanned
+  const uint2* wait_edge;         // (awaited rule, target); target bit 31: origin = the set the rule started in
   const int32_t* gather_state;    // bit 31: a predicted start state (its items begin in the current set)
   const uint32_t* class_bits;     // [C][8]
   const EntryDev* entries;        // [S]; meaningful for scannable states

@@ -69,18 +69,21 @@ __device__ __forceinline__ bool advance_waiters(const GrammarDev& g, const Chart
   for (int i = b; i < e; ++i) {
     const uint32_t s2 = src_st[i];
     const int32_t o2 = src_org[i];
-    for (int w = g.wait_begin[s2]; w < g.wait_begin[s2 + 1]; ++w) {
-      if (g.wait_rule[w] != rule) continue;
-      const uint32_t t = g.wait_target[w];
-      if (!add_item(st, org, start, cnt, cap, t & ~kSelf, (t & kSelf) ? o : o2)) return false;
+    const int4 rec = *reinterpret_cast<const int4*>(&g.state[s2].scan_begin);          // .w = wait_begin
+    const int wait_end = g.state[s2].wait_end;
+    for (int w = rec.w; w < wait_end; ++w) {
+      const uint2 we = g.wait_edge[w];
+      if (we.x != rule) continue;
+      if (!add_item(st, org, start, cnt, cap, we.y & ~kSelf, (we.y & kSelf) ? o : o2)) return false;
     }
   }
   return true;
 }
 
+// class_bits may point to a shared-memory copy of g.class_bits
 template <typename LsbT>
-__device__ __forceinline__ int token_walk(const GrammarDev& g, const Chart& c, const uint8_t* __restrict__ bytes, int len, bool own_edges_first,
-                                          uint32_t* st, int32_t* org, int cap, LsbT* lsb, int* flags, uint32_t* exit_mask) {
+__device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* class_bits, const Chart& c, const uint8_t* __restrict__ bytes, int len,
+                                          bool own_edges_first, uint32_t* st, int32_t* org, int cap, LsbT* lsb, int* flags, uint32_t* exit_mask) {
   int cnt = 0;
   const uint32_t* cur_st = c.i_st;
   const int32_t* cur_org = c.i_org;
@@ -96,19 +99,19 @@ __device__ __forceinline__ int token_walk(const GrammarDev& g, const Chart& c, c
     for (int i = cur_b; i < cur_e; ++i) {
       const uint32_t s = cur_st[i];
       const int32_t o = cur_org[i];
-      const int e0 = g.scan_begin[s];
-      const int e1 = (k == 0 && own_edges_first) ? g.scan_own_end[s] : g.scan_begin[s + 1];
-      for (int e = e0; e < e1; ++e) {
-        if (g.class_bits[g.scan_class[e] * 8 + word] & bit) {
-          const uint32_t t = g.scan_target[e];
-          if (!add_item(st, org, start, cnt, cap, t & ~kSelf, (t & kSelf) ? self_idx : o)) { *flags |= kWalkOverflow; return k; }
+      const int4 rec = *reinterpret_cast<const int4*>(&g.state[s].scan_begin);   // scan_begin, scan_own_end, scan_end, wait_begin
+      const int e1 = (k == 0 && own_edges_first) ? rec.y : rec.z;
+      for (int e = rec.x; e < e1; ++e) {
+        const uint2 se = g.scan_edge[e];
+        if (class_bits[se.x * 8 + word] & bit) {
+          if (!add_item(st, org, start, cnt, cap, se.y & ~kSelf, (se.y & kSelf) ? self_idx : o)) { *flags |= kWalkOverflow; return k; }
         }
       }
     }
     if (cnt == start) return k;
     // complete (cascades through the growing set)
     for (int q = start; q < cnt; ++q) {
-      const uint32_t info = g.state_info[st[q]];
+      const uint32_t info = g.state[st[q]].info;
       if (!(info >> 31)) continue;
       const int32_t o = org[q];
       if (o < 0) {
@@ -123,6 +126,14 @@ __device__ __forceinline__ int token_walk(const GrammarDev& g, const Chart& c, c
   return len;
 }
 
+// byte-class bitsets staged in shared memory when they fit (the hottest table of a walk)
+constexpr int kSharedClasses = 256;
+__device__ __forceinline__ const uint32_t* stage_class_bits(const GrammarDev& g, uint32_t* sh) {
+  if (g.n_classes > kSharedClasses) return g.class_bits;
+  for (int i = threadIdx.x; i < g.n_classes * 8; i += blockDim.x) sh[i] = g.class_bits[i];
+  return sh;
+}
+
 // ------------------------------------------------------------------------------------------
 // Cache build (Section 3.4; appendix on the adaptive token mask cache): classify every
 // (scannable state, token) pair.  grid.y = position, grid.x * block = token rank (trie order).
@@ -135,8 +146,10 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
                 int2* __restrict__ overflow, int* __restrict__ overflow_count, int overflow_cap) {
   __shared__ uint32_t sh_st[1];
   __shared__ int32_t sh_org[1];
+  __shared__ uint32_t sh_class[kSharedClasses * 8];
   const int pos = blockIdx.y;
   if (threadIdx.x == 0) { sh_st[0] = (uint32_t)positions[pos]; sh_org[0] = -1; }
+  const uint32_t* class_bits = stage_class_bits(g, sh_class);
   __syncthreads();
   const int rank = blockIdx.x * blockDim.x + threadIdx.x;
   int cls = 0;
@@ -153,7 +166,7 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
       Chart c;
       c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1;
       c.i_st = sh_st; c.i_org = sh_org; c.i_cnt = 1; c.i_idx = 0;
-      consumed = token_walk<int16_t>(g, c, v.bytes + off, len, true, st, org, kFastCap, lsb, &flags, nullptr);
+      consumed = token_walk<int16_t>(g, class_bits, c, v.bytes + off, len, true, st, org, kFastCap, lsb, &flags, nullptr);
     }
     if (flags & kWalkOverflow) {
       int slot = atomicAdd(overflow_count, 1);
@@ -187,7 +200,7 @@ __global__ void classify_slow_kernel(GrammarDev g, VocabDev v, const int32_t* __
   const int len = (int)(v.offset[rank + 1] - off);
   if (len > kSlowMaxBytes) { atomicExch(failed, 1); return; }
   int flags = 0;
-  int consumed = token_walk<int32_t>(g, c, v.bytes + off, len, true, scratch_st + (size_t)i * kSlowCap,
+  int consumed = token_walk<int32_t>(g, g.class_bits, c, v.bytes + off, len, true, scratch_st + (size_t)i * kSlowCap,
                                      scratch_org + (size_t)i * kSlowCap, kSlowCap, scratch_lsb + (size_t)i * (kSlowMaxBytes + 2), &flags, nullptr);
   if (flags & kWalkOverflow) { atomicExch(failed, 1); return; }
   int cls = consumed == len ? 1 : ((flags & kWalkUncertain) ? 2 : 0);
@@ -321,9 +334,11 @@ __global__ void __launch_bounds__(256)
 exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, const EntryDev* __restrict__ entries) {
   __shared__ uint32_t sh_st[1];
   __shared__ int32_t sh_org[1];
+  __shared__ uint32_t sh_class[kSharedClasses * 8];
   const int p = blockIdx.x;
   const EntryDev e = entries[p];
   if (threadIdx.x == 0) { sh_st[0] = (uint32_t)positions[p]; sh_org[0] = -1; }
+  const uint32_t* class_bits = stage_class_bits(g, sh_class);
   __syncthreads();
   uint32_t* out = const_cast<uint32_t*>(e.unc_exit);
   for (int k = threadIdx.x; k < e.n_unc; k += blockDim.x) {
@@ -339,7 +354,7 @@ exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, con
       Chart c;
       c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1;
       c.i_st = sh_st; c.i_org = sh_org; c.i_cnt = 1; c.i_idx = 0;
-      token_walk<int16_t>(g, c, v.bytes + off, len, true, st, org, kFastCap, lsb, &flags, &mask);
+      token_walk<int16_t>(g, class_bits, c, v.bytes + off, len, true, st, org, kFastCap, lsb, &flags, &mask);
       if (flags & kWalkOverflow) mask = 0;
     }
     out[k] = mask;
@@ -367,7 +382,7 @@ __device__ __forceinline__ bool root_complete(const MatcherDev& m, const Grammar
   const int n = m.n_sets - 1;
   for (int i = m.set_begin[n]; i < m.set_begin[n + 1]; ++i) {
     if (m.item_origin[i] != 0) continue;
-    const uint32_t info = g.state_info[m.item_state[i]];
+    const uint32_t info = g.state[m.item_state[i]].info;
     if ((info >> 31) && (info & 0x7FFFFFFFu) == (uint32_t)g.root_rule) return true;
   }
   return false;
@@ -402,7 +417,7 @@ __global__ void accept_kernel(MatcherDev* const* __restrict__ matchers, int batc
         int flags = 0;
         const int room = min(m.cap_items - n_items, 32000);
         const Chart c = chart_of_history(m.item_state, m.item_origin, m.set_begin, n_sets - 1);
-        const int consumed = token_walk<int16_t>(g, c, v.bytes + off + done, piece, false, m.item_state + n_items, m.item_origin + n_items,
+        const int consumed = token_walk<int16_t>(g, g.class_bits, c, v.bytes + off + done, piece, false, m.item_state + n_items, m.item_origin + n_items,
                                                  room, lsb, &flags, nullptr);
         if (flags & kWalkOverflow) { st = -6; break; }
         if (consumed < piece) { st = -7; break; }
@@ -459,7 +474,8 @@ merge_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
     const int n = m.n_sets - 1;
     for (int i = m.set_begin[n]; i < m.set_begin[n + 1]; ++i) {
       const uint32_t s = m.item_state[i];
-      for (int gi = g.gather_begin[s]; gi < g.gather_begin[s + 1]; ++gi) {
+      const StateRec rec = g.state[s];
+      for (int gi = rec.gather_begin; gi < rec.gather_end; ++gi) {
         const EntryDev e = g.entries[g.gather_state[gi] & 0x7FFFFFFF];
         if (e.kind == 2) {
           for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] |= e.data[w0 + w];
@@ -524,13 +540,16 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
   const GrammarDev& g = *m.grammar;
   const int n = m.n_sets - 1;
   const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
+  __shared__ uint32_t sh_class[kSharedClasses * 8];
+  const uint32_t* class_bits = stage_class_bits(g, sh_class);
   if (threadIdx.x == 0) {
     int ne = 0, fail = 0;
     ent_cum[0] = 0;
     if (!m.terminated) {
       for (int i = 0; i < hist.i_cnt && !fail; ++i) {
         const uint32_t s = hist.i_st[i];
-        for (int gi = g.gather_begin[s]; gi < g.gather_begin[s + 1]; ++gi) {
+        const StateRec rec = g.state[s];
+        for (int gi = rec.gather_begin; gi < rec.gather_end; ++gi) {
           const int q = g.gather_state[gi] & 0x7FFFFFFF;
           const int origin = g.gather_state[gi] < 0 ? n : hist.i_org[i];     // predicted start states begin here
           bool seen = false;
@@ -555,17 +574,17 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
     int32_t* org = cont_org[e];
     int cnt = 0;
     int16_t no_local[2] = {0, 0};
-    bool ok = advance_waiters(g, hist, g.state_info[ent_state[e]] & 0x7FFFFFFFu, ent_origin[e], st, org, no_local, 0, cnt, kContCap);
+    bool ok = advance_waiters(g, hist, g.state[ent_state[e]].info & 0x7FFFFFFFu, ent_origin[e], st, org, no_local, 0, cnt, kContCap);
     for (int q = 0; ok && q < cnt; ++q) {
-      const uint32_t info = g.state_info[st[q]];
+      const uint32_t info = g.state[st[q]].info;
       if (info >> 31) ok = advance_waiters(g, hist, info & 0x7FFFFFFFu, org[q], st, org, no_local, 0, cnt, kContCap);
     }
     if (!ok) sh_fail = 1;
     cont_cnt[e] = ok ? cnt : 0;
     uint32_t first[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     for (int q = 0; q < cont_cnt[e]; ++q)
-      for (int x = g.scan_begin[st[q]]; x < g.scan_begin[st[q] + 1]; ++x) {
-        const uint32_t* cb = g.class_bits + g.scan_class[x] * 8;
+      for (int x = g.state[st[q]].scan_begin; x < g.state[st[q]].scan_end; ++x) {
+        const uint32_t* cb = class_bits + g.scan_edge[x].x * 8;
 #pragma unroll
         for (int w = 0; w < 8; ++w) first[w] |= cb[w];
       }
@@ -592,7 +611,7 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
         int32_t org[kFastCap];
         int16_t lsb[kFastMaxBytes + 2];
         int flags = 0;
-        pass = token_walk<int16_t>(g, hist, v.bytes + off, len, false, st, org, kFastCap, lsb, &flags, nullptr) == len;
+        pass = token_walk<int16_t>(g, class_bits, hist, v.bytes + off, len, false, st, org, kFastCap, lsb, &flags, nullptr) == len;
         overflow = (flags & kWalkOverflow) != 0;
       }
     } else {
@@ -607,7 +626,7 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
         int flags = 0;
         Chart c = hist;
         c.i_st = cont_st[e]; c.i_org = cont_org[e]; c.i_cnt = cont_cnt[e]; c.i_idx = n + at;
-        pass = token_walk<int16_t>(g, c, v.bytes + off + at, len - at, false, st, org, kFastCap, lsb, &flags, nullptr) == len - at;
+        pass = token_walk<int16_t>(g, class_bits, c, v.bytes + off + at, len - at, false, st, org, kFastCap, lsb, &flags, nullptr) == len - at;
         overflow = (flags & kWalkOverflow) != 0;
       }
     }
@@ -637,6 +656,27 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
 // (neither read nor written); one whose tokens are all disallowed is overwritten without being
 // read; only mixed vectors are read, blended and written back.
 // ------------------------------------------------------------------------------------------
+template <int ELEMS>
+__device__ __forceinline__ uint4 blend_ninf(uint4 x, uint32_t bits) {
+  if (ELEMS == 8) {
+    uint32_t p[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (!((bits >> (2 * k)) & 1u)) p[k] = (p[k] & 0xFFFF0000u) | 0xFF80u;
+      if (!((bits >> (2 * k + 1)) & 1u)) p[k] = (p[k] & 0x0000FFFFu) | 0xFF800000u;
+    }
+    return make_uint4(p[0], p[1], p[2], p[3]);
+  }
+  if (!(bits & 1u)) x.x = 0xFF800000u;
+  if (!(bits & 2u)) x.y = 0xFF800000u;
+  if (!(bits & 4u)) x.z = 0xFF800000u;
+  if (!(bits & 8u)) x.w = 0xFF800000u;
+  return x;
+}
+
+// grid = (blocks per row, rows).  Each thread handles four vectors per iteration: the four mask
+// tests first, then the loads of the mixed vectors (independent, all in flight together), then
+// the stores.
 template <int ELEMS>   // elements per 16-byte vector: 8 (bf16) or 4 (fp32)
 __global__ void __launch_bounds__(256)
 apply_kernel(void* __restrict__ logits, int vocab_size, long long row_stride_elems, const uint32_t* __restrict__ bitmask,
@@ -649,27 +689,24 @@ apply_kernel(void* __restrict__ logits, int vocab_size, long long row_stride_ele
                                 : make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
   uint4* base = ELEMS == 8 ? (uint4*)((uint16_t*)logits + (long long)r * row_stride_elems)
                            : (uint4*)((uint32_t*)logits + (long long)r * row_stride_elems);
-  for (int vi = blockIdx.x * blockDim.x + threadIdx.x; vi < n_vec; vi += gridDim.x * blockDim.x) {
-    const int first = vi * ELEMS;
-    const uint32_t bits = (__ldg(&mrow[first >> 5]) >> (first & 31)) & kAll;
-    if (bits == kAll) continue;
-    if (bits == 0) { base[vi] = ninf; continue; }
-    uint4 x = base[vi];
-    if (ELEMS == 8) {
-      uint32_t p[4] = {x.x, x.y, x.z, x.w};
+  const int stride = gridDim.x * blockDim.x;
+  for (int v0 = blockIdx.x * blockDim.x + threadIdx.x; v0 < n_vec; v0 += 4 * stride) {
+    uint32_t bits[4];
+    uint4 x[4];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        if (!((bits >> (2 * k)) & 1u)) p[k] = (p[k] & 0xFFFF0000u) | 0xFF80u;
-        if (!((bits >> (2 * k + 1)) & 1u)) p[k] = (p[k] & 0x0000FFFFu) | 0xFF800000u;
-      }
-      x = make_uint4(p[0], p[1], p[2], p[3]);
-    } else {
-      if (!(bits & 1u)) x.x = 0xFF800000u;
-      if (!(bits & 2u)) x.y = 0xFF800000u;
-      if (!(bits & 4u)) x.z = 0xFF800000u;
-      if (!(bits & 8u)) x.w = 0xFF800000u;
+    for (int u = 0; u < 4; ++u) {
+      const int vi = v0 + u * stride;
+      const int first = vi * ELEMS;
+      bits[u] = vi < n_vec ? ((__ldg(&mrow[first >> 5]) >> (first & 31)) & kAll) : kAll;
     }
-    base[vi] = x;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (bits[u] != kAll && bits[u] != 0) x[u] = base[v0 + u * stride];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (bits[u] == kAll) continue;
+      base[v0 + u * stride] = bits[u] == 0 ? ninf : blend_ninf<ELEMS>(x[u], bits[u]);
+    }
   }
   // ragged tail (vocab_size not a multiple of the vector width)
   if (blockIdx.x == 0) {
