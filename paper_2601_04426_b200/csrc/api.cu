@@ -189,17 +189,28 @@ static xg_status_t upload_grammar(xg_grammar* g) {
   // one blob, sections 16-byte aligned
   size_t total = 0;
   auto reserve = [&](size_t bytes) { size_t at = total; total += (bytes + 15) & ~size_t(15); return at; };
+  // classes of exactly one byte are encoded in place (no bitset lookup on the device)
+  std::vector<uint32_t> class_code(f.n_classes);
+  for (int c = 0; c < f.n_classes; ++c) {
+    int count = 0, byte = 0;
+    for (int b = 0; b < 256; ++b) if ((f.class_bits[(size_t)c * 8 + (b >> 5)] >> (b & 31)) & 1u) { ++count; byte = b; }
+    class_code[c] = count == 1 ? (kLiteral | (uint32_t)byte) : (uint32_t)c;
+  }
+  std::vector<uint2> scan(f.scan_class.size()), wait(f.wait_rule.size());
+  for (size_t e = 0; e < scan.size(); ++e) scan[e] = make_uint2(class_code[f.scan_class[e]], f.scan_target[e]);
+  for (size_t e = 0; e < wait.size(); ++e) wait[e] = make_uint2(f.wait_rule[e], f.wait_target[e]);
   std::vector<StateRec> recs(f.n_states);
   for (int s = 0; s < f.n_states; ++s) {
     StateRec& r = recs[s];
-    r.scan_begin = f.scan_begin[s]; r.scan_own_end = f.scan_own_end[s]; r.scan_end = f.scan_begin[s + 1];
-    r.wait_begin = f.wait_begin[s]; r.wait_end = f.wait_begin[s + 1];
-    r.gather_begin = f.gather_begin[s]; r.gather_end = f.gather_begin[s + 1];
+    const int n_own = f.scan_own_end[s] - f.scan_begin[s], n_scan = f.scan_begin[s + 1] - f.scan_begin[s];
+    const int n_wait = f.wait_begin[s + 1] - f.wait_begin[s], n_gather = f.gather_begin[s + 1] - f.gather_begin[s];
+    if (n_scan > 65535 || n_wait > 65535 || n_gather > 65535) return set_error(XG_ERR_CAPACITY, "a state predicts more than 65535 edges");
+    r.scan_begin = f.scan_begin[s]; r.n_own_n_scan = (uint32_t)n_own | ((uint32_t)n_scan << 16);
+    r.wait_begin = f.wait_begin[s]; r.n_wait_n_gather = (uint32_t)n_wait | ((uint32_t)n_gather << 16);
+    r.gather_begin = f.gather_begin[s];
     r.info = (uint32_t)f.state_rule[s] | (f.state_final[s] ? 0x80000000u : 0u);
+    r.edge0_class = n_scan ? scan[f.scan_begin[s]].x : 0; r.edge0_target = n_scan ? scan[f.scan_begin[s]].y : 0;
   }
-  std::vector<uint2> scan(f.scan_class.size()), wait(f.wait_rule.size());
-  for (size_t e = 0; e < scan.size(); ++e) scan[e] = make_uint2(f.scan_class[e], f.scan_target[e]);
-  for (size_t e = 0; e < wait.size(); ++e) wait[e] = make_uint2(f.wait_rule[e], f.wait_target[e]);
   size_t o_rec = reserve(recs.size() * sizeof(StateRec)), o_scan = reserve(scan.size() * sizeof(uint2)), o_wait = reserve(wait.size() * sizeof(uint2)),
          o_gs = reserve(f.gather_state.size() * 4), o_cb = reserve(f.class_bits.size() * 4),
          o_en = reserve((size_t)f.n_states * sizeof(EntryDev)), o_self = reserve(sizeof(GrammarDev));
@@ -663,7 +674,7 @@ xg_status_t xg_accept_token(xg_matcher_t* const* matchers, int32_t batch, const 
   xg_status_t st = batch_slot(matchers, batch, &tok, &slot);
   if (st != XG_OK) return st;
   if (!token_ids_dev) return set_error(XG_ERR_INVALID_ARG, "token_ids_dev is NULL");
-  accept_kernel<<<(batch + 31) / 32, 32, 0, (cudaStream_t)stream>>>(slot->dev_matchers, batch, tok->dev, token_ids_dev, status_dev);
+  accept_kernel<<<(batch + 3) / 4, 128, 0, (cudaStream_t)stream>>>(slot->dev_matchers, batch, tok->dev, token_ids_dev, status_dev);
   XG_CUDA(cudaGetLastError());
   return XG_OK;
 }

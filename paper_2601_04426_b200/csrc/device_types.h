@@ -33,13 +33,20 @@ struct EntryDev {
 };
 
 // Everything a walk needs to know about one automaton state, in one 32-byte record (two 16-byte
-// loads): the scan list [scan_begin, scan_end) with the state's own edges first
-// [scan_begin, scan_own_end), the wait list, the gather list, and rule id | (accepting << 31).
+// loads).  The scan list is scan_edge[scan_begin .. +n_scan) with the state's own edges first
+// (n_own of them); its first edge is repeated inline, so the long literal chains of a schema
+// grammar cost one load per byte.  A byte-class code is either a class id or, for a class of
+// exactly one byte, kLiteral | byte (no bitset lookup).
 struct __align__(16) StateRec {
-  int32_t scan_begin, scan_own_end, scan_end, wait_begin;
-  int32_t wait_end, gather_begin, gather_end;
-  uint32_t info;
+  int32_t scan_begin;
+  uint32_t n_own_n_scan;       // n_own | n_scan << 16
+  int32_t wait_begin;
+  uint32_t n_wait_n_gather;    // n_wait | n_gather << 16
+  int32_t gather_begin;
+  uint32_t info;               // rule id | accepting << 31
+  uint32_t edge0_class, edge0_target;
 };
+constexpr uint32_t kLiteral = 0x80000000u;
 
 struct GrammarDev {
   int32_t n_states, n_rules, n_classes;

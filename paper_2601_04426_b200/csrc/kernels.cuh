@@ -69,9 +69,9 @@ __device__ __forceinline__ bool advance_waiters(const GrammarDev& g, const Chart
   for (int i = b; i < e; ++i) {
     const uint32_t s2 = src_st[i];
     const int32_t o2 = src_org[i];
-    const int4 rec = *reinterpret_cast<const int4*>(&g.state[s2].scan_begin);          // .w = wait_begin
-    const int wait_end = g.state[s2].wait_end;
-    for (int w = rec.w; w < wait_end; ++w) {
+    const uint4 rec = *reinterpret_cast<const uint4*>(&g.state[s2]);
+    const int wait_end = (int)rec.z + (int)(rec.w & 0xFFFFu);
+    for (int w = (int)rec.z; w < wait_end; ++w) {
       const uint2 we = g.wait_edge[w];
       if (we.x != rule) continue;
       if (!add_item(st, org, start, cnt, cap, we.y & ~kSelf, (we.y & kSelf) ? o : o2)) return false;
@@ -99,13 +99,16 @@ __device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* c
     for (int i = cur_b; i < cur_e; ++i) {
       const uint32_t s = cur_st[i];
       const int32_t o = cur_org[i];
-      const int4 rec = *reinterpret_cast<const int4*>(&g.state[s].scan_begin);   // scan_begin, scan_own_end, scan_end, wait_begin
-      const int e1 = (k == 0 && own_edges_first) ? rec.y : rec.z;
-      for (int e = rec.x; e < e1; ++e) {
-        const uint2 se = g.scan_edge[e];
-        if (class_bits[se.x * 8 + word] & bit) {
-          if (!add_item(st, org, start, cnt, cap, se.y & ~kSelf, (se.y & kSelf) ? self_idx : o)) { *flags |= kWalkOverflow; return k; }
-        }
+      const uint4 ra = *reinterpret_cast<const uint4*>(&g.state[s]);
+      const int n_edges = (k == 0 && own_edges_first) ? (int)(ra.y & 0xFFFFu) : (int)(ra.y >> 16);
+      if (n_edges == 0) continue;
+      const uint4 rb = *(reinterpret_cast<const uint4*>(&g.state[s]) + 1);
+      uint2 se = make_uint2(rb.z, rb.w);                      // the first edge is inline
+      for (int e = 0;;) {
+        const bool hit = (se.x & kLiteral) ? ((se.x & 0xFFu) == byte) : ((class_bits[se.x * 8 + word] & bit) != 0);
+        if (hit && !add_item(st, org, start, cnt, cap, se.y & ~kSelf, (se.y & kSelf) ? self_idx : o)) { *flags |= kWalkOverflow; return k; }
+        if (++e >= n_edges) break;
+        se = g.scan_edge[(int)ra.x + e];
       }
     }
     if (cnt == start) return k;
@@ -388,20 +391,31 @@ __device__ __forceinline__ bool root_complete(const MatcherDev& m, const Grammar
   return false;
 }
 
-// Accept one sampled token per request (Section 2.2 "trace the output"): the walk writes its
-// sets straight behind the request's history; they are committed only if every byte survived.
-__global__ void accept_kernel(MatcherDev* const* __restrict__ matchers, int batch, VocabDev v,
-                              const int32_t* __restrict__ token_ids, int32_t* __restrict__ status) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+// Accept one sampled token per request (Section 2.2 "trace the output").  One warp per request:
+// requests follow unrelated paths, so sharing a warp between them would serialise their walks.
+// Lane 0 walks the token's bytes into local arrays; if every byte survived, the warp appends the
+// new sets behind the request's history and lane 0 commits the counters.
+__global__ void __launch_bounds__(128)
+accept_kernel(MatcherDev* const* __restrict__ matchers, int batch, VocabDev v,
+              const int32_t* __restrict__ token_ids, int32_t* __restrict__ status) {
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
   if (b >= batch) return;
   MatcherDev& m = *matchers[b];
   const GrammarDev& g = *m.grammar;
+  __shared__ uint32_t sh_st[4][kFastCap];
+  __shared__ int32_t sh_org[4][kFastCap];
+  __shared__ int16_t sh_lsb[4][kFastMaxBytes + 2];
+  uint32_t* w_st = sh_st[threadIdx.x >> 5];
+  int32_t* w_org = sh_org[threadIdx.x >> 5];
+  int16_t* lsb = sh_lsb[threadIdx.x >> 5];
   int st = 0;   // XG_OK
   const int tok = token_ids[b];
   if (m.terminated) st = -8;
   else if (tok < 0 || tok >= v.vocab_size) st = -7;
   else if (tok == v.eos_id) {
-    if (root_complete(m, g)) m.terminated = 1; else st = -7;
+    if (lane == 0) { if (root_complete(m, g)) m.terminated = 1; else st = -7; }
+    st = __shfl_sync(0xFFFFFFFFu, st, 0);
   } else {
     const int rank = v.id_to_rank[tok];
     const uint32_t off = v.offset[rank];
@@ -412,26 +426,33 @@ __global__ void accept_kernel(MatcherDev* const* __restrict__ matchers, int batc
       int done = 0;
       while (done < len && st == 0) {            // long tokens go through in pieces
         const int piece = min(len - done, kFastMaxBytes);
-        if (n_sets + piece > m.cap_sets) { st = -6; break; }
-        int16_t lsb[kFastMaxBytes + 2];
-        int flags = 0;
-        const int room = min(m.cap_items - n_items, 32000);
-        const Chart c = chart_of_history(m.item_state, m.item_origin, m.set_begin, n_sets - 1);
-        const int consumed = token_walk<int16_t>(g, g.class_bits, c, v.bytes + off + done, piece, false, m.item_state + n_items, m.item_origin + n_items,
-                                                 room, lsb, &flags, nullptr);
-        if (flags & kWalkOverflow) { st = -6; break; }
-        if (consumed < piece) { st = -7; break; }
+        int made = 0;
+        if (n_sets + piece > m.cap_sets) st = -6;
+        else if (lane == 0) {
+          int flags = 0;
+          const Chart c = chart_of_history(m.item_state, m.item_origin, m.set_begin, n_sets - 1);
+          const int consumed = token_walk<int16_t>(g, g.class_bits, c, v.bytes + off + done, piece, false, w_st, w_org, kFastCap, lsb, &flags, nullptr);
+          if (flags & kWalkOverflow) st = -6;
+          else if (consumed < piece) st = -7;
+          else { made = lsb[piece + 1]; if (n_items + made > m.cap_items) st = -6; }
+        }
+        st = __shfl_sync(0xFFFFFFFFu, st, 0);
+        made = __shfl_sync(0xFFFFFFFFu, made, 0);
+        if (st != 0) break;
+        __syncwarp();
         // origins written by the walk are already chart indices (its base is set n_sets - 1);
-        // publish the boundaries of the new sets
-        for (int j = 1; j <= piece; ++j) m.set_begin[n_sets + j] = n_items + lsb[j + 1];
-        n_items += lsb[piece + 1];
+        // append the new sets behind the history (visible to the next piece; committed below)
+        for (int q = lane; q < made; q += 32) { m.item_state[n_items + q] = w_st[q]; m.item_origin[n_items + q] = w_org[q]; }
+        for (int j = 1 + lane; j <= piece; j += 32) m.set_begin[n_sets + j] = n_items + lsb[j + 1];
+        __syncwarp();
+        n_items += made;
         n_sets += piece;
         done += piece;
       }
-      if (st == 0) { m.n_sets = n_sets; m.n_items = n_items; }
+      if (st == 0 && lane == 0) { m.n_sets = n_sets; m.n_items = n_items; }
     }
   }
-  if (status) status[b] = st;
+  if (status && lane == 0) status[b] = st;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -475,7 +496,7 @@ merge_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
     for (int i = m.set_begin[n]; i < m.set_begin[n + 1]; ++i) {
       const uint32_t s = m.item_state[i];
       const StateRec rec = g.state[s];
-      for (int gi = rec.gather_begin; gi < rec.gather_end; ++gi) {
+      for (int gi = rec.gather_begin; gi < rec.gather_begin + (int)(rec.n_wait_n_gather >> 16); ++gi) {
         const EntryDev e = g.entries[g.gather_state[gi] & 0x7FFFFFFF];
         if (e.kind == 2) {
           for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] |= e.data[w0 + w];
@@ -549,7 +570,7 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
       for (int i = 0; i < hist.i_cnt && !fail; ++i) {
         const uint32_t s = hist.i_st[i];
         const StateRec rec = g.state[s];
-        for (int gi = rec.gather_begin; gi < rec.gather_end; ++gi) {
+        for (int gi = rec.gather_begin; gi < rec.gather_begin + (int)(rec.n_wait_n_gather >> 16); ++gi) {
           const int q = g.gather_state[gi] & 0x7FFFFFFF;
           const int origin = g.gather_state[gi] < 0 ? n : hist.i_org[i];     // predicted start states begin here
           bool seen = false;
@@ -568,8 +589,8 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
   }
   __syncthreads();
   // continuation set of every entry: complete rule(q) started at its origin, with cascades
-  if ((int)threadIdx.x < n_ent) {
-    const int e = threadIdx.x;
+  for (int e = threadIdx.x >> 5; e < n_ent; e += blockDim.x >> 5) {     // one warp per entry: their chains differ
+    if (threadIdx.x & 31) continue;
     uint32_t* st = cont_st[e];
     int32_t* org = cont_org[e];
     int cnt = 0;
@@ -583,8 +604,10 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
     cont_cnt[e] = ok ? cnt : 0;
     uint32_t first[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     for (int q = 0; q < cont_cnt[e]; ++q)
-      for (int x = g.state[st[q]].scan_begin; x < g.state[st[q]].scan_end; ++x) {
-        const uint32_t* cb = class_bits + g.scan_edge[x].x * 8;
+      for (int x = g.state[st[q]].scan_begin; x < g.state[st[q]].scan_begin + (int)(g.state[st[q]].n_own_n_scan >> 16); ++x) {
+        const uint32_t code = g.scan_edge[x].x;
+        if (code & kLiteral) { first[(code & 0xFFu) >> 5] |= 1u << (code & 31u); continue; }
+        const uint32_t* cb = class_bits + code * 8;
 #pragma unroll
         for (int w = 0; w < 8; ++w) first[w] |= cb[w];
       }
@@ -594,44 +617,71 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
   __syncthreads();
   const int total = ent_cum[n_ent];
   uint32_t* row = (uint32_t*)bitmask + (long long)b * row_stride;
-  for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < total; j += gridDim.x * blockDim.x) {
-    int e = 0;
-    while (j >= ent_cum[e + 1]) ++e;
-    const int k = j - ent_cum[e];
-    const int rank = (int)ent_rank[e][k];
-    uint32_t exits = ent_exit[e][k];
-    const uint32_t off = v.offset[rank];
-    const int len = (int)(v.offset[rank + 1] - off);
-    bool pass = false, overflow = false;
-    if (exits == 0) {
-      // no exit record (very long token, or its walk overflowed at build time): walk in full
-      if (len > kFastMaxBytes) overflow = true;
-      else {
-        uint32_t st[kFastCap];
-        int32_t org[kFastCap];
-        int16_t lsb[kFastMaxBytes + 2];
-        int flags = 0;
-        pass = token_walk<int16_t>(g, class_bits, hist, v.bytes + off, len, false, st, org, kFastCap, lsb, &flags, nullptr) == len;
-        overflow = (flags & kWalkOverflow) != 0;
-      }
-    } else {
-      while (exits && !pass && !overflow) {
-        const int at = __ffs(exits) - 1;
-        exits &= exits - 1;
-        const uint32_t byte = v.bytes[off + at];
-        if (!((cont_first[e][byte >> 5] >> (byte & 31)) & 1u)) continue;
-        uint32_t st[kFastCap];
-        int32_t org[kFastCap];
-        int16_t lsb[kFastMaxBytes + 2];
-        int flags = 0;
-        Chart c = hist;
-        c.i_st = cont_st[e]; c.i_org = cont_org[e]; c.i_cnt = cont_cnt[e]; c.i_idx = n + at;
-        pass = token_walk<int16_t>(g, class_bits, c, v.bytes + off + at, len - at, false, st, org, kFastCap, lsb, &flags, nullptr) == len - at;
-        overflow = (flags & kWalkOverflow) != 0;
+  const int stride = gridDim.x * blockDim.x;
+  constexpr int kUnroll = 4;
+  for (int j0 = blockIdx.x * blockDim.x + threadIdx.x; j0 < total; j0 += kUnroll * stride) {
+    // filter phase: four candidates per thread with their loads in flight together; nearly all
+    // of them end here, on the first-byte test of their (usually single) exit
+    int ent[kUnroll], rank[kUnroll];
+    uint32_t exits[kUnroll], off[kUnroll], nxt[kUnroll], byte0[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int j = j0 + u * stride;
+      rank[u] = -1;
+      exits[u] = 0;
+      if (j < total) {
+        int e = 0;
+        while (j >= ent_cum[e + 1]) ++e;
+        ent[u] = e;
+        rank[u] = (int)ent_rank[e][j - ent_cum[e]];
+        exits[u] = ent_exit[e][j - ent_cum[e]];
       }
     }
-    if (overflow) sh_fail = 1;
-    else if (pass) { const int id = v.rank_to_id[rank]; atomicOr(&row[id >> 5], 1u << (id & 31)); }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u)
+      if (rank[u] >= 0) { off[u] = v.offset[rank[u]]; nxt[u] = v.offset[rank[u] + 1]; }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u)
+      if (rank[u] >= 0 && exits[u]) byte0[u] = v.bytes[off[u] + __ffs(exits[u]) - 1];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      if (rank[u] < 0) continue;
+      const int e = ent[u];
+      const int len = (int)(nxt[u] - off[u]);
+      bool pass = false, overflow = false;
+      if (exits[u] == 0) {
+        // no exit record (very long token, or its walk overflowed at build time): walk in full
+        if (len > kFastMaxBytes) overflow = true;
+        else {
+          uint32_t st[kFastCap];
+          int32_t org[kFastCap];
+          int16_t lsb[kFastMaxBytes + 2];
+          int flags = 0;
+          pass = token_walk<int16_t>(g, class_bits, hist, v.bytes + off[u], len, false, st, org, kFastCap, lsb, &flags, nullptr) == len;
+          overflow = (flags & kWalkOverflow) != 0;
+        }
+      } else {
+        uint32_t left = exits[u];
+        bool first = true;
+        while (left && !pass && !overflow) {
+          const int at = __ffs(left) - 1;
+          left &= left - 1;
+          const uint32_t byte = first ? byte0[u] : v.bytes[off[u] + at];
+          first = false;
+          if (!((cont_first[e][byte >> 5] >> (byte & 31)) & 1u)) continue;
+          uint32_t st[kFastCap];
+          int32_t org[kFastCap];
+          int16_t lsb[kFastMaxBytes + 2];
+          int flags = 0;
+          Chart c = hist;
+          c.i_st = cont_st[e]; c.i_org = cont_org[e]; c.i_cnt = cont_cnt[e]; c.i_idx = n + at;
+          pass = token_walk<int16_t>(g, class_bits, c, v.bytes + off[u] + at, len - at, false, st, org, kFastCap, lsb, &flags, nullptr) == len - at;
+          overflow = (flags & kWalkOverflow) != 0;
+        }
+      }
+      if (overflow) sh_fail = 1;
+      else if (pass) { const int id = v.rank_to_id[rank[u]]; atomicOr(&row[id >> 5], 1u << (id & 31)); }
+    }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
