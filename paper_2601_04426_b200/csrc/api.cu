@@ -506,7 +506,8 @@ xg_status_t xg_matcher_create(const xg_grammar_t* g, const xg_matcher_options_t*
   if (max_items <= 0) max_items = 4 * max_sets;
   std::unique_ptr<xg_matcher> m(new xg_matcher());
   m->grammar = g;
-  const size_t o_items = 256, o_org = o_items + (size_t)max_items * 4, o_sb = o_org + (size_t)max_items * 4;
+  const size_t o_plan = 256, o_items = o_plan + ((sizeof(StepPlan) + 255) & ~size_t(255)), o_org = o_items + (size_t)max_items * 4,
+               o_sb = o_org + (size_t)max_items * 4;
   const size_t total = o_sb + ((size_t)max_sets + 1) * 4;
   XG_CUDA(cudaMalloc(&m->block, total));
   uint8_t* d = (uint8_t*)m->block;
@@ -516,6 +517,7 @@ xg_status_t xg_matcher_create(const xg_grammar_t* g, const xg_matcher_options_t*
   h.item_origin = (int32_t*)(d + o_org);
   h.set_begin = (int32_t*)(d + o_sb);
   h.cap_sets = max_sets; h.cap_items = max_items;
+  h.plan = (StepPlan*)(d + o_plan);
   m->dev = (MatcherDev*)d;
   cudaError_t err = cudaMemcpyAsync(m->dev, &h, sizeof h, cudaMemcpyHostToDevice, (cudaStream_t)stream);
   if (err == cudaSuccess) { matcher_reset_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(m->dev); err = cudaGetLastError(); }

@@ -59,6 +59,28 @@ struct GrammarDev {
   const EntryDev* entries;        // [S]; meaningful for scannable states
 };
 
+// What the next mask needs from the current Earley set, worked out once when the set is made
+// (by accept or reset) instead of by every block of the fill kernels:
+//   * the cache entries to merge (scannable states of the set, predicted ones included);
+//   * the entries that have uncertain tokens, as (state, origin) pairs, with for each the
+//     continuation set -- what the chart looks like right after that state's rule completes --
+//     and the bytes that set can scan;
+//   * whether EOS is allowed.
+constexpr int kPlanMergeMax = 64;
+constexpr int kPlanCheckMax = 32;
+constexpr int kContCap = 16;
+struct StepPlan {
+  int32_t n_merge, n_check, eos_ok, overflow;
+  int32_t merge_state[kPlanMergeMax];
+  int32_t check_state[kPlanCheckMax];
+  int32_t check_origin[kPlanCheckMax];
+  int32_t check_cum[kPlanCheckMax + 1];      // running totals of uncertain tokens
+  int32_t cont_cnt[kPlanCheckMax];
+  uint32_t cont_first[kPlanCheckMax][8];
+  uint32_t cont_st[kPlanCheckMax][kContCap];
+  int32_t cont_org[kPlanCheckMax][kContCap];
+};
+
 // One request's Earley chart.  Only "kernel" items (made by scan or complete) are stored; the
 // predicted items of a set are implied by the grammar's per-state lists.
 struct MatcherDev {
@@ -70,6 +92,7 @@ struct MatcherDev {
   int32_t cap_sets, cap_items;
   int32_t terminated;
   int32_t pad;
+  StepPlan* plan;
 };
 
 constexpr uint32_t kSelf = 0x80000000u;

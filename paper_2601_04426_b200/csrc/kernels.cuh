@@ -367,18 +367,6 @@ exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, con
 // ------------------------------------------------------------------------------------------
 // matcher state
 // ------------------------------------------------------------------------------------------
-__global__ void matcher_reset_kernel(MatcherDev* m) {
-  if (threadIdx.x == 0 && blockIdx.x == 0) {
-    m->item_state[0] = (uint32_t)m->grammar->root_start;
-    m->item_origin[0] = 0;
-    m->set_begin[0] = 0;
-    m->set_begin[1] = 1;
-    m->n_sets = 1;
-    m->n_items = 1;
-    m->terminated = 0;
-  }
-}
-
 // is the root rule complete in the current set (EOS allowed)?
 __device__ __forceinline__ bool root_complete(const MatcherDev& m, const GrammarDev& g) {
   if (m.n_sets == 1 && g.root_nullable) return true;
@@ -389,6 +377,88 @@ __device__ __forceinline__ bool root_complete(const MatcherDev& m, const Grammar
     if ((info >> 31) && (info & 0x7FFFFFFFu) == (uint32_t)g.root_rule) return true;
   }
   return false;
+}
+
+// Build the step plan of the request's current set.  One warp: lane 0 lists the entries, then
+// one lane per entry completes that entry's rule into its continuation set.
+__device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g, int lane) {
+  StepPlan& p = *m.plan;
+  const int n = m.n_sets - 1;
+  const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
+  int n_check = 0;
+  if (lane == 0) {
+    int n_merge = 0, overflow = 0;
+    p.check_cum[0] = 0;
+    for (int i = 0; i < hist.i_cnt && !overflow; ++i) {
+      const uint32_t s = hist.i_st[i];
+      const StateRec rec = g.state[s];
+      for (int gi = rec.gather_begin; gi < rec.gather_begin + (int)(rec.n_wait_n_gather >> 16); ++gi) {
+        const int code = g.gather_state[gi];
+        const int q = code & 0x7FFFFFFF;
+        const int origin = code < 0 ? n : hist.i_org[i];          // predicted start states begin here
+        bool seen = false;
+        for (int z = 0; z < n_merge; ++z) seen = seen || p.merge_state[z] == q;
+        if (!seen) { if (n_merge == kPlanMergeMax) { overflow = 1; break; } p.merge_state[n_merge++] = q; }
+        const int n_unc = g.entries[q].n_unc;
+        if (n_unc == 0) continue;
+        seen = false;
+        for (int z = 0; z < n_check; ++z) seen = seen || (p.check_state[z] == q && p.check_origin[z] == origin);
+        if (seen) continue;
+        if (n_check == kPlanCheckMax) { overflow = 1; break; }
+        p.check_state[n_check] = q; p.check_origin[n_check] = origin;
+        p.check_cum[n_check + 1] = p.check_cum[n_check] + n_unc;
+        ++n_check;
+      }
+    }
+    p.n_merge = n_merge; p.n_check = n_check; p.overflow = overflow;
+    p.eos_ok = root_complete(m, g) ? 1 : 0;
+  }
+  n_check = __shfl_sync(0xFFFFFFFFu, n_check, 0);
+  __syncwarp();
+  // continuation set of every entry: complete rule(q) started at its origin, with cascades
+  bool bad = false;
+  for (int e = lane; e < n_check; e += 32) {
+    uint32_t* st = p.cont_st[e];
+    int32_t* org = p.cont_org[e];
+    int cnt = 0;
+    int16_t no_local[2] = {0, 0};
+    bool ok = advance_waiters(g, hist, g.state[p.check_state[e]].info & 0x7FFFFFFFu, p.check_origin[e], st, org, no_local, 0, cnt, kContCap);
+    for (int q = 0; ok && q < cnt; ++q) {
+      const uint32_t info = g.state[st[q]].info;
+      if (info >> 31) ok = advance_waiters(g, hist, info & 0x7FFFFFFFu, org[q], st, org, no_local, 0, cnt, kContCap);
+    }
+    if (!ok) { bad = true; cnt = 0; }
+    p.cont_cnt[e] = cnt;
+    uint32_t first[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int q = 0; q < cnt; ++q) {
+      const StateRec rec = g.state[st[q]];
+      for (int x = 0; x < (int)(rec.n_own_n_scan >> 16); ++x) {
+        const uint32_t code = x == 0 ? rec.edge0_class : g.scan_edge[rec.scan_begin + x].x;
+        if (code & kLiteral) { first[(code & 0xFFu) >> 5] |= 1u << (code & 31u); continue; }
+        const uint32_t* cb = g.class_bits + code * 8;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) first[w] |= cb[w];
+      }
+    }
+#pragma unroll
+    for (int w = 0; w < 8; ++w) p.cont_first[e][w] = first[w];
+  }
+  if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) p.overflow = 1;
+}
+
+__global__ void matcher_reset_kernel(MatcherDev* m) {      // one warp
+  if (blockIdx.x != 0 || threadIdx.x >= 32) return;
+  if (threadIdx.x == 0) {
+    m->item_state[0] = (uint32_t)m->grammar->root_start;
+    m->item_origin[0] = 0;
+    m->set_begin[0] = 0;
+    m->set_begin[1] = 1;
+    m->n_sets = 1;
+    m->n_items = 1;
+    m->terminated = 0;
+  }
+  __syncwarp();
+  prepare_plan(*m, *m->grammar, threadIdx.x);
 }
 
 // Accept one sampled token per request (Section 2.2 "trace the output").  One warp per request:
@@ -449,7 +519,11 @@ accept_kernel(MatcherDev* const* __restrict__ matchers, int batch, VocabDev v,
         n_sets += piece;
         done += piece;
       }
-      if (st == 0 && lane == 0) { m.n_sets = n_sets; m.n_items = n_items; }
+      if (st == 0) {
+        if (lane == 0) { m.n_sets = n_sets; m.n_items = n_items; }
+        __syncwarp();
+        prepare_plan(m, g, lane);      // the next mask's plan, while the new set is still hot
+      }
     }
   }
   if (status && lane == 0) status[b] = st;
@@ -482,43 +556,39 @@ merge_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
   const int w0 = blockIdx.x * chunk, w1 = min(v.n_words, w0 + chunk);
   const int nw = max(0, w1 - w0);
   for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] = 0;
-  const bool dead = m.terminated != 0;
+  const StepPlan& plan = *m.plan;
+  const int st0 = m.terminated ? -8 : (plan.overflow ? -6 : 0);
   if (blockIdx.x == 0 && threadIdx.x == 0) {
-    const int s = dead ? -8 : 0;
-    status[b] = s;
-    if (status_user) status_user[b] = s;
+    status[b] = st0;
+    if (status_user) status_user[b] = st0;
     done_count[b] = 0;
   }
   __syncthreads();
-  if (!dead && nw > 0) {
+  if (st0 == 0 && nw > 0) {
     const uint32_t id_lo = (uint32_t)w0 * 32u, id_hi = (uint32_t)w1 * 32u;
-    const int n = m.n_sets - 1;
-    for (int i = m.set_begin[n]; i < m.set_begin[n + 1]; ++i) {
-      const uint32_t s = m.item_state[i];
-      const StateRec rec = g.state[s];
-      for (int gi = rec.gather_begin; gi < rec.gather_begin + (int)(rec.n_wait_n_gather >> 16); ++gi) {
-        const EntryDev e = g.entries[g.gather_state[gi] & 0x7FFFFFFF];
-        if (e.kind == 2) {
-          for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] |= e.data[w0 + w];
-        } else if (e.kind == 0) {
-          const int lo = lower_bound_u32(e.data, e.n_list, id_lo), hi = lower_bound_u32(e.data, e.n_list, id_hi);
-          for (int k = lo + threadIdx.x; k < hi; k += blockDim.x) { const uint32_t id = e.data[k]; atomicOr(&row[(id >> 5) - w0], 1u << (id & 31)); }
-        } else {
-          // accepted = everything except the rejected and the uncertain tokens
-          const uint32_t tail = (v.vocab_size & 31) ? ((1u << (v.vocab_size & 31)) - 1) : 0xFFFFFFFFu;
-          for (int w = threadIdx.x; w < nw; w += blockDim.x) tmp[w] = (w0 + w == v.n_words - 1) ? tail : 0xFFFFFFFFu;
-          __syncthreads();
-          int lo = lower_bound_u32(e.data, e.n_list, id_lo), hi = lower_bound_u32(e.data, e.n_list, id_hi);
-          for (int k = lo + threadIdx.x; k < hi; k += blockDim.x) { const uint32_t id = e.data[k]; atomicAnd(&tmp[(id >> 5) - w0], ~(1u << (id & 31))); }
-          lo = lower_bound_u32(e.unc_id, e.n_unc, id_lo); hi = lower_bound_u32(e.unc_id, e.n_unc, id_hi);
-          for (int k = lo + threadIdx.x; k < hi; k += blockDim.x) { const uint32_t id = e.unc_id[k]; atomicAnd(&tmp[(id >> 5) - w0], ~(1u << (id & 31))); }
-          __syncthreads();
-          for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] |= tmp[w];
-        }
+    const int n_merge = plan.n_merge;
+    for (int k = 0; k < n_merge; ++k) {
+      const EntryDev e = g.entries[plan.merge_state[k]];
+      if (e.kind == 2) {
+        for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] |= e.data[w0 + w];
+      } else if (e.kind == 0) {
+        const int lo = lower_bound_u32(e.data, e.n_list, id_lo), hi = lower_bound_u32(e.data, e.n_list, id_hi);
+        for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) { const uint32_t id = e.data[i]; atomicOr(&row[(id >> 5) - w0], 1u << (id & 31)); }
+      } else {
+        // accepted = everything except the rejected and the uncertain tokens
+        const uint32_t tail = (v.vocab_size & 31) ? ((1u << (v.vocab_size & 31)) - 1) : 0xFFFFFFFFu;
+        for (int w = threadIdx.x; w < nw; w += blockDim.x) tmp[w] = (w0 + w == v.n_words - 1) ? tail : 0xFFFFFFFFu;
         __syncthreads();
+        int lo = lower_bound_u32(e.data, e.n_list, id_lo), hi = lower_bound_u32(e.data, e.n_list, id_hi);
+        for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) { const uint32_t id = e.data[i]; atomicAnd(&tmp[(id >> 5) - w0], ~(1u << (id & 31))); }
+        lo = lower_bound_u32(e.unc_id, e.n_unc, id_lo); hi = lower_bound_u32(e.unc_id, e.n_unc, id_hi);
+        for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) { const uint32_t id = e.unc_id[i]; atomicAnd(&tmp[(id >> 5) - w0], ~(1u << (id & 31))); }
+        __syncthreads();
+        for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] |= tmp[w];
       }
+      __syncthreads();
     }
-    if (threadIdx.x == 0 && v.eos_id >= 0 && (uint32_t)v.eos_id >= id_lo && (uint32_t)v.eos_id < id_hi && root_complete(m, g))
+    if (threadIdx.x == 0 && v.eos_id >= 0 && (uint32_t)v.eos_id >= id_lo && (uint32_t)v.eos_id < id_hi && plan.eos_ok)
       row[(v.eos_id >> 5) - w0] |= 1u << (v.eos_id & 31);
     __syncthreads();
   }
@@ -538,86 +608,47 @@ merge_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
 // Tokens are taken in trie order, one per lane, so neighbouring lanes share prefixes.
 // The last block of a request to finish clears the row if anything overflowed.
 // ------------------------------------------------------------------------------------------
-constexpr int kMaxStepEntries = 48;
-constexpr int kContCap = 16;
 
 __global__ void __launch_bounds__(256)
 check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __restrict__ bitmask, long long row_stride,
              int32_t* __restrict__ status_user, int32_t* __restrict__ status, int32_t* __restrict__ done_count) {
-  __shared__ const uint32_t* ent_rank[kMaxStepEntries];
-  __shared__ const uint32_t* ent_exit[kMaxStepEntries];
-  __shared__ int ent_cum[kMaxStepEntries + 1];
-  __shared__ int ent_state[kMaxStepEntries];
-  __shared__ int ent_origin[kMaxStepEntries];
-  __shared__ uint32_t cont_st[kMaxStepEntries][kContCap];
-  __shared__ int32_t cont_org[kMaxStepEntries][kContCap];
-  __shared__ int cont_cnt[kMaxStepEntries];
-  __shared__ uint32_t cont_first[kMaxStepEntries][8];
-  __shared__ int n_ent;
+  __shared__ const uint32_t* ent_rank[kPlanCheckMax];
+  __shared__ const uint32_t* ent_exit[kPlanCheckMax];
+  __shared__ int ent_cum[kPlanCheckMax + 1];
+  __shared__ uint32_t cont_st[kPlanCheckMax][kContCap];
+  __shared__ int32_t cont_org[kPlanCheckMax][kContCap];
+  __shared__ int cont_cnt[kPlanCheckMax];
+  __shared__ uint32_t cont_first[kPlanCheckMax][8];
+  __shared__ uint32_t sh_class[kSharedClasses * 8];
   __shared__ int sh_fail;
   __shared__ int sh_last;
   const int b = blockIdx.y;
   const MatcherDev& m = *matchers[b];
   const GrammarDev& g = *m.grammar;
+  const StepPlan& plan = *m.plan;
   const int n = m.n_sets - 1;
-  const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
-  __shared__ uint32_t sh_class[kSharedClasses * 8];
-  const uint32_t* class_bits = stage_class_bits(g, sh_class);
-  if (threadIdx.x == 0) {
-    int ne = 0, fail = 0;
-    ent_cum[0] = 0;
-    if (!m.terminated) {
-      for (int i = 0; i < hist.i_cnt && !fail; ++i) {
-        const uint32_t s = hist.i_st[i];
-        const StateRec rec = g.state[s];
-        for (int gi = rec.gather_begin; gi < rec.gather_begin + (int)(rec.n_wait_n_gather >> 16); ++gi) {
-          const int q = g.gather_state[gi] & 0x7FFFFFFF;
-          const int origin = g.gather_state[gi] < 0 ? n : hist.i_org[i];     // predicted start states begin here
-          bool seen = false;
-          for (int z = 0; z < ne; ++z) seen = seen || (ent_state[z] == q && ent_origin[z] == origin);
-          if (seen) continue;
-          const EntryDev& e = g.entries[q];
-          if (e.n_unc == 0) continue;
-          if (ne == kMaxStepEntries) { fail = 1; break; }
-          ent_state[ne] = q; ent_origin[ne] = origin; ent_rank[ne] = e.unc_rank; ent_exit[ne] = e.unc_exit;
-          ent_cum[ne + 1] = ent_cum[ne] + e.n_unc; ++ne;
-        }
-      }
-    }
-    n_ent = ne;
-    sh_fail = fail;
-  }
-  __syncthreads();
-  // continuation set of every entry: complete rule(q) started at its origin, with cascades
-  for (int e = threadIdx.x >> 5; e < n_ent; e += blockDim.x >> 5) {     // one warp per entry: their chains differ
-    if (threadIdx.x & 31) continue;
-    uint32_t* st = cont_st[e];
-    int32_t* org = cont_org[e];
-    int cnt = 0;
-    int16_t no_local[2] = {0, 0};
-    bool ok = advance_waiters(g, hist, g.state[ent_state[e]].info & 0x7FFFFFFFu, ent_origin[e], st, org, no_local, 0, cnt, kContCap);
-    for (int q = 0; ok && q < cnt; ++q) {
-      const uint32_t info = g.state[st[q]].info;
-      if (info >> 31) ok = advance_waiters(g, hist, info & 0x7FFFFFFFu, org[q], st, org, no_local, 0, cnt, kContCap);
-    }
-    if (!ok) sh_fail = 1;
-    cont_cnt[e] = ok ? cnt : 0;
-    uint32_t first[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    for (int q = 0; q < cont_cnt[e]; ++q)
-      for (int x = g.state[st[q]].scan_begin; x < g.state[st[q]].scan_begin + (int)(g.state[st[q]].n_own_n_scan >> 16); ++x) {
-        const uint32_t code = g.scan_edge[x].x;
-        if (code & kLiteral) { first[(code & 0xFFu) >> 5] |= 1u << (code & 31u); continue; }
-        const uint32_t* cb = class_bits + code * 8;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) first[w] |= cb[w];
-      }
-#pragma unroll
-    for (int w = 0; w < 8; ++w) cont_first[e][w] = first[w];
-  }
-  __syncthreads();
-  const int total = ent_cum[n_ent];
-  uint32_t* row = (uint32_t*)bitmask + (long long)b * row_stride;
+  const bool live = !m.terminated && !plan.overflow;
+  const int n_ent = live ? plan.n_check : 0;
+  const int total = n_ent ? plan.check_cum[n_ent] : 0;
   const int stride = gridDim.x * blockDim.x;
+  if (threadIdx.x == 0) sh_fail = 0;
+  if (blockIdx.x * (int)blockDim.x < total) {         // blocks without candidates only take part in the count below
+    const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
+    const uint32_t* class_bits = stage_class_bits(g, sh_class);
+    // the plan's arrays for the live entries, copied with coalesced loads
+    for (int i = threadIdx.x; i < n_ent; i += blockDim.x) {
+      const EntryDev& e = g.entries[plan.check_state[i]];
+      ent_rank[i] = e.unc_rank; ent_exit[i] = e.unc_exit;
+      cont_cnt[i] = plan.cont_cnt[i];
+    }
+    for (int i = threadIdx.x; i <= n_ent; i += blockDim.x) ent_cum[i] = plan.check_cum[i];
+    for (int i = threadIdx.x; i < n_ent * kContCap; i += blockDim.x) {
+      (&cont_st[0][0])[i] = (&plan.cont_st[0][0])[i];
+      (&cont_org[0][0])[i] = (&plan.cont_org[0][0])[i];
+    }
+    for (int i = threadIdx.x; i < n_ent * 8; i += blockDim.x) (&cont_first[0][0])[i] = (&plan.cont_first[0][0])[i];
+    __syncthreads();
+    uint32_t* row = (uint32_t*)bitmask + (long long)b * row_stride;
   constexpr int kUnroll = 4;
   for (int j0 = blockIdx.x * blockDim.x + threadIdx.x; j0 < total; j0 += kUnroll * stride) {
     // filter phase: four candidates per thread with their loads in flight together; nearly all
@@ -683,6 +714,7 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
       else if (pass) { const int id = v.rank_to_id[rank[u]]; atomicOr(&row[id >> 5], 1u << (id & 31)); }
     }
   }
+  }
   __syncthreads();
   if (threadIdx.x == 0) {
     if (sh_fail) atomicExch(&status[b], -6);
@@ -694,6 +726,7 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
     __threadfence();
     const int s = *(volatile int32_t*)&status[b];
     if (s == -6) {
+      uint32_t* row = (uint32_t*)bitmask + (long long)b * row_stride;
       for (int w = threadIdx.x; w < v.n_words; w += blockDim.x) row[w] = 0;
       if (threadIdx.x == 0 && status_user) status_user[b] = -6;
     }
