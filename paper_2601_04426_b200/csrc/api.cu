@@ -211,11 +211,17 @@ static xg_status_t upload_grammar(xg_grammar* g) {
     r.info = (uint32_t)f.state_rule[s] | (f.state_final[s] ? 0x80000000u : 0u);
     r.edge0_class = n_scan ? scan[f.scan_begin[s]].x : 0; r.edge0_target = n_scan ? scan[f.scan_begin[s]].y : 0;
   }
+  std::vector<uint32_t> state_first((size_t)f.n_states * 8, 0);
+  for (int s = 0; s < f.n_states; ++s)
+    for (int e = f.scan_begin[s]; e < f.scan_begin[s + 1]; ++e)
+      for (int w = 0; w < 8; ++w) state_first[(size_t)s * 8 + w] |= f.class_bits[(size_t)f.scan_class[e] * 8 + w];
+  size_t o_first = reserve(state_first.size() * 4);
   size_t o_rec = reserve(recs.size() * sizeof(StateRec)), o_scan = reserve(scan.size() * sizeof(uint2)), o_wait = reserve(wait.size() * sizeof(uint2)),
          o_gs = reserve(f.gather_state.size() * 4), o_cb = reserve(f.class_bits.size() * 4),
          o_en = reserve((size_t)f.n_states * sizeof(EntryDev)), o_self = reserve(sizeof(GrammarDev));
   std::vector<uint8_t> host(total, 0);
   auto put = [&](size_t at, const void* src, size_t bytes) { if (bytes) std::memcpy(host.data() + at, src, bytes); };
+  put(o_first, state_first.data(), state_first.size() * 4);
   put(o_rec, recs.data(), recs.size() * sizeof(StateRec));
   put(o_scan, scan.data(), scan.size() * sizeof(uint2));
   put(o_wait, wait.data(), wait.size() * sizeof(uint2));
@@ -232,6 +238,7 @@ static xg_status_t upload_grammar(xg_grammar* g) {
   v.wait_edge = (const uint2*)(d + o_wait);
   v.gather_state = (const int32_t*)(d + o_gs);
   v.class_bits = (const uint32_t*)(d + o_cb);
+  v.state_first = (const uint32_t*)(d + o_first);
   v.entries = (const EntryDev*)(d + o_en);
   put(o_self, &v, sizeof(GrammarDev));
   g->dev = (GrammarDev*)(d + o_self);

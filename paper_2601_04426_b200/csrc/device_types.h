@@ -1,5 +1,6 @@
 // Plain structs shared by host code and kernels (all pointers are device pointers).
 #pragma once
+#include <cstddef>
 #include <cstdint>
 
 namespace xg {
@@ -56,6 +57,7 @@ struct GrammarDev {
   const uint2* wait_edge;         // (awaited rule, target); target bit 31: origin = the set the rule started in
   const int32_t* gather_state;    // bit 31: a predicted start state (its items begin in the current set)
   const uint32_t* class_bits;     // [C][8]
+  const uint32_t* state_first;    // [S][8] bytes that the state's scan list (own and predicted edges) can take
   const EntryDev* entries;        // [S]; meaningful for scannable states
 };
 
@@ -69,17 +71,18 @@ struct GrammarDev {
 constexpr int kPlanMergeMax = 64;
 constexpr int kPlanCheckMax = 32;
 constexpr int kContCap = 16;
-struct StepPlan {
+struct __align__(16) StepPlan {
   int32_t n_merge, n_check, eos_ok, overflow;
+  uint32_t cont_first[kPlanCheckMax][8];     // read and written as 16-byte vectors: keep 16-byte aligned
+  uint32_t cont_st[kPlanCheckMax][kContCap];
+  int32_t cont_org[kPlanCheckMax][kContCap];
   int32_t merge_state[kPlanMergeMax];
   int32_t check_state[kPlanCheckMax];
   int32_t check_origin[kPlanCheckMax];
-  int32_t check_cum[kPlanCheckMax + 1];      // running totals of uncertain tokens
   int32_t cont_cnt[kPlanCheckMax];
-  uint32_t cont_first[kPlanCheckMax][8];
-  uint32_t cont_st[kPlanCheckMax][kContCap];
-  int32_t cont_org[kPlanCheckMax][kContCap];
+  int32_t check_cum[kPlanCheckMax + 1];      // running totals of uncertain tokens
 };
+static_assert(offsetof(StepPlan, cont_first) % 16 == 0, "cont_first must be 16-byte aligned");
 
 // One request's Earley chart.  Only "kernel" items (made by scan or complete) are stored; the
 // predicted items of a set are implied by the grammar's per-state lists.

@@ -429,19 +429,15 @@ __device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g,
     }
     if (!ok) { bad = true; cnt = 0; }
     p.cont_cnt[e] = cnt;
-    uint32_t first[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    uint4 fa = make_uint4(0, 0, 0, 0), fb = make_uint4(0, 0, 0, 0);
     for (int q = 0; q < cnt; ++q) {
-      const StateRec rec = g.state[st[q]];
-      for (int x = 0; x < (int)(rec.n_own_n_scan >> 16); ++x) {
-        const uint32_t code = x == 0 ? rec.edge0_class : g.scan_edge[rec.scan_begin + x].x;
-        if (code & kLiteral) { first[(code & 0xFFu) >> 5] |= 1u << (code & 31u); continue; }
-        const uint32_t* cb = g.class_bits + code * 8;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) first[w] |= cb[w];
-      }
+      const uint4* sf = reinterpret_cast<const uint4*>(g.state_first + (size_t)st[q] * 8);
+      const uint4 a = sf[0], c = sf[1];
+      fa.x |= a.x; fa.y |= a.y; fa.z |= a.z; fa.w |= a.w;
+      fb.x |= c.x; fb.y |= c.y; fb.z |= c.z; fb.w |= c.w;
     }
-#pragma unroll
-    for (int w = 0; w < 8; ++w) p.cont_first[e][w] = first[w];
+    uint4* out = reinterpret_cast<uint4*>(p.cont_first[e]);
+    out[0] = fa; out[1] = fb;
   }
   if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) p.overflow = 1;
 }
