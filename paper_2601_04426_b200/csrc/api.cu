@@ -429,7 +429,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     g->stats.total_uncertain += c.y;
     g->stats.total_rejected += tok->vocab_size - c.x - c.y;
     g->stats.kind_count[e.kind]++;
-    g->stats.cache_bytes += 4LL * ((e.kind == 2 ? tok->n_words : e.n_list) + 3LL * e.n_unc);
+    g->stats.cache_bytes += 4LL * ((e.kind == 2 ? tok->n_words : e.n_list) + 3LL * e.n_unc + (e.n_unc + 3) / 4);
   }
   *out = g.release();
   return XG_OK;
@@ -607,6 +607,13 @@ xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t ba
   if (st != XG_OK) return st;
   if (!bitmask_dev || row_stride_words < tok->n_words) return set_error(XG_ERR_INVALID_ARG, "bad bitmask buffer");
   const int W = tok->n_words;
+  if ((W + kClusterBlocks - 1) / kClusterBlocks <= kMergeMaxChunkWords) {
+    // one launch: a cluster of eight blocks per request keeps the row in distributed shared memory
+    fill_cluster_kernel<<<dim3(kClusterBlocks, batch), 256, 0, (cudaStream_t)stream>>>(slot->dev_matchers, tok->dev, bitmask_dev,
+                                                                                      (long long)row_stride_words, status_dev);
+    XG_CUDA(cudaGetLastError());
+    return XG_OK;
+  }
   int chunks = std::max((W + kMergeMaxChunkWords - 1) / kMergeMaxChunkWords, std::min(8, (W + 127) / 128));
   dim3 grid_merge(chunks, batch);
   merge_kernel<<<grid_merge, 256, 0, (cudaStream_t)stream>>>(slot->dev_matchers, tok->dev, bitmask_dev, (long long)row_stride_words,

@@ -27,6 +27,7 @@ struct EntryDev {
   const uint32_t* unc_id;    // [n_unc] ascending token ids
   const uint32_t* unc_rank;  // [n_unc] ascending ranks
   const uint32_t* unc_exit;  // [n_unc] parallel to unc_rank: bit j = the token leaves the entry's rule after j bytes
+  const uint8_t* unc_byte;   // [n_unc] parallel to unc_rank: the token's byte at its first exit (what the context must scan)
   int32_t kind;              // xg_store_kind_t
   int32_t n_list;            // list length (0 for bitset)
   int32_t n_unc;

@@ -2,6 +2,7 @@
 // dense contraction, so no tensor cores; the rules that matter are coalesced streaming, work
 // that follows the trie order of the vocabulary, and grids sized to fill 148 SMs.
 #pragma once
+#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -258,7 +259,7 @@ plan_kernel(const int2* __restrict__ counts, int n_pos, int vocab_size, int n_wo
     if (nr < n_list) { kind = 1; n_list = nr; }
     if (n_words < n_list) { kind = 2; n_list = 0; }
     plan[p].kind = kind; plan[p].n_list = n_list; plan[p].n_acc = na; plan[p].n_unc = nu;
-    local += (kind == 2 ? n_words : n_list) + 3LL * nu;
+    local += (kind == 2 ? n_words : n_list) + 3LL * nu + (nu + 3) / 4;
   }
   sums[threadIdx.x] = local;
   __syncthreads();
@@ -271,7 +272,7 @@ plan_kernel(const int2* __restrict__ counts, int n_pos, int vocab_size, int n_wo
   long long run = sums[threadIdx.x] - local;
   for (int p = lo; p < hi; ++p) {
     plan[p].offset_words = run;
-    run += (plan[p].kind == 2 ? n_words : plan[p].n_list) + 3LL * plan[p].n_unc;
+    run += (plan[p].kind == 2 ? n_words : plan[p].n_list) + 3LL * plan[p].n_unc + (plan[p].n_unc + 3) / 4;
   }
   if (threadIdx.x == blockDim.x - 1) *total_words = sums[threadIdx.x];
 }
@@ -325,6 +326,7 @@ pack_kernel(const uint32_t* __restrict__ acc_id, const uint32_t* __restrict__ un
   if (threadIdx.x == 0) {
     EntryDev e;
     e.data = data; e.unc_id = out_uid; e.unc_rank = out_urank; e.unc_exit = out_urank + pl.n_unc;
+    e.unc_byte = reinterpret_cast<const uint8_t*>(out_urank + 2 * (size_t)pl.n_unc);
     e.kind = pl.kind; e.n_list = pl.n_list; e.n_unc = pl.n_unc; e.n_acc = pl.n_acc;
     entries[p] = e;
   }
@@ -344,6 +346,7 @@ exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, con
   const uint32_t* class_bits = stage_class_bits(g, sh_class);
   __syncthreads();
   uint32_t* out = const_cast<uint32_t*>(e.unc_exit);
+  uint8_t* out_byte = const_cast<uint8_t*>(e.unc_byte);
   for (int k = threadIdx.x; k < e.n_unc; k += blockDim.x) {
     const int rank = (int)e.unc_rank[k];
     const uint32_t off = v.offset[rank];
@@ -361,6 +364,7 @@ exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, con
       if (flags & kWalkOverflow) mask = 0;
     }
     out[k] = mask;
+    out_byte[k] = mask ? v.bytes[off + __ffs(mask) - 1] : 0;
   }
 }
 
@@ -727,6 +731,154 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
       if (threadIdx.x == 0 && status_user) status_user[b] = -6;
     }
   }
+}
+
+// ------------------------------------------------------------------------------------------
+// Per-step mask in one launch: a thread-block cluster of eight blocks per request.  Block r of
+// the cluster keeps slice r of the request's row in its shared memory.
+//   1. every block merges the accepted sets of the plan's entries into its own slice;
+//   2. cluster barrier; the blocks share the uncertain candidates (trie order, one token per
+//      lane); a token that passes is OR-ed into the slice of the block that owns its id, through
+//      distributed shared memory;
+//   3. cluster barrier; every block writes its slice with coalesced stores.
+// No global atomics, no scratch words, and the row never makes a round trip through L2.
+// Used when a slice fits (vocabularies up to 8 x 2048 x 32 tokens); larger vocabularies take the
+// two-kernel path above.
+// ------------------------------------------------------------------------------------------
+constexpr int kClusterBlocks = 8;
+
+__global__ void __cluster_dims__(kClusterBlocks, 1, 1) __launch_bounds__(256, 4)
+fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __restrict__ bitmask, long long row_stride,
+                    int32_t* __restrict__ status_user) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  __shared__ uint32_t row[kMergeMaxChunkWords];
+  __shared__ uint32_t tmp[kMergeMaxChunkWords];
+  __shared__ const uint32_t* ent_rank[kPlanCheckMax];
+  __shared__ const uint32_t* ent_exit[kPlanCheckMax];
+  __shared__ const uint8_t* ent_byte[kPlanCheckMax];
+  __shared__ int ent_cum[kPlanCheckMax + 1];
+  __shared__ uint32_t cont_st[kPlanCheckMax][kContCap];
+  __shared__ int32_t cont_org[kPlanCheckMax][kContCap];
+  __shared__ int cont_cnt[kPlanCheckMax];
+  __shared__ uint32_t cont_first[kPlanCheckMax][8];
+  __shared__ uint32_t sh_class[kSharedClasses * 8];
+  __shared__ int sh_fail;          // block 0's copy collects the whole cluster's failures
+
+  const int b = blockIdx.y;
+  const int rank = (int)cluster.block_rank();
+  const MatcherDev& m = *matchers[b];
+  const GrammarDev& g = *m.grammar;
+  const StepPlan& plan = *m.plan;
+  const int chunk = (v.n_words + kClusterBlocks - 1) / kClusterBlocks;
+  const int w0 = rank * chunk, w1 = min(v.n_words, w0 + chunk);
+  const int nw = max(0, w1 - w0);
+  for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] = 0;
+  const int st0 = m.terminated ? -8 : (plan.overflow ? -6 : 0);
+  if (threadIdx.x == 0) sh_fail = 0;
+  const int n_ent = st0 == 0 ? plan.n_check : 0;
+  const int total = n_ent ? plan.check_cum[n_ent] : 0;
+  __syncthreads();
+  // 1. merge
+  if (st0 == 0 && nw > 0) {
+    const uint32_t id_lo = (uint32_t)w0 * 32u, id_hi = (uint32_t)w1 * 32u;
+    const int n_merge = plan.n_merge;
+    for (int k = 0; k < n_merge; ++k) {
+      const EntryDev e = g.entries[plan.merge_state[k]];
+      if (e.kind == 2) {
+        for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] |= e.data[w0 + w];
+      } else if (e.kind == 0) {
+        const int lo = lower_bound_u32(e.data, e.n_list, id_lo), hi = lower_bound_u32(e.data, e.n_list, id_hi);
+        for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) { const uint32_t id = e.data[i]; atomicOr(&row[(id >> 5) - w0], 1u << (id & 31)); }
+      } else {
+        const uint32_t tail = (v.vocab_size & 31) ? ((1u << (v.vocab_size & 31)) - 1) : 0xFFFFFFFFu;
+        for (int w = threadIdx.x; w < nw; w += blockDim.x) tmp[w] = (w0 + w == v.n_words - 1) ? tail : 0xFFFFFFFFu;
+        __syncthreads();
+        int lo = lower_bound_u32(e.data, e.n_list, id_lo), hi = lower_bound_u32(e.data, e.n_list, id_hi);
+        for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) { const uint32_t id = e.data[i]; atomicAnd(&tmp[(id >> 5) - w0], ~(1u << (id & 31))); }
+        lo = lower_bound_u32(e.unc_id, e.n_unc, id_lo); hi = lower_bound_u32(e.unc_id, e.n_unc, id_hi);
+        for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) { const uint32_t id = e.unc_id[i]; atomicAnd(&tmp[(id >> 5) - w0], ~(1u << (id & 31))); }
+        __syncthreads();
+        for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] |= tmp[w];
+      }
+      __syncthreads();
+    }
+    if (threadIdx.x == 0 && v.eos_id >= 0 && (uint32_t)v.eos_id >= id_lo && (uint32_t)v.eos_id < id_hi && plan.eos_ok)
+      row[(v.eos_id >> 5) - w0] |= 1u << (v.eos_id & 31);
+  }
+  // 2. check (the plan and its arrays are the same for the whole cluster: `total` is uniform)
+  if (total > 0) {
+    const int n = m.n_sets - 1;
+    const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
+    const uint32_t* class_bits = stage_class_bits(g, sh_class);
+    for (int i = threadIdx.x; i < n_ent; i += blockDim.x) {
+      const EntryDev& e = g.entries[plan.check_state[i]];
+      ent_rank[i] = e.unc_rank; ent_exit[i] = e.unc_exit; ent_byte[i] = e.unc_byte;
+      cont_cnt[i] = plan.cont_cnt[i];
+    }
+    for (int i = threadIdx.x; i <= n_ent; i += blockDim.x) ent_cum[i] = plan.check_cum[i];
+    for (int i = threadIdx.x; i < n_ent * kContCap; i += blockDim.x) {
+      (&cont_st[0][0])[i] = (&plan.cont_st[0][0])[i];
+      (&cont_org[0][0])[i] = (&plan.cont_org[0][0])[i];
+    }
+    for (int i = threadIdx.x; i < n_ent * 8; i += blockDim.x) (&cont_first[0][0])[i] = (&plan.cont_first[0][0])[i];
+    cluster.sync();            // every slice is merged (and this block's staging is visible)
+    const int stride = kClusterBlocks * blockDim.x;
+    auto walk_one = [&](int trank, uint32_t off, int e, int at) {
+      const int len = (int)(v.offset[trank + 1] - off);
+      bool pass = false, overflow = len - at > kFastMaxBytes;
+      if (!overflow) {
+        uint32_t st[kFastCap];
+        int32_t org[kFastCap];
+        int16_t lsb[kFastMaxBytes + 2];
+        int flags = 0;
+        Chart c = hist;
+        if (at > 0) { c.i_st = cont_st[e]; c.i_org = cont_org[e]; c.i_cnt = cont_cnt[e]; c.i_idx = n + at; }
+        pass = token_walk<int16_t>(g, class_bits, c, v.bytes + off + at, len - at, false, st, org, kFastCap, lsb, &flags, nullptr) == len - at;
+        overflow = (flags & kWalkOverflow) != 0;
+      }
+      if (overflow) atomicOr(cluster.map_shared_rank(&sh_fail, 0), 1);
+      return pass && !overflow;
+    };
+    for (int j = rank * blockDim.x + threadIdx.x; j < total; j += stride) {
+      // per candidate: its exit mask and the byte at its first exit, both streamed in list order;
+      // the token's rank and bytes are only touched by the few that survive the bit test
+      int e = 0;
+      while (j >= ent_cum[e + 1]) ++e;
+      const int k = j - ent_cum[e];
+      uint32_t left = ent_exit[e][k];
+      bool pass = false;
+      int trank = -1;
+      if (left == 0) {                // no exit record (very long token, or its build-time walk overflowed): walk in full
+        trank = (int)ent_rank[e][k];
+        pass = walk_one(trank, v.offset[trank], e, 0);
+      } else {
+        uint32_t byte = ent_byte[e][k];
+        if (!((cont_first[e][byte >> 5] >> (byte & 31)) & 1u)) left &= left - 1;
+        if (left == 0) continue;                        // the usual end of a candidate
+        trank = (int)ent_rank[e][k];
+        const uint32_t off = v.offset[trank];
+        while (left && !pass) {
+          const int at = __ffs(left) - 1;
+          left &= left - 1;
+          byte = v.bytes[off + at];
+          if ((cont_first[e][byte >> 5] >> (byte & 31)) & 1u) pass = walk_one(trank, off, e, at);
+        }
+      }
+      if (pass) {
+        const int id = v.rank_to_id[trank];
+        const int word = id >> 5, owner = word / chunk;
+        atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
+      }
+    }
+    cluster.sync();            // every remote OR has landed
+  } else __syncthreads();
+  // 3. write the slice
+  const int failed = total > 0 ? *cluster.map_shared_rank(&sh_fail, 0) : 0;
+  const bool clear = st0 != 0 || failed;
+  for (int w = threadIdx.x; w < nw; w += blockDim.x) bitmask[(long long)b * row_stride + w0 + w] = clear ? 0 : (int32_t)row[w];
+  if (rank == 0 && threadIdx.x == 0 && status_user) status_user[b] = st0 != 0 ? st0 : (failed ? -6 : 0);
+  if (total > 0) cluster.sync();      // block 0's shared memory must outlive the reads above
 }
 
 // ------------------------------------------------------------------------------------------
