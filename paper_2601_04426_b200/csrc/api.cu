@@ -254,32 +254,29 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
   const size_t row_bytes = (size_t)W * 4;
   const size_t budget = size_t(768) << 20;                         // scratch rows per batch
   const int per_batch = (int)std::max<size_t>(1, std::min<size_t>(std::min<size_t>(states.size(), 65535), budget / (3 * row_bytes)));
-  int32_t* d_pos = nullptr;
-  uint32_t* d_rows = nullptr;
-  int2* d_counts = nullptr;
-  PackPlan* d_plan = nullptr;
-  long long* d_total = nullptr;
-  EntryDev* d_entries = nullptr;
-  int2* d_over = nullptr;
-  int* d_over_count = nullptr;
+  // build scratch lives in the pool and is reused by later compiles (no allocation per grammar)
   const int over_cap = 1 << 16;
-  auto cleanup = [&]() { cudaFree(d_pos); cudaFree(d_rows); cudaFree(d_counts); cudaFree(d_plan); cudaFree(d_total); cudaFree(d_entries); cudaFree(d_over); cudaFree(d_over_count); };
+  CachePool& pool = *g->pool;
+  int32_t* d_pos = (int32_t*)pool.scratch(0, per_batch * sizeof(int32_t));
+  uint32_t* d_rows = (uint32_t*)pool.scratch(1, 3 * row_bytes * per_batch);
+  int2* d_counts = (int2*)pool.scratch(2, per_batch * sizeof(int2));
+  PackPlan* d_plan = (PackPlan*)pool.scratch(3, per_batch * sizeof(PackPlan));
+  long long* d_total = (long long*)pool.scratch(4, sizeof(long long));
+  EntryDev* d_entries = (EntryDev*)pool.scratch(5, per_batch * sizeof(EntryDev));
+  int2* d_over = (int2*)pool.scratch(6, over_cap * sizeof(int2));
+  int* d_over_count = (int*)pool.scratch(7, 2 * sizeof(int));
+  if (!d_pos || !d_rows || !d_counts || !d_plan || !d_total || !d_entries || !d_over || !d_over_count)
+    return set_error(XG_ERR_OOM, "cache build scratch allocation failed");
+  auto cleanup = [&]() {};
 #define XG_CUDA_C(expr) do { cudaError_t e__ = (expr); if (e__ != cudaSuccess) { cleanup(); return set_error(XG_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)); } } while (0)
-  XG_CUDA_C(cudaMalloc(&d_pos, per_batch * sizeof(int32_t)));
-  XG_CUDA_C(cudaMalloc(&d_rows, 3 * row_bytes * per_batch));
-  XG_CUDA_C(cudaMalloc(&d_counts, per_batch * sizeof(int2)));
-  XG_CUDA_C(cudaMalloc(&d_plan, per_batch * sizeof(PackPlan)));
-  XG_CUDA_C(cudaMalloc(&d_total, sizeof(long long)));
-  XG_CUDA_C(cudaMalloc(&d_entries, per_batch * sizeof(EntryDev)));
-  XG_CUDA_C(cudaMalloc(&d_over, over_cap * sizeof(int2)));
-  XG_CUDA_C(cudaMalloc(&d_over_count, 2 * sizeof(int)));
   for (size_t begin = 0; begin < states.size(); begin += per_batch) {
     const int n = (int)std::min<size_t>(per_batch, states.size() - begin);
     uint32_t* acc = d_rows;
     uint32_t* unc = d_rows + (size_t)per_batch * W;
     uint32_t* unr = d_rows + 2 * (size_t)per_batch * W;
     XG_CUDA_C(cudaMemcpyAsync(d_pos, states.data() + begin, n * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
-    XG_CUDA_C(cudaMemsetAsync(d_rows, 0, 3 * row_bytes * per_batch, stream));
+    XG_CUDA_C(cudaMemsetAsync(acc, 0, row_bytes * n, stream));      // the rank-ordered row is fully written by ballots
+    XG_CUDA_C(cudaMemsetAsync(unc, 0, row_bytes * n, stream));
     XG_CUDA_C(cudaMemsetAsync(d_over_count, 0, 2 * sizeof(int), stream));
     dim3 grid((V + 255) / 256, n);
     classify_kernel<<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, acc, unc, unr, d_over, d_over_count, over_cap);

@@ -559,6 +559,22 @@ Fsm determinize(const Fsm& f, int max_states) {
       }
     for (auto& kv : by_rule) { int t = state_of(kv.second); d.ref(cur, kv.first, t); }
     if (byte_edges.empty()) continue;
+    // common case: the byte sets do not overlap, so every edge keeps its single target
+    {
+      ByteSet seen;
+      bool disjoint = true;
+      for (const Edge* e : byte_edges) {
+        for (int w = 0; w < 8 && disjoint; ++w) disjoint = (seen.w[w] & e->set.w[w]) == 0;
+        if (!disjoint) break;
+        seen.merge(e->set);
+      }
+      if (disjoint) {
+        std::map<int, ByteSet> by_target;
+        for (const Edge* e : byte_edges) by_target[e->to].merge(e->set);
+        for (auto& kv : by_target) { std::vector<int> tg{kv.first}; int t = state_of(tg); d.bytes(cur, kv.second, t); }
+        continue;
+      }
+    }
     std::map<std::vector<int>, ByteSet> groups;      // target subset -> bytes
     std::vector<int> targets;
     for (int b = 0; b < 256; ++b) {
@@ -574,8 +590,61 @@ Fsm determinize(const Fsm& f, int max_states) {
   return d;
 }
 
+// Minimisation of an acyclic deterministic automaton in one bottom-up pass: in reverse
+// topological order, two states are equivalent iff they agree on acceptance and on their edges
+// into already-merged targets.  Returns false (and leaves `out` alone) if the automaton has a cycle.
+bool minimize_acyclic(const Fsm& f, Fsm& out) {
+  const int n = f.size();
+  std::vector<int> indeg(n, 0), order;
+  for (int s = 0; s < n; ++s) for (const Edge& e : f.out[s]) ++indeg[e.to];
+  for (int s = 0; s < n; ++s) if (!indeg[s]) order.push_back(s);
+  for (size_t q = 0; q < order.size(); ++q) for (const Edge& e : f.out[order[q]]) if (--indeg[e.to] == 0) order.push_back(e.to);
+  if ((int)order.size() != n) return false;
+  typedef std::pair<std::vector<std::pair<int, ByteSet>>, std::vector<std::pair<int, int>>> Sig;
+  std::map<std::pair<int, Sig>, int> cls_of;
+  std::vector<int> cls(n, -1);
+  for (int k = n - 1; k >= 0; --k) {
+    const int s = order[k];
+    std::map<int, ByteSet> by_cls;
+    std::vector<std::pair<int, int>> refs;
+    for (const Edge& e : f.out[s]) {
+      if (e.kind == Edge::kBytes) by_cls[cls[e.to]].merge(e.set);
+      else refs.emplace_back(e.rule, cls[e.to]);
+    }
+    std::sort(refs.begin(), refs.end());
+    auto key = std::make_pair((int)f.fin[s], Sig{std::vector<std::pair<int, ByteSet>>(by_cls.begin(), by_cls.end()), refs});
+    auto it = cls_of.find(key);
+    if (it == cls_of.end()) it = cls_of.emplace(key, (int)cls_of.size()).first;
+    cls[s] = it->second;
+  }
+  Fsm m;
+  m.has_tag_dispatch = f.has_tag_dispatch;
+  const int n_cls = (int)cls_of.size();
+  for (int b = 0; b < n_cls; ++b) m.add();
+  std::vector<char> done(n_cls, 0);
+  m.start = cls[f.start];
+  for (int s = 0; s < n; ++s) {
+    const int b = cls[s];
+    if (f.fin[s]) m.fin[b] = 1;
+    if (done[b]) continue;
+    done[b] = 1;
+    std::map<int, ByteSet> by_cls;
+    for (const Edge& e : f.out[s]) {
+      if (e.kind == Edge::kBytes) by_cls[cls[e.to]].merge(e.set);
+      else m.ref(b, e.rule, cls[e.to]);
+    }
+    for (auto& kv : by_cls) m.bytes(b, kv.second, kv.first);
+  }
+  out = m;
+  return true;
+}
+
 // merge equivalent states of a deterministic automaton (partition refinement on sparse signatures)
 Fsm minimize(const Fsm& f) {
+  {
+    Fsm quick;
+    if (minimize_acyclic(f, quick)) return quick;
+  }
   int n = f.size();
   std::vector<int> block(n);
   for (int s = 0; s < n; ++s) block[s] = f.fin[s] ? 1 : 0;

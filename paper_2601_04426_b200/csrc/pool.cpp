@@ -18,6 +18,20 @@ uint64_t hash_fold(uint64_t h, uint64_t x) {
 
 CachePool::~CachePool() {
   for (void* p : chunks_) cudaFree(p);
+  for (auto& s : scratch_) cudaFree(s.first);
+}
+
+void* CachePool::scratch(int slot, size_t bytes) {
+  if ((int)scratch_.size() <= slot) scratch_.resize(slot + 1, {nullptr, 0});
+  auto& s = scratch_[slot];
+  if (s.second < bytes) {
+    cudaFree(s.first);
+    s = {nullptr, 0};
+    size_t want = bytes + bytes / 4;
+    if (cudaMalloc(&s.first, want) != cudaSuccess) { s.first = nullptr; return nullptr; }
+    s.second = want;
+  }
+  return s.first;
 }
 
 void* CachePool::allocate_device(size_t bytes) {

@@ -45,12 +45,15 @@ class CachePool {
   PoolRule& rule(int id) { return rules_[id]; }
   size_t n_rules() const { return rules_.size(); }
   void* allocate_device(size_t bytes);      // lives as long as the pool
+  // reusable build scratch (grow-only, one buffer per slot; call with `mu` held)
+  void* scratch(int slot, size_t bytes);
 
  private:
   const void* owner_;
   std::vector<PoolRule> rules_;
   std::unordered_map<uint64_t, std::vector<int>> by_hash_;
   std::vector<void*> chunks_;
+  std::vector<std::pair<void*, size_t>> scratch_;
   int find_or_add(uint64_t hash, std::vector<uint64_t>&& serial);
 };
 

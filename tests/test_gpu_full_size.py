@@ -74,3 +74,25 @@ def test_full_size_sampled_parity(name, steps, sample):
         assert compared == len(sample)
     finally:
         s.close()
+
+
+def test_vocabulary_too_large_for_one_cluster_takes_the_two_kernel_path():
+    """Above 8 x 2048 x 32 = 524 288 tokens a row slice no longer fits the cluster kernel's shared
+    memory and the fill runs as merge + check kernels; masks must not change."""
+    import torch
+    from paper_2601_04426_b200 import engine
+    w = inputs.make_workload("C1", steps=6, vocab_size=524288 + 4096)
+    s = engine.Session(w)
+    ov = O.Vocab(w.vocab.tokens, w.vocab.eos_id, w.vocab.special_ids)
+    om = O.Matcher(O.Grammar(SE.grammar_text(w.grammars[0].kind, w.grammars[0].text)))
+    try:
+        for step, tok in enumerate(w.trajectories[0]):
+            s.fill()
+            assert np.array_equal(s.mask_numpy()[0], om.mask(ov)), step
+            s.accept([tok])
+            assert int(s.accept_status.cpu()[0]) == 0
+            if om.accept_token(ov, tok) == 2:
+                om.reset()
+                s.reset(0)
+    finally:
+        s.close()
