@@ -29,7 +29,8 @@ if ROOT not in sys.path:
 
 from paper_2601_04426_b200 import inputs  # noqa: E402
 
-SHAPES = {"C1": (1, 8192), "C2": (1, 128256), "C3": (128, 151936), "C4": (64, 128256), "C5": (256, 200064)}
+SHAPES = {"C1": (1, 8192), "C2": (1, 128256), "C3": (128, 151936), "C4": (64, 128256), "C5": (256, 200064),
+          "T5": (16, 128256), "T20": (16, 128256), "T50": (16, 128256), "T100": (16, 128256)}
 
 
 def measured_peaks():

@@ -175,7 +175,8 @@ def schema_to_ebnf(schema_text: str, root: str = "root", prefix: str = "") -> st
 def tag_dispatch_to_ebnf(spec_text: str, root: str = "root") -> str:
     """{"tags": [{"tag": t, "end": e, "tools": [{"name": n, "schema": s}, ...]}, ...], "stop_strs": [...]}
 
-    Tag t dispatches to  ( call_1 | ... | call_n ) e  with  call_k = {"name": "n_k", "arguments": <s_k>}.
+    Tag t dispatches to  ( call_1 | ... | call_n ) e  with  call_k = {"name": "n_k", "arguments": <s_k>},
+    or, when the tag entry has "bare": true, call_k = <s_k> alone.
     """
     spec = json.loads(spec_text) if isinstance(spec_text, str) else spec_text
     rules: List[str] = []
@@ -186,8 +187,11 @@ def tag_dispatch_to_ebnf(spec_text: str, root: str = "root") -> str:
             prefix = "t%d_%d_" % (ti, ki)
             sub = schema_to_ebnf(tool["schema"], root=prefix + "args", prefix=prefix)
             rules.append(sub.rstrip("\n"))
-            head = '{"name": %s, "arguments": ' % json_literal(tool["name"])
-            rules.append('%scall ::= %s %sargs "}"' % (prefix, ebnf_quote(head), prefix))
+            if tag.get("bare"):
+                rules.append('%scall ::= %sargs' % (prefix, prefix))
+            else:
+                head = '{"name": %s, "arguments": ' % json_literal(tool["name"])
+                rules.append('%scall ::= %s %sargs "}"' % (prefix, ebnf_quote(head), prefix))
             calls.append(prefix + "call")
         rules.append("tag_%d ::= ( %s ) %s" % (ti, " | ".join(calls), ebnf_quote(tag.get("end", ""))))
         pairs.append("(%s, tag_%d)" % (ebnf_quote(tag["tag"]), ti))

@@ -1261,7 +1261,9 @@ std::string tag_dispatch_to_ebnf(const std::string& spec_json) {
       SchemaLowering low(schema->get("$defs"), prefix);
       std::string args = low.lower(*schema);
       for (auto& r : low.rules) rules += r + "\n";
-      rules += prefix + "call ::= " + literal("{\"name\": " + json_string_text(name->text) + ", \"arguments\": ") + " " + args + " \"}\"\n";
+      const Json* bare = tag.get("bare");
+      if (bare && bare->type == Json::kBool && bare->boolean) rules += prefix + "call ::= " + args + "\n";      // the tag names the tool: arguments only
+      else rules += prefix + "call ::= " + literal("{\"name\": " + json_string_text(name->text) + ", \"arguments\": ") + " " + args + " \"}\"\n";
       calls += (k ? " | " : "") + prefix + "call";
     }
     std::string rule = "dispatch_" + std::to_string(ti);

@@ -459,6 +459,11 @@ def make_tool_set(rng: Rng, n_tools: int) -> List[dict]:
     return tools
 
 
+def function_tags_spec(tools: List[dict]) -> dict:
+    """One tag per tool: `<function=NAME>` dispatches to that tool's argument object, then `</function>`."""
+    return {"tags": [{"tag": "<function=%s>" % t["name"], "end": "</function>", "bare": True, "tools": [t]} for t in tools], "stop_strs": []}
+
+
 def tag_dispatch_spec(tools: List[dict], tag: str = "<tool_call>", end: str = "</tool_call>") -> dict:
     """One tag that dispatches to `(call_1 | ... | call_n) end`, call_k = {"name": ..., "arguments": ...}."""
     return {"tags": [{"tag": tag, "end": end, "tools": tools}], "stop_strs": []}
@@ -480,6 +485,43 @@ def sample_tool_text(rng: Rng, tools: List[dict], tag: str, end: str, n_calls: i
         out.append(tag + '{"name": "%s", "arguments": %s}' % (tool["name"], args) + end)
         prev = c
     out.append(free(max(1, words_total - prev)))
+    return "".join(out)
+
+
+def make_function_tags(rng: Rng, n_tags: int, tag_len: int = 20) -> List[dict]:
+    """`n_tags` tools whose tags share the prefix `<function=` and are `tag_len` bytes long in total
+    (the shape of the paper's tag-count experiment, Section 4.1), each with a small argument schema."""
+    tools, names = [], set()
+    body = tag_len - len("<function=") - 1
+    while len(tools) < n_tags:
+        name = _word(rng, body, body)
+        if name in names:
+            continue
+        names.add(name)
+        schema = make_object_schema(rng, rng.randint(1, 4), 1, kinds=("string", "integer", "number", "boolean", "enum"), enum_size=3)
+        tools.append({"name": name, "schema": schema})
+    return tools
+
+
+def function_tags_ebnf(tools: List[dict], stop_strs: Sequence[str] = ()) -> Tuple[str, List[str]]:
+    """Grammar text: one tag per tool, `<function=NAME>` -> arguments object then `</function>`.
+    The argument grammars are given as one JSON-schema-shaped EBNF rule each by the caller's own
+    lowering; here only the dispatching skeleton is spelled, with rule names args_<i>."""
+    pairs = ", ".join('("<function=%s>", call_%d)' % (t["name"], i) for i, t in enumerate(tools))
+    stops = ", ".join(json.dumps(s) for s in stop_strs)
+    head = "root ::= TagDispatch(%s, stop_strs=(%s))\n" % (pairs, stops)
+    calls = "".join('call_%d ::= args_%d "</function>"\n' % (i, i) for i in range(len(tools)))
+    return head + calls, ["args_%d" % i for i in range(len(tools))]
+
+
+def sample_function_text(rng: Rng, tools: List[dict], n_calls: int, n_words: int) -> str:
+    def free(k: int) -> str:
+        return " ".join(_word(rng, 2, 8) for _ in range(k)) + rng.choice([" ", ". ", "\n"])
+    out = [free(max(1, n_words // (n_calls + 1)))]
+    for _ in range(n_calls):
+        tool = rng.choice(tools)
+        out.append("<function=%s>%s</function>" % (tool["name"], sample_document(tool["schema"], rng)))
+        out.append(free(max(1, n_words // (n_calls + 1))))
     return "".join(out)
 
 
@@ -519,13 +561,18 @@ _SHAPES = {
     "C3": (151936,   16,  4.0, 0.3,    0.0,  128,  128,  "bf16"),
     "C4": (128256,   16,  4.0, 0.3,    0.0,  64,   512,  "f32"),
     "C5": (200064,   24,  4.5, 0.0,    0.1,  256,  256,  "bf16"),
+    # many-tag TagDispatch (Section 4.1's tag-count experiment): 5 / 20 / 50 / 100 tags of 20 bytes with a common prefix
+    "T5": (128256,   16,  4.0, 0.3,    0.0,  16,   128,  "bf16"),
+    "T20": (128256,  16,  4.0, 0.3,    0.0,  16,   128,  "bf16"),
+    "T50": (128256,  16,  4.0, 0.3,    0.0,  16,   128,  "bf16"),
+    "T100": (128256, 16,  4.0, 0.3,    0.0,  16,   128,  "bf16"),
 }
 
 _vocab_cache: Dict[Tuple, Vocab] = {}
 
 
 def config_seed(name: str) -> int:
-    return BASE_SEED * 10 + int(name[1])
+    return BASE_SEED * 10 + (int(name[1]) if name[0] == "C" else 1000 + int(name[1:]))
 
 
 def config_vocab(name: str, vocab_size: Optional[int] = None) -> Vocab:
@@ -533,7 +580,7 @@ def config_vocab(name: str, vocab_size: Optional[int] = None) -> Vocab:
     if vocab_size is not None:
         V = vocab_size
     # C2 and C4 share one Llama-3-sized vocabulary
-    seed_name = "C2" if name == "C4" else name
+    seed_name = "C2" if (name == "C4" or name[0] == "T") else name
     key = (seed_name, V)
     if key not in _vocab_cache:
         _vocab_cache[key] = make_vocab(config_seed(seed_name) ^ 0x5EED, V, lmax, mean, lead, utf8)
@@ -624,6 +671,14 @@ def make_workload(name: str, batch: Optional[int] = None, steps: Optional[int] =
             t, d = _trajectory(tok, vocab.eos_id, S, lambda: sample_any_json(rr, depth).encode("utf-8"))
             request_grammar.append(0); trajs.append(t); docs_all.append(d)
             meta.setdefault("depths", []).append(depth)
+    elif name[0] == "T":
+        tools = make_function_tags(rng.fork(3), int(name[1:]))
+        grammars.append(GrammarSpec("tag_dispatch", json.dumps(function_tags_spec(tools))))
+        meta["tools"] = tools
+        for b in range(B):
+            rr = rng.fork(100 + b)
+            t, d = _trajectory(tok, vocab.eos_id, S, lambda: sample_function_text(rr, tools, rr.randint(1, 3), 40).encode())
+            request_grammar.append(0); trajs.append(t); docs_all.append(d)
     else:
         raise KeyError(name)
     return Workload(name=name, vocab=vocab, grammars=grammars, request_grammar=request_grammar,

@@ -90,7 +90,7 @@ def _mutate(rng, doc, alphabet):
     return doc[:pos] + b + doc[pos + 1:] if kind == 0 else (doc[:pos] + doc[pos + 1:] if kind == 1 else doc[:pos] + b + doc[pos:])
 
 
-@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4", "C5"])
+@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4", "C5", "T20"])
 def test_workload_grammars_same_language_as_oracle(name):
     w = inputs.make_workload(name, batch=3, steps=40)
     rng = inputs.Rng(17)
@@ -114,7 +114,7 @@ def test_workload_grammars_same_language_as_oracle(name):
                         assert tm.can_terminate() == O.accepts(og, mut), mut
 
 
-@pytest.mark.parametrize("name,vsize,steps", [("C1", 2048, 40), ("C4", 2048, 60), ("C5", 4096, 30)])
+@pytest.mark.parametrize("name,vsize,steps", [("C1", 2048, 40), ("C4", 2048, 60), ("C5", 4096, 30), ("T5", 2048, 50)])
 def test_masks_plain_equals_merged_equals_oracle(name, vsize, steps):
     """The cache classification plus the merge rule reproduces the plain definition, step by step."""
     w = inputs.make_workload(name, batch=1, steps=steps, vocab_size=vsize)

@@ -92,6 +92,12 @@ def test_c5_recursive_json_with_utf8():
     _run_trajectories(w, {0, 7, 31, 63}, check_requests={1})
 
 
+def test_many_tag_dispatch_batch():
+    """Twenty tags with a common prefix (the paper's tag-count experiment, Section 4.1)."""
+    w = inputs.make_workload("T20", batch=4, steps=90, vocab_size=16384)
+    _run_trajectories(w, {0, 20, 45, 89}, check_requests={1})
+
+
 def test_hand_worked_masks_on_gpu():
     torch, engine = _engine()
     from golden_util import load_mask_fixture
