@@ -763,6 +763,14 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   __shared__ int cont_cnt[kPlanCheckMax];
   __shared__ uint32_t cont_first[kPlanCheckMax][8];
   __shared__ uint32_t sh_class[kSharedClasses * 8];
+  // uncertain tokens too long for the per-thread arrays (33..255 bytes; rare) are queued and walked one at a time
+  // by thread 0 in this block-wide scratch
+  constexpr int kLongQueue = 32, kLongCap = 1024;
+  __shared__ int long_q[kLongQueue];
+  __shared__ int long_n;
+  __shared__ uint32_t long_st[kLongCap];
+  __shared__ int32_t long_org[kLongCap];
+  __shared__ int16_t long_lsb[kSlowMaxBytes + 2];
   __shared__ int sh_fail;          // block 0's copy collects the whole cluster's failures
 
   const int b = blockIdx.y;
@@ -775,7 +783,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   const int nw = max(0, w1 - w0);
   for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] = 0;
   const int st0 = m.terminated ? -8 : (plan.overflow ? -6 : 0);
-  if (threadIdx.x == 0) sh_fail = 0;
+  if (threadIdx.x == 0) { sh_fail = 0; long_n = 0; }
   const int n_ent = st0 == 0 ? plan.n_check : 0;
   const int total = n_ent ? plan.check_cum[n_ent] : 0;
   __syncthreads();
@@ -851,6 +859,11 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
       int trank = -1;
       if (left == 0) {                // no exit record (very long token, or its build-time walk overflowed): walk in full
         trank = (int)ent_rank[e][k];
+        if ((int)(v.offset[trank + 1] - v.offset[trank]) > kFastMaxBytes) {
+          const int slot = atomicAdd(&long_n, 1);
+          if (slot < kLongQueue) long_q[slot] = trank; else atomicOr(cluster.map_shared_rank(&sh_fail, 0), 1);
+          continue;
+        }
         pass = walk_one(trank, v.offset[trank], e, 0);
       } else {
         uint32_t byte = ent_byte[e][k];
@@ -869,6 +882,22 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
         const int id = v.rank_to_id[trank];
         const int word = id >> 5, owner = word / chunk;
         atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int i = 0; i < min(long_n, kLongQueue); ++i) {
+        const int trank = long_q[i];
+        const uint32_t off = v.offset[trank];
+        const int len = (int)(v.offset[trank + 1] - off);
+        int flags = 0;
+        const bool pass = token_walk<int16_t>(g, class_bits, hist, v.bytes + off, len, false, long_st, long_org, kLongCap, long_lsb, &flags, nullptr) == len;
+        if (flags & kWalkOverflow) atomicOr(cluster.map_shared_rank(&sh_fail, 0), 1);
+        else if (pass) {
+          const int id = v.rank_to_id[trank];
+          const int word = id >> 5, owner = word / chunk;
+          atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
+        }
       }
     }
     cluster.sync();            // every remote OR has landed

@@ -316,3 +316,91 @@ def test_history_capacity_is_reported_not_overrun():
     bits = O.unpack_bits(mask.cpu().numpy().view(np.uint32)[0], len(toks))
     assert bits[ord("a")] and bits[eos] and bits[toks.index(b"aaaa")] and bits.sum() == 3
     m.close(); g.close(); tok.close()
+
+
+def test_long_tokens_up_to_255_bytes():
+    """Tokens beyond the per-thread walk arrays (33..255 bytes): classified by the exact slow path at
+    build time, accepted in pieces, and checked against the full state when uncertain."""
+    torch, engine = _engine()
+    base = [bytes([b]) for b in range(256)]
+    long_tokens = [b"a" * 33, b"ab" * 40, b"x" * 255, b"a" * 40 + b"}", b"a" * 100 + b"}}", b"b" * 64 + b'}, "k": {', b"z" * 200 + b"}!", b'{"' + b"q" * 60]
+    toks = base + long_tokens + [b""]
+    toks += [b"\xfe\xff%d" % i for i in range(-len(toks) % 32)]
+    eos = toks.index(b"")
+    ebnf = 'root ::= obj\nobj ::= "{" [a-z]* "}" | "{" "\\"" [a-z]* "\\": " obj "}"\n'
+    tok = B.Tokenizer(toks, eos)
+    g = B.Grammar(tok, "ebnf", ebnf, inline_max_states=0)
+    ov = O.Vocab(toks, eos)
+    og = O.Grammar(ebnf)
+    # cache entries against the oracle's classification on the exported tables
+    t = g.tables()
+    scal = {k: t.pop(k) for k in ("n_rules", "n_states", "n_classes", "root_rule", "root_nullable")}
+    tb = O.Tables(scal["n_rules"], scal["n_states"], scal["n_classes"], scal["root_rule"], scal["root_nullable"], **t)
+    saw_long_uncertain = False
+    for s_ in tb.scannable_states():
+        e = g.cache_entry(s_)
+        cls = tb.classify(ov, s_)
+        acc, unc = _entry_sets(e, len(toks))
+        assert acc == set(np.nonzero(cls == 1)[0].tolist()) and unc == set(np.nonzero(cls == 2)[0].tolist()), s_
+        saw_long_uncertain |= any(len(toks[i]) > 32 for i in unc)
+    assert saw_long_uncertain
+    m = B.Matcher(g)
+    batch = B.Batch([m])
+    om = O.Matcher(og)
+    mask = torch.zeros((1, tok.words), dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ids = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for piece in [b"{", b'"', b"q" * 3, b'": ', b"{", b"a" * 33, b"ab" * 40, b"a" * 40 + b"}", b"}"]:
+        batch.fill_next_token_bitmask(mask.data_ptr(), tok.words, st.data_ptr())
+        assert int(st.cpu()[0]) == 0
+        assert np.array_equal(mask.cpu().numpy().view(np.uint32)[0], om.mask(ov)), piece
+        tid = toks.index(piece) if piece in toks else None
+        if tid is None:
+            for byte in piece:
+                ids[0] = byte
+                batch.accept_token(ids.data_ptr(), st.data_ptr())
+                assert int(st.cpu()[0]) == 0
+                assert om.accept_token(ov, byte) == 1
+        else:
+            ids[0] = tid
+            batch.accept_token(ids.data_ptr(), st.data_ptr())
+            assert int(st.cpu()[0]) == 0, piece
+            assert om.accept_token(ov, tid) == 1
+    batch.fill_next_token_bitmask(mask.data_ptr(), tok.words, st.data_ptr())
+    assert np.array_equal(mask.cpu().numpy().view(np.uint32)[0], om.mask(ov))
+    m.close(); g.close(); tok.close()
+
+
+def test_item_sets_beyond_the_fast_path():
+    """Sixty alternatives that all start with the same byte give Earley sets of sixty items: the cache is
+    still built exactly (slow path), while the run-time calls report XG_ERR_CAPACITY instead of guessing."""
+    torch, engine = _engine()
+    toks = [bytes([b]) for b in range(256)] + [b"xa", b"xab", b"xq7", b"x", b"xa9!", b""]
+    toks += [b"\xfe\xff%d" % i for i in range(-len(toks) % 32)]
+    eos = toks.index(b"")
+    rules = "\n".join('alt%d ::= "x" [a-z]* "%d" "!"?' % (i, i % 10) for i in range(60))
+    ebnf = "root ::= " + " | ".join("alt%d" % i for i in range(60)) + "\n" + rules + "\n"
+    tok = B.Tokenizer(toks, eos)
+    g = B.Grammar(tok, "ebnf", ebnf, inline_max_states=0)
+    ov = O.Vocab(toks, eos)
+    t = g.tables()
+    scal = {k: t.pop(k) for k in ("n_rules", "n_states", "n_classes", "root_rule", "root_nullable")}
+    tb = O.Tables(scal["n_rules"], scal["n_states"], scal["n_classes"], scal["root_rule"], scal["root_nullable"], **t)
+    for s_ in tb.scannable_states()[::7]:
+        e = g.cache_entry(s_)
+        cls = tb.classify(ov, s_)
+        acc, unc = _entry_sets(e, len(toks))
+        assert acc == set(np.nonzero(cls == 1)[0].tolist()) and unc == set(np.nonzero(cls == 2)[0].tolist()), s_
+    m = B.Matcher(g)
+    batch = B.Batch([m])
+    mask = torch.zeros((1, tok.words), dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    batch.fill_next_token_bitmask(mask.data_ptr(), tok.words, st.data_ptr())
+    om = O.Matcher(O.Grammar(ebnf))
+    assert int(st.cpu()[0]) == 0 and np.array_equal(mask.cpu().numpy().view(np.uint32)[0], om.mask(ov))
+    ids = torch.tensor([toks.index(b"x")], dtype=torch.int32, device="cuda")
+    batch.accept_token(ids.data_ptr(), st.data_ptr())
+    assert int(st.cpu()[0]) == B.XG_ERR_CAPACITY          # sixty items do not fit; the state is unchanged
+    batch.fill_next_token_bitmask(mask.data_ptr(), tok.words, st.data_ptr())
+    assert int(st.cpu()[0]) == 0 and np.array_equal(mask.cpu().numpy().view(np.uint32)[0], om.mask(ov))
+    m.close(); g.close(); tok.close()
