@@ -275,8 +275,9 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
     uint32_t* unc = d_rows + (size_t)per_batch * W;
     uint32_t* unr = d_rows + 2 * (size_t)per_batch * W;
     XG_CUDA_C(cudaMemcpyAsync(d_pos, states.data() + begin, n * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
-    XG_CUDA_C(cudaMemsetAsync(acc, 0, row_bytes * n, stream));      // the rank-ordered row is fully written by ballots
+    XG_CUDA_C(cudaMemsetAsync(acc, 0, row_bytes * n, stream));      // blocks with nothing to scan leave their part of the rows untouched
     XG_CUDA_C(cudaMemsetAsync(unc, 0, row_bytes * n, stream));
+    XG_CUDA_C(cudaMemsetAsync(unr, 0, row_bytes * n, stream));
     XG_CUDA_C(cudaMemsetAsync(d_over_count, 0, 2 * sizeof(int), stream));
     dim3 grid((V + 255) / 256, n);
     classify_kernel<<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, acc, unc, unr, d_over, d_over_count, over_cap);

@@ -151,14 +151,48 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
   __shared__ uint32_t sh_st[1];
   __shared__ int32_t sh_org[1];
   __shared__ uint32_t sh_class[kSharedClasses * 8];
+  __shared__ uint32_t sh_first[8];          // bytes the position's own edges can take
+  __shared__ int sh_skip;
   const int pos = blockIdx.y;
-  if (threadIdx.x == 0) { sh_st[0] = (uint32_t)positions[pos]; sh_org[0] = -1; }
+  const int state = positions[pos];
+  const int rank = blockIdx.x * blockDim.x + threadIdx.x;
+  if (threadIdx.x < 8) {
+    // own first-byte set, and an early exit for the whole block: the tokens of a block are a
+    // contiguous run of the trie order, so their first bytes span [first of the first token,
+    // first of the last]; most (position, block) pairs have nothing in common
+    const StateRec rec = g.state[state];
+    uint32_t w = 0;
+    for (int e = 0; e < (int)(rec.n_own_n_scan & 0xFFFFu); ++e) {
+      const uint32_t code = e == 0 ? rec.edge0_class : g.scan_edge[rec.scan_begin + e].x;
+      if (code & kLiteral) w |= ((code & 0xFFu) >> 5) == threadIdx.x ? 1u << (code & 31u) : 0u;
+      else w |= g.class_bits[code * 8 + threadIdx.x];
+    }
+    sh_first[threadIdx.x] = w;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int r0 = blockIdx.x * blockDim.x, r1 = min(v.vocab_size, r0 + (int)blockDim.x) - 1;
+    // empty tokens sort first; treat them as byte 0
+    const uint32_t o0 = v.offset[r0], o1 = v.offset[r1];
+    const int b0 = v.offset[r0 + 1] > o0 ? v.bytes[o0] : 0, b1 = v.offset[r1 + 1] > o1 ? v.bytes[o1] : 0;
+    bool any = false;
+    for (int b = b0; b <= b1 && !any; ++b) any = (sh_first[b >> 5] >> (b & 31)) & 1u;
+    sh_skip = any ? 0 : 1;
+    sh_st[0] = (uint32_t)state; sh_org[0] = -1;
+  }
+  __syncthreads();
+  if (sh_skip) return;                       // every token of the block is rejected on its first byte (rows are pre-zeroed)
   const uint32_t* class_bits = stage_class_bits(g, sh_class);
   __syncthreads();
-  const int rank = blockIdx.x * blockDim.x + threadIdx.x;
   int cls = 0;
-  if (rank < v.vocab_size && !v.never[rank]) {
-    const uint32_t off = v.offset[rank];
+  bool live = rank < v.vocab_size && !v.never[rank];
+  uint32_t off = 0;
+  if (live) {
+    off = v.offset[rank];
+    const uint32_t first_byte = v.bytes[off];
+    live = (sh_first[first_byte >> 5] >> (first_byte & 31)) & 1u;             // else rejected on the first byte
+  }
+  if (live) {
     const int len = (int)(v.offset[rank + 1] - off);
     int flags = 0;
     int consumed = 0;
