@@ -43,7 +43,10 @@ def measured_peaks():
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons (read-only NVML queries, every millisecond) while the
+    measured passes run; falls back to polling nvidia-smi if the NVML binding is missing."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
     def __init__(self, index: int = 0):
         super().__init__(daemon=True)
@@ -51,13 +54,36 @@ class ClockSampler(threading.Thread):
         self.samples = []
         self.reasons = set()
         self.stop_flag = threading.Event()
+        self.max_mhz = None
         self.proc = None
 
     def run(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = self.index
+            if visible:
+                try:
+                    phys = int(visible.split(",")[self.index])
+                except ValueError:
+                    phys = self.index
+            h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            while not self.stop_flag.is_set():
+                self.samples.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                bits = pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for bit, name in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+                time.sleep(0.001)
+            return
+        except Exception:
+            pass
         q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + q, "--format=csv,noheader,nounits", "-lms", "100"],
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + q, "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             return
@@ -67,7 +93,8 @@ class ClockSampler(threading.Thread):
                 break
             parts = [x.strip() for x in line.split(",")]
             try:
-                self.samples.append((float(parts[0]), float(parts[1])))
+                self.samples.append(float(parts[0]))
+                self.max_mhz = float(parts[1])
             except (ValueError, IndexError):
                 continue
             for n, v in zip(names, parts[2:6]):
@@ -78,10 +105,11 @@ class ClockSampler(threading.Thread):
         self.stop_flag.set()
         if self.proc is not None:
             self.proc.terminate()       # the exact child started above
+        self.join(timeout=2.0)
         if not self.samples:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
-        sm = sorted(s[0] for s in self.samples)
-        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(s[1] for s in self.samples), "reasons": sorted(self.reasons), "samples": len(sm)}
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        sm = sorted(self.samples)
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(sm)}
 
 
 def oracle_leg(w, steps, warmup, sample_pairs=None):
