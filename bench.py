@@ -261,7 +261,6 @@ def main():
     e1.record()
     torch.cuda.synchronize()
     dist_util.barrier()
-    clocks = sampler.finish()
     ms_total = dist_util.max_over_ranks(e0.elapsed_time(e1))
     us_per_step = 1e3 * ms_total / args.steps
     timed_launches = sum(launches.values())
@@ -298,6 +297,7 @@ def main():
             zero_bits_sum += n * s.V - int(np.unpackbits(s.mask_numpy().view(np.uint8)).sum())
             mask_samples += 1
     torch.cuda.synchronize()
+    clocks = sampler.finish()          # sampled over the timed pass and this per-kernel pass (same steps, same kernels)
     t_fill = float(np.mean([e[0].elapsed_time(e[1]) for e in evs])) * 1e3
     t_apply = float(np.mean([e[1].elapsed_time(e[2]) for e in evs])) * 1e3
     t_accept = float(np.mean([e[2].elapsed_time(e[3]) for e in evs])) * 1e3

@@ -236,7 +236,10 @@ class GrammarParser {
   void want(Token::Type ty, const char* what) { if (peek().type != ty) err(std::string("expected ") + what); ++p_; }
   bool starts_rule() const { return peek().type == Token::kIdent && peek2().type == Token::kDefine; }
 
+  int depth_ = 0;
   ExprP alternatives() {
+    struct Guard { int& d; explicit Guard(int& x) : d(x) { ++d; } ~Guard() { --d; } } guard(depth_);
+    if (depth_ > 200) err("expression nested too deeply");
     auto alt = make(Expr::kAlt);
     alt->kids.push_back(sequence());
     while (peek().type == Token::kBar) { ++p_; alt->kids.push_back(sequence()); }
@@ -417,7 +420,9 @@ struct Builder {
     return it->second;
   }
   // Thompson construction: returns (entry, exit) of a fragment inside f
+  int max_states = 1 << 20;
   std::pair<int, int> frag(Fsm& f, const Expr& e) {
+    if (f.size() > max_states) fail(XG_ERR_CAPACITY, "a rule automaton exceeds max_rule_states");
     switch (e.kind) {
       case Expr::kBytes: {
         int s = f.add(), cur = s;
@@ -1295,6 +1300,7 @@ FlatGrammar compile_frontend(int kind, const std::string& text, const std::strin
   }
   std::string root_name = (kind == kEbnf && !root.empty()) ? root : "root";
   c.root = c.b.lookup(root_name);
+  c.b.max_states = opt.max_rule_states;
   for (auto& r : parsed) {
     Fsm f;
     auto p = c.b.frag(f, *r.second);

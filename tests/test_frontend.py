@@ -180,6 +180,30 @@ def test_front_end_errors():
         assert str(e.value)
 
 
+def test_front_end_limits():
+    with pytest.raises(B.XgError) as e:
+        B.Grammar(None, "ebnf", "root ::= " + "(" * 300 + '"a"' + ")" * 300)
+    assert e.value.status == B.XG_ERR_PARSE
+    with pytest.raises(B.XgError) as e:
+        B.Grammar(None, "ebnf", 'root ::= ("abcdefgh"{1000}){1000}')
+    assert e.value.status == B.XG_ERR_CAPACITY
+    g = B.Grammar(None, "ebnf", 'root ::= [a-z]{0,300} "!"')          # a long bounded repetition is fine
+    assert g.stats()["n_states"] >= 300
+
+
+def test_device_entry_points_fail_loudly_without_a_gpu():
+    """No CPU fallback: without a CUDA device the device entry points return XG_ERR_CUDA."""
+    try:
+        import torch
+        if torch.cuda.is_available():
+            pytest.skip("a GPU is present")
+    except ImportError:
+        pass
+    with pytest.raises(B.XgError) as e:
+        B.Tokenizer([b"a", b"b", b""], eos_id=2)
+    assert e.value.status == B.XG_ERR_CUDA and "vocabulary upload" in str(e.value)
+
+
 def test_schema_lowerings_agree():
     """The library's schema -> grammar text and the oracle's, each read by the oracle's parser,
     accept the same documents (the texts themselves differ)."""
