@@ -360,6 +360,7 @@ def main():
         "cache_build": {"seconds": build_ms / 1e3, "compile_wall_s": compile_s, "pairs_classified": pairs, "pairs_per_s": pairs / max(build_ms / 1e3, 1e-9),
                         "pairs_dense": pairs_dense, "pairs_dense_per_s": pairs_dense / max(build_ms / 1e3, 1e-9),
                         "entries_built": sum(x["n_entries_built"] for x in stats), "entries_reused": sum(x["n_entries_reused"] for x in stats),
+                        "uncertain_total": sum(x["total_uncertain"] for x in stats), "uncertain_after_lookahead": sum(x["total_checked"] for x in stats),
                         "cache_bytes_unique_upper": sum(x["cache_bytes"] for x in stats)},
         "roofline": roofline,
         "e2e": {"value": e2e_us, "unit": "us/step", "h2d_bytes_per_step": bytes_one + 4 * n, "d2h_bytes_per_step": bytes_one, "steps": e2e_steps},

@@ -161,6 +161,8 @@ typedef struct {
   int32_t pad;
   int64_t cache_bytes;          /* device bytes of this grammar's entries (shared ones included) */
   double frontend_ms, cache_build_ms;   /* host front end; GPU classification + packing */
+  int64_t total_checked;        /* uncertain tokens left after this grammar's lookahead narrowed the lists (Section 3.3):
+                                   what the per-step check actually streams; <= total_uncertain */
 } xg_grammar_stats_t;
 xg_status_t xg_grammar_stats(const xg_grammar_t* g, xg_grammar_stats_t* out);
 

@@ -78,6 +78,7 @@ struct xg_grammar {
   GrammarDev host_view{};               // device pointers
   GrammarDev* dev = nullptr;            // the same struct in device memory
   void* blob = nullptr;
+  void* lookahead_arena = nullptr;      // this grammar's narrowed check lists
   xg_grammar_stats_t stats{};
   // buffers behind xg_grammar_get_cache_entry's view
   mutable std::vector<int32_t> view_list, view_unc;
@@ -211,17 +212,15 @@ static xg_status_t upload_grammar(xg_grammar* g) {
     r.info = (uint32_t)f.state_rule[s] | (f.state_final[s] ? 0x80000000u : 0u);
     r.edge0_class = n_scan ? scan[f.scan_begin[s]].x : 0; r.edge0_target = n_scan ? scan[f.scan_begin[s]].y : 0;
   }
-  std::vector<uint32_t> state_first((size_t)f.n_states * 8, 0);
-  for (int s = 0; s < f.n_states; ++s)
-    for (int e = f.scan_begin[s]; e < f.scan_begin[s + 1]; ++e)
-      for (int w = 0; w < 8; ++w) state_first[(size_t)s * 8 + w] |= f.class_bits[(size_t)f.scan_class[e] * 8 + w];
-  size_t o_first = reserve(state_first.size() * 4);
+  const std::vector<uint32_t>& state_first = f.state_first;
+  size_t o_first = reserve(state_first.size() * 4), o_follow = reserve(f.rule_follow.size() * 4);
   size_t o_rec = reserve(recs.size() * sizeof(StateRec)), o_scan = reserve(scan.size() * sizeof(uint2)), o_wait = reserve(wait.size() * sizeof(uint2)),
          o_gs = reserve(f.gather_state.size() * 4), o_cb = reserve(f.class_bits.size() * 4),
          o_en = reserve((size_t)f.n_states * sizeof(EntryDev)), o_self = reserve(sizeof(GrammarDev));
   std::vector<uint8_t> host(total, 0);
   auto put = [&](size_t at, const void* src, size_t bytes) { if (bytes) std::memcpy(host.data() + at, src, bytes); };
   put(o_first, state_first.data(), state_first.size() * 4);
+  put(o_follow, f.rule_follow.data(), f.rule_follow.size() * 4);
   put(o_rec, recs.data(), recs.size() * sizeof(StateRec));
   put(o_scan, scan.data(), scan.size() * sizeof(uint2));
   put(o_wait, wait.data(), wait.size() * sizeof(uint2));
@@ -239,6 +238,7 @@ static xg_status_t upload_grammar(xg_grammar* g) {
   v.gather_state = (const int32_t*)(d + o_gs);
   v.class_bits = (const uint32_t*)(d + o_cb);
   v.state_first = (const uint32_t*)(d + o_first);
+  v.rule_follow = (const uint32_t*)(d + o_follow);
   v.entries = (const EntryDev*)(d + o_en);
   put(o_self, &v, sizeof(GrammarDev));
   g->dev = (GrammarDev*)(d + o_self);
@@ -322,6 +322,45 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
   }
   cleanup();
 #undef XG_CUDA_C
+  return XG_OK;
+}
+
+// Lookahead pass (Section 3.3): the pool's entries are context-free; each grammar narrows their
+// uncertain lists with its own follow sets.  Count, exclusive scan on the host (a few thousand
+// numbers), compact.  The grammar's entry headers must already be on the device.
+static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>& scannable, cudaStream_t stream) {
+  std::vector<int32_t> states;
+  for (int s : scannable) if (g->entries[s].n_unc > 0) states.push_back(s);
+  if (states.empty()) return XG_OK;
+  const int n = (int)states.size();
+  if (n > 2000000) return set_error(XG_ERR_CAPACITY, "too many cache entries with uncertain tokens");
+  CachePool& pool = *g->pool;
+  int32_t* d_states = (int32_t*)pool.scratch(11, (size_t)n * 4);
+  int32_t* d_counts = (int32_t*)pool.scratch(12, (size_t)n * 4);
+  long long* d_offsets = (long long*)pool.scratch(13, (size_t)n * 8);
+  if (!d_states || !d_counts || !d_offsets) return set_error(XG_ERR_OOM, "lookahead scratch allocation failed");
+  XG_CUDA(cudaMemcpyAsync(d_states, states.data(), (size_t)n * 4, cudaMemcpyHostToDevice, stream));
+  lookahead_count_kernel<<<n, 256, 0, stream>>>(g->host_view, g->tok->dev, d_states, d_counts);
+  XG_CUDA(cudaGetLastError());
+  std::vector<int32_t> counts(n);
+  XG_CUDA(cudaMemcpyAsync(counts.data(), d_counts, (size_t)n * 4, cudaMemcpyDeviceToHost, stream));
+  XG_CUDA(cudaStreamSynchronize(stream));
+  std::vector<long long> offsets(n);
+  long long total = 0;
+  for (int k = 0; k < n; ++k) { offsets[k] = total; total += 2LL * counts[k] + (counts[k] + 3) / 4; }
+  XG_CUDA(cudaMalloc(&g->lookahead_arena, (size_t)std::max<long long>(total, 1) * 4));
+  XG_CUDA(cudaMemcpyAsync(d_offsets, offsets.data(), (size_t)n * 8, cudaMemcpyHostToDevice, stream));
+  lookahead_compact_kernel<<<n, 256, 0, stream>>>(g->host_view, g->tok->dev, d_states, d_offsets, d_counts, (uint32_t*)g->lookahead_arena);
+  XG_CUDA(cudaGetLastError());
+  XG_CUDA(cudaStreamSynchronize(stream));
+  uint32_t* arena = (uint32_t*)g->lookahead_arena;
+  for (int k = 0; k < n; ++k) {
+    EntryDev& e = g->entries[states[k]];
+    e.chk_rank = arena + offsets[k];
+    e.chk_exit = e.chk_rank + counts[k];
+    e.chk_byte = reinterpret_cast<const uint8_t*>(e.chk_exit + counts[k]);
+    e.n_chk = counts[k];
+  }
   return XG_OK;
 }
 
@@ -416,6 +455,8 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     ++g->stats.n_entries_reused;
   }
   st = upload_grammar(g.get());       // now with the entry headers
+  if (st == XG_OK) st = narrow_check_lists(g.get(), scannable, (cudaStream_t)stream);
+  if (st == XG_OK) st = upload_grammar(g.get());       // and with this grammar's narrowed check lists
   if (st != XG_OK) { xg_grammar_destroy(g.release()); return st; }
   g->stats.cache_build_ms = now_ms() - t1;
   g->stats.n_entries_built = (int)to_build.size();
@@ -425,6 +466,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     const int2 c = g->entry_counts[s];
     g->stats.total_accepted += c.x;
     g->stats.total_uncertain += c.y;
+    g->stats.total_checked += e.n_chk;
     g->stats.total_rejected += tok->vocab_size - c.x - c.y;
     g->stats.kind_count[e.kind]++;
     g->stats.cache_bytes += 4LL * ((e.kind == 2 ? tok->n_words : e.n_list) + 3LL * e.n_unc + (e.n_unc + 3) / 4);
@@ -436,6 +478,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
 void xg_grammar_destroy(xg_grammar_t* g) {
   if (!g) return;
   cudaFree(g->blob);
+  cudaFree(g->lookahead_arena);
   delete g;
 }
 

@@ -28,6 +28,14 @@ struct EntryDev {
   const uint32_t* unc_rank;  // [n_unc] ascending ranks
   const uint32_t* unc_exit;  // [n_unc] parallel to unc_rank: bit j = the token leaves the entry's rule after j bytes
   const uint8_t* unc_byte;   // [n_unc] parallel to unc_rank: the token's byte at its first exit (what the context must scan)
+  // The list the run-time check walks.  In the pool it is the uncertain list itself; a grammar
+  // narrows it with its own lookahead (Section 3.3): exits whose next byte can never follow the
+  // rule anywhere in that grammar are dropped, and tokens left without an exit with them.
+  const uint32_t* chk_rank;
+  const uint32_t* chk_exit;
+  const uint8_t* chk_byte;
+  int32_t n_chk;
+  int32_t pad2;
   int32_t kind;              // xg_store_kind_t
   int32_t n_list;            // list length (0 for bitset)
   int32_t n_unc;
@@ -59,6 +67,7 @@ struct GrammarDev {
   const int32_t* gather_state;    // bit 31: a predicted start state (its items begin in the current set)
   const uint32_t* class_bits;     // [C][8]
   const uint32_t* state_first;    // [S][8] bytes that the state's scan list (own and predicted edges) can take
+  const uint32_t* rule_follow;    // [R][8] bytes that can follow a completed rule somewhere in this grammar
   const EntryDev* entries;        // [S]; meaningful for scannable states
 };
 

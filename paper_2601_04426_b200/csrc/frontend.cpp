@@ -989,6 +989,25 @@ struct Compiler {
       g.wait_begin.push_back((int)g.wait_rule.size());
       g.gather_begin.push_back((int)g.gather_state.size());
     }
+    g.state_first.assign((size_t)S * 8, 0);
+    for (int s = 0; s < S; ++s)
+      for (int e = g.scan_begin[s]; e < g.scan_begin[s + 1]; ++e)
+        for (int w = 0; w < 8; ++w) g.state_first[(size_t)s * 8 + w] |= g.class_bits[(size_t)g.scan_class[e] * 8 + w];
+    g.rule_follow.assign((size_t)R * 8, 0);
+    bool changed = true;
+    while (changed) {
+      changed = false;
+      for (int s = 0; s < S; ++s)
+        for (int e = g.redge_begin[s]; e < g.redge_begin[s + 1]; ++e) {
+          const int r = g.redge_rule[e], t = g.redge_target[e];
+          for (int w = 0; w < 8; ++w) {
+            uint32_t add = g.state_first[(size_t)t * 8 + w];
+            if (g.state_final[t]) add |= g.rule_follow[(size_t)g.state_rule[t] * 8 + w];
+            uint32_t& dst = g.rule_follow[(size_t)r * 8 + w];
+            if ((dst | add) != dst) { dst |= add; changed = true; }
+          }
+        }
+    }
   }
 };
 

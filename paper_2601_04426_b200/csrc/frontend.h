@@ -60,6 +60,10 @@ struct FlatGrammar {
   std::vector<int32_t> wait_begin;
   std::vector<uint32_t> wait_rule, wait_target;
   std::vector<int32_t> gather_begin, gather_state;
+  // state_first[s] = bytes the scan list of s (own and predicted edges) can take; rule_follow[r] = bytes that can
+  // come right after rule r completes, anywhere in this grammar (the lookahead of Section 3.3): the first bytes
+  // of every state a reference to r leads to, plus, where that state is accepting, the follow set of its own rule
+  std::vector<uint32_t> state_first, rule_follow;          // [S][8], [R][8]
 };
 
 enum GrammarKind { kEbnf = 0, kJsonSchema = 1, kTagDispatchJson = 2 };

@@ -362,6 +362,7 @@ pack_kernel(const uint32_t* __restrict__ acc_id, const uint32_t* __restrict__ un
     e.data = data; e.unc_id = out_uid; e.unc_rank = out_urank; e.unc_exit = out_urank + pl.n_unc;
     e.unc_byte = reinterpret_cast<const uint8_t*>(out_urank + 2 * (size_t)pl.n_unc);
     e.kind = pl.kind; e.n_list = pl.n_list; e.n_unc = pl.n_unc; e.n_acc = pl.n_acc;
+    e.chk_rank = e.unc_rank; e.chk_exit = e.unc_exit; e.chk_byte = e.unc_byte; e.n_chk = pl.n_unc; e.pad2 = 0;
     entries[p] = e;
   }
 }
@@ -402,6 +403,76 @@ exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, con
   }
 }
 
+// Lookahead (Section 3.3): narrow each entry's uncertain list with the grammar's follow set of
+// the entry's rule.  An exit survives iff the byte after it can follow the rule somewhere in this
+// grammar; a token survives iff it keeps an exit (tokens without an exit record are kept).
+// First pass counts, second pass compacts in list order.
+__device__ __forceinline__ uint32_t narrow_exits(const VocabDev& v, const uint32_t* __restrict__ follow, int rank, uint32_t exits) {
+  if (exits == 0) return 0;
+  const uint32_t off = v.offset[rank];
+  uint32_t keep = 0;
+  for (uint32_t left = exits; left; left &= left - 1) {
+    const int at = __ffs(left) - 1;
+    const uint32_t byte = v.bytes[off + at];
+    if ((follow[byte >> 5] >> (byte & 31)) & 1u) keep |= 1u << at;
+  }
+  return keep;
+}
+
+__global__ void __launch_bounds__(256)
+lookahead_count_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ states, int32_t* __restrict__ counts) {
+  __shared__ int sh[8];
+  const int q = states[blockIdx.x];
+  const EntryDev e = g.entries[q];
+  const uint32_t* follow = g.rule_follow + (size_t)(g.state[q].info & 0x7FFFFFFFu) * 8;
+  int mine = 0;
+  for (int k = threadIdx.x; k < e.n_unc; k += blockDim.x) {
+    const uint32_t exits = e.unc_exit[k];
+    mine += (exits == 0 || narrow_exits(v, follow, (int)e.unc_rank[k], exits) != 0) ? 1 : 0;
+  }
+  mine = block_reduce_sum(mine, sh);
+  if (threadIdx.x == 0) counts[blockIdx.x] = mine;
+}
+
+__global__ void __launch_bounds__(256)
+lookahead_compact_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ states, const long long* __restrict__ offsets,
+                         const int32_t* __restrict__ counts, uint32_t* __restrict__ arena) {
+  __shared__ int sh_scan[256];
+  const int q = states[blockIdx.x];
+  const EntryDev e = g.entries[q];
+  const uint32_t* follow = g.rule_follow + (size_t)(g.state[q].info & 0x7FFFFFFFu) * 8;
+  const int n_out = counts[blockIdx.x];
+  uint32_t* out_rank = arena + offsets[blockIdx.x];
+  uint32_t* out_exit = out_rank + n_out;
+  uint8_t* out_byte = reinterpret_cast<uint8_t*>(out_exit + n_out);
+  const int per = (e.n_unc + blockDim.x - 1) / blockDim.x;
+  const int lo = min(e.n_unc, (int)threadIdx.x * per), hi = min(e.n_unc, lo + per);
+  int mine = 0;
+  for (int k = lo; k < hi; ++k) {
+    const uint32_t exits = e.unc_exit[k];
+    mine += (exits == 0 || narrow_exits(v, follow, (int)e.unc_rank[k], exits) != 0) ? 1 : 0;
+  }
+  sh_scan[threadIdx.x] = mine;
+  __syncthreads();
+  for (int off = 1; off < (int)blockDim.x; off <<= 1) {
+    int add = (int)threadIdx.x >= off ? sh_scan[threadIdx.x - off] : 0;
+    __syncthreads();
+    sh_scan[threadIdx.x] += add;
+    __syncthreads();
+  }
+  int at = sh_scan[threadIdx.x] - mine;
+  for (int k = lo; k < hi; ++k) {
+    const uint32_t exits = e.unc_exit[k];
+    const int rank = (int)e.unc_rank[k];
+    const uint32_t keep = narrow_exits(v, follow, rank, exits);
+    if (exits != 0 && keep == 0) continue;
+    out_rank[at] = (uint32_t)rank;
+    out_exit[at] = keep;
+    out_byte[at] = keep ? v.bytes[v.offset[rank] + __ffs(keep) - 1] : 0;
+    ++at;
+  }
+}
+
 // ------------------------------------------------------------------------------------------
 // matcher state
 // ------------------------------------------------------------------------------------------
@@ -437,7 +508,7 @@ __device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g,
         bool seen = false;
         for (int z = 0; z < n_merge; ++z) seen = seen || p.merge_state[z] == q;
         if (!seen) { if (n_merge == kPlanMergeMax) { overflow = 1; break; } p.merge_state[n_merge++] = q; }
-        const int n_unc = g.entries[q].n_unc;
+        const int n_unc = g.entries[q].n_chk;
         if (n_unc == 0) continue;
         seen = false;
         for (int z = 0; z < n_check; ++z) seen = seen || (p.check_state[z] == q && p.check_origin[z] == origin);
@@ -672,7 +743,7 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
     // the plan's arrays for the live entries, copied with coalesced loads
     for (int i = threadIdx.x; i < n_ent; i += blockDim.x) {
       const EntryDev& e = g.entries[plan.check_state[i]];
-      ent_rank[i] = e.unc_rank; ent_exit[i] = e.unc_exit;
+      ent_rank[i] = e.chk_rank; ent_exit[i] = e.chk_exit;
       cont_cnt[i] = plan.cont_cnt[i];
     }
     for (int i = threadIdx.x; i <= n_ent; i += blockDim.x) ent_cum[i] = plan.check_cum[i];
@@ -855,7 +926,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
     const uint32_t* class_bits = stage_class_bits(g, sh_class);
     for (int i = threadIdx.x; i < n_ent; i += blockDim.x) {
       const EntryDev& e = g.entries[plan.check_state[i]];
-      ent_rank[i] = e.unc_rank; ent_exit[i] = e.unc_exit; ent_byte[i] = e.unc_byte;
+      ent_rank[i] = e.chk_rank; ent_exit[i] = e.chk_exit; ent_byte[i] = e.chk_byte;
       cont_cnt[i] = plan.cont_cnt[i];
     }
     for (int i = threadIdx.x; i <= n_ent; i += blockDim.x) ent_cum[i] = plan.check_cum[i];
