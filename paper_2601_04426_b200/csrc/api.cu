@@ -650,8 +650,12 @@ xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t ba
   const int W = tok->n_words;
   if ((W + kClusterBlocks - 1) / kClusterBlocks <= kMergeMaxChunkWords) {
     // one launch: a cluster of eight blocks per request keeps the row in distributed shared memory
-    fill_cluster_kernel<<<dim3(kClusterBlocks, batch), 256, 0, (cudaStream_t)stream>>>(slot->dev_matchers, tok->dev, bitmask_dev,
-                                                                                      (long long)row_stride_words, status_dev);
+    // eight blocks per request; 128 threads each once the batch alone fills the machine (a block
+    // of 256 threads halves the number of requests in flight), 256 for small batches (latency)
+    const int threads = batch >= 64 ? 128 : 256;
+    const size_t smem = 2 * sizeof(uint32_t) * (size_t)((W + kClusterBlocks - 1) / kClusterBlocks);
+    fill_cluster_kernel<<<dim3(kClusterBlocks, batch), threads, smem, (cudaStream_t)stream>>>(slot->dev_matchers, tok->dev, bitmask_dev,
+                                                                                             (long long)row_stride_words, status_dev);
     XG_CUDA(cudaGetLastError());
     return XG_OK;
   }

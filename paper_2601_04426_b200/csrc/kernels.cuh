@@ -857,8 +857,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
                     int32_t* __restrict__ status_user) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
-  __shared__ uint32_t row[kMergeMaxChunkWords];
-  __shared__ uint32_t tmp[kMergeMaxChunkWords];
+  extern __shared__ uint32_t dyn_smem[];          // this block's row slice and a scratch slice: 2 x ceil(W / 8) words
   __shared__ const uint32_t* ent_rank[kPlanCheckMax];
   __shared__ const uint32_t* ent_exit[kPlanCheckMax];
   __shared__ const uint8_t* ent_byte[kPlanCheckMax];
@@ -870,7 +869,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   __shared__ uint32_t sh_class[kSharedClasses * 8];
   // uncertain tokens too long for the per-thread arrays (33..255 bytes; rare) are queued and walked one at a time
   // by thread 0 in this block-wide scratch
-  constexpr int kLongQueue = 32, kLongCap = 1024;
+  constexpr int kLongQueue = 32, kLongCap = 512;
   __shared__ int long_q[kLongQueue];
   __shared__ int long_n;
   __shared__ uint32_t long_st[kLongCap];
@@ -884,6 +883,8 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   const GrammarDev& g = *m.grammar;
   const StepPlan& plan = *m.plan;
   const int chunk = (v.n_words + kClusterBlocks - 1) / kClusterBlocks;
+  uint32_t* row = dyn_smem;
+  uint32_t* tmp = dyn_smem + chunk;
   const int w0 = rank * chunk, w1 = min(v.n_words, w0 + chunk);
   const int nw = max(0, w1 - w0);
   for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] = 0;
