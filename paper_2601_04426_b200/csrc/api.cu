@@ -648,15 +648,27 @@ xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t ba
   if (st != XG_OK) return st;
   if (!bitmask_dev || row_stride_words < tok->n_words) return set_error(XG_ERR_INVALID_ARG, "bad bitmask buffer");
   const int W = tok->n_words;
-  if ((W + kClusterBlocks - 1) / kClusterBlocks <= kMergeMaxChunkWords) {
-    // one launch: a cluster of eight blocks per request keeps the row in distributed shared memory
-    // eight blocks per request; 128 threads each once the batch alone fills the machine (a block
-    // of 256 threads halves the number of requests in flight), 256 for small batches (latency)
-    const int threads = batch >= 64 ? 128 : 256;
-    const size_t smem = 2 * sizeof(uint32_t) * (size_t)((W + kClusterBlocks - 1) / kClusterBlocks);
-    fill_cluster_kernel<<<dim3(kClusterBlocks, batch), threads, smem, (cudaStream_t)stream>>>(slot->dev_matchers, tok->dev, bitmask_dev,
-                                                                                             (long long)row_stride_words, status_dev);
-    XG_CUDA(cudaGetLastError());
+  if ((W + kMaxClusterBlocks - 1) / kMaxClusterBlocks <= kMergeMaxChunkWords) {
+    // One launch: a cluster of blocks per request keeps the row in distributed shared memory.
+    // Eight blocks per request; 256 threads each while that leaves the whole batch resident (the
+    // kernel runs at 64 registers per thread: 1024 threads per SM), else 128.
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int per_request = sms * 1024 / batch;
+    int blocks = kMaxClusterBlocks, threads = 256;
+    if (per_request < 2048) threads = 128;     // measured: fewer blocks or narrower blocks than this are slower even at batch 256
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks, batch);
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = 2 * sizeof(uint32_t) * (size_t)((W + blocks - 1) / blocks);
+    cfg.stream = (cudaStream_t)stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = blocks; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    XG_CUDA(cudaLaunchKernelEx(&cfg, fill_cluster_kernel, (MatcherDev* const*)slot->dev_matchers, tok->dev, bitmask_dev,
+                               (long long)row_stride_words, status_dev));
     return XG_OK;
   }
   int chunks = std::max((W + kMergeMaxChunkWords - 1) / kMergeMaxChunkWords, std::min(8, (W + 127) / 128));

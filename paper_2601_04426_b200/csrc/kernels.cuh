@@ -839,25 +839,26 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
 }
 
 // ------------------------------------------------------------------------------------------
-// Per-step mask in one launch: a thread-block cluster of eight blocks per request.  Block r of
-// the cluster keeps slice r of the request's row in its shared memory.
+// Per-step mask in one launch: a thread-block cluster of two to eight blocks per request.  Block
+// r of the cluster keeps slice r of the request's row in its shared memory.
 //   1. every block merges the accepted sets of the plan's entries into its own slice;
 //   2. cluster barrier; the blocks share the uncertain candidates (trie order, one token per
 //      lane); a token that passes is OR-ed into the slice of the block that owns its id, through
 //      distributed shared memory;
 //   3. cluster barrier; every block writes its slice with coalesced stores.
 // No global atomics, no scratch words, and the row never makes a round trip through L2.
-// Used when a slice fits (vocabularies up to 8 x 2048 x 32 tokens); larger vocabularies take the
-// two-kernel path above.
+// The host picks cluster and block size so that the whole batch is resident at once.  Used when
+// a slice fits (at most 2048 words per block); larger vocabularies take the two-kernel path above.
 // ------------------------------------------------------------------------------------------
-constexpr int kClusterBlocks = 8;
+constexpr int kMaxClusterBlocks = 8;      // the portable cluster size limit
 
-__global__ void __cluster_dims__(kClusterBlocks, 1, 1) __launch_bounds__(256, 4)
+// launched with a cluster of gridDim.x blocks (2, 4 or 8) along x
+__global__ void __launch_bounds__(256, 4)
 fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __restrict__ bitmask, long long row_stride,
                     int32_t* __restrict__ status_user) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
-  extern __shared__ uint32_t dyn_smem[];          // this block's row slice and a scratch slice: 2 x ceil(W / 8) words
+  extern __shared__ uint32_t dyn_smem[];          // this block's row slice and a scratch slice: 2 x ceil(W / blocks) words
   __shared__ const uint32_t* ent_rank[kPlanCheckMax];
   __shared__ const uint32_t* ent_exit[kPlanCheckMax];
   __shared__ const uint8_t* ent_byte[kPlanCheckMax];
@@ -882,7 +883,8 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   const MatcherDev& m = *matchers[b];
   const GrammarDev& g = *m.grammar;
   const StepPlan& plan = *m.plan;
-  const int chunk = (v.n_words + kClusterBlocks - 1) / kClusterBlocks;
+  const int n_blocks = (int)gridDim.x;
+  const int chunk = (v.n_words + n_blocks - 1) / n_blocks;
   uint32_t* row = dyn_smem;
   uint32_t* tmp = dyn_smem + chunk;
   const int w0 = rank * chunk, w1 = min(v.n_words, w0 + chunk);
@@ -937,7 +939,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
     }
     for (int i = threadIdx.x; i < n_ent * 8; i += blockDim.x) (&cont_first[0][0])[i] = (&plan.cont_first[0][0])[i];
     cluster.sync();            // every slice is merged (and this block's staging is visible)
-    const int stride = kClusterBlocks * blockDim.x;
+    const int stride = n_blocks * blockDim.x;
     auto walk_one = [&](int trank, uint32_t off, int e, int at) {
       const int len = (int)(v.offset[trank + 1] - off);
       bool pass = false, overflow = len - at > kFastMaxBytes;
