@@ -81,6 +81,19 @@ void xg_tokenizer_destroy(xg_tokenizer_t* tok);
  * A pool belongs to one tokenizer and must outlive the grammars compiled with it. */
 xg_status_t xg_cache_pool_create(const xg_tokenizer_t* tok, xg_cache_pool_t** out);
 void xg_cache_pool_destroy(xg_cache_pool_t* pool);
+/* Size limit of the pool's device memory (Section 3.3: at the limit the least recently used entries
+ * are evicted).  Entries are evicted in the batches they were built in, oldest use first, and only
+ * once no live grammar uses any entry of the batch; a later compile rebuilds what it misses.
+ * max_bytes <= 0: no limit (the default).  May synchronise the device when it evicts. */
+xg_status_t xg_cache_pool_set_limit(xg_cache_pool_t* pool, int64_t max_bytes);
+typedef struct {
+  int64_t bytes;             /* device bytes held now */
+  int64_t evicted_bytes;     /* total evicted so far */
+  int64_t evicted_chunks;
+  int32_t live_rules;        /* rule automata whose entries are in the pool */
+  int32_t chunks;            /* batches of entries held now */
+} xg_cache_pool_stats_t;
+xg_status_t xg_cache_pool_stats(xg_cache_pool_t* pool, xg_cache_pool_stats_t* out);
 
 typedef struct {
   uint32_t struct_size;       /* sizeof(xg_compile_options_t), for versioning */

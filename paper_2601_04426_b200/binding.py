@@ -25,7 +25,7 @@ KIND_BY_NAME = {"ebnf": XG_EBNF, "json_schema": XG_JSON_SCHEMA, "tag_dispatch": 
 DTYPE_BY_NAME = {"f32": XG_F32, "bf16": XG_BF16}
 
 EXPORTS = [
-    "xg_last_error", "xg_tokenizer_create", "xg_tokenizer_destroy", "xg_cache_pool_create", "xg_cache_pool_destroy",
+    "xg_last_error", "xg_tokenizer_create", "xg_tokenizer_destroy", "xg_cache_pool_create", "xg_cache_pool_destroy", "xg_cache_pool_set_limit", "xg_cache_pool_stats",
     "xg_compile_grammar", "xg_grammar_destroy", "xg_grammar_get_tables", "xg_grammar_get_rule_hashes", "xg_grammar_get_cache_entry", "xg_grammar_stats",
     "xg_matcher_create", "xg_matcher_reset", "xg_matcher_destroy", "xg_matcher_is_terminated",
     "xg_fill_next_token_bitmask", "xg_fill_next_token_bitmask_static", "xg_apply_token_bitmask", "xg_accept_token",
@@ -45,6 +45,10 @@ class CompileOptions(C.Structure):
 
 class MatcherOptions(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("max_sets", C.c_int32), ("max_items", C.c_int32)]
+
+
+class PoolStats(C.Structure):
+    _fields_ = [("bytes", C.c_int64), ("evicted_bytes", C.c_int64), ("evicted_chunks", C.c_int64), ("live_rules", C.c_int32), ("chunks", C.c_int32)]
 
 
 class GrammarTables(C.Structure):
@@ -85,6 +89,8 @@ def lib():
         L.xg_cache_pool_create.argtypes = [vp, C.POINTER(vp)]
         L.xg_cache_pool_destroy.argtypes = [vp]
         L.xg_cache_pool_destroy.restype = None
+        L.xg_cache_pool_set_limit.argtypes = [vp, i64]
+        L.xg_cache_pool_stats.argtypes = [vp, C.POINTER(PoolStats)]
         L.xg_compile_grammar.argtypes = [vp, vp, C.c_int, C.c_char_p, C.c_size_t, C.c_char_p, C.POINTER(CompileOptions), vp, C.POINTER(vp)]
         L.xg_grammar_destroy.argtypes = [vp]
         L.xg_grammar_destroy.restype = None
@@ -135,6 +141,14 @@ class CachePool:
         h = C.c_void_p()
         _check(lib().xg_cache_pool_create(tokenizer.h, C.byref(h)))
         self.h = h
+
+    def set_limit(self, max_bytes: int):
+        _check(lib().xg_cache_pool_set_limit(self.h, int(max_bytes)))
+
+    def stats(self) -> dict:
+        s = PoolStats()
+        _check(lib().xg_cache_pool_stats(self.h, C.byref(s)))
+        return {n: getattr(s, n) for n, _ in PoolStats._fields_}
 
     def close(self):
         if getattr(self, "h", None):

@@ -79,6 +79,8 @@ struct xg_grammar {
   GrammarDev* dev = nullptr;            // the same struct in device memory
   void* blob = nullptr;
   void* lookahead_arena = nullptr;      // this grammar's narrowed check lists
+  std::vector<int> entry_chunk;         // [n_states] pool chunk that holds the state's entry (-1: none)
+  std::vector<int> chunk_refs;          // pool chunks this grammar keeps alive
   xg_grammar_stats_t stats{};
   // buffers behind xg_grammar_get_cache_entry's view
   mutable std::vector<int32_t> view_list, view_unc;
@@ -181,6 +183,23 @@ xg_status_t xg_cache_pool_create(const xg_tokenizer_t* tok, xg_cache_pool_t** ou
   return XG_OK;
 }
 void xg_cache_pool_destroy(xg_cache_pool_t* pool) { delete pool; }
+
+xg_status_t xg_cache_pool_set_limit(xg_cache_pool_t* pool, int64_t max_bytes) {
+  if (!pool) return set_error(XG_ERR_INVALID_ARG, "NULL pool");
+  std::lock_guard<std::mutex> lock(pool->impl->mu);
+  pool->impl->set_limit(max_bytes);
+  pool->impl->enforce_limit();
+  return XG_OK;
+}
+
+xg_status_t xg_cache_pool_stats(xg_cache_pool_t* pool, xg_cache_pool_stats_t* out) {
+  if (!pool || !out) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
+  std::lock_guard<std::mutex> lock(pool->impl->mu);
+  const CachePool::Stats s = pool->impl->stats();
+  out->bytes = s.bytes; out->evicted_bytes = s.evicted_bytes; out->evicted_chunks = s.evicted_chunks;
+  out->live_rules = s.live_rules; out->chunks = s.chunks;
+  return XG_OK;
+}
 
 // ---------------------------------------------------------------------------------------------
 // grammar compilation
@@ -308,7 +327,8 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
     long long total_words = 0;
     XG_CUDA_C(cudaMemcpyAsync(&total_words, d_total, sizeof(long long), cudaMemcpyDeviceToHost, stream));
     XG_CUDA_C(cudaStreamSynchronize(stream));
-    uint32_t* arena = (uint32_t*)g->pool->allocate_device((size_t)std::max<long long>(total_words, 1) * 4);
+    int chunk_id = -1;
+    uint32_t* arena = (uint32_t*)g->pool->allocate_device((size_t)std::max<long long>(total_words, 1) * 4, &chunk_id);
     if (!arena) { cleanup(); return set_error(XG_ERR_OOM, "cache arena allocation failed"); }
     pack_kernel<<<n, 256, 0, stream>>>(acc, unc, unr, d_plan, V, W, arena, d_entries);
     exit_kernel<<<n, 256, 0, stream>>>(g->host_view, v, d_pos, d_entries);
@@ -318,7 +338,7 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
     XG_CUDA_C(cudaMemcpyAsync(built.data(), d_entries, n * sizeof(EntryDev), cudaMemcpyDeviceToHost, stream));
     XG_CUDA_C(cudaMemcpyAsync(counts.data(), d_counts, n * sizeof(int2), cudaMemcpyDeviceToHost, stream));
     XG_CUDA_C(cudaStreamSynchronize(stream));
-    for (int k = 0; k < n; ++k) { g->entries[states[begin + k]] = built[k]; g->entry_counts[states[begin + k]] = counts[k]; }
+    for (int k = 0; k < n; ++k) { g->entries[states[begin + k]] = built[k]; g->entry_counts[states[begin + k]] = counts[k]; g->entry_chunk[states[begin + k]] = chunk_id; }
   }
   cleanup();
 #undef XG_CUDA_C
@@ -401,18 +421,26 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   g->pool = pool ? pool->impl : std::make_shared<CachePool>((const void*)tok);
   g->entries.assign(f.n_states, EntryDev{});
   g->entry_counts.assign(f.n_states, make_int2(0, 0));
+  g->entry_chunk.assign(f.n_states, -1);
   const double t1 = now_ms();
   xg_status_t st = upload_grammar(g.get());
   if (st != XG_OK) { xg_grammar_destroy(g.release()); return st; }
   // cross-grammar cache (Section 3.3): rules whose canonical structure is already in the pool
   // reuse its entries; the others are classified now and registered afterwards
-  std::lock_guard<std::mutex> pool_lock(g->pool->mu);
+  const std::shared_ptr<CachePool> pool_keep = g->pool;      // outlives the lock below on every path
+  std::lock_guard<std::mutex> pool_lock(pool_keep->mu);
+  bool retained = false;
+  auto fail = [&](xg_status_t status) {                       // the lock is held: give the chunks back without taking it again
+    if (retained) pool_keep->release_held(g->chunk_refs);
+    g->chunk_refs.clear();
+    xg_grammar_destroy(g.release());
+    return status;
+  };
   RuleInterning in;
   try {
     in = g->pool->intern(f);
   } catch (const std::exception& e) {
-    xg_grammar_destroy(g.release());
-    return set_error(XG_ERR_OOM, e.what());
+    return fail(set_error(XG_ERR_OOM, e.what()));
   }
   std::vector<int> rule_first(f.n_rules + 1, f.n_states);
   for (int s = f.n_states - 1; s >= 0; --s) rule_first[f.state_rule[s]] = s;
@@ -428,6 +456,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
       g->entries[s] = pr.entries[canon_of[s]];
       g->entry_counts[s] = pr.counts[canon_of[s]];
       ++g->stats.n_entries_reused;
+      for (int c : pr.chunks) if (std::find(g->chunk_refs.begin(), g->chunk_refs.end(), c) == g->chunk_refs.end()) g->chunk_refs.push_back(c);
     } else {
       auto it = builder_of.find(in.pool_id[r]);
       if (it == builder_of.end()) it = builder_of.emplace(in.pool_id[r], r).first;
@@ -435,16 +464,25 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     }
   }
   st = build_entries(g.get(), to_build, (cudaStream_t)stream);
-  if (st != XG_OK) { xg_grammar_destroy(g.release()); return st; }
+  if (st != XG_OK) return fail(st);
   for (auto& kv : builder_of) {
     PoolRule& pr = g->pool->rule(kv.first);
     const int r = kv.second;
     const int n_local = (int)in.canon[r].size();
     pr.entries.resize(n_local);
     pr.counts.resize(n_local);
-    for (int k = 0; k < n_local; ++k) { pr.entries[k] = g->entries[rule_first[r] + in.canon[r][k]]; pr.counts[k] = g->entry_counts[rule_first[r] + in.canon[r][k]]; }
+    for (int k = 0; k < n_local; ++k) {
+      const int s = rule_first[r] + in.canon[r][k];
+      pr.entries[k] = g->entries[s]; pr.counts[k] = g->entry_counts[s];
+      const int c = g->entry_chunk[s];
+      if (c >= 0 && std::find(pr.chunks.begin(), pr.chunks.end(), c) == pr.chunks.end()) { pr.chunks.push_back(c); g->pool->note_rule_in_chunk(kv.first, c); }
+    }
+    for (int c : pr.chunks) if (std::find(g->chunk_refs.begin(), g->chunk_refs.end(), c) == g->chunk_refs.end()) g->chunk_refs.push_back(c);
     pr.built = true;
   }
+  g->pool->retain(g->chunk_refs);
+  retained = true;
+  g->pool->enforce_limit();
   for (int s : scannable) {                           // duplicates of a rule inside this grammar
     const int r = f.state_rule[s];
     auto it = builder_of.find(in.pool_id[r]);
@@ -457,7 +495,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   st = upload_grammar(g.get());       // now with the entry headers
   if (st == XG_OK) st = narrow_check_lists(g.get(), scannable, (cudaStream_t)stream);
   if (st == XG_OK) st = upload_grammar(g.get());       // and with this grammar's narrowed check lists
-  if (st != XG_OK) { xg_grammar_destroy(g.release()); return st; }
+  if (st != XG_OK) return fail(st);
   g->stats.cache_build_ms = now_ms() - t1;
   g->stats.n_entries_built = (int)to_build.size();
   g->stats.pairs_classified = (int64_t)to_build.size() * tok->vocab_size;
@@ -479,6 +517,7 @@ void xg_grammar_destroy(xg_grammar_t* g) {
   if (!g) return;
   cudaFree(g->blob);
   cudaFree(g->lookahead_arena);
+  if (g->pool && !g->chunk_refs.empty()) g->pool->release(g->chunk_refs);
   delete g;
 }
 

@@ -17,7 +17,7 @@ uint64_t hash_fold(uint64_t h, uint64_t x) {
 }
 
 CachePool::~CachePool() {
-  for (void* p : chunks_) cudaFree(p);
+  for (auto& c : chunks_) cudaFree(c.ptr);
   for (auto& s : scratch_) cudaFree(s.first);
 }
 
@@ -34,11 +34,61 @@ void* CachePool::scratch(int slot, size_t bytes) {
   return s.first;
 }
 
-void* CachePool::allocate_device(size_t bytes) {
+void* CachePool::allocate_device(size_t bytes, int* chunk_id) {
   void* p = nullptr;
   if (cudaMalloc(&p, bytes) != cudaSuccess) return nullptr;
-  chunks_.push_back(p);
+  Chunk c;
+  c.ptr = p; c.bytes = bytes; c.last_use = ++clock_;
+  chunks_.push_back(c);
+  bytes_ += (long long)bytes;
+  *chunk_id = (int)chunks_.size() - 1;
   return p;
+}
+
+void CachePool::retain(const std::vector<int>& chunk_ids) {
+  for (int c : chunk_ids) { ++chunks_[c].refs; chunks_[c].last_use = ++clock_; }
+}
+
+void CachePool::release(const std::vector<int>& chunk_ids) {
+  std::lock_guard<std::mutex> lock(mu);
+  release_held(chunk_ids);
+}
+
+void CachePool::release_held(const std::vector<int>& chunk_ids) {
+  for (int c : chunk_ids) --chunks_[c].refs;
+  enforce_limit();
+}
+
+void CachePool::enforce_limit() {
+  if (limit_ <= 0) return;
+  while (bytes_ > limit_) {
+    int victim = -1;
+    for (int c = 0; c < (int)chunks_.size(); ++c)
+      if (chunks_[c].ptr && chunks_[c].refs == 0 && (victim < 0 || chunks_[c].last_use < chunks_[victim].last_use)) victim = c;
+    if (victim < 0) return;               // everything left is in use
+    Chunk& ch = chunks_[victim];
+    for (int r : ch.rules) {              // the rules of this chunk leave the pool (a later compile rebuilds them)
+      PoolRule& pr = rules_[r];
+      if (!pr.built) continue;
+      auto& bucket = by_hash_[pr.hash];
+      bucket.erase(std::remove(bucket.begin(), bucket.end(), r), bucket.end());
+      pr.built = false;
+      pr.serial.clear(); pr.entries.clear(); pr.counts.clear(); pr.chunks.clear();
+    }
+    cudaDeviceSynchronize();              // nothing may still be reading the chunk
+    cudaFree(ch.ptr);
+    bytes_ -= (long long)ch.bytes;
+    ++evicted_chunks_; evicted_bytes_ += (long long)ch.bytes;
+    ch.ptr = nullptr; ch.bytes = 0; ch.rules.clear();
+  }
+}
+
+CachePool::Stats CachePool::stats() const {
+  Stats s;
+  s.bytes = bytes_; s.evicted_chunks = evicted_chunks_; s.evicted_bytes = evicted_bytes_;
+  for (auto& r : rules_) s.live_rules += r.built ? 1 : 0;
+  for (auto& c : chunks_) s.chunks += c.ptr ? 1 : 0;
+  return s;
 }
 
 int CachePool::find_or_add(uint64_t hash, std::vector<uint64_t>&& serial) {

@@ -18,6 +18,7 @@ struct PoolRule {
   std::vector<uint64_t> serial;      // canonical serialisation (the exact identity of the rule)
   uint64_t hash = 0;
   bool built = false;
+  std::vector<int> chunks;           // device chunks that hold this rule's entries
   std::vector<EntryDev> entries;     // by canonical state index
   std::vector<int2> counts;          // (accepted, uncertain) by canonical state index
 };
@@ -44,7 +45,18 @@ class CachePool {
   RuleInterning intern(const FlatGrammar& g);
   PoolRule& rule(int id) { return rules_[id]; }
   size_t n_rules() const { return rules_.size(); }
-  void* allocate_device(size_t bytes);      // lives as long as the pool
+  // Device memory for one batch of freshly built entries.  Chunks are the unit of eviction
+  // (Section 3.3 bounds the cross-grammar cache by a size limit with least-recently-used
+  // eviction): a chunk may go once no live grammar uses any entry in it.
+  void* allocate_device(size_t bytes, int* chunk_id);
+  void retain(const std::vector<int>& chunk_ids);          // a grammar starts using these chunks
+  void release(const std::vector<int>& chunk_ids);         // ... and stops (locks `mu` itself)
+  void release_held(const std::vector<int>& chunk_ids);    // the same with `mu` already held
+  void set_limit(long long bytes) { limit_ = bytes; }
+  void enforce_limit();                                      // evict least recently used idle chunks (call with `mu` held)
+  void note_rule_in_chunk(int rule_id, int chunk_id) { chunks_[chunk_id].rules.push_back(rule_id); }
+  struct Stats { long long bytes = 0, evicted_chunks = 0, evicted_bytes = 0; int live_rules = 0, chunks = 0; };
+  Stats stats() const;
   // reusable build scratch (grow-only, one buffer per slot; call with `mu` held)
   void* scratch(int slot, size_t bytes);
 
@@ -52,7 +64,10 @@ class CachePool {
   const void* owner_;
   std::vector<PoolRule> rules_;
   std::unordered_map<uint64_t, std::vector<int>> by_hash_;
-  std::vector<void*> chunks_;
+  struct Chunk { void* ptr = nullptr; size_t bytes = 0; int refs = 0; uint64_t last_use = 0; std::vector<int> rules; };
+  std::vector<Chunk> chunks_;
+  long long limit_ = 0, bytes_ = 0, evicted_chunks_ = 0, evicted_bytes_ = 0;
+  uint64_t clock_ = 0;
   std::vector<std::pair<void*, size_t>> scratch_;
   int find_or_add(uint64_t hash, std::vector<uint64_t>&& serial);
 };

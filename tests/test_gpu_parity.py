@@ -206,6 +206,78 @@ def test_cross_grammar_pool_reuses_entries():
     pool.close(); tok.close()
 
 
+def _scannable(g):
+    t = g.tables()
+    return [s for s in range(t["n_states"]) if t["cedge_begin"][s + 1] > t["cedge_begin"][s]]
+
+
+def _same_entries(a, b, stride=1):
+    for s in _scannable(a)[::stride]:
+        ea, eb = a.cache_entry(s), b.cache_entry(s)
+        assert ea["kind"] == eb["kind"] and np.array_equal(ea["list"], eb["list"]) and np.array_equal(ea["uncertain"], eb["uncertain"]), s
+
+
+def test_pool_limit_never_evicts_entries_in_use():
+    """Section 3.3: the pool has a size limit; eviction must not touch what a live grammar reads."""
+    torch, engine = _engine()
+    w = inputs.make_workload("C3", batch=4, steps=2, vocab_size=4096)
+    v = w.vocab
+    tok = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
+    pool = B.CachePool(tok)
+    shared = [B.Grammar(tok, g.kind, g.text, pool=pool) for g in w.grammars]
+    private = [B.Grammar(tok, g.kind, g.text) for g in w.grammars]
+    before = pool.stats()
+    assert before["bytes"] > 0 and before["evicted_chunks"] == 0 and before["live_rules"] > 0
+    pool.set_limit(1)                           # far below what is held, but all of it is in use
+    assert pool.stats() == before
+    last = shared.pop()
+    last.close()                                # what only this grammar used may go now
+    after = pool.stats()
+    assert after["evicted_chunks"] >= 1 and after["bytes"] < before["bytes"] and after["live_rules"] < before["live_rules"]
+    assert after["bytes"] + after["evicted_bytes"] == before["bytes"]
+    for a, b in zip(shared, private):           # the survivors still read valid memory
+        _same_entries(a, b, stride=17)
+    # the evicted rules are rebuilt on demand, with the same result
+    again = B.Grammar(tok, w.grammars[3].kind, w.grammars[3].text, pool=pool)
+    assert again.stats()["n_entries_built"] > 0
+    _same_entries(again, private[3], stride=7)
+    for g in shared + private + [again]:
+        g.close()
+    assert pool.stats()["bytes"] <= 1 or pool.stats()["chunks"] == 0
+    pool.close(); tok.close()
+
+
+def test_pool_evicts_in_least_recently_used_order():
+    torch, engine = _engine()
+    w = inputs.make_workload("C1", batch=1, steps=2, vocab_size=4096)
+    v = w.vocab
+    tok = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
+    pool = B.CachePool(tok)
+    texts = {k: 'root ::= "%s"+ [0-9]' % k for k in "abc"}
+
+    def compile_and_drop(k):
+        g = B.Grammar(tok, "ebnf", texts[k], pool=pool)
+        built = g.stats()["n_entries_built"]
+        g.close()
+        return built
+
+    assert all(compile_and_drop(k) > 0 for k in "abc")       # use order: a, b, c
+    assert compile_and_drop("a") == 0                        # now: b, c, a
+    s = pool.stats()
+    assert s["chunks"] == 3 and s["evicted_chunks"] == 0
+    pool.set_limit(s["bytes"] - 1)                           # one batch of entries has to go: b's
+    s = pool.stats()
+    assert s["chunks"] == 2 and s["evicted_chunks"] == 1
+    assert compile_and_drop("a") == 0 and compile_and_drop("c") == 0
+    assert compile_and_drop("b") > 0                         # rebuilt; to stay under the limit the oldest idle one (a) went
+    assert pool.stats()["evicted_chunks"] == 2
+    assert compile_and_drop("c") == 0 and compile_and_drop("a") > 0
+    pool.set_limit(0)                                        # no limit again: nothing more is evicted
+    n = pool.stats()["evicted_chunks"]
+    assert compile_and_drop("b") >= 0 and compile_and_drop("c") >= 0 and pool.stats()["evicted_chunks"] == n
+    pool.close(); tok.close()
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("rows,vocab,stride_pad", [(1, 8192, 0), (3, 1000, 8), (5, 32 * 7 + 5, 16), (2, 151936, 0)])
 def test_apply_matches_oracle(dtype, rows, vocab, stride_pad):
