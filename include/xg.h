@@ -84,10 +84,13 @@ void xg_cache_pool_destroy(xg_cache_pool_t* pool);
 /* Size limit of the pool's device memory (Section 3.3: at the limit the least recently used entries
  * are evicted).  Entries are evicted in the batches they were built in, oldest use first, and only
  * once no live grammar uses any entry of the batch; a later compile rebuilds what it misses.
+ * The limit counts the entries' bytes; the pool takes device memory in slabs (at most 64 MiB each)
+ * and returns a slab when nothing in it is live.
  * max_bytes <= 0: no limit (the default).  May synchronise the device when it evicts. */
 xg_status_t xg_cache_pool_set_limit(xg_cache_pool_t* pool, int64_t max_bytes);
 typedef struct {
-  int64_t bytes;             /* device bytes held now */
+  int64_t bytes;             /* bytes of cache entries held now (what the limit bounds) */
+  int64_t reserved_bytes;    /* device memory the pool's slabs hold, grammars' own tables included */
   int64_t evicted_bytes;     /* total evicted so far */
   int64_t evicted_chunks;
   int32_t live_rules;        /* rule automata whose entries are in the pool */

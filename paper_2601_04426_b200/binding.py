@@ -48,7 +48,7 @@ class MatcherOptions(C.Structure):
 
 
 class PoolStats(C.Structure):
-    _fields_ = [("bytes", C.c_int64), ("evicted_bytes", C.c_int64), ("evicted_chunks", C.c_int64), ("live_rules", C.c_int32), ("chunks", C.c_int32)]
+    _fields_ = [("bytes", C.c_int64), ("reserved_bytes", C.c_int64), ("evicted_bytes", C.c_int64), ("evicted_chunks", C.c_int64), ("live_rules", C.c_int32), ("chunks", C.c_int32)]
 
 
 class GrammarTables(C.Structure):

@@ -196,7 +196,7 @@ xg_status_t xg_cache_pool_stats(xg_cache_pool_t* pool, xg_cache_pool_stats_t* ou
   if (!pool || !out) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
   std::lock_guard<std::mutex> lock(pool->impl->mu);
   const CachePool::Stats s = pool->impl->stats();
-  out->bytes = s.bytes; out->evicted_bytes = s.evicted_bytes; out->evicted_chunks = s.evicted_chunks;
+  out->bytes = s.bytes; out->reserved_bytes = s.reserved; out->evicted_bytes = s.evicted_bytes; out->evicted_chunks = s.evicted_chunks;
   out->live_rules = s.live_rules; out->chunks = s.chunks;
   return XG_OK;
 }
@@ -246,7 +246,10 @@ static xg_status_t upload_grammar(xg_grammar* g) {
   put(o_gs, f.gather_state.data(), f.gather_state.size() * 4);
   put(o_cb, f.class_bits.data(), f.class_bits.size() * 4);
   put(o_en, g->entries.data(), g->entries.size() * sizeof(EntryDev));
-  if (!g->blob) XG_CUDA(cudaMalloc(&g->blob, total));
+  if (!g->blob) {                        // from the pool's slabs (the caller holds the pool's lock)
+    g->blob = g->pool->allocate_plain(total);
+    if (!g->blob) return set_error(XG_ERR_OOM, "grammar table allocation failed");
+  }
   uint8_t* d = (uint8_t*)g->blob;
   GrammarDev& v = g->host_view;
   v.n_states = f.n_states; v.n_rules = f.n_rules; v.n_classes = f.n_classes;
@@ -368,7 +371,8 @@ static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>&
   std::vector<long long> offsets(n);
   long long total = 0;
   for (int k = 0; k < n; ++k) { offsets[k] = total; total += 2LL * counts[k] + (counts[k] + 3) / 4; }
-  XG_CUDA(cudaMalloc(&g->lookahead_arena, (size_t)std::max<long long>(total, 1) * 4));
+  g->lookahead_arena = pool.allocate_plain((size_t)std::max<long long>(total, 1) * 4);
+  if (!g->lookahead_arena) return set_error(XG_ERR_OOM, "check list allocation failed");
   XG_CUDA(cudaMemcpyAsync(d_offsets, offsets.data(), (size_t)n * 8, cudaMemcpyHostToDevice, stream));
   lookahead_compact_kernel<<<n, 256, 0, stream>>>(g->host_view, g->tok->dev, d_states, d_offsets, d_counts, (uint32_t*)g->lookahead_arena);
   XG_CUDA(cudaGetLastError());
@@ -423,19 +427,22 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   g->entry_counts.assign(f.n_states, make_int2(0, 0));
   g->entry_chunk.assign(f.n_states, -1);
   const double t1 = now_ms();
-  xg_status_t st = upload_grammar(g.get());
-  if (st != XG_OK) { xg_grammar_destroy(g.release()); return st; }
-  // cross-grammar cache (Section 3.3): rules whose canonical structure is already in the pool
-  // reuse its entries; the others are classified now and registered afterwards
   const std::shared_ptr<CachePool> pool_keep = g->pool;      // outlives the lock below on every path
   std::lock_guard<std::mutex> pool_lock(pool_keep->mu);
   bool retained = false;
-  auto fail = [&](xg_status_t status) {                       // the lock is held: give the chunks back without taking it again
+  auto fail = [&](xg_status_t status) {                       // the lock is held: give everything back without taking it again
+    cudaDeviceSynchronize();
     if (retained) pool_keep->release_held(g->chunk_refs);
     g->chunk_refs.clear();
+    pool_keep->free_plain(g->blob); pool_keep->free_plain(g->lookahead_arena);
+    g->blob = g->lookahead_arena = nullptr;
     xg_grammar_destroy(g.release());
     return status;
   };
+  xg_status_t st = upload_grammar(g.get());
+  if (st != XG_OK) return fail(st);
+  // cross-grammar cache (Section 3.3): rules whose canonical structure is already in the pool
+  // reuse its entries; the others are classified now and registered afterwards
   RuleInterning in;
   try {
     in = g->pool->intern(f);
@@ -515,9 +522,13 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
 
 void xg_grammar_destroy(xg_grammar_t* g) {
   if (!g) return;
-  cudaFree(g->blob);
-  cudaFree(g->lookahead_arena);
-  if (g->pool && !g->chunk_refs.empty()) g->pool->release(g->chunk_refs);
+  if (g->pool && (g->blob || g->lookahead_arena || !g->chunk_refs.empty())) {
+    cudaDeviceSynchronize();             // its tables go back to the pool's slabs: nothing may still read them
+    std::lock_guard<std::mutex> lock(g->pool->mu);
+    g->pool->free_plain(g->blob);
+    g->pool->free_plain(g->lookahead_arena);
+    g->pool->release_held(g->chunk_refs);
+  }
   delete g;
 }
 

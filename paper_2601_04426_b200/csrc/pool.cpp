@@ -2,6 +2,7 @@
 
 #include <algorithm>
 #include <functional>
+#include <iterator>
 
 namespace xg {
 
@@ -16,8 +17,72 @@ uint64_t hash_fold(uint64_t h, uint64_t x) {
   return z ^ (z >> 31);
 }
 
+DeviceArena::~DeviceArena() {
+  for (auto& s : slabs_) if (s.base) cudaFree(s.base);
+}
+
+void* DeviceArena::alloc(size_t bytes) {
+  bytes = (std::max<size_t>(bytes, 1) + 255) & ~size_t(255);
+  int slab = -1;
+  size_t offset = 0;
+  for (int i = 0; i < (int)slabs_.size() && slab < 0; ++i) {
+    if (!slabs_[i].base || slabs_[i].bytes - slabs_[i].used < bytes) continue;
+    for (auto& blk : slabs_[i].free_blocks)
+      if (blk.second >= bytes) { slab = i; offset = blk.first; break; }
+  }
+  if (slab < 0) {
+    const size_t want = std::max(bytes, std::min<size_t>(size_t(64) << 20, std::max<size_t>(size_t(1) << 20, reserved_)));
+    void* base = nullptr;
+    size_t got = want;
+    if (cudaMalloc(&base, got) != cudaSuccess) {
+      cudaGetLastError();
+      got = bytes;
+      if (got == want || cudaMalloc(&base, got) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    }
+    for (slab = 0; slab < (int)slabs_.size() && slabs_[slab].base; ++slab) {}
+    if (slab == (int)slabs_.size()) slabs_.emplace_back();
+    Slab& s = slabs_[slab];
+    s.base = (char*)base; s.bytes = got; s.used = 0;
+    s.free_blocks.clear();
+    s.free_blocks[0] = got;
+    reserved_ += got;
+    offset = 0;
+  }
+  Slab& s = slabs_[slab];
+  const size_t len = s.free_blocks[offset];
+  s.free_blocks.erase(offset);
+  if (len > bytes) s.free_blocks[offset + bytes] = len - bytes;
+  s.used += bytes;
+  void* p = s.base + offset;
+  live_[p] = std::make_pair(slab, bytes);
+  return p;
+}
+
+void DeviceArena::free(void* p) {
+  auto it = live_.find(p);
+  if (it == live_.end()) return;
+  const int slab = it->second.first;
+  size_t bytes = it->second.second;
+  live_.erase(it);
+  Slab& s = slabs_[slab];
+  s.used -= bytes;
+  if (s.used == 0) {                     // nothing left in it: back to the driver
+    cudaFree(s.base);
+    reserved_ -= s.bytes;
+    s = Slab();
+    return;
+  }
+  size_t offset = (size_t)((char*)p - s.base);
+  auto next = s.free_blocks.lower_bound(offset);
+  if (next != s.free_blocks.end() && offset + bytes == next->first) { bytes += next->second; next = s.free_blocks.erase(next); }
+  if (next != s.free_blocks.begin()) {
+    auto prev = std::prev(next);
+    if (prev->first + prev->second == offset) { prev->second += bytes; return; }
+  }
+  s.free_blocks[offset] = bytes;
+}
+
 CachePool::~CachePool() {
-  for (auto& c : chunks_) cudaFree(c.ptr);
   for (auto& s : scratch_) cudaFree(s.first);
 }
 
@@ -35,8 +100,8 @@ void* CachePool::scratch(int slot, size_t bytes) {
 }
 
 void* CachePool::allocate_device(size_t bytes, int* chunk_id) {
-  void* p = nullptr;
-  if (cudaMalloc(&p, bytes) != cudaSuccess) return nullptr;
+  void* p = arena_.alloc(bytes);
+  if (!p) return nullptr;
   Chunk c;
   c.ptr = p; c.bytes = bytes; c.last_use = ++clock_;
   chunks_.push_back(c);
@@ -76,7 +141,7 @@ void CachePool::enforce_limit() {
       pr.serial.clear(); pr.entries.clear(); pr.counts.clear(); pr.chunks.clear();
     }
     cudaDeviceSynchronize();              // nothing may still be reading the chunk
-    cudaFree(ch.ptr);
+    arena_.free(ch.ptr);
     bytes_ -= (long long)ch.bytes;
     ++evicted_chunks_; evicted_bytes_ += (long long)ch.bytes;
     ch.ptr = nullptr; ch.bytes = 0; ch.rules.clear();
@@ -85,7 +150,7 @@ void CachePool::enforce_limit() {
 
 CachePool::Stats CachePool::stats() const {
   Stats s;
-  s.bytes = bytes_; s.evicted_chunks = evicted_chunks_; s.evicted_bytes = evicted_bytes_;
+  s.bytes = bytes_; s.reserved = (long long)arena_.reserved(); s.evicted_chunks = evicted_chunks_; s.evicted_bytes = evicted_bytes_;
   for (auto& r : rules_) s.live_rules += r.built ? 1 : 0;
   for (auto& c : chunks_) s.chunks += c.ptr ? 1 : 0;
   return s;

@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <map>
 #include <mutex>
 #include <unordered_map>
 #include <vector>
@@ -34,6 +35,25 @@ struct RuleInterning {
 // graph, Algorithm 2's refinement on cycles.
 RuleInterning structural_hashes(const FlatGrammar& g);
 
+// Device memory in slabs with a first-fit free list.  Compiling a grammar needs a handful of
+// device buffers (its tables, a batch of cache entries, its narrowed check lists); taking each
+// from the driver costs a driver allocation apiece, which on a busy host takes from tens of
+// microseconds to tens of milliseconds.  Slabs grow geometrically up to 64 MiB, so a pool that
+// serves many grammars asks the driver a few dozen times in its life.  Not thread-safe: the
+// owner serialises calls.
+class DeviceArena {
+ public:
+  ~DeviceArena();
+  void* alloc(size_t bytes);            // 256-byte aligned; nullptr when the device is out of memory
+  void free(void* p);                   // p from alloc(); an empty slab goes back to the driver
+  size_t reserved() const { return reserved_; }
+ private:
+  struct Slab { char* base = nullptr; size_t bytes = 0, used = 0; std::map<size_t, size_t> free_blocks; };   // offset -> length
+  std::vector<Slab> slabs_;
+  std::unordered_map<void*, std::pair<int, size_t>> live_;      // block -> (slab, bytes)
+  size_t reserved_ = 0;
+};
+
 class CachePool {
  public:
   explicit CachePool(const void* owner) : owner_(owner) {}
@@ -49,13 +69,16 @@ class CachePool {
   // (Section 3.3 bounds the cross-grammar cache by a size limit with least-recently-used
   // eviction): a chunk may go once no live grammar uses any entry in it.
   void* allocate_device(size_t bytes, int* chunk_id);
+  // Plain device memory from the pool's slabs for a grammar's own tables (not subject to the limit).
+  void* allocate_plain(size_t bytes) { return arena_.alloc(bytes); }
+  void free_plain(void* p) { if (p) arena_.free(p); }
   void retain(const std::vector<int>& chunk_ids);          // a grammar starts using these chunks
   void release(const std::vector<int>& chunk_ids);         // ... and stops (locks `mu` itself)
   void release_held(const std::vector<int>& chunk_ids);    // the same with `mu` already held
   void set_limit(long long bytes) { limit_ = bytes; }
   void enforce_limit();                                      // evict least recently used idle chunks (call with `mu` held)
   void note_rule_in_chunk(int rule_id, int chunk_id) { chunks_[chunk_id].rules.push_back(rule_id); }
-  struct Stats { long long bytes = 0, evicted_chunks = 0, evicted_bytes = 0; int live_rules = 0, chunks = 0; };
+  struct Stats { long long bytes = 0, reserved = 0, evicted_chunks = 0, evicted_bytes = 0; int live_rules = 0, chunks = 0; };
   Stats stats() const;
   // reusable build scratch (grow-only, one buffer per slot; call with `mu` held)
   void* scratch(int slot, size_t bytes);
@@ -66,6 +89,7 @@ class CachePool {
   std::unordered_map<uint64_t, std::vector<int>> by_hash_;
   struct Chunk { void* ptr = nullptr; size_t bytes = 0; int refs = 0; uint64_t last_use = 0; std::vector<int> rules; };
   std::vector<Chunk> chunks_;
+  DeviceArena arena_;
   long long limit_ = 0, bytes_ = 0, evicted_chunks_ = 0, evicted_bytes_ = 0;
   uint64_t clock_ = 0;
   std::vector<std::pair<void*, size_t>> scratch_;
