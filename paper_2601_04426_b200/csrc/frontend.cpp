@@ -13,6 +13,7 @@
 #include <map>
 #include <memory>
 #include <set>
+#include <unordered_map>
 
 #include "xg.h"
 
@@ -538,15 +539,16 @@ Fsm determinize(const Fsm& f, int max_states) {
   Fsm d;
   d.has_tag_dispatch = f.has_tag_dispatch;
   std::map<std::vector<int>, int> index;
+  std::vector<int> single(f.size(), -1);              // subsets of one state, the common case
   std::vector<std::vector<int>> subsets;
   auto state_of = [&](std::vector<int>& set) {
     std::sort(set.begin(), set.end());
     set.erase(std::unique(set.begin(), set.end()), set.end());
-    auto it = index.find(set);
-    if (it != index.end()) return it->second;
+    if (set.size() == 1) { if (single[set[0]] >= 0) return single[set[0]]; }
+    else { auto it = index.find(set); if (it != index.end()) return it->second; }
     int id = d.add();
     if (id >= max_states) fail(XG_ERR_CAPACITY, "a rule automaton exceeds max_rule_states");
-    index[set] = id;
+    if (set.size() == 1) single[set[0]] = id; else index[set] = id;
     subsets.push_back(set);
     for (int s : set) if (f.fin[s]) d.fin[id] = 1;
     return id;
@@ -595,6 +597,73 @@ Fsm determinize(const Fsm& f, int max_states) {
   return d;
 }
 
+// Equal word sequences get equal ids, numbered in order of first appearance.
+struct SignatureTable {
+  std::unordered_map<uint64_t, std::vector<int>> buckets;
+  std::vector<uint32_t> words;                         // every distinct signature, back to back
+  std::vector<std::pair<size_t, size_t>> span;         // id -> (begin, length)
+  int size() const { return (int)span.size(); }
+  int intern(const std::vector<uint32_t>& sig) {
+    uint64_t h = 0x9E3779B97F4A7C15ull ^ sig.size();
+    for (uint32_t x : sig) { h ^= x; h *= 0xBF58476D1CE4E5B9ull; h ^= h >> 29; }
+    std::vector<int>& bucket = buckets[h];
+    for (int id : bucket)
+      if (span[id].second == sig.size() && std::equal(sig.begin(), sig.end(), words.begin() + span[id].first)) return id;
+    const int id = (int)span.size();
+    span.emplace_back(words.size(), sig.size());
+    words.insert(words.end(), sig.begin(), sig.end());
+    bucket.push_back(id);
+    return id;
+  }
+};
+
+// The outgoing edges of state s with targets replaced by their class: byte sets merged per
+// class (ascending class), then the reference edges (ascending rule, class).
+struct ClassEdges {
+  std::vector<std::pair<int, ByteSet>> bytes;
+  std::vector<std::pair<int, int>> refs;
+  void collect(const Fsm& f, int s, const std::vector<int>& cls) {
+    bytes.clear(); refs.clear();
+    for (const Edge& e : f.out[s]) {
+      if (e.kind == Edge::kBytes) {
+        const int c = cls[e.to];
+        size_t k = 0;
+        while (k < bytes.size() && bytes[k].first != c) ++k;
+        if (k == bytes.size()) bytes.emplace_back(c, e.set); else bytes[k].second.merge(e.set);
+      } else refs.emplace_back(e.rule, cls[e.to]);
+    }
+    std::sort(bytes.begin(), bytes.end(), [](const std::pair<int, ByteSet>& a, const std::pair<int, ByteSet>& b) { return a.first < b.first; });
+    std::sort(refs.begin(), refs.end());
+  }
+  void signature(int head, std::vector<uint32_t>& sig) const {
+    sig.clear();
+    sig.push_back((uint32_t)head);
+    sig.push_back((uint32_t)bytes.size());
+    for (auto& b : bytes) { sig.push_back((uint32_t)b.first); sig.insert(sig.end(), b.second.w.begin(), b.second.w.end()); }
+    for (auto& r : refs) { sig.push_back((uint32_t)r.first); sig.push_back((uint32_t)r.second); }
+  }
+};
+
+// the quotient automaton of a partition (classes numbered 0 .. n_cls-1)
+Fsm quotient(const Fsm& f, const std::vector<int>& cls, int n_cls) {
+  Fsm m;
+  m.has_tag_dispatch = f.has_tag_dispatch;
+  for (int b = 0; b < n_cls; ++b) m.add();
+  std::vector<char> done(n_cls, 0);
+  m.start = cls[f.start];
+  ClassEdges ce;
+  for (int s = 0; s < f.size(); ++s) {
+    const int b = cls[s];
+    if (f.fin[s]) m.fin[b] = 1;
+    if (done[b]) continue;
+    done[b] = 1;
+    ce.collect(f, s, cls);
+    for (const Edge& e : f.out[s]) if (e.kind == Edge::kRef) m.ref(b, e.rule, cls[e.to]);
+    for (auto& kv : ce.bytes) m.bytes(b, kv.second, kv.first);
+  }
+  return m;
+}
+
 // Minimisation of an acyclic deterministic automaton in one bottom-up pass: in reverse
 // topological order, two states are equivalent iff they agree on acceptance and on their edges
 // into already-merged targets.  Returns false (and leaves `out` alone) if the automaton has a cycle.
@@ -605,96 +674,92 @@ bool minimize_acyclic(const Fsm& f, Fsm& out) {
   for (int s = 0; s < n; ++s) if (!indeg[s]) order.push_back(s);
   for (size_t q = 0; q < order.size(); ++q) for (const Edge& e : f.out[order[q]]) if (--indeg[e.to] == 0) order.push_back(e.to);
   if ((int)order.size() != n) return false;
-  typedef std::pair<std::vector<std::pair<int, ByteSet>>, std::vector<std::pair<int, int>>> Sig;
-  std::map<std::pair<int, Sig>, int> cls_of;
+  SignatureTable table;
   std::vector<int> cls(n, -1);
+  ClassEdges ce;
+  std::vector<uint32_t> sig;
   for (int k = n - 1; k >= 0; --k) {
     const int s = order[k];
-    std::map<int, ByteSet> by_cls;
-    std::vector<std::pair<int, int>> refs;
-    for (const Edge& e : f.out[s]) {
-      if (e.kind == Edge::kBytes) by_cls[cls[e.to]].merge(e.set);
-      else refs.emplace_back(e.rule, cls[e.to]);
-    }
-    std::sort(refs.begin(), refs.end());
-    auto key = std::make_pair((int)f.fin[s], Sig{std::vector<std::pair<int, ByteSet>>(by_cls.begin(), by_cls.end()), refs});
-    auto it = cls_of.find(key);
-    if (it == cls_of.end()) it = cls_of.emplace(key, (int)cls_of.size()).first;
-    cls[s] = it->second;
+    ce.collect(f, s, cls);
+    ce.signature((int)f.fin[s], sig);
+    cls[s] = table.intern(sig);
   }
-  Fsm m;
-  m.has_tag_dispatch = f.has_tag_dispatch;
-  const int n_cls = (int)cls_of.size();
-  for (int b = 0; b < n_cls; ++b) m.add();
-  std::vector<char> done(n_cls, 0);
-  m.start = cls[f.start];
-  for (int s = 0; s < n; ++s) {
-    const int b = cls[s];
-    if (f.fin[s]) m.fin[b] = 1;
-    if (done[b]) continue;
-    done[b] = 1;
-    std::map<int, ByteSet> by_cls;
-    for (const Edge& e : f.out[s]) {
-      if (e.kind == Edge::kBytes) by_cls[cls[e.to]].merge(e.set);
-      else m.ref(b, e.rule, cls[e.to]);
-    }
-    for (auto& kv : by_cls) m.bytes(b, kv.second, kv.first);
-  }
-  out = m;
+  out = quotient(f, cls, table.size());
   return true;
 }
 
-// merge equivalent states of a deterministic automaton (partition refinement on sparse signatures)
+// Merge equivalent states of a deterministic automaton: partition refinement on sparse
+// signatures.  A state's signature (its edges with targets replaced by their blocks) is only
+// recomputed after one of its targets changed block, and when a block splits the largest part
+// keeps the block's id, so a state changes id O(log n) times.
 Fsm minimize(const Fsm& f) {
   {
     Fsm quick;
     if (minimize_acyclic(f, quick)) return quick;
   }
-  int n = f.size();
+  const int n = f.size();
+  std::vector<std::vector<int>> pred(n);
+  for (int s = 0; s < n; ++s) for (const Edge& e : f.out[s]) pred[e.to].push_back(s);
   std::vector<int> block(n);
-  for (int s = 0; s < n; ++s) block[s] = f.fin[s] ? 1 : 0;
-  int n_blocks = 0;
-  typedef std::pair<std::vector<std::pair<int, ByteSet>>, std::vector<std::pair<int, int>>> Sig;
-  while (true) {
-    std::map<std::pair<int, Sig>, int> sig_id;
-    std::vector<int> nb(n);
+  std::vector<std::vector<int>> members;
+  {
+    int id_of[2] = {-1, -1};
     for (int s = 0; s < n; ++s) {
-      std::map<int, ByteSet> by_block;
-      std::vector<std::pair<int, int>> refs;
-      for (const Edge& e : f.out[s]) {
-        if (e.kind == Edge::kBytes) by_block[block[e.to]].merge(e.set);
-        else refs.emplace_back(e.rule, block[e.to]);
+      int& id = id_of[f.fin[s] ? 1 : 0];
+      if (id < 0) { id = (int)members.size(); members.emplace_back(); }
+      block[s] = id;
+      members[id].push_back(s);
+    }
+  }
+  SignatureTable table;
+  std::vector<int> sig_id(n, -1), work(n), touched;
+  std::vector<char> queued(n, 1), block_touched;
+  for (int s = 0; s < n; ++s) work[s] = s;
+  ClassEdges ce;
+  std::vector<uint32_t> sig;
+  while (!work.empty()) {
+    touched.clear();
+    block_touched.assign(members.size(), 0);
+    for (int s : work) {
+      ce.collect(f, s, block);
+      ce.signature(0, sig);
+      sig_id[s] = table.intern(sig);
+      queued[s] = 0;
+      if (!block_touched[block[s]]) { block_touched[block[s]] = 1; touched.push_back(block[s]); }
+    }
+    work.clear();
+    for (int b : touched) {
+      {
+        std::vector<int>& in_place = members[b];
+        std::sort(in_place.begin(), in_place.end(), [&](int x, int y) { return sig_id[x] != sig_id[y] ? sig_id[x] < sig_id[y] : x < y; });
+        if (sig_id[in_place.front()] == sig_id[in_place.back()]) continue;
       }
-      std::sort(refs.begin(), refs.end());
-      Sig sig{std::vector<std::pair<int, ByteSet>>(by_block.begin(), by_block.end()), refs};
-      auto key = std::make_pair(block[s], sig);
-      auto it = sig_id.find(key);
-      if (it == sig_id.end()) it = sig_id.emplace(key, (int)sig_id.size()).first;
-      nb[s] = it->second;
+      const std::vector<int> mem = members[b];      // a copy: `members` grows below
+      size_t best_begin = 0, best_len = 0;                    // the largest part stays
+      for (size_t i = 0; i < mem.size();) {
+        size_t j = i;
+        while (j < mem.size() && sig_id[mem[j]] == sig_id[mem[i]]) ++j;
+        if (j - i > best_len) { best_len = j - i; best_begin = i; }
+        i = j;
+      }
+      std::vector<int> stay(mem.begin() + best_begin, mem.begin() + best_begin + best_len);
+      for (size_t i = 0; i < mem.size();) {
+        size_t j = i;
+        while (j < mem.size() && sig_id[mem[j]] == sig_id[mem[i]]) ++j;
+        if (i != best_begin) {
+          const int id = (int)members.size();
+          members.emplace_back(mem.begin() + i, mem.begin() + j);
+          for (size_t k = i; k < j; ++k) {
+            block[mem[k]] = id;
+            for (int p : pred[mem[k]]) if (!queued[p]) { queued[p] = 1; work.push_back(p); }
+          }
+        }
+        i = j;
+      }
+      members[b] = stay;
     }
-    int count = (int)sig_id.size();
-    block = nb;
-    if (count == n_blocks) break;
-    n_blocks = count;
   }
-  Fsm m;
-  m.has_tag_dispatch = f.has_tag_dispatch;
-  for (int b = 0; b < n_blocks; ++b) m.add();
-  std::vector<char> done(n_blocks, 0);
-  m.start = block[f.start];
-  for (int s = 0; s < n; ++s) {
-    int b = block[s];
-    if (f.fin[s]) m.fin[b] = 1;
-    if (done[b]) continue;
-    done[b] = 1;
-    std::map<int, ByteSet> by_block;
-    for (const Edge& e : f.out[s]) {
-      if (e.kind == Edge::kBytes) by_block[block[e.to]].merge(e.set);
-      else m.ref(b, e.rule, block[e.to]);
-    }
-    for (auto& kv : by_block) m.bytes(b, kv.second, kv.first);
-  }
-  return m;
+  return quotient(f, block, (int)members.size());
 }
 
 // breadth-first renumbering from the start state with edges in a fixed order; drops unreachable
@@ -784,8 +849,10 @@ struct Compiler {
 
   // Rules that derive at least one string; then: drop references to the others, and every state
   // that cannot reach an accepting state.
-  void trim() {
+  // Returns, per rule, whether anything was removed (an untouched rule keeps its automaton as is).
+  std::vector<char> trim() {
     int R = n_rules();
+    std::vector<char> touched(R, 0);
     std::vector<char> productive(R, 0);
     auto live_states = [&](const Fsm& f) {
       int n = f.size();
@@ -826,8 +893,12 @@ struct Compiler {
           g.out[id[s]].push_back(c);
         }
       }
-      f = g;
+      size_t edges_before = 0, edges_after = 0;
+      for (auto& es : f.out) edges_before += es.size();
+      for (auto& es : g.out) edges_after += es.size();
+      if (g.size() != f.size() || edges_after != edges_before) { f = g; touched[r] = 1; }
     }
+    return touched;
   }
 
   // for each rule, whether it can reach itself through references
@@ -856,7 +927,8 @@ struct Compiler {
   // A rule used a few times may also be somewhat larger as long as size x uses stays bounded
   // (a character rule repeated by a bounded string must not stay a rule of its own: every
   // multi-byte token would leave it and become context-dependent).
-  void inline_small_rules() {
+  void inline_small_rules(std::vector<char>& renormalized) {
+    renormalized.assign(n_rules(), 0);
     if (opt.inline_max_states <= 0) return;
     const int single_use_max = std::max(64, opt.inline_max_states);
     int R = n_rules();
@@ -897,7 +969,7 @@ struct Compiler {
         }
         g.out[s] = keep;
       }
-      if (changed) b.rules[r] = normalize(g, opt.max_rule_states);
+      if (changed) { b.rules[r] = normalize(g, opt.max_rule_states); renormalized[r] = 1; }
       candidate[r] = !rec[r] && r != root && b.rules[r].size() <= single_use_max;
     };
     for (int r = 0; r < R; ++r) process(r);
@@ -1330,10 +1402,11 @@ FlatGrammar compile_frontend(int kind, const std::string& text, const std::strin
   }
   c.remove_nullability();
   for (Fsm& f : c.b.rules) f = normalize(f, opt.max_rule_states);
-  c.trim();
-  c.inline_small_rules();
-  c.trim();
-  for (Fsm& f : c.b.rules) f = canonical_order(minimize(f));
+  std::vector<char> stale = c.trim(), renormalized;           // stale: trimmed since it was last minimised
+  c.inline_small_rules(renormalized);
+  const std::vector<char> trimmed_again = c.trim();
+  for (int r = 0; r < c.n_rules(); ++r)
+    if (trimmed_again[r] || (stale[r] && !renormalized[r])) c.b.rules[r] = canonical_order(minimize(c.b.rules[r]));
   return c.flatten();
 }
 
