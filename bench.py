@@ -30,7 +30,8 @@ if ROOT not in sys.path:
 from paper_2601_04426_b200 import inputs  # noqa: E402
 
 SHAPES = {"C1": (1, 8192), "C2": (1, 128256), "C3": (128, 151936), "C4": (64, 128256), "C5": (256, 200064),
-          "T5": (16, 128256), "T20": (16, 128256), "T50": (16, 128256), "T100": (16, 128256)}
+          "T5": (16, 128256), "T20": (16, 128256), "T50": (16, 128256), "T100": (16, 128256),
+          "R256": (16, 128256), "R1024": (16, 128256), "R4096": (16, 128256)}
 
 
 def measured_peaks():
@@ -153,6 +154,8 @@ def main():
     ap.add_argument("--workload", default="C3", choices=sorted(SHAPES))
     ap.add_argument("--batch", type=int, default=None, help="shrink the batch (debugging only; the line then names it)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-state-compression", action="store_true",
+                    help="build one cache entry per scannable state (ablation of the repetition state compression)")
     args = ap.parse_args()
     warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
@@ -191,7 +194,7 @@ def main():
     wt.close()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
-    s = engine.Session(w, device="cuda:%d" % local_rank)
+    s = engine.Session(w, device="cuda:%d" % local_rank, state_compression=not args.no_state_compression)
     torch.cuda.synchronize()
     compile_s = time.perf_counter() - t0
     stats = [g.stats() for g in s.grammars]
@@ -385,6 +388,8 @@ def main():
         "cache_build": {"seconds": build_ms / 1e3, "compile_wall_s": compile_s, "pairs_classified": pairs, "pairs_per_s": pairs / max(build_ms / 1e3, 1e-9),
                         "pairs_dense": pairs_dense, "pairs_dense_per_s": pairs_dense / max(build_ms / 1e3, 1e-9),
                         "entries_built": sum(x["n_entries_built"] for x in stats), "entries_reused": sum(x["n_entries_reused"] for x in stats),
+                        "entries_shared_by_state_compression": sum(x["n_entries_shared"] for x in stats), "states": sum(x["n_states"] for x in stats),
+                        "frontend_ms": sum(x["frontend_ms"] for x in stats),
                         "uncertain_total": sum(x["total_uncertain"] for x in stats), "uncertain_after_lookahead": sum(x["total_checked"] for x in stats),
                         "cache_bytes_unique_upper": sum(x["cache_bytes"] for x in stats)},
         "roofline": roofline,

@@ -104,6 +104,8 @@ typedef struct {
                                  states into their users; 0 = never; negative = default (16). */
   int32_t max_rule_states;    /* XG_ERR_CAPACITY if one rule's automaton grows past this.  <= 0 = default (1<<20). */
   int32_t build_cache;        /* 0 = front end only (tables, no device work).  Otherwise build. */
+  int32_t no_state_compression; /* non-zero: build one cache entry per scannable state even where repetition
+                                 state compression (Section 3.6) would let states share one. */
 } xg_compile_options_t;
 
 /* ---- grammar compilation (Section 3.5 "compilation stage"; Sections 3.2, 3.3, 3.4) ---------
@@ -152,6 +154,16 @@ xg_status_t xg_grammar_get_tables(const xg_grammar_t* g, xg_grammar_tables_t* ho
  * compares canonical serialisations, so a collision can never share an entry. */
 xg_status_t xg_grammar_get_rule_hashes(const xg_grammar_t* g, uint64_t* out);
 
+/* Repetition state compression (Section 3.6).  A bounded repetition R{l,r} is kept as explicit
+ * automaton states (the count k of the paper's state (R{l,r}, k) is the state itself), but cache
+ * entries are built once per class of states that no token can tell apart: states of one rule
+ * whose automata agree when unrolled `depth` edges deep.  With depth = the longest token in bytes
+ * their accepted / rejected / uncertain sets are identical, so inside a long repetition only the
+ * copies within `depth` of the bounds get entries of their own.  out (host, [n_states]): for each
+ * state the smallest state of its class.  depth < 0: the tokenizer's longest token (grammars
+ * compiled without a tokenizer: XG_ERR_INVALID_ARG).  Host work only. */
+xg_status_t xg_grammar_get_state_classes(const xg_grammar_t* g, int32_t depth, int32_t* out);
+
 /* One cache entry, copied to the host (valid until the next call on this grammar or its
  * destruction).  list = accepted ids (XG_STORE_ACCEPT_LIST) or rejected ids
  * (XG_STORE_REJECT_LIST), ascending; bitset = accepted bits (XG_STORE_BITSET), ceil(V/32) words;
@@ -179,6 +191,8 @@ typedef struct {
   double frontend_ms, cache_build_ms;   /* host front end; GPU classification + packing */
   int64_t total_checked;        /* uncertain tokens left after this grammar's lookahead narrowed the lists (Section 3.3):
                                    what the per-step check actually streams; <= total_uncertain */
+  int64_t n_entries_shared;     /* scannable states that use the entry of an equivalent state of their rule
+                                   (repetition state compression, Section 3.6) instead of one of their own */
 } xg_grammar_stats_t;
 xg_status_t xg_grammar_stats(const xg_grammar_t* g, xg_grammar_stats_t* out);
 

@@ -26,7 +26,7 @@ DTYPE_BY_NAME = {"f32": XG_F32, "bf16": XG_BF16}
 
 EXPORTS = [
     "xg_last_error", "xg_tokenizer_create", "xg_tokenizer_destroy", "xg_cache_pool_create", "xg_cache_pool_destroy", "xg_cache_pool_set_limit", "xg_cache_pool_stats",
-    "xg_compile_grammar", "xg_grammar_destroy", "xg_grammar_get_tables", "xg_grammar_get_rule_hashes", "xg_grammar_get_cache_entry", "xg_grammar_stats",
+    "xg_compile_grammar", "xg_grammar_destroy", "xg_grammar_get_tables", "xg_grammar_get_rule_hashes", "xg_grammar_get_cache_entry", "xg_grammar_get_state_classes", "xg_grammar_stats",
     "xg_matcher_create", "xg_matcher_reset", "xg_matcher_destroy", "xg_matcher_is_terminated",
     "xg_fill_next_token_bitmask", "xg_fill_next_token_bitmask_static", "xg_apply_token_bitmask", "xg_accept_token",
 ]
@@ -40,7 +40,8 @@ class XgError(RuntimeError):
 
 
 class CompileOptions(C.Structure):
-    _fields_ = [("struct_size", C.c_uint32), ("inline_max_states", C.c_int32), ("max_rule_states", C.c_int32), ("build_cache", C.c_int32)]
+    _fields_ = [("struct_size", C.c_uint32), ("inline_max_states", C.c_int32), ("max_rule_states", C.c_int32), ("build_cache", C.c_int32),
+                ("no_state_compression", C.c_int32)]
 
 
 class MatcherOptions(C.Structure):
@@ -65,7 +66,8 @@ class CacheEntryView(C.Structure):
 class GrammarStats(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_rules", "n_states", "n_scannable", "n_classes", "n_entries_built", "n_entries_reused")] + \
                [(n, C.c_int64) for n in ("pairs_classified", "total_accepted", "total_rejected", "total_uncertain")] + \
-               [("kind_count", C.c_int32 * 3), ("pad", C.c_int32), ("cache_bytes", C.c_int64), ("frontend_ms", C.c_double), ("cache_build_ms", C.c_double), ("total_checked", C.c_int64)]
+               [("kind_count", C.c_int32 * 3), ("pad", C.c_int32), ("cache_bytes", C.c_int64), ("frontend_ms", C.c_double), ("cache_build_ms", C.c_double), ("total_checked", C.c_int64),
+                ("n_entries_shared", C.c_int64)]
 
 
 _lib = None
@@ -97,6 +99,7 @@ def lib():
         L.xg_grammar_get_tables.argtypes = [vp, C.POINTER(GrammarTables)]
         L.xg_grammar_get_rule_hashes.argtypes = [vp, vp]
         L.xg_grammar_get_cache_entry.argtypes = [vp, i32, C.POINTER(CacheEntryView)]
+        L.xg_grammar_get_state_classes.argtypes = [vp, i32, vp]
         L.xg_grammar_stats.argtypes = [vp, C.POINTER(GrammarStats)]
         L.xg_matcher_create.argtypes = [vp, C.POINTER(MatcherOptions), vp, C.POINTER(vp)]
         L.xg_matcher_reset.argtypes = [vp, vp]
@@ -158,10 +161,10 @@ class CachePool:
 
 class Grammar:
     def __init__(self, tokenizer: Optional[Tokenizer], kind, text: str, pool: Optional[CachePool] = None, root: Optional[str] = None,
-                 inline_max_states: int = -1, build_cache: bool = True, stream: int = 0):
+                 inline_max_states: int = -1, build_cache: bool = True, stream: int = 0, state_compression: bool = True):
         kind = KIND_BY_NAME.get(kind, kind)
         raw = text.encode("utf-8") if isinstance(text, str) else text
-        opt = CompileOptions(C.sizeof(CompileOptions), inline_max_states, 0, 1 if build_cache else 0)
+        opt = CompileOptions(C.sizeof(CompileOptions), inline_max_states, 0, 1 if build_cache else 0, 0 if state_compression else 1)
         h = C.c_void_p()
         _check(lib().xg_compile_grammar(tokenizer.h if tokenizer else None, pool.h if pool else None, kind, raw, len(raw),
                                         root.encode() if root else None, C.byref(opt), stream, C.byref(h)))
@@ -196,6 +199,13 @@ class Grammar:
         _check(lib().xg_grammar_stats(self.h, C.byref(s)))
         out = np.zeros(s.n_rules, dtype=np.uint64)
         _check(lib().xg_grammar_get_rule_hashes(self.h, out.ctypes.data))
+        return out
+
+    def state_classes(self, depth: int = -1) -> np.ndarray:
+        s = GrammarStats()
+        _check(lib().xg_grammar_stats(self.h, C.byref(s)))
+        out = np.zeros(s.n_states, dtype=np.int32)
+        _check(lib().xg_grammar_get_state_classes(self.h, int(depth), out.ctypes.data))
         return out
 
     def cache_entry(self, state: int) -> dict:

@@ -351,9 +351,9 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
 // Lookahead pass (Section 3.3): the pool's entries are context-free; each grammar narrows their
 // uncertain lists with its own follow sets.  Count, exclusive scan on the host (a few thousand
 // numbers), compact.  The grammar's entry headers must already be on the device.
-static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>& scannable, cudaStream_t stream) {
+static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>& scannable, const std::vector<int32_t>& rep, cudaStream_t stream) {
   std::vector<int32_t> states;
-  for (int s : scannable) if (g->entries[s].n_unc > 0) states.push_back(s);
+  for (int s : scannable) if (g->entries[s].n_unc > 0 && rep[s] == s) states.push_back(s);      // one list per shared entry
   if (states.empty()) return XG_OK;
   const int n = (int)states.size();
   if (n > 2000000) return set_error(XG_ERR_CAPACITY, "too many cache entries with uncertain tokens");
@@ -385,6 +385,12 @@ static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>&
     e.chk_byte = reinterpret_cast<const uint8_t*>(e.chk_exit + counts[k]);
     e.n_chk = counts[k];
   }
+  for (int s : scannable) {
+    if (rep[s] == s) continue;
+    const EntryDev& r = g->entries[rep[s]];
+    EntryDev& e = g->entries[s];
+    e.chk_rank = r.chk_rank; e.chk_exit = r.chk_exit; e.chk_byte = r.chk_byte; e.n_chk = r.n_chk;
+  }
   return XG_OK;
 }
 
@@ -394,12 +400,13 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   *out = nullptr;
   if (!text) return set_error(XG_ERR_INVALID_ARG, "text is NULL");
   FrontendOptions fo;
-  bool build_cache = tok != nullptr;
+  bool build_cache = tok != nullptr, compress = true;
   if (opt) {
     if (opt->struct_size < 8) return set_error(XG_ERR_INVALID_ARG, "bad options struct_size");
     if (opt->inline_max_states >= 0) fo.inline_max_states = opt->inline_max_states;
     if (opt->struct_size >= 12 && opt->max_rule_states > 0) fo.max_rule_states = opt->max_rule_states;
     if (opt->struct_size >= 16 && opt->build_cache == 0) build_cache = false;
+    if (opt->struct_size >= 20 && opt->no_state_compression != 0) compress = false;
   }
   if (pool && pool->impl->owner() != (const void*)tok) return set_error(XG_ERR_INVALID_ARG, "the pool belongs to another tokenizer");
   std::unique_ptr<xg_grammar> g(new xg_grammar());
@@ -454,6 +461,11 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   std::vector<int> canon_of(f.n_states, -1);          // state -> canonical index inside its rule
   for (int r = 0; r < f.n_rules; ++r)
     for (size_t k = 0; k < in.canon[r].size(); ++k) canon_of[rule_first[r] + in.canon[r][k]] = (int)k;
+  // Repetition state compression (Section 3.6): states of a rule that no token of this vocabulary
+  // can tell apart share the entry of their class representative
+  std::vector<int32_t> rep(f.n_states);
+  if (compress && tok->dev.max_len > 0) rep = bounded_equivalence(f, tok->dev.max_len);
+  else for (int s = 0; s < f.n_states; ++s) rep[s] = s;
   std::map<int, int> builder_of;                      // pool rule -> the rule of this grammar that builds it
   std::vector<int32_t> to_build;
   for (int s : scannable) {
@@ -467,11 +479,19 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     } else {
       auto it = builder_of.find(in.pool_id[r]);
       if (it == builder_of.end()) it = builder_of.emplace(in.pool_id[r], r).first;
-      if (it->second == r) to_build.push_back(s);
+      if (it->second == r) {
+        if (rep[s] == s) to_build.push_back(s); else ++g->stats.n_entries_shared;
+      }
     }
   }
   st = build_entries(g.get(), to_build, (cudaStream_t)stream);
   if (st != XG_OK) return fail(st);
+  for (int s : scannable) {                           // the other members of each class
+    if (rep[s] == s) continue;
+    auto it = builder_of.find(in.pool_id[f.state_rule[s]]);
+    if (it == builder_of.end() || it->second != f.state_rule[s]) continue;
+    g->entries[s] = g->entries[rep[s]]; g->entry_counts[s] = g->entry_counts[rep[s]]; g->entry_chunk[s] = g->entry_chunk[rep[s]];
+  }
   for (auto& kv : builder_of) {
     PoolRule& pr = g->pool->rule(kv.first);
     const int r = kv.second;
@@ -500,7 +520,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     ++g->stats.n_entries_reused;
   }
   st = upload_grammar(g.get());       // now with the entry headers
-  if (st == XG_OK) st = narrow_check_lists(g.get(), scannable, (cudaStream_t)stream);
+  if (st == XG_OK) st = narrow_check_lists(g.get(), scannable, rep, (cudaStream_t)stream);
   if (st == XG_OK) st = upload_grammar(g.get());       // and with this grammar's narrowed check lists
   if (st != XG_OK) return fail(st);
   g->stats.cache_build_ms = now_ms() - t1;
@@ -514,7 +534,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     g->stats.total_checked += e.n_chk;
     g->stats.total_rejected += tok->vocab_size - c.x - c.y;
     g->stats.kind_count[e.kind]++;
-    g->stats.cache_bytes += 4LL * ((e.kind == 2 ? tok->n_words : e.n_list) + 3LL * e.n_unc + (e.n_unc + 3) / 4);
+    if (rep[s] == s) g->stats.cache_bytes += 4LL * ((e.kind == 2 ? tok->n_words : e.n_list) + 3LL * e.n_unc + (e.n_unc + 3) / 4);
   }
   *out = g.release();
   return XG_OK;
@@ -552,6 +572,21 @@ xg_status_t xg_grammar_get_rule_hashes(const xg_grammar_t* g, uint64_t* out) {
     for (int r = 0; r < g->flat.n_rules; ++r) out[r] = in.hash[r];
   } catch (const std::exception& e) {
     return set_error(XG_ERR_OOM, e.what());
+  }
+  return XG_OK;
+}
+
+xg_status_t xg_grammar_get_state_classes(const xg_grammar_t* g, int32_t depth, int32_t* out) {
+  if (!g || !out) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
+  if (depth < 0) {
+    if (!g->tok) return set_error(XG_ERR_INVALID_ARG, "depth < 0 needs a grammar compiled with a tokenizer");
+    depth = g->tok->dev.max_len;
+  }
+  try {
+    const std::vector<int32_t> rep = bounded_equivalence(g->flat, depth);
+    std::memcpy(out, rep.data(), rep.size() * sizeof(int32_t));
+  } catch (const std::bad_alloc&) {
+    return set_error(XG_ERR_OOM, "out of host memory");
   }
   return XG_OK;
 }

@@ -1410,4 +1410,114 @@ FlatGrammar compile_frontend(int kind, const std::string& text, const std::strin
   return c.flatten();
 }
 
+
+// Repetition state compression (Section 3.6), as an equivalence on automaton states.  A cache
+// entry only records how tokens of at most `depth` bytes behave from its state, so two states of
+// one rule whose automata agree when unrolled `depth` edges deep (every edge consumes at least
+// one byte: no rule derives the empty string) have the same entry.  Inside a bounded repetition
+// R{l,r} almost all copies of R are alike in this sense -- only the copies within `depth` of the
+// bounds differ -- so the number of entries to build stays bounded however large r is, while the
+// explicit states keep the exact count k of (R{l,r}, k) for the run-time check.
+//   level 0:   same rule, same acceptance;
+//   level d+1: level 0, and the same edges (byte class or referenced rule) into level-d classes.
+// Returns, per state, the smallest state of its class after `depth` rounds of refinement (a
+// partition at least as fine as level `depth`, at most as fine as full bisimulation).
+std::vector<int32_t> bounded_equivalence(const FlatGrammar& g, int depth) {
+  const int S = g.n_states;
+  // predecessors (CSR): whose signature goes stale when a state changes class
+  std::vector<int> pred_begin(S + 1, 0), pred;
+  for (int t : g.cedge_target) ++pred_begin[t + 1];
+  for (int t : g.redge_target) ++pred_begin[t + 1];
+  for (int s = 0; s < S; ++s) pred_begin[s + 1] += pred_begin[s];
+  pred.resize(pred_begin[S]);
+  {
+    std::vector<int> at(pred_begin.begin(), pred_begin.end() - 1);
+    for (int s = 0; s < S; ++s) {
+      for (int e = g.cedge_begin[s]; e < g.cedge_begin[s + 1]; ++e) pred[at[g.cedge_target[e]]++] = s;
+      for (int e = g.redge_begin[s]; e < g.redge_begin[s + 1]; ++e) pred[at[g.redge_target[e]]++] = s;
+    }
+  }
+  // level 0
+  std::vector<int> block(S), count;
+  {
+    SignatureTable table;
+    std::vector<uint32_t> sig(2);
+    for (int s = 0; s < S; ++s) {
+      sig[0] = (uint32_t)g.state_rule[s]; sig[1] = g.state_final[s];
+      block[s] = table.intern(sig);
+      if (block[s] == (int)count.size()) count.push_back(0);
+      ++count[block[s]];
+    }
+  }
+  // One round per level.  A state's signature (its edges with targets replaced by their classes)
+  // is recomputed only after one of its targets moved to a new class.  All members of a class
+  // carry the same signature once a round is over, so a round only has to place the recomputed
+  // states: those that still match their class's standing signature stay, every other group
+  // becomes a new class (when the whole class was recomputed, its largest group keeps the id).
+  // A round costs in proportion to what changed, not to S.
+  SignatureTable table;
+  std::vector<int> sig_id(S, -1), standing(count.size(), -1), work(S);
+  std::vector<char> queued(S, 1);
+  for (int s = 0; s < S; ++s) work[s] = s;
+  std::vector<uint32_t> sig;
+  std::vector<std::pair<uint32_t, uint32_t>> edges;
+  std::vector<int> moved;
+  for (int level = 0; level < depth && !work.empty(); ++level) {
+    for (int s : work) {
+      sig.clear();
+      edges.clear();
+      for (int e = g.cedge_begin[s]; e < g.cedge_begin[s + 1]; ++e) edges.emplace_back((uint32_t)g.cedge_class[e], (uint32_t)block[g.cedge_target[e]]);
+      std::sort(edges.begin(), edges.end());
+      sig.push_back((uint32_t)edges.size());
+      for (auto& p : edges) { sig.push_back(p.first); sig.push_back(p.second); }
+      edges.clear();
+      for (int e = g.redge_begin[s]; e < g.redge_begin[s + 1]; ++e) edges.emplace_back((uint32_t)g.redge_rule[e], (uint32_t)block[g.redge_target[e]]);
+      std::sort(edges.begin(), edges.end());
+      for (auto& p : edges) { sig.push_back(p.first); sig.push_back(p.second); }
+      sig_id[s] = table.intern(sig);
+      queued[s] = 0;
+    }
+    std::sort(work.begin(), work.end(), [&](int x, int y) {
+      if (block[x] != block[y]) return block[x] < block[y];
+      return sig_id[x] != sig_id[y] ? sig_id[x] < sig_id[y] : x < y;
+    });
+    moved.clear();
+    for (size_t lo = 0; lo < work.size();) {
+      const int b = block[work[lo]];
+      size_t hi = lo;
+      while (hi < work.size() && block[work[hi]] == b) ++hi;
+      int keep = standing[b];
+      if ((int)(hi - lo) == count[b]) {               // nobody holds the standing signature any more: the largest group stays
+        size_t best = 0;
+        for (size_t i = lo; i < hi;) {
+          size_t j = i;
+          while (j < hi && sig_id[work[j]] == sig_id[work[i]]) ++j;
+          if (j - i > best) { best = j - i; keep = sig_id[work[i]]; }
+          i = j;
+        }
+        standing[b] = keep;
+      }
+      for (size_t i = lo; i < hi;) {
+        size_t j = i;
+        while (j < hi && sig_id[work[j]] == sig_id[work[i]]) ++j;
+        if (sig_id[work[i]] != keep) {
+          const int id = (int)count.size();
+          count.push_back((int)(j - i));
+          standing.push_back(sig_id[work[i]]);
+          count[b] -= (int)(j - i);
+          for (size_t k = i; k < j; ++k) { block[work[k]] = id; moved.push_back(work[k]); }
+        }
+        i = j;
+      }
+      lo = hi;
+    }
+    work.clear();
+    for (int s : moved)
+      for (int q = pred_begin[s]; q < pred_begin[s + 1]; ++q) if (!queued[pred[q]]) { queued[pred[q]] = 1; work.push_back(pred[q]); }
+  }
+  std::vector<int32_t> first(count.size(), -1), rep(S);
+  for (int s = 0; s < S; ++s) { if (first[block[s]] < 0) first[block[s]] = s; rep[s] = first[block[s]]; }
+  return rep;
+}
+
 }  // namespace xg

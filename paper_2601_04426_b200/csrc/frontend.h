@@ -71,6 +71,11 @@ enum GrammarKind { kEbnf = 0, kJsonSchema = 1, kTagDispatchJson = 2 };
 // Throws FrontendError.
 FlatGrammar compile_frontend(int kind, const std::string& text, const std::string& root, const FrontendOptions& opt);
 
+// Repetition state compression (Section 3.6): states of one rule that agree when their automata
+// are unrolled `depth` edges deep share one cache entry.  Returns the class representative (the
+// smallest such state) of every state.
+std::vector<int32_t> bounded_equivalence(const FlatGrammar& g, int depth);
+
 // The two text-to-text lowerings (exposed for tests and diagnostics).
 std::string json_schema_to_ebnf(const std::string& schema_json, const std::string& root_name, const std::string& prefix);
 std::string tag_dispatch_to_ebnf(const std::string& spec_json);

@@ -17,7 +17,7 @@ from . import inputs
 class Session:
     """One tokenizer, its compiled grammars and one matcher per request of a workload."""
 
-    def __init__(self, workload: inputs.Workload, share_pool: bool = True, device: str = "cuda:0"):
+    def __init__(self, workload: inputs.Workload, share_pool: bool = True, device: str = "cuda:0", state_compression: bool = True):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         self.device = torch.device(device)
@@ -26,7 +26,8 @@ class Session:
         v = workload.vocab
         self.tokenizer = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
         self.pool = B.CachePool(self.tokenizer) if share_pool else None
-        self.grammars: List[B.Grammar] = [B.Grammar(self.tokenizer, g.kind, g.text, pool=self.pool) for g in workload.grammars]
+        self.grammars: List[B.Grammar] = [B.Grammar(self.tokenizer, g.kind, g.text, pool=self.pool, state_compression=state_compression)
+                                          for g in workload.grammars]
         self.matchers = [B.Matcher(self.grammars[gi]) for gi in workload.request_grammar]
         self.batch = B.Batch(self.matchers)
         self.V, self.W, self.n = v.size, self.tokenizer.words, len(self.matchers)

@@ -566,13 +566,19 @@ _SHAPES = {
     "T20": (128256,  16,  4.0, 0.3,    0.0,  16,   128,  "bf16"),
     "T50": (128256,  16,  4.0, 0.3,    0.0,  16,   128,  "bf16"),
     "T100": (128256, 16,  4.0, 0.3,    0.0,  16,   128,  "bf16"),
+    # long bounded repetitions (Section 3.6: minLength / maxLength / minItems / maxItems in the hundreds to thousands)
+    "R256": (128256,  16,  4.0, 0.3,    0.0,  16,   256,  "bf16"),
+    "R1024": (128256, 16,  4.0, 0.3,    0.0,  16,   256,  "bf16"),
+    "R4096": (128256, 16,  4.0, 0.3,    0.0,  16,   256,  "bf16"),
 }
 
 _vocab_cache: Dict[Tuple, Vocab] = {}
 
 
 def config_seed(name: str) -> int:
-    return BASE_SEED * 10 + (int(name[1]) if name[0] == "C" else 1000 + int(name[1:]))
+    if name[0] == "C":
+        return BASE_SEED * 10 + int(name[1])
+    return BASE_SEED * 10 + (1000 if name[0] == "T" else 100000) + int(name[1:])
 
 
 def config_vocab(name: str, vocab_size: Optional[int] = None) -> Vocab:
@@ -580,7 +586,7 @@ def config_vocab(name: str, vocab_size: Optional[int] = None) -> Vocab:
     if vocab_size is not None:
         V = vocab_size
     # C2 and C4 share one Llama-3-sized vocabulary
-    seed_name = "C2" if (name == "C4" or name[0] == "T") else name
+    seed_name = "C2" if (name == "C4" or name[0] in "TR") else name
     key = (seed_name, V)
     if key not in _vocab_cache:
         _vocab_cache[key] = make_vocab(config_seed(seed_name) ^ 0x5EED, V, lmax, mean, lead, utf8)
@@ -679,6 +685,29 @@ def make_workload(name: str, batch: Optional[int] = None, steps: Optional[int] =
             rr = rng.fork(100 + b)
             t, d = _trajectory(tok, vocab.eos_id, S, lambda: sample_function_text(rr, tools, rr.randint(1, 3), 40).encode())
             request_grammar.append(0); trajs.append(t); docs_all.append(d)
+    elif name[0] == "R":
+        # four orderings of one set of bounded properties, so that within the step budget different
+        # requests are inside different repetitions; lengths are drawn up to the bounds
+        n = int(name[1:])
+        r = rng.fork(1)
+        props = [
+            (_word(r, 3, 8), {"type": "string", "maxLength": n}),
+            (_word(r, 3, 8), {"type": "string", "minLength": n // 2, "maxLength": n}),
+            (_word(r, 3, 8), {"type": "array", "items": {"type": "integer"}, "maxItems": n // 8}),
+            (_word(r, 3, 8), {"type": "array", "items": {"type": "string", "maxLength": 8}, "minItems": n // 16, "maxItems": n // 8}),
+        ]
+        schemas = []
+        for k in range(4):
+            order = props[k:] + props[:k]
+            schema = {"type": "object", "properties": dict(order), "required": [key for key, _ in order]}
+            schemas.append(schema)
+            grammars.append(GrammarSpec("json_schema", json.dumps(schema)))
+        meta["bound"] = n
+        for b in range(B):
+            rr = rng.fork(100 + b)
+            schema = schemas[b % 4]
+            t, d = _trajectory(tok, vocab.eos_id, S, lambda: sample_document(schema, rr).encode())
+            request_grammar.append(b % 4); trajs.append(t); docs_all.append(d)
     else:
         raise KeyError(name)
     return Workload(name=name, vocab=vocab, grammars=grammars, request_grammar=request_grammar,
