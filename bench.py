@@ -154,6 +154,9 @@ def main():
     ap.add_argument("--workload", default="C3", choices=sorted(SHAPES))
     ap.add_argument("--batch", type=int, default=None, help="shrink the batch (debugging only; the line then names it)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--jit-sweep", default=None,
+                    help="comma-separated K values (or 'full'): compile just in time with K entries precomputed and report "
+                         "compile time and per-step time avg / P99 / max over the trajectory (the shape of the paper's K sweep)")
     ap.add_argument("--no-state-compression", action="store_true",
                     help="build one cache entry per scannable state (ablation of the repetition state compression)")
     args = ap.parse_args()
@@ -186,6 +189,11 @@ def main():
     XB.lib()          # fails loudly if the CUDA library is missing
 
     w = inputs.make_workload(args.workload, batch=args.batch)
+    if args.jit_sweep:
+        if rank == 0:
+            print(json.dumps(jit_sweep(w, args, local_rank)))
+        dist_util.finish()
+        return 0
     if world > 1:     # weak scaling: every rank serves its own batch of requests (no data-path collective)
         w = dist_util.rotate_requests(w, rank)
     # one small compile first, so that the reported build time holds no context creation or lazy module loading
@@ -404,6 +412,62 @@ def main():
         print(json.dumps(line))
     dist_util.finish()
     return 0
+
+
+def jit_sweep(w, args, local_rank):
+    """Per-step time with the cache built just in time (Section 3.5): for each K, compile with K entries
+    precomputed, then run the trajectory once from a cold pool (entries arrive while decoding) and once more
+    warm.  A step = fill + apply + accept + the service call and whatever cache-build kernels it enqueued."""
+    import torch
+    from paper_2601_04426_b200 import binding as XB
+    from paper_2601_04426_b200 import engine
+    wt = XB.Tokenizer([bytes([i]) for i in range(256)] + [b""], 256, [])
+    XB.Grammar(wt, "ebnf", 'root ::= [a-z]+ "."').close()
+    wt.close()
+    rows = []
+    n = w.batch
+    for k_text in args.jit_sweep.split(","):
+        full = k_text == "full"
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        s = engine.Session(w, device="cuda:%d" % local_rank, jit=not full, jit_precompute=0 if full else int(k_text))
+        torch.cuda.synchronize()
+        compile_s = time.perf_counter() - t0
+        stats = [g.stats() for g in s.grammars]
+        logits = engine.logits_tensor(inputs.make_logits(w.logits_seed, min(n, 8), s.V, w.dtype), s.device)
+        logits = logits.repeat((n + logits.shape[0] - 1) // logits.shape[0], 1)[:n].contiguous()
+        traj = torch.from_numpy(np.asarray([[w.trajectories[b][t] for b in range(n)] for t in range(w.steps)], dtype=np.int32)).to(s.device)
+        eos_at = {t: [b for b in range(n) if w.trajectories[b][t] == w.vocab.eos_id] for t in range(w.steps)}
+        passes = {}
+        for label in ("cold", "warm"):
+            if label == "warm" and not full:
+                s.jit_service(wait=True)          # whatever the cold pass left in flight or unreported
+            for b in range(n):
+                s.reset(b)
+            torch.cuda.synchronize()
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(w.steps + 1)]
+            evs[0].record()
+            for t in range(w.steps):
+                s.fill()
+                s.apply(logits)
+                s.accept_device(traj[t])
+                for b in eos_at[t]:
+                    s.reset(b)
+                if not full:
+                    s.jit_service(wait=False)
+                evs[t + 1].record()
+                evs[t + 1].synchronize()        # a decode loop waits here for the sampled tokens: the host never runs ahead of the GPU
+            torch.cuda.synchronize()
+            us = np.asarray([evs[t].elapsed_time(evs[t + 1]) * 1e3 for t in range(w.steps)])
+            passes[label] = {"avg_us": float(us.mean()), "p99_us": float(np.percentile(us, 99)), "max_us": float(us.max())}
+        js = s.jit_service(wait=True) if not full else {"n_built": 0, "n_pool_hits": 0, "n_missing": 0}
+        rows.append({"K": k_text, "compile_wall_s": compile_s, "cache_build_ms": sum(x["cache_build_ms"] for x in stats),
+                     "frontend_ms": sum(x["frontend_ms"] for x in stats),
+                     "entries_built_at_compile": sum(x["n_entries_built"] for x in stats), "entries_built_just_in_time": js["n_built"],
+                     "pool_hits": js["n_pool_hits"], "entries_never_built": js["n_missing"], "steps": w.steps, **{k + "_" + kk: vv for k, p in passes.items() for kk, vv in p.items()}})
+        s.close()
+    return {"metric": "per-step us with just-in-time cache build (eager launches: fill, apply, accept, service)", "workload": w.name, "batch": n,
+            "vocab": w.vocab.size, "rows": rows}
 
 
 def _with_batch(w, batch):

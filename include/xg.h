@@ -106,6 +106,11 @@ typedef struct {
   int32_t build_cache;        /* 0 = front end only (tables, no device work).  Otherwise build. */
   int32_t no_state_compression; /* non-zero: build one cache entry per scannable state even where repetition
                                  state compression (Section 3.6) would let states share one. */
+  int32_t jit;                /* non-zero: just-in-time cache (Section 3.5).  The compile builds only the
+                                 jit_precompute costliest entries that the pool does not already hold; the others
+                                 are built when a matcher first visits their state (xg_jit_service). */
+  int32_t jit_precompute;     /* K of Section 3.5's configurable JIT: entries to build at compile time, the
+                                 costliest first (cost = tokens that survive the state's first-byte test). */
 } xg_compile_options_t;
 
 /* ---- grammar compilation (Section 3.5 "compilation stage"; Sections 3.2, 3.3, 3.4) ---------
@@ -167,7 +172,8 @@ xg_status_t xg_grammar_get_state_classes(const xg_grammar_t* g, int32_t depth, i
 /* One cache entry, copied to the host (valid until the next call on this grammar or its
  * destruction).  list = accepted ids (XG_STORE_ACCEPT_LIST) or rejected ids
  * (XG_STORE_REJECT_LIST), ascending; bitset = accepted bits (XG_STORE_BITSET), ceil(V/32) words;
- * uncertain = ascending ids.  Returns XG_ERR_INVALID_ARG if `state` is not scannable.
+ * uncertain = ascending ids.  Returns XG_ERR_INVALID_ARG if `state` is not scannable, or if a
+ * just-in-time grammar has not built (and confirmed, see xg_jit_service) its entry yet.
  * Synchronises the device. */
 typedef struct {
   int32_t state, kind;
@@ -196,6 +202,32 @@ typedef struct {
 } xg_grammar_stats_t;
 xg_status_t xg_grammar_stats(const xg_grammar_t* g, xg_grammar_stats_t* out);
 
+/* ---- just-in-time cache build (Section 3.5) ------------------------------------------------
+ * A grammar compiled with opt->jit starts with (nearly) no cache entries.  Masks are exact from the
+ * first step on: while a scannable state of a matcher's current Earley set has no entry yet, the
+ * fill kernel takes that request's mask from the plain definition (every token walked against the
+ * full Earley state) and reports the state in a device-side ring.  xg_jit_service, called between
+ * decode steps, reads the ring and gets the missing entries: from the pool if another grammar has
+ * built them since (a cache hit), else by enqueueing the cache-build kernels on `stream`; the new
+ * entries become visible to later fills in stream order.  States that are never visited are never
+ * built.
+ *   - The call never waits for the GPU unless wait != 0: it polls events, copies a few KB and
+ *     enqueues kernels.  A miss reported by the fill of step t is picked up by the service call
+ *     after step t+1 at the earliest, so a new state costs a few fallback steps.
+ *   - wait != 0: also synchronises `stream` repeatedly until nothing is reported and nothing is in
+ *     flight (what a caller does while the model prefills, and what tests use).
+ *   - Use one stream for the fills, accepts and service calls of all just-in-time grammars of a
+ *     pool, or order them with events: publishing an entry races with a fill running elsewhere.
+ *   - Entries that arrive just in time get the grammar's lookahead narrowing like those of a full compile.
+ * grammars: host array of n handles; those compiled without jit are skipped.  out may be NULL. */
+typedef struct {
+  int32_t n_built;        /* entries built just in time so far, over the given grammars (one per class of states) */
+  int32_t n_pool_hits;    /* visited entries found in the pool instead of being built */
+  int32_t n_in_flight;    /* entries whose build is enqueued and not yet confirmed */
+  int32_t n_missing;      /* entries (classes of scannable states) still not built */
+} xg_jit_stats_t;
+xg_status_t xg_jit_service(xg_grammar_t* const* grammars, int32_t n, void* stream, int32_t wait, xg_jit_stats_t* out);
+
 /* ---- matcher: one request's Earley state (Section 3.4) ------------------------------------ */
 typedef struct {
   uint32_t struct_size;
@@ -215,6 +247,8 @@ xg_status_t xg_matcher_is_terminated(const xg_matcher_t* m, void* stream, int32_
  * XGrammar's cache: a token accepted by the cache of at least one current scannable state is
  * allowed; otherwise, if some cache calls it uncertain, it is checked against the matcher's full
  * Earley state; otherwise it is rejected.  EOS is allowed iff the root rule is complete.
+ * (Just-in-time grammars: a request with an entry still missing gets the same mask from a walk of
+ * the whole vocabulary against its full Earley state.)
  * status_dev (device, [batch], may be NULL) receives XG_OK, XG_ERR_TERMINATED or XG_ERR_CAPACITY
  * per matcher; rows of matchers whose status is not XG_OK are all zero. */
 xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t batch,

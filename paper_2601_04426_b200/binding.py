@@ -26,7 +26,7 @@ DTYPE_BY_NAME = {"f32": XG_F32, "bf16": XG_BF16}
 
 EXPORTS = [
     "xg_last_error", "xg_tokenizer_create", "xg_tokenizer_destroy", "xg_cache_pool_create", "xg_cache_pool_destroy", "xg_cache_pool_set_limit", "xg_cache_pool_stats",
-    "xg_compile_grammar", "xg_grammar_destroy", "xg_grammar_get_tables", "xg_grammar_get_rule_hashes", "xg_grammar_get_cache_entry", "xg_grammar_get_state_classes", "xg_grammar_stats",
+    "xg_compile_grammar", "xg_grammar_destroy", "xg_grammar_get_tables", "xg_grammar_get_rule_hashes", "xg_grammar_get_cache_entry", "xg_grammar_get_state_classes", "xg_grammar_stats", "xg_jit_service",
     "xg_matcher_create", "xg_matcher_reset", "xg_matcher_destroy", "xg_matcher_is_terminated",
     "xg_fill_next_token_bitmask", "xg_fill_next_token_bitmask_static", "xg_apply_token_bitmask", "xg_accept_token",
 ]
@@ -41,7 +41,11 @@ class XgError(RuntimeError):
 
 class CompileOptions(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("inline_max_states", C.c_int32), ("max_rule_states", C.c_int32), ("build_cache", C.c_int32),
-                ("no_state_compression", C.c_int32)]
+                ("no_state_compression", C.c_int32), ("jit", C.c_int32), ("jit_precompute", C.c_int32)]
+
+
+class JitStats(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_built", "n_pool_hits", "n_in_flight", "n_missing")]
 
 
 class MatcherOptions(C.Structure):
@@ -100,6 +104,7 @@ def lib():
         L.xg_grammar_get_rule_hashes.argtypes = [vp, vp]
         L.xg_grammar_get_cache_entry.argtypes = [vp, i32, C.POINTER(CacheEntryView)]
         L.xg_grammar_get_state_classes.argtypes = [vp, i32, vp]
+        L.xg_jit_service.argtypes = [vp, i32, vp, i32, C.POINTER(JitStats)]
         L.xg_grammar_stats.argtypes = [vp, C.POINTER(GrammarStats)]
         L.xg_matcher_create.argtypes = [vp, C.POINTER(MatcherOptions), vp, C.POINTER(vp)]
         L.xg_matcher_reset.argtypes = [vp, vp]
@@ -161,10 +166,12 @@ class CachePool:
 
 class Grammar:
     def __init__(self, tokenizer: Optional[Tokenizer], kind, text: str, pool: Optional[CachePool] = None, root: Optional[str] = None,
-                 inline_max_states: int = -1, build_cache: bool = True, stream: int = 0, state_compression: bool = True):
+                 inline_max_states: int = -1, build_cache: bool = True, stream: int = 0, state_compression: bool = True,
+                 jit: bool = False, jit_precompute: int = 0):
         kind = KIND_BY_NAME.get(kind, kind)
         raw = text.encode("utf-8") if isinstance(text, str) else text
-        opt = CompileOptions(C.sizeof(CompileOptions), inline_max_states, 0, 1 if build_cache else 0, 0 if state_compression else 1)
+        opt = CompileOptions(C.sizeof(CompileOptions), inline_max_states, 0, 1 if build_cache else 0, 0 if state_compression else 1,
+                             1 if jit else 0, int(jit_precompute))
         h = C.c_void_p()
         _check(lib().xg_compile_grammar(tokenizer.h if tokenizer else None, pool.h if pool else None, kind, raw, len(raw),
                                         root.encode() if root else None, C.byref(opt), stream, C.byref(h)))
@@ -223,6 +230,14 @@ class Grammar:
         d = {n: getattr(s, n) for n, _ in GrammarStats._fields_ if n not in ("kind_count", "pad")}
         d["kind_count"] = list(s.kind_count)
         return d
+
+
+def jit_service(grammars: Sequence["Grammar"], stream: int = 0, wait: bool = False) -> dict:
+    """Advance the just-in-time cache builds of `grammars` (see xg_jit_service)."""
+    arr = (C.c_void_p * len(grammars))(*[g.h for g in grammars])
+    st = JitStats()
+    _check(lib().xg_jit_service(arr, len(grammars), stream, 1 if wait else 0, C.byref(st)))
+    return {n: getattr(st, n) for n, _ in JitStats._fields_}
 
 
 class Matcher:

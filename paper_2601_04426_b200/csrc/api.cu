@@ -64,9 +64,52 @@ struct xg_tokenizer {
   std::vector<void*> allocations;
   std::vector<int32_t> rank_to_id, id_to_rank;
   int32_t vocab_size = 0, n_words = 0;
+  int64_t first_byte_count[256] = {};     // tokens (other than EOS / special / empty) by first byte
   mutable std::mutex mu;
   mutable std::vector<BatchSlot> batch_slots;
   mutable uint64_t use_counter = 0;
+};
+
+// Host side of the just-in-time cache build (Section 3.5).  The cycle belongs to the pool: a snapshot of
+// the pool's miss ring is copied to pinned memory; once it has arrived, the reported states are served from
+// the pool or their builds are enqueued, grammar by grammar; once the builds' results have arrived, they are
+// recorded and the cycle restarts.  One snapshot and one event per step, however many grammars decode.
+constexpr int kJitBatchMax = 64;          // entries per build (one grammar, one set of launches)
+constexpr int kJitCycleEntries = 512;     // entries per cycle, over all grammars
+constexpr int kJitCycleBuilds = 128;      // builds per cycle
+struct JitHostResult {                    // pinned; written by asynchronous copies
+  JitRing ring;
+  EntryDev entries[kJitCycleEntries];
+  int2 counts[kJitCycleEntries];
+  int result[kJitCycleBuilds][2];
+  long long total_words[kJitCycleBuilds];
+};
+struct JitFlight {                        // one enqueued build
+  xg_grammar* g;
+  std::vector<int32_t> reps;
+  int chunk, entry_offset, index;
+};
+struct JitPool {
+  JitRing* d_ring = nullptr;
+  JitHostResult* h = nullptr;
+  cudaEvent_t ev = nullptr;
+  int phase = 0;                          // 0 idle, 1 snapshot on its way, 2 builds on their way
+  uint32_t ring_seen = 0;
+  std::vector<xg_grammar*> slots;         // the pool's just-in-time grammars by slot (nullptr once destroyed)
+  std::vector<JitFlight> flights;
+};
+struct JitState {                         // per grammar
+  bool enabled = false;
+  int slot = -1;
+  std::vector<int32_t> rep;                    // state -> class representative
+  std::vector<int32_t> member_begin, members;  // representative -> the states of its class (CSR over all states)
+  std::vector<uint8_t> status;                 // per representative: 0 missing, 1 build in flight, 2 built
+  int32_t* d_rep = nullptr;
+  int32_t* d_pub_state = nullptr;              // [kJitBatchMax] staging of pool hits
+  EntryDev* d_pub_entry = nullptr;
+  RuleInterning in;
+  std::vector<int> canon_of, rule_first;
+  int n_built = 0, n_pool_hits = 0, n_missing = 0, n_in_flight = 0;
 };
 
 struct xg_grammar {
@@ -82,6 +125,7 @@ struct xg_grammar {
   std::vector<int> entry_chunk;         // [n_states] pool chunk that holds the state's entry (-1: none)
   std::vector<int> chunk_refs;          // pool chunks this grammar keeps alive
   xg_grammar_stats_t stats{};
+  JitState jit;
   // buffers behind xg_grammar_get_cache_entry's view
   mutable std::vector<int32_t> view_list, view_unc;
   mutable std::vector<uint32_t> view_bits;
@@ -149,6 +193,7 @@ xg_status_t xg_tokenizer_create(const uint8_t* bytes, const int64_t* offsets, in
     if (offsets[id + 1] > offsets[id]) arena.insert(arena.end(), bytes + offsets[id], bytes + offsets[id + 1]);
     off[r + 1] = (uint32_t)arena.size();
     never_rank[r] = (never[id] || offsets[id + 1] == offsets[id]) ? 1 : 0;
+    if (!never_rank[r]) ++t->first_byte_count[bytes[offsets[id]]];
   }
   arena.resize(arena.size() + 16, 0);
   cudaError_t err = cudaSuccess;
@@ -262,6 +307,8 @@ static xg_status_t upload_grammar(xg_grammar* g) {
   v.state_first = (const uint32_t*)(d + o_first);
   v.rule_follow = (const uint32_t*)(d + o_follow);
   v.entries = (const EntryDev*)(d + o_en);
+  v.miss_ring = g->jit.slot >= 0 ? ((JitPool*)g->pool->jit_host)->d_ring : nullptr;
+  v.jit_slot = g->jit.slot;
   put(o_self, &v, sizeof(GrammarDev));
   g->dev = (GrammarDev*)(d + o_self);
   XG_CUDA(cudaMemcpy(g->blob, host.data(), total, cudaMemcpyHostToDevice));
@@ -333,8 +380,8 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
     int chunk_id = -1;
     uint32_t* arena = (uint32_t*)g->pool->allocate_device((size_t)std::max<long long>(total_words, 1) * 4, &chunk_id);
     if (!arena) { cleanup(); return set_error(XG_ERR_OOM, "cache arena allocation failed"); }
-    pack_kernel<<<n, 256, 0, stream>>>(acc, unc, unr, d_plan, V, W, arena, d_entries);
-    exit_kernel<<<n, 256, 0, stream>>>(g->host_view, v, d_pos, d_entries);
+    pack_kernel<<<n, 256, 0, stream>>>(acc, unc, unr, d_plan, V, W, arena, d_entries, nullptr);
+    exit_kernel<<<n, 256, 0, stream>>>(g->host_view, v, d_pos, d_entries, nullptr);
     XG_CUDA_C(cudaGetLastError());
     std::vector<EntryDev> built(n);
     std::vector<int2> counts(n);
@@ -363,7 +410,7 @@ static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>&
   long long* d_offsets = (long long*)pool.scratch(13, (size_t)n * 8);
   if (!d_states || !d_counts || !d_offsets) return set_error(XG_ERR_OOM, "lookahead scratch allocation failed");
   XG_CUDA(cudaMemcpyAsync(d_states, states.data(), (size_t)n * 4, cudaMemcpyHostToDevice, stream));
-  lookahead_count_kernel<<<n, 256, 0, stream>>>(g->host_view, g->tok->dev, d_states, d_counts);
+  lookahead_count_kernel<<<n, 256, 0, stream>>>(g->host_view, g->tok->dev, d_states, d_counts, nullptr);
   XG_CUDA(cudaGetLastError());
   std::vector<int32_t> counts(n);
   XG_CUDA(cudaMemcpyAsync(counts.data(), d_counts, (size_t)n * 4, cudaMemcpyDeviceToHost, stream));
@@ -374,7 +421,7 @@ static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>&
   g->lookahead_arena = pool.allocate_plain((size_t)std::max<long long>(total, 1) * 4);
   if (!g->lookahead_arena) return set_error(XG_ERR_OOM, "check list allocation failed");
   XG_CUDA(cudaMemcpyAsync(d_offsets, offsets.data(), (size_t)n * 8, cudaMemcpyHostToDevice, stream));
-  lookahead_compact_kernel<<<n, 256, 0, stream>>>(g->host_view, g->tok->dev, d_states, d_offsets, d_counts, (uint32_t*)g->lookahead_arena);
+  lookahead_compact_kernel<<<n, 256, 0, stream>>>(g->host_view, g->tok->dev, d_states, d_offsets, d_counts, (uint32_t*)g->lookahead_arena, nullptr);
   XG_CUDA(cudaGetLastError());
   XG_CUDA(cudaStreamSynchronize(stream));
   uint32_t* arena = (uint32_t*)g->lookahead_arena;
@@ -394,19 +441,349 @@ static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>&
   return XG_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// just-in-time cache build (Section 3.5)
+// ---------------------------------------------------------------------------------------------
+// device scratch of the just-in-time builds: the pool's, separate from the compile-time build's (which may be
+// running on another stream) and sized once for a full batch, so it is never reallocated inside a decode loop
+struct JitScratch {
+  int32_t* pos; uint32_t* rows; int2* counts; PackPlan* plan; long long* total; EntryDev* entries; int2* over; int* over_count; int* result;
+  int32_t* list_counts; long long* list_offsets; int* go_lists; int* one;
+};
+static bool jit_scratch(CachePool& pool, int W, JitScratch* sc) {
+  const size_t row_bytes = (size_t)W * 4;
+  sc->pos = (int32_t*)pool.scratch(20, kJitBatchMax * sizeof(int32_t));
+  sc->rows = (uint32_t*)pool.scratch(21, 3 * row_bytes * kJitBatchMax);
+  sc->counts = (int2*)pool.scratch(22, kJitBatchMax * sizeof(int2));
+  sc->plan = (PackPlan*)pool.scratch(23, kJitBatchMax * sizeof(PackPlan));
+  sc->total = (long long*)pool.scratch(24, sizeof(long long));
+  sc->entries = (EntryDev*)pool.scratch(25, kJitBatchMax * sizeof(EntryDev));
+  sc->over = (int2*)pool.scratch(26, 64 * sizeof(int2));
+  sc->over_count = (int*)pool.scratch(27, 2 * sizeof(int));
+  sc->result = (int*)pool.scratch(28, 2 * sizeof(int));
+  sc->list_counts = (int32_t*)pool.scratch(29, kJitBatchMax * sizeof(int32_t));
+  sc->list_offsets = (long long*)pool.scratch(30, kJitBatchMax * sizeof(long long));
+  sc->go_lists = (int*)pool.scratch(31, sizeof(int));
+  sc->one = (int*)pool.scratch(32, sizeof(int));            // holds 1 (set when a grammar registers)
+  return sc->one && sc->list_counts && sc->list_offsets && sc->go_lists && sc->pos && sc->rows && sc->counts && sc->plan && sc->total && sc->entries && sc->over && sc->over_count && sc->result;
+}
+
+static void jit_pool_free(void* p) {
+  JitPool* jp = (JitPool*)p;
+  cudaFree(jp->d_ring);
+  if (jp->h) cudaFreeHost(jp->h);
+  if (jp->ev) cudaEventDestroy(jp->ev);
+  delete jp;
+}
+
+// undo jit_allocate (call with the pool's lock held)
+static void jit_release(xg_grammar* g) {
+  cudaDeviceSynchronize();               // a build of this grammar may still be on its way
+  if (g->pool) g->pool->free_plain(g->jit.d_rep);
+  g->jit.d_rep = nullptr; g->jit.d_pub_state = nullptr; g->jit.d_pub_entry = nullptr;
+  JitPool* jp = g->pool ? (JitPool*)g->pool->jit_host : nullptr;
+  if (jp && g->jit.slot >= 0) {
+    jp->slots[g->jit.slot] = nullptr;
+    jp->flights.erase(std::remove_if(jp->flights.begin(), jp->flights.end(), [&](const JitFlight& fl) { return fl.g == g; }), jp->flights.end());
+  }
+  g->jit.slot = -1;
+  g->jit.enabled = false;
+}
+
+// per-grammar device arrays, the pool's ring and scratch; registers the grammar in the pool (call with the pool's lock held)
+static xg_status_t jit_allocate(xg_grammar* g) {
+  JitState& j = g->jit;
+  CachePool& pool = *g->pool;
+  JitScratch sc;
+  if (!jit_scratch(pool, g->tok->n_words, &sc) || !pool.jit_arena(0, false)) return set_error(XG_ERR_OOM, "just-in-time scratch allocation failed");
+  const int one = 1;
+  XG_CUDA(cudaMemcpy(sc.one, &one, sizeof(int), cudaMemcpyHostToDevice));
+  if (!pool.jit_host) {
+    JitPool* jp = new JitPool();
+    pool.jit_host = jp;
+    pool.jit_host_free = jit_pool_free;
+    XG_CUDA(cudaMalloc(&jp->d_ring, sizeof(JitRing)));
+    XG_CUDA(cudaMemset(jp->d_ring, 0, sizeof(JitRing)));
+    XG_CUDA(cudaHostAlloc(&jp->h, sizeof(JitHostResult), cudaHostAllocDefault));
+    std::memset(jp->h, 0, sizeof(JitHostResult));
+    XG_CUDA(cudaEventCreateWithFlags(&jp->ev, cudaEventDisableTiming));
+  }
+  JitPool* jp = (JitPool*)pool.jit_host;
+  if (!jp->d_ring || !jp->h || !jp->ev) return set_error(XG_ERR_CUDA, "the pool's just-in-time state is incomplete");
+  // one block from the pool's slabs: [rep | staged states | staged entries]
+  const size_t S = (size_t)std::max(g->flat.n_states, 1);
+  const size_t o_state = (S * 4 + 255) & ~size_t(255), o_entry = o_state + 256;
+  static_assert(kJitBatchMax * sizeof(int32_t) <= 256, "staging area too small");
+  char* block = (char*)pool.allocate_plain(o_entry + kJitBatchMax * sizeof(EntryDev));
+  if (!block) return set_error(XG_ERR_OOM, "just-in-time tables allocation failed");
+  j.d_rep = (int32_t*)block;
+  j.d_pub_state = (int32_t*)(block + o_state);
+  j.d_pub_entry = (EntryDev*)(block + o_entry);
+  for (size_t k = 0; k < jp->slots.size() && j.slot < 0; ++k) if (!jp->slots[k]) { jp->slots[k] = g; j.slot = (int)k; }
+  if (j.slot < 0) { jp->slots.push_back(g); j.slot = (int)jp->slots.size() - 1; }
+  return XG_OK;
+}
+
+// the host's record of entries that now exist on the device for the representatives `reps`:
+// grammar copy for every class member, pool registration, chunk references
+static void jit_record(xg_grammar* g, const std::vector<int32_t>& reps, const EntryDev* entries, const int2* counts, int chunk) {
+  JitState& j = g->jit;
+  const FlatGrammar& f = g->flat;
+  CachePool& pool = *g->pool;
+  for (size_t k = 0; k < reps.size(); ++k) {
+    const int r = reps[k];
+    const int rule = f.state_rule[r];
+    PoolRule& pr = pool.rule(j.in.pool_id[rule]);
+    const int n_local = (int)j.in.canon[rule].size();
+    pr.entries.resize(n_local); pr.counts.resize(n_local); pr.have.resize(n_local, 0);
+    for (int q = j.member_begin[r]; q < j.member_begin[r + 1]; ++q) {
+      const int s = j.members[q];
+      g->entries[s] = entries[k]; g->entry_counts[s] = counts[k]; g->entry_chunk[s] = chunk;
+      const int c = j.canon_of[s];
+      if (c >= 0 && !pr.have[c]) { pr.entries[c] = entries[k]; pr.counts[c] = counts[k]; pr.have[c] = 1; }
+    }
+    pr.built = true;
+    if (chunk >= 0 && std::find(pr.chunks.begin(), pr.chunks.end(), chunk) == pr.chunks.end()) { pr.chunks.push_back(chunk); pool.note_rule_in_chunk(j.in.pool_id[rule], chunk); }
+    if (j.status[r] != 2) { j.status[r] = 2; --j.n_missing; }
+  }
+  if (chunk >= 0 && std::find(g->chunk_refs.begin(), g->chunk_refs.end(), chunk) == g->chunk_refs.end()) {
+    g->chunk_refs.push_back(chunk);
+    pool.retain(std::vector<int>{chunk});
+  }
+}
+
+// This grammar's lookahead narrows the check lists of the entries just published for `d_states` (only in its own
+// device copy of the headers: the pool keeps them context-free).  `go`: device flag, the step is skipped when it is 0.
+static void jit_enqueue_narrowing(xg_grammar* g, const JitScratch& sc, const CachePool::JitArena* arena, const int32_t* d_states, int n,
+                                  const int* go, cudaStream_t stream) {
+  EntryDev* dev_entries = const_cast<EntryDev*>(g->host_view.entries);
+  lookahead_count_kernel<<<n, 256, 0, stream>>>(g->host_view, g->tok->dev, d_states, sc.list_counts, go);
+  jit_reserve_lists_kernel<<<1, 32, 0, stream>>>(sc.list_counts, n, sc.list_offsets, arena->d_used, arena->cap_words, go, sc.go_lists);
+  lookahead_compact_kernel<<<n, 256, 0, stream>>>(g->host_view, g->tok->dev, d_states, sc.list_offsets, sc.list_counts, arena->base, sc.go_lists);
+  jit_patch_lists_kernel<<<(g->flat.n_states + 255) / 256, 256, 0, stream>>>(dev_entries, g->jit.d_rep, g->flat.n_states, d_states, sc.list_counts,
+                                                                             sc.list_offsets, arena->base, n, sc.go_lists);
+}
+
+// publish host-side entry headers for `reps` (pool hits, or entries built by the synchronous path)
+static xg_status_t jit_publish_from_host(xg_grammar* g, const std::vector<int32_t>& reps, const std::vector<EntryDev>& entries, cudaStream_t stream) {
+  JitState& j = g->jit;
+  for (size_t begin = 0; begin < reps.size(); begin += kJitBatchMax) {
+    const int n = (int)std::min<size_t>(kJitBatchMax, reps.size() - begin);
+    // pageable sources: the runtime stages them before these calls return
+    XG_CUDA(cudaMemcpyAsync(j.d_pub_state, reps.data() + begin, n * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+    XG_CUDA(cudaMemcpyAsync(j.d_pub_entry, entries.data() + begin, n * sizeof(EntryDev), cudaMemcpyHostToDevice, stream));
+    jit_publish_kernel<<<(g->flat.n_states + 255) / 256, 256, 0, stream>>>(const_cast<EntryDev*>(g->host_view.entries), j.d_rep, g->flat.n_states,
+                                                                           j.d_pub_state, j.d_pub_entry, n, nullptr);
+    const CachePool::JitArena* arena = g->pool->jit_arena(0, false);
+    JitScratch sc;
+    if (arena && jit_scratch(*g->pool, g->tok->n_words, &sc)) {
+      if (std::find(g->chunk_refs.begin(), g->chunk_refs.end(), arena->chunk) == g->chunk_refs.end()) {
+        g->chunk_refs.push_back(arena->chunk);
+        g->pool->retain(std::vector<int>{arena->chunk});
+      }
+      jit_enqueue_narrowing(g, sc, arena, j.d_pub_state, n, sc.one, stream);
+    }
+    XG_CUDA(cudaGetLastError());
+  }
+  return XG_OK;
+}
+
+// Enqueue the build of `reps` (at most kJitBatchMax, one grammar) without any host round trip; its
+// results go to slice (`entry_offset`, `index`) of the pool's pinned result block.
+static xg_status_t jit_enqueue_build(JitPool* jp, xg_grammar* g, const std::vector<int32_t>& reps, bool renew_arena, long long min_words,
+                                     int entry_offset, int index, cudaStream_t stream) {
+  JitState& j = g->jit;
+  CachePool& pool = *g->pool;
+  const VocabDev& v = g->tok->dev;
+  const int W = v.n_words, V = v.vocab_size, n = (int)reps.size();
+  const size_t row_bytes = (size_t)W * 4;
+  const CachePool::JitArena* arena = pool.jit_arena(min_words, renew_arena);
+  if (!arena) return set_error(XG_ERR_OOM, "just-in-time arena allocation failed");
+  JitScratch sc;
+  if (!jit_scratch(pool, W, &sc)) return set_error(XG_ERR_OOM, "just-in-time scratch allocation failed");
+  if (std::find(g->chunk_refs.begin(), g->chunk_refs.end(), arena->chunk) == g->chunk_refs.end()) {     // in use from now on
+    g->chunk_refs.push_back(arena->chunk);
+    pool.retain(std::vector<int>{arena->chunk});
+  }
+  uint32_t* acc = sc.rows;
+  uint32_t* unc = sc.rows + (size_t)kJitBatchMax * W;
+  uint32_t* unr = sc.rows + 2 * (size_t)kJitBatchMax * W;
+  XG_CUDA(cudaMemcpyAsync(sc.pos, reps.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+  XG_CUDA(cudaMemsetAsync(acc, 0, row_bytes * n, stream));
+  XG_CUDA(cudaMemsetAsync(unc, 0, row_bytes * n, stream));
+  XG_CUDA(cudaMemsetAsync(unr, 0, row_bytes * n, stream));
+  XG_CUDA(cudaMemsetAsync(sc.over_count, 0, 2 * sizeof(int), stream));
+  classify_kernel<<<dim3((V + 255) / 256, n), 256, 0, stream>>>(g->host_view, v, sc.pos, acc, unc, unr, sc.over, sc.over_count, 64);
+  count_kernel<<<n, 256, 0, stream>>>(acc, unc, W, sc.counts);
+  plan_kernel<<<1, 1024, 0, stream>>>(sc.counts, n, V, W, sc.plan, sc.total);
+  jit_reserve_kernel<<<1, 32, 0, stream>>>(sc.plan, n, sc.total, arena->d_used, arena->cap_words, sc.over_count, sc.result);
+  pack_kernel<<<n, 256, 0, stream>>>(acc, unc, unr, sc.plan, V, W, arena->base, sc.entries, sc.result);
+  exit_kernel<<<n, 256, 0, stream>>>(g->host_view, v, sc.pos, sc.entries, sc.result);
+  jit_publish_kernel<<<(g->flat.n_states + 255) / 256, 256, 0, stream>>>(const_cast<EntryDev*>(g->host_view.entries), j.d_rep, g->flat.n_states,
+                                                                         sc.pos, sc.entries, n, sc.result);
+  jit_enqueue_narrowing(g, sc, arena, sc.pos, n, sc.result, stream);
+  XG_CUDA(cudaGetLastError());
+  // the scratch is reused by the next build in stream order: take the results out first
+  XG_CUDA(cudaMemcpyAsync(jp->h->entries + entry_offset, sc.entries, n * sizeof(EntryDev), cudaMemcpyDeviceToHost, stream));
+  XG_CUDA(cudaMemcpyAsync(jp->h->counts + entry_offset, sc.counts, n * sizeof(int2), cudaMemcpyDeviceToHost, stream));
+  XG_CUDA(cudaMemcpyAsync(jp->h->result[index], sc.result, 2 * sizeof(int), cudaMemcpyDeviceToHost, stream));
+  XG_CUDA(cudaMemcpyAsync(&jp->h->total_words[index], sc.total, sizeof(long long), cudaMemcpyDeviceToHost, stream));
+  JitFlight fl;
+  fl.g = g; fl.reps = reps; fl.chunk = arena->chunk; fl.entry_offset = entry_offset; fl.index = index;
+  jp->flights.push_back(fl);
+  for (int r : reps) j.status[r] = 1;
+  j.n_in_flight += n;
+  return XG_OK;
+}
+
+// One pool's cycle over the grammars in `eligible`.  *idle = true once a snapshot taken inside this
+// call held nothing new and nothing is in flight (only reachable with wait).
+static xg_status_t jit_advance(CachePool& pool, const std::vector<xg_grammar*>& eligible, cudaStream_t stream, bool wait, bool* idle) {
+  JitPool* jp = (JitPool*)pool.jit_host;
+  bool fresh = false;            // the snapshot being looked at was taken inside this call
+  *idle = false;
+  for (int guard = 0; guard < 100000; ++guard) {
+    if (jp->phase == 0) {
+      bool any_missing = false;
+      for (xg_grammar* g : eligible) any_missing = any_missing || g->jit.n_missing > 0;
+      if (!any_missing) { *idle = true; return XG_OK; }           // everything is built: nothing can be reported any more
+      XG_CUDA(cudaMemcpyAsync(&jp->h->ring, jp->d_ring, sizeof(JitRing), cudaMemcpyDeviceToHost, stream));
+      XG_CUDA(cudaEventRecord(jp->ev, stream));
+      jp->phase = 1;
+      fresh = true;
+      if (!wait) return XG_OK;
+      continue;
+    }
+    if (wait) XG_CUDA(cudaEventSynchronize(jp->ev));
+    else {
+      cudaError_t q = cudaEventQuery(jp->ev);
+      if (q == cudaErrorNotReady) return XG_OK;
+      if (q != cudaSuccess) return set_error(XG_ERR_CUDA, std::string("just-in-time event: ") + cudaGetErrorString(q));
+    }
+    if (jp->phase == 2) {                      // the builds have finished
+      std::vector<JitFlight> flights;
+      flights.swap(jp->flights);
+      jp->phase = 0;
+      std::vector<JitFlight> again;
+      for (JitFlight& fl : flights) {
+        xg_grammar* g = fl.g;
+        g->jit.n_in_flight -= (int)fl.reps.size();
+        const int* result = jp->h->result[fl.index];
+        if (result[0] == 1) {
+          jit_record(g, fl.reps, jp->h->entries + fl.entry_offset, jp->h->counts + fl.entry_offset, fl.chunk);
+          g->jit.n_built += (int)fl.reps.size();
+        } else if (result[1] == 1) {           // no room: the same states again, in a larger arena
+          for (int r : fl.reps) g->jit.status[r] = 0;
+          again.push_back(fl);
+        } else {                               // a walk left the fast path: the exact build with its host round trips
+          for (int r : fl.reps) g->jit.status[r] = 0;
+          xg_status_t st = build_entries(g, fl.reps, stream);
+          if (st != XG_OK) return st;
+          std::vector<EntryDev> es;
+          std::vector<int2> cs;
+          for (int r : fl.reps) { es.push_back(g->entries[r]); cs.push_back(g->entry_counts[r]); }
+          st = jit_publish_from_host(g, fl.reps, es, stream);
+          if (st != XG_OK) return st;
+          for (size_t k = 0; k < fl.reps.size(); ++k) jit_record(g, std::vector<int32_t>{fl.reps[k]}, &es[k], &cs[k], g->entry_chunk[fl.reps[k]]);
+          g->jit.n_built += (int)fl.reps.size();
+        }
+      }
+      if (!again.empty()) {
+        long long need = 1 << 16;
+        for (JitFlight& fl : again) need += jp->h->total_words[fl.index];
+        bool renew = true;
+        for (JitFlight& fl : again) {
+          xg_status_t st = jit_enqueue_build(jp, fl.g, fl.reps, renew, need, fl.entry_offset, fl.index, stream);
+          if (st != XG_OK) return st;
+          renew = false;
+        }
+        XG_CUDA(cudaEventRecord(jp->ev, stream));
+        jp->phase = 2;
+        if (!wait) return XG_OK;
+      }
+      continue;
+    }
+    // phase 1: a snapshot of the miss ring has arrived
+    jp->phase = 0;
+    const uint32_t count = jp->h->ring.count;
+    uint32_t from = jp->ring_seen;
+    if (count - from > (uint32_t)kJitRingCap) from = count - kJitRingCap;
+    std::vector<std::pair<xg_grammar*, std::vector<int32_t>>> want;      // in order of first report
+    for (uint32_t i = from; i != count; ++i) {
+      const int2 m = jp->h->ring.miss[i % kJitRingCap];
+      if (m.x < 0 || m.x >= (int)jp->slots.size()) continue;
+      xg_grammar* g = jp->slots[m.x];
+      if (!g || std::find(eligible.begin(), eligible.end(), g) == eligible.end()) continue;
+      if (m.y < 0 || m.y >= g->flat.n_states) continue;
+      const int r = g->jit.rep[m.y];
+      if (g->jit.status[r] != 0) continue;
+      size_t w = 0;
+      while (w < want.size() && want[w].first != g) ++w;
+      if (w == want.size()) want.emplace_back(g, std::vector<int32_t>());
+      if (std::find(want[w].second.begin(), want[w].second.end(), r) == want[w].second.end()) want[w].second.push_back(r);
+    }
+    jp->ring_seen = count;
+    if (want.empty()) {
+      if (wait && fresh) { *idle = true; return XG_OK; }
+      continue;                                // take a fresh snapshot
+    }
+    fresh = false;
+    int entry_offset = 0, index = 0;
+    for (auto& gw : want) {
+      xg_grammar* g = gw.first;
+      JitState& j = g->jit;
+      const FlatGrammar& f = g->flat;
+      // cache hit (Section 3.5): the pool already holds the entry (another grammar has built it since)
+      std::vector<int32_t> hit_reps, build_reps;
+      std::vector<EntryDev> hit_entries;
+      std::vector<int2> hit_counts;
+      for (int r : gw.second) {
+        const PoolRule& pr = pool.rule(j.in.pool_id[f.state_rule[r]]);
+        const int c = j.canon_of[r];
+        if (pr.built && c >= 0 && c < (int)pr.have.size() && pr.have[c]) {
+          hit_reps.push_back(r); hit_entries.push_back(pr.entries[c]); hit_counts.push_back(pr.counts[c]);
+          for (int ch : pr.chunks)
+            if (std::find(g->chunk_refs.begin(), g->chunk_refs.end(), ch) == g->chunk_refs.end()) { g->chunk_refs.push_back(ch); pool.retain(std::vector<int>{ch}); }
+        } else if ((int)build_reps.size() < kJitBatchMax && entry_offset + (int)build_reps.size() < kJitCycleEntries && index < kJitCycleBuilds)
+          build_reps.push_back(r);                   // what does not fit this cycle is reported again by a later fill
+      }
+      if (!hit_reps.empty()) {
+        xg_status_t st = jit_publish_from_host(g, hit_reps, hit_entries, stream);
+        if (st != XG_OK) return st;
+        for (size_t k = 0; k < hit_reps.size(); ++k) jit_record(g, std::vector<int32_t>{hit_reps[k]}, &hit_entries[k], &hit_counts[k], -1);
+        j.n_pool_hits += (int)hit_reps.size();
+      }
+      if (!build_reps.empty()) {
+        xg_status_t st = jit_enqueue_build(jp, g, build_reps, false, 0, entry_offset, index, stream);
+        if (st != XG_OK) return st;
+        entry_offset += (int)build_reps.size();
+        ++index;
+      }
+    }
+    if (!jp->flights.empty()) {
+      XG_CUDA(cudaEventRecord(jp->ev, stream));
+      jp->phase = 2;
+      if (!wait) return XG_OK;
+    }
+  }
+  return set_error(XG_ERR_TIMEOUT, "just-in-time service did not settle");
+}
+
 xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool, xg_grammar_kind_t kind, const char* text, size_t len,
                                const char* root_rule, const xg_compile_options_t* opt, void* stream, xg_grammar_t** out) {
   if (!out) return set_error(XG_ERR_INVALID_ARG, "out is NULL");
   *out = nullptr;
   if (!text) return set_error(XG_ERR_INVALID_ARG, "text is NULL");
   FrontendOptions fo;
-  bool build_cache = tok != nullptr, compress = true;
+  bool build_cache = tok != nullptr, compress = true, jit = false;
+  int jit_precompute = 0;
   if (opt) {
     if (opt->struct_size < 8) return set_error(XG_ERR_INVALID_ARG, "bad options struct_size");
     if (opt->inline_max_states >= 0) fo.inline_max_states = opt->inline_max_states;
     if (opt->struct_size >= 12 && opt->max_rule_states > 0) fo.max_rule_states = opt->max_rule_states;
     if (opt->struct_size >= 16 && opt->build_cache == 0) build_cache = false;
     if (opt->struct_size >= 20 && opt->no_state_compression != 0) compress = false;
+    if (opt->struct_size >= 28 && opt->jit != 0) { jit = true; jit_precompute = std::max(0, opt->jit_precompute); }
   }
   if (pool && pool->impl->owner() != (const void*)tok) return set_error(XG_ERR_INVALID_ARG, "the pool belongs to another tokenizer");
   std::unique_ptr<xg_grammar> g(new xg_grammar());
@@ -443,10 +820,16 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     g->chunk_refs.clear();
     pool_keep->free_plain(g->blob); pool_keep->free_plain(g->lookahead_arena);
     g->blob = g->lookahead_arena = nullptr;
+    jit_release(g.get());
     xg_grammar_destroy(g.release());
     return status;
   };
-  xg_status_t st = upload_grammar(g.get());
+  xg_status_t st = XG_OK;
+  if (jit) {
+    st = jit_allocate(g.get());
+    if (st != XG_OK) return fail(st);
+  }
+  st = upload_grammar(g.get());
   if (st != XG_OK) return fail(st);
   // cross-grammar cache (Section 3.3): rules whose canonical structure is already in the pool
   // reuse its entries; the others are classified now and registered afterwards
@@ -468,15 +851,20 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   else for (int s = 0; s < f.n_states; ++s) rep[s] = s;
   std::map<int, int> builder_of;                      // pool rule -> the rule of this grammar that builds it
   std::vector<int32_t> to_build;
+  auto in_pool = [&](int s) {
+    const PoolRule& pr = g->pool->rule(in.pool_id[f.state_rule[s]]);
+    return pr.built && canon_of[s] < (int)pr.have.size() && pr.have[canon_of[s]];
+  };
   for (int s : scannable) {
     const int r = f.state_rule[s];
     PoolRule& pr = g->pool->rule(in.pool_id[r]);
-    if (pr.built) {
+    if (in_pool(s)) {
       g->entries[s] = pr.entries[canon_of[s]];
       g->entry_counts[s] = pr.counts[canon_of[s]];
       ++g->stats.n_entries_reused;
       for (int c : pr.chunks) if (std::find(g->chunk_refs.begin(), g->chunk_refs.end(), c) == g->chunk_refs.end()) g->chunk_refs.push_back(c);
     } else {
+      g->entries[s].kind = kEntryNotBuilt;
       auto it = builder_of.find(in.pool_id[r]);
       if (it == builder_of.end()) it = builder_of.emplace(in.pool_id[r], r).first;
       if (it->second == r) {
@@ -484,10 +872,28 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
       }
     }
   }
+  if (jit) {
+    // configurable JIT (Section 3.5): only the K costliest of the missing entries are built now.
+    // Cost of an entry = the tokens that pass its state's own first-byte test (the others are
+    // rejected before a walk starts).
+    std::vector<std::pair<int64_t, int32_t>> cost;
+    for (int s : to_build) {
+      int64_t c = 0;
+      uint32_t own[8] = {};
+      for (int e = f.cedge_begin[s]; e < f.cedge_begin[s + 1]; ++e)
+        for (int w = 0; w < 8; ++w) own[w] |= f.class_bits[(size_t)f.cedge_class[e] * 8 + w];
+      for (int b = 0; b < 256; ++b) if ((own[b >> 5] >> (b & 31)) & 1u) c += tok->first_byte_count[b];
+      cost.emplace_back(-c, s);
+    }
+    std::sort(cost.begin(), cost.end());
+    to_build.clear();
+    for (int k = 0; k < (int)cost.size() && k < jit_precompute; ++k) to_build.push_back(cost[k].second);
+    std::sort(to_build.begin(), to_build.end());
+  }
   st = build_entries(g.get(), to_build, (cudaStream_t)stream);
   if (st != XG_OK) return fail(st);
   for (int s : scannable) {                           // the other members of each class
-    if (rep[s] == s) continue;
+    if (rep[s] == s || g->entries[s].kind != kEntryNotBuilt) continue;
     auto it = builder_of.find(in.pool_id[f.state_rule[s]]);
     if (it == builder_of.end() || it->second != f.state_rule[s]) continue;
     g->entries[s] = g->entries[rep[s]]; g->entry_counts[s] = g->entry_counts[rep[s]]; g->entry_chunk[s] = g->entry_chunk[rep[s]];
@@ -498,14 +904,17 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     const int n_local = (int)in.canon[r].size();
     pr.entries.resize(n_local);
     pr.counts.resize(n_local);
+    pr.have.resize(n_local, 0);
     for (int k = 0; k < n_local; ++k) {
       const int s = rule_first[r] + in.canon[r][k];
+      if (pr.have[k] || g->entries[s].kind == kEntryNotBuilt) continue;
       pr.entries[k] = g->entries[s]; pr.counts[k] = g->entry_counts[s];
+      pr.have[k] = 1;
+      pr.built = true;
       const int c = g->entry_chunk[s];
       if (c >= 0 && std::find(pr.chunks.begin(), pr.chunks.end(), c) == pr.chunks.end()) { pr.chunks.push_back(c); g->pool->note_rule_in_chunk(kv.first, c); }
     }
     for (int c : pr.chunks) if (std::find(g->chunk_refs.begin(), g->chunk_refs.end(), c) == g->chunk_refs.end()) g->chunk_refs.push_back(c);
-    pr.built = true;
   }
   g->pool->retain(g->chunk_refs);
   retained = true;
@@ -514,10 +923,27 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     const int r = f.state_rule[s];
     auto it = builder_of.find(in.pool_id[r]);
     if (it == builder_of.end() || it->second == r) continue;
+    if (!in_pool(s)) continue;                        // a just-in-time grammar: not built yet
     const PoolRule& pr = g->pool->rule(in.pool_id[r]);
     g->entries[s] = pr.entries[canon_of[s]];
     g->entry_counts[s] = pr.counts[canon_of[s]];
     ++g->stats.n_entries_reused;
+  }
+  if (jit) {
+    JitState& j = g->jit;
+    j.rep = rep;
+    j.in = in; j.canon_of = canon_of; j.rule_first = rule_first;
+    j.status.assign(f.n_states, 2);
+    std::vector<int32_t> count(f.n_states + 1, 0);
+    for (int s2 = 0; s2 < f.n_states; ++s2) ++count[rep[s2] + 1];
+    for (int s2 = 0; s2 < f.n_states; ++s2) count[s2 + 1] += count[s2];
+    j.member_begin = count;
+    j.members.resize(f.n_states);
+    { std::vector<int32_t> at(count.begin(), count.end() - 1); for (int s2 = 0; s2 < f.n_states; ++s2) j.members[at[rep[s2]]++] = s2; }
+    for (int s2 : scannable) if (rep[s2] == s2 && g->entries[s2].kind == kEntryNotBuilt) { j.status[s2] = 0; ++j.n_missing; }
+    if (cudaMemcpy(j.d_rep, rep.data(), (size_t)f.n_states * 4, cudaMemcpyHostToDevice) != cudaSuccess)
+      return fail(set_error(XG_ERR_CUDA, "upload of the state classes failed"));
+    j.enabled = true;
   }
   st = upload_grammar(g.get());       // now with the entry headers
   if (st == XG_OK) st = narrow_check_lists(g.get(), scannable, rep, (cudaStream_t)stream);
@@ -528,6 +954,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   g->stats.pairs_classified = (int64_t)to_build.size() * tok->vocab_size;
   for (int s : scannable) {
     const EntryDev& e = g->entries[s];
+    if (e.kind == kEntryNotBuilt) continue;
     const int2 c = g->entry_counts[s];
     g->stats.total_accepted += c.x;
     g->stats.total_uncertain += c.y;
@@ -540,8 +967,39 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   return XG_OK;
 }
 
+xg_status_t xg_jit_service(xg_grammar_t* const* grammars, int32_t n, void* stream, int32_t wait, xg_jit_stats_t* out) {
+  if (n < 0 || (n > 0 && !grammars)) return set_error(XG_ERR_INVALID_ARG, "bad grammar array");
+  std::vector<std::pair<CachePool*, std::vector<xg_grammar*>>> pools;      // the just-in-time grammars by pool
+  for (int i = 0; i < n; ++i) {
+    xg_grammar* g = grammars[i];
+    if (!g) return set_error(XG_ERR_INVALID_ARG, "NULL grammar");
+    if (!g->jit.enabled) continue;
+    size_t k = 0;
+    while (k < pools.size() && pools[k].first != g->pool.get()) ++k;
+    if (k == pools.size()) pools.emplace_back(g->pool.get(), std::vector<xg_grammar*>());
+    if (std::find(pools[k].second.begin(), pools[k].second.end(), g) == pools[k].second.end()) pools[k].second.push_back(g);
+  }
+  xg_jit_stats_t total{};
+  for (auto& pg : pools) {
+    std::lock_guard<std::mutex> lock(pg.first->mu);
+    bool idle = false;
+    xg_status_t st = jit_advance(*pg.first, pg.second, (cudaStream_t)stream, wait != 0, &idle);
+    if (st != XG_OK) return st;
+    for (xg_grammar* g : pg.second) {
+      total.n_built += g->jit.n_built; total.n_pool_hits += g->jit.n_pool_hits;
+      total.n_in_flight += g->jit.n_in_flight; total.n_missing += g->jit.n_missing;
+    }
+  }
+  if (out) *out = total;
+  return XG_OK;
+}
+
 void xg_grammar_destroy(xg_grammar_t* g) {
   if (!g) return;
+  if (g->jit.d_rep || g->jit.slot >= 0) {
+    std::lock_guard<std::mutex> lock(g->pool->mu);
+    jit_release(g);
+  }
   if (g->pool && (g->blob || g->lookahead_arena || !g->chunk_refs.empty())) {
     cudaDeviceSynchronize();             // its tables go back to the pool's slabs: nothing may still read them
     std::lock_guard<std::mutex> lock(g->pool->mu);
@@ -597,6 +1055,7 @@ xg_status_t xg_grammar_get_cache_entry(const xg_grammar_t* g, int32_t state, xg_
   const FlatGrammar& f = g->flat;
   if (state < 0 || state >= f.n_states || f.cedge_begin[state + 1] == f.cedge_begin[state]) return set_error(XG_ERR_INVALID_ARG, "state is not scannable");
   const EntryDev& e = g->entries[state];
+  if (e.kind == kEntryNotBuilt) return set_error(XG_ERR_INVALID_ARG, "the entry of this state has not been built yet (just-in-time grammar)");
   const int2 c = g->entry_counts[state];
   XG_CUDA(cudaDeviceSynchronize());
   view->state = state; view->kind = e.kind;

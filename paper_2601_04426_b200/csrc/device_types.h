@@ -3,6 +3,8 @@
 #include <cstddef>
 #include <cstdint>
 
+#include <vector_types.h>
+
 namespace xg {
 
 // Vocabulary, sorted by token bytes (trie order): tokens that share a prefix are adjacent, so
@@ -36,10 +38,21 @@ struct EntryDev {
   const uint8_t* chk_byte;
   int32_t n_chk;
   int32_t pad2;
-  int32_t kind;              // xg_store_kind_t
+  int32_t kind;              // xg_store_kind_t; kEntryNotBuilt while a just-in-time grammar has not built it yet
   int32_t n_list;            // list length (0 for bitset)
   int32_t n_unc;
   int32_t n_acc;
+};
+
+constexpr int32_t kEntryNotBuilt = -1;
+
+// Just-in-time cache build (Section 3.5): the fill kernels report the scannable states whose
+// entry they found missing here; the host reads the ring between steps and builds them.
+constexpr int kJitRingCap = 1024;
+struct JitRing {                  // one per cache pool, shared by its just-in-time grammars
+  uint32_t count;                 // reports so far (monotonic); report i is miss[i % kJitRingCap]
+  uint32_t pad[3];
+  int2 miss[kJitRingCap];         // (the grammar's slot in the pool, state)
 };
 
 // Everything a walk needs to know about one automaton state, in one 32-byte record (two 16-byte
@@ -69,6 +82,9 @@ struct GrammarDev {
   const uint32_t* state_first;    // [S][8] bytes that the state's scan list (own and predicted edges) can take
   const uint32_t* rule_follow;    // [R][8] bytes that can follow a completed rule somewhere in this grammar
   const EntryDev* entries;        // [S]; meaningful for scannable states
+  JitRing* miss_ring;             // just-in-time grammars only (else nullptr)
+  int32_t jit_slot;               // this grammar's number in the ring's reports
+  int32_t pad3;
 };
 
 // What the next mask needs from the current Earley set, worked out once when the set is made
@@ -81,6 +97,7 @@ struct GrammarDev {
 constexpr int kPlanMergeMax = 64;
 constexpr int kPlanCheckMax = 32;
 constexpr int kContCap = 16;
+constexpr int kPlanMissingMax = 8;
 struct __align__(16) StepPlan {
   int32_t n_merge, n_check, eos_ok, overflow;
   uint32_t cont_first[kPlanCheckMax][8];     // read and written as 16-byte vectors: keep 16-byte aligned
@@ -91,6 +108,10 @@ struct __align__(16) StepPlan {
   int32_t check_origin[kPlanCheckMax];
   int32_t cont_cnt[kPlanCheckMax];
   int32_t check_cum[kPlanCheckMax + 1];      // running totals of uncertain tokens
+  // just-in-time grammars: scannable states of the current set whose entry is not built yet.  While there are any,
+  // the step's mask comes from walking the whole vocabulary against the full Earley state (the plain definition).
+  int32_t n_missing;                         // may exceed kPlanMissingMax; the first kPlanMissingMax are listed
+  int32_t missing_state[kPlanMissingMax];
 };
 static_assert(offsetof(StepPlan, cont_first) % 16 == 0, "cont_first must be 16-byte aligned");
 

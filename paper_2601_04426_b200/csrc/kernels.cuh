@@ -336,8 +336,10 @@ __device__ __forceinline__ void compact_bits(F word_fn, int n_words, uint32_t* _
 
 __global__ void __launch_bounds__(256)
 pack_kernel(const uint32_t* __restrict__ acc_id, const uint32_t* __restrict__ unc_id, const uint32_t* __restrict__ unc_rank,
-            const PackPlan* __restrict__ plan, int vocab_size, int n_words, uint32_t* __restrict__ arena, EntryDev* __restrict__ entries) {
+            const PackPlan* __restrict__ plan, int vocab_size, int n_words, uint32_t* __restrict__ arena, EntryDev* __restrict__ entries,
+            const int* __restrict__ go) {
   __shared__ int sh_scan[256];
+  if (go && !*go) return;                 // a just-in-time build that found no room (see jit_reserve_kernel)
   const int p = blockIdx.x;
   const PackPlan pl = plan[p];
   const uint32_t* a = acc_id + (size_t)p * n_words;
@@ -371,7 +373,8 @@ pack_kernel(const uint32_t* __restrict__ acc_id, const uint32_t* __restrict__ un
 // the entry's rule (bit j = after j bytes).  The run-time check restarts there instead of
 // re-walking the part of the token that the cache already decided.  0 = unknown (walk in full).
 __global__ void __launch_bounds__(256)
-exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, const EntryDev* __restrict__ entries) {
+exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, const EntryDev* __restrict__ entries, const int* __restrict__ go) {
+  if (go && !*go) return;
   __shared__ uint32_t sh_st[1];
   __shared__ int32_t sh_org[1];
   __shared__ uint32_t sh_class[kSharedClasses * 8];
@@ -420,8 +423,9 @@ __device__ __forceinline__ uint32_t narrow_exits(const VocabDev& v, const uint32
 }
 
 __global__ void __launch_bounds__(256)
-lookahead_count_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ states, int32_t* __restrict__ counts) {
+lookahead_count_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ states, int32_t* __restrict__ counts, const int* __restrict__ go) {
   __shared__ int sh[8];
+  if (go && !*go) return;
   const int q = states[blockIdx.x];
   const EntryDev e = g.entries[q];
   const uint32_t* follow = g.rule_follow + (size_t)(g.state[q].info & 0x7FFFFFFFu) * 8;
@@ -436,8 +440,9 @@ lookahead_count_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ sta
 
 __global__ void __launch_bounds__(256)
 lookahead_compact_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ states, const long long* __restrict__ offsets,
-                         const int32_t* __restrict__ counts, uint32_t* __restrict__ arena) {
+                         const int32_t* __restrict__ counts, uint32_t* __restrict__ arena, const int* __restrict__ go) {
   __shared__ int sh_scan[256];
+  if (go && !*go) return;
   const int q = states[blockIdx.x];
   const EntryDev e = g.entries[q];
   const uint32_t* follow = g.rule_follow + (size_t)(g.state[q].info & 0x7FFFFFFFu) * 8;
@@ -474,6 +479,77 @@ lookahead_compact_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ s
 }
 
 // ------------------------------------------------------------------------------------------
+// Just-in-time cache build (Section 3.5): the same classify / count / plan / pack / exit kernels,
+// enqueued between decode steps without a host round trip.  The two things the host does in the
+// compile-time build -- sizing the arena from the plan's total and checking for walks that left
+// the fast path -- happen here on the device.
+// ------------------------------------------------------------------------------------------
+// result[0]: 1 = go on, 0 = stop (result[1] says why: 1 = no room in the arena, 2 = a token walk
+// needs the exact slow path, which only the host can set up)
+__global__ void jit_reserve_kernel(PackPlan* __restrict__ plan, int n_pos, const long long* __restrict__ total_words,
+                                   unsigned long long* __restrict__ arena_used, long long arena_cap,
+                                   const int* __restrict__ overflow_count, int* __restrict__ result) {
+  if (blockIdx.x != 0 || threadIdx.x != 0) return;
+  result[0] = 0; result[1] = 0;
+  if (*overflow_count > 0) { result[1] = 2; return; }
+  const unsigned long long need = (unsigned long long)max(*total_words, 1LL);
+  const unsigned long long base = atomicAdd(arena_used, need);
+  if (base + need > (unsigned long long)arena_cap) { result[1] = 1; return; }
+  for (int p = 0; p < n_pos; ++p) plan[p].offset_words += (long long)base;
+  result[0] = 1;
+}
+
+// Make freshly built entries visible to the fill kernels: every state whose class representative
+// was built takes the representative's entry.  `built_state` / `built_entry`: the n entries.
+__global__ void __launch_bounds__(256)
+jit_publish_kernel(EntryDev* __restrict__ entries, const int32_t* __restrict__ rep, int n_states,
+                   const int32_t* __restrict__ built_state, const EntryDev* __restrict__ built_entry, int n, const int* __restrict__ go) {
+  if (go && !*go) return;
+  const int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s >= n_states) return;
+  const int r = rep[s];
+  for (int k = 0; k < n; ++k)
+    if (built_state[k] == r) { entries[s] = built_entry[k]; return; }
+}
+
+// Lookahead narrowing of just-built entries (Section 3.3), again without the host: room for the
+// narrowed check lists comes from the same arena.  If there is none the entries simply keep their
+// whole uncertain lists as check lists.
+__global__ void jit_reserve_lists_kernel(const int32_t* __restrict__ counts, int n, long long* __restrict__ offsets,
+                                         unsigned long long* __restrict__ arena_used, long long arena_cap,
+                                         const int* __restrict__ go, int* __restrict__ go_lists) {
+  if (blockIdx.x != 0 || threadIdx.x != 0) return;
+  *go_lists = 0;
+  if (!*go) return;
+  unsigned long long need = 1;
+  for (int k = 0; k < n; ++k) need += 2ull * counts[k] + (counts[k] + 3) / 4;
+  const unsigned long long base = atomicAdd(arena_used, need);
+  if (base + need > (unsigned long long)arena_cap) return;
+  long long run = (long long)base;
+  for (int k = 0; k < n; ++k) { offsets[k] = run; run += 2LL * counts[k] + (counts[k] + 3) / 4; }
+  *go_lists = 1;
+}
+
+__global__ void __launch_bounds__(256)
+jit_patch_lists_kernel(EntryDev* __restrict__ entries, const int32_t* __restrict__ rep, int n_states, const int32_t* __restrict__ built_state,
+                       const int32_t* __restrict__ counts, const long long* __restrict__ offsets, const uint32_t* __restrict__ arena, int n,
+                       const int* __restrict__ go_lists) {
+  if (!*go_lists) return;
+  const int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s >= n_states) return;
+  const int r = rep[s];
+  for (int k = 0; k < n; ++k)
+    if (built_state[k] == r) {
+      EntryDev& e = entries[s];
+      e.chk_rank = arena + offsets[k];
+      e.chk_exit = e.chk_rank + counts[k];
+      e.chk_byte = reinterpret_cast<const uint8_t*>(e.chk_exit + counts[k]);
+      e.n_chk = counts[k];
+      return;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // matcher state
 // ------------------------------------------------------------------------------------------
 // is the root rule complete in the current set (EOS allowed)?
@@ -496,7 +572,7 @@ __device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g,
   const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
   int n_check = 0;
   if (lane == 0) {
-    int n_merge = 0, overflow = 0;
+    int n_merge = 0, overflow = 0, n_missing = 0;
     p.check_cum[0] = 0;
     for (int i = 0; i < hist.i_cnt && !overflow; ++i) {
       const uint32_t s = hist.i_st[i];
@@ -506,6 +582,11 @@ __device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g,
         const int q = code & 0x7FFFFFFF;
         const int origin = code < 0 ? n : hist.i_org[i];          // predicted start states begin here
         bool seen = false;
+        if (g.entries[q].kind == kEntryNotBuilt) {                // a just-in-time grammar has not built this entry yet
+          for (int z = 0; z < min(n_missing, kPlanMissingMax); ++z) seen = seen || p.missing_state[z] == q;
+          if (!seen) { if (n_missing < kPlanMissingMax) p.missing_state[n_missing] = q; ++n_missing; }
+          continue;
+        }
         for (int z = 0; z < n_merge; ++z) seen = seen || p.merge_state[z] == q;
         if (!seen) { if (n_merge == kPlanMergeMax) { overflow = 1; break; } p.merge_state[n_merge++] = q; }
         const int n_unc = g.entries[q].n_chk;
@@ -519,7 +600,7 @@ __device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g,
         ++n_check;
       }
     }
-    p.n_merge = n_merge; p.n_check = n_check; p.overflow = overflow;
+    p.n_merge = n_merge; p.n_check = n_check; p.overflow = overflow; p.n_missing = n_missing;
     p.eos_ok = root_complete(m, g) ? 1 : 0;
   }
   n_check = __shfl_sync(0xFFFFFFFFu, n_check, 0);
@@ -647,6 +728,29 @@ __device__ __forceinline__ int lower_bound_u32(const uint32_t* __restrict__ a, i
   return lo;
 }
 
+// Just-in-time grammars (Section 3.5): while an entry of the current set is not built, the mask
+// is the plain definition -- every token walked against the full Earley state.  The bytes the
+// current set can scan at all (OR of the per-state first-byte sets) reject most tokens before a
+// walk starts.  One warp computes it.
+__device__ __forceinline__ void current_first_bytes(const GrammarDev& g, const Chart& hist, uint32_t* out8, int lane) {
+  if (lane < 8) {
+    uint32_t w = 0;
+    for (int i = 0; i < hist.i_cnt; ++i) w |= g.state_first[(size_t)hist.i_st[i] * 8 + lane];
+    out8[lane] = w;
+  }
+}
+
+// report the plan's missing entries to the host (one thread per request and step)
+__device__ __forceinline__ void report_missing(const GrammarDev& g, const StepPlan& plan) {
+  JitRing* ring = g.miss_ring;
+  if (!ring) return;
+  const int n = min(plan.n_missing, kPlanMissingMax);
+  for (int z = 0; z < n; ++z) {
+    const uint32_t slot = atomicAdd(&ring->count, 1u);
+    ring->miss[slot % kJitRingCap] = make_int2(g.jit_slot, plan.missing_state[z]);
+  }
+}
+
 constexpr int kMergeMaxChunkWords = 2048;
 
 __global__ void __launch_bounds__(256)
@@ -733,10 +837,35 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
   const StepPlan& plan = *m.plan;
   const int n = m.n_sets - 1;
   const bool live = !m.terminated && !plan.overflow;
-  const int n_ent = live ? plan.n_check : 0;
+  const bool fallback = live && plan.n_missing > 0;   // an entry is not built yet: walk the whole vocabulary instead
+  const int n_ent = (live && !fallback) ? plan.n_check : 0;
   const int total = n_ent ? plan.check_cum[n_ent] : 0;
   const int stride = gridDim.x * blockDim.x;
   if (threadIdx.x == 0) sh_fail = 0;
+  if (fallback) {
+    __shared__ uint32_t set_first[8];
+    const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
+    const uint32_t* class_bits = stage_class_bits(g, sh_class);
+    current_first_bytes(g, hist, set_first, threadIdx.x);
+    if (blockIdx.x == 0 && threadIdx.x == 0) report_missing(g, plan);
+    __syncthreads();
+    uint32_t* row = (uint32_t*)bitmask + (long long)b * row_stride;
+    for (int r = blockIdx.x * blockDim.x + threadIdx.x; r < v.vocab_size; r += stride) {
+      if (v.never[r]) continue;
+      const uint32_t off = v.offset[r];
+      const int len = (int)(v.offset[r + 1] - off);
+      const uint32_t byte = v.bytes[off];
+      if (!((set_first[byte >> 5] >> (byte & 31)) & 1u)) continue;
+      if (len > kFastMaxBytes) { sh_fail = 1; continue; }
+      uint32_t st[kFastCap];
+      int32_t org[kFastCap];
+      int16_t lsb[kFastMaxBytes + 2];
+      int flags = 0;
+      const bool pass = token_walk<int16_t>(g, class_bits, hist, v.bytes + off, len, false, st, org, kFastCap, lsb, &flags, nullptr) == len;
+      if (flags & kWalkOverflow) sh_fail = 1;
+      else if (pass) { const int id = v.rank_to_id[r]; atomicOr(&row[id >> 5], 1u << (id & 31)); }
+    }
+  } else
   if (blockIdx.x * (int)blockDim.x < total) {         // blocks without candidates only take part in the count below
     const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
     const uint32_t* class_bits = stage_class_bits(g, sh_class);
@@ -892,8 +1021,10 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] = 0;
   const int st0 = m.terminated ? -8 : (plan.overflow ? -6 : 0);
   if (threadIdx.x == 0) { sh_fail = 0; long_n = 0; }
-  const int n_ent = st0 == 0 ? plan.n_check : 0;
+  const bool fallback = st0 == 0 && plan.n_missing > 0;   // an entry is not built yet: walk the whole vocabulary instead
+  const int n_ent = (st0 == 0 && !fallback) ? plan.n_check : 0;
   const int total = n_ent ? plan.check_cum[n_ent] : 0;
+  __shared__ uint32_t set_first[8];
   __syncthreads();
   // 1. merge
   if (st0 == 0 && nw > 0) {
@@ -922,8 +1053,8 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
     if (threadIdx.x == 0 && v.eos_id >= 0 && (uint32_t)v.eos_id >= id_lo && (uint32_t)v.eos_id < id_hi && plan.eos_ok)
       row[(v.eos_id >> 5) - w0] |= 1u << (v.eos_id & 31);
   }
-  // 2. check (the plan and its arrays are the same for the whole cluster: `total` is uniform)
-  if (total > 0) {
+  // 2. check (the plan and its arrays are the same for the whole cluster: `total` and `fallback` are uniform)
+  if (total > 0 || fallback) {
     const int n = m.n_sets - 1;
     const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
     const uint32_t* class_bits = stage_class_bits(g, sh_class);
@@ -938,6 +1069,10 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
       (&cont_org[0][0])[i] = (&plan.cont_org[0][0])[i];
     }
     for (int i = threadIdx.x; i < n_ent * 8; i += blockDim.x) (&cont_first[0][0])[i] = (&plan.cont_first[0][0])[i];
+    if (fallback) {
+      current_first_bytes(g, hist, set_first, threadIdx.x);
+      if (rank == 0 && threadIdx.x == 0) report_missing(g, plan);
+    }
     cluster.sync();            // every slice is merged (and this block's staging is visible)
     const int stride = n_blocks * blockDim.x;
     auto walk_one = [&](int trank, uint32_t off, int e, int at) {
@@ -956,6 +1091,25 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
       if (overflow) atomicOr(cluster.map_shared_rank(&sh_fail, 0), 1);
       return pass && !overflow;
     };
+    if (fallback) {
+      // the plain definition: every token against the full Earley state, in trie order
+      for (int r = rank * blockDim.x + threadIdx.x; r < v.vocab_size; r += stride) {
+        if (v.never[r]) continue;
+        const uint32_t off = v.offset[r];
+        const uint32_t byte = v.bytes[off];
+        if (!((set_first[byte >> 5] >> (byte & 31)) & 1u)) continue;
+        if ((int)(v.offset[r + 1] - off) > kFastMaxBytes) {
+          const int slot = atomicAdd(&long_n, 1);
+          if (slot < kLongQueue) long_q[slot] = r; else atomicOr(cluster.map_shared_rank(&sh_fail, 0), 1);
+          continue;
+        }
+        if (walk_one(r, off, 0, 0)) {
+          const int id = v.rank_to_id[r];
+          const int word = id >> 5, owner = word / chunk;
+          atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
+        }
+      }
+    }
     for (int j = rank * blockDim.x + threadIdx.x; j < total; j += stride) {
       // per candidate: its exit mask and the byte at its first exit, both streamed in list order;
       // the token's rank and bytes are only touched by the few that survive the bit test
@@ -1011,11 +1165,11 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
     cluster.sync();            // every remote OR has landed
   } else __syncthreads();
   // 3. write the slice
-  const int failed = total > 0 ? *cluster.map_shared_rank(&sh_fail, 0) : 0;
+  const int failed = (total > 0 || fallback) ? *cluster.map_shared_rank(&sh_fail, 0) : 0;
   const bool clear = st0 != 0 || failed;
   for (int w = threadIdx.x; w < nw; w += blockDim.x) bitmask[(long long)b * row_stride + w0 + w] = clear ? 0 : (int32_t)row[w];
   if (rank == 0 && threadIdx.x == 0 && status_user) status_user[b] = st0 != 0 ? st0 : (failed ? -6 : 0);
-  if (total > 0) cluster.sync();      // block 0's shared memory must outlive the reads above
+  if (total > 0 || fallback) cluster.sync();      // block 0's shared memory must outlive the reads above
 }
 
 // ------------------------------------------------------------------------------------------

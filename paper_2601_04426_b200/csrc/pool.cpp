@@ -84,6 +84,25 @@ void DeviceArena::free(void* p) {
 
 CachePool::~CachePool() {
   for (auto& s : scratch_) cudaFree(s.first);
+  cudaFree(jit_.d_used);
+  if (jit_host && jit_host_free) jit_host_free(jit_host);
+}
+
+const CachePool::JitArena* CachePool::jit_arena(long long min_words, bool renew) {
+  if (jit_.base && !renew && jit_.cap_words >= min_words) return &jit_;
+  // the old chunk stays in the pool for the entries already in it; new builds go to the new one
+  long long words = std::max<long long>(min_words, jit_.base ? std::min<long long>(2 * jit_.cap_words, (64LL << 20)) : (8LL << 20));
+  JitArena a;
+  a.base = (uint32_t*)allocate_device((size_t)words * 4, &a.chunk);
+  if (!a.base) return nullptr;
+  if (cudaMalloc(&a.d_used, sizeof(unsigned long long)) != cudaSuccess || cudaMemset(a.d_used, 0, sizeof(unsigned long long)) != cudaSuccess) {
+    cudaFree(a.d_used);
+    return nullptr;                      // the chunk stays registered and idle: the limit's eviction returns it
+  }
+  a.cap_words = words;
+  cudaFree(jit_.d_used);
+  jit_ = a;
+  return &jit_;
 }
 
 void* CachePool::scratch(int slot, size_t bytes) {
@@ -138,8 +157,9 @@ void CachePool::enforce_limit() {
       auto& bucket = by_hash_[pr.hash];
       bucket.erase(std::remove(bucket.begin(), bucket.end(), r), bucket.end());
       pr.built = false;
-      pr.serial.clear(); pr.entries.clear(); pr.counts.clear(); pr.chunks.clear();
+      pr.serial.clear(); pr.entries.clear(); pr.counts.clear(); pr.chunks.clear(); pr.have.clear();
     }
+    if (victim == jit_.chunk) { cudaFree(jit_.d_used); jit_ = JitArena(); }
     cudaDeviceSynchronize();              // nothing may still be reading the chunk
     arena_.free(ch.ptr);
     bytes_ -= (long long)ch.bytes;

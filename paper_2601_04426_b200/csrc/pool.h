@@ -18,8 +18,10 @@ namespace xg {
 struct PoolRule {
   std::vector<uint64_t> serial;      // canonical serialisation (the exact identity of the rule)
   uint64_t hash = 0;
-  bool built = false;
+  bool built = false;                // at least one entry of this rule is in the pool
   std::vector<int> chunks;           // device chunks that hold this rule's entries
+  std::vector<char> have;            // by canonical state index: the entry is in the pool (a just-in-time
+                                     // grammar adds the entries of a rule one visited state at a time)
   std::vector<EntryDev> entries;     // by canonical state index
   std::vector<int2> counts;          // (accepted, uncertain) by canonical state index
 };
@@ -83,6 +85,17 @@ class CachePool {
   // reusable build scratch (grow-only, one buffer per slot; call with `mu` held)
   void* scratch(int slot, size_t bytes);
 
+  // Arena of the just-in-time builds (Section 3.5).  A build that runs inside the decode loop
+  // cannot stop to learn its size on the host, so it takes its space on the device: a counter of
+  // words used, bumped by the build itself.  One chunk at a time; when a build does not fit, the
+  // host opens a larger one and the build is repeated.
+  struct JitArena { uint32_t* base = nullptr; long long cap_words = 0; unsigned long long* d_used = nullptr; int chunk = -1; };
+  // the current arena, or a fresh one of at least `min_words` when there is none or `renew` is set (call with `mu` held)
+  const JitArena* jit_arena(long long min_words, bool renew);
+  // host-side state of the just-in-time service (owned here, defined by the API layer)
+  void* jit_host = nullptr;
+  void (*jit_host_free)(void*) = nullptr;
+
  private:
   const void* owner_;
   std::vector<PoolRule> rules_;
@@ -93,6 +106,7 @@ class CachePool {
   long long limit_ = 0, bytes_ = 0, evicted_chunks_ = 0, evicted_bytes_ = 0;
   uint64_t clock_ = 0;
   std::vector<std::pair<void*, size_t>> scratch_;
+  JitArena jit_;
   int find_or_add(uint64_t hash, std::vector<uint64_t>&& serial);
 };
 

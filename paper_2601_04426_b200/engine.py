@@ -17,7 +17,8 @@ from . import inputs
 class Session:
     """One tokenizer, its compiled grammars and one matcher per request of a workload."""
 
-    def __init__(self, workload: inputs.Workload, share_pool: bool = True, device: str = "cuda:0", state_compression: bool = True):
+    def __init__(self, workload: inputs.Workload, share_pool: bool = True, device: str = "cuda:0", state_compression: bool = True,
+                 jit: bool = False, jit_precompute: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         self.device = torch.device(device)
@@ -26,7 +27,8 @@ class Session:
         v = workload.vocab
         self.tokenizer = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
         self.pool = B.CachePool(self.tokenizer) if share_pool else None
-        self.grammars: List[B.Grammar] = [B.Grammar(self.tokenizer, g.kind, g.text, pool=self.pool, state_compression=state_compression)
+        self.grammars: List[B.Grammar] = [B.Grammar(self.tokenizer, g.kind, g.text, pool=self.pool, state_compression=state_compression,
+                                                    jit=jit, jit_precompute=jit_precompute)
                                           for g in workload.grammars]
         self.matchers = [B.Matcher(self.grammars[gi]) for gi in workload.request_grammar]
         self.batch = B.Batch(self.matchers)
@@ -53,6 +55,10 @@ class Session:
         dtype = {torch.float32: "f32", torch.bfloat16: "bf16", torch.int16: "bf16", torch.uint16: "bf16"}[logits.dtype]
         B.apply_token_bitmask(logits.data_ptr(), dtype, logits.shape[0], self.V, logits.stride(0), self.bitmask.data_ptr(), self.W,
                               rows.data_ptr() if rows is not None else 0, int(rows.numel()) if rows is not None else 0, self.stream())
+
+    def jit_service(self, wait: bool = False) -> dict:
+        """Between decode steps: pick up the cache entries the last fills found missing (just-in-time grammars)."""
+        return B.jit_service(self.grammars, self.stream(), wait)
 
     def mask_numpy(self) -> np.ndarray:
         return self.bitmask.cpu().numpy().view(np.uint32)
