@@ -176,12 +176,18 @@ def tag_dispatch_to_ebnf(spec_text: str, root: str = "root") -> str:
     """{"tags": [{"tag": t, "end": e, "tools": [{"name": n, "schema": s}, ...]}, ...], "stop_strs": [...]}
 
     Tag t dispatches to  ( call_1 | ... | call_n ) e  with  call_k = {"name": "n_k", "arguments": <s_k>},
-    or, when the tag entry has "bare": true, call_k = <s_k> alone.
+    or, when the tag entry has "bare": true, call_k = <s_k> alone.  A tag entry with "text": true has no
+    tools: its body is free text that ends with the entry's "end" string.
     """
     spec = json.loads(spec_text) if isinstance(spec_text, str) else spec_text
     rules: List[str] = []
     pairs = []
     for ti, tag in enumerate(spec["tags"]):
+        if tag.get("text"):
+            # a channel whose body is free text up to its end marker (Section 3.2's stop strings)
+            rules.append("tag_%d ::= TagDispatch(stop_strs=(%s))" % (ti, ebnf_quote(tag["end"])))
+            pairs.append("(%s, tag_%d)" % (ebnf_quote(tag["tag"]), ti))
+            continue
         calls = []
         for ki, tool in enumerate(tag["tools"]):
             prefix = "t%d_%d_" % (ti, ki)

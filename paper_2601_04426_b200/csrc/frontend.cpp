@@ -321,7 +321,7 @@ class GrammarParser {
       if (peek().type == Token::kComma) ++p_;
     }
     ++p_;
-    if (e->tag.tags.empty()) err("TagDispatch needs at least one tag");
+    if (e->tag.tags.empty() && e->tag.stops.empty()) err("TagDispatch needs at least one tag or stop string");
     return e;
   }
 };
@@ -1347,6 +1347,15 @@ std::string tag_dispatch_to_ebnf(const std::string& spec_json) {
     const Json* tools = tag.get("tools");
     const Json* end = tag.get("end");
     if (!text || text->type != Json::kString || text->text.empty()) fail(XG_ERR_PARSE, "TagDispatch spec: missing tag string");
+    const Json* free_text = tag.get("text");
+    if (free_text && free_text->type == Json::kBool && free_text->boolean) {
+      // a channel whose body is free text up to its end marker: a TagDispatch without tags that stops at the marker
+      if (!end || end->type != Json::kString || end->text.empty()) fail(XG_ERR_PARSE, "TagDispatch spec: a text channel needs a non-empty \"end\"");
+      std::string rule = "dispatch_" + std::to_string(ti);
+      rules += rule + " ::= TagDispatch(stop_strs=(" + literal(end->text) + "))\n";
+      pairs += (ti ? ", " : "") + std::string("(") + literal(text->text) + ", " + rule + ")";
+      continue;
+    }
     if (!tools || tools->type != Json::kArray || tools->items.empty()) fail(XG_ERR_PARSE, "TagDispatch spec: \"tools\" must be a non-empty array");
     std::string calls;
     for (size_t k = 0; k < tools->items.size(); ++k) {

@@ -488,6 +488,32 @@ def sample_tool_text(rng: Rng, tools: List[dict], tag: str, end: str, n_calls: i
     return "".join(out)
 
 
+# a channelised response protocol: every message names its channel; text channels run to an end marker, tool
+# channels carry the arguments of one tool, a final marker ends the response (Sections 1 and 3.2)
+CH_START, CH_CHANNEL, CH_MESSAGE, CH_END, CH_CALL, CH_RETURN = "<|start|>assistant", "<|channel|>", "<|message|>", "<|end|>", "<|call|>", "<|return|>"
+
+
+def channel_spec(tools: List[dict]) -> dict:
+    tags = [{"tag": CH_CHANNEL + name + CH_MESSAGE, "text": True, "end": CH_END} for name in ("analysis", "final")]
+    tags += [{"tag": "%scommentary to=functions.%s%s" % (CH_CHANNEL, t["name"], CH_MESSAGE), "end": CH_CALL, "bare": True, "tools": [t]} for t in tools]
+    return {"tags": tags, "stop_strs": [CH_RETURN]}
+
+
+def sample_channel_text(rng: Rng, tools: List[dict], n_messages: int) -> str:
+    def free(k: int) -> str:
+        return " ".join(_word(rng, 2, 8) for _ in range(k)) + rng.choice(["", ".", "\n"])
+    out: List[str] = []
+    for _ in range(n_messages):
+        out.append(CH_START)
+        if rng.below(2):
+            out.append(CH_CHANNEL + "analysis" + CH_MESSAGE + free(rng.randint(3, 14)) + CH_END)
+        else:
+            tool = rng.choice(tools)
+            out.append("%scommentary to=functions.%s%s%s%s" % (CH_CHANNEL, tool["name"], CH_MESSAGE, sample_document(tool["schema"], rng), CH_CALL))
+    out.append(CH_START + CH_CHANNEL + "final" + CH_MESSAGE + free(rng.randint(4, 16)) + CH_END + CH_RETURN)
+    return "".join(out)
+
+
 def make_function_tags(rng: Rng, n_tags: int, tag_len: int = 20) -> List[dict]:
     """`n_tags` tools whose tags share the prefix `<function=` and are `tag_len` bytes long in total
     (the shape of the paper's tag-count experiment, Section 4.1), each with a small argument schema."""
@@ -566,6 +592,9 @@ _SHAPES = {
     "T20": (128256,  16,  4.0, 0.3,    0.0,  16,   128,  "bf16"),
     "T50": (128256,  16,  4.0, 0.3,    0.0,  16,   128,  "bf16"),
     "T100": (128256, 16,  4.0, 0.3,    0.0,  16,   128,  "bf16"),
+    # channelised response protocol with 16 / 64 tools (text channels with stop strings, one tool channel per tool)
+    "H16": (128256,  16,  4.0, 0.3,    0.0,  32,   256,  "bf16"),
+    "H64": (128256,  16,  4.0, 0.3,    0.0,  32,   256,  "bf16"),
     # long bounded repetitions (Section 3.6: minLength / maxLength / minItems / maxItems in the hundreds to thousands)
     "R256": (128256,  16,  4.0, 0.3,    0.0,  16,   256,  "bf16"),
     "R1024": (128256, 16,  4.0, 0.3,    0.0,  16,   256,  "bf16"),
@@ -578,7 +607,7 @@ _vocab_cache: Dict[Tuple, Vocab] = {}
 def config_seed(name: str) -> int:
     if name[0] == "C":
         return BASE_SEED * 10 + int(name[1])
-    return BASE_SEED * 10 + (1000 if name[0] == "T" else 100000) + int(name[1:])
+    return BASE_SEED * 10 + {"T": 1000, "R": 100000, "H": 200000}[name[0]] + int(name[1:])
 
 
 def config_vocab(name: str, vocab_size: Optional[int] = None) -> Vocab:
@@ -586,7 +615,7 @@ def config_vocab(name: str, vocab_size: Optional[int] = None) -> Vocab:
     if vocab_size is not None:
         V = vocab_size
     # C2 and C4 share one Llama-3-sized vocabulary
-    seed_name = "C2" if (name == "C4" or name[0] in "TR") else name
+    seed_name = "C2" if (name == "C4" or name[0] in "TRH") else name
     key = (seed_name, V)
     if key not in _vocab_cache:
         _vocab_cache[key] = make_vocab(config_seed(seed_name) ^ 0x5EED, V, lmax, mean, lead, utf8)
@@ -684,6 +713,14 @@ def make_workload(name: str, batch: Optional[int] = None, steps: Optional[int] =
         for b in range(B):
             rr = rng.fork(100 + b)
             t, d = _trajectory(tok, vocab.eos_id, S, lambda: sample_function_text(rr, tools, rr.randint(1, 3), 40).encode())
+            request_grammar.append(0); trajs.append(t); docs_all.append(d)
+    elif name[0] == "H":
+        tools = make_tool_set(rng.fork(3), int(name[1:]))
+        grammars.append(GrammarSpec("tag_dispatch", json.dumps(channel_spec(tools))))
+        meta["tools"] = tools
+        for b in range(B):
+            rr = rng.fork(100 + b)
+            t, d = _trajectory(tok, vocab.eos_id, S, lambda: sample_channel_text(rr, tools, rr.randint(1, 4)).encode())
             request_grammar.append(0); trajs.append(t); docs_all.append(d)
     elif name[0] == "R":
         # four orderings of one set of bounded properties, so that within the step budget different

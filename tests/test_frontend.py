@@ -56,6 +56,8 @@ def test_tables_same_language_as_oracle_on_small_grammars(inline):
     _same_language('root ::= TagDispatch(("ab", g), stop_strs=("xb")) "!"\ng ::= "a"', "abx!", 6, inline_max_states=inline)
     _same_language('root ::= TagDispatch(("ab", g))\ng ::= "x" "x"?', "abx", 7, inline_max_states=inline)
     _same_language('root ::= "q"? TagDispatch(("<a>", r0), ("<<b", r1)) \nr0 ::= "0"\nr1 ::= "1" root?', "<>ab01q", 5, inline_max_states=inline)
+    # a text channel: a TagDispatch without tags that runs to its stop string, nested in a dispatching one
+    _same_language('root ::= TagDispatch(("<a", body), stop_strs=("!"))\nbody ::= TagDispatch(stop_strs=("a>", ">>"))', "<a>!", 7, inline_max_states=inline)
 
 
 def test_tables_invariants():
@@ -90,7 +92,7 @@ def _mutate(rng, doc, alphabet):
     return doc[:pos] + b + doc[pos + 1:] if kind == 0 else (doc[:pos] + doc[pos + 1:] if kind == 1 else doc[:pos] + b + doc[pos:])
 
 
-@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4", "C5", "T20"])
+@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4", "C5", "T20", "H16", "R256"])
 def test_workload_grammars_same_language_as_oracle(name):
     w = inputs.make_workload(name, batch=3, steps=40)
     rng = inputs.Rng(17)
@@ -114,7 +116,7 @@ def test_workload_grammars_same_language_as_oracle(name):
                         assert tm.can_terminate() == O.accepts(og, mut), mut
 
 
-@pytest.mark.parametrize("name,vsize,steps", [("C1", 2048, 40), ("C4", 2048, 60), ("C5", 4096, 30), ("T5", 2048, 50)])
+@pytest.mark.parametrize("name,vsize,steps", [("C1", 2048, 40), ("C4", 2048, 60), ("C5", 4096, 30), ("T5", 2048, 50), ("H16", 2048, 70)])
 def test_masks_plain_equals_merged_equals_oracle(name, vsize, steps):
     """The cache classification plus the merge rule reproduces the plain definition, step by step."""
     w = inputs.make_workload(name, batch=1, steps=steps, vocab_size=vsize)

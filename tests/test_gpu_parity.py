@@ -98,6 +98,12 @@ def test_many_tag_dispatch_batch():
     _run_trajectories(w, {0, 20, 45, 89}, check_requests={1})
 
 
+def test_channel_protocol_batch():
+    """Text channels that run to a stop string, tool channels, a final stop string (Sections 1, 3.2)."""
+    w = inputs.make_workload("H16", batch=6, steps=140, vocab_size=16384)
+    _run_trajectories(w, {0, 1, 15, 40, 80, 139}, check_requests={4})
+
+
 def test_hand_worked_masks_on_gpu():
     torch, engine = _engine()
     from golden_util import load_mask_fixture

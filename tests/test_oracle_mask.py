@@ -117,6 +117,42 @@ def test_tagdispatch_with_stop_string_equals_plain_lowering():
         assert O.is_prefix(td, s.encode()) == O.is_prefix(plain, s.encode()), s
 
 
+def test_text_channel_is_free_text_up_to_its_first_stop_string():
+    """A TagDispatch without tags (a text channel): accepts exactly the strings that end with a stop
+    string and hold no earlier occurrence of one; checked with str.find and with the plain lowering."""
+    td = O.Grammar('root ::= TagDispatch(stop_strs=("ab", "bb"))')
+    plain = O.Grammar("""
+        root ::= n0
+        n0 ::= "a" na | "b" nb | "x" n0
+        na ::= "a" na | "b" | "x" n0
+        nb ::= "a" na | "b" | "x" n0
+    """)
+    for s in all_strings("abx", 7):
+        ends = [s.find(p) + 2 for p in ("ab", "bb") if s.find(p) >= 0]
+        member = bool(ends) and min(ends) == len(s)
+        assert O.accepts(td, s.encode()) == member == O.accepts(plain, s.encode()), s
+        assert O.is_prefix(td, s.encode()) == (not ends or min(ends) == len(s)) == O.is_prefix(plain, s.encode()), s
+
+
+def test_channel_protocol_lowering_accepts_generated_text():
+    rng = inputs.Rng(9)
+    tools = inputs.make_tool_set(rng, 4)
+    g = O.Grammar(SE.tag_dispatch_to_ebnf(json.dumps(inputs.channel_spec(tools))))
+    for _ in range(8):
+        text = inputs.sample_channel_text(rng, tools, rng.randint(1, 4)).encode()
+        m = O.Matcher(g)
+        assert m.accept_bytes(text) and m.can_terminate()
+        assert not O.is_prefix(g, text + b"x")                        # the final marker ends the response
+        m2 = O.Matcher(g)
+        assert m2.accept_bytes(text[:-len(inputs.CH_RETURN)]) and not m2.can_terminate()
+        if b"commentary" in text:                                     # inside a tool channel only the arguments grammar applies
+            at = text.index(b"<|message|>", text.index(b"commentary")) + len(b"<|message|>")
+            assert O.is_prefix(g, text[:at] + b"{") and not O.is_prefix(g, text[:at] + b"x")
+        at = text.index(b"analysis<|message|>") + len(b"analysis<|message|>") if b"analysis" in text else None
+        if at:                                                        # a text channel takes anything, tags included, up to its end marker
+            assert O.is_prefix(g, text[:at] + b"<|channel|>final<|message|>{ x")
+
+
 def test_tagdispatch_fires_at_earliest_ending_tag():
     tags = ["<a>", "<bc>", "<<b>"]
     g = O.Grammar('root ::= TagDispatch(("<a>", r0), ("<bc>", r1), ("<<b>", r2))\nr0 ::= "0"\nr1 ::= "1"\nr2 ::= "2"')
