@@ -111,6 +111,9 @@ typedef struct {
                                  are built when a matcher first visits their state (xg_jit_service). */
   int32_t jit_precompute;     /* K of Section 3.5's configurable JIT: entries to build at compile time, the
                                  costliest first (cost = tokens that survive the state's first-byte test). */
+  int64_t jit_arena_bytes;    /* size of the pool's first just-in-time arena (entries built inside the decode loop take
+                                 their space from it on the device); when one fills up the next is twice as large.
+                                 <= 0 = default (32 MiB).  Only the pool's first just-in-time compile sets it. */
 } xg_compile_options_t;
 
 /* ---- grammar compilation (Section 3.5 "compilation stage"; Sections 3.2, 3.3, 3.4) ---------

@@ -41,7 +41,7 @@ class XgError(RuntimeError):
 
 class CompileOptions(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("inline_max_states", C.c_int32), ("max_rule_states", C.c_int32), ("build_cache", C.c_int32),
-                ("no_state_compression", C.c_int32), ("jit", C.c_int32), ("jit_precompute", C.c_int32)]
+                ("no_state_compression", C.c_int32), ("jit", C.c_int32), ("jit_precompute", C.c_int32), ("jit_arena_bytes", C.c_int64)]
 
 
 class JitStats(C.Structure):
@@ -167,11 +167,11 @@ class CachePool:
 class Grammar:
     def __init__(self, tokenizer: Optional[Tokenizer], kind, text: str, pool: Optional[CachePool] = None, root: Optional[str] = None,
                  inline_max_states: int = -1, build_cache: bool = True, stream: int = 0, state_compression: bool = True,
-                 jit: bool = False, jit_precompute: int = 0):
+                 jit: bool = False, jit_precompute: int = 0, jit_arena_bytes: int = 0):
         kind = KIND_BY_NAME.get(kind, kind)
         raw = text.encode("utf-8") if isinstance(text, str) else text
         opt = CompileOptions(C.sizeof(CompileOptions), inline_max_states, 0, 1 if build_cache else 0, 0 if state_compression else 1,
-                             1 if jit else 0, int(jit_precompute))
+                             1 if jit else 0, int(jit_precompute), int(jit_arena_bytes))
         h = C.c_void_p()
         _check(lib().xg_compile_grammar(tokenizer.h if tokenizer else None, pool.h if pool else None, kind, raw, len(raw),
                                         root.encode() if root else None, C.byref(opt), stream, C.byref(h)))

@@ -44,6 +44,29 @@ T* device_copy(const std::vector<T>& v, cudaError_t* err) {
   return p;
 }
 
+// launch with programmatic stream serialisation (see step_kernel_prologue in kernels.cuh)
+template <typename... KArgs, typename... Args>
+cudaError_t launch_step_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, int cluster_x, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attrs[2];
+  int n = 0;
+  attrs[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attrs[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster_x > 1) {
+    attrs[n].id = cudaLaunchAttributeClusterDimension;
+    attrs[n].val.clusterDim.x = cluster_x; attrs[n].val.clusterDim.y = 1; attrs[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attrs;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 double now_ms() {
   return std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now().time_since_epoch()).count();
 }
@@ -491,11 +514,11 @@ static void jit_release(xg_grammar* g) {
 }
 
 // per-grammar device arrays, the pool's ring and scratch; registers the grammar in the pool (call with the pool's lock held)
-static xg_status_t jit_allocate(xg_grammar* g) {
+static xg_status_t jit_allocate(xg_grammar* g, long long first_arena_words) {
   JitState& j = g->jit;
   CachePool& pool = *g->pool;
   JitScratch sc;
-  if (!jit_scratch(pool, g->tok->n_words, &sc) || !pool.jit_arena(0, false)) return set_error(XG_ERR_OOM, "just-in-time scratch allocation failed");
+  if (!jit_scratch(pool, g->tok->n_words, &sc) || !pool.jit_arena(0, false, first_arena_words)) return set_error(XG_ERR_OOM, "just-in-time scratch allocation failed");
   const int one = 1;
   XG_CUDA(cudaMemcpy(sc.one, &one, sizeof(int), cudaMemcpyHostToDevice));
   if (!pool.jit_host) {
@@ -777,6 +800,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   FrontendOptions fo;
   bool build_cache = tok != nullptr, compress = true, jit = false;
   int jit_precompute = 0;
+  long long jit_arena_words = 0;
   if (opt) {
     if (opt->struct_size < 8) return set_error(XG_ERR_INVALID_ARG, "bad options struct_size");
     if (opt->inline_max_states >= 0) fo.inline_max_states = opt->inline_max_states;
@@ -784,6 +808,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     if (opt->struct_size >= 16 && opt->build_cache == 0) build_cache = false;
     if (opt->struct_size >= 20 && opt->no_state_compression != 0) compress = false;
     if (opt->struct_size >= 28 && opt->jit != 0) { jit = true; jit_precompute = std::max(0, opt->jit_precompute); }
+    if (opt->struct_size >= 40 && opt->jit_arena_bytes > 0) jit_arena_words = std::max<long long>(1024, opt->jit_arena_bytes / 4);
   }
   if (pool && pool->impl->owner() != (const void*)tok) return set_error(XG_ERR_INVALID_ARG, "the pool belongs to another tokenizer");
   std::unique_ptr<xg_grammar> g(new xg_grammar());
@@ -826,7 +851,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   };
   xg_status_t st = XG_OK;
   if (jit) {
-    st = jit_allocate(g.get());
+    st = jit_allocate(g.get(), jit_arena_words);
     if (st != XG_OK) return fail(st);
   }
   st = upload_grammar(g.get());
@@ -1201,17 +1226,8 @@ xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t ba
     const int per_request = sms * 1024 / batch;
     int blocks = kMaxClusterBlocks, threads = 256;
     if (per_request < 2048) threads = 128;     // measured: fewer blocks or narrower blocks than this are slower even at batch 256
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(blocks, batch);
-    cfg.blockDim = dim3(threads);
-    cfg.dynamicSmemBytes = 2 * sizeof(uint32_t) * (size_t)((W + blocks - 1) / blocks);
-    cfg.stream = (cudaStream_t)stream;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = blocks; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
-    XG_CUDA(cudaLaunchKernelEx(&cfg, fill_cluster_kernel, (MatcherDev* const*)slot->dev_matchers, tok->dev, bitmask_dev,
+    XG_CUDA(launch_step_kernel(fill_cluster_kernel, dim3(blocks, batch), dim3(threads), 2 * sizeof(uint32_t) * (size_t)((W + blocks - 1) / blocks),
+                               (cudaStream_t)stream, blocks, (MatcherDev* const*)slot->dev_matchers, tok->dev, bitmask_dev,
                                (long long)row_stride_words, status_dev));
     return XG_OK;
   }
@@ -1291,8 +1307,8 @@ xg_status_t xg_accept_token(xg_matcher_t* const* matchers, int32_t batch, const 
   xg_status_t st = batch_slot(matchers, batch, &tok, &slot);
   if (st != XG_OK) return st;
   if (!token_ids_dev) return set_error(XG_ERR_INVALID_ARG, "token_ids_dev is NULL");
-  accept_kernel<<<(batch + 3) / 4, 128, 0, (cudaStream_t)stream>>>(slot->dev_matchers, batch, tok->dev, token_ids_dev, status_dev);
-  XG_CUDA(cudaGetLastError());
+  XG_CUDA(launch_step_kernel(accept_kernel, dim3((batch + 3) / 4), dim3(128), 0, (cudaStream_t)stream, 1, (MatcherDev* const*)slot->dev_matchers,
+                             (int)batch, tok->dev, token_ids_dev, status_dev));
   return XG_OK;
 }
 
@@ -1319,12 +1335,11 @@ xg_status_t xg_apply_token_bitmask(void* logits_dev, xg_dtype_t dtype, int32_t b
   if (rows > 65535) return set_error(XG_ERR_INVALID_ARG, "more than 65535 rows");
   dim3 grid(bx, rows);
   if (dtype == XG_BF16)
-    apply_kernel<8><<<grid, 256, 0, (cudaStream_t)stream>>>(logits_dev, vocab_size, (long long)logits_row_stride_elems, (const uint32_t*)bitmask_dev,
-                                                            (long long)mask_row_stride_words, row_indices_dev);
+    XG_CUDA(launch_step_kernel(apply_kernel<8>, grid, dim3(256), 0, (cudaStream_t)stream, 1, logits_dev, (int)vocab_size, (long long)logits_row_stride_elems,
+                               (const uint32_t*)bitmask_dev, (long long)mask_row_stride_words, row_indices_dev));
   else
-    apply_kernel<4><<<grid, 256, 0, (cudaStream_t)stream>>>(logits_dev, vocab_size, (long long)logits_row_stride_elems, (const uint32_t*)bitmask_dev,
-                                                            (long long)mask_row_stride_words, row_indices_dev);
-  XG_CUDA(cudaGetLastError());
+    XG_CUDA(launch_step_kernel(apply_kernel<4>, grid, dim3(256), 0, (cudaStream_t)stream, 1, logits_dev, (int)vocab_size, (long long)logits_row_stride_elems,
+                               (const uint32_t*)bitmask_dev, (long long)mask_row_stride_words, row_indices_dev));
   return XG_OK;
 }
 

@@ -13,6 +13,17 @@ namespace xg {
 
 enum : int { kWalkUncertain = 1, kWalkOverflow = 2 };
 
+// Programmatic dependent launch: the three kernels of a decode step are short, so the gap between
+// one kernel's end and the next one's start is a large share of the step.  Each of them lets the
+// next kernel of the stream be scheduled at once (its blocks become resident as room appears) and
+// itself waits, before it touches any memory, until the previous kernel has finished and its
+// writes are visible.  The order of all memory accesses is that of plain stream order.  Both are
+// no-ops for a launch without the programmatic-serialisation attribute.
+__device__ __forceinline__ void step_kernel_prologue() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 constexpr int kFastCap = 48;     // items a token walk may create before it falls back
 constexpr int kFastMaxBytes = 32;
 constexpr int kSlowCap = 2048;
@@ -654,6 +665,7 @@ __global__ void matcher_reset_kernel(MatcherDev* m) {      // one warp
 __global__ void __launch_bounds__(128)
 accept_kernel(MatcherDev* const* __restrict__ matchers, int batch, VocabDev v,
               const int32_t* __restrict__ token_ids, int32_t* __restrict__ status) {
+  step_kernel_prologue();
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (b >= batch) return;
@@ -1007,6 +1019,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   __shared__ int16_t long_lsb[kSlowMaxBytes + 2];
   __shared__ int sh_fail;          // block 0's copy collects the whole cluster's failures
 
+  step_kernel_prologue();
   const int b = blockIdx.y;
   const int rank = (int)cluster.block_rank();
   const MatcherDev& m = *matchers[b];
@@ -1203,6 +1216,7 @@ template <int ELEMS>   // elements per 16-byte vector: 8 (bf16) or 4 (fp32)
 __global__ void __launch_bounds__(256)
 apply_kernel(void* __restrict__ logits, int vocab_size, long long row_stride_elems, const uint32_t* __restrict__ bitmask,
              long long mask_stride, const int32_t* __restrict__ row_indices) {
+  step_kernel_prologue();
   const int r = row_indices ? row_indices[blockIdx.y] : blockIdx.y;
   const uint32_t* mrow = bitmask + (long long)r * mask_stride;
   const int n_vec = vocab_size / ELEMS;

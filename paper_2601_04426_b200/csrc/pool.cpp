@@ -88,10 +88,10 @@ CachePool::~CachePool() {
   if (jit_host && jit_host_free) jit_host_free(jit_host);
 }
 
-const CachePool::JitArena* CachePool::jit_arena(long long min_words, bool renew) {
+const CachePool::JitArena* CachePool::jit_arena(long long min_words, bool renew, long long first_words) {
   if (jit_.base && !renew && jit_.cap_words >= min_words) return &jit_;
   // the old chunk stays in the pool for the entries already in it; new builds go to the new one
-  long long words = std::max<long long>(min_words, jit_.base ? std::min<long long>(2 * jit_.cap_words, (64LL << 20)) : (8LL << 20));
+  long long words = std::max<long long>(min_words, jit_.base ? std::min<long long>(2 * jit_.cap_words, (64LL << 20)) : (first_words > 0 ? first_words : (8LL << 20)));
   JitArena a;
   a.base = (uint32_t*)allocate_device((size_t)words * 4, &a.chunk);
   if (!a.base) return nullptr;

@@ -91,7 +91,8 @@ class CachePool {
   // host opens a larger one and the build is repeated.
   struct JitArena { uint32_t* base = nullptr; long long cap_words = 0; unsigned long long* d_used = nullptr; int chunk = -1; };
   // the current arena, or a fresh one of at least `min_words` when there is none or `renew` is set (call with `mu` held)
-  const JitArena* jit_arena(long long min_words, bool renew);
+  // `first_words` > 0 sizes the very first arena (default 8 Mi words)
+  const JitArena* jit_arena(long long min_words, bool renew, long long first_words = 0);
   // host-side state of the just-in-time service (owned here, defined by the API layer)
   void* jit_host = nullptr;
   void (*jit_host_free)(void*) = nullptr;

@@ -18,7 +18,7 @@ class Session:
     """One tokenizer, its compiled grammars and one matcher per request of a workload."""
 
     def __init__(self, workload: inputs.Workload, share_pool: bool = True, device: str = "cuda:0", state_compression: bool = True,
-                 jit: bool = False, jit_precompute: int = 0):
+                 jit: bool = False, jit_precompute: int = 0, jit_arena_bytes: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         self.device = torch.device(device)
@@ -28,7 +28,7 @@ class Session:
         self.tokenizer = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
         self.pool = B.CachePool(self.tokenizer) if share_pool else None
         self.grammars: List[B.Grammar] = [B.Grammar(self.tokenizer, g.kind, g.text, pool=self.pool, state_compression=state_compression,
-                                                    jit=jit, jit_precompute=jit_precompute)
+                                                    jit=jit, jit_precompute=jit_precompute, jit_arena_bytes=jit_arena_bytes)
                                           for g in workload.grammars]
         self.matchers = [B.Matcher(self.grammars[gi]) for gi in workload.request_grammar]
         self.batch = B.Batch(self.matchers)

@@ -178,3 +178,90 @@ def test_allocation_free_fill_and_many_grammars():
     s, final, _, _ = _drive(w, 6, "each", static_fill=True)
     assert final["n_built"] + final["n_pool_hits"] > 0
     s.close()
+
+
+def test_arena_that_is_too_small_is_replaced_by_a_larger_one():
+    """Builds that find no room in the pool's just-in-time arena are repeated in a larger arena;
+    the masks are exact meanwhile and afterwards."""
+    w = inputs.make_workload("C1", steps=50)
+    s, final, _, _ = _drive(w, 2, "wait", jit_arena_bytes=4096)
+    assert final["n_built"] > 0 and final["n_in_flight"] == 0
+    pool = s.pool.stats()
+    assert pool["chunks"] >= 2                   # the first arena (4 KiB) and at least one successor
+    s.close()
+
+
+def test_long_tokens_take_the_exact_build_path():
+    """A vocabulary with tokens beyond the fast path's 32 bytes: the just-in-time build notices on the
+    device that it cannot finish, and the service call falls back to the exact build."""
+    import torch
+    base = [bytes([b]) for b in range(256)]
+    long_tokens = [b"a" * 33, b"ab" * 40, b"x" * 255, b"a" * 40 + b"}", b"a" * 100 + b"}}", b"b" * 64 + b'}, "k": {', b'{"' + b"q" * 60]
+    toks = base + long_tokens + [b""]
+    toks += [b"\xfe\xff%d" % i for i in range(-len(toks) % 32)]
+    eos = toks.index(b"")
+    ebnf = 'root ::= obj\nobj ::= "{" [a-z]* "}" | "{" "\\"" [a-z]* "\\": " obj "}"\n'
+    tok = B.Tokenizer(toks, eos)
+    g = B.Grammar(tok, "ebnf", ebnf, inline_max_states=0, jit=True)
+    full = B.Grammar(tok, "ebnf", ebnf, inline_max_states=0)
+    ov = O.Vocab(toks, eos)
+    om = O.Matcher(O.Grammar(ebnf))
+    m = B.Matcher(g)
+    batch = B.Batch([m])
+    mask = torch.zeros((1, tok.words), dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ids = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for piece in [b"{", b'"', b"q", b"q", b'"', b":", b" ", b"{", b"a" * 33, b"ab" * 40, b"a" * 40 + b"}", b"}"]:
+        for _ in range(2):                       # once from the whole-vocabulary walk, once more after the service call
+            batch.fill_next_token_bitmask(mask.data_ptr(), tok.words, st.data_ptr())
+            assert int(st.cpu()[0]) == 0
+            assert np.array_equal(mask.cpu().numpy().view(np.uint32)[0], om.mask(ov)), piece
+            B.jit_service([g], 0, True)
+            m2 = B.Matcher(g)                    # a fresh matcher fed the same bytes sees the published entries
+            m2.close()
+        tid = toks.index(piece)
+        ids[0] = tid
+        batch.accept_token(ids.data_ptr(), st.data_ptr())
+        assert int(st.cpu()[0]) == 0, piece
+        assert om.accept_token(ov, tid) == 1
+    stats = B.jit_service([g], 0, True)
+    assert stats["n_built"] > 0
+    t = full.tables()
+    compared = 0
+    for s_ in [x for x in range(t["n_states"]) if t["cedge_begin"][x + 1] > t["cedge_begin"][x]]:
+        try:
+            e = g.cache_entry(s_)
+        except B.XgError:
+            continue
+        ref = full.cache_entry(s_)
+        assert e["kind"] == ref["kind"] and np.array_equal(e["list"], ref["list"]) and np.array_equal(e["uncertain"], ref["uncertain"]), s_
+        compared += 1
+    assert compared > 0
+    m.close(); g.close(); full.close(); tok.close()
+
+
+def test_teardown_with_builds_in_flight_and_pool_accounting():
+    import torch
+    from paper_2601_04426_b200 import engine
+    w = inputs.make_workload("C3", batch=4, steps=12, vocab_size=8192)
+    s = engine.Session(w, jit=True)
+    for step in range(6):
+        s.fill()
+        s.accept([w.trajectories[b][step] for b in range(s.n)])
+        s.jit_service(wait=False)                # leaves a snapshot or builds on their way
+    pool, tokenizer = s.pool, s.tokenizer
+    before = pool.stats()
+    assert before["bytes"] > 0
+    pool.set_limit(1)                            # everything held is in use by the live grammars
+    assert pool.stats()["evicted_chunks"] == 0
+    for m in s.matchers:                         # matchers and grammars go while work may be pending
+        m.close()
+    for g in s.grammars:
+        g.close()
+    after = pool.stats()
+    assert after["bytes"] == 0 and after["chunks"] == 0
+    # the pool is still usable: a new just-in-time grammar starts from nothing
+    g = B.Grammar(tokenizer, w.grammars[0].kind, w.grammars[0].text, pool=pool, jit=True, jit_precompute=3)
+    assert g.stats()["n_entries_built"] == 3
+    g.close()
+    pool.close(); tokenizer.close()
