@@ -354,6 +354,20 @@ def main():
                           "frac": (4.0 * n * W + elt * alone_zero_bits) / (t_apply_alone * 1e-6) / 1e9 / peak,
                           "conventional_gbs": apply_conv_bytes / (t_apply_alone * 1e-6) / 1e9}}
 
+    # The other two step kernels are bound by latency, not by a memory or arithmetic pipe.  What can be said against a
+    # peak is their issue rate: warp instructions per launch (ncu, profiles/step_kernels_c3.txt; C3 only, void once
+    # the kernels change) over the launch time, against 148 SMs x 4 schedulers x the SM clock.
+    props = torch.cuda.get_device_properties(local_rank)
+    issue_peak = props.multi_processor_count * 4 * (clocks["sm_max_mhz"] or 1965.0) * 1e6
+    warp_insts = {"fill": 1665453.0, "accept": 104371.0} if (args.workload == "C3" and n == 128) else {}
+    latency_bound = {}
+    for name, t_us in (("fill", t_fill), ("accept", t_accept)):
+        wi = warp_insts.get(name)
+        latency_bound[name] = {"kernel": "fill_cluster_kernel" if name == "fill" else "accept_kernel", "bound": "alu",
+                               "achieved": (wi / (t_us * 1e-6)) if wi else None, "peak": issue_peak, "unit": "warp instructions/s",
+                               "frac": (wi / (t_us * 1e-6) / issue_peak) if wi else None, "warp_instructions_per_launch": wi,
+                               "us_per_launch": t_us, "note": "latency-bound: chains of dependent loads, issue slots 4-11 % busy under ncu"}
+
     # ---- end to end through the C ABI with host buffers ---------------------------------------
     e2e_steps = max(3, min(args.steps, 12))
     host_in = torch.empty((n, s.V), dtype=tdtype).pin_memory()
@@ -401,6 +415,7 @@ def main():
                         "uncertain_total": sum(x["total_uncertain"] for x in stats), "uncertain_after_lookahead": sum(x["total_checked"] for x in stats),
                         "cache_bytes_unique_upper": sum(x["cache_bytes"] for x in stats)},
         "roofline": roofline,
+        "roofline_latency_bound_kernels": latency_bound,
         "e2e": {"value": e2e_us, "unit": "us/step", "h2d_bytes_per_step": bytes_one + 4 * n, "d2h_bytes_per_step": bytes_one, "steps": e2e_steps},
         "gpu_launches": timed_launches,
     }

@@ -1,5 +1,6 @@
 // C ABI of the token-mask library: argument checking, device memory, launches.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
 #include <chrono>
@@ -66,6 +67,12 @@ cudaError_t launch_step_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, 
   cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
+
+// a named range around every entry point that does device work, for timelines (costs nothing without a profiler)
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+};
 
 double now_ms() {
   return std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now().time_since_epoch()).count();
@@ -173,6 +180,7 @@ const char* xg_last_error(void) { return g_last_error.c_str(); }
 // ---------------------------------------------------------------------------------------------
 xg_status_t xg_tokenizer_create(const uint8_t* bytes, const int64_t* offsets, int32_t vocab_size, int32_t eos_token_id,
                                 const int32_t* special_ids, int32_t n_special, void* stream, xg_tokenizer_t** out) {
+  NvtxRange nvtx_range("xg_tokenizer_create");
   (void)stream;
   if (!out) return set_error(XG_ERR_INVALID_ARG, "out is NULL");
   *out = nullptr;
@@ -794,6 +802,7 @@ static xg_status_t jit_advance(CachePool& pool, const std::vector<xg_grammar*>& 
 
 xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool, xg_grammar_kind_t kind, const char* text, size_t len,
                                const char* root_rule, const xg_compile_options_t* opt, void* stream, xg_grammar_t** out) {
+  NvtxRange nvtx_range("xg_compile_grammar");
   if (!out) return set_error(XG_ERR_INVALID_ARG, "out is NULL");
   *out = nullptr;
   if (!text) return set_error(XG_ERR_INVALID_ARG, "text is NULL");
@@ -993,6 +1002,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
 }
 
 xg_status_t xg_jit_service(xg_grammar_t* const* grammars, int32_t n, void* stream, int32_t wait, xg_jit_stats_t* out) {
+  NvtxRange nvtx_range("xg_jit_service");
   if (n < 0 || (n > 0 && !grammars)) return set_error(XG_ERR_INVALID_ARG, "bad grammar array");
   std::vector<std::pair<CachePool*, std::vector<xg_grammar*>>> pools;      // the just-in-time grammars by pool
   for (int i = 0; i < n; ++i) {
@@ -1211,6 +1221,7 @@ static xg_status_t batch_slot(xg_matcher_t* const* matchers, int32_t batch, cons
 
 xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t batch, int32_t* bitmask_dev, int64_t row_stride_words,
                                        int32_t* status_dev, void* stream) {
+  NvtxRange nvtx_range("xg_fill_next_token_bitmask");
   const xg_tokenizer* tok = nullptr;
   BatchSlot* slot = nullptr;
   xg_status_t st = batch_slot(matchers, batch, &tok, &slot);
@@ -1274,6 +1285,7 @@ static xg_status_t static_fill_scratch(StaticFillScratch** out) {
 
 xg_status_t xg_fill_next_token_bitmask_static(xg_matcher_t* const* matchers, int32_t batch, int32_t* bitmask_dev, int64_t row_stride_words,
                                               int32_t* status_dev, void* stream) {
+  NvtxRange nvtx_range("xg_fill_next_token_bitmask_static");
   if (!matchers || batch <= 0) return set_error(XG_ERR_INVALID_ARG, "empty batch");
   if (batch > XG_STATIC_FILL_MAX_BATCH)
     return set_error(XG_ERR_CAPACITY, "batch of " + std::to_string(batch) + " requests exceeds the static scratch limit of " +
@@ -1302,6 +1314,7 @@ xg_status_t xg_fill_next_token_bitmask_static(xg_matcher_t* const* matchers, int
 }
 
 xg_status_t xg_accept_token(xg_matcher_t* const* matchers, int32_t batch, const int32_t* token_ids_dev, int32_t* status_dev, void* stream) {
+  NvtxRange nvtx_range("xg_accept_token");
   const xg_tokenizer* tok = nullptr;
   BatchSlot* slot = nullptr;
   xg_status_t st = batch_slot(matchers, batch, &tok, &slot);
@@ -1315,6 +1328,7 @@ xg_status_t xg_accept_token(xg_matcher_t* const* matchers, int32_t batch, const 
 xg_status_t xg_apply_token_bitmask(void* logits_dev, xg_dtype_t dtype, int32_t batch, int32_t vocab_size, int64_t logits_row_stride_elems,
                                    const int32_t* bitmask_dev, int64_t mask_row_stride_words, const int32_t* row_indices_dev,
                                    int32_t n_rows, void* stream) {
+  NvtxRange nvtx_range("xg_apply_token_bitmask");
   if (!logits_dev || !bitmask_dev) return set_error(XG_ERR_INVALID_ARG, "NULL buffer");
   if (dtype != XG_F32 && dtype != XG_BF16) return set_error(XG_ERR_INVALID_ARG, "unknown dtype");
   if (vocab_size <= 0 || logits_row_stride_elems < vocab_size || mask_row_stride_words < (vocab_size + 31) / 32)

@@ -193,6 +193,24 @@ def test_front_end_limits():
     assert g.stats()["n_states"] >= 300
 
 
+def test_just_in_time_and_class_calls_on_the_host():
+    """What needs no device: the service call over nothing or over grammars without a cache is a no-op, the
+    class export checks its arguments, and the just-in-time options do not change the front end's tables."""
+    assert B.jit_service([], 0, False) == {"n_built": 0, "n_pool_hits": 0, "n_in_flight": 0, "n_missing": 0}
+    text = 'root ::= "[" [a-z]{2,40} "]"'
+    plain = B.Grammar(None, "ebnf", text)
+    jit = B.Grammar(None, "ebnf", text, jit=True, jit_precompute=3, state_compression=False)
+    assert B.jit_service([plain, jit], 0, True)["n_missing"] == 0        # compiled without a tokenizer: not just-in-time grammars
+    ta, tb = plain.tables(), jit.tables()
+    assert all(np.array_equal(ta[k], tb[k]) for k in ta)
+    with pytest.raises(B.XgError) as e:
+        plain.state_classes(-1)                                          # the default depth needs a tokenizer
+    assert e.value.status == B.XG_ERR_INVALID_ARG
+    rep0, rep9 = plain.state_classes(0), plain.state_classes(9)
+    assert len(np.unique(rep0)) <= len(np.unique(rep9)) <= len(rep9)
+    assert (rep9 <= np.arange(len(rep9))).all() and (rep9[rep9] == rep9).all()
+
+
 def test_device_entry_points_fail_loudly_without_a_gpu():
     """No CPU fallback: without a CUDA device the device entry points return XG_ERR_CUDA."""
     try:
