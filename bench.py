@@ -369,32 +369,64 @@ def main():
                                "us_per_launch": t_us, "note": "latency-bound: chains of dependent loads, issue slots 4-11 % busy under ncu"}
 
     # ---- end to end through the C ABI with host buffers ---------------------------------------
-    e2e_steps = max(3, min(args.steps, 12))
+    # Every step: the step's logits come from pinned host memory, the masked logits go back to pinned host memory,
+    # the step's token ids come from the host.  Two device buffers and two copy streams, as a serving loop would
+    # have them: the upload of step t+1 and the download of step t-1 overlap the kernels of step t (PCIe is full
+    # duplex); every dependency is an event, nothing is skipped.
+    e2e_steps = max(4, min(args.steps, 16))
     host_in = torch.empty((n, s.V), dtype=tdtype).pin_memory()
     host_in.copy_(ring[0].cpu())
-    host_out = torch.empty((n, s.V), dtype=tdtype).pin_memory()
+    host_out = [torch.empty((n, s.V), dtype=tdtype).pin_memory() for _ in range(2)]
     host_traj = traj.cpu().pin_memory()
-    restart()
-    dev_buf = ring[0]
+    dev_buf = [ring[0], ring[1 % ring_n]]
+    main = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
     torch.cuda.synchronize()
     h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for phase in ("warm", "timed"):
         restart()
+        torch.cuda.synchronize()
         if phase == "timed":
-            torch.cuda.synchronize()
             h0.record()
+        ev_in = [None, None]
+        ev_out = [None, None]
+        ev_applied = [None, None]
+
+        def upload(t):
+            k = t % 2
+            with torch.cuda.stream(s_in):
+                if ev_out[k] is not None:
+                    s_in.wait_event(ev_out[k])          # the buffer's previous contents have left the device
+                dev_buf[k].copy_(host_in, non_blocking=True)
+                ev_in[k] = torch.cuda.Event()
+                ev_in[k].record(s_in)
+
+        if phase == "timed":
+            s_in.wait_event(h0)
+        upload(0)
         for t in range(e2e_steps):
-            dev_buf.copy_(host_in, non_blocking=True)
+            k = t % 2
+            if t + 1 < e2e_steps:
+                upload(t + 1)
             s.fill()
-            s.apply(dev_buf)
-            host_out.copy_(dev_buf, non_blocking=True)
+            main.wait_event(ev_in[k])
+            s.apply(dev_buf[k])
+            ev_applied[k] = torch.cuda.Event()
+            ev_applied[k].record(main)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_applied[k])
+                host_out[k].copy_(dev_buf[k], non_blocking=True)
+                ev_out[k] = torch.cuda.Event()
+                ev_out[k].record(s_out)
             s.tokens.copy_(host_traj[t], non_blocking=True)
             s.accept_device(s.tokens)
             for b in eos_at[t]:
                 s.reset(b)
+        main.wait_event(ev_out[0])
+        main.wait_event(ev_out[1])
         if phase == "timed":
             h1.record()
-            torch.cuda.synchronize()
+        torch.cuda.synchronize()
     e2e_us = dist_util.max_over_ranks(h0.elapsed_time(h1)) * 1e3 / e2e_steps
 
     line = {
