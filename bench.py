@@ -441,6 +441,8 @@ def main():
         "apply_gbs": apply_gbs,
         "cache_build": {"seconds": build_ms / 1e3, "compile_wall_s": compile_s, "pairs_classified": pairs, "pairs_per_s": pairs / max(build_ms / 1e3, 1e-9),
                         "pairs_dense": pairs_dense, "pairs_dense_per_s": pairs_dense / max(build_ms / 1e3, 1e-9),
+                        "classify_kernel_ms": sum(x["classify_ms"] for x in stats),
+                        "pairs_per_s_classify_kernel": pairs / max(sum(x["classify_ms"] for x in stats) / 1e3, 1e-9),
                         "entries_built": sum(x["n_entries_built"] for x in stats), "entries_reused": sum(x["n_entries_reused"] for x in stats),
                         "entries_shared_by_state_compression": sum(x["n_entries_shared"] for x in stats), "states": sum(x["n_states"] for x in stats),
                         "frontend_ms": sum(x["frontend_ms"] for x in stats),

@@ -202,6 +202,7 @@ typedef struct {
                                    what the per-step check actually streams; <= total_uncertain */
   int64_t n_entries_shared;     /* scannable states that use the entry of an equivalent state of their rule
                                    (repetition state compression, Section 3.6) instead of one of their own */
+  double classify_ms;           /* device time of the classification kernel alone (inside cache_build_ms) */
 } xg_grammar_stats_t;
 xg_status_t xg_grammar_stats(const xg_grammar_t* g, xg_grammar_stats_t* out);
 

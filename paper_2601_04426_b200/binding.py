@@ -71,7 +71,7 @@ class GrammarStats(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_rules", "n_states", "n_scannable", "n_classes", "n_entries_built", "n_entries_reused")] + \
                [(n, C.c_int64) for n in ("pairs_classified", "total_accepted", "total_rejected", "total_uncertain")] + \
                [("kind_count", C.c_int32 * 3), ("pad", C.c_int32), ("cache_bytes", C.c_int64), ("frontend_ms", C.c_double), ("cache_build_ms", C.c_double), ("total_checked", C.c_int64),
-                ("n_entries_shared", C.c_int64)]
+                ("n_entries_shared", C.c_int64), ("classify_ms", C.c_double)]
 
 
 _lib = None

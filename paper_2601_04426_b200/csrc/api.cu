@@ -238,6 +238,13 @@ xg_status_t xg_tokenizer_create(const uint8_t* bytes, const int64_t* offsets, in
   if (err == cudaSuccess) t->dev.rank_to_id = keep(device_copy(t->rank_to_id, &err));
   if (err == cudaSuccess) t->dev.id_to_rank = keep(device_copy(t->id_to_rank, &err));
   if (err == cudaSuccess) t->dev.never = keep(device_copy(never_rank, &err));
+  std::vector<uint16_t> block_first((vocab_size + 255) / 256);
+  for (size_t vb = 0; vb < block_first.size(); ++vb) {          // empty tokens sort first: they count as byte 0
+    const int r0 = (int)vb * 256, r1 = std::min(vocab_size, r0 + 256) - 1;
+    const unsigned lo = off[r0 + 1] > off[r0] ? arena[off[r0]] : 0u, hi = off[r1 + 1] > off[r1] ? arena[off[r1]] : 0u;
+    block_first[vb] = (uint16_t)(lo | (hi << 8));
+  }
+  if (err == cudaSuccess) t->dev.block_first = keep(device_copy(block_first, &err));
   if (err != cudaSuccess) {
     for (void* p : t->allocations) cudaFree(p);
     return set_error(XG_ERR_CUDA, std::string("vocabulary upload: ") + cudaGetErrorString(err));
@@ -379,12 +386,16 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
     XG_CUDA_C(cudaMemsetAsync(unc, 0, row_bytes * n, stream));
     XG_CUDA_C(cudaMemsetAsync(unr, 0, row_bytes * n, stream));
     XG_CUDA_C(cudaMemsetAsync(d_over_count, 0, 2 * sizeof(int), stream));
-    dim3 grid((V + 255) / 256, n);
+    dim3 grid(((V + 255) / 256 + kClassifySpan - 1) / kClassifySpan, n);
+    cudaEvent_t* ev = pool.timing_events();            // device time of the classification itself, for the statistics
+    if (ev) cudaEventRecord(ev[0], stream);
     classify_kernel<<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, acc, unc, unr, d_over, d_over_count, over_cap);
     XG_CUDA_C(cudaGetLastError());
+    if (ev) cudaEventRecord(ev[1], stream);
     int over[2] = {0, 0};
     XG_CUDA_C(cudaMemcpyAsync(over, d_over_count, 2 * sizeof(int), cudaMemcpyDeviceToHost, stream));
     XG_CUDA_C(cudaStreamSynchronize(stream));
+    if (ev) { float ms = 0.f; if (cudaEventElapsedTime(&ms, ev[0], ev[1]) == cudaSuccess) g->stats.classify_ms += ms; }
     if (over[0] > over_cap) { cleanup(); return set_error(XG_ERR_CAPACITY, "too many token walks exceeded the fast path"); }
     for (int done = 0; done < over[0];) {          // exact fallback, a bounded number of pairs per round
       const int round = std::min(over[0] - done, 4096);
@@ -644,7 +655,7 @@ static xg_status_t jit_enqueue_build(JitPool* jp, xg_grammar* g, const std::vect
   XG_CUDA(cudaMemsetAsync(unc, 0, row_bytes * n, stream));
   XG_CUDA(cudaMemsetAsync(unr, 0, row_bytes * n, stream));
   XG_CUDA(cudaMemsetAsync(sc.over_count, 0, 2 * sizeof(int), stream));
-  classify_kernel<<<dim3((V + 255) / 256, n), 256, 0, stream>>>(g->host_view, v, sc.pos, acc, unc, unr, sc.over, sc.over_count, 64);
+  classify_kernel<<<dim3(((V + 255) / 256 + kClassifySpan - 1) / kClassifySpan, n), 256, 0, stream>>>(g->host_view, v, sc.pos, acc, unc, unr, sc.over, sc.over_count, 64);
   count_kernel<<<n, 256, 0, stream>>>(acc, unc, W, sc.counts);
   plan_kernel<<<1, 1024, 0, stream>>>(sc.counts, n, V, W, sc.plan, sc.total);
   jit_reserve_kernel<<<1, 32, 0, stream>>>(sc.plan, n, sc.total, arena->d_used, arena->cap_words, sc.over_count, sc.result);

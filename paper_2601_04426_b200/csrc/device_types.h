@@ -19,6 +19,7 @@ struct VocabDev {
   const int32_t* rank_to_id; // [V]
   const int32_t* id_to_rank; // [V]
   const uint8_t* never;      // [V] by rank: 1 = EOS, special or zero-length (never classified)
+  const uint16_t* block_first; // [ceil(V / 256)]: first byte of the first token of a block of 256 ranks | first byte of its last << 8
 };
 
 // One adaptive cache entry (Section 3.4): the accepted/rejected split in its smallest form plus

@@ -597,22 +597,41 @@ Fsm determinize(const Fsm& f, int max_states) {
   return d;
 }
 
-// Equal word sequences get equal ids, numbered in order of first appearance.
+// Equal word sequences get equal ids, numbered in order of first appearance.  Open addressing on a
+// 64-bit hash of the words; a hit is confirmed against the stored words.
 struct SignatureTable {
-  std::unordered_map<uint64_t, std::vector<int>> buckets;
   std::vector<uint32_t> words;                         // every distinct signature, back to back
   std::vector<std::pair<size_t, size_t>> span;         // id -> (begin, length)
+  std::vector<uint64_t> slot_hash;
+  std::vector<int> slot_id;                            // -1 = empty
   int size() const { return (int)span.size(); }
+  void grow() {
+    const size_t cap = slot_id.empty() ? 64 : slot_id.size() * 2;
+    std::vector<uint64_t> nh(cap, 0);
+    std::vector<int> ni(cap, -1);
+    for (size_t k = 0; k < slot_id.size(); ++k) {
+      if (slot_id[k] < 0) continue;
+      size_t at = (size_t)slot_hash[k] & (cap - 1);
+      while (ni[at] >= 0) at = (at + 1) & (cap - 1);
+      nh[at] = slot_hash[k]; ni[at] = slot_id[k];
+    }
+    slot_hash.swap(nh); slot_id.swap(ni);
+  }
   int intern(const std::vector<uint32_t>& sig) {
     uint64_t h = 0x9E3779B97F4A7C15ull ^ sig.size();
     for (uint32_t x : sig) { h ^= x; h *= 0xBF58476D1CE4E5B9ull; h ^= h >> 29; }
-    std::vector<int>& bucket = buckets[h];
-    for (int id : bucket)
-      if (span[id].second == sig.size() && std::equal(sig.begin(), sig.end(), words.begin() + span[id].first)) return id;
+    if (span.size() * 2 >= slot_id.size()) grow();
+    const size_t mask = slot_id.size() - 1;
+    size_t at = (size_t)h & mask;
+    while (slot_id[at] >= 0) {
+      const int id = slot_id[at];
+      if (slot_hash[at] == h && span[id].second == sig.size() && std::equal(sig.begin(), sig.end(), words.begin() + span[id].first)) return id;
+      at = (at + 1) & mask;
+    }
     const int id = (int)span.size();
     span.emplace_back(words.size(), sig.size());
     words.insert(words.end(), sig.begin(), sig.end());
-    bucket.push_back(id);
+    slot_hash[at] = h; slot_id[at] = id;
     return id;
   }
 };

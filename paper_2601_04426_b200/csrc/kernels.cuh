@@ -155,6 +155,8 @@ __device__ __forceinline__ const uint32_t* stage_class_bits(const GrammarDev& g,
 // Accepted and uncertain bits are scattered into id-ordered rows; the uncertain bits are also
 // ballot-packed in rank order (the order later walks use).
 // ------------------------------------------------------------------------------------------
+constexpr int kClassifySpan = 8;      // vocabulary blocks of 256 ranks per thread block
+
 __global__ void __launch_bounds__(256)
 classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
                 uint32_t* __restrict__ acc_id, uint32_t* __restrict__ unc_id, uint32_t* __restrict__ unc_rank,
@@ -163,14 +165,11 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
   __shared__ int32_t sh_org[1];
   __shared__ uint32_t sh_class[kSharedClasses * 8];
   __shared__ uint32_t sh_first[8];          // bytes the position's own edges can take
-  __shared__ int sh_skip;
+  __shared__ uint32_t sh_live;              // which of this block's vocabulary blocks hold a token that survives its first byte
   const int pos = blockIdx.y;
   const int state = positions[pos];
-  const int rank = blockIdx.x * blockDim.x + threadIdx.x;
+  const int n_vblocks = (v.vocab_size + 255) >> 8;
   if (threadIdx.x < 8) {
-    // own first-byte set, and an early exit for the whole block: the tokens of a block are a
-    // contiguous run of the trie order, so their first bytes span [first of the first token,
-    // first of the last]; most (position, block) pairs have nothing in common
     const StateRec rec = g.state[state];
     uint32_t w = 0;
     for (int e = 0; e < (int)(rec.n_own_n_scan & 0xFFFFu); ++e) {
@@ -181,55 +180,63 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
     sh_first[threadIdx.x] = w;
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
-    const int r0 = blockIdx.x * blockDim.x, r1 = min(v.vocab_size, r0 + (int)blockDim.x) - 1;
-    // empty tokens sort first; treat them as byte 0
-    const uint32_t o0 = v.offset[r0], o1 = v.offset[r1];
-    const int b0 = v.offset[r0 + 1] > o0 ? v.bytes[o0] : 0, b1 = v.offset[r1 + 1] > o1 ? v.bytes[o1] : 0;
+  if (threadIdx.x < 32) {
+    // The tokens of a vocabulary block are a contiguous run of the trie order, so their first bytes span
+    // [first of the first token, first of the last] (a table of the tokenizer); most (position, block) pairs
+    // have nothing in common with the position's own first-byte set and are rejected here as a whole.
     bool any = false;
-    for (int b = b0; b <= b1 && !any; ++b) any = (sh_first[b >> 5] >> (b & 31)) & 1u;
-    sh_skip = any ? 0 : 1;
-    sh_st[0] = (uint32_t)state; sh_org[0] = -1;
+    const int vb = blockIdx.x * kClassifySpan + (int)threadIdx.x;
+    if (threadIdx.x < kClassifySpan && vb < n_vblocks) {
+      const uint32_t span = v.block_first[vb];
+      for (int b = (int)(span & 0xFFu); b <= (int)(span >> 8) && !any; ++b) any = (sh_first[b >> 5] >> (b & 31)) & 1u;
+    }
+    const uint32_t live = __ballot_sync(0xFFFFFFFFu, any);
+    if (threadIdx.x == 0) { sh_live = live; sh_st[0] = (uint32_t)state; sh_org[0] = -1; }
   }
   __syncthreads();
-  if (sh_skip) return;                       // every token of the block is rejected on its first byte (rows are pre-zeroed)
+  const uint32_t live_blocks = sh_live;
+  if (live_blocks == 0) return;              // every token here is rejected on its first byte (the rows are pre-zeroed)
   const uint32_t* class_bits = stage_class_bits(g, sh_class);
   __syncthreads();
-  int cls = 0;
-  bool live = rank < v.vocab_size && !v.never[rank];
-  uint32_t off = 0;
-  if (live) {
-    off = v.offset[rank];
-    const uint32_t first_byte = v.bytes[off];
-    live = (sh_first[first_byte >> 5] >> (first_byte & 31)) & 1u;             // else rejected on the first byte
-  }
-  if (live) {
-    const int len = (int)(v.offset[rank + 1] - off);
-    int flags = 0;
-    int consumed = 0;
-    if (len > kFastMaxBytes) flags = kWalkOverflow;
-    else {
-      uint32_t st[kFastCap];
-      int32_t org[kFastCap];
-      int16_t lsb[kFastMaxBytes + 2];
-      Chart c;
-      c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1;
-      c.i_st = sh_st; c.i_org = sh_org; c.i_cnt = 1; c.i_idx = 0;
-      consumed = token_walk<int16_t>(g, class_bits, c, v.bytes + off, len, true, st, org, kFastCap, lsb, &flags, nullptr);
+  for (int i = 0; i < kClassifySpan; ++i) {
+    if (!((live_blocks >> i) & 1u)) continue;
+    const int rank = ((blockIdx.x * kClassifySpan + i) << 8) + (int)threadIdx.x;
+    int cls = 0;
+    bool live = rank < v.vocab_size && !v.never[rank];
+    uint32_t off = 0;
+    if (live) {
+      off = v.offset[rank];
+      const uint32_t first_byte = v.bytes[off];
+      live = (sh_first[first_byte >> 5] >> (first_byte & 31)) & 1u;             // else rejected on the first byte
     }
-    if (flags & kWalkOverflow) {
-      int slot = atomicAdd(overflow_count, 1);
-      if (slot < overflow_cap) overflow[slot] = make_int2(pos, rank);
-    } else if (consumed == len) cls = 1;
-    else if (flags & kWalkUncertain) cls = 2;
-    if (cls) {
-      const int id = v.rank_to_id[rank];
-      uint32_t* row = (cls == 1 ? acc_id : unc_id) + (size_t)pos * v.n_words;
-      atomicOr(&row[id >> 5], 1u << (id & 31));
+    if (live) {
+      const int len = (int)(v.offset[rank + 1] - off);
+      int flags = 0;
+      int consumed = 0;
+      if (len > kFastMaxBytes) flags = kWalkOverflow;
+      else {
+        uint32_t st[kFastCap];
+        int32_t org[kFastCap];
+        int16_t lsb[kFastMaxBytes + 2];
+        Chart c;
+        c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1;
+        c.i_st = sh_st; c.i_org = sh_org; c.i_cnt = 1; c.i_idx = 0;
+        consumed = token_walk<int16_t>(g, class_bits, c, v.bytes + off, len, true, st, org, kFastCap, lsb, &flags, nullptr);
+      }
+      if (flags & kWalkOverflow) {
+        int slot = atomicAdd(overflow_count, 1);
+        if (slot < overflow_cap) overflow[slot] = make_int2(pos, rank);
+      } else if (consumed == len) cls = 1;
+      else if (flags & kWalkUncertain) cls = 2;
+      if (cls) {
+        const int id = v.rank_to_id[rank];
+        uint32_t* row = (cls == 1 ? acc_id : unc_id) + (size_t)pos * v.n_words;
+        atomicOr(&row[id >> 5], 1u << (id & 31));
+      }
     }
+    const uint32_t ballot = __ballot_sync(0xFFFFFFFFu, cls == 2);
+    if ((threadIdx.x & 31) == 0 && rank < v.vocab_size) unc_rank[(size_t)pos * v.n_words + (rank >> 5)] = ballot;
   }
-  const uint32_t ballot = __ballot_sync(0xFFFFFFFFu, cls == 2);
-  if ((threadIdx.x & 31) == 0 && rank < v.vocab_size) unc_rank[(size_t)pos * v.n_words + (rank >> 5)] = ballot;
 }
 
 // exact fallback for the pairs whose walk did not fit the fast path's fixed arrays

@@ -86,6 +86,15 @@ CachePool::~CachePool() {
   for (auto& s : scratch_) cudaFree(s.first);
   cudaFree(jit_.d_used);
   if (jit_host && jit_host_free) jit_host_free(jit_host);
+  for (cudaEvent_t e : timing_) if (e) cudaEventDestroy(e);
+}
+
+cudaEvent_t* CachePool::timing_events() {
+  if (!timing_[0]) {
+    if (cudaEventCreate(&timing_[0]) != cudaSuccess) { timing_[0] = nullptr; return nullptr; }
+    if (cudaEventCreate(&timing_[1]) != cudaSuccess) { cudaEventDestroy(timing_[0]); timing_[0] = timing_[1] = nullptr; return nullptr; }
+  }
+  return timing_;
 }
 
 const CachePool::JitArena* CachePool::jit_arena(long long min_words, bool renew, long long first_words) {

@@ -93,6 +93,8 @@ class CachePool {
   // the current arena, or a fresh one of at least `min_words` when there is none or `renew` is set (call with `mu` held)
   // `first_words` > 0 sizes the very first arena (default 8 Mi words)
   const JitArena* jit_arena(long long min_words, bool renew, long long first_words = 0);
+  // two events for timing a build step on the device (created on first use; nullptr if that fails)
+  cudaEvent_t* timing_events();
   // host-side state of the just-in-time service (owned here, defined by the API layer)
   void* jit_host = nullptr;
   void (*jit_host_free)(void*) = nullptr;
@@ -108,6 +110,7 @@ class CachePool {
   uint64_t clock_ = 0;
   std::vector<std::pair<void*, size_t>> scratch_;
   JitArena jit_;
+  cudaEvent_t timing_[2] = {nullptr, nullptr};
   int find_or_add(uint64_t hash, std::vector<uint64_t>&& serial);
 };
 
