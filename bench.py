@@ -157,6 +157,7 @@ def main():
     ap.add_argument("--jit-sweep", default=None,
                     help="comma-separated K values (or 'full'): compile just in time with K entries precomputed and report "
                          "compile time and per-step time avg / P99 / max over the trajectory (the shape of the paper's K sweep)")
+    ap.add_argument("--compile-threads", type=int, default=0, help="host threads compiling the grammars (0 = one per core, at most 16)")
     ap.add_argument("--no-state-compression", action="store_true",
                     help="build one cache entry per scannable state (ablation of the repetition state compression)")
     args = ap.parse_args()
@@ -202,7 +203,7 @@ def main():
     wt.close()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
-    s = engine.Session(w, device="cuda:%d" % local_rank, state_compression=not args.no_state_compression)
+    s = engine.Session(w, device="cuda:%d" % local_rank, state_compression=not args.no_state_compression, compile_threads=args.compile_threads)
     torch.cuda.synchronize()
     compile_s = time.perf_counter() - t0
     stats = [g.stats() for g in s.grammars]
@@ -439,7 +440,7 @@ def main():
         "clocks": clocks,
         "kernels_us": {"fill": t_fill, "apply": t_apply, "accept": t_accept},
         "apply_gbs": apply_gbs,
-        "cache_build": {"seconds": build_ms / 1e3, "compile_wall_s": compile_s, "pairs_classified": pairs, "pairs_per_s": pairs / max(build_ms / 1e3, 1e-9),
+        "cache_build": {"seconds": build_ms / 1e3, "compile_wall_s": compile_s, "compile_threads": args.compile_threads or min(16, os.cpu_count() or 1), "pairs_classified": pairs, "pairs_per_s": pairs / max(build_ms / 1e3, 1e-9),
                         "pairs_dense": pairs_dense, "pairs_dense_per_s": pairs_dense / max(build_ms / 1e3, 1e-9),
                         "classify_kernel_ms": sum(x["classify_ms"] for x in stats),
                         "pairs_per_s_classify_kernel": pairs / max(sum(x["classify_ms"] for x in stats) / 1e3, 1e-9),

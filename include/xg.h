@@ -126,6 +126,8 @@ typedef struct {
  * xg_grammar_get_tables but cannot make matchers, and no CUDA call is made.
  * pool may be NULL (a private pool is used).  root_rule: EBNF only, NULL = "root".
  * Synchronous: the cache is complete when the call returns.
+ * May be called from several host threads at once, also with one pool: the front ends run side
+ * by side, the cache builds of one pool take turns (each thread must have the device current).
  * Errors: XG_ERR_PARSE, XG_ERR_UNSUPPORTED, XG_ERR_CAPACITY, XG_ERR_CUDA, XG_ERR_OOM. */
 xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool, xg_grammar_kind_t kind,
                                const char* text, size_t len, const char* root_rule,

@@ -855,9 +855,9 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   g->entries.assign(f.n_states, EntryDev{});
   g->entry_counts.assign(f.n_states, make_int2(0, 0));
   g->entry_chunk.assign(f.n_states, -1);
-  const double t1 = now_ms();
   const std::shared_ptr<CachePool> pool_keep = g->pool;      // outlives the lock below on every path
   std::lock_guard<std::mutex> pool_lock(pool_keep->mu);
+  const double t1 = now_ms();                                 // the cache build proper: not the wait for another thread's compile
   bool retained = false;
   auto fail = [&](xg_status_t status) {                       // the lock is held: give everything back without taking it again
     cudaDeviceSynchronize();

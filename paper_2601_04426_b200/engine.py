@@ -5,6 +5,8 @@ pointers through `binding`, and moves results to numpy.  It needs a CUDA device.
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
 from typing import List, Optional, Sequence
 
 import numpy as np
@@ -18,7 +20,7 @@ class Session:
     """One tokenizer, its compiled grammars and one matcher per request of a workload."""
 
     def __init__(self, workload: inputs.Workload, share_pool: bool = True, device: str = "cuda:0", state_compression: bool = True,
-                 jit: bool = False, jit_precompute: int = 0, jit_arena_bytes: int = 0):
+                 jit: bool = False, jit_precompute: int = 0, jit_arena_bytes: int = 0, compile_threads: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         self.device = torch.device(device)
@@ -27,9 +29,19 @@ class Session:
         v = workload.vocab
         self.tokenizer = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
         self.pool = B.CachePool(self.tokenizer) if share_pool else None
-        self.grammars: List[B.Grammar] = [B.Grammar(self.tokenizer, g.kind, g.text, pool=self.pool, state_compression=state_compression,
-                                                    jit=jit, jit_precompute=jit_precompute, jit_arena_bytes=jit_arena_bytes)
-                                          for g in workload.grammars]
+        # xg_compile_grammar may be called from several threads: the host front ends run side by side, the
+        # cache builds take turns on the pool.  compile_threads: 0 = one per core (at most 16), 1 = in this thread.
+        def compile_one(g):
+            torch.cuda.set_device(self.device)
+            return B.Grammar(self.tokenizer, g.kind, g.text, pool=self.pool, state_compression=state_compression,
+                             jit=jit, jit_precompute=jit_precompute, jit_arena_bytes=jit_arena_bytes)
+        n_threads = compile_threads if compile_threads > 0 else min(16, os.cpu_count() or 1)
+        n_threads = max(1, min(n_threads, len(workload.grammars)))
+        if n_threads == 1:
+            self.grammars: List[B.Grammar] = [compile_one(g) for g in workload.grammars]
+        else:
+            with ThreadPoolExecutor(max_workers=n_threads) as ex:
+                self.grammars = list(ex.map(compile_one, workload.grammars))
         self.matchers = [B.Matcher(self.grammars[gi]) for gi in workload.request_grammar]
         self.batch = B.Batch(self.matchers)
         self.V, self.W, self.n = v.size, self.tokenizer.words, len(self.matchers)
