@@ -284,3 +284,20 @@ def test_structural_hash_on_cycles():
     assert set(_hashes(renamed, root="p").tolist()) == set(ha.tolist())
     other = 'a ::= "1" b | "x"\nb ::= "2" c | "y"\nc ::= "4" a | "z"'
     assert not set(_hashes(other, root="a").tolist()) & set(ha.tolist())
+
+
+def test_front_end_is_reentrant():
+    """Several threads compiling at once get the tables a single thread gets."""
+    from concurrent.futures import ThreadPoolExecutor
+    w = inputs.make_workload("C3", batch=12, steps=2)
+
+    def tables(spec):
+        t = B.Grammar(None, spec.kind, spec.text).tables()
+        return {k: (v.copy() if hasattr(v, "copy") else v) for k, v in t.items()}
+
+    serial = [tables(g) for g in w.grammars]
+    with ThreadPoolExecutor(max_workers=6) as ex:
+        threaded = list(ex.map(tables, w.grammars * 3))
+    for i, t in enumerate(threaded):
+        ref = serial[i % len(serial)]
+        assert all(np.array_equal(ref[k], t[k]) for k in ref), i

@@ -485,3 +485,19 @@ def test_item_sets_beyond_the_fast_path():
     batch.fill_next_token_bitmask(mask.data_ptr(), tok.words, st.data_ptr())
     assert int(st.cpu()[0]) == 0 and np.array_equal(mask.cpu().numpy().view(np.uint32)[0], om.mask(ov))
     m.close(); g.close(); tok.close()
+
+
+def test_threaded_compile_into_one_pool_builds_the_same_cache():
+    """Grammars compiled from eight threads into a shared pool: the same entries as from one thread, and
+    between them exactly as many built + reused entries (who builds a shared rule is a matter of timing)."""
+    torch, engine = _engine()
+    w = inputs.make_workload("C3", batch=12, steps=2, vocab_size=8192)
+    a = engine.Session(w, compile_threads=8)
+    b = engine.Session(w, compile_threads=1)
+    sa, sb = [g.stats() for g in a.grammars], [g.stats() for g in b.grammars]
+    total = lambda st: sum(x["n_entries_built"] + x["n_entries_reused"] + x["n_entries_shared"] for x in st)
+    assert total(sa) == total(sb)
+    assert sum(x["n_entries_built"] for x in sa) == sum(x["n_entries_built"] for x in sb)
+    for ga, gb in zip(a.grammars, b.grammars):
+        _same_entries(ga, gb, stride=37)
+    a.close(); b.close()
