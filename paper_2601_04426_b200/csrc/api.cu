@@ -856,6 +856,20 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   g->entry_counts.assign(f.n_states, make_int2(0, 0));
   g->entry_chunk.assign(f.n_states, -1);
   const std::shared_ptr<CachePool> pool_keep = g->pool;      // outlives the lock below on every path
+  // what needs neither the pool nor the device comes before the lock, so that threads compiling side by side
+  // only take turns for the pool lookups and the cache build: rule hashes and canonical orders (Section 3.3), and
+  // the classes of states that share a cache entry (repetition state compression, Section 3.6)
+  std::shared_ptr<const void> prepared;
+  std::vector<int32_t> rep(f.n_states);
+  const double t_pre = now_ms();
+  try {
+    prepared = prepare_interning(f);
+    if (compress && tok->dev.max_len > 0) rep = bounded_equivalence(f, tok->dev.max_len);
+    else for (int s = 0; s < f.n_states; ++s) rep[s] = s;
+  } catch (const std::exception& e) {
+    return set_error(XG_ERR_OOM, e.what());
+  }
+  const double pre_ms = now_ms() - t_pre;
   std::lock_guard<std::mutex> pool_lock(pool_keep->mu);
   const double t1 = now_ms();                                 // the cache build proper: not the wait for another thread's compile
   bool retained = false;
@@ -880,7 +894,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   // reuse its entries; the others are classified now and registered afterwards
   RuleInterning in;
   try {
-    in = g->pool->intern(f);
+    in = g->pool->intern(f, prepared);
   } catch (const std::exception& e) {
     return fail(set_error(XG_ERR_OOM, e.what()));
   }
@@ -889,11 +903,8 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   std::vector<int> canon_of(f.n_states, -1);          // state -> canonical index inside its rule
   for (int r = 0; r < f.n_rules; ++r)
     for (size_t k = 0; k < in.canon[r].size(); ++k) canon_of[rule_first[r] + in.canon[r][k]] = (int)k;
-  // Repetition state compression (Section 3.6): states of a rule that no token of this vocabulary
-  // can tell apart share the entry of their class representative
-  std::vector<int32_t> rep(f.n_states);
-  if (compress && tok->dev.max_len > 0) rep = bounded_equivalence(f, tok->dev.max_len);
-  else for (int s = 0; s < f.n_states; ++s) rep[s] = s;
+  // (`rep`: states of a rule that no token of this vocabulary can tell apart share the entry of their class
+  // representative)
   std::map<int, int> builder_of;                      // pool rule -> the rule of this grammar that builds it
   std::vector<int32_t> to_build;
   auto in_pool = [&](int s) {
@@ -994,7 +1005,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   if (st == XG_OK) st = narrow_check_lists(g.get(), scannable, rep, (cudaStream_t)stream);
   if (st == XG_OK) st = upload_grammar(g.get());       // and with this grammar's narrowed check lists
   if (st != XG_OK) return fail(st);
-  g->stats.cache_build_ms = now_ms() - t1;
+  g->stats.cache_build_ms = now_ms() - t1 + pre_ms;
   g->stats.n_entries_built = (int)to_build.size();
   g->stats.pairs_classified = (int64_t)to_build.size() * tok->vocab_size;
   for (int s : scannable) {

@@ -1,6 +1,7 @@
 #include "pool.h"
 
 #include <algorithm>
+#include <memory>
 #include <functional>
 #include <iterator>
 
@@ -355,8 +356,13 @@ Analysis analyse(const FlatGrammar& g) {
 
 RuleInterning structural_hashes(const FlatGrammar& g) { return analyse(g).out; }
 
-RuleInterning CachePool::intern(const FlatGrammar& g) {
-  Analysis a = analyse(g);
+// the part of interning that needs no pool: shapes, canonical state orders, hashes
+std::shared_ptr<const void> prepare_interning(const FlatGrammar& g) {
+  return std::shared_ptr<const void>(new Analysis(analyse(g)), [](const void* p) { delete static_cast<const Analysis*>(p); });
+}
+
+RuleInterning CachePool::intern(const FlatGrammar& g, const std::shared_ptr<const void>& prepared) {
+  Analysis a = prepared ? *static_cast<const Analysis*>(prepared.get()) : analyse(g);
   RuleInterning& out = a.out;
   const int R = g.n_rules;
   // exact identities: serialise each rule with its callees named by pool id; members of a

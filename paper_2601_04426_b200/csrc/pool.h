@@ -6,6 +6,7 @@
 
 #include <cstdint>
 #include <map>
+#include <memory>
 #include <mutex>
 #include <unordered_map>
 #include <vector>
@@ -36,6 +37,9 @@ struct RuleInterning {
 // Hashes and canonical state orders only (no pool): Algorithm 1 bottom-up over the reference
 // graph, Algorithm 2's refinement on cycles.
 RuleInterning structural_hashes(const FlatGrammar& g);
+// The pool-independent part of CachePool::intern (rule shapes, canonical orders, hashes): needs no lock, so
+// threads that compile side by side only take turns for the pool lookups and the cache build.
+std::shared_ptr<const void> prepare_interning(const FlatGrammar& g);
 
 // Device memory in slabs with a first-fit free list.  Compiling a grammar needs a handful of
 // device buffers (its tables, a batch of cache entries, its narrowed check lists); taking each
@@ -64,7 +68,8 @@ class CachePool {
   std::mutex mu;                            // one compile at a time per pool
 
   // find-or-create pool rules for every rule of `g`, callees first (call with `mu` held)
-  RuleInterning intern(const FlatGrammar& g);
+  // `prepared` (optional): the result of prepare_interning(g), computed without the lock
+  RuleInterning intern(const FlatGrammar& g, const std::shared_ptr<const void>& prepared = nullptr);
   PoolRule& rule(int id) { return rules_[id]; }
   size_t n_rules() const { return rules_.size(); }
   // Device memory for one batch of freshly built entries.  Chunks are the unit of eviction
