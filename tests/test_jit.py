@@ -265,3 +265,13 @@ def test_teardown_with_builds_in_flight_and_pool_accounting():
     assert g.stats()["n_entries_built"] == 3
     g.close()
     pool.close(); tokenizer.close()
+
+
+def test_just_in_time_entries_serve_whole_classes_of_states():
+    """Long repetitions: one entry built just in time is published to every state of its class
+    (repetition state compression), so a string of hundreds of characters costs a handful of builds."""
+    w = inputs.make_workload("R256", batch=4, steps=150, vocab_size=8192)
+    s, final, _, stats = _drive(w, 6, "each")
+    assert 0 < final["n_built"] < 400
+    assert sum(x["n_states"] for x in stats) > 20 * final["n_built"]
+    s.close()
