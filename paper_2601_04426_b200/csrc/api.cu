@@ -152,6 +152,7 @@ struct xg_grammar {
   GrammarDev* dev = nullptr;            // the same struct in device memory
   void* blob = nullptr;
   void* lookahead_arena = nullptr;      // this grammar's narrowed check lists
+  size_t entries_offset = 0;            // where the entry headers sit inside `blob`
   std::vector<int> entry_chunk;         // [n_states] pool chunk that holds the state's entry (-1: none)
   std::vector<int> chunk_refs;          // pool chunks this grammar keeps alive
   xg_grammar_stats_t stats{};
@@ -287,6 +288,14 @@ xg_status_t xg_cache_pool_stats(xg_cache_pool_t* pool, xg_cache_pool_stats_t* ou
 // ---------------------------------------------------------------------------------------------
 // grammar compilation
 // ---------------------------------------------------------------------------------------------
+// the entry headers alone, once the tables are on the device (the headers change twice during a compile: when the
+// entries are built, and when this grammar's lookahead has narrowed their check lists)
+static xg_status_t upload_entry_headers(xg_grammar* g) {
+  if (!g->blob) return set_error(XG_ERR_INVALID_ARG, "internal: tables not uploaded yet");
+  XG_CUDA(cudaMemcpy((uint8_t*)g->blob + g->entries_offset, g->entries.data(), g->entries.size() * sizeof(EntryDev), cudaMemcpyHostToDevice));
+  return XG_OK;
+}
+
 static xg_status_t upload_grammar(xg_grammar* g) {
   const FlatGrammar& f = g->flat;
   // one blob, sections 16-byte aligned
@@ -345,6 +354,7 @@ static xg_status_t upload_grammar(xg_grammar* g) {
   v.state_first = (const uint32_t*)(d + o_first);
   v.rule_follow = (const uint32_t*)(d + o_follow);
   v.entries = (const EntryDev*)(d + o_en);
+  g->entries_offset = o_en;
   v.miss_ring = g->jit.slot >= 0 ? ((JitPool*)g->pool->jit_host)->d_ring : nullptr;
   v.jit_slot = g->jit.slot;
   put(o_self, &v, sizeof(GrammarDev));
@@ -1001,9 +1011,9 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
       return fail(set_error(XG_ERR_CUDA, "upload of the state classes failed"));
     j.enabled = true;
   }
-  st = upload_grammar(g.get());       // now with the entry headers
+  st = upload_entry_headers(g.get());       // now with the entry headers
   if (st == XG_OK) st = narrow_check_lists(g.get(), scannable, rep, (cudaStream_t)stream);
-  if (st == XG_OK) st = upload_grammar(g.get());       // and with this grammar's narrowed check lists
+  if (st == XG_OK) st = upload_entry_headers(g.get());       // and with this grammar's narrowed check lists
   if (st != XG_OK) return fail(st);
   g->stats.cache_build_ms = now_ms() - t1 + pre_ms;
   g->stats.n_entries_built = (int)to_build.size();
