@@ -290,6 +290,7 @@ def main():
     spin_cycles = int(2.0e5)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     zero_bits_sum, mask_samples = 0, 0
+    fill_work = {"merge_bytes": 0, "check_bytes": 0, "row_bytes": 0, "check_tokens": 0, "steps": 0}
     for i in range(total):
         t = i % w.steps
         if t == 0 and i > 0:
@@ -313,6 +314,12 @@ def main():
         if ev and (i - warmup) % 10 == 0:            # masked fraction, sampled (synchronises; outside the event intervals)
             zero_bits_sum += n * s.V - int(np.unpackbits(s.mask_numpy().view(np.uint8)).sum())
             mask_samples += 1
+            if (i - warmup) % 10 == 0:                 # what the next fill streams: cache entries merged, candidates tested, row written
+                for m in s.matchers:
+                    fw = m.next_fill_work(s.stream())
+                    fill_work["merge_bytes"] += fw["merge_bytes"]; fill_work["check_bytes"] += fw["check_bytes"]
+                    fill_work["row_bytes"] += fw["row_bytes"]; fill_work["check_tokens"] += fw["check_tokens"]
+                fill_work["steps"] += 1
     torch.cuda.synchronize()
     eager_us = {"fill": float(np.mean([e[0].elapsed_time(e[1]) for e in evs])) * 1e3,
                 "apply": float(np.mean([e[1].elapsed_time(e[2]) for e in evs])) * 1e3,
@@ -368,6 +375,13 @@ def main():
                                "achieved": (wi / (t_us * 1e-6)) if wi else None, "peak": issue_peak, "unit": "warp instructions/s",
                                "frac": (wi / (t_us * 1e-6) / issue_peak) if wi else None, "warp_instructions_per_launch": wi,
                                "us_per_launch": t_us, "note": "latency-bound: chains of dependent loads, issue slots 4-11 % busy under ncu"}
+
+    fw_steps = max(fill_work["steps"], 1)
+    fill_bytes = (fill_work["merge_bytes"] + fill_work["check_bytes"] + fill_work["row_bytes"]) / fw_steps
+    fill_stream = {"bytes_per_launch": fill_bytes, "merge_bytes": fill_work["merge_bytes"] / fw_steps, "check_bytes": fill_work["check_bytes"] / fw_steps,
+                   "row_bytes": fill_work["row_bytes"] / fw_steps, "uncertain_candidates_per_launch": fill_work["check_tokens"] / fw_steps,
+                   "gbs": fill_bytes / (t_fill * 1e-6) / 1e9, "frac_of_hbm_peak": fill_bytes / (t_fill * 1e-6) / 1e9 / peak,
+                   "sampled_steps": fill_work["steps"]}
 
     # ---- end to end through the C ABI with host buffers ---------------------------------------
     # Every step: the step's logits come from pinned host memory, the masked logits go back to pinned host memory,
@@ -451,6 +465,7 @@ def main():
                         "cache_bytes_unique_upper": sum(x["cache_bytes"] for x in stats)},
         "roofline": roofline,
         "roofline_latency_bound_kernels": latency_bound,
+        "fill_streaming": fill_stream,
         "e2e": {"value": e2e_us, "unit": "us/step", "h2d_bytes_per_step": bytes_one + 4 * n, "d2h_bytes_per_step": bytes_one, "steps": e2e_steps},
         "gpu_launches": timed_launches,
     }

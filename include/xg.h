@@ -246,6 +246,18 @@ void xg_matcher_destroy(xg_matcher_t* m);
 /* *out = 1 iff EOS has been accepted.  Synchronises `stream`. */
 xg_status_t xg_matcher_is_terminated(const xg_matcher_t* m, void* stream, int32_t* out);
 
+/* What the next xg_fill_next_token_bitmask has to stream for this matcher (for measurements): the
+ * bytes of the cache entries it merges (bitsets in full, lists in full -- a block reads only its
+ * slice of a list, but all blocks together read all of it), the uncertain candidates it tests
+ * (5 bytes each: exit mask and first-exit byte) and the row it writes.  List lengths and check
+ * counts are the compile-time ones (entries that arrived just in time count with their whole
+ * uncertain list).  Synchronises `stream`. */
+typedef struct {
+  int32_t n_merge, n_check, n_missing, pad;
+  int64_t merge_bytes, check_tokens, check_bytes, row_bytes;
+} xg_fill_work_t;
+xg_status_t xg_matcher_next_fill_work(const xg_matcher_t* m, void* stream, xg_fill_work_t* out);
+
 /* ---- per decode step ----------------------------------------------------------------------
  * xg_fill_next_token_bitmask: for each of `batch` matchers (host array of handles, all on one
  * tokenizer, grammars may differ) write its next-token bitmask into

@@ -27,7 +27,7 @@ DTYPE_BY_NAME = {"f32": XG_F32, "bf16": XG_BF16}
 EXPORTS = [
     "xg_last_error", "xg_tokenizer_create", "xg_tokenizer_destroy", "xg_cache_pool_create", "xg_cache_pool_destroy", "xg_cache_pool_set_limit", "xg_cache_pool_stats",
     "xg_compile_grammar", "xg_grammar_destroy", "xg_grammar_get_tables", "xg_grammar_get_rule_hashes", "xg_grammar_get_cache_entry", "xg_grammar_get_state_classes", "xg_grammar_stats", "xg_jit_service",
-    "xg_matcher_create", "xg_matcher_reset", "xg_matcher_destroy", "xg_matcher_is_terminated",
+    "xg_matcher_create", "xg_matcher_reset", "xg_matcher_destroy", "xg_matcher_is_terminated", "xg_matcher_next_fill_work",
     "xg_fill_next_token_bitmask", "xg_fill_next_token_bitmask_static", "xg_apply_token_bitmask", "xg_accept_token",
 ]
 XG_STATIC_FILL_MAX_BATCH = 1024
@@ -42,6 +42,11 @@ class XgError(RuntimeError):
 class CompileOptions(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("inline_max_states", C.c_int32), ("max_rule_states", C.c_int32), ("build_cache", C.c_int32),
                 ("no_state_compression", C.c_int32), ("jit", C.c_int32), ("jit_precompute", C.c_int32), ("jit_arena_bytes", C.c_int64)]
+
+
+class FillWork(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_merge", "n_check", "n_missing", "pad")] + \
+               [(n, C.c_int64) for n in ("merge_bytes", "check_tokens", "check_bytes", "row_bytes")]
 
 
 class JitStats(C.Structure):
@@ -111,6 +116,7 @@ def lib():
         L.xg_matcher_destroy.argtypes = [vp]
         L.xg_matcher_destroy.restype = None
         L.xg_matcher_is_terminated.argtypes = [vp, vp, C.POINTER(i32)]
+        L.xg_matcher_next_fill_work.argtypes = [vp, vp, C.POINTER(FillWork)]
         L.xg_fill_next_token_bitmask.argtypes = [vp, i32, vp, i64, vp, vp]
         L.xg_fill_next_token_bitmask_static.argtypes = [vp, i32, vp, i64, vp, vp]
         L.xg_apply_token_bitmask.argtypes = [vp, C.c_int, i32, i32, i64, vp, i64, vp, i32, vp]
@@ -250,6 +256,11 @@ class Matcher:
 
     def reset(self, stream: int = 0):
         _check(lib().xg_matcher_reset(self.h, stream))
+
+    def next_fill_work(self, stream: int = 0) -> dict:
+        w = FillWork()
+        _check(lib().xg_matcher_next_fill_work(self.h, stream, C.byref(w)))
+        return {n: getattr(w, n) for n, _ in FillWork._fields_ if n != "pad"}
 
     def is_terminated(self, stream: int = 0) -> bool:
         out = C.c_int32(0)

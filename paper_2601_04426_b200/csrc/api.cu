@@ -1214,6 +1214,33 @@ xg_status_t xg_matcher_is_terminated(const xg_matcher_t* m, void* stream, int32_
   return XG_OK;
 }
 
+xg_status_t xg_matcher_next_fill_work(const xg_matcher_t* m, void* stream, xg_fill_work_t* out) {
+  if (!m || !out) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
+  const xg_grammar* g = m->grammar;
+  MatcherDev h;
+  XG_CUDA(cudaMemcpyAsync(&h, m->dev, sizeof h, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+  XG_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  std::unique_ptr<StepPlan> plan(new StepPlan());
+  XG_CUDA(cudaMemcpyAsync(plan.get(), h.plan, sizeof(StepPlan), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+  XG_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  xg_fill_work_t w{};
+  const int64_t W = g->tok->n_words;
+  w.row_bytes = 4 * W;
+  if (!h.terminated && !plan->overflow) {
+    w.n_merge = plan->n_merge; w.n_check = plan->n_check; w.n_missing = plan->n_missing;
+    for (int k = 0; k < plan->n_merge; ++k) {
+      const EntryDev& e = g->entries[plan->merge_state[k]];
+      if (e.kind == XG_STORE_BITSET) w.merge_bytes += 4 * W;
+      else if (e.kind == XG_STORE_ACCEPT_LIST) w.merge_bytes += 4LL * e.n_list;
+      else if (e.kind == XG_STORE_REJECT_LIST) w.merge_bytes += 4LL * e.n_list + 4LL * e.n_unc;
+    }
+    w.check_tokens = plan->n_check ? plan->check_cum[plan->n_check] : 0;
+    w.check_bytes = 5 * w.check_tokens;
+  }
+  *out = w;
+  return XG_OK;
+}
+
 // device-side array of matcher pointers for this exact batch (built once, then reused)
 static xg_status_t batch_slot(xg_matcher_t* const* matchers, int32_t batch, const xg_tokenizer** tok_out, BatchSlot** slot_out) {
   if (!matchers || batch <= 0) return set_error(XG_ERR_INVALID_ARG, "empty batch");

@@ -501,3 +501,21 @@ def test_threaded_compile_into_one_pool_builds_the_same_cache():
     for ga, gb in zip(a.grammars, b.grammars):
         _same_entries(ga, gb, stride=37)
     a.close(); b.close()
+
+
+def test_next_fill_work_counts_the_plan():
+    """The measurement call: merged entries, uncertain candidates and the row of the next fill."""
+    torch, engine = _engine()
+    w = inputs.make_workload("C5", batch=2, steps=12, vocab_size=8192)
+    s = engine.Session(w)
+    for step in range(12):
+        fw = s.matchers[0].next_fill_work(s.stream())
+        assert fw["row_bytes"] == 4 * s.W and fw["n_missing"] == 0
+        assert fw["n_merge"] >= 1 and fw["merge_bytes"] > 0
+        assert fw["check_bytes"] == 5 * fw["check_tokens"] and fw["n_check"] <= fw["n_merge"] * 2 + 2
+        s.fill()
+        s.accept([w.trajectories[b][step] for b in range(s.n)])
+        for b in range(s.n):
+            if w.trajectories[b][step] == w.vocab.eos_id:
+                s.reset(b)
+    s.close()
