@@ -741,10 +741,36 @@ accept_kernel(MatcherDev* const* __restrict__ matchers, int batch, VocabDev v,
 // into it (bitsets streamed with coalesced loads, sorted lists cut to the slice by binary
 // search) and writes the slice once.
 // ------------------------------------------------------------------------------------------
+// First index whose element is >= key, in a sorted list.  Called by whole warps with the same
+// arguments: 32 probes per round, so a list of a few thousand ids takes three rounds of
+// independent loads where a binary search would chain a dozen dependent ones.
 __device__ __forceinline__ int lower_bound_u32(const uint32_t* __restrict__ a, int n, uint32_t key) {
-  int lo = 0, hi = n;
-  while (lo < hi) { int mid = (lo + hi) >> 1; if (a[mid] < key) lo = mid + 1; else hi = mid; }
+  const int lane = threadIdx.x & 31;
+  int lo = 0, hi = n;                       // the answer lies in [lo, hi]
+  while (lo < hi) {
+    const int step = (hi - lo + 31) >> 5;
+    const int pos = lo + (lane + 1) * step - 1;                      // ascending with the lane
+    const bool less = pos < hi && a[pos] < key;
+    const int below = __popc(__ballot_sync(0xFFFFFFFFu, less));      // the probes below the key are the first `below` lanes
+    const int first_not_less = lo + (below + 1) * step - 1;          // the probe of lane `below`, if it exists
+    lo += below * step;
+    hi = first_not_less < hi ? first_not_less : hi;
+  }
   return lo;
+}
+
+// Visit the ids of a sorted list that fall into [id_lo, id_hi), all threads of the block together.  A short list
+// is simply read in full by every block of the cluster (one round of independent loads, no search at all); a
+// long one is cut to the slice first.
+constexpr int kScanWholeList = 1024;
+template <typename F>
+__device__ __forceinline__ void for_ids_in_slice(const uint32_t* __restrict__ list, int n, uint32_t id_lo, uint32_t id_hi, F visit) {
+  if (n <= kScanWholeList) {
+    for (int i = threadIdx.x; i < n; i += blockDim.x) { const uint32_t id = list[i]; if (id >= id_lo && id < id_hi) visit(id); }
+  } else {
+    const int lo = lower_bound_u32(list, n, id_lo), hi = lo + lower_bound_u32(list + lo, n - lo, id_hi);
+    for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) visit(list[i]);
+  }
 }
 
 // Just-in-time grammars (Section 3.5): while an entry of the current set is not built, the mask
@@ -1055,16 +1081,13 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
       if (e.kind == 2) {
         for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] |= e.data[w0 + w];
       } else if (e.kind == 0) {
-        const int lo = lower_bound_u32(e.data, e.n_list, id_lo), hi = lower_bound_u32(e.data, e.n_list, id_hi);
-        for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) { const uint32_t id = e.data[i]; atomicOr(&row[(id >> 5) - w0], 1u << (id & 31)); }
+        for_ids_in_slice(e.data, e.n_list, id_lo, id_hi, [&](uint32_t id) { atomicOr(&row[(id >> 5) - w0], 1u << (id & 31)); });
       } else {
         const uint32_t tail = (v.vocab_size & 31) ? ((1u << (v.vocab_size & 31)) - 1) : 0xFFFFFFFFu;
         for (int w = threadIdx.x; w < nw; w += blockDim.x) tmp[w] = (w0 + w == v.n_words - 1) ? tail : 0xFFFFFFFFu;
         __syncthreads();
-        int lo = lower_bound_u32(e.data, e.n_list, id_lo), hi = lower_bound_u32(e.data, e.n_list, id_hi);
-        for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) { const uint32_t id = e.data[i]; atomicAnd(&tmp[(id >> 5) - w0], ~(1u << (id & 31))); }
-        lo = lower_bound_u32(e.unc_id, e.n_unc, id_lo); hi = lower_bound_u32(e.unc_id, e.n_unc, id_hi);
-        for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) { const uint32_t id = e.unc_id[i]; atomicAnd(&tmp[(id >> 5) - w0], ~(1u << (id & 31))); }
+        for_ids_in_slice(e.data, e.n_list, id_lo, id_hi, [&](uint32_t id) { atomicAnd(&tmp[(id >> 5) - w0], ~(1u << (id & 31))); });
+        for_ids_in_slice(e.unc_id, e.n_unc, id_lo, id_hi, [&](uint32_t id) { atomicAnd(&tmp[(id >> 5) - w0], ~(1u << (id & 31))); });
         __syncthreads();
         for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] |= tmp[w];
       }
