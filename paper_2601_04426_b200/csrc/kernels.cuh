@@ -83,10 +83,17 @@ __device__ __forceinline__ bool advance_waiters(const GrammarDev& g, const Chart
     const int32_t o2 = src_org[i];
     const uint4 rec = *reinterpret_cast<const uint4*>(&g.state[s2]);
     const int wait_end = (int)rec.z + (int)(rec.w & 0xFFFFu);
-    for (int w = (int)rec.z; w < wait_end; ++w) {
-      const uint2 we = g.wait_edge[w];
-      if (we.x != rule) continue;
-      if (!add_item(st, org, start, cnt, cap, we.y & ~kSelf, (we.y & kSelf) ? o : o2)) return false;
+    // four edges at a time: their loads are issued together, then compared (one at a time, each load would be
+    // waited for before the next is even issued)
+    for (int w = (int)rec.z; w < wait_end; w += 4) {
+      uint2 we[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) we[u] = w + u < wait_end ? g.wait_edge[w + u] : make_uint2(0xFFFFFFFFu, 0u);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (we[u].x != rule) continue;
+        if (!add_item(st, org, start, cnt, cap, we[u].y & ~kSelf, (we[u].y & kSelf) ? o : o2)) return false;
+      }
     }
   }
   return true;
@@ -115,12 +122,18 @@ __device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* c
       const int n_edges = (k == 0 && own_edges_first) ? (int)(ra.y & 0xFFFFu) : (int)(ra.y >> 16);
       if (n_edges == 0) continue;
       const uint4 rb = *(reinterpret_cast<const uint4*>(&g.state[s]) + 1);
-      uint2 se = make_uint2(rb.z, rb.w);                      // the first edge is inline
-      for (int e = 0;;) {
-        const bool hit = (se.x & kLiteral) ? ((se.x & 0xFFu) == byte) : ((class_bits[se.x * 8 + word] & bit) != 0);
-        if (hit && !add_item(st, org, start, cnt, cap, se.y & ~kSelf, (se.y & kSelf) ? self_idx : o)) { *flags |= kWalkOverflow; return k; }
-        if (++e >= n_edges) break;
-        se = g.scan_edge[(int)ra.x + e];
+      // the first edge is inline in the record; the others are fetched four at a time (loads issued together, then tested)
+      for (int e = 0; e < n_edges; e += 4) {
+        uint2 se[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          se[u] = (e + u == 0) ? make_uint2(rb.z, rb.w) : (e + u < n_edges ? g.scan_edge[(int)ra.x + e + u] : make_uint2(kLiteral | 0x100u, 0u));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (e + u >= n_edges) break;
+          const bool hit = (se[u].x & kLiteral) ? ((se[u].x & 0x1FFu) == byte) : ((class_bits[se[u].x * 8 + word] & bit) != 0);
+          if (hit && !add_item(st, org, start, cnt, cap, se[u].y & ~kSelf, (se[u].y & kSelf) ? self_idx : o)) { *flags |= kWalkOverflow; return k; }
+        }
       }
     }
     if (cnt == start) return k;
