@@ -31,7 +31,7 @@ from paper_2601_04426_b200 import inputs  # noqa: E402
 
 SHAPES = {"C1": (1, 8192), "C2": (1, 128256), "C3": (128, 151936), "C4": (64, 128256), "C5": (256, 200064),
           "T5": (16, 128256), "T20": (16, 128256), "T50": (16, 128256), "T100": (16, 128256),
-          "H16": (32, 128256), "H64": (32, 128256), "R256": (16, 128256), "R1024": (16, 128256), "R4096": (16, 128256)}
+          "H16": (32, 128256), "H64": (32, 128256), "P10": (8, 128256), "P100": (8, 128256), "P500": (8, 128256), "R256": (16, 128256), "R1024": (16, 128256), "R4096": (16, 128256)}
 
 
 def measured_peaks():

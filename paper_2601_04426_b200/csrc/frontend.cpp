@@ -410,7 +410,10 @@ struct AhoCorasick {
   }
 };
 
+constexpr int kKeepDispatchedRules = 8;
+
 struct Builder {
+  std::set<int> keep_as_rule;             // rules that inlining leaves alone
   std::vector<std::string> names;
   std::map<std::string, int> ids;
   std::vector<Fsm> rules;
@@ -487,6 +490,10 @@ struct Builder {
     int exit = f.add();
     std::vector<int> dispatch(n_tags, -1);       // state holding the reference edge of tag j
     for (int j = 0; j < n_tags; ++j) { dispatch[j] = f.add(); f.ref(dispatch[j], lookup(spec.tag_rules[j]), node_state[0]); }
+    // A dispatch over many tags is a menu of independent structures (one tool each): their rules are kept as
+    // rules, so that requests which offer different subsets of a tool pool still share the cache entries of the
+    // tools they have in common (Section 3.3; inlined into the dispatching automaton they would be unique to it).
+    if (n_tags >= kKeepDispatchedRules) for (int j = 0; j < n_tags; ++j) keep_as_rule.insert(lookup(spec.tag_rules[j]));
     for (int u = 0; u < n_nodes; ++u) {
       if (node_state[u] < 0) continue;
       std::map<int, ByteSet> by_target;          // target state -> bytes
@@ -989,7 +996,7 @@ struct Compiler {
         g.out[s] = keep;
       }
       if (changed) { b.rules[r] = normalize(g, opt.max_rule_states); renormalized[r] = 1; }
-      candidate[r] = !rec[r] && r != root && b.rules[r].size() <= single_use_max;
+      candidate[r] = !rec[r] && r != root && b.rules[r].size() <= single_use_max && !b.keep_as_rule.count(r);
     };
     for (int r = 0; r < R; ++r) process(r);
   }

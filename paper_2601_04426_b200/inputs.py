@@ -514,6 +514,16 @@ def sample_channel_text(rng: Rng, tools: List[dict], n_messages: int) -> str:
     return "".join(out)
 
 
+_tool_pool_cache: List[dict] = []
+
+
+def _tool_pool() -> List[dict]:
+    """The seeded pool of 1 908 tools (the size of the tool pool in Section 4.1) with distinct names."""
+    if not _tool_pool_cache:
+        _tool_pool_cache.extend(make_function_tags(Rng(BASE_SEED * 10 + 300000), 1908, tag_len=24))
+    return _tool_pool_cache
+
+
 def make_function_tags(rng: Rng, n_tags: int, tag_len: int = 20) -> List[dict]:
     """`n_tags` tools whose tags share the prefix `<function=` and are `tag_len` bytes long in total
     (the shape of the paper's tag-count experiment, Section 4.1), each with a small argument schema."""
@@ -595,6 +605,11 @@ _SHAPES = {
     # channelised response protocol with 16 / 64 tools (text channels with stop strings, one tool channel per tool)
     "H16": (128256,  16,  4.0, 0.3,    0.0,  32,   256,  "bf16"),
     "H64": (128256,  16,  4.0, 0.3,    0.0,  32,   256,  "bf16"),
+    # inter-request dynamism (Section 4.1): every request draws its own subset of 10 / 100 / 500 tools from one pool of
+    # 1 908 tools, one `<function=NAME>` tag per tool; what the requests share are the tools' argument grammars
+    "P10": (128256,  16,  4.0, 0.3,    0.0,  8,    64,   "bf16"),
+    "P100": (128256, 16,  4.0, 0.3,    0.0,  8,    64,   "bf16"),
+    "P500": (128256, 16,  4.0, 0.3,    0.0,  8,    64,   "bf16"),
     # long bounded repetitions (Section 3.6: minLength / maxLength / minItems / maxItems in the hundreds to thousands)
     "R256": (128256,  16,  4.0, 0.3,    0.0,  16,   256,  "bf16"),
     "R1024": (128256, 16,  4.0, 0.3,    0.0,  16,   256,  "bf16"),
@@ -607,7 +622,7 @@ _vocab_cache: Dict[Tuple, Vocab] = {}
 def config_seed(name: str) -> int:
     if name[0] == "C":
         return BASE_SEED * 10 + int(name[1])
-    return BASE_SEED * 10 + {"T": 1000, "R": 100000, "H": 200000}[name[0]] + int(name[1:])
+    return BASE_SEED * 10 + {"T": 1000, "R": 100000, "H": 200000, "P": 300000}[name[0]] + int(name[1:])
 
 
 def config_vocab(name: str, vocab_size: Optional[int] = None) -> Vocab:
@@ -615,7 +630,7 @@ def config_vocab(name: str, vocab_size: Optional[int] = None) -> Vocab:
     if vocab_size is not None:
         V = vocab_size
     # C2 and C4 share one Llama-3-sized vocabulary
-    seed_name = "C2" if (name == "C4" or name[0] in "TRH") else name
+    seed_name = "C2" if (name == "C4" or name[0] in "TRHP") else name
     key = (seed_name, V)
     if key not in _vocab_cache:
         _vocab_cache[key] = make_vocab(config_seed(seed_name) ^ 0x5EED, V, lmax, mean, lead, utf8)
@@ -714,6 +729,21 @@ def make_workload(name: str, batch: Optional[int] = None, steps: Optional[int] =
             rr = rng.fork(100 + b)
             t, d = _trajectory(tok, vocab.eos_id, S, lambda: sample_function_text(rr, tools, rr.randint(1, 3), 40).encode())
             request_grammar.append(0); trajs.append(t); docs_all.append(d)
+    elif name[0] == "P":
+        pool_tools = _tool_pool()
+        k = int(name[1:])
+        for b in range(B):
+            sr = rng.fork(50 + b)
+            picked = sorted({sr.below(len(pool_tools)) for _ in range(4 * k)})
+            sr2 = rng.fork(70 + b)
+            while len(picked) > k:
+                picked.pop(sr2.below(len(picked)))
+            tools = [pool_tools[i] for i in picked]
+            grammars.append(GrammarSpec("tag_dispatch", json.dumps(function_tags_spec(tools))))
+            rr = rng.fork(100 + b)
+            t, d = _trajectory(tok, vocab.eos_id, S, lambda: sample_function_text(rr, tools, rr.randint(1, 3), 30).encode())
+            request_grammar.append(b); trajs.append(t); docs_all.append(d)
+        meta["pool_size"] = len(pool_tools)
     elif name[0] == "H":
         tools = make_tool_set(rng.fork(3), int(name[1:]))
         grammars.append(GrammarSpec("tag_dispatch", json.dumps(channel_spec(tools))))

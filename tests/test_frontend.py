@@ -92,7 +92,7 @@ def _mutate(rng, doc, alphabet):
     return doc[:pos] + b + doc[pos + 1:] if kind == 0 else (doc[:pos] + doc[pos + 1:] if kind == 1 else doc[:pos] + b + doc[pos:])
 
 
-@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4", "C5", "T20", "H16", "R256"])
+@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4", "C5", "T20", "H16", "R256", "P10"])
 def test_workload_grammars_same_language_as_oracle(name):
     w = inputs.make_workload(name, batch=3, steps=40)
     rng = inputs.Rng(17)

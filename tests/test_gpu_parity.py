@@ -519,3 +519,18 @@ def test_next_fill_work_counts_the_plan():
             if w.trajectories[b][step] == w.vocab.eos_id:
                 s.reset(b)
     s.close()
+
+
+def test_tool_pool_requests_share_the_tools_they_have_in_common():
+    """Inter-request dynamism (Section 4.1): every request offers its own subset of one tool pool.  The masks are
+    exact, and requests compiled later find the entries of the tools that earlier requests already offered."""
+    torch, engine = _engine()
+    w = inputs.make_workload("P100", batch=6, steps=40, vocab_size=8192)
+    names = [set(t["tag"] for t in json.loads(g.text)["tags"]) for g in w.grammars]
+    assert all(len(n) == 100 for n in names) and len(set.union(*names)) > 300 and any(names[0] & n for n in names[1:])
+    _run_trajectories(w, {0, 13, 39}, check_requests={2})
+    s = engine.Session(w, compile_threads=1)
+    stats = [g.stats() for g in s.grammars]
+    assert stats[0]["n_entries_reused"] < stats[-1]["n_entries_reused"]          # the pool fills up as requests arrive
+    assert sum(x["n_entries_reused"] for x in stats[1:]) > 0
+    s.close()
