@@ -1237,13 +1237,14 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
 template <int ELEMS>
 __device__ __forceinline__ uint4 blend_ninf(uint4 x, uint32_t bits) {
   if (ELEMS == 8) {
-    uint32_t p[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      if (!((bits >> (2 * k)) & 1u)) p[k] = (p[k] & 0xFFFF0000u) | 0xFF80u;
-      if (!((bits >> (2 * k + 1)) & 1u)) p[k] = (p[k] & 0x0000FFFFu) | 0xFF800000u;
-    }
-    return make_uint4(p[0], p[1], p[2], p[3]);
+    // four allowed-bits -> four bytes of 0x00 / 0xFF (a multiply spreads the bits to the bytes' low bits, a second
+    // one fills the bytes), then each byte is doubled into the 16-bit lane it stands for
+    const uint32_t lo = (((bits & 0xFu) * 0x00204081u) & 0x01010101u) * 0xFFu;
+    const uint32_t hi = ((((bits >> 4) & 0xFu) * 0x00204081u) & 0x01010101u) * 0xFFu;
+    const uint32_t k0 = __byte_perm(lo, 0u, 0x1100), k1 = __byte_perm(lo, 0u, 0x3322);
+    const uint32_t k2 = __byte_perm(hi, 0u, 0x1100), k3 = __byte_perm(hi, 0u, 0x3322);
+    constexpr uint32_t kNinf2 = 0xFF80FF80u;
+    return make_uint4((x.x & k0) | (kNinf2 & ~k0), (x.y & k1) | (kNinf2 & ~k1), (x.z & k2) | (kNinf2 & ~k2), (x.w & k3) | (kNinf2 & ~k3));
   }
   if (!(bits & 1u)) x.x = 0xFF800000u;
   if (!(bits & 2u)) x.y = 0xFF800000u;
