@@ -354,7 +354,7 @@ def main():
     dominant = max((("fill", t_fill), ("apply", t_apply), ("accept", t_accept)), key=lambda x: x[1])[0]
     # bytes per launch by ncu (profiles/step_kernels_c3.txt): DRAM reads + bytes written towards L2, which the logits ring
     # turns into DRAM write-backs; measured on C3 only, and void once apply_kernel changes
-    traffic = 46.0e6 if (args.workload == "C3" and n == 128) else None
+    traffic = 50.6e6 if (args.workload == "C3" and n == 128) else None
     roofline = {"kernel": "apply_kernel", "bound": "hbm", "achieved": apply_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": apply_gbs / peak, "traffic": traffic, "us_per_launch": t_apply, "masked_fraction": masked_frac,
                 "conventional_gbs": apply_conv_bytes / (t_apply * 1e-6) / 1e9, "dominant_by_time": dominant,
@@ -368,7 +368,7 @@ def main():
     # the kernels change) over the launch time, against 148 SMs x 4 schedulers x the SM clock.
     props = torch.cuda.get_device_properties(local_rank)
     issue_peak = props.multi_processor_count * 4 * (clocks["sm_max_mhz"] or 1965.0) * 1e6
-    warp_insts = {"fill": 1665453.0, "accept": 104371.0} if (args.workload == "C3" and n == 128) else {}
+    warp_insts = {"fill": 1431770.0, "accept": 117728.0} if (args.workload == "C3" and n == 128) else {}
     latency_bound = {}
     for name, t_us in (("fill", t_fill), ("accept", t_accept)):
         wi = warp_insts.get(name)
