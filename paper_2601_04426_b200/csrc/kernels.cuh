@@ -1281,11 +1281,11 @@ apply_kernel(void* __restrict__ logits, int vocab_size, long long row_stride_ele
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u)
-      if (bits[u] != kAll && bits[u] != 0) x[u] = base[v0 + u * stride];
+      if (bits[u] != kAll && bits[u] != 0) x[u] = __ldcs(&base[v0 + u * stride]);
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       if (bits[u] == kAll) continue;
-      base[v0 + u * stride] = bits[u] == 0 ? ninf : blend_ninf<ELEMS>(x[u], bits[u]);
+      __stcs(&base[v0 + u * stride], bits[u] == 0 ? ninf : blend_ninf<ELEMS>(x[u], bits[u]));
     }
   }
   // ragged tail (vocab_size not a multiple of the vector width)
