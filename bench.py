@@ -154,6 +154,8 @@ def main():
     ap.add_argument("--workload", default="C3", choices=sorted(SHAPES))
     ap.add_argument("--batch", type=int, default=None, help="shrink the batch (debugging only; the line then names it)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fused-accept-fill", action="store_true",
+                    help="step = apply, then accept and the next mask's fill in one launch, instead of fill, apply, accept as three launches")
     ap.add_argument("--jit-sweep", default=None,
                     help="comma-separated K values (or 'full'): compile just in time with K entries precomputed and report "
                          "compile time and per-step time avg / P99 / max over the trajectory (the shape of the paper's K sweep)")
@@ -221,28 +223,39 @@ def main():
     base = engine.logits_tensor(inputs.make_logits(w.logits_seed, min(n, 8), s.V, w.dtype), s.device)
     ring = [base.repeat((n + base.shape[0] - 1) // base.shape[0], 1)[:n].contiguous() for _ in range(ring_n)]
     traj = torch.from_numpy(np.asarray([[w.trajectories[b][t] for b in range(n)] for t in range(w.steps)], dtype=np.int32)).to(s.device)      # [steps, n]
-    eos_at = {t: [b for b in range(n) if w.trajectories[b][t] == w.vocab.eos_id] for t in range(w.steps)}
     total = warmup + args.steps
-    launches = {"accept": 0, "fill": 0, "apply": 0, "reset": 0}      # this library's kernels only
+    launches = {"accept": 0, "fill": 0, "apply": 0, "reset": 0, "accept_fill": 0}      # this library's kernels only
+    fused = args.fused_accept_fill
 
-    def restart():
+    def restart(first_mask=False):
         for b in range(n):
             s.reset(b)
+        launches["reset"] += n
+        if first_mask:
+            s.fill()
+            launches["fill"] += 1
 
-    # The decode loop is launch-bound (three short kernels per step), so the timed loop replays
-    # CUDA graphs, as a serving engine's decode loop does: one graph per trajectory step holding
-    # fill + apply + accept, with the step's token ids read straight from the resident trajectory
-    # table and the logits buffer taken from the ring.
+    # The decode loop is launch-bound (short kernels), so the timed loop replays CUDA graphs, as a
+    # serving engine's decode loop does: one graph per trajectory step, with the step's token ids
+    # read straight from the resident trajectory table and the logits buffer taken from the ring.
+    # A step fills the mask, masks the logits and accepts the step's token: three launches.  A
+    # request that accepts end of sequence starts its next document in the accept launch.
+    # (--fused-accept-fill: apply, then accept and the next mask's fill in one launch.)  Either
+    # way every step runs accept, fill and apply once for every request.
 
     def step_body(buf, t):
-        s.fill()
-        s.apply(buf)
-        s.accept_device(traj[t])
+        if fused:
+            s.apply(buf)
+            s.accept_fill_device(traj[t], restart_on_eos=True)
+        else:
+            s.fill()
+            s.apply(buf)
+            s.accept_device(traj[t], restart_on_eos=True)
 
     for k in range(ring_n):              # eager warm-up of every call before capture (first-use set-up)
         step_body(ring[k], 0)
     torch.cuda.synchronize()
-    restart()
+    restart(fused)
     graphs = []
     for t in range(w.steps):
         gph = torch.cuda.CUDAGraph()
@@ -250,17 +263,18 @@ def main():
             step_body(ring[t % ring_n], t)
         graphs.append(gph)
     torch.cuda.synchronize()
-    restart()
+    restart(fused)
 
     def one_step(i):
         t = i % w.steps
         if t == 0 and i > 0:
-            restart()
+            restart(fused)
         graphs[t].replay()
-        for b in eos_at[t]:
-            s.reset(b)
-            launches["reset"] += 1
-        launches["fill"] += 1; launches["apply"] += 1; launches["accept"] += 1
+        launches["apply"] += 1
+        if fused:
+            launches["accept_fill"] += 1
+        else:
+            launches["fill"] += 1; launches["accept"] += 1
 
     # ---- pass A: the headline number (events only around the timed region) --------------------
     for i in range(warmup):
@@ -306,11 +320,9 @@ def main():
         s.apply(buf)
         if ev:
             ev[2].record()
-        s.accept_device(traj[t])
+        s.accept_device(traj[t], restart_on_eos=True)
         if ev:
             ev[3].record()
-        for b in eos_at[t]:
-            s.reset(b)
         if ev and (i - warmup) % 10 == 0:            # masked fraction, sampled (synchronises; outside the event intervals)
             zero_bits_sum += n * s.V - int(np.unpackbits(s.mask_numpy().view(np.uint8)).sum())
             mask_samples += 1
@@ -324,6 +336,24 @@ def main():
     eager_us = {"fill": float(np.mean([e[0].elapsed_time(e[1]) for e in evs])) * 1e3,
                 "apply": float(np.mean([e[1].elapsed_time(e[2]) for e in evs])) * 1e3,
                 "accept": float(np.mean([e[2].elapsed_time(e[3]) for e in evs])) * 1e3}
+
+    # the one-launch accept-and-fill, timed the same way (apply in front of it, as in the step)
+    restart(True)
+    evf = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+    for i in range(total):
+        t = i % w.steps
+        if t == 0 and i > 0:
+            restart(True)
+        ev = evf[i - warmup] if i >= warmup else None
+        torch.cuda._sleep(spin_cycles)
+        s.apply(ring[i % ring_n])
+        if ev:
+            ev[0].record()
+        s.accept_fill_device(traj[t], restart_on_eos=True)
+        if ev:
+            ev[1].record()
+    torch.cuda.synchronize()
+    eager_us["accept_fill"] = float(np.mean([e[0].elapsed_time(e[1]) for e in evf])) * 1e3
 
     # ---- apply alone: launches back to back over the logits ring (the last step's mask) ---------
     # The intervals above hold the launch gap of a short kernel; a stream of launches does not.
@@ -400,7 +430,7 @@ def main():
     torch.cuda.synchronize()
     h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for phase in ("warm", "timed"):
-        restart()
+        restart(fused)
         torch.cuda.synchronize()
         if phase == "timed":
             h0.record()
@@ -424,7 +454,8 @@ def main():
             k = t % 2
             if t + 1 < e2e_steps:
                 upload(t + 1)
-            s.fill()
+            if not fused:
+                s.fill()
             main.wait_event(ev_in[k])
             s.apply(dev_buf[k])
             ev_applied[k] = torch.cuda.Event()
@@ -435,9 +466,10 @@ def main():
                 ev_out[k] = torch.cuda.Event()
                 ev_out[k].record(s_out)
             s.tokens.copy_(host_traj[t], non_blocking=True)
-            s.accept_device(s.tokens)
-            for b in eos_at[t]:
-                s.reset(b)
+            if fused:
+                s.accept_fill_device(s.tokens, restart_on_eos=True)
+            else:
+                s.accept_device(s.tokens, restart_on_eos=True)
         main.wait_event(ev_out[0])
         main.wait_event(ev_out[1])
         if phase == "timed":
@@ -449,11 +481,11 @@ def main():
         "metric": metric, "value": us_per_step, "unit": "us/step", "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": us_per_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "int32", "data": "synthetic",
-        "config": {"workload": args.workload, "batch": n, "global_batch": n * world, "vocab": s.V, "logits_dtype": w.dtype, "launch": "one CUDA graph per trajectory step (fill, apply, accept)",
+        "config": {"workload": args.workload, "batch": n, "global_batch": n * world, "vocab": s.V, "logits_dtype": w.dtype, "launch": "one CUDA graph per trajectory step: " + ("apply, then accept + fill of the next mask in one launch" if fused else "fill, apply, accept"),
                    "grammars": len(w.grammars), "l2": "logits ring of %d buffers (%.0f MB) > 2 x L2" % (ring_n, ring_n * bytes_one / 1e6),
                    "parallelism": "replicas x%d" % world},
         "clocks": clocks,
-        "kernels_us": {"fill": t_fill, "apply": t_apply, "accept": t_accept},
+        "kernels_us": {"fill": t_fill, "apply": t_apply, "accept": t_accept, "accept_fill": eager_us["accept_fill"]},
         "apply_gbs": apply_gbs,
         "cache_build": {"seconds": build_ms / 1e3, "compile_wall_s": compile_s, "compile_threads": args.compile_threads or min(16, os.cpu_count() or 1), "pairs_classified": pairs, "pairs_per_s": pairs / max(build_ms / 1e3, 1e-9),
                         "pairs_dense": pairs_dense, "pairs_dense_per_s": pairs_dense / max(build_ms / 1e3, 1e-9),

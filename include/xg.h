@@ -315,6 +315,32 @@ xg_status_t xg_apply_token_bitmask(void* logits_dev, xg_dtype_t dtype, int32_t b
 xg_status_t xg_accept_token(xg_matcher_t* const* matchers, int32_t batch, const int32_t* token_ids_dev,
                             int32_t* status_dev, void* stream);
 
+/* xg_accept_token_ex: xg_accept_token with one option.  restart_on_eos != 0: a request that
+ * accepts the end-of-sequence token is put back into its initial state in the same launch (what
+ * xg_matcher_reset would do in a launch of its own) instead of terminating -- for slots that
+ * begin the next document of the same grammar at once.  restart_on_eos == 0 is xg_accept_token. */
+xg_status_t xg_accept_token_ex(xg_matcher_t* const* matchers, int32_t batch, const int32_t* token_ids_dev,
+                               int32_t* status_dev, int32_t restart_on_eos, void* stream);
+
+/* xg_accept_token_and_fill_next_bitmask: xg_accept_token followed by xg_fill_next_token_bitmask
+ * on the same batch, in one launch (Section 2.2: after a token is sampled the engine traces it
+ * and generates the next step's mask; the two steps always follow each other in a decode loop).
+ * The result is the one the two calls give in that order: accept_status_dev (device, [batch],
+ * may be NULL) receives what xg_accept_token would report; a request whose token was rejected
+ * keeps its state, and its mask row is the mask of that unchanged state; a request that
+ * terminated gets an all-zero row and XG_ERR_TERMINATED in fill_status_dev (device, [batch], may
+ * be NULL).  restart_on_eos != 0: a request that accepts the end-of-sequence token is put back
+ * into its initial state (as by xg_matcher_reset) instead of terminating, and its row is the
+ * mask of the grammar's start -- for slots that begin the next document of the same grammar at
+ * once.  Where the vocabulary is too large for the one-launch fill the call enqueues the two
+ * steps one after the other.  Other arguments, layout and errors: as in the two calls it
+ * replaces. */
+xg_status_t xg_accept_token_and_fill_next_bitmask(xg_matcher_t* const* matchers, int32_t batch,
+                                                  const int32_t* token_ids_dev, int32_t* accept_status_dev,
+                                                  int32_t restart_on_eos, int32_t* bitmask_dev,
+                                                  int64_t row_stride_words, int32_t* fill_status_dev,
+                                                  void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -29,6 +29,7 @@ EXPORTS = [
     "xg_compile_grammar", "xg_grammar_destroy", "xg_grammar_get_tables", "xg_grammar_get_rule_hashes", "xg_grammar_get_cache_entry", "xg_grammar_get_state_classes", "xg_grammar_stats", "xg_jit_service",
     "xg_matcher_create", "xg_matcher_reset", "xg_matcher_destroy", "xg_matcher_is_terminated", "xg_matcher_next_fill_work",
     "xg_fill_next_token_bitmask", "xg_fill_next_token_bitmask_static", "xg_apply_token_bitmask", "xg_accept_token",
+    "xg_accept_token_ex", "xg_accept_token_and_fill_next_bitmask",
 ]
 XG_STATIC_FILL_MAX_BATCH = 1024
 
@@ -121,6 +122,8 @@ def lib():
         L.xg_fill_next_token_bitmask_static.argtypes = [vp, i32, vp, i64, vp, vp]
         L.xg_apply_token_bitmask.argtypes = [vp, C.c_int, i32, i32, i64, vp, i64, vp, i32, vp]
         L.xg_accept_token.argtypes = [vp, i32, vp, vp, vp]
+        L.xg_accept_token_ex.argtypes = [vp, i32, vp, vp, i32, vp]
+        L.xg_accept_token_and_fill_next_bitmask.argtypes = [vp, i32, vp, vp, i32, vp, i64, vp, vp]
         _lib = L
     return _lib
 
@@ -289,8 +292,16 @@ class Batch:
         XG_STATIC_FILL_MAX_BATCH requests; calls must not overlap on the GPU)."""
         _check(lib().xg_fill_next_token_bitmask_static(self.handles, self.n, bitmask_ptr, row_stride_words, status_ptr or None, stream))
 
-    def accept_token(self, token_ids_ptr: int, status_ptr: int = 0, stream: int = 0):
-        _check(lib().xg_accept_token(self.handles, self.n, token_ids_ptr, status_ptr or None, stream))
+    def accept_token(self, token_ids_ptr: int, status_ptr: int = 0, stream: int = 0, restart_on_eos: bool = False):
+        if restart_on_eos:
+            _check(lib().xg_accept_token_ex(self.handles, self.n, token_ids_ptr, status_ptr or None, 1, stream))
+        else:
+            _check(lib().xg_accept_token(self.handles, self.n, token_ids_ptr, status_ptr or None, stream))
+
+    def accept_token_and_fill_next_bitmask(self, token_ids_ptr: int, accept_status_ptr: int, restart_on_eos: bool, bitmask_ptr: int,
+                                           row_stride_words: int, fill_status_ptr: int = 0, stream: int = 0):
+        _check(lib().xg_accept_token_and_fill_next_bitmask(self.handles, self.n, token_ids_ptr, accept_status_ptr or None, 1 if restart_on_eos else 0,
+                                                           bitmask_ptr, row_stride_words, fill_status_ptr or None, stream))
 
 
 def apply_token_bitmask(logits_ptr: int, dtype, batch: int, vocab_size: int, logits_row_stride: int, bitmask_ptr: int,

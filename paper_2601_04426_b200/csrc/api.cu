@@ -1278,9 +1278,9 @@ static xg_status_t batch_slot(xg_matcher_t* const* matchers, int32_t batch, cons
   return XG_OK;
 }
 
-xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t batch, int32_t* bitmask_dev, int64_t row_stride_words,
-                                       int32_t* status_dev, void* stream) {
-  NvtxRange nvtx_range("xg_fill_next_token_bitmask");
+// accept (when token_ids_dev is given) and fill; the two public entry points below are this
+static xg_status_t accept_and_fill(xg_matcher_t* const* matchers, int32_t batch, const int32_t* token_ids_dev, int32_t* accept_status_dev,
+                                   int restart_on_eos, int32_t* bitmask_dev, int64_t row_stride_words, int32_t* status_dev, void* stream) {
   const xg_tokenizer* tok = nullptr;
   BatchSlot* slot = nullptr;
   xg_status_t st = batch_slot(matchers, batch, &tok, &slot);
@@ -1296,10 +1296,20 @@ xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t ba
     const int per_request = sms * 1024 / batch;
     int blocks = kMaxClusterBlocks, threads = 256;
     if (per_request < 2048) threads = 128;     // measured: fewer blocks or narrower blocks than this are slower even at batch 256
-    XG_CUDA(launch_step_kernel(fill_cluster_kernel, dim3(blocks, batch), dim3(threads), 2 * sizeof(uint32_t) * (size_t)((W + blocks - 1) / blocks),
-                               (cudaStream_t)stream, blocks, (MatcherDev* const*)slot->dev_matchers, tok->dev, bitmask_dev,
-                               (long long)row_stride_words, status_dev));
+    const size_t smem = 2 * sizeof(uint32_t) * (size_t)((W + blocks - 1) / blocks);
+    if (token_ids_dev)
+      XG_CUDA(launch_step_kernel(fill_cluster_kernel<true>, dim3(blocks, batch), dim3(threads), smem, (cudaStream_t)stream, blocks,
+                                 (MatcherDev* const*)slot->dev_matchers, tok->dev, bitmask_dev, (long long)row_stride_words, status_dev,
+                                 token_ids_dev, accept_status_dev, restart_on_eos));
+    else
+      XG_CUDA(launch_step_kernel(fill_cluster_kernel<false>, dim3(blocks, batch), dim3(threads), smem, (cudaStream_t)stream, blocks,
+                                 (MatcherDev* const*)slot->dev_matchers, tok->dev, bitmask_dev, (long long)row_stride_words, status_dev,
+                                 (const int32_t*)nullptr, (int32_t*)nullptr, 0));
     return XG_OK;
+  }
+  if (token_ids_dev) {
+    XG_CUDA(launch_step_kernel(accept_kernel, dim3((batch + 3) / 4), dim3(128), 0, (cudaStream_t)stream, 1, (MatcherDev* const*)slot->dev_matchers,
+                               (int)batch, tok->dev, token_ids_dev, accept_status_dev, restart_on_eos));
   }
   int chunks = std::max((W + kMergeMaxChunkWords - 1) / kMergeMaxChunkWords, std::min(8, (W + 127) / 128));
   dim3 grid_merge(chunks, batch);
@@ -1310,6 +1320,20 @@ xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t ba
                                                              status_dev, slot->status, slot->done_count);
   XG_CUDA(cudaGetLastError());
   return XG_OK;
+}
+
+xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t batch, int32_t* bitmask_dev, int64_t row_stride_words,
+                                       int32_t* status_dev, void* stream) {
+  NvtxRange nvtx_range("xg_fill_next_token_bitmask");
+  return accept_and_fill(matchers, batch, nullptr, nullptr, 0, bitmask_dev, row_stride_words, status_dev, stream);
+}
+
+xg_status_t xg_accept_token_and_fill_next_bitmask(xg_matcher_t* const* matchers, int32_t batch, const int32_t* token_ids_dev,
+                                                  int32_t* accept_status_dev, int32_t restart_on_eos, int32_t* bitmask_dev,
+                                                  int64_t row_stride_words, int32_t* fill_status_dev, void* stream) {
+  NvtxRange nvtx_range("xg_accept_token_and_fill_next_bitmask");
+  if (!token_ids_dev) return set_error(XG_ERR_INVALID_ARG, "token_ids_dev is NULL");
+  return accept_and_fill(matchers, batch, token_ids_dev, accept_status_dev, restart_on_eos ? 1 : 0, bitmask_dev, row_stride_words, fill_status_dev, stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1373,6 +1397,11 @@ xg_status_t xg_fill_next_token_bitmask_static(xg_matcher_t* const* matchers, int
 }
 
 xg_status_t xg_accept_token(xg_matcher_t* const* matchers, int32_t batch, const int32_t* token_ids_dev, int32_t* status_dev, void* stream) {
+  return xg_accept_token_ex(matchers, batch, token_ids_dev, status_dev, 0, stream);
+}
+
+xg_status_t xg_accept_token_ex(xg_matcher_t* const* matchers, int32_t batch, const int32_t* token_ids_dev, int32_t* status_dev,
+                               int32_t restart_on_eos, void* stream) {
   NvtxRange nvtx_range("xg_accept_token");
   const xg_tokenizer* tok = nullptr;
   BatchSlot* slot = nullptr;
@@ -1380,7 +1409,7 @@ xg_status_t xg_accept_token(xg_matcher_t* const* matchers, int32_t batch, const 
   if (st != XG_OK) return st;
   if (!token_ids_dev) return set_error(XG_ERR_INVALID_ARG, "token_ids_dev is NULL");
   XG_CUDA(launch_step_kernel(accept_kernel, dim3((batch + 3) / 4), dim3(128), 0, (cudaStream_t)stream, 1, (MatcherDev* const*)slot->dev_matchers,
-                             (int)batch, tok->dev, token_ids_dev, status_dev));
+                             (int)batch, tok->dev, token_ids_dev, status_dev, restart_on_eos ? 1 : 0));
   return XG_OK;
 }
 

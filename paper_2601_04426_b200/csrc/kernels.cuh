@@ -663,87 +663,98 @@ __device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g,
   if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) p.overflow = 1;
 }
 
+// the matcher's initial state: one item, the root rule's start state at origin 0 (lane 0 writes)
+__device__ __forceinline__ void matcher_restart(MatcherDev& m, const GrammarDev& g) {
+  m.item_state[0] = (uint32_t)g.root_start;
+  m.item_origin[0] = 0;
+  m.set_begin[0] = 0;
+  m.set_begin[1] = 1;
+  m.n_sets = 1;
+  m.n_items = 1;
+  m.terminated = 0;
+}
+
 __global__ void matcher_reset_kernel(MatcherDev* m) {      // one warp
   if (blockIdx.x != 0 || threadIdx.x >= 32) return;
-  if (threadIdx.x == 0) {
-    m->item_state[0] = (uint32_t)m->grammar->root_start;
-    m->item_origin[0] = 0;
-    m->set_begin[0] = 0;
-    m->set_begin[1] = 1;
-    m->n_sets = 1;
-    m->n_items = 1;
-    m->terminated = 0;
-  }
+  if (threadIdx.x == 0) matcher_restart(*m, *m->grammar);
   __syncwarp();
   prepare_plan(*m, *m->grammar, threadIdx.x);
 }
 
-// Accept one sampled token per request (Section 2.2 "trace the output").  One warp per request:
-// requests follow unrelated paths, so sharing a warp between them would serialise their walks.
-// Lane 0 walks the token's bytes into local arrays; if every byte survived, the warp appends the
-// new sets behind the request's history and lane 0 commits the counters.
+// Accept one sampled token of one request (Section 2.2 "trace the output"), by one warp.  Lane 0
+// walks the token's bytes into the warp's scratch (w_st, w_org: kFastCap items, lsb: kFastMaxBytes
+// + 2); if every byte survived, the warp appends the new sets behind the request's history, lane
+// 0 commits the counters and the warp builds the plan of the next mask.  A rejected token leaves
+// the matcher as it was.  With restart_on_eos an accepted end-of-sequence token puts the matcher
+// back into its initial state instead of terminating it.  Returns the status, the same in every lane.
+__device__ __forceinline__ int accept_one(MatcherDev& m, const GrammarDev& g, const VocabDev& v, int tok, bool restart_on_eos, int lane,
+                                          uint32_t* w_st, int32_t* w_org, int16_t* lsb) {
+  int st = 0;   // XG_OK
+  if (m.terminated) return -8;
+  if (tok < 0 || tok >= v.vocab_size) return -7;
+  if (tok == v.eos_id) {
+    if (lane == 0) {
+      if (!root_complete(m, g)) st = -7;
+      else if (restart_on_eos) matcher_restart(m, g);
+      else m.terminated = 1;
+    }
+    st = __shfl_sync(0xFFFFFFFFu, st, 0);
+    if (st == 0 && restart_on_eos) { __syncwarp(); prepare_plan(m, g, lane); }
+    return st;
+  }
+  const int rank = v.id_to_rank[tok];
+  const uint32_t off = v.offset[rank];
+  const int len = (int)(v.offset[rank + 1] - off);
+  if (v.never[rank] || len == 0) return -7;
+  int n_sets = m.n_sets, n_items = m.n_items;
+  int done = 0;
+  while (done < len && st == 0) {            // long tokens go through in pieces
+    const int piece = min(len - done, kFastMaxBytes);
+    int made = 0;
+    if (n_sets + piece > m.cap_sets) st = -6;
+    else if (lane == 0) {
+      int flags = 0;
+      const Chart c = chart_of_history(m.item_state, m.item_origin, m.set_begin, n_sets - 1);
+      const int consumed = token_walk<int16_t>(g, g.class_bits, c, v.bytes + off + done, piece, false, w_st, w_org, kFastCap, lsb, &flags, nullptr);
+      if (flags & kWalkOverflow) st = -6;
+      else if (consumed < piece) st = -7;
+      else { made = lsb[piece + 1]; if (n_items + made > m.cap_items) st = -6; }
+    }
+    st = __shfl_sync(0xFFFFFFFFu, st, 0);
+    made = __shfl_sync(0xFFFFFFFFu, made, 0);
+    if (st != 0) break;
+    __syncwarp();
+    // origins written by the walk are already chart indices (its base is set n_sets - 1);
+    // append the new sets behind the history (visible to the next piece; committed below)
+    for (int q = lane; q < made; q += 32) { m.item_state[n_items + q] = w_st[q]; m.item_origin[n_items + q] = w_org[q]; }
+    for (int j = 1 + lane; j <= piece; j += 32) m.set_begin[n_sets + j] = n_items + lsb[j + 1];
+    __syncwarp();
+    n_items += made;
+    n_sets += piece;
+    done += piece;
+  }
+  if (st == 0) {
+    if (lane == 0) { m.n_sets = n_sets; m.n_items = n_items; }
+    __syncwarp();
+    prepare_plan(m, g, lane);      // the next mask's plan, while the new set is still hot
+  }
+  return st;
+}
+
+// One warp per request: requests follow unrelated paths, so sharing a warp between them would
+// serialise their walks.
 __global__ void __launch_bounds__(128)
 accept_kernel(MatcherDev* const* __restrict__ matchers, int batch, VocabDev v,
-              const int32_t* __restrict__ token_ids, int32_t* __restrict__ status) {
+              const int32_t* __restrict__ token_ids, int32_t* __restrict__ status, int restart_on_eos) {
   step_kernel_prologue();
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (b >= batch) return;
   MatcherDev& m = *matchers[b];
-  const GrammarDev& g = *m.grammar;
   __shared__ uint32_t sh_st[4][kFastCap];
   __shared__ int32_t sh_org[4][kFastCap];
   __shared__ int16_t sh_lsb[4][kFastMaxBytes + 2];
-  uint32_t* w_st = sh_st[threadIdx.x >> 5];
-  int32_t* w_org = sh_org[threadIdx.x >> 5];
-  int16_t* lsb = sh_lsb[threadIdx.x >> 5];
-  int st = 0;   // XG_OK
-  const int tok = token_ids[b];
-  if (m.terminated) st = -8;
-  else if (tok < 0 || tok >= v.vocab_size) st = -7;
-  else if (tok == v.eos_id) {
-    if (lane == 0) { if (root_complete(m, g)) m.terminated = 1; else st = -7; }
-    st = __shfl_sync(0xFFFFFFFFu, st, 0);
-  } else {
-    const int rank = v.id_to_rank[tok];
-    const uint32_t off = v.offset[rank];
-    const int len = (int)(v.offset[rank + 1] - off);
-    if (v.never[rank] || len == 0) st = -7;
-    else {
-      int n_sets = m.n_sets, n_items = m.n_items;
-      int done = 0;
-      while (done < len && st == 0) {            // long tokens go through in pieces
-        const int piece = min(len - done, kFastMaxBytes);
-        int made = 0;
-        if (n_sets + piece > m.cap_sets) st = -6;
-        else if (lane == 0) {
-          int flags = 0;
-          const Chart c = chart_of_history(m.item_state, m.item_origin, m.set_begin, n_sets - 1);
-          const int consumed = token_walk<int16_t>(g, g.class_bits, c, v.bytes + off + done, piece, false, w_st, w_org, kFastCap, lsb, &flags, nullptr);
-          if (flags & kWalkOverflow) st = -6;
-          else if (consumed < piece) st = -7;
-          else { made = lsb[piece + 1]; if (n_items + made > m.cap_items) st = -6; }
-        }
-        st = __shfl_sync(0xFFFFFFFFu, st, 0);
-        made = __shfl_sync(0xFFFFFFFFu, made, 0);
-        if (st != 0) break;
-        __syncwarp();
-        // origins written by the walk are already chart indices (its base is set n_sets - 1);
-        // append the new sets behind the history (visible to the next piece; committed below)
-        for (int q = lane; q < made; q += 32) { m.item_state[n_items + q] = w_st[q]; m.item_origin[n_items + q] = w_org[q]; }
-        for (int j = 1 + lane; j <= piece; j += 32) m.set_begin[n_sets + j] = n_items + lsb[j + 1];
-        __syncwarp();
-        n_items += made;
-        n_sets += piece;
-        done += piece;
-      }
-      if (st == 0) {
-        if (lane == 0) { m.n_sets = n_sets; m.n_items = n_items; }
-        __syncwarp();
-        prepare_plan(m, g, lane);      // the next mask's plan, while the new set is still hot
-      }
-    }
-  }
+  const int st = accept_one(m, *m.grammar, v, token_ids[b], restart_on_eos != 0, lane, sh_st[threadIdx.x >> 5], sh_org[threadIdx.x >> 5], sh_lsb[threadIdx.x >> 5]);
   if (status && lane == 0) status[b] = st;
 }
 
@@ -1034,15 +1045,22 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
 //      distributed shared memory;
 //   3. cluster barrier; every block writes its slice with coalesced stores.
 // No global atomics, no scratch words, and the row never makes a round trip through L2.
+// With kAccept the launch first accepts one sampled token per request (the first warp of the
+// cluster's block 0, as in accept_kernel; the rest of the cluster waits at a cluster barrier) and
+// then fills the mask of the state it reached: in a decode loop the two always follow each other,
+// and one launch saves a kernel boundary and lets a request with a slow accept and a short fill
+// overlap one with the opposite mix.
 // The host picks cluster and block size so that the whole batch is resident at once.  Used when
 // a slice fits (at most 2048 words per block); larger vocabularies take the two-kernel path above.
 // ------------------------------------------------------------------------------------------
 constexpr int kMaxClusterBlocks = 8;      // the portable cluster size limit
 
 // launched with a cluster of gridDim.x blocks (2, 4 or 8) along x
+template <bool kAccept>
 __global__ void __launch_bounds__(256, 4)
 fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __restrict__ bitmask, long long row_stride,
-                    int32_t* __restrict__ status_user) {
+                    int32_t* __restrict__ status_user, const int32_t* __restrict__ token_ids, int32_t* __restrict__ accept_status,
+                    int restart_on_eos) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ uint32_t dyn_smem[];          // this block's row slice and a scratch slice: 2 x ceil(W / blocks) words
@@ -1078,6 +1096,15 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   const int w0 = rank * chunk, w1 = min(v.n_words, w0 + chunk);
   const int nw = max(0, w1 - w0);
   for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] = 0;
+  if (kAccept) {
+    // nothing of the request's state or plan is read before this barrier; its release/acquire pair makes what the
+    // accepting warp wrote visible to the whole cluster
+    if (rank == 0 && threadIdx.x < 32) {
+      const int st = accept_one(*matchers[b], g, v, token_ids[b], restart_on_eos != 0, (int)threadIdx.x, long_st, long_org, long_lsb);
+      if (accept_status && threadIdx.x == 0) accept_status[b] = st;
+    }
+    cluster.sync();
+  }
   const int st0 = m.terminated ? -8 : (plan.overflow ? -6 : 0);
   if (threadIdx.x == 0) { sh_fail = 0; long_n = 0; }
   const bool fallback = st0 == 0 && plan.n_missing > 0;   // an entry is not built yet: walk the whole vocabulary instead

@@ -56,12 +56,21 @@ class Session:
     def fill(self) -> None:
         self.batch.fill_next_token_bitmask(self.bitmask.data_ptr(), self.W, self.status.data_ptr(), self.stream())
 
-    def accept(self, token_ids: Sequence[int]) -> None:
+    def accept(self, token_ids: Sequence[int], restart_on_eos: bool = False) -> None:
         self.tokens.copy_(torch.as_tensor(np.asarray(token_ids, dtype=np.int32)))
-        self.batch.accept_token(self.tokens.data_ptr(), self.accept_status.data_ptr(), self.stream())
+        self.batch.accept_token(self.tokens.data_ptr(), self.accept_status.data_ptr(), self.stream(), restart_on_eos)
 
-    def accept_device(self, token_ids: torch.Tensor) -> None:
-        self.batch.accept_token(token_ids.data_ptr(), self.accept_status.data_ptr(), self.stream())
+    def accept_device(self, token_ids: torch.Tensor, restart_on_eos: bool = False) -> None:
+        self.batch.accept_token(token_ids.data_ptr(), self.accept_status.data_ptr(), self.stream(), restart_on_eos)
+
+    def accept_fill(self, token_ids: Sequence[int], restart_on_eos: bool = False) -> None:
+        self.tokens.copy_(torch.as_tensor(np.asarray(token_ids, dtype=np.int32)))
+        self.accept_fill_device(self.tokens, restart_on_eos)
+
+    def accept_fill_device(self, token_ids: torch.Tensor, restart_on_eos: bool = False) -> None:
+        """Accept one token per request and fill the next step's mask, in one launch."""
+        self.batch.accept_token_and_fill_next_bitmask(token_ids.data_ptr(), self.accept_status.data_ptr(), restart_on_eos,
+                                                      self.bitmask.data_ptr(), self.W, self.status.data_ptr(), self.stream())
 
     def apply(self, logits: torch.Tensor, rows: Optional[torch.Tensor] = None) -> None:
         dtype = {torch.float32: "f32", torch.bfloat16: "bf16", torch.int16: "bf16", torch.uint16: "bf16"}[logits.dtype]

@@ -28,9 +28,12 @@ def _oracle_side(w):
     return ov, grammars, matchers
 
 
-def _run_trajectories(w, check_steps, check_requests=None):
+def _run_trajectories(w, check_steps, check_requests=None, fused=False, restart=False):
     """Drive GPU and oracle along the seeded trajectories; compare masks where asked, and the
-    cheap invariants everywhere (sampled token allowed, statuses, termination)."""
+    cheap invariants everywhere (sampled token allowed, statuses, termination).  fused: after the
+    first fill every step is one accept-and-fill launch that restarts a request at end of
+    sequence, instead of accept, reset and fill.  restart: the accept call restarts a request at
+    end of sequence (no reset call)."""
     torch, engine = _engine()
     s = engine.Session(w)
     ov, _, oms = _oracle_side(w)
@@ -38,7 +41,8 @@ def _run_trajectories(w, check_steps, check_requests=None):
     compared = 0
     try:
         for step in range(w.steps):
-            s.fill()
+            if step == 0 or not fused:
+                s.fill()
             mask = s.mask_numpy()
             status = s.status.cpu().numpy()
             assert (status == 0).all(), (step, status)
@@ -52,16 +56,20 @@ def _run_trajectories(w, check_steps, check_requests=None):
                         raise AssertionError("step %d request %d: %d differing tokens, e.g. %r (gpu=%d)" % (
                             step, b, len(diff), [w.vocab.tokens[t] for t in diff[:8]], int((mask[b, diff[0] >> 5] >> (diff[0] & 31)) & 1)))
                     compared += 1
-            s.accept(toks)
+            if fused:
+                s.accept_fill(toks, restart_on_eos=True)
+            else:
+                s.accept(toks, restart_on_eos=restart)
             ast = s.accept_status.cpu().numpy()
             assert (ast == 0).all(), (step, ast)
             for b in range(n):
                 r = oms[b].accept_token(ov, toks[b])
                 assert r in (1, 2)
                 if r == 2:
-                    assert s.matchers[b].is_terminated()
+                    assert s.matchers[b].is_terminated() != (fused or restart)
                     oms[b].reset()
-                    s.reset(b)
+                    if not (fused or restart):
+                        s.reset(b)
         return compared
     finally:
         s.close()
