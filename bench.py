@@ -384,7 +384,7 @@ def main():
     dominant = max((("fill", t_fill), ("apply", t_apply), ("accept", t_accept)), key=lambda x: x[1])[0]
     # bytes per launch by ncu (profiles/step_kernels_c3.txt): DRAM reads + bytes written towards L2, which the logits ring
     # turns into DRAM write-backs; measured on C3 only, and void once apply_kernel changes
-    traffic = 50.6e6 if (args.workload == "C3" and n == 128) else None
+    traffic = 50.9e6 if (args.workload == "C3" and n == 128) else None
     roofline = {"kernel": "apply_kernel", "bound": "hbm", "achieved": apply_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": apply_gbs / peak, "traffic": traffic, "us_per_launch": t_apply, "masked_fraction": masked_frac,
                 "conventional_gbs": apply_conv_bytes / (t_apply * 1e-6) / 1e9, "dominant_by_time": dominant,
