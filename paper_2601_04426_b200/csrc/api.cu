@@ -1429,11 +1429,14 @@ xg_status_t xg_apply_token_bitmask(void* logits_dev, xg_dtype_t dtype, int32_t b
     return set_error(XG_ERR_INVALID_ARG, "logits rows must start on 16-byte boundaries");
   const int elems = 16 / elt;
   const int n_vec = vocab_size / elems;
-  // about eight blocks of 256 threads per SM in total (one full wave), split evenly over the rows
+  // Enough blocks per row that every thread makes one pass of four vectors (measured: C3 9.4 us per launch against
+  // 11.1 with half as many blocks and two passes, C5 27.7 against 31.7; more and narrower passes are slower again),
+  // and for small batches at least about eight blocks of 256 threads per SM in total.
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int per_row_max = std::max(1, (n_vec + 255) / 256);
-  const int bx = std::max(1, std::min(per_row_max, (sms * 8 + rows / 2) / rows));
+  const int one_pass = (n_vec + 1023) / 1024;
+  const int bx = std::max(1, std::min(per_row_max, std::max(one_pass, (sms * 8 + rows / 2) / rows)));
   if (rows > 65535) return set_error(XG_ERR_INVALID_ARG, "more than 65535 rows");
   dim3 grid(bx, rows);
   if (dtype == XG_BF16)
