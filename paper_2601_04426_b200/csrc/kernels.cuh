@@ -1200,22 +1200,23 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
       while (j >= ent_cum[e + 1]) ++e;
       const int k = j - ent_cum[e];
       uint32_t left = ent_exit[e][k];
+      const int trank = (int)ent_rank[e][k];      // read together with the exit mask: one dependent load less for the survivors
       bool pass = false;
-      int trank = -1;
+      int id = -1;
       if (left == 0) {                // no exit record (very long token, or its build-time walk overflowed): walk in full
-        trank = (int)ent_rank[e][k];
         if ((int)(v.offset[trank + 1] - v.offset[trank]) > kFastMaxBytes) {
           const int slot = atomicAdd(&long_n, 1);
           if (slot < kLongQueue) long_q[slot] = trank; else atomicOr(cluster.map_shared_rank(&sh_fail, 0), 1);
           continue;
         }
+        id = v.rank_to_id[trank];
         pass = walk_one(trank, v.offset[trank], e, 0);
       } else {
         uint32_t byte = ent_byte[e][k];
         if (!((cont_first[e][byte >> 5] >> (byte & 31)) & 1u)) left &= left - 1;
         if (left == 0) continue;                        // the usual end of a candidate
-        trank = (int)ent_rank[e][k];
         const uint32_t off = v.offset[trank];
+        id = v.rank_to_id[trank];                       // requested before the walk, needed after it
         while (left && !pass) {
           const int at = __ffs(left) - 1;
           left &= left - 1;
@@ -1224,7 +1225,6 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
         }
       }
       if (pass) {
-        const int id = v.rank_to_id[trank];
         const int word = id >> 5, owner = word / chunk;
         atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
       }
