@@ -690,8 +690,19 @@ __global__ void matcher_reset_kernel(MatcherDev* m) {      // one warp
 __device__ __forceinline__ int accept_one(MatcherDev& m, const GrammarDev& g, const VocabDev& v, int tok, bool restart_on_eos, int lane,
                                           uint32_t* w_st, int32_t* w_org, int16_t* lsb) {
   int st = 0;   // XG_OK
+  // The token's bytes and the request's current set are each a few dependent loads away (id -> rank -> offset ->
+  // bytes; counters -> set bounds -> first item -> its state record).  Both chains are requested before anything is
+  // tested, so that they travel together instead of one after the other.
+  const bool tok_ok = tok >= 0 && tok < v.vocab_size;
+  const int rank = v.id_to_rank[tok_ok ? tok : 0];
+  int n_sets = m.n_sets, n_items = m.n_items;
+  const Chart c0 = chart_of_history(m.item_state, m.item_origin, m.set_begin, n_sets - 1);
+  const uint32_t off = v.offset[rank];
+  const int len = (int)(v.offset[rank + 1] - off);
+  const bool never = v.never[rank] != 0;
+  if (c0.i_cnt > 0) asm volatile("prefetch.global.L1 [%0];" ::"l"(&g.state[c0.i_st[0]]));
   if (m.terminated) return -8;
-  if (tok < 0 || tok >= v.vocab_size) return -7;
+  if (!tok_ok) return -7;
   if (tok == v.eos_id) {
     if (lane == 0) {
       if (!root_complete(m, g)) st = -7;
@@ -702,11 +713,7 @@ __device__ __forceinline__ int accept_one(MatcherDev& m, const GrammarDev& g, co
     if (st == 0 && restart_on_eos) { __syncwarp(); prepare_plan(m, g, lane); }
     return st;
   }
-  const int rank = v.id_to_rank[tok];
-  const uint32_t off = v.offset[rank];
-  const int len = (int)(v.offset[rank + 1] - off);
-  if (v.never[rank] || len == 0) return -7;
-  int n_sets = m.n_sets, n_items = m.n_items;
+  if (never || len == 0) return -7;
   int done = 0;
   while (done < len && st == 0) {            // long tokens go through in pieces
     const int piece = min(len - done, kFastMaxBytes);
@@ -714,7 +721,7 @@ __device__ __forceinline__ int accept_one(MatcherDev& m, const GrammarDev& g, co
     if (n_sets + piece > m.cap_sets) st = -6;
     else if (lane == 0) {
       int flags = 0;
-      const Chart c = chart_of_history(m.item_state, m.item_origin, m.set_begin, n_sets - 1);
+      const Chart c = done == 0 ? c0 : chart_of_history(m.item_state, m.item_origin, m.set_begin, n_sets - 1);
       const int consumed = token_walk<int16_t>(g, g.class_bits, c, v.bytes + off + done, piece, false, w_st, w_org, kFastCap, lsb, &flags, nullptr);
       if (flags & kWalkOverflow) st = -6;
       else if (consumed < piece) st = -7;
@@ -1081,7 +1088,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   __shared__ uint32_t long_st[kLongCap];
   __shared__ int32_t long_org[kLongCap];
   __shared__ int16_t long_lsb[kSlowMaxBytes + 2];
-  __shared__ int sh_fail;          // block 0's copy collects the whole cluster's failures
+  __shared__ int sh_fail;          // set in every block of the cluster when any of them fails
 
   step_kernel_prologue();
   const int b = blockIdx.y;
@@ -1158,6 +1165,9 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
     }
     cluster.sync();            // every slice is merged (and this block's staging is visible)
     const int stride = n_blocks * blockDim.x;
+    // a failure (rare) is recorded in every block's flag, so that each block reads its own at the end and no block has to
+    // outlive the others' reads
+    auto fail_everywhere = [&]() { for (int r = 0; r < n_blocks; ++r) atomicOr(cluster.map_shared_rank(&sh_fail, r), 1); };
     auto walk_one = [&](int trank, uint32_t off, int e, int at) {
       const int len = (int)(v.offset[trank + 1] - off);
       bool pass = false, overflow = len - at > kFastMaxBytes;
@@ -1171,7 +1181,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
         pass = token_walk<int16_t>(g, class_bits, c, v.bytes + off + at, len - at, false, st, org, kFastCap, lsb, &flags, nullptr) == len - at;
         overflow = (flags & kWalkOverflow) != 0;
       }
-      if (overflow) atomicOr(cluster.map_shared_rank(&sh_fail, 0), 1);
+      if (overflow) fail_everywhere();
       return pass && !overflow;
     };
     if (fallback) {
@@ -1183,7 +1193,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
         if (!((set_first[byte >> 5] >> (byte & 31)) & 1u)) continue;
         if ((int)(v.offset[r + 1] - off) > kFastMaxBytes) {
           const int slot = atomicAdd(&long_n, 1);
-          if (slot < kLongQueue) long_q[slot] = r; else atomicOr(cluster.map_shared_rank(&sh_fail, 0), 1);
+          if (slot < kLongQueue) long_q[slot] = r; else fail_everywhere();
           continue;
         }
         if (walk_one(r, off, 0, 0)) {
@@ -1206,7 +1216,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
       if (left == 0) {                // no exit record (very long token, or its build-time walk overflowed): walk in full
         if ((int)(v.offset[trank + 1] - v.offset[trank]) > kFastMaxBytes) {
           const int slot = atomicAdd(&long_n, 1);
-          if (slot < kLongQueue) long_q[slot] = trank; else atomicOr(cluster.map_shared_rank(&sh_fail, 0), 1);
+          if (slot < kLongQueue) long_q[slot] = trank; else fail_everywhere();
           continue;
         }
         id = v.rank_to_id[trank];
@@ -1237,7 +1247,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
         const int len = (int)(v.offset[trank + 1] - off);
         int flags = 0;
         const bool pass = token_walk<int16_t>(g, class_bits, hist, v.bytes + off, len, false, long_st, long_org, kLongCap, long_lsb, &flags, nullptr) == len;
-        if (flags & kWalkOverflow) atomicOr(cluster.map_shared_rank(&sh_fail, 0), 1);
+        if (flags & kWalkOverflow) fail_everywhere();
         else if (pass) {
           const int id = v.rank_to_id[trank];
           const int word = id >> 5, owner = word / chunk;
@@ -1248,11 +1258,10 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
     cluster.sync();            // every remote OR has landed
   } else __syncthreads();
   // 3. write the slice
-  const int failed = (total > 0 || fallback) ? *cluster.map_shared_rank(&sh_fail, 0) : 0;
+  const int failed = (total > 0 || fallback) ? sh_fail : 0;
   const bool clear = st0 != 0 || failed;
   for (int w = threadIdx.x; w < nw; w += blockDim.x) bitmask[(long long)b * row_stride + w0 + w] = clear ? 0 : (int32_t)row[w];
   if (rank == 0 && threadIdx.x == 0 && status_user) status_user[b] = st0 != 0 ? st0 : (failed ? -6 : 0);
-  if (total > 0 || fallback) cluster.sync();      // block 0's shared memory must outlive the reads above
 }
 
 // ------------------------------------------------------------------------------------------
