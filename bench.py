@@ -430,7 +430,7 @@ def main():
     # the kernels change) over the launch time, against 148 SMs x 4 schedulers x the SM clock.
     props = torch.cuda.get_device_properties(local_rank)
     issue_peak = props.multi_processor_count * 4 * (clocks["sm_max_mhz"] or 1965.0) * 1e6
-    warp_insts = {"fill": 1431770.0, "accept": 117728.0} if (args.workload == "C3" and n == 128) else {}
+    warp_insts = {"fill": 1354736.0, "accept": 121532.0} if (args.workload == "C3" and n == 128) else {}
     latency_bound = {}
     for name, t_us in (("fill", t_fill), ("accept", t_accept)):
         wi = warp_insts.get(name)
