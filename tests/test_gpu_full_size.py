@@ -94,5 +94,13 @@ def test_vocabulary_too_large_for_one_cluster_takes_the_two_kernel_path():
             if om.accept_token(ov, tok) == 2:
                 om.reset()
                 s.reset(0)
+        # the accept-and-fill entry point on this path: accept kernel, then the two fill kernels
+        s.reset(0); om.reset()
+        for step, tok in enumerate(w.trajectories[0][:4]):
+            s.accept_fill([tok], restart_on_eos=True)
+            assert int(s.accept_status.cpu()[0]) == 0 and int(s.status.cpu()[0]) == 0
+            if om.accept_token(ov, tok) == 2:
+                om.reset()
+            assert np.array_equal(s.mask_numpy()[0], om.mask(ov)), step
     finally:
         s.close()
