@@ -169,6 +169,24 @@ def test_classification_partition_and_soundness():
         tm.accept_bytes(w.vocab.tokens[tok])
 
 
+def test_classification_against_hand_worked_table():
+    """Section 3.4 on paper: every token at every scannable state of a two-rule grammar, from both
+    sides -- a token wrongly called uncertain (an inner rule ended, the state's own did not) fails
+    here just as one wrongly called accepted or rejected."""
+    from golden_util import load_classify_fixture, state_at_path
+    ebnf, tokens, cases = load_classify_fixture("classify_bracket_item.txt")
+    ov = O.Vocab([t.encode() for t in tokens], tokens.index(""))
+    tb, g = tables_of("ebnf", ebnf, inline_max_states=0)
+    t = g.tables()
+    assert t["n_rules"] == 2                              # `item` was kept as a rule of its own
+    states = [state_at_path(t, path) for path, _, _ in cases]
+    assert sorted(states) == tb.scannable_states()        # the fixture covers every scannable state
+    for s, (path, acc, unc) in zip(states, cases):
+        cls = tb.classify(ov, s)
+        assert sorted(tokens[i] for i in np.nonzero(cls == 1)[0]) == sorted(acc), path
+        assert sorted(tokens[i] for i in np.nonzero(cls == 2)[0]) == sorted(unc), path
+
+
 def test_front_end_errors():
     cases = [("ebnf", 'root ::= "a', B.XG_ERR_PARSE), ("ebnf", "root ::= missing", B.XG_ERR_PARSE), ("ebnf", 'x ::= "a"', B.XG_ERR_PARSE),
              ("ebnf", 'root ::= "a"{3,2}', B.XG_ERR_PARSE), ("json_schema", "{", B.XG_ERR_PARSE),
