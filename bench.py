@@ -113,21 +113,20 @@ class ClockSampler(threading.Thread):
         return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(sm)}
 
 
-def oracle_leg(w, steps, warmup, sample_pairs=None):
-    """The CPU oracle, as it stands, on a bounded sample: a few (request, step) masks plus the
-    apply of one row each, scaled to a whole batch step."""
+def oracle_leg(w, steps, warmup, threads=None, n_req=None, budget_s=25.0):
+    """The CPU oracle, as it stands, on a bounded sample: the masks of the first requests of the batch along
+    their trajectories plus the apply of one row each, scaled to a whole batch step.  The same (request, step)
+    pairs whatever arm calls it, so the figures of the two arms can be compared."""
     from oracle import oracle as O
     from oracle import schema_ebnf as SE
-    threads = O.default_threads()
+    threads = threads or O.default_threads()
     ov = O.Vocab(w.vocab.tokens, w.vocab.eos_id, w.vocab.special_ids)
-    n_req = min(w.batch, 4)
+    n_req = min(w.batch, len(w.request_grammar), n_req or 16)
     oms = [O.Matcher(O.Grammar(SE.grammar_text(w.grammars[w.request_grammar[b]].kind, w.grammars[w.request_grammar[b]].text))) for b in range(n_req)]
     logits = inputs.make_logits(w.logits_seed, 1, w.vocab.size, w.dtype)
     per_step = []
-    total_steps = warmup + steps
-    budget_s = 25.0
     t_begin = time.perf_counter()
-    for step in range(min(total_steps, w.steps)):
+    for step in range(min(warmup + steps, w.steps)):
         t0 = time.perf_counter()
         for b in range(n_req):
             mask = oms[b].mask(ov, threads)
@@ -142,7 +141,57 @@ def oracle_leg(w, steps, warmup, sample_pairs=None):
         if time.perf_counter() - t_begin > budget_s and len(per_step) >= 1:
             break
     us = 1e6 * float(np.mean(per_step))
-    return us, threads, "%d steps x %d of %d requests (mask + apply of each), scaled to the batch" % (len(per_step), n_req, w.batch)
+    sample = "steps %d..%d x the first %d of %d requests (mask + apply of each), scaled x%.1f to the batch" % (
+        warmup, warmup + len(per_step) - 1, n_req, w.batch, w.batch / n_req)
+    return us, threads, sample
+
+
+def oracle_cache_build_leg(w, n_scannable_total, threads, n_positions=48, budget_s=10.0):
+    """The oracle's classification (accepted / uncertain / rejected of every token at one scannable state,
+    from the flattened tables) on a seeded sample of positions of the first grammar, extrapolated to the
+    workload's scannable positions."""
+    from oracle import oracle as O
+    from paper_2601_04426_b200 import binding as XB
+    ov = O.Vocab(w.vocab.tokens, w.vocab.eos_id, w.vocab.special_ids)
+    g = XB.Grammar(None, w.grammars[0].kind, w.grammars[0].text)          # host front end only: the tables
+    t = g.tables()
+    scal = {k: t.pop(k) for k in ("n_rules", "n_states", "n_classes", "root_rule", "root_nullable")}
+    tb = O.Tables(scal["n_rules"], scal["n_states"], scal["n_classes"], scal["root_rule"], scal["root_nullable"], **t)
+    states = tb.scannable_states()
+    rng = inputs.Rng(inputs.config_seed(w.name) ^ 0xB111D)
+    picked = [states[rng.below(len(states))] for _ in range(min(n_positions, len(states)))]
+    t0 = time.perf_counter()
+    done = 0
+    for st in picked:
+        tb.classify(ov, st, threads)
+        done += 1
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    g.close()
+    pairs_per_s = done * w.vocab.size / dt
+    return {"pairs_per_s": pairs_per_s, "seconds_extrapolated": n_scannable_total * w.vocab.size / pairs_per_s, "cores": threads,
+            "sample": "%d seeded positions of grammar 0 x the whole vocabulary, extrapolated to %d scannable positions" % (done, n_scannable_total)}
+
+
+def kernels_sha():
+    """First 16 hex digits of the SHA-256 of the kernel source: ncu figures are tied to the kernels they were taken on."""
+    import hashlib
+    with open(os.path.join(ROOT, "paper_2601_04426_b200", "csrc", "kernels.cuh"), "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:16]
+
+
+def ncu_figures(workload, batch):
+    """Counters read from ncu captures (profiles/ncu_counters.json), or {} when they were taken on another
+    version of the kernels or on another workload."""
+    path = os.path.join(ROOT, "profiles", "ncu_counters.json")
+    if not os.path.exists(path):
+        return {}
+    with open(path) as f:
+        rec = json.load(f)
+    if rec.get("kernels_sha16") != kernels_sha():
+        return {}
+    return rec.get("workloads", {}).get("%s/%d" % (workload, batch), {})
 
 
 def main():
@@ -154,8 +203,9 @@ def main():
     ap.add_argument("--workload", default="C3", choices=sorted(SHAPES))
     ap.add_argument("--batch", type=int, default=None, help="shrink the batch (debugging only; the line then names it)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--fused-accept-fill", action="store_true",
-                    help="step = apply, then accept and the next mask's fill in one launch, instead of fill, apply, accept as three launches")
+    ap.add_argument("--step", default="three", choices=["three", "fill_apply", "accept_fill"],
+                    help="how a step is launched: 'three' = fill, apply, accept as three launches (default); 'fill_apply' = fill and apply "
+                         "in one launch, then accept; 'accept_fill' = apply, then accept and the next mask's fill in one launch")
     ap.add_argument("--jit-sweep", default=None,
                     help="comma-separated K values (or 'full'): compile just in time with K entries precomputed and report "
                          "compile time and per-step time avg / P99 / max over the trajectory (the shape of the paper's K sweep)")
@@ -173,7 +223,7 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return 0
-        w = inputs.make_workload(args.workload, batch=min(args.batch or B0, 4))
+        w = inputs.make_workload(args.workload, batch=min(args.batch or B0, 16))
         w_full_batch = args.batch or B0
         us, threads, sample = oracle_leg(_with_batch(w, w_full_batch), args.steps, args.warmup)
         line = {"impl": "reference", "metric": metric, "value": us, "unit": "us/step", "n_gpus": args.gpus, "steps": args.steps,
@@ -224,123 +274,128 @@ def main():
     ring = [base.repeat((n + base.shape[0] - 1) // base.shape[0], 1)[:n].contiguous() for _ in range(ring_n)]
     traj = torch.from_numpy(np.asarray([[w.trajectories[b][t] for b in range(n)] for t in range(w.steps)], dtype=np.int32)).to(s.device)      # [steps, n]
     total = warmup + args.steps
-    launches = {"accept": 0, "fill": 0, "apply": 0, "reset": 0, "accept_fill": 0}      # this library's kernels only
-    fused = args.fused_accept_fill
-
-    def restart(first_mask=False):
-        for b in range(n):
-            s.reset(b)
-        launches["reset"] += n
-        if first_mask:
-            s.fill()
-            launches["fill"] += 1
+    launches = {"accept": 0, "fill": 0, "apply": 0, "reset": 0, "accept_fill": 0, "fill_apply": 0}      # this library's kernels only
 
     # The decode loop is launch-bound (short kernels), so the timed loop replays CUDA graphs, as a
     # serving engine's decode loop does: one graph per trajectory step, with the step's token ids
     # read straight from the resident trajectory table and the logits buffer taken from the ring.
-    # A step fills the mask, masks the logits and accepts the step's token: three launches.  A
-    # request that accepts end of sequence starts its next document in the accept launch.
-    # (--fused-accept-fill: apply, then accept and the next mask's fill in one launch.)  Either
-    # way every step runs accept, fill and apply once for every request.
+    # Every way of launching a step runs accept, fill and apply once for every request; a request
+    # that accepts end of sequence starts its next document in the accept launch.
+    #   three        fill, apply, accept                                      (3 launches, the default)
+    #   fill_apply   fill + apply in one launch, accept                       (2 launches)
+    #   accept_fill  apply, accept + fill of the next mask in one launch      (2 launches; needs a first fill)
+    #   no_apply     fill, accept: not a step -- the three-launch step without its apply, for apply's in-step cost
+    def body_of(mode):
+        def body(buf, t):
+            if mode == "fill_apply":
+                s.fill_apply(buf)
+                s.accept_device(traj[t], restart_on_eos=True)
+            elif mode == "three":
+                s.fill(); s.apply(buf)
+                s.accept_device(traj[t], restart_on_eos=True)
+            elif mode == "accept_fill":
+                s.apply(buf)
+                s.accept_fill_device(traj[t], restart_on_eos=True)
+            else:
+                s.fill()
+                s.accept_device(traj[t], restart_on_eos=True)
+        return body
 
-    def step_body(buf, t):
-        if fused:
-            s.apply(buf)
-            s.accept_fill_device(traj[t], restart_on_eos=True)
-        else:
+    per_step_launches = {"fill_apply": {"fill_apply": 1, "accept": 1}, "three": {"fill": 1, "apply": 1, "accept": 1},
+                         "accept_fill": {"apply": 1, "accept_fill": 1}, "no_apply": {"fill": 1, "accept": 1}}
+
+    def restart(mode):
+        for b in range(n):
+            s.reset(b)
+        launches["reset"] += n
+        if mode == "accept_fill":
             s.fill()
-            s.apply(buf)
-            s.accept_device(traj[t], restart_on_eos=True)
+            launches["fill"] += 1
 
-    for k in range(ring_n):              # eager warm-up of every call before capture (first-use set-up)
-        step_body(ring[k], 0)
-    torch.cuda.synchronize()
-    restart(fused)
-    graphs = []
-    for t in range(w.steps):
-        gph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(gph):
-            step_body(ring[t % ring_n], t)
-        graphs.append(gph)
-    torch.cuda.synchronize()
-    restart(fused)
+    def capture(mode, group=1):
+        """One graph per `group` consecutive trajectory steps."""
+        body = body_of(mode)
+        restart(mode)
+        torch.cuda.synchronize()
+        graphs = []
+        for t0_ in range(0, w.steps - group + 1, group):
+            gph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gph):
+                for t in range(t0_, t0_ + group):
+                    body(ring[t % ring_n], t)
+            graphs.append(gph)
+        torch.cuda.synchronize()
+        return graphs
 
-    def one_step(i):
-        t = i % w.steps
-        if t == 0 and i > 0:
-            restart(fused)
-        graphs[t].replay()
-        launches["apply"] += 1
-        if fused:
-            launches["accept_fill"] += 1
-        else:
-            launches["fill"] += 1; launches["accept"] += 1
+    def replay_pass(mode, graphs, n_replays, n_warm, group=1, count=False):
+        """Replays graph i % len(graphs) for i in [0, n_warm + n_replays); returns us per step of the last n_replays."""
+        restart(mode)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for i in range(n_warm + n_replays):
+            if i == n_warm:
+                if count:
+                    for k in launches:
+                        launches[k] = 0
+                dist_util.barrier()
+                torch.cuda.synchronize()
+                e0.record()
+            if i % len(graphs) == 0 and i > 0:
+                restart(mode)
+            graphs[i % len(graphs)].replay()
+            for k, c in per_step_launches[mode].items():
+                launches[k] += c * group
+        e1.record()
+        torch.cuda.synchronize()
+        dist_util.barrier()
+        return dist_util.max_over_ranks(e0.elapsed_time(e1)) * 1e3 / (n_replays * group)
+
+    for mode in ("three", "fill_apply", "accept_fill"):      # eager warm-up of every call before capture (first-use set-up)
+        restart(mode)
+        for k in range(ring_n):
+            body_of(mode)(ring[k], 0)
+    torch.cuda.synchronize()
 
     # ---- pass A: the headline number (events only around the timed region) --------------------
-    for i in range(warmup):
-        one_step(i)
-    for k in launches:
-        launches[k] = 0
     sampler = ClockSampler(local_rank)
     sampler.start()
-    dist_util.barrier()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(warmup, total):
-        one_step(i)
-    e1.record()
-    torch.cuda.synchronize()
-    dist_util.barrier()
-    ms_total = dist_util.max_over_ranks(e0.elapsed_time(e1))
-    us_per_step = 1e3 * ms_total / args.steps
+    graphs = capture(args.step)
+    us_per_step = replay_pass(args.step, graphs, args.steps, warmup, count=True)
     timed_launches = sum(launches.values())
+    del graphs
 
-    # ---- pass A2: the same steps with eight of them per graph (context, not the headline) ------
+    # ---- the same steps launched the other ways, and eight steps per graph (context, not the headline) ------
     # A serving engine's decode graph holds the model's forward pass too, so the launch of the
     # graph is shared with everything else in the step.  With eight steps per graph, seven of
     # eight step boundaries are kernel-to-kernel edges like the ones inside a step.
+    by_mode = {args.step: us_per_step}
+    for mode in ("fill_apply", "three", "accept_fill", "no_apply"):
+        if mode not in by_mode:
+            g2 = capture(mode)
+            by_mode[mode] = replay_pass(mode, g2, args.steps, warmup)
+            del g2
     group = 8
     multi_us = None
     if w.steps % group == 0 and args.steps >= group:
-        restart(fused)
-        torch.cuda.synchronize()
-        multi = []
-        for t0 in range(0, w.steps, group):
-            gph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(gph):
-                for t in range(t0, t0 + group):
-                    step_body(ring[t % ring_n], t)
-            multi.append(gph)
-        torch.cuda.synchronize()
-        n_groups = max(1, args.steps // group)
-        for phase in ("warm", "timed"):
-            restart(fused)
-            torch.cuda.synchronize()
-            m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            m0.record()
-            for i in range(n_groups):
-                if i % len(multi) == 0 and i > 0:
-                    restart(fused)
-                multi[i % len(multi)].replay()
-            m1.record()
-            torch.cuda.synchronize()
-        multi_us = dist_util.max_over_ranks(m0.elapsed_time(m1)) * 1e3 / (n_groups * group)
-        del multi
+        g8 = capture(args.step, group)
+        multi_us = replay_pass(args.step, g8, max(1, args.steps // group), max(1, warmup // group), group)
+        del g8
+    # what the apply kernel adds to a replayed three-launch step (launch overlap and kernel boundary included)
+    t_apply_in_step = max(by_mode["three"] - by_mode["no_apply"], 1e-3)
 
     # ---- pass B: per-kernel device times over the same steps -----------------------------------
     # Eager calls with events between them.  A short spin kernel in front of every step lets the
     # host queue the whole step before the GPU starts it, so the event intervals are device time
     # (kernel + launch gap) rather than host issue time.
-    restart()
+    restart("three")
     spin_cycles = int(2.0e5)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     zero_bits_sum, mask_samples = 0, 0
+    sector_stats = np.zeros(3)
     fill_work = {"merge_bytes": 0, "check_bytes": 0, "row_bytes": 0, "check_tokens": 0, "steps": 0}
     for i in range(total):
         t = i % w.steps
         if t == 0 and i > 0:
-            restart()
+            restart("three")
         buf = ring[i % ring_n]
         ev = evs[i - warmup] if i >= warmup else None
         torch.cuda._sleep(spin_cycles)
@@ -356,36 +411,47 @@ def main():
         if ev:
             ev[3].record()
         if ev and (i - warmup) % 10 == 0:            # masked fraction, sampled (synchronises; outside the event intervals)
-            zero_bits_sum += n * s.V - int(np.unpackbits(s.mask_numpy().view(np.uint8)).sum())
+            bits = np.unpackbits(s.mask_numpy().view(np.uint8), axis=1, bitorder="little")[:, :s.V]
+            zero_bits_sum += n * s.V - int(bits.sum())
             mask_samples += 1
-            if (i - warmup) % 10 == 0:                 # what the next fill streams: cache entries merged, candidates tested, row written
-                for m in s.matchers:
-                    fw = m.next_fill_work(s.stream())
-                    fill_work["merge_bytes"] += fw["merge_bytes"]; fill_work["check_bytes"] += fw["check_bytes"]
-                    fill_work["row_bytes"] += fw["row_bytes"]; fill_work["check_tokens"] += fw["check_tokens"]
-                fill_work["steps"] += 1
+            # the 32-byte sectors of the logits by what the mask does to them: untouched, overwritten, read and rewritten
+            per_sector = 32 // elt
+            sec = bits[:, :s.V // per_sector * per_sector].reshape(n, -1, per_sector).sum(axis=2)
+            sector_stats += [int((sec == per_sector).sum()), int((sec == 0).sum()), int(((sec > 0) & (sec < per_sector)).sum())]
+            for m in s.matchers:                       # what the next fill streams: cache entries merged, candidates tested, row written
+                fw = m.next_fill_work(s.stream())
+                fill_work["merge_bytes"] += fw["merge_bytes"]; fill_work["check_bytes"] += fw["check_bytes"]
+                fill_work["row_bytes"] += fw["row_bytes"]; fill_work["check_tokens"] += fw["check_tokens"]
+            fill_work["steps"] += 1
     torch.cuda.synchronize()
     eager_us = {"fill": float(np.mean([e[0].elapsed_time(e[1]) for e in evs])) * 1e3,
                 "apply": float(np.mean([e[1].elapsed_time(e[2]) for e in evs])) * 1e3,
                 "accept": float(np.mean([e[2].elapsed_time(e[3]) for e in evs])) * 1e3}
 
-    # the one-launch accept-and-fill, timed the same way (apply in front of it, as in the step)
-    restart(True)
-    evf = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
-    for i in range(total):
-        t = i % w.steps
-        if t == 0 and i > 0:
-            restart(True)
-        ev = evf[i - warmup] if i >= warmup else None
-        torch.cuda._sleep(spin_cycles)
-        s.apply(ring[i % ring_n])
-        if ev:
-            ev[0].record()
-        s.accept_fill_device(traj[t], restart_on_eos=True)
-        if ev:
-            ev[1].record()
-    torch.cuda.synchronize()
-    eager_us["accept_fill"] = float(np.mean([e[0].elapsed_time(e[1]) for e in evf])) * 1e3
+    # the two-in-one launches, timed the same way
+    for name, mode in (("accept_fill", "accept_fill"), ("fill_apply", "fill_apply")):
+        restart(mode)
+        evf = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+        for i in range(total):
+            t = i % w.steps
+            if t == 0 and i > 0:
+                restart(mode)
+            ev = evf[i - warmup] if i >= warmup else None
+            torch.cuda._sleep(spin_cycles)
+            if mode == "accept_fill":
+                s.apply(ring[i % ring_n])
+            if ev:
+                ev[0].record()
+            if mode == "accept_fill":
+                s.accept_fill_device(traj[t], restart_on_eos=True)
+            else:
+                s.fill_apply(ring[i % ring_n])
+            if ev:
+                ev[1].record()
+            if mode == "fill_apply":
+                s.accept_device(traj[t], restart_on_eos=True)
+        torch.cuda.synchronize()
+        eager_us[name] = float(np.mean([e[0].elapsed_time(e[1]) for e in evf])) * 1e3
 
     # ---- apply alone: launches back to back over the logits ring (the last step's mask) ---------
     # The intervals above hold the launch gap of a short kernel; a stream of launches does not.
@@ -411,33 +477,45 @@ def main():
     masked_frac = zero_bits / float(n * s.V)
     apply_alg_bytes = 4.0 * n * W + elt * zero_bits
     apply_conv_bytes = 2.0 * elt * n * s.V + 4.0 * n * W
+    # what has to cross the memory interface in 32-byte sectors: the mask, every sector with a masked logit written,
+    # every sector that mixes allowed and masked logits read first
+    sec_untouched, sec_overwritten, sec_mixed = (sector_stats / max(mask_samples, 1)).tolist()
+    apply_sector_bytes = 4.0 * n * W + 32.0 * (sec_overwritten + 2 * sec_mixed)
     peak, peak_kind = measured_peaks()
-    apply_gbs = apply_alg_bytes / (t_apply * 1e-6) / 1e9
+    ncu = ncu_figures(args.workload, n)
+    traffic = ncu.get("apply_kernel", {}).get("dram_bytes")          # ncu: DRAM bytes read + written per launch; None once the kernels changed
+    apply_gbs = apply_alg_bytes / (t_apply_in_step * 1e-6) / 1e9
     dominant = max((("fill", t_fill), ("apply", t_apply), ("accept", t_accept)), key=lambda x: x[1])[0]
-    # bytes per launch by ncu (profiles/step_kernels_c3.txt): DRAM reads + bytes written towards L2, which the logits ring
-    # turns into DRAM write-backs; measured on C3 only, and void once apply_kernel changes
-    traffic = 50.9e6 if (args.workload == "C3" and n == 128) else None
-    roofline = {"kernel": "apply_kernel", "bound": "hbm", "achieved": apply_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                "frac": apply_gbs / peak, "traffic": traffic, "us_per_launch": t_apply, "masked_fraction": masked_frac,
-                "conventional_gbs": apply_conv_bytes / (t_apply * 1e-6) / 1e9, "dominant_by_time": dominant,
-                "alone": {"how": "%d launches back to back over the logits ring (queued behind a primer kernel), last step's mask" % reps, "us_per_launch": t_apply_alone,
-                          "achieved": (4.0 * n * W + elt * alone_zero_bits) / (t_apply_alone * 1e-6) / 1e9,
-                          "frac": (4.0 * n * W + elt * alone_zero_bits) / (t_apply_alone * 1e-6) / 1e9 / peak,
-                          "conventional_gbs": apply_conv_bytes / (t_apply_alone * 1e-6) / 1e9}}
 
-    # The other two step kernels are bound by latency, not by a memory or arithmetic pipe.  What can be said against a
-    # peak is their issue rate: warp instructions per launch (ncu, profiles/step_kernels_c3.txt; C3 only, void once
-    # the kernels change) over the launch time, against 148 SMs x 4 schedulers x the SM clock.
+    def apply_at(t_us, zb=None):
+        alg = apply_alg_bytes if zb is None else 4.0 * n * W + elt * zb
+        return {"us_per_launch": t_us, "achieved": alg / (t_us * 1e-6) / 1e9, "frac": alg / (t_us * 1e-6) / 1e9 / peak,
+                "sector_traffic_gbs": apply_sector_bytes / (t_us * 1e-6) / 1e9, "sector_traffic_frac": apply_sector_bytes / (t_us * 1e-6) / 1e9 / peak,
+                "ncu_traffic_frac": (traffic / (t_us * 1e-6) / 1e9 / peak) if traffic else None,
+                "conventional_gbs": apply_conv_bytes / (t_us * 1e-6) / 1e9}
+
+    roofline = {"kernel": "apply_kernel", "bound": "hbm", "achieved": apply_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": apply_gbs / peak, "traffic": traffic, "us_per_launch": t_apply_in_step,
+                "how": "in-graph: replayed three-launch step (fill, apply, accept) minus the same step without its apply",
+                "masked_fraction": masked_frac, "algorithmic_bytes": apply_alg_bytes,
+                "sector_bytes": apply_sector_bytes, "sectors": {"untouched": sec_untouched, "overwritten": sec_overwritten, "read_and_rewritten": sec_mixed},
+                "in_step": apply_at(t_apply_in_step), "dominant_by_time": dominant,
+                "eager_event_interval": apply_at(t_apply),
+                "alone": dict(apply_at(t_apply_alone, alone_zero_bits),
+                              how="%d launches back to back over the logits ring (queued behind a primer kernel), last step's mask" % reps)}
+
+    # The fill and accept kernels are bound by latency, not by a memory or arithmetic pipe.  What can be said against a
+    # peak is their issue rate: warp instructions per launch (ncu) over the launch time, against 148 SMs x 4 schedulers
+    # x the SM clock.
     props = torch.cuda.get_device_properties(local_rank)
     issue_peak = props.multi_processor_count * 4 * (clocks["sm_max_mhz"] or 1965.0) * 1e6
-    warp_insts = {"fill": 1354736.0, "accept": 121532.0} if (args.workload == "C3" and n == 128) else {}
     latency_bound = {}
-    for name, t_us in (("fill", t_fill), ("accept", t_accept)):
-        wi = warp_insts.get(name)
-        latency_bound[name] = {"kernel": "fill_cluster_kernel" if name == "fill" else "accept_kernel", "bound": "alu",
+    for name, kernel, t_us in (("fill", "fill_cluster_kernel", t_fill), ("accept", "accept_kernel", t_accept)):
+        wi = ncu.get(kernel, {}).get("warp_instructions")
+        latency_bound[name] = {"kernel": kernel, "bound": "alu",
                                "achieved": (wi / (t_us * 1e-6)) if wi else None, "peak": issue_peak, "unit": "warp instructions/s",
                                "frac": (wi / (t_us * 1e-6) / issue_peak) if wi else None, "warp_instructions_per_launch": wi,
-                               "us_per_launch": t_us, "note": "latency-bound: chains of dependent loads, issue slots 4-11 % busy under ncu"}
+                               "us_per_launch": t_us, "note": "latency-bound: chains of dependent loads"}
 
     fw_steps = max(fill_work["steps"], 1)
     fill_bytes = (fill_work["merge_bytes"] + fill_work["check_bytes"] + fill_work["row_bytes"]) / fw_steps
@@ -445,12 +523,19 @@ def main():
                    "row_bytes": fill_work["row_bytes"] / fw_steps, "uncertain_candidates_per_launch": fill_work["check_tokens"] / fw_steps,
                    "gbs": fill_bytes / (t_fill * 1e-6) / 1e9, "frac_of_hbm_peak": fill_bytes / (t_fill * 1e-6) / 1e9 / peak,
                    "sampled_steps": fill_work["steps"]}
+    t_fa = eager_us["fill_apply"]
+    fused = {"kernel": "fill_cluster_kernel with the apply tail", "us_per_launch": t_fa, "us_fill_then_apply_as_two_launches": t_fill + t_apply,
+             "algorithmic_bytes": apply_alg_bytes - 4.0 * n * W + fill_bytes,
+             "achieved_gbs": (apply_alg_bytes - 4.0 * n * W + fill_bytes) / (t_fa * 1e-6) / 1e9,
+             "frac_of_hbm_peak": (apply_alg_bytes - 4.0 * n * W + fill_bytes) / (t_fa * 1e-6) / 1e9 / peak,
+             "note": "the launch lasts as long as its slowest request's token walks; the logits traffic of the other rows overlaps them"}
 
     # ---- end to end through the C ABI with host buffers ---------------------------------------
     # Every step: the step's logits come from pinned host memory, the masked logits go back to pinned host memory,
     # the step's token ids come from the host.  Two device buffers and two copy streams, as a serving loop would
     # have them: the upload of step t+1 and the download of step t-1 overlap the kernels of step t (PCIe is full
     # duplex); every dependency is an event, nothing is skipped.
+    e2e_mode = args.step if args.step != "no_apply" else "fill_apply"
     e2e_steps = max(4, min(args.steps, 16))
     host_in = torch.empty((n, s.V), dtype=tdtype).pin_memory()
     host_in.copy_(ring[0].cpu())
@@ -462,7 +547,7 @@ def main():
     torch.cuda.synchronize()
     h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for phase in ("warm", "timed"):
-        restart(fused)
+        restart(e2e_mode)
         torch.cuda.synchronize()
         if phase == "timed":
             h0.record()
@@ -486,10 +571,13 @@ def main():
             k = t % 2
             if t + 1 < e2e_steps:
                 upload(t + 1)
-            if not fused:
+            if e2e_mode == "three":
                 s.fill()
             main.wait_event(ev_in[k])
-            s.apply(dev_buf[k])
+            if e2e_mode == "fill_apply":
+                s.fill_apply(dev_buf[k])
+            else:
+                s.apply(dev_buf[k])
             ev_applied[k] = torch.cuda.Event()
             ev_applied[k].record(main)
             with torch.cuda.stream(s_out):
@@ -498,7 +586,7 @@ def main():
                 ev_out[k] = torch.cuda.Event()
                 ev_out[k].record(s_out)
             s.tokens.copy_(host_traj[t], non_blocking=True)
-            if fused:
+            if e2e_mode == "accept_fill":
                 s.accept_fill_device(s.tokens, restart_on_eos=True)
             else:
                 s.accept_device(s.tokens, restart_on_eos=True)
@@ -509,21 +597,38 @@ def main():
         torch.cuda.synchronize()
     e2e_us = dist_util.max_over_ranks(h0.elapsed_time(h1)) * 1e3 / e2e_steps
 
+    launch_text = {"fill_apply": "fill + apply in one launch, then accept", "three": "fill, apply, accept",
+                   "accept_fill": "apply, then accept + fill of the next mask in one launch"}[args.step]
+    classify_ms = sum(x["classify_ms"] for x in stats)
+    # the work behind a classified pair: token bytes the walks consume (viable trie nodes, no sharing between tokens),
+    # counted in a second compile of the first grammars into a pool of their own (the timed compile does not count)
+    cpool = XB.CachePool(s.tokenizer)
+    counted = [XB.Grammar(s.tokenizer, g.kind, g.text, pool=cpool, count_node_visits=True) for g in w.grammars[:16]]
+    cstats = [g.stats() for g in counted]
+    visits_per_pair = sum(x["node_visits"] for x in cstats) / max(sum(x["pairs_classified"] for x in cstats), 1)
+    for g in counted:
+        g.close()
+    cpool.close()
     line = {
         "metric": metric, "value": us_per_step, "unit": "us/step", "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": us_per_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "int32", "data": "synthetic",
-        "config": {"workload": args.workload, "batch": n, "global_batch": n * world, "vocab": s.V, "logits_dtype": w.dtype, "launch": "one CUDA graph per trajectory step: " + ("apply, then accept + fill of the next mask in one launch" if fused else "fill, apply, accept"),
+        "config": {"workload": args.workload, "batch": n, "global_batch": n * world, "vocab": s.V, "logits_dtype": w.dtype, "launch": "one CUDA graph per trajectory step: " + launch_text,
                    "grammars": len(w.grammars), "l2": "logits ring of %d buffers (%.0f MB) > 2 x L2" % (ring_n, ring_n * bytes_one / 1e6),
                    "parallelism": "replicas x%d" % world},
         "clocks": clocks,
+        "us_per_step_by_launch_structure": by_mode,
         "us_per_step_with_8_steps_per_graph": multi_us,
-        "kernels_us": {"fill": t_fill, "apply": t_apply, "accept": t_accept, "accept_fill": eager_us["accept_fill"]},
+        "kernels_us": {"fill": t_fill, "apply": t_apply, "accept": t_accept, "accept_fill": eager_us["accept_fill"], "fill_apply": eager_us["fill_apply"],
+                       "apply_in_step": t_apply_in_step},
         "apply_gbs": apply_gbs,
         "cache_build": {"seconds": build_ms / 1e3, "compile_wall_s": compile_s, "compile_threads": args.compile_threads or min(16, os.cpu_count() or 1), "pairs_classified": pairs, "pairs_per_s": pairs / max(build_ms / 1e3, 1e-9),
+                        "pairs_per_s_of_wall_time": pairs / max(compile_s, 1e-9),
                         "pairs_dense": pairs_dense, "pairs_dense_per_s": pairs_dense / max(build_ms / 1e3, 1e-9),
-                        "classify_kernel_ms": sum(x["classify_ms"] for x in stats),
-                        "pairs_per_s_classify_kernel": pairs / max(sum(x["classify_ms"] for x in stats) / 1e3, 1e-9),
+                        "classify_kernel_ms": classify_ms,
+                        "pairs_per_s_classify_kernel": pairs / max(classify_ms / 1e3, 1e-9),
+                        "viable_node_visits_per_pair": visits_per_pair,
+                        "viable_node_visits_per_s": visits_per_pair * pairs / max(classify_ms / 1e3, 1e-9),
                         "entries_built": sum(x["n_entries_built"] for x in stats), "entries_reused": sum(x["n_entries_reused"] for x in stats),
                         "entries_shared_by_state_compression": sum(x["n_entries_shared"] for x in stats), "states": sum(x["n_states"] for x in stats),
                         "frontend_ms": sum(x["frontend_ms"] for x in stats),
@@ -532,12 +637,17 @@ def main():
         "roofline": roofline,
         "roofline_latency_bound_kernels": latency_bound,
         "fill_streaming": fill_stream,
+        "fill_and_apply_in_one_launch": fused,
         "e2e": {"value": e2e_us, "unit": "us/step", "h2d_bytes_per_step": bytes_one + 4 * n, "d2h_bytes_per_step": bytes_one, "steps": e2e_steps},
         "gpu_launches": timed_launches,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        us, threads, sample = oracle_leg(w, min(args.steps, 6), 0)
-        line["cpu_baseline"] = {"value": us, "unit": "us/step", "cores": threads, "kind": "oracle", "sample": sample}
+        us, threads, sample = oracle_leg(w, args.steps, args.warmup)
+        us1, _, sample1 = oracle_leg(w, args.steps, args.warmup, threads=1, n_req=4, budget_s=12.0)
+        n_built = sum(x["n_entries_built"] for x in stats)
+        line["cpu_baseline"] = {"value": us, "unit": "us/step", "cores": threads, "kind": "oracle", "sample": sample,
+                                "single_thread": {"value": us1, "unit": "us/step", "us_per_mask": us1 / n, "sample": sample1},
+                                "cache_build": {"all_cores": oracle_cache_build_leg(w, n_built, threads), "single_thread": oracle_cache_build_leg(w, n_built, 1, n_positions=12, budget_s=6.0)}}
     s.close()
     if rank == 0:
         print(json.dumps(line))

@@ -114,6 +114,9 @@ typedef struct {
   int64_t jit_arena_bytes;    /* size of the pool's first just-in-time arena (entries built inside the decode loop take
                                  their space from it on the device); when one fills up the next is twice as large.
                                  <= 0 = default (32 MiB).  Only the pool's first just-in-time compile sets it. */
+  int32_t count_node_visits;  /* non-zero: the classification also counts the token bytes its walks consume
+                                 (xg_grammar_stats_t.node_visits); statistics only, costs an atomic per warp. */
+  int32_t reserved;
 } xg_compile_options_t;
 
 /* ---- grammar compilation (Section 3.5 "compilation stage"; Sections 3.2, 3.3, 3.4) ---------
@@ -205,6 +208,8 @@ typedef struct {
   int64_t n_entries_shared;     /* scannable states that use the entry of an equivalent state of their rule
                                    (repetition state compression, Section 3.6) instead of one of their own */
   double classify_ms;           /* device time of the classification kernel alone (inside cache_build_ms) */
+  int64_t node_visits;          /* with opt->count_node_visits: token bytes consumed by the classification walks of this
+                                   compile, i.e. viable trie nodes visited without sharing between tokens (else 0) */
 } xg_grammar_stats_t;
 xg_status_t xg_grammar_stats(const xg_grammar_t* g, xg_grammar_stats_t* out);
 
@@ -340,6 +345,22 @@ xg_status_t xg_accept_token_and_fill_next_bitmask(xg_matcher_t* const* matchers,
                                                   int32_t restart_on_eos, int32_t* bitmask_dev,
                                                   int64_t row_stride_words, int32_t* fill_status_dev,
                                                   void* stream);
+
+/* xg_fill_and_apply_token_bitmask: xg_fill_next_token_bitmask followed by xg_apply_token_bitmask on
+ * rows 0..batch-1 of logits_dev, in one launch (Section 2.1: the mask is generated, then the logits of
+ * the tokens it rules out are set to -inf).  Each request's mask row is applied to its logits row
+ * straight from the on-chip copy the fill has just produced, so the mask is not read back from
+ * memory, there is no kernel boundary between the two steps, and the rows of requests whose fill is
+ * short are masked while other requests still check their uncertain tokens.  The results are exactly
+ * those of the two calls in that order: bitmask_dev and status_dev as xg_fill_next_token_bitmask
+ * writes them (the row of a request whose status is not XG_OK is all zero, so all of its logits
+ * become -inf); logits as xg_apply_token_bitmask leaves them (same layout, alignment rule, dtype and
+ * bit patterns; logits row i belongs to matchers[i]).  Where the vocabulary is too large for the
+ * one-launch fill the call enqueues the steps one after the other. */
+xg_status_t xg_fill_and_apply_token_bitmask(xg_matcher_t* const* matchers, int32_t batch,
+                                            int32_t* bitmask_dev, int64_t row_stride_words,
+                                            int32_t* status_dev, void* logits_dev, xg_dtype_t dtype,
+                                            int64_t logits_row_stride_elems, void* stream);
 
 #ifdef __cplusplus
 }

@@ -29,7 +29,7 @@ EXPORTS = [
     "xg_compile_grammar", "xg_grammar_destroy", "xg_grammar_get_tables", "xg_grammar_get_rule_hashes", "xg_grammar_get_cache_entry", "xg_grammar_get_state_classes", "xg_grammar_stats", "xg_jit_service",
     "xg_matcher_create", "xg_matcher_reset", "xg_matcher_destroy", "xg_matcher_is_terminated", "xg_matcher_next_fill_work",
     "xg_fill_next_token_bitmask", "xg_fill_next_token_bitmask_static", "xg_apply_token_bitmask", "xg_accept_token",
-    "xg_accept_token_ex", "xg_accept_token_and_fill_next_bitmask",
+    "xg_accept_token_ex", "xg_accept_token_and_fill_next_bitmask", "xg_fill_and_apply_token_bitmask",
 ]
 XG_STATIC_FILL_MAX_BATCH = 1024
 
@@ -42,7 +42,8 @@ class XgError(RuntimeError):
 
 class CompileOptions(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("inline_max_states", C.c_int32), ("max_rule_states", C.c_int32), ("build_cache", C.c_int32),
-                ("no_state_compression", C.c_int32), ("jit", C.c_int32), ("jit_precompute", C.c_int32), ("jit_arena_bytes", C.c_int64)]
+                ("no_state_compression", C.c_int32), ("jit", C.c_int32), ("jit_precompute", C.c_int32), ("jit_arena_bytes", C.c_int64),
+                ("count_node_visits", C.c_int32), ("reserved", C.c_int32)]
 
 
 class FillWork(C.Structure):
@@ -77,7 +78,7 @@ class GrammarStats(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_rules", "n_states", "n_scannable", "n_classes", "n_entries_built", "n_entries_reused")] + \
                [(n, C.c_int64) for n in ("pairs_classified", "total_accepted", "total_rejected", "total_uncertain")] + \
                [("kind_count", C.c_int32 * 3), ("pad", C.c_int32), ("cache_bytes", C.c_int64), ("frontend_ms", C.c_double), ("cache_build_ms", C.c_double), ("total_checked", C.c_int64),
-                ("n_entries_shared", C.c_int64), ("classify_ms", C.c_double)]
+                ("n_entries_shared", C.c_int64), ("classify_ms", C.c_double), ("node_visits", C.c_int64)]
 
 
 _lib = None
@@ -124,6 +125,7 @@ def lib():
         L.xg_accept_token.argtypes = [vp, i32, vp, vp, vp]
         L.xg_accept_token_ex.argtypes = [vp, i32, vp, vp, i32, vp]
         L.xg_accept_token_and_fill_next_bitmask.argtypes = [vp, i32, vp, vp, i32, vp, i64, vp, vp]
+        L.xg_fill_and_apply_token_bitmask.argtypes = [vp, i32, vp, i64, vp, vp, C.c_int, i64, vp]
         _lib = L
     return _lib
 
@@ -176,11 +178,11 @@ class CachePool:
 class Grammar:
     def __init__(self, tokenizer: Optional[Tokenizer], kind, text: str, pool: Optional[CachePool] = None, root: Optional[str] = None,
                  inline_max_states: int = -1, build_cache: bool = True, stream: int = 0, state_compression: bool = True,
-                 jit: bool = False, jit_precompute: int = 0, jit_arena_bytes: int = 0):
+                 jit: bool = False, jit_precompute: int = 0, jit_arena_bytes: int = 0, count_node_visits: bool = False):
         kind = KIND_BY_NAME.get(kind, kind)
         raw = text.encode("utf-8") if isinstance(text, str) else text
         opt = CompileOptions(C.sizeof(CompileOptions), inline_max_states, 0, 1 if build_cache else 0, 0 if state_compression else 1,
-                             1 if jit else 0, int(jit_precompute), int(jit_arena_bytes))
+                             1 if jit else 0, int(jit_precompute), int(jit_arena_bytes), 1 if count_node_visits else 0, 0)
         h = C.c_void_p()
         _check(lib().xg_compile_grammar(tokenizer.h if tokenizer else None, pool.h if pool else None, kind, raw, len(raw),
                                         root.encode() if root else None, C.byref(opt), stream, C.byref(h)))
@@ -291,6 +293,11 @@ class Batch:
         """Same masks as fill_next_token_bitmask, without any device allocation (at most
         XG_STATIC_FILL_MAX_BATCH requests; calls must not overlap on the GPU)."""
         _check(lib().xg_fill_next_token_bitmask_static(self.handles, self.n, bitmask_ptr, row_stride_words, status_ptr or None, stream))
+
+    def fill_and_apply_token_bitmask(self, bitmask_ptr: int, row_stride_words: int, status_ptr: int, logits_ptr: int, dtype,
+                                     logits_row_stride: int, stream: int = 0):
+        _check(lib().xg_fill_and_apply_token_bitmask(self.handles, self.n, bitmask_ptr, row_stride_words, status_ptr or None, logits_ptr,
+                                                     DTYPE_BY_NAME.get(dtype, dtype), logits_row_stride, stream))
 
     def accept_token(self, token_ids_ptr: int, status_ptr: int = 0, stream: int = 0, restart_on_eos: bool = False):
         if restart_on_eos:

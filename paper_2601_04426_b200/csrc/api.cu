@@ -156,6 +156,7 @@ struct xg_grammar {
   std::vector<int> entry_chunk;         // [n_states] pool chunk that holds the state's entry (-1: none)
   std::vector<int> chunk_refs;          // pool chunks this grammar keeps alive
   xg_grammar_stats_t stats{};
+  bool count_visits = false;            // add up the bytes the classification walks consume (statistics only)
   JitState jit;
   // buffers behind xg_grammar_get_cache_entry's view
   mutable std::vector<int32_t> view_list, view_unc;
@@ -399,7 +400,17 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
     dim3 grid(((V + 255) / 256 + kClassifySpan - 1) / kClassifySpan, n);
     cudaEvent_t* ev = pool.timing_events();            // device time of the classification itself, for the statistics
     if (ev) cudaEventRecord(ev[0], stream);
-    classify_kernel<<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, acc, unc, unr, d_over, d_over_count, over_cap);
+    if (g->count_visits) {
+      unsigned long long* d_visits = (unsigned long long*)pool.scratch(8, sizeof(unsigned long long));
+      if (!d_visits) return set_error(XG_ERR_OOM, "cache build scratch allocation failed");
+      XG_CUDA_C(cudaMemsetAsync(d_visits, 0, sizeof(unsigned long long), stream));
+      classify_kernel<true><<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, acc, unc, unr, d_over, d_over_count, over_cap, d_visits);
+      unsigned long long visits = 0;
+      XG_CUDA_C(cudaMemcpyAsync(&visits, d_visits, sizeof visits, cudaMemcpyDeviceToHost, stream));
+      XG_CUDA_C(cudaStreamSynchronize(stream));
+      g->stats.node_visits += (int64_t)visits;
+    } else
+    classify_kernel<false><<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, acc, unc, unr, d_over, d_over_count, over_cap, nullptr);
     XG_CUDA_C(cudaGetLastError());
     if (ev) cudaEventRecord(ev[1], stream);
     int over[2] = {0, 0};
@@ -409,14 +420,13 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
     if (over[0] > over_cap) { cleanup(); return set_error(XG_ERR_CAPACITY, "too many token walks exceeded the fast path"); }
     for (int done = 0; done < over[0];) {          // exact fallback, a bounded number of pairs per round
       const int round = std::min(over[0] - done, 4096);
-      uint32_t* s_st = nullptr; int32_t* s_org = nullptr; int32_t* s_lsb = nullptr;
-      cudaError_t e1 = cudaMalloc(&s_st, (size_t)round * kSlowCap * 4), e2 = cudaMalloc(&s_org, (size_t)round * kSlowCap * 4),
-                  e3 = cudaMalloc(&s_lsb, (size_t)round * (kSlowMaxBytes + 2) * 4);
-      if (e1 == cudaSuccess && e2 == cudaSuccess && e3 == cudaSuccess)
-        classify_slow_kernel<<<(round + 63) / 64, 64, 0, stream>>>(g->host_view, v, d_pos, d_over + done, round, s_st, s_org, s_lsb, acc, unc, unr, d_over_count + 1);
-      cudaError_t e4 = cudaStreamSynchronize(stream);
-      cudaFree(s_st); cudaFree(s_org); cudaFree(s_lsb);
-      if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) { cleanup(); return set_error(XG_ERR_CUDA, "slow classification failed"); }
+      // the exact walks' scratch comes from the pool too (grow-only, reused by later compiles)
+      uint32_t* s_st = (uint32_t*)pool.scratch(9, (size_t)round * kSlowCap * 4);
+      int32_t* s_org = (int32_t*)pool.scratch(10, (size_t)round * kSlowCap * 4);
+      int32_t* s_lsb = (int32_t*)pool.scratch(14, (size_t)round * (kSlowMaxBytes + 2) * 4);
+      if (!s_st || !s_org || !s_lsb) { cleanup(); return set_error(XG_ERR_OOM, "slow classification scratch allocation failed"); }
+      classify_slow_kernel<<<(round + 63) / 64, 64, 0, stream>>>(g->host_view, v, d_pos, d_over + done, round, s_st, s_org, s_lsb, acc, unc, unr, d_over_count + 1);
+      if (cudaStreamSynchronize(stream) != cudaSuccess) { cleanup(); return set_error(XG_ERR_CUDA, "slow classification failed"); }
       done += round;
     }
     if (over[0] > 0) {
@@ -665,7 +675,7 @@ static xg_status_t jit_enqueue_build(JitPool* jp, xg_grammar* g, const std::vect
   XG_CUDA(cudaMemsetAsync(unc, 0, row_bytes * n, stream));
   XG_CUDA(cudaMemsetAsync(unr, 0, row_bytes * n, stream));
   XG_CUDA(cudaMemsetAsync(sc.over_count, 0, 2 * sizeof(int), stream));
-  classify_kernel<<<dim3(((V + 255) / 256 + kClassifySpan - 1) / kClassifySpan, n), 256, 0, stream>>>(g->host_view, v, sc.pos, acc, unc, unr, sc.over, sc.over_count, 64);
+  classify_kernel<false><<<dim3(((V + 255) / 256 + kClassifySpan - 1) / kClassifySpan, n), 256, 0, stream>>>(g->host_view, v, sc.pos, acc, unc, unr, sc.over, sc.over_count, 64, nullptr);
   count_kernel<<<n, 256, 0, stream>>>(acc, unc, W, sc.counts);
   plan_kernel<<<1, 1024, 0, stream>>>(sc.counts, n, V, W, sc.plan, sc.total);
   jit_reserve_kernel<<<1, 32, 0, stream>>>(sc.plan, n, sc.total, arena->d_used, arena->cap_words, sc.over_count, sc.result);
@@ -828,7 +838,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   *out = nullptr;
   if (!text) return set_error(XG_ERR_INVALID_ARG, "text is NULL");
   FrontendOptions fo;
-  bool build_cache = tok != nullptr, compress = true, jit = false;
+  bool build_cache = tok != nullptr, compress = true, jit = false, count_visits = false;
   int jit_precompute = 0;
   long long jit_arena_words = 0;
   if (opt) {
@@ -839,9 +849,11 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     if (opt->struct_size >= 20 && opt->no_state_compression != 0) compress = false;
     if (opt->struct_size >= 28 && opt->jit != 0) { jit = true; jit_precompute = std::max(0, opt->jit_precompute); }
     if (opt->struct_size >= 40 && opt->jit_arena_bytes > 0) jit_arena_words = std::max<long long>(1024, opt->jit_arena_bytes / 4);
+    if (opt->struct_size >= 44 && opt->count_node_visits != 0) count_visits = true;
   }
   if (pool && pool->impl->owner() != (const void*)tok) return set_error(XG_ERR_INVALID_ARG, "the pool belongs to another tokenizer");
   std::unique_ptr<xg_grammar> g(new xg_grammar());
+  g->count_visits = count_visits;
   const double t0 = now_ms();
   try {
     g->flat = compile_frontend((int)kind, std::string(text, len), root_rule ? root_rule : "root", fo);
@@ -1278,9 +1290,13 @@ static xg_status_t batch_slot(xg_matcher_t* const* matchers, int32_t batch, cons
   return XG_OK;
 }
 
-// accept (when token_ids_dev is given) and fill; the two public entry points below are this
+static xg_status_t apply_rows(void* logits_dev, xg_dtype_t dtype, int32_t rows, int32_t vocab_size, int64_t logits_row_stride_elems,
+                              const int32_t* bitmask_dev, int64_t mask_row_stride_words, const int32_t* row_indices_dev, void* stream);
+
+// accept (when token_ids_dev is given), fill, and apply (when logits_dev is given)
 static xg_status_t accept_and_fill(xg_matcher_t* const* matchers, int32_t batch, const int32_t* token_ids_dev, int32_t* accept_status_dev,
-                                   int restart_on_eos, int32_t* bitmask_dev, int64_t row_stride_words, int32_t* status_dev, void* stream) {
+                                   int restart_on_eos, int32_t* bitmask_dev, int64_t row_stride_words, int32_t* status_dev, void* stream,
+                                   void* logits_dev = nullptr, xg_dtype_t dtype = XG_F32, int64_t logits_row_stride_elems = 0) {
   const xg_tokenizer* tok = nullptr;
   BatchSlot* slot = nullptr;
   xg_status_t st = batch_slot(matchers, batch, &tok, &slot);
@@ -1297,14 +1313,21 @@ static xg_status_t accept_and_fill(xg_matcher_t* const* matchers, int32_t batch,
     int blocks = kMaxClusterBlocks, threads = 256;
     if (per_request < 2048) threads = 128;     // measured: fewer blocks or narrower blocks than this are slower even at batch 256
     const size_t smem = 2 * sizeof(uint32_t) * (size_t)((W + blocks - 1) / blocks);
+    MatcherDev* const* dm = slot->dev_matchers;
+    const dim3 grid(blocks, batch), block(threads);
+    cudaStream_t cs = (cudaStream_t)stream;
     if (token_ids_dev)
-      XG_CUDA(launch_step_kernel(fill_cluster_kernel<true>, dim3(blocks, batch), dim3(threads), smem, (cudaStream_t)stream, blocks,
-                                 (MatcherDev* const*)slot->dev_matchers, tok->dev, bitmask_dev, (long long)row_stride_words, status_dev,
-                                 token_ids_dev, accept_status_dev, restart_on_eos));
+      XG_CUDA(launch_step_kernel(fill_cluster_kernel<true, 0>, grid, block, smem, cs, blocks, dm, tok->dev, bitmask_dev, (long long)row_stride_words,
+                                 status_dev, token_ids_dev, accept_status_dev, restart_on_eos, (void*)nullptr, 0LL));
+    else if (!logits_dev)
+      XG_CUDA(launch_step_kernel(fill_cluster_kernel<false, 0>, grid, block, smem, cs, blocks, dm, tok->dev, bitmask_dev, (long long)row_stride_words,
+                                 status_dev, (const int32_t*)nullptr, (int32_t*)nullptr, 0, (void*)nullptr, 0LL));
+    else if (dtype == XG_BF16)
+      XG_CUDA(launch_step_kernel(fill_cluster_kernel<false, 8>, grid, block, smem, cs, blocks, dm, tok->dev, bitmask_dev, (long long)row_stride_words,
+                                 status_dev, (const int32_t*)nullptr, (int32_t*)nullptr, 0, logits_dev, (long long)logits_row_stride_elems));
     else
-      XG_CUDA(launch_step_kernel(fill_cluster_kernel<false>, dim3(blocks, batch), dim3(threads), smem, (cudaStream_t)stream, blocks,
-                                 (MatcherDev* const*)slot->dev_matchers, tok->dev, bitmask_dev, (long long)row_stride_words, status_dev,
-                                 (const int32_t*)nullptr, (int32_t*)nullptr, 0));
+      XG_CUDA(launch_step_kernel(fill_cluster_kernel<false, 4>, grid, block, smem, cs, blocks, dm, tok->dev, bitmask_dev, (long long)row_stride_words,
+                                 status_dev, (const int32_t*)nullptr, (int32_t*)nullptr, 0, logits_dev, (long long)logits_row_stride_elems));
     return XG_OK;
   }
   if (token_ids_dev) {
@@ -1319,6 +1342,7 @@ static xg_status_t accept_and_fill(xg_matcher_t* const* matchers, int32_t batch,
   check_kernel<<<grid_check, 256, 0, (cudaStream_t)stream>>>(slot->dev_matchers, tok->dev, bitmask_dev, (long long)row_stride_words,
                                                              status_dev, slot->status, slot->done_count);
   XG_CUDA(cudaGetLastError());
+  if (logits_dev) return apply_rows(logits_dev, dtype, batch, tok->vocab_size, logits_row_stride_elems, bitmask_dev, row_stride_words, nullptr, stream);
   return XG_OK;
 }
 
@@ -1334,6 +1358,20 @@ xg_status_t xg_accept_token_and_fill_next_bitmask(xg_matcher_t* const* matchers,
   NvtxRange nvtx_range("xg_accept_token_and_fill_next_bitmask");
   if (!token_ids_dev) return set_error(XG_ERR_INVALID_ARG, "token_ids_dev is NULL");
   return accept_and_fill(matchers, batch, token_ids_dev, accept_status_dev, restart_on_eos ? 1 : 0, bitmask_dev, row_stride_words, fill_status_dev, stream);
+}
+
+xg_status_t xg_fill_and_apply_token_bitmask(xg_matcher_t* const* matchers, int32_t batch, int32_t* bitmask_dev, int64_t row_stride_words,
+                                            int32_t* status_dev, void* logits_dev, xg_dtype_t dtype, int64_t logits_row_stride_elems,
+                                            void* stream) {
+  NvtxRange nvtx_range("xg_fill_and_apply_token_bitmask");
+  if (!logits_dev) return set_error(XG_ERR_INVALID_ARG, "logits_dev is NULL");
+  if (dtype != XG_F32 && dtype != XG_BF16) return set_error(XG_ERR_INVALID_ARG, "unknown dtype");
+  if (!matchers || batch <= 0 || !matchers[0]) return set_error(XG_ERR_INVALID_ARG, "empty batch");
+  const int elt = dtype == XG_BF16 ? 2 : 4;
+  if (logits_row_stride_elems < matchers[0]->grammar->tok->vocab_size) return set_error(XG_ERR_INVALID_ARG, "bad shape or stride");
+  if (((uintptr_t)logits_dev & 15) || ((logits_row_stride_elems * elt) & 15))
+    return set_error(XG_ERR_INVALID_ARG, "logits rows must start on 16-byte boundaries");
+  return accept_and_fill(matchers, batch, nullptr, nullptr, 0, bitmask_dev, row_stride_words, status_dev, stream, logits_dev, dtype, logits_row_stride_elems);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1417,11 +1455,16 @@ xg_status_t xg_apply_token_bitmask(void* logits_dev, xg_dtype_t dtype, int32_t b
                                    const int32_t* bitmask_dev, int64_t mask_row_stride_words, const int32_t* row_indices_dev,
                                    int32_t n_rows, void* stream) {
   NvtxRange nvtx_range("xg_apply_token_bitmask");
+  const int rows = row_indices_dev ? n_rows : batch;
+  return apply_rows(logits_dev, dtype, rows, vocab_size, logits_row_stride_elems, bitmask_dev, mask_row_stride_words, row_indices_dev, stream);
+}
+
+static xg_status_t apply_rows(void* logits_dev, xg_dtype_t dtype, int32_t rows, int32_t vocab_size, int64_t logits_row_stride_elems,
+                              const int32_t* bitmask_dev, int64_t mask_row_stride_words, const int32_t* row_indices_dev, void* stream) {
   if (!logits_dev || !bitmask_dev) return set_error(XG_ERR_INVALID_ARG, "NULL buffer");
   if (dtype != XG_F32 && dtype != XG_BF16) return set_error(XG_ERR_INVALID_ARG, "unknown dtype");
   if (vocab_size <= 0 || logits_row_stride_elems < vocab_size || mask_row_stride_words < (vocab_size + 31) / 32)
     return set_error(XG_ERR_INVALID_ARG, "bad shape or stride");
-  const int rows = row_indices_dev ? n_rows : batch;
   if (rows == 0 && row_indices_dev) return XG_OK;
   if (rows <= 0) return set_error(XG_ERR_INVALID_ARG, "no rows");
   const int elt = dtype == XG_BF16 ? 2 : 4;

@@ -927,27 +927,7 @@ struct Compiler {
     return touched;
   }
 
-  // for each rule, whether it can reach itself through references
-  std::vector<char> recursive_rules() {
-    int R = n_rules();
-    std::vector<std::set<int>> adj(R);
-    for (int r = 0; r < R; ++r) for (auto& es : b.rules[r].out) for (const Edge& e : es) if (e.kind == Edge::kRef) adj[r].insert(e.rule);
-    std::vector<char> rec(R, 0);
-    for (int r = 0; r < R; ++r) {
-      std::vector<char> seen(R, 0);
-      std::vector<int> stack(adj[r].begin(), adj[r].end());
-      while (!stack.empty()) {
-        int u = stack.back(); stack.pop_back();
-        if (u == r) { rec[r] = 1; break; }
-        if (seen[u]) continue;
-        seen[u] = 1;
-        for (int v : adj[u]) stack.push_back(v);
-      }
-    }
-    return rec;
-  }
-
-  // Replace references to small non-recursive rules by a copy of their automaton.  A rule that
+  // Replace references to small rules by a copy of their automaton.  A rule that
   // is referenced from a single place may be larger (inlining it duplicates nothing); this also
   // folds alternatives such as the tool calls of a TagDispatch into one deterministic automaton.
   // A rule used a few times may also be somewhat larger as long as size x uses stays bounded
@@ -958,7 +938,6 @@ struct Compiler {
     if (opt.inline_max_states <= 0) return;
     const int single_use_max = std::max(64, opt.inline_max_states);
     int R = n_rules();
-    std::vector<char> rec = recursive_rules();
     std::vector<int> uses(R, 0);
     for (const Fsm& f : b.rules) for (auto& es : f.out) for (const Edge& e : es) if (e.kind == Edge::kRef) ++uses[e.rule];
     std::vector<char> candidate(R, 0), done(R, 0);
@@ -996,7 +975,15 @@ struct Compiler {
         g.out[s] = keep;
       }
       if (changed) { b.rules[r] = normalize(g, opt.max_rule_states); renormalized[r] = 1; }
-      candidate[r] = !rec[r] && r != root && b.rules[r].size() <= single_use_max && !b.keep_as_rule.count(r);
+      // A rule on a cycle of references may be copied into its users too: each rule is finished before anything
+      // copies it and is copied as it then stands, so the expansion ends; a cycle keeps the rule whose processing
+      // began first, which ends up referring to itself (any-JSON: object, member and array fold into value).  One
+      // level of nesting is then one rule, not three: a closing bracket completes one rule instead of a cascade,
+      // and tokens that run from a string into the punctuation behind it stay inside their rule (Section 3.4: only
+      // tokens that leave the rule are context-dependent).
+      bool self_reference = false;
+      for (auto& es : b.rules[r].out) for (const Edge& e : es) self_reference = self_reference || (e.kind == Edge::kRef && e.rule == r);
+      candidate[r] = !self_reference && r != root && b.rules[r].size() <= single_use_max && !b.keep_as_rule.count(r);
     };
     for (int r = 0; r < R; ++r) process(r);
   }

@@ -170,10 +170,13 @@ __device__ __forceinline__ const uint32_t* stage_class_bits(const GrammarDev& g,
 // ------------------------------------------------------------------------------------------
 constexpr int kClassifySpan = 8;      // vocabulary blocks of 256 ranks per thread block
 
+// kCount: also add up the bytes the walks consume (viable trie nodes visited, without any sharing between tokens)
+// into *visits -- the work the classification actually does, as opposed to the (position, token) pairs it decides.
+template <bool kCount>
 __global__ void __launch_bounds__(256)
 classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
                 uint32_t* __restrict__ acc_id, uint32_t* __restrict__ unc_id, uint32_t* __restrict__ unc_rank,
-                int2* __restrict__ overflow, int* __restrict__ overflow_count, int overflow_cap) {
+                int2* __restrict__ overflow, int* __restrict__ overflow_count, int overflow_cap, unsigned long long* __restrict__ visits) {
   __shared__ uint32_t sh_st[1];
   __shared__ int32_t sh_org[1];
   __shared__ uint32_t sh_class[kSharedClasses * 8];
@@ -214,7 +217,7 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
   for (int i = 0; i < kClassifySpan; ++i) {
     if (!((live_blocks >> i) & 1u)) continue;
     const int rank = ((blockIdx.x * kClassifySpan + i) << 8) + (int)threadIdx.x;
-    int cls = 0;
+    int cls = 0, walked = 0;
     bool live = rank < v.vocab_size && !v.never[rank];
     uint32_t off = 0;
     if (live) {
@@ -235,6 +238,7 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
         c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1;
         c.i_st = sh_st; c.i_org = sh_org; c.i_cnt = 1; c.i_idx = 0;
         consumed = token_walk<int16_t>(g, class_bits, c, v.bytes + off, len, true, st, org, kFastCap, lsb, &flags, nullptr);
+        walked = consumed;
       }
       if (flags & kWalkOverflow) {
         int slot = atomicAdd(overflow_count, 1);
@@ -249,6 +253,10 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
     }
     const uint32_t ballot = __ballot_sync(0xFFFFFFFFu, cls == 2);
     if ((threadIdx.x & 31) == 0 && rank < v.vocab_size) unc_rank[(size_t)pos * v.n_words + (rank >> 5)] = ballot;
+    if (kCount) {
+      const int sum = __reduce_add_sync(0xFFFFFFFFu, walked);
+      if ((threadIdx.x & 31) == 0 && sum) atomicAdd(visits, (unsigned long long)sum);
+    }
   }
 }
 
@@ -1044,6 +1052,83 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
 }
 
 // ------------------------------------------------------------------------------------------
+// Mask apply (Section 2.1): logits of disallowed tokens become -inf, in place, one pass.
+// One 16-byte vector per thread and step.  A vector whose tokens are all allowed is skipped
+// (neither read nor written); one whose tokens are all disallowed is overwritten without being
+// read; only mixed vectors are read, blended and written back.
+// ------------------------------------------------------------------------------------------
+template <int ELEMS>
+__device__ __forceinline__ uint4 blend_ninf(uint4 x, uint32_t bits) {
+  if (ELEMS == 8) {
+    // four allowed-bits -> four bytes of 0x00 / 0xFF (a multiply spreads the bits to the bytes' low bits, a second
+    // one fills the bytes), then each byte is doubled into the 16-bit lane it stands for
+    const uint32_t lo = (((bits & 0xFu) * 0x00204081u) & 0x01010101u) * 0xFFu;
+    const uint32_t hi = ((((bits >> 4) & 0xFu) * 0x00204081u) & 0x01010101u) * 0xFFu;
+    const uint32_t k0 = __byte_perm(lo, 0u, 0x1100), k1 = __byte_perm(lo, 0u, 0x3322);
+    const uint32_t k2 = __byte_perm(hi, 0u, 0x1100), k3 = __byte_perm(hi, 0u, 0x3322);
+    constexpr uint32_t kNinf2 = 0xFF80FF80u;
+    return make_uint4((x.x & k0) | (kNinf2 & ~k0), (x.y & k1) | (kNinf2 & ~k1), (x.z & k2) | (kNinf2 & ~k2), (x.w & k3) | (kNinf2 & ~k3));
+  }
+  if (!(bits & 1u)) x.x = 0xFF800000u;
+  if (!(bits & 2u)) x.y = 0xFF800000u;
+  if (!(bits & 4u)) x.z = 0xFF800000u;
+  if (!(bits & 8u)) x.w = 0xFF800000u;
+  return x;
+}
+
+// The vectors [v_begin, v_end) of one row, by `n_threads` threads of which this is thread `tid`; word_at(w) gives
+// word w of the row's mask.  Each thread handles four vectors per iteration: the four mask tests first, then the
+// loads of the mixed vectors (independent, all in flight together), then the stores.
+template <int ELEMS, typename MaskFn>   // elements per 16-byte vector: 8 (bf16) or 4 (fp32)
+__device__ __forceinline__ void apply_vectors(uint4* __restrict__ base, int v_begin, int v_end, int tid, int n_threads, MaskFn word_at) {
+  constexpr uint32_t kAll = (1u << ELEMS) - 1;
+  const uint4 ninf = ELEMS == 8 ? make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u)
+                                : make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
+  for (int v0 = v_begin + tid; v0 < v_end; v0 += 4 * n_threads) {
+    uint32_t bits[4];
+    uint4 x[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int vi = v0 + u * n_threads;
+      const int first = vi * ELEMS;
+      bits[u] = vi < v_end ? ((word_at(first >> 5) >> (first & 31)) & kAll) : kAll;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (bits[u] != kAll && bits[u] != 0) x[u] = __ldcs(&base[v0 + u * n_threads]);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (bits[u] == kAll) continue;
+      __stcs(&base[v0 + u * n_threads], bits[u] == 0 ? ninf : blend_ninf<ELEMS>(x[u], bits[u]));
+    }
+  }
+}
+
+// the elements behind a row's last whole vector (vocab_size not a multiple of the vector width)
+template <int ELEMS, typename MaskFn>
+__device__ __forceinline__ void apply_ragged_tail(void* row_base, int vocab_size, int tid, int n_threads, MaskFn word_at) {
+  for (int c = (vocab_size / ELEMS) * ELEMS + tid; c < vocab_size; c += n_threads) {
+    if ((word_at(c >> 5) >> (c & 31)) & 1u) continue;
+    if (ELEMS == 8) ((uint16_t*)row_base)[c] = 0xFF80u;
+    else ((uint32_t*)row_base)[c] = 0xFF800000u;
+  }
+}
+
+// grid = (blocks per row, rows)
+template <int ELEMS>
+__global__ void __launch_bounds__(256)
+apply_kernel(void* __restrict__ logits, int vocab_size, long long row_stride_elems, const uint32_t* __restrict__ bitmask,
+             long long mask_stride, const int32_t* __restrict__ row_indices) {
+  step_kernel_prologue();
+  const int r = row_indices ? row_indices[blockIdx.y] : blockIdx.y;
+  const uint32_t* mrow = bitmask + (long long)r * mask_stride;
+  void* row_base = ELEMS == 8 ? (void*)((uint16_t*)logits + (long long)r * row_stride_elems) : (void*)((uint32_t*)logits + (long long)r * row_stride_elems);
+  auto word_at = [&](int w) { return __ldg(&mrow[w]); };
+  apply_vectors<ELEMS>((uint4*)row_base, 0, vocab_size / ELEMS, blockIdx.x * blockDim.x + threadIdx.x, gridDim.x * blockDim.x, word_at);
+  if (blockIdx.x == 0) apply_ragged_tail<ELEMS>(row_base, vocab_size, threadIdx.x, blockDim.x, word_at);
+}
+
+// ------------------------------------------------------------------------------------------
 // Per-step mask in one launch: a thread-block cluster of two to eight blocks per request.  Block
 // r of the cluster keeps slice r of the request's row in its shared memory.
 //   1. every block merges the accepted sets of the plan's entries into its own slice;
@@ -1057,17 +1142,21 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
 // then fills the mask of the state it reached: in a decode loop the two always follow each other,
 // and one launch saves a kernel boundary and lets a request with a slow accept and a short fill
 // overlap one with the opposite mix.
+// With kApplyElems (8: bf16 logits, 4: fp32) each block also masks its slice of the request's logits row from
+// the slice it has just written, still in shared memory: the mask is not read back from global memory, there is
+// no kernel boundary between fill and apply, and the rows of requests whose fill is short are masked while
+// other requests still walk their uncertain tokens.
 // The host picks cluster and block size so that the whole batch is resident at once.  Used when
 // a slice fits (at most 2048 words per block); larger vocabularies take the two-kernel path above.
 // ------------------------------------------------------------------------------------------
 constexpr int kMaxClusterBlocks = 8;      // the portable cluster size limit
 
 // launched with a cluster of gridDim.x blocks (2, 4 or 8) along x
-template <bool kAccept>
+template <bool kAccept, int kApplyElems>
 __global__ void __launch_bounds__(256, 4)
 fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __restrict__ bitmask, long long row_stride,
                     int32_t* __restrict__ status_user, const int32_t* __restrict__ token_ids, int32_t* __restrict__ accept_status,
-                    int restart_on_eos) {
+                    int restart_on_eos, void* __restrict__ logits, long long logits_row_stride_elems) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ uint32_t dyn_smem[];          // this block's row slice and a scratch slice: 2 x ceil(W / blocks) words
@@ -1262,75 +1351,13 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   const bool clear = st0 != 0 || failed;
   for (int w = threadIdx.x; w < nw; w += blockDim.x) bitmask[(long long)b * row_stride + w0 + w] = clear ? 0 : (int32_t)row[w];
   if (rank == 0 && threadIdx.x == 0 && status_user) status_user[b] = st0 != 0 ? st0 : (failed ? -6 : 0);
-}
-
-// ------------------------------------------------------------------------------------------
-// Mask apply (Section 2.1): logits of disallowed tokens become -inf, in place, one pass.
-// One 16-byte vector per thread and step.  A vector whose tokens are all allowed is skipped
-// (neither read nor written); one whose tokens are all disallowed is overwritten without being
-// read; only mixed vectors are read, blended and written back.
-// ------------------------------------------------------------------------------------------
-template <int ELEMS>
-__device__ __forceinline__ uint4 blend_ninf(uint4 x, uint32_t bits) {
-  if (ELEMS == 8) {
-    // four allowed-bits -> four bytes of 0x00 / 0xFF (a multiply spreads the bits to the bytes' low bits, a second
-    // one fills the bytes), then each byte is doubled into the 16-bit lane it stands for
-    const uint32_t lo = (((bits & 0xFu) * 0x00204081u) & 0x01010101u) * 0xFFu;
-    const uint32_t hi = ((((bits >> 4) & 0xFu) * 0x00204081u) & 0x01010101u) * 0xFFu;
-    const uint32_t k0 = __byte_perm(lo, 0u, 0x1100), k1 = __byte_perm(lo, 0u, 0x3322);
-    const uint32_t k2 = __byte_perm(hi, 0u, 0x1100), k3 = __byte_perm(hi, 0u, 0x3322);
-    constexpr uint32_t kNinf2 = 0xFF80FF80u;
-    return make_uint4((x.x & k0) | (kNinf2 & ~k0), (x.y & k1) | (kNinf2 & ~k1), (x.z & k2) | (kNinf2 & ~k2), (x.w & k3) | (kNinf2 & ~k3));
-  }
-  if (!(bits & 1u)) x.x = 0xFF800000u;
-  if (!(bits & 2u)) x.y = 0xFF800000u;
-  if (!(bits & 4u)) x.z = 0xFF800000u;
-  if (!(bits & 8u)) x.w = 0xFF800000u;
-  return x;
-}
-
-// grid = (blocks per row, rows).  Each thread handles four vectors per iteration: the four mask
-// tests first, then the loads of the mixed vectors (independent, all in flight together), then
-// the stores.
-template <int ELEMS>   // elements per 16-byte vector: 8 (bf16) or 4 (fp32)
-__global__ void __launch_bounds__(256)
-apply_kernel(void* __restrict__ logits, int vocab_size, long long row_stride_elems, const uint32_t* __restrict__ bitmask,
-             long long mask_stride, const int32_t* __restrict__ row_indices) {
-  step_kernel_prologue();
-  const int r = row_indices ? row_indices[blockIdx.y] : blockIdx.y;
-  const uint32_t* mrow = bitmask + (long long)r * mask_stride;
-  const int n_vec = vocab_size / ELEMS;
-  constexpr uint32_t kAll = (1u << ELEMS) - 1;
-  const uint4 ninf = ELEMS == 8 ? make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u)
-                                : make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
-  uint4* base = ELEMS == 8 ? (uint4*)((uint16_t*)logits + (long long)r * row_stride_elems)
-                           : (uint4*)((uint32_t*)logits + (long long)r * row_stride_elems);
-  const int stride = gridDim.x * blockDim.x;
-  for (int v0 = blockIdx.x * blockDim.x + threadIdx.x; v0 < n_vec; v0 += 4 * stride) {
-    uint32_t bits[4];
-    uint4 x[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int vi = v0 + u * stride;
-      const int first = vi * ELEMS;
-      bits[u] = vi < n_vec ? ((__ldg(&mrow[first >> 5]) >> (first & 31)) & kAll) : kAll;
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-      if (bits[u] != kAll && bits[u] != 0) x[u] = __ldcs(&base[v0 + u * stride]);
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      if (bits[u] == kAll) continue;
-      __stcs(&base[v0 + u * stride], bits[u] == 0 ? ninf : blend_ninf<ELEMS>(x[u], bits[u]));
-    }
-  }
-  // ragged tail (vocab_size not a multiple of the vector width)
-  if (blockIdx.x == 0) {
-    for (int c = n_vec * ELEMS + threadIdx.x; c < vocab_size; c += blockDim.x) {
-      if ((mrow[c >> 5] >> (c & 31)) & 1u) continue;
-      if (ELEMS == 8) ((uint16_t*)logits)[(long long)r * row_stride_elems + c] = 0xFF80u;
-      else ((uint32_t*)logits)[(long long)r * row_stride_elems + c] = 0xFF800000u;
-    }
+  // 4. mask this slice of the request's logits (nobody writes `row` any more: every remote OR landed before the barrier)
+  if (kApplyElems != 0 && nw > 0) {
+    constexpr int kE = kApplyElems == 0 ? 8 : kApplyElems;
+    void* row_base = kE == 8 ? (void*)((uint16_t*)logits + (long long)b * logits_row_stride_elems) : (void*)((uint32_t*)logits + (long long)b * logits_row_stride_elems);
+    auto word_at = [&](int w) { return clear ? 0u : row[w - w0]; };
+    apply_vectors<kE>((uint4*)row_base, w0 * 32 / kE, min(v.vocab_size / kE, w1 * 32 / kE), threadIdx.x, blockDim.x, word_at);
+    if (w1 == v.n_words) apply_ragged_tail<kE>(row_base, v.vocab_size, threadIdx.x, blockDim.x, word_at);
   }
 }
 

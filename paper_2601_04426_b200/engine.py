@@ -77,6 +77,12 @@ class Session:
         B.apply_token_bitmask(logits.data_ptr(), dtype, logits.shape[0], self.V, logits.stride(0), self.bitmask.data_ptr(), self.W,
                               rows.data_ptr() if rows is not None else 0, int(rows.numel()) if rows is not None else 0, self.stream())
 
+    def fill_apply(self, logits: torch.Tensor) -> None:
+        """Fill every request's mask and apply it to its logits row, in one launch."""
+        dtype = {torch.float32: "f32", torch.bfloat16: "bf16", torch.int16: "bf16", torch.uint16: "bf16"}[logits.dtype]
+        self.batch.fill_and_apply_token_bitmask(self.bitmask.data_ptr(), self.W, self.status.data_ptr(), logits.data_ptr(), dtype,
+                                                logits.stride(0), self.stream())
+
     def jit_service(self, wait: bool = False) -> dict:
         """Between decode steps: pick up the cache entries the last fills found missing (just-in-time grammars)."""
         return B.jit_service(self.grammars, self.stream(), wait)
