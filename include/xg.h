@@ -43,7 +43,8 @@ enum {
   XG_ERR_UNSUPPORTED = -3,    /* schema keyword or construct outside the supported subset */
   XG_ERR_OOM = -4,
   XG_ERR_CUDA = -5,           /* a CUDA runtime call failed, or no usable device */
-  XG_ERR_CAPACITY = -6,       /* a fixed-capacity structure (item sets, history) overflowed */
+  XG_ERR_CAPACITY = -6,       /* a capacity was exhausted: the matcher's history (max_sets / max_items), or an Earley
+                                 set beyond even the exact slow path (2048 items per token walk) */
   XG_ERR_TOKEN_REJECTED = -7, /* xg_accept_token: the token is not allowed in this state */
   XG_ERR_TERMINATED = -8,     /* the matcher already accepted EOS */
   XG_ERR_TIMEOUT = -9
@@ -272,8 +273,17 @@ xg_status_t xg_matcher_next_fill_work(const xg_matcher_t* m, void* stream, xg_fi
  * Earley state; otherwise it is rejected.  EOS is allowed iff the root rule is complete.
  * (Just-in-time grammars: a request with an entry still missing gets the same mask from a walk of
  * the whole vocabulary against its full Earley state.)
+ * Token walks run in small fixed arrays; a walk that does not fit them (an Earley set of more than 48
+ * items, a token longer than 32 bytes) is redone exactly in a large per-matcher scratch, and a state
+ * with more scannable entries than the step plan lists takes its mask from the plain definition, so
+ * such states cost time, never a wrong or missing bit.  XG_ERR_CAPACITY is left for walks beyond that
+ * scratch (2048 items, or more than 1024 such tokens in one step).
  * status_dev (device, [batch], may be NULL) receives XG_OK, XG_ERR_TERMINATED or XG_ERR_CAPACITY
- * per matcher; rows of matchers whose status is not XG_OK are all zero. */
+ * per matcher; rows of matchers whose status is not XG_OK are all zero.
+ * The first call with a list of matchers uploads the list (one asynchronous copy on `stream`); the
+ * library caches the 64 most recently used lists, so a decode loop whose batch changes by a request
+ * per step neither allocates nor synchronises the device once its largest batch has been seen.  Calls
+ * on one tokenizer must be ordered among themselves (one stream, or events). */
 xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t batch,
                                        int32_t* bitmask_dev, int64_t row_stride_words,
                                        int32_t* status_dev, void* stream);
@@ -291,10 +301,10 @@ xg_status_t xg_fill_next_token_bitmask(xg_matcher_t* const* matchers, int32_t ba
  *   - batch > XG_STATIC_FILL_MAX_BATCH returns XG_ERR_CAPACITY and does nothing.
  *   - The first call on each device looks up the array's device address; make that first call
  *     before any stream capture begins.
- *   - Every call on a device uses the same array: the request table and the per-request words
- *     are rewritten at the start of each call, so nothing is carried over from the previous one,
- *     but two calls whose GPU work overlaps (different streams) race; keep them on one stream or
- *     order them with events.
+ *   - Every call on a device uses the same array: a small kernel at the head of each call rewrites
+ *     the request table (which travels as a launch parameter, not through a host buffer) and clears
+ *     the per-request words, so nothing is carried over from the previous call, but two calls whose
+ *     GPU work overlaps (different streams) race; keep them on one stream or order them with events.
  * Arguments, layout, statuses and errors are otherwise those of xg_fill_next_token_bitmask. */
 #define XG_STATIC_FILL_MAX_BATCH 1024
 xg_status_t xg_fill_next_token_bitmask_static(xg_matcher_t* const* matchers, int32_t batch,

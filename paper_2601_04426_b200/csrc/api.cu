@@ -80,13 +80,30 @@ double now_ms() {
 
 }  // namespace
 
-// the device array of matcher pointers (and the per-request scratch words) of one batch
+// Device arrays of matcher pointers, one per batch composition.  A decode loop calls with the same list of
+// matchers step after step, or with one that differs in a request or two (continuous batching): the list is looked
+// up among the cached compositions; a new one takes the least recently used entry and is uploaded with one
+// asynchronous copy from the entry's own pinned staging buffer on the caller's stream.  After the tables have grown
+// to the largest batch in use there is no allocation, no device-wide synchronisation and no blocking copy.
+constexpr int kBatchEntries = 64;
 struct BatchSlot {
   std::vector<xg_matcher_t*> key;
-  MatcherDev** dev_matchers = nullptr;
-  int32_t* status = nullptr;       // [batch]
-  int32_t* done_count = nullptr;   // [batch]
+  MatcherDev** dev_matchers = nullptr;   // [cap], inside the tokenizer's slab
+  MatcherDev** staging = nullptr;        // [cap], pinned host memory
+  cudaEvent_t uploaded = nullptr;        // the last upload from `staging` (an entry is reused only after it)
+  bool upload_recorded = false;
+  bool in_graph = false;                 // uploaded inside a stream capture: the graph's copy node reads `staging` at
+                                         // every replay, so the entry is never reused
+  int32_t* status = nullptr;             // [cap] scratch words of the two-kernel fill (shared by all entries)
+  int32_t* done_count = nullptr;
   uint64_t last_use = 0;
+};
+struct BatchTables {
+  int cap = 0;                           // requests per entry
+  MatcherDev** dev_slab = nullptr;       // [kBatchEntries][cap]
+  MatcherDev** host_slab = nullptr;      // pinned, same shape
+  int32_t* words = nullptr;              // status[cap], done_count[cap]
+  std::vector<BatchSlot> slots;
 };
 
 struct xg_tokenizer {
@@ -96,7 +113,7 @@ struct xg_tokenizer {
   int32_t vocab_size = 0, n_words = 0;
   int64_t first_byte_count[256] = {};     // tokens (other than EOS / special / empty) by first byte
   mutable std::mutex mu;
-  mutable std::vector<BatchSlot> batch_slots;
+  mutable BatchTables batches;
   mutable uint64_t use_counter = 0;
 };
 
@@ -257,7 +274,9 @@ xg_status_t xg_tokenizer_create(const uint8_t* bytes, const int64_t* offsets, in
 
 void xg_tokenizer_destroy(xg_tokenizer_t* t) {
   if (!t) return;
-  for (auto& s : t->batch_slots) { cudaFree(s.dev_matchers); cudaFree(s.status); cudaFree(s.done_count); }
+  for (auto& s : t->batches.slots) if (s.uploaded) cudaEventDestroy(s.uploaded);
+  cudaFree(t->batches.dev_slab); cudaFree(t->batches.words);
+  if (t->batches.host_slab) cudaFreeHost(t->batches.host_slab);
   for (void* p : t->allocations) cudaFree(p);
   delete t;
 }
@@ -1179,7 +1198,9 @@ xg_status_t xg_matcher_create(const xg_grammar_t* g, const xg_matcher_options_t*
   m->grammar = g;
   const size_t o_plan = 256, o_items = o_plan + ((sizeof(StepPlan) + 255) & ~size_t(255)), o_org = o_items + (size_t)max_items * 4,
                o_sb = o_org + (size_t)max_items * 4;
-  const size_t total = o_sb + ((size_t)max_sets + 1) * 4;
+  const size_t o_slow_st = (o_sb + ((size_t)max_sets + 1) * 4 + 255) & ~size_t(255), o_slow_org = o_slow_st + (size_t)kSlowCap * 4,
+               o_slow_lsb = o_slow_org + (size_t)kSlowCap * 4, o_slow_q = o_slow_lsb + (size_t)(kSlowMaxBytes + 2) * 4;
+  const size_t total = o_slow_q + (size_t)kSlowQueue * 4;
   XG_CUDA(cudaMalloc(&m->block, total));
   uint8_t* d = (uint8_t*)m->block;
   MatcherDev h{};
@@ -1189,6 +1210,8 @@ xg_status_t xg_matcher_create(const xg_grammar_t* g, const xg_matcher_options_t*
   h.set_begin = (int32_t*)(d + o_sb);
   h.cap_sets = max_sets; h.cap_items = max_items;
   h.plan = (StepPlan*)(d + o_plan);
+  h.slow_st = (uint32_t*)(d + o_slow_st); h.slow_org = (int32_t*)(d + o_slow_org);
+  h.slow_lsb = (int32_t*)(d + o_slow_lsb); h.slow_q = (int32_t*)(d + o_slow_q);
   m->dev = (MatcherDev*)d;
   cudaError_t err = cudaMemcpyAsync(m->dev, &h, sizeof h, cudaMemcpyHostToDevice, (cudaStream_t)stream);
   if (err == cudaSuccess) { matcher_reset_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(m->dev); err = cudaGetLastError(); }
@@ -1210,7 +1233,7 @@ void xg_matcher_destroy(xg_matcher_t* m) {
   if (m->grammar && m->grammar->tok) {       // forget cached batches that contain this matcher
     const xg_tokenizer* t = m->grammar->tok;
     std::lock_guard<std::mutex> lock(t->mu);
-    for (auto& s : t->batch_slots)
+    for (auto& s : t->batches.slots)
       if (std::find(s.key.begin(), s.key.end(), m) != s.key.end()) s.key.clear();
   }
   cudaFree(m->block);
@@ -1253,34 +1276,63 @@ xg_status_t xg_matcher_next_fill_work(const xg_matcher_t* m, void* stream, xg_fi
   return XG_OK;
 }
 
-// device-side array of matcher pointers for this exact batch (built once, then reused)
-static xg_status_t batch_slot(xg_matcher_t* const* matchers, int32_t batch, const xg_tokenizer** tok_out, BatchSlot** slot_out) {
+// (re)allocate the batch tables for `cap` requests per composition; only when a batch is larger than any before
+static xg_status_t grow_batch_tables(BatchTables& bt, int cap) {
+  XG_CUDA(cudaDeviceSynchronize());              // the old tables may still be in use
+  for (auto& s : bt.slots) if (s.uploaded) cudaEventDestroy(s.uploaded);
+  bt.slots.clear();
+  cudaFree(bt.dev_slab); cudaFree(bt.words);
+  if (bt.host_slab) cudaFreeHost(bt.host_slab);
+  bt.dev_slab = nullptr; bt.words = nullptr; bt.host_slab = nullptr; bt.cap = 0;
+  XG_CUDA(cudaMalloc(&bt.dev_slab, sizeof(void*) * (size_t)cap * kBatchEntries));
+  XG_CUDA(cudaMalloc(&bt.words, sizeof(int32_t) * 2 * (size_t)cap));
+  XG_CUDA(cudaHostAlloc(&bt.host_slab, sizeof(void*) * (size_t)cap * kBatchEntries, cudaHostAllocDefault));
+  bt.cap = cap;
+  bt.slots.resize(kBatchEntries);
+  for (int k = 0; k < kBatchEntries; ++k) {
+    BatchSlot& s = bt.slots[k];
+    s.dev_matchers = bt.dev_slab + (size_t)k * cap;
+    s.staging = bt.host_slab + (size_t)k * cap;
+    s.status = bt.words; s.done_count = bt.words + cap;
+    XG_CUDA(cudaEventCreateWithFlags(&s.uploaded, cudaEventDisableTiming));
+  }
+  return XG_OK;
+}
+
+// device-side array of matcher pointers for this batch composition (see BatchTables)
+static xg_status_t batch_slot(xg_matcher_t* const* matchers, int32_t batch, cudaStream_t stream, const xg_tokenizer** tok_out, BatchSlot** slot_out) {
   if (!matchers || batch <= 0) return set_error(XG_ERR_INVALID_ARG, "empty batch");
   if (batch > 65535) return set_error(XG_ERR_INVALID_ARG, "batch larger than 65535");
   for (int i = 0; i < batch; ++i) if (!matchers[i]) return set_error(XG_ERR_INVALID_ARG, "NULL matcher in batch");
   const xg_tokenizer* tok = matchers[0]->grammar->tok;
   for (int i = 1; i < batch; ++i) if (matchers[i]->grammar->tok != tok) return set_error(XG_ERR_INVALID_ARG, "matchers of one batch must share a tokenizer");
   std::lock_guard<std::mutex> lock(tok->mu);
+  BatchTables& bt = tok->batches;
+  if (batch > bt.cap) {
+    int cap = std::max(256, bt.cap);
+    while (cap < batch) cap *= 2;
+    xg_status_t st = grow_batch_tables(bt, cap);
+    if (st != XG_OK) return st;
+  }
   BatchSlot* hit = nullptr;
-  for (auto& s : tok->batch_slots)
+  for (auto& s : bt.slots)
     if ((int)s.key.size() == batch && std::memcmp(s.key.data(), matchers, sizeof(void*) * batch) == 0) { hit = &s; break; }
   if (!hit) {
-    if (tok->batch_slots.size() < 16) tok->batch_slots.emplace_back();
-    BatchSlot* victim = &tok->batch_slots[0];
-    for (auto& s : tok->batch_slots) {
+    BatchSlot* victim = nullptr;
+    for (auto& s : bt.slots) {
+      if (s.in_graph && !s.key.empty()) continue;
       if (s.key.empty()) { victim = &s; break; }
-      if (s.last_use < victim->last_use) victim = &s;
+      if (!victim || s.last_use < victim->last_use) victim = &s;
     }
-    XG_CUDA(cudaDeviceSynchronize());            // the victim's arrays may still be in use
-    cudaFree(victim->dev_matchers); cudaFree(victim->status); cudaFree(victim->done_count);
-    victim->dev_matchers = nullptr; victim->status = nullptr; victim->done_count = nullptr;
-    victim->key.clear();
-    std::vector<MatcherDev*> ptrs(batch);
-    for (int i = 0; i < batch; ++i) ptrs[i] = matchers[i]->dev;
-    XG_CUDA(cudaMalloc(&victim->dev_matchers, sizeof(void*) * batch));
-    XG_CUDA(cudaMalloc(&victim->status, sizeof(int32_t) * batch));
-    XG_CUDA(cudaMalloc(&victim->done_count, sizeof(int32_t) * batch));
-    XG_CUDA(cudaMemcpy(victim->dev_matchers, ptrs.data(), sizeof(void*) * batch, cudaMemcpyHostToDevice));
+    if (!victim) return set_error(XG_ERR_CAPACITY, "every cached batch composition belongs to a captured graph");
+    if (victim->upload_recorded) XG_CUDA(cudaEventSynchronize(victim->uploaded));      // its staging buffer is free again (long done, normally)
+    for (int i = 0; i < batch; ++i) victim->staging[i] = matchers[i]->dev;
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    XG_CUDA(cudaStreamIsCapturing(stream, &capturing));
+    XG_CUDA(cudaMemcpyAsync(victim->dev_matchers, victim->staging, sizeof(void*) * batch, cudaMemcpyHostToDevice, stream));
+    victim->in_graph = capturing != cudaStreamCaptureStatusNone;
+    victim->upload_recorded = false;
+    if (!victim->in_graph) { XG_CUDA(cudaEventRecord(victim->uploaded, stream)); victim->upload_recorded = true; }
     victim->key.assign(matchers, matchers + batch);
     hit = victim;
   }
@@ -1299,7 +1351,7 @@ static xg_status_t accept_and_fill(xg_matcher_t* const* matchers, int32_t batch,
                                    void* logits_dev = nullptr, xg_dtype_t dtype = XG_F32, int64_t logits_row_stride_elems = 0) {
   const xg_tokenizer* tok = nullptr;
   BatchSlot* slot = nullptr;
-  xg_status_t st = batch_slot(matchers, batch, &tok, &slot);
+  xg_status_t st = batch_slot(matchers, batch, (cudaStream_t)stream, &tok, &slot);
   if (st != XG_OK) return st;
   if (!bitmask_dev || row_stride_words < tok->n_words) return set_error(XG_ERR_INVALID_ARG, "bad bitmask buffer");
   const int W = tok->n_words;
@@ -1386,6 +1438,18 @@ struct StaticFillScratch {
 };
 static __device__ __align__(256) unsigned char g_static_fill_scratch[sizeof(StaticFillScratch)];
 
+// the request table of one call, passed to the set-up kernel by value (8 KiB of launch parameters)
+struct StaticFillTable {
+  MatcherDev* matchers[XG_STATIC_FILL_MAX_BATCH];
+};
+static __global__ void static_fill_setup_kernel(StaticFillScratch* sc, const __grid_constant__ StaticFillTable table, int batch) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= batch) return;
+  sc->matchers[i] = table.matchers[i];
+  sc->status[i] = 0;
+  sc->done_count[i] = 0;
+}
+
 // The symbol above is only a host-side stand-in; kernels need its device address, which differs
 // per device.  Looked up once per device, with that device current.
 static xg_status_t static_fill_scratch(StaticFillScratch** out) {
@@ -1411,11 +1475,11 @@ xg_status_t xg_fill_next_token_bitmask_static(xg_matcher_t* const* matchers, int
   if (batch > XG_STATIC_FILL_MAX_BATCH)
     return set_error(XG_ERR_CAPACITY, "batch of " + std::to_string(batch) + " requests exceeds the static scratch limit of " +
                                           std::to_string(XG_STATIC_FILL_MAX_BATCH) + "; use xg_fill_next_token_bitmask or split the batch");
-  MatcherDev* ptrs[XG_STATIC_FILL_MAX_BATCH];
+  StaticFillTable table;
   for (int i = 0; i < batch; ++i) {
     if (!matchers[i]) return set_error(XG_ERR_INVALID_ARG, "NULL matcher in batch");
     if (matchers[i]->grammar->tok != matchers[0]->grammar->tok) return set_error(XG_ERR_INVALID_ARG, "matchers of one batch must share a tokenizer");
-    ptrs[i] = matchers[i]->dev;
+    table.matchers[i] = matchers[i]->dev;
   }
   const xg_tokenizer* tok = matchers[0]->grammar->tok;
   if (!bitmask_dev || row_stride_words < tok->n_words) return set_error(XG_ERR_INVALID_ARG, "bad bitmask buffer");
@@ -1423,9 +1487,9 @@ xg_status_t xg_fill_next_token_bitmask_static(xg_matcher_t* const* matchers, int
   xg_status_t st = static_fill_scratch(&sc);
   if (st != XG_OK) return st;
   cudaStream_t cs = (cudaStream_t)stream;
-  // the array keeps the previous call's contents: rewrite the request table, clear the words
-  XG_CUDA(cudaMemcpyAsync(sc->matchers, ptrs, sizeof(MatcherDev*) * batch, cudaMemcpyHostToDevice, cs));
-  XG_CUDA(cudaMemsetAsync(sc->status, 0, 2 * sizeof(int32_t) * XG_STATIC_FILL_MAX_BATCH, cs));
+  // the array keeps the previous call's contents: the request table is rewritten and the words cleared by a small
+  // kernel that gets the table as a launch parameter (no host buffer has to outlive the call)
+  static_fill_setup_kernel<<<(batch + 255) / 256, 256, 0, cs>>>(sc, table, batch);
   const int W = tok->n_words;
   int chunks = std::max((W + kMergeMaxChunkWords - 1) / kMergeMaxChunkWords, std::min(8, (W + 127) / 128));
   merge_kernel<<<dim3(chunks, batch), 256, 0, cs>>>(sc->matchers, tok->dev, bitmask_dev, (long long)row_stride_words, status_dev, sc->status, sc->done_count);
@@ -1443,7 +1507,7 @@ xg_status_t xg_accept_token_ex(xg_matcher_t* const* matchers, int32_t batch, con
   NvtxRange nvtx_range("xg_accept_token");
   const xg_tokenizer* tok = nullptr;
   BatchSlot* slot = nullptr;
-  xg_status_t st = batch_slot(matchers, batch, &tok, &slot);
+  xg_status_t st = batch_slot(matchers, batch, (cudaStream_t)stream, &tok, &slot);
   if (st != XG_OK) return st;
   if (!token_ids_dev) return set_error(XG_ERR_INVALID_ARG, "token_ids_dev is NULL");
   XG_CUDA(launch_step_kernel(accept_kernel, dim3((batch + 3) / 4), dim3(128), 0, (cudaStream_t)stream, 1, (MatcherDev* const*)slot->dev_matchers,

@@ -126,9 +126,16 @@ struct MatcherDev {
   int32_t n_sets, n_items;
   int32_t cap_sets, cap_items;
   int32_t terminated;
-  int32_t pad;
+  int32_t slow_n;            // tokens queued for the exact slow walk by the fill that is running (reset by every fill)
   StepPlan* plan;
+  // Exact slow path (one user at a time): a token walk that does not fit the fixed per-thread arrays -- more than
+  // kFastCap items, or a token beyond kFastMaxBytes bytes -- is redone here, up to kSlowCap items and 255 bytes.
+  uint32_t* slow_st;         // [kSlowCap]
+  int32_t* slow_org;         // [kSlowCap]
+  int32_t* slow_lsb;         // [257]
+  int32_t* slow_q;           // [kSlowQueue] token ranks waiting for a slow walk
 };
+constexpr int kSlowQueue = 1024;
 
 constexpr uint32_t kSelf = 0x80000000u;
 

@@ -725,24 +725,32 @@ __device__ __forceinline__ int accept_one(MatcherDev& m, const GrammarDev& g, co
   int done = 0;
   while (done < len && st == 0) {            // long tokens go through in pieces
     const int piece = min(len - done, kFastMaxBytes);
-    int made = 0;
+    int made = 0, slow = 0;
     if (n_sets + piece > m.cap_sets) st = -6;
     else if (lane == 0) {
       int flags = 0;
       const Chart c = done == 0 ? c0 : chart_of_history(m.item_state, m.item_origin, m.set_begin, n_sets - 1);
-      const int consumed = token_walk<int16_t>(g, g.class_bits, c, v.bytes + off + done, piece, false, w_st, w_org, kFastCap, lsb, &flags, nullptr);
+      int consumed = token_walk<int16_t>(g, g.class_bits, c, v.bytes + off + done, piece, false, w_st, w_org, kFastCap, lsb, &flags, nullptr);
+      if (flags & kWalkOverflow) {       // the sets do not fit the warp's scratch: the same walk again, exactly, in the matcher's large one
+        flags = 0;
+        slow = 1;
+        consumed = token_walk<int32_t>(g, g.class_bits, c, v.bytes + off + done, piece, false, m.slow_st, m.slow_org, kSlowCap, m.slow_lsb, &flags, nullptr);
+      }
       if (flags & kWalkOverflow) st = -6;
       else if (consumed < piece) st = -7;
-      else { made = lsb[piece + 1]; if (n_items + made > m.cap_items) st = -6; }
+      else { made = slow ? m.slow_lsb[piece + 1] : lsb[piece + 1]; if (n_items + made > m.cap_items) st = -6; }
     }
     st = __shfl_sync(0xFFFFFFFFu, st, 0);
     made = __shfl_sync(0xFFFFFFFFu, made, 0);
+    slow = __shfl_sync(0xFFFFFFFFu, slow, 0);
     if (st != 0) break;
     __syncwarp();
     // origins written by the walk are already chart indices (its base is set n_sets - 1);
     // append the new sets behind the history (visible to the next piece; committed below)
-    for (int q = lane; q < made; q += 32) { m.item_state[n_items + q] = w_st[q]; m.item_origin[n_items + q] = w_org[q]; }
-    for (int j = 1 + lane; j <= piece; j += 32) m.set_begin[n_sets + j] = n_items + lsb[j + 1];
+    const uint32_t* src_st = slow ? m.slow_st : w_st;
+    const int32_t* src_org = slow ? m.slow_org : w_org;
+    for (int q = lane; q < made; q += 32) { m.item_state[n_items + q] = src_st[q]; m.item_origin[n_items + q] = src_org[q]; }
+    for (int j = 1 + lane; j <= piece; j += 32) m.set_begin[n_sets + j] = n_items + (slow ? m.slow_lsb[j + 1] : (int)lsb[j + 1]);
     __syncwarp();
     n_items += made;
     n_sets += piece;
@@ -837,6 +845,34 @@ __device__ __forceinline__ void report_missing(const GrammarDev& g, const StepPl
 
 constexpr int kMergeMaxChunkWords = 2048;
 
+// A token whose walk does not fit the per-thread arrays (more than kFastCap items, or longer than kFastMaxBytes)
+// is queued on its request for the exact slow walk; false when the queue is full (the request then fails).
+__device__ __forceinline__ bool queue_slow_walk(MatcherDev* m, int token_rank) {
+  const int slot = atomicAdd(&m->slow_n, 1);
+  if (slot >= kSlowQueue) return false;
+  m->slow_q[slot] = token_rank;
+  return true;
+}
+
+// The queued tokens, one after the other, by one thread: each walked in full from the request's current set (the
+// plain definition) in the matcher's large scratch; allow(id) records a token that passes.  false: a walk exceeded
+// even that scratch, or the queue had overflowed.
+template <typename F>
+__device__ __forceinline__ bool run_slow_walks(MatcherDev* m, const GrammarDev& g, const VocabDev& v, const Chart& hist, F allow) {
+  const int n = m->slow_n;
+  if (n > kSlowQueue) return false;
+  for (int i = 0; i < n; ++i) {
+    const int trank = m->slow_q[i];
+    const uint32_t off = v.offset[trank];
+    const int len = (int)(v.offset[trank + 1] - off);
+    int flags = 0;
+    const bool pass = token_walk<int32_t>(g, g.class_bits, hist, v.bytes + off, len, false, m->slow_st, m->slow_org, kSlowCap, m->slow_lsb, &flags, nullptr) == len;
+    if (flags & kWalkOverflow) return false;
+    if (pass) allow(v.rank_to_id[trank]);
+  }
+  return true;
+}
+
 __global__ void __launch_bounds__(256)
 merge_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __restrict__ bitmask, long long row_stride,
              int32_t* __restrict__ status_user, int32_t* __restrict__ status, int32_t* __restrict__ done_count) {
@@ -850,11 +886,12 @@ merge_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
   const int nw = max(0, w1 - w0);
   for (int w = threadIdx.x; w < nw; w += blockDim.x) row[w] = 0;
   const StepPlan& plan = *m.plan;
-  const int st0 = m.terminated ? -8 : (plan.overflow ? -6 : 0);
+  const int st0 = m.terminated ? -8 : 0;
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     status[b] = st0;
     if (status_user) status_user[b] = st0;
     done_count[b] = 0;
+    matchers[b]->slow_n = 0;
   }
   __syncthreads();
   if (st0 == 0 && nw > 0) {
@@ -920,8 +957,10 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
   const GrammarDev& g = *m.grammar;
   const StepPlan& plan = *m.plan;
   const int n = m.n_sets - 1;
-  const bool live = !m.terminated && !plan.overflow;
-  const bool fallback = live && plan.n_missing > 0;   // an entry is not built yet: walk the whole vocabulary instead
+  MatcherDev* mw = matchers[b];
+  const bool live = !m.terminated;
+  // an entry is not built yet, or the plan did not fit its fixed arrays: walk the whole vocabulary instead
+  const bool fallback = live && (plan.n_missing > 0 || plan.overflow);
   const int n_ent = (live && !fallback) ? plan.n_check : 0;
   const int total = n_ent ? plan.check_cum[n_ent] : 0;
   const int stride = gridDim.x * blockDim.x;
@@ -931,7 +970,7 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
     const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
     const uint32_t* class_bits = stage_class_bits(g, sh_class);
     current_first_bytes(g, hist, set_first, threadIdx.x);
-    if (blockIdx.x == 0 && threadIdx.x == 0) report_missing(g, plan);
+    if (blockIdx.x == 0 && threadIdx.x == 0 && plan.n_missing > 0) report_missing(g, plan);
     __syncthreads();
     uint32_t* row = (uint32_t*)bitmask + (long long)b * row_stride;
     for (int r = blockIdx.x * blockDim.x + threadIdx.x; r < v.vocab_size; r += stride) {
@@ -940,13 +979,13 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
       const int len = (int)(v.offset[r + 1] - off);
       const uint32_t byte = v.bytes[off];
       if (!((set_first[byte >> 5] >> (byte & 31)) & 1u)) continue;
-      if (len > kFastMaxBytes) { sh_fail = 1; continue; }
+      if (len > kFastMaxBytes) { if (!queue_slow_walk(mw, r)) sh_fail = 1; continue; }
       uint32_t st[kFastCap];
       int32_t org[kFastCap];
       int16_t lsb[kFastMaxBytes + 2];
       int flags = 0;
       const bool pass = token_walk<int16_t>(g, class_bits, hist, v.bytes + off, len, false, st, org, kFastCap, lsb, &flags, nullptr) == len;
-      if (flags & kWalkOverflow) sh_fail = 1;
+      if (flags & kWalkOverflow) { if (!queue_slow_walk(mw, r)) sh_fail = 1; }
       else if (pass) { const int id = v.rank_to_id[r]; atomicOr(&row[id >> 5], 1u << (id & 31)); }
     }
   } else
@@ -1000,7 +1039,7 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
       bool pass = false, overflow = false;
       if (exits[u] == 0) {
         // no exit record (very long token, or its walk overflowed at build time): walk in full
-        if (len > kFastMaxBytes) overflow = true;
+        if (len > kFastMaxBytes) overflow = true;      // (queued for the slow walk below)
         else {
           uint32_t st[kFastCap];
           int32_t org[kFastCap];
@@ -1028,7 +1067,7 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
           overflow = (flags & kWalkOverflow) != 0;
         }
       }
-      if (overflow) sh_fail = 1;
+      if (overflow) { if (!queue_slow_walk(mw, rank[u])) sh_fail = 1; }       // the whole token again, exactly
       else if (pass) { const int id = v.rank_to_id[rank[u]]; atomicOr(&row[id >> 5], 1u << (id & 31)); }
     }
   }
@@ -1042,6 +1081,14 @@ check_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __re
   __syncthreads();
   if (sh_last) {
     __threadfence();
+    // every block of the request has finished: the queued slow walks, by one thread
+    if (threadIdx.x == 0 && *(volatile int32_t*)&mw->slow_n > 0) {
+      uint32_t* row = (uint32_t*)bitmask + (long long)b * row_stride;
+      const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
+      if (!run_slow_walks(mw, g, v, hist, [&](int id) { row[id >> 5] |= 1u << (id & 31); })) status[b] = -6;
+      __threadfence();
+    }
+    __syncthreads();
     const int s = *(volatile int32_t*)&status[b];
     if (s == -6) {
       uint32_t* row = (uint32_t*)bitmask + (long long)b * row_stride;
@@ -1169,19 +1216,17 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   __shared__ int cont_cnt[kPlanCheckMax];
   __shared__ uint32_t cont_first[kPlanCheckMax][8];
   __shared__ uint32_t sh_class[kSharedClasses * 8];
-  // uncertain tokens too long for the per-thread arrays (33..255 bytes; rare) are queued and walked one at a time
-  // by thread 0 in this block-wide scratch
-  constexpr int kLongQueue = 32, kLongCap = 512;
-  __shared__ int long_q[kLongQueue];
-  __shared__ int long_n;
-  __shared__ uint32_t long_st[kLongCap];
-  __shared__ int32_t long_org[kLongCap];
-  __shared__ int16_t long_lsb[kSlowMaxBytes + 2];
+  // scratch of the accepting warp (kAccept)
+  __shared__ uint32_t acc_st[kAccept ? kFastCap : 1];
+  __shared__ int32_t acc_org[kAccept ? kFastCap : 1];
+  __shared__ int16_t acc_lsb[kAccept ? kFastMaxBytes + 2 : 1];
   __shared__ int sh_fail;          // set in every block of the cluster when any of them fails
+  __shared__ int sh_slow;          // set in every block of the cluster when a token was queued for the exact slow walk
 
   step_kernel_prologue();
   const int b = blockIdx.y;
   const int rank = (int)cluster.block_rank();
+  MatcherDev* mw = matchers[b];
   const MatcherDev& m = *matchers[b];
   const GrammarDev& g = *m.grammar;
   const StepPlan& plan = *m.plan;
@@ -1196,14 +1241,15 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
     // nothing of the request's state or plan is read before this barrier; its release/acquire pair makes what the
     // accepting warp wrote visible to the whole cluster
     if (rank == 0 && threadIdx.x < 32) {
-      const int st = accept_one(*matchers[b], g, v, token_ids[b], restart_on_eos != 0, (int)threadIdx.x, long_st, long_org, long_lsb);
+      const int st = accept_one(*matchers[b], g, v, token_ids[b], restart_on_eos != 0, (int)threadIdx.x, acc_st, acc_org, acc_lsb);
       if (accept_status && threadIdx.x == 0) accept_status[b] = st;
     }
     cluster.sync();
   }
-  const int st0 = m.terminated ? -8 : (plan.overflow ? -6 : 0);
-  if (threadIdx.x == 0) { sh_fail = 0; long_n = 0; }
-  const bool fallback = st0 == 0 && plan.n_missing > 0;   // an entry is not built yet: walk the whole vocabulary instead
+  const int st0 = m.terminated ? -8 : 0;
+  if (threadIdx.x == 0) { sh_fail = 0; sh_slow = 0; }
+  // an entry is not built yet, or the plan did not fit its fixed arrays: walk the whole vocabulary instead
+  const bool fallback = st0 == 0 && (plan.n_missing > 0 || plan.overflow);
   const int n_ent = (st0 == 0 && !fallback) ? plan.n_check : 0;
   const int total = n_ent ? plan.check_cum[n_ent] : 0;
   __shared__ uint32_t set_first[8];
@@ -1250,13 +1296,19 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
     for (int i = threadIdx.x; i < n_ent * 8; i += blockDim.x) (&cont_first[0][0])[i] = (&plan.cont_first[0][0])[i];
     if (fallback) {
       current_first_bytes(g, hist, set_first, threadIdx.x);
-      if (rank == 0 && threadIdx.x == 0) report_missing(g, plan);
+      if (rank == 0 && threadIdx.x == 0 && plan.n_missing > 0) report_missing(g, plan);
     }
-    cluster.sync();            // every slice is merged (and this block's staging is visible)
+    if (rank == 0 && threadIdx.x == 0) mw->slow_n = 0;
+    cluster.sync();            // every slice is merged (and this block's staging, and the emptied slow queue, are visible)
     const int stride = n_blocks * blockDim.x;
     // a failure (rare) is recorded in every block's flag, so that each block reads its own at the end and no block has to
     // outlive the others' reads
     auto fail_everywhere = [&]() { for (int r = 0; r < n_blocks; ++r) atomicOr(cluster.map_shared_rank(&sh_fail, r), 1); };
+    // a walk that does not fit the per-thread arrays: the token is queued for the exact slow walk after the others
+    auto walk_slowly = [&](int trank) {
+      if (!queue_slow_walk(mw, trank)) fail_everywhere();
+      for (int r = 0; r < n_blocks; ++r) atomicOr(cluster.map_shared_rank(&sh_slow, r), 1);
+    };
     auto walk_one = [&](int trank, uint32_t off, int e, int at) {
       const int len = (int)(v.offset[trank + 1] - off);
       bool pass = false, overflow = len - at > kFastMaxBytes;
@@ -1270,7 +1322,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
         pass = token_walk<int16_t>(g, class_bits, c, v.bytes + off + at, len - at, false, st, org, kFastCap, lsb, &flags, nullptr) == len - at;
         overflow = (flags & kWalkOverflow) != 0;
       }
-      if (overflow) fail_everywhere();
+      if (overflow) walk_slowly(trank);
       return pass && !overflow;
     };
     if (fallback) {
@@ -1280,11 +1332,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
         const uint32_t off = v.offset[r];
         const uint32_t byte = v.bytes[off];
         if (!((set_first[byte >> 5] >> (byte & 31)) & 1u)) continue;
-        if ((int)(v.offset[r + 1] - off) > kFastMaxBytes) {
-          const int slot = atomicAdd(&long_n, 1);
-          if (slot < kLongQueue) long_q[slot] = r; else fail_everywhere();
-          continue;
-        }
+        if ((int)(v.offset[r + 1] - off) > kFastMaxBytes) { walk_slowly(r); continue; }
         if (walk_one(r, off, 0, 0)) {
           const int id = v.rank_to_id[r];
           const int word = id >> 5, owner = word / chunk;
@@ -1303,11 +1351,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
       bool pass = false;
       int id = -1;
       if (left == 0) {                // no exit record (very long token, or its build-time walk overflowed): walk in full
-        if ((int)(v.offset[trank + 1] - v.offset[trank]) > kFastMaxBytes) {
-          const int slot = atomicAdd(&long_n, 1);
-          if (slot < kLongQueue) long_q[slot] = trank; else fail_everywhere();
-          continue;
-        }
+        if ((int)(v.offset[trank + 1] - v.offset[trank]) > kFastMaxBytes) { walk_slowly(trank); continue; }
         id = v.rank_to_id[trank];
         pass = walk_one(trank, v.offset[trank], e, 0);
       } else {
@@ -1328,23 +1372,18 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
         atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
       }
     }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      for (int i = 0; i < min(long_n, kLongQueue); ++i) {
-        const int trank = long_q[i];
-        const uint32_t off = v.offset[trank];
-        const int len = (int)(v.offset[trank + 1] - off);
-        int flags = 0;
-        const bool pass = token_walk<int16_t>(g, class_bits, hist, v.bytes + off, len, false, long_st, long_org, kLongCap, long_lsb, &flags, nullptr) == len;
-        if (flags & kWalkOverflow) fail_everywhere();
-        else if (pass) {
-          const int id = v.rank_to_id[trank];
+    __threadfence();           // queued tokens are visible to the block that walks them
+    cluster.sync();            // every remote OR has landed
+    if (sh_slow) {             // (the same in every block of the cluster)
+      if (rank == 0 && threadIdx.x == 0) {
+        const bool ok = run_slow_walks(mw, g, v, hist, [&](int id) {
           const int word = id >> 5, owner = word / chunk;
           atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
-        }
+        });
+        if (!ok) fail_everywhere();
       }
+      cluster.sync();
     }
-    cluster.sync();            // every remote OR has landed
   } else __syncthreads();
   // 3. write the slice
   const int failed = (total > 0 || fallback) ? sh_fail : 0;

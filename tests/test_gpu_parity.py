@@ -531,13 +531,62 @@ def test_long_tokens_up_to_255_bytes():
     batch.fill_next_token_bitmask(mask.data_ptr(), tok.words, st.data_ptr())
     assert np.array_equal(mask.cpu().numpy().view(np.uint32)[0], om.mask(ov))
     m.close(); g.close(); tok.close()
+    # the same through the two-kernel fill of the allocation-free entry point, and with a just-in-time grammar whose
+    # entries are all missing (the whole vocabulary, long tokens included, is walked against the Earley state)
+    feed = [b"{", b'"', b"q", b"q", b'"', b":", b" ", b"{", b"a" * 33, b"ab" * 40, b"a" * 40 + b"}", b"}"]
+    _drive(ebnf, toks, eos, feed, static_too=True)
+    tok = B.Tokenizer(toks, eos)
+    gj = B.Grammar(tok, "ebnf", ebnf, inline_max_states=0, jit=True, jit_precompute=0)
+    mj = B.Matcher(gj)
+    bj = B.Batch([mj])
+    om = O.Matcher(og)
+    for piece in feed:
+        for fill in (bj.fill_next_token_bitmask, bj.fill_next_token_bitmask_static):
+            fill(mask.data_ptr(), tok.words, st.data_ptr())
+            assert int(st.cpu()[0]) == 0 and np.array_equal(mask.cpu().numpy().view(np.uint32)[0], om.mask(ov)), piece
+        ids[0] = toks.index(piece)
+        bj.accept_token(ids.data_ptr(), st.data_ptr())
+        assert int(st.cpu()[0]) == 0 and om.accept_token(ov, toks.index(piece)) == 1
+    mj.close(); gj.close(); tok.close()
+
+
+def _drive(ebnf, toks, eos, feed, inline=0, static_too=False):
+    """Feed `feed` (token byte strings) to a matcher of grammar `ebnf`, comparing every mask (and the static
+    entry point's, when asked) and every accept status with the oracle."""
+    torch, engine = _engine()
+    tok = B.Tokenizer(toks, eos)
+    g = B.Grammar(tok, "ebnf", ebnf, inline_max_states=inline)
+    ov = O.Vocab(toks, eos)
+    om = O.Matcher(O.Grammar(ebnf))
+    m = B.Matcher(g)
+    batch = B.Batch([m])
+    mask = torch.zeros((1, tok.words), dtype=torch.int32, device="cuda")
+    mask2 = torch.zeros((1, tok.words), dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ids = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for piece in list(feed) + [None]:
+        batch.fill_next_token_bitmask(mask.data_ptr(), tok.words, st.data_ptr())
+        ref = om.mask(ov)
+        assert int(st.cpu()[0]) == 0 and np.array_equal(mask.cpu().numpy().view(np.uint32)[0], ref), piece
+        if static_too:
+            batch.fill_next_token_bitmask_static(mask2.data_ptr(), tok.words, st.data_ptr())
+            assert int(st.cpu()[0]) == 0 and np.array_equal(mask2.cpu().numpy().view(np.uint32)[0], ref), piece
+        if piece is None:
+            break
+        ids[0] = toks.index(piece)
+        batch.accept_token(ids.data_ptr(), st.data_ptr())
+        assert int(st.cpu()[0]) == 0, piece
+        assert om.accept_token(ov, toks.index(piece)) == 1
+    m.close(); g.close(); tok.close()
 
 
 def test_item_sets_beyond_the_fast_path():
-    """Sixty alternatives that all start with the same byte give Earley sets of sixty items: the cache is
-    still built exactly (slow path), while the run-time calls report XG_ERR_CAPACITY instead of guessing."""
+    """Sixty alternatives that all start with the same byte give Earley sets of sixty items, more than the fixed
+    arrays of a token walk hold: the cache is built by the exact slow path, the token is accepted through the
+    matcher's large scratch, the step plan that does not fit makes the fill walk the whole vocabulary, and the walks
+    that overflow there are redone one by one -- every mask still equals the oracle's, through both fill paths."""
     torch, engine = _engine()
-    toks = [bytes([b]) for b in range(256)] + [b"xa", b"xab", b"xq7", b"x", b"xa9!", b""]
+    toks = [bytes([b]) for b in range(256)] + [b"xa", b"xab", b"xq7", b"x", b"xa9!", b"q7", b"b3!", b""]
     toks += [b"\xfe\xff%d" % i for i in range(-len(toks) % 32)]
     eos = toks.index(b"")
     rules = "\n".join('alt%d ::= "x" [a-z]* "%d" "!"?' % (i, i % 10) for i in range(60))
@@ -545,27 +594,24 @@ def test_item_sets_beyond_the_fast_path():
     tok = B.Tokenizer(toks, eos)
     g = B.Grammar(tok, "ebnf", ebnf, inline_max_states=0)
     ov = O.Vocab(toks, eos)
-    t = g.tables()
-    scal = {k: t.pop(k) for k in ("n_rules", "n_states", "n_classes", "root_rule", "root_nullable")}
-    tb = O.Tables(scal["n_rules"], scal["n_states"], scal["n_classes"], scal["root_rule"], scal["root_nullable"], **t)
+    tb, _ = _oracle_tables(g)
     for s_ in tb.scannable_states()[::7]:
-        e = g.cache_entry(s_)
-        cls = tb.classify(ov, s_)
-        acc, unc = _entry_sets(e, len(toks))
-        assert acc == set(np.nonzero(cls == 1)[0].tolist()) and unc == set(np.nonzero(cls == 2)[0].tolist()), s_
-    m = B.Matcher(g)
-    batch = B.Batch([m])
-    mask = torch.zeros((1, tok.words), dtype=torch.int32, device="cuda")
-    st = torch.zeros(1, dtype=torch.int32, device="cuda")
-    batch.fill_next_token_bitmask(mask.data_ptr(), tok.words, st.data_ptr())
-    om = O.Matcher(O.Grammar(ebnf))
-    assert int(st.cpu()[0]) == 0 and np.array_equal(mask.cpu().numpy().view(np.uint32)[0], om.mask(ov))
-    ids = torch.tensor([toks.index(b"x")], dtype=torch.int32, device="cuda")
-    batch.accept_token(ids.data_ptr(), st.data_ptr())
-    assert int(st.cpu()[0]) == B.XG_ERR_CAPACITY          # sixty items do not fit; the state is unchanged
-    batch.fill_next_token_bitmask(mask.data_ptr(), tok.words, st.data_ptr())
-    assert int(st.cpu()[0]) == 0 and np.array_equal(mask.cpu().numpy().view(np.uint32)[0], om.mask(ov))
-    m.close(); g.close(); tok.close()
+        _check_entry(g, tb, ov, s_, tok.words)
+    g.close(); tok.close()
+    _drive(ebnf, toks, eos, [b"x", b"a", b"q7", b"!"], static_too=True)
+    _drive(ebnf, toks, eos, [b"xab", b"b3!"], static_too=True)
+
+
+def test_more_entries_to_check_than_the_plan_holds():
+    """Forty rules predicted at one position, each with tokens that run past its end: more (state, origin) entries
+    with uncertain tokens than the step plan lists.  The fill then takes the mask from the plain definition."""
+    toks = [bytes([b]) for b in range(256)] + [b"a0;", b"b1;;", b"c2", b"a0", b";", b"z9;a", b"m3;m", b""]
+    toks += [b"\xfe\xff%d" % i for i in range(-len(toks) % 32)]
+    eos = toks.index(b"")
+    letters = "abcdefghijklmnopqrstuvwxyzABCDEFGHIJKLMN"
+    rules = "\n".join('r%d ::= "%s" [0-9]+' % (i, letters[i]) for i in range(40))
+    ebnf = 'root ::= (item ";")+\nitem ::= ' + " | ".join("r%d" % i for i in range(40)) + "\n" + rules + "\n"
+    _drive(ebnf, toks, eos, [b"a0;", b"c2", b";", b"m3;m", b"7", b";"], static_too=True)
 
 
 def test_threaded_compile_into_one_pool_builds_the_same_cache():
@@ -615,3 +661,46 @@ def test_tool_pool_requests_share_the_tools_they_have_in_common():
     assert stats[0]["n_entries_reused"] < stats[-1]["n_entries_reused"]          # the pool fills up as requests arrive
     assert sum(x["n_entries_reused"] for x in stats[1:]) > 0
     s.close()
+
+
+def test_changing_batch_compositions_need_no_allocation_and_no_device_synchronisation():
+    """Continuous batching: every step one request leaves the batch and another joins, so every step's list of
+    matchers is new to the library.  Masks and accepts stay exact, and after the first steps the calls allocate no
+    device memory (the per-batch tables are a fixed set of slots that are reused)."""
+    torch, engine = _engine()
+    w = inputs.make_workload("C3", batch=12, steps=200, vocab_size=8192)
+    s = engine.Session(w)
+    ov, _, oms = _oracle_side(w)
+    n = s.n
+    pos = [0] * n                                         # next trajectory step of every request
+    mask = torch.zeros((8, s.W), dtype=torch.int32, device=s.device)
+    st = torch.zeros(8, dtype=torch.int32, device=s.device)
+    ids = torch.zeros(8, dtype=torch.int32, device=s.device)
+    free_after_warmup = None
+    try:
+        for step in range(200):
+            members = [(step + k) % n for k in range(8)]          # a window of 8 requests that slides by one every step
+            batch = B.Batch([s.matchers[b] for b in members])
+            batch.fill_next_token_bitmask(mask.data_ptr(), s.W, st.data_ptr(), s.stream())
+            got = mask.cpu().numpy().view(np.uint32)
+            assert (st.cpu().numpy() == 0).all()
+            toks = []
+            for k, b in enumerate(members):
+                if step % 5 == 0 or k == 7:
+                    assert np.array_equal(got[k], oms[b].mask(ov)), (step, b)
+                t = w.trajectories[b][pos[b] % w.steps]
+                pos[b] += 1
+                toks.append(t)
+            ids.copy_(torch.tensor(toks, dtype=torch.int32))
+            batch.accept_token(ids.data_ptr(), st.data_ptr(), s.stream(), restart_on_eos=True)
+            assert (st.cpu().numpy() == 0).all(), step
+            for k, b in enumerate(members):
+                if oms[b].accept_token(ov, toks[k]) == 2:
+                    oms[b].reset()
+            if step == 20:
+                torch.cuda.synchronize()
+                free_after_warmup = torch.cuda.mem_get_info()[0]
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_after_warmup
+    finally:
+        s.close()

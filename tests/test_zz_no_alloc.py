@@ -82,3 +82,65 @@ def test_static_fill_rejects_oversized_batches_and_bad_buffers():
         assert (rows == s.bitmask[0]).all()
     finally:
         s.close()
+
+
+def test_static_fill_allocates_no_device_memory_where_the_regular_call_does():
+    """The property the entry point exists for.  A batch composition that neither call has seen before: the static
+    call must leave the device's free memory as it was; the regular call, whose per-batch tables grow on first use
+    of a larger batch, serves (with a much larger batch) as the control that the probe would notice an allocation."""
+    import torch
+    from paper_2601_04426_b200 import engine
+    w = inputs.make_workload("C1", steps=2, vocab_size=2048)
+    s = engine.Session(w)
+    try:
+        n_big = 1000
+        many = B.Batch([s.matchers[0]] * n_big)
+        rows = torch.zeros((n_big, s.W), dtype=torch.int32, device=s.device)
+        n_control = 40000                                    # large enough for its tables (tens of MB) to show in the free memory
+        control = B.Batch([s.matchers[0]] * n_control)
+        rows2 = torch.zeros((n_control, s.W), dtype=torch.int32, device=s.device)
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        many.fill_next_token_bitmask_static(rows.data_ptr(), s.W)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 == free0                                # nothing allocated
+        control.fill_next_token_bitmask(rows2.data_ptr(), s.W)      # the regular call grows its per-batch tables here
+        torch.cuda.synchronize()
+        free2, _ = torch.cuda.mem_get_info()
+        assert free2 < free1
+        s.fill()
+        assert (rows == s.bitmask[0]).all() and (rows2 == s.bitmask[0]).all()
+    finally:
+        s.close()
+
+
+def test_static_fill_serves_a_just_in_time_grammar_with_missing_entries():
+    """A grammar whose cache entries are not built yet: the static call, like the regular one, takes the mask from a
+    walk of the whole vocabulary; both equal the oracle's mask."""
+    import torch
+    from oracle import oracle as O
+    from oracle import schema_ebnf as SE
+    w = inputs.make_workload("C1", steps=6, vocab_size=4096)
+    v = w.vocab
+    tok = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
+    g = B.Grammar(tok, w.grammars[0].kind, w.grammars[0].text, jit=True, jit_precompute=0)
+    m = B.Matcher(g)
+    batch = B.Batch([m])
+    ov = O.Vocab(v.tokens, v.eos_id, v.special_ids)
+    om = O.Matcher(O.Grammar(SE.grammar_text(w.grammars[0].kind, w.grammars[0].text)))
+    mask = torch.zeros((1, tok.words), dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ids = torch.zeros(1, dtype=torch.int32, device="cuda")
+    try:
+        for t in w.trajectories[0]:
+            for fill in (batch.fill_next_token_bitmask_static, batch.fill_next_token_bitmask):
+                mask.fill_(-1)
+                fill(mask.data_ptr(), tok.words, st.data_ptr())
+                assert int(st.cpu()[0]) == 0 and np.array_equal(mask.cpu().numpy().view(np.uint32)[0], om.mask(ov))
+            ids[0] = t
+            batch.accept_token(ids.data_ptr(), st.data_ptr())
+            if om.accept_token(ov, t) == 2:
+                break
+    finally:
+        m.close(); g.close(); tok.close()
