@@ -47,7 +47,8 @@ enum {
                                  set beyond even the exact slow path (2048 items per token walk) */
   XG_ERR_TOKEN_REJECTED = -7, /* xg_accept_token: the token is not allowed in this state */
   XG_ERR_TERMINATED = -8,     /* the matcher already accepted EOS */
-  XG_ERR_TIMEOUT = -9
+  XG_ERR_TIMEOUT = -9,
+  XG_ERR_BOUNDS = -10         /* bounds-checking build only: a kernel met an index outside its table (xg_debug_bounds_check) */
 };
 
 typedef enum { XG_EBNF = 0, XG_JSON_SCHEMA = 1, XG_TAG_DISPATCH_JSON = 2 } xg_grammar_kind_t;
@@ -62,6 +63,17 @@ typedef struct xg_matcher xg_matcher_t;
 
 /* Message of the last failing call on this thread ("" if none).  Valid until the next call. */
 const char* xg_last_error(void);
+
+/* ---- bounds-checking build -----------------------------------------------------------------
+ * The library can be built with -DXG_DEBUG_BOUNDS (paper_2601_04426_b200/build.py builds that variant
+ * as libxg_dbg.so): its kernels range-check every index into a grammar table, the vocabulary arena, a
+ * request's chart and another block's shared memory before using it.  A failed check records the first
+ * violation in a device word and skips the access; nothing traps.  xg_debug_bounds_check synchronises
+ * `stream`, returns XG_OK when no check has failed since the last call and XG_ERR_BOUNDS (message: which
+ * table, index, limit) otherwise, and clears the word.  In the regular build the checks do not exist and
+ * the call returns XG_OK.  xg_debug_bounds_enabled: 1 in the checking build, else 0. */
+int32_t xg_debug_bounds_enabled(void);
+xg_status_t xg_debug_bounds_check(void* stream);
 
 /* ---- vocabulary ---------------------------------------------------------------------------
  * The token set V of the tokenizer (appendix "Formal Definitions": V is the vocabulary).
@@ -89,6 +101,12 @@ void xg_cache_pool_destroy(xg_cache_pool_t* pool);
  * and returns a slab when nothing in it is live.
  * max_bytes <= 0: no limit (the default).  May synchronise the device when it evicts. */
 xg_status_t xg_cache_pool_set_limit(xg_cache_pool_t* pool, int64_t max_bytes);
+/* Take `bytes` of device memory for the pool now (Section 3.5: what can be prepared before requests arrive
+ * is).  Taking memory from the driver costs tens of microseconds per MiB; a pool that grows while grammars
+ * compile pays that inside their compile times, a server that knows its cache budget pays it once at start-up.
+ * The reservation is kept until the pool is destroyed and is used before any further memory is taken.
+ * XG_ERR_OOM if the device has no room.  Synchronous. */
+xg_status_t xg_cache_pool_reserve(xg_cache_pool_t* pool, int64_t bytes);
 typedef struct {
   int64_t bytes;             /* bytes of cache entries held now (what the limit bounds) */
   int64_t reserved_bytes;    /* device memory the pool's slabs hold, grammars' own tables included */

@@ -17,7 +17,7 @@ from . import build as _build
 
 XG_OK = 0
 XG_ERR_INVALID_ARG, XG_ERR_PARSE, XG_ERR_UNSUPPORTED, XG_ERR_OOM, XG_ERR_CUDA = -1, -2, -3, -4, -5
-XG_ERR_CAPACITY, XG_ERR_TOKEN_REJECTED, XG_ERR_TERMINATED, XG_ERR_TIMEOUT = -6, -7, -8, -9
+XG_ERR_CAPACITY, XG_ERR_TOKEN_REJECTED, XG_ERR_TERMINATED, XG_ERR_TIMEOUT, XG_ERR_BOUNDS = -6, -7, -8, -9, -10
 XG_EBNF, XG_JSON_SCHEMA, XG_TAG_DISPATCH_JSON = 0, 1, 2
 XG_F32, XG_BF16 = 0, 1
 XG_STORE_ACCEPT_LIST, XG_STORE_REJECT_LIST, XG_STORE_BITSET = 0, 1, 2
@@ -25,7 +25,7 @@ KIND_BY_NAME = {"ebnf": XG_EBNF, "json_schema": XG_JSON_SCHEMA, "tag_dispatch": 
 DTYPE_BY_NAME = {"f32": XG_F32, "bf16": XG_BF16}
 
 EXPORTS = [
-    "xg_last_error", "xg_tokenizer_create", "xg_tokenizer_destroy", "xg_cache_pool_create", "xg_cache_pool_destroy", "xg_cache_pool_set_limit", "xg_cache_pool_stats",
+    "xg_last_error", "xg_debug_bounds_enabled", "xg_debug_bounds_check", "xg_tokenizer_create", "xg_tokenizer_destroy", "xg_cache_pool_create", "xg_cache_pool_destroy", "xg_cache_pool_set_limit", "xg_cache_pool_reserve", "xg_cache_pool_stats",
     "xg_compile_grammar", "xg_grammar_destroy", "xg_grammar_get_tables", "xg_grammar_get_rule_hashes", "xg_grammar_get_cache_entry", "xg_grammar_get_state_classes", "xg_grammar_stats", "xg_jit_service",
     "xg_matcher_create", "xg_matcher_reset", "xg_matcher_destroy", "xg_matcher_is_terminated", "xg_matcher_next_fill_work",
     "xg_fill_next_token_bitmask", "xg_fill_next_token_bitmask_static", "xg_apply_token_bitmask", "xg_accept_token",
@@ -85,17 +85,25 @@ _lib = None
 
 
 def lib_path() -> str:
-    return _build.LIB
+    return _build.LIB_DEBUG if os.environ.get("XG_DEBUG_BOUNDS") == "1" else _build.LIB
+
+
+def debug_bounds_check(stream: int = 0):
+    """Raises XgError(XG_ERR_BOUNDS) if a kernel of the bounds-checking build met an index outside its table."""
+    _check(lib().xg_debug_bounds_check(stream))
 
 
 def lib():
-    """Load (building first if the sources are newer) libxg.so.  Raises if that is impossible."""
+    """Load (building first if the sources are newer) libxg.so -- or, with XG_DEBUG_BOUNDS=1 in the environment,
+    the bounds-checking variant libxg_dbg.so.  Raises if that is impossible."""
     global _lib
     if _lib is None:
-        path = _build.build()
+        path = _build.build(debug_bounds=os.environ.get("XG_DEBUG_BOUNDS") == "1")
         L = C.CDLL(path)
         vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
         L.xg_last_error.restype = C.c_char_p
+        L.xg_debug_bounds_enabled.restype = i32
+        L.xg_debug_bounds_check.argtypes = [vp]
         L.xg_tokenizer_create.argtypes = [vp, vp, i32, i32, vp, i32, vp, C.POINTER(vp)]
         L.xg_tokenizer_destroy.argtypes = [vp]
         L.xg_tokenizer_destroy.restype = None
@@ -103,6 +111,7 @@ def lib():
         L.xg_cache_pool_destroy.argtypes = [vp]
         L.xg_cache_pool_destroy.restype = None
         L.xg_cache_pool_set_limit.argtypes = [vp, i64]
+        L.xg_cache_pool_reserve.argtypes = [vp, i64]
         L.xg_cache_pool_stats.argtypes = [vp, C.POINTER(PoolStats)]
         L.xg_compile_grammar.argtypes = [vp, vp, C.c_int, C.c_char_p, C.c_size_t, C.c_char_p, C.POINTER(CompileOptions), vp, C.POINTER(vp)]
         L.xg_grammar_destroy.argtypes = [vp]
@@ -163,6 +172,9 @@ class CachePool:
 
     def set_limit(self, max_bytes: int):
         _check(lib().xg_cache_pool_set_limit(self.h, int(max_bytes)))
+
+    def reserve(self, n_bytes: int):
+        _check(lib().xg_cache_pool_reserve(self.h, int(n_bytes)))
 
     def stats(self) -> dict:
         s = PoolStats()

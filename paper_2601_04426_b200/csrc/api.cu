@@ -252,6 +252,8 @@ xg_status_t xg_tokenizer_create(const uint8_t* bytes, const int64_t* offsets, in
   t->dev.n_words = t->n_words;
   t->dev.eos_id = eos_token_id;
   t->dev.max_len = max_len;
+  t->dev.n_bytes = (uint32_t)arena.size();
+  t->dev.pad = 0;
   t->dev.bytes = keep(device_copy(arena, &err));
   if (err == cudaSuccess) t->dev.offset = keep(device_copy(off, &err));
   if (err == cudaSuccess) t->dev.rank_to_id = keep(device_copy(t->rank_to_id, &err));
@@ -281,6 +283,35 @@ void xg_tokenizer_destroy(xg_tokenizer_t* t) {
   delete t;
 }
 
+// ---------------------------------------------------------------------------------------------
+// bounds-checking build
+// ---------------------------------------------------------------------------------------------
+int32_t xg_debug_bounds_enabled(void) {
+#ifdef XG_DEBUG_BOUNDS
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+xg_status_t xg_debug_bounds_check(void* stream) {
+#ifdef XG_DEBUG_BOUNDS
+  static const char* what_name[] = {"?", "automaton state", "scan edge", "wait edge", "gather entry", "byte class", "token rank", "token bytes",
+                                    "chart set", "chart item", "walk item", "plan entry", "mask row word", "cluster block", "check list entry", "cache entry"};
+  XG_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  unsigned long long word = 0, zero = 0;
+  XG_CUDA(cudaMemcpyFromSymbol(&word, g_bounds_violation, sizeof word));
+  if (!word) return XG_OK;
+  XG_CUDA(cudaMemcpyToSymbol(g_bounds_violation, &zero, sizeof zero));
+  const int what = (int)((word >> 48) & 0x7FFF);
+  return set_error(XG_ERR_BOUNDS, std::string("bounds violation in a kernel: ") + (what >= 1 && what <= 15 ? what_name[what] : "?") + " index " +
+                                      std::to_string((long long)((word >> 24) & 0xFFFFFF)) + " (low 24 bits), limit " + std::to_string((long long)(word & 0xFFFFFF)));
+#else
+  (void)stream;
+  return XG_OK;
+#endif
+}
+
 xg_status_t xg_cache_pool_create(const xg_tokenizer_t* tok, xg_cache_pool_t** out) {
   if (!tok || !out) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
   *out = new xg_cache_pool{std::make_shared<CachePool>((const void*)tok)};
@@ -293,6 +324,13 @@ xg_status_t xg_cache_pool_set_limit(xg_cache_pool_t* pool, int64_t max_bytes) {
   std::lock_guard<std::mutex> lock(pool->impl->mu);
   pool->impl->set_limit(max_bytes);
   pool->impl->enforce_limit();
+  return XG_OK;
+}
+
+xg_status_t xg_cache_pool_reserve(xg_cache_pool_t* pool, int64_t bytes) {
+  if (!pool || bytes < 0) return set_error(XG_ERR_INVALID_ARG, "bad argument");
+  std::lock_guard<std::mutex> lock(pool->impl->mu);
+  if (!pool->impl->reserve((size_t)bytes)) return set_error(XG_ERR_OOM, "the device has no room for the reservation");
   return XG_OK;
 }
 
@@ -310,13 +348,17 @@ xg_status_t xg_cache_pool_stats(xg_cache_pool_t* pool, xg_cache_pool_stats_t* ou
 // ---------------------------------------------------------------------------------------------
 // the entry headers alone, once the tables are on the device (the headers change twice during a compile: when the
 // entries are built, and when this grammar's lookahead has narrowed their check lists)
-static xg_status_t upload_entry_headers(xg_grammar* g) {
+static xg_status_t upload_entry_headers(xg_grammar* g, cudaStream_t stream) {
   if (!g->blob) return set_error(XG_ERR_INVALID_ARG, "internal: tables not uploaded yet");
-  XG_CUDA(cudaMemcpy((uint8_t*)g->blob + g->entries_offset, g->entries.data(), g->entries.size() * sizeof(EntryDev), cudaMemcpyHostToDevice));
+  const size_t bytes = g->entries.size() * sizeof(EntryDev);
+  void* stage = g->pool->pinned(1, bytes);            // (the caller synchronises between two uploads of the headers)
+  if (!stage) return set_error(XG_ERR_OOM, "pinned staging allocation failed");
+  std::memcpy(stage, g->entries.data(), bytes);
+  XG_CUDA(cudaMemcpyAsync((uint8_t*)g->blob + g->entries_offset, stage, bytes, cudaMemcpyHostToDevice, stream));
   return XG_OK;
 }
 
-static xg_status_t upload_grammar(xg_grammar* g) {
+static xg_status_t upload_grammar(xg_grammar* g, cudaStream_t stream) {
   const FlatGrammar& f = g->flat;
   // one blob, sections 16-byte aligned
   size_t total = 0;
@@ -348,8 +390,10 @@ static xg_status_t upload_grammar(xg_grammar* g) {
   size_t o_rec = reserve(recs.size() * sizeof(StateRec)), o_scan = reserve(scan.size() * sizeof(uint2)), o_wait = reserve(wait.size() * sizeof(uint2)),
          o_gs = reserve(f.gather_state.size() * 4), o_cb = reserve(f.class_bits.size() * 4),
          o_en = reserve((size_t)f.n_states * sizeof(EntryDev)), o_self = reserve(sizeof(GrammarDev));
-  std::vector<uint8_t> host(total, 0);
-  auto put = [&](size_t at, const void* src, size_t bytes) { if (bytes) std::memcpy(host.data() + at, src, bytes); };
+  uint8_t* host = (uint8_t*)g->pool->pinned(0, total);       // (every compile ends with a synchronisation: the slot is free again)
+  if (!host) return set_error(XG_ERR_OOM, "pinned staging allocation failed");
+  std::memset(host, 0, total);
+  auto put = [&](size_t at, const void* src, size_t bytes) { if (bytes) std::memcpy(host + at, src, bytes); };
   put(o_first, state_first.data(), state_first.size() * 4);
   put(o_follow, f.rule_follow.data(), f.rule_follow.size() * 4);
   put(o_rec, recs.data(), recs.size() * sizeof(StateRec));
@@ -377,9 +421,10 @@ static xg_status_t upload_grammar(xg_grammar* g) {
   g->entries_offset = o_en;
   v.miss_ring = g->jit.slot >= 0 ? ((JitPool*)g->pool->jit_host)->d_ring : nullptr;
   v.jit_slot = g->jit.slot;
+  v.n_scan_edges = (int32_t)scan.size(); v.n_wait_edges = (int32_t)wait.size(); v.n_gather = (int32_t)f.gather_state.size();
   put(o_self, &v, sizeof(GrammarDev));
   g->dev = (GrammarDev*)(d + o_self);
-  XG_CUDA(cudaMemcpy(g->blob, host.data(), total, cudaMemcpyHostToDevice));
+  XG_CUDA(cudaMemcpyAsync(g->blob, host, total, cudaMemcpyHostToDevice, stream));
   return XG_OK;
 }
 
@@ -395,6 +440,7 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
   const int over_cap = 1 << 16;
   CachePool& pool = *g->pool;
   int32_t* d_pos = (int32_t*)pool.scratch(0, per_batch * sizeof(int32_t));
+  int32_t* h_pos = (int32_t*)pool.pinned(4, per_batch * sizeof(int32_t));
   uint32_t* d_rows = (uint32_t*)pool.scratch(1, 3 * row_bytes * per_batch);
   int2* d_counts = (int2*)pool.scratch(2, per_batch * sizeof(int2));
   PackPlan* d_plan = (PackPlan*)pool.scratch(3, per_batch * sizeof(PackPlan));
@@ -402,7 +448,7 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
   EntryDev* d_entries = (EntryDev*)pool.scratch(5, per_batch * sizeof(EntryDev));
   int2* d_over = (int2*)pool.scratch(6, over_cap * sizeof(int2));
   int* d_over_count = (int*)pool.scratch(7, 2 * sizeof(int));
-  if (!d_pos || !d_rows || !d_counts || !d_plan || !d_total || !d_entries || !d_over || !d_over_count)
+  if (!h_pos || !d_pos || !d_rows || !d_counts || !d_plan || !d_total || !d_entries || !d_over || !d_over_count)
     return set_error(XG_ERR_OOM, "cache build scratch allocation failed");
   auto cleanup = [&]() {};
 #define XG_CUDA_C(expr) do { cudaError_t e__ = (expr); if (e__ != cudaSuccess) { cleanup(); return set_error(XG_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)); } } while (0)
@@ -411,7 +457,8 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
     uint32_t* acc = d_rows;
     uint32_t* unc = d_rows + (size_t)per_batch * W;
     uint32_t* unr = d_rows + 2 * (size_t)per_batch * W;
-    XG_CUDA_C(cudaMemcpyAsync(d_pos, states.data() + begin, n * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+    std::memcpy(h_pos, states.data() + begin, n * sizeof(int32_t));       // (the previous batch ended with a synchronisation)
+    XG_CUDA_C(cudaMemcpyAsync(d_pos, h_pos, n * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
     XG_CUDA_C(cudaMemsetAsync(acc, 0, row_bytes * n, stream));      // blocks with nothing to scan leave their part of the rows untouched
     XG_CUDA_C(cudaMemsetAsync(unc, 0, row_bytes * n, stream));
     XG_CUDA_C(cudaMemsetAsync(unr, 0, row_bytes * n, stream));
@@ -432,8 +479,15 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
     classify_kernel<false><<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, acc, unc, unr, d_over, d_over_count, over_cap, nullptr);
     XG_CUDA_C(cudaGetLastError());
     if (ev) cudaEventRecord(ev[1], stream);
+    // count and plan are enqueued behind the classification at once; walks that left the fast path are rare, and when
+    // there are some the two small kernels are simply run again after the exact fallback
+    count_kernel<<<n, 256, 0, stream>>>(acc, unc, W, d_counts);
+    plan_kernel<<<1, 1024, 0, stream>>>(d_counts, n, V, W, d_plan, d_total);
+    XG_CUDA_C(cudaGetLastError());
     int over[2] = {0, 0};
+    long long total_words = 0;
     XG_CUDA_C(cudaMemcpyAsync(over, d_over_count, 2 * sizeof(int), cudaMemcpyDeviceToHost, stream));
+    XG_CUDA_C(cudaMemcpyAsync(&total_words, d_total, sizeof(long long), cudaMemcpyDeviceToHost, stream));
     XG_CUDA_C(cudaStreamSynchronize(stream));
     if (ev) { float ms = 0.f; if (cudaEventElapsedTime(&ms, ev[0], ev[1]) == cudaSuccess) g->stats.classify_ms += ms; }
     if (over[0] > over_cap) { cleanup(); return set_error(XG_ERR_CAPACITY, "too many token walks exceeded the fast path"); }
@@ -451,13 +505,12 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
     if (over[0] > 0) {
       XG_CUDA_C(cudaMemcpy(over, d_over_count, 2 * sizeof(int), cudaMemcpyDeviceToHost));
       if (over[1]) { cleanup(); return set_error(XG_ERR_CAPACITY, "an Earley item set exceeded the supported size during cache build"); }
+      count_kernel<<<n, 256, 0, stream>>>(acc, unc, W, d_counts);
+      plan_kernel<<<1, 1024, 0, stream>>>(d_counts, n, V, W, d_plan, d_total);
+      XG_CUDA_C(cudaGetLastError());
+      XG_CUDA_C(cudaMemcpyAsync(&total_words, d_total, sizeof(long long), cudaMemcpyDeviceToHost, stream));
+      XG_CUDA_C(cudaStreamSynchronize(stream));
     }
-    count_kernel<<<n, 256, 0, stream>>>(acc, unc, W, d_counts);
-    plan_kernel<<<1, 1024, 0, stream>>>(d_counts, n, V, W, d_plan, d_total);
-    XG_CUDA_C(cudaGetLastError());
-    long long total_words = 0;
-    XG_CUDA_C(cudaMemcpyAsync(&total_words, d_total, sizeof(long long), cudaMemcpyDeviceToHost, stream));
-    XG_CUDA_C(cudaStreamSynchronize(stream));
     int chunk_id = -1;
     uint32_t* arena = (uint32_t*)g->pool->allocate_device((size_t)std::max<long long>(total_words, 1) * 4, &chunk_id);
     if (!arena) { cleanup(); return set_error(XG_ERR_OOM, "cache arena allocation failed"); }
@@ -479,7 +532,8 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
 // Lookahead pass (Section 3.3): the pool's entries are context-free; each grammar narrows their
 // uncertain lists with its own follow sets.  Count, exclusive scan on the host (a few thousand
 // numbers), compact.  The grammar's entry headers must already be on the device.
-static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>& scannable, const std::vector<int32_t>& rep, cudaStream_t stream) {
+static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>& scannable, const std::vector<int32_t>& rep, cudaStream_t stream, bool* narrowed) {
+  *narrowed = false;
   std::vector<int32_t> states;
   for (int s : scannable) if (g->entries[s].n_unc > 0 && rep[s] == s) states.push_back(s);      // one list per shared entry
   if (states.empty()) return XG_OK;
@@ -490,7 +544,11 @@ static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>&
   int32_t* d_counts = (int32_t*)pool.scratch(12, (size_t)n * 4);
   long long* d_offsets = (long long*)pool.scratch(13, (size_t)n * 8);
   if (!d_states || !d_counts || !d_offsets) return set_error(XG_ERR_OOM, "lookahead scratch allocation failed");
-  XG_CUDA(cudaMemcpyAsync(d_states, states.data(), (size_t)n * 4, cudaMemcpyHostToDevice, stream));
+  int32_t* h_states = (int32_t*)pool.pinned(2, (size_t)n * 4);
+  long long* h_offsets = (long long*)pool.pinned(3, (size_t)n * 8);
+  if (!h_states || !h_offsets) return set_error(XG_ERR_OOM, "pinned staging allocation failed");
+  std::memcpy(h_states, states.data(), (size_t)n * 4);
+  XG_CUDA(cudaMemcpyAsync(d_states, h_states, (size_t)n * 4, cudaMemcpyHostToDevice, stream));
   lookahead_count_kernel<<<n, 256, 0, stream>>>(g->host_view, g->tok->dev, d_states, d_counts, nullptr);
   XG_CUDA(cudaGetLastError());
   std::vector<int32_t> counts(n);
@@ -501,10 +559,10 @@ static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>&
   for (int k = 0; k < n; ++k) { offsets[k] = total; total += 2LL * counts[k] + (counts[k] + 3) / 4; }
   g->lookahead_arena = pool.allocate_plain((size_t)std::max<long long>(total, 1) * 4);
   if (!g->lookahead_arena) return set_error(XG_ERR_OOM, "check list allocation failed");
-  XG_CUDA(cudaMemcpyAsync(d_offsets, offsets.data(), (size_t)n * 8, cudaMemcpyHostToDevice, stream));
+  std::memcpy(h_offsets, offsets.data(), (size_t)n * 8);
+  XG_CUDA(cudaMemcpyAsync(d_offsets, h_offsets, (size_t)n * 8, cudaMemcpyHostToDevice, stream));
   lookahead_compact_kernel<<<n, 256, 0, stream>>>(g->host_view, g->tok->dev, d_states, d_offsets, d_counts, (uint32_t*)g->lookahead_arena, nullptr);
-  XG_CUDA(cudaGetLastError());
-  XG_CUDA(cudaStreamSynchronize(stream));
+  XG_CUDA(cudaGetLastError());          // (the caller synchronises once the narrowed headers are on their way too)
   uint32_t* arena = (uint32_t*)g->lookahead_arena;
   for (int k = 0; k < n; ++k) {
     EntryDev& e = g->entries[states[k]];
@@ -519,6 +577,7 @@ static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>&
     EntryDev& e = g->entries[s];
     e.chk_rank = r.chk_rank; e.chk_exit = r.chk_exit; e.chk_byte = r.chk_byte; e.n_chk = r.n_chk;
   }
+  *narrowed = true;
   return XG_OK;
 }
 
@@ -929,7 +988,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     st = jit_allocate(g.get(), jit_arena_words);
     if (st != XG_OK) return fail(st);
   }
-  st = upload_grammar(g.get());
+  st = upload_grammar(g.get(), (cudaStream_t)stream);
   if (st != XG_OK) return fail(st);
   // cross-grammar cache (Section 3.3): rules whose canonical structure is already in the pool
   // reuse its entries; the others are classified now and registered afterwards
@@ -1042,9 +1101,11 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
       return fail(set_error(XG_ERR_CUDA, "upload of the state classes failed"));
     j.enabled = true;
   }
-  st = upload_entry_headers(g.get());       // now with the entry headers
-  if (st == XG_OK) st = narrow_check_lists(g.get(), scannable, rep, (cudaStream_t)stream);
-  if (st == XG_OK) st = upload_entry_headers(g.get());       // and with this grammar's narrowed check lists
+  st = upload_entry_headers(g.get(), (cudaStream_t)stream);       // now with the entry headers
+  bool narrowed = false;
+  if (st == XG_OK) st = narrow_check_lists(g.get(), scannable, rep, (cudaStream_t)stream, &narrowed);      // (synchronises after its first kernel)
+  if (st == XG_OK && narrowed) st = upload_entry_headers(g.get(), (cudaStream_t)stream);       // and with this grammar's narrowed check lists
+  if (st == XG_OK && cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) st = set_error(XG_ERR_CUDA, "cache build failed on the device");
   if (st != XG_OK) return fail(st);
   g->stats.cache_build_ms = now_ms() - t1 + pre_ms;
   g->stats.n_entries_built = (int)to_build.size();

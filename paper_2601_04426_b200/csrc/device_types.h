@@ -7,6 +7,20 @@
 
 namespace xg {
 
+// Bounds-checking build (-DXG_DEBUG_BOUNDS): every index into a grammar table, the vocabulary arena, a request's
+// chart or another block's shared memory is range-checked before use.  A check that fails records the first
+// violation in a device word (what, index, limit) and makes the code skip the access -- it never traps.  The
+// host reads the word with xg_debug_bounds_check.  Without the flag the checks compile to nothing.
+enum : int {
+  kBoundState = 1, kBoundScanEdge, kBoundWaitEdge, kBoundGather, kBoundClass, kBoundTokenRank, kBoundTokenBytes,
+  kBoundChartSet, kBoundChartItem, kBoundWalkItem, kBoundPlanEntry, kBoundRowWord, kBoundClusterBlock, kBoundCheckList, kBoundEntry
+};
+#ifdef XG_DEBUG_BOUNDS
+#define XG_BOUND(index, limit, what) ::xg::bound_ok((long long)(index), (long long)(limit), (what))
+#else
+#define XG_BOUND(index, limit, what) true
+#endif
+
 // Vocabulary, sorted by token bytes (trie order): tokens that share a prefix are adjacent, so
 // neighbouring lanes of a warp walk the same automaton path for the shared prefix.
 struct VocabDev {
@@ -20,6 +34,8 @@ struct VocabDev {
   const int32_t* id_to_rank; // [V]
   const uint8_t* never;      // [V] by rank: 1 = EOS, special or zero-length (never classified)
   const uint16_t* block_first; // [ceil(V / 256)]: first byte of the first token of a block of 256 ranks | first byte of its last << 8
+  uint32_t n_bytes;            // size of the arena (for the bounds-checking build)
+  uint32_t pad;
 };
 
 // One adaptive cache entry (Section 3.4): the accepted/rejected split in its smallest form plus
@@ -85,7 +101,7 @@ struct GrammarDev {
   const EntryDev* entries;        // [S]; meaningful for scannable states
   JitRing* miss_ring;             // just-in-time grammars only (else nullptr)
   int32_t jit_slot;               // this grammar's number in the ring's reports
-  int32_t pad3;
+  int32_t n_scan_edges, n_wait_edges, n_gather;      // table sizes (for the bounds-checking build)
 };
 
 // What the next mask needs from the current Earley set, worked out once when the set is made

@@ -13,6 +13,16 @@ namespace xg {
 
 enum : int { kWalkUncertain = 1, kWalkOverflow = 2 };
 
+#ifdef XG_DEBUG_BOUNDS
+// first violation: 1 << 63 | what << 48 | (index & 0xFFFFFF) << 24 | (limit & 0xFFFFFF)
+__device__ unsigned long long g_bounds_violation = 0ull;
+__device__ __forceinline__ bool bound_ok(long long index, long long limit, int what) {
+  if (index >= 0 && index < limit) return true;
+  atomicCAS(&g_bounds_violation, 0ull, (1ull << 63) | ((unsigned long long)what << 48) | (((unsigned long long)index & 0xFFFFFFull) << 24) | ((unsigned long long)limit & 0xFFFFFFull));
+  return false;
+}
+#endif
+
 // Programmatic dependent launch: the three kernels of a decode step are short, so the gap between
 // one kernel's end and the next one's start is a large share of the step.  Each of them lets the
 // next kernel of the stream be scheduled at once (its blocks become resident as room appears) and
@@ -50,6 +60,7 @@ struct Chart {
   const uint32_t* i_st;
   const int32_t* i_org;
   int i_cnt, i_idx;
+  int h_items;          // items in the history (bounds-checking build)
 };
 
 __device__ __forceinline__ Chart chart_of_history(const uint32_t* h_st, const int32_t* h_org, const int32_t* h_sb, int n) {
@@ -57,6 +68,7 @@ __device__ __forceinline__ Chart chart_of_history(const uint32_t* h_st, const in
   c.h_st = h_st; c.h_org = h_org; c.h_sb = h_sb; c.n = n;
   const int b = h_sb[n];
   c.i_st = h_st + b; c.i_org = h_org + b; c.i_cnt = h_sb[n + 1] - b; c.i_idx = n;
+  c.h_items = h_sb[n + 1];
   return c;
 }
 
@@ -75,14 +87,23 @@ __device__ __forceinline__ bool advance_waiters(const GrammarDev& g, const Chart
   const uint32_t* src_st;
   const int32_t* src_org;
   int b, e;
-  if (o < c.i_idx) { src_st = c.h_st; src_org = c.h_org; b = c.h_sb[o]; e = c.h_sb[o + 1]; }
+  if (o < c.i_idx) {
+    if (!XG_BOUND(o, c.n + 1, kBoundChartSet)) return true;
+    src_st = c.h_st; src_org = c.h_org; b = c.h_sb[o]; e = c.h_sb[o + 1];
+    if (!XG_BOUND(e, c.h_items + 1, kBoundChartItem) || !XG_BOUND(b, e + 1, kBoundChartItem)) return true;
+  }
   else if (o == c.i_idx) { src_st = c.i_st; src_org = c.i_org; b = 0; e = c.i_cnt; }
-  else { src_st = st; src_org = org; b = lsb[o - c.i_idx]; e = lsb[o - c.i_idx + 1]; }
+  else {
+    src_st = st; src_org = org; b = lsb[o - c.i_idx]; e = lsb[o - c.i_idx + 1];
+    if (!XG_BOUND(e, cnt + 1, kBoundWalkItem) || !XG_BOUND(b, e + 1, kBoundWalkItem)) return true;
+  }
   for (int i = b; i < e; ++i) {
     const uint32_t s2 = src_st[i];
     const int32_t o2 = src_org[i];
+    if (!XG_BOUND(s2, g.n_states, kBoundState)) continue;
     const uint4 rec = *reinterpret_cast<const uint4*>(&g.state[s2]);
     const int wait_end = (int)rec.z + (int)(rec.w & 0xFFFFu);
+    if (!XG_BOUND(wait_end, g.n_wait_edges + 1, kBoundWaitEdge)) continue;
     // four edges at a time: their loads are issued together, then compared (one at a time, each load would be
     // waited for before the next is even issued)
     for (int w = (int)rec.z; w < wait_end; w += 4) {
@@ -118,9 +139,11 @@ __device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* c
     for (int i = cur_b; i < cur_e; ++i) {
       const uint32_t s = cur_st[i];
       const int32_t o = cur_org[i];
+      if (!XG_BOUND(s, g.n_states, kBoundState)) continue;
       const uint4 ra = *reinterpret_cast<const uint4*>(&g.state[s]);
       const int n_edges = (k == 0 && own_edges_first) ? (int)(ra.y & 0xFFFFu) : (int)(ra.y >> 16);
       if (n_edges == 0) continue;
+      if (!XG_BOUND((int)ra.x + n_edges, g.n_scan_edges + 1, kBoundScanEdge)) continue;
       const uint4 rb = *(reinterpret_cast<const uint4*>(&g.state[s]) + 1);
       // the first edge is inline in the record; the others are fetched four at a time (loads issued together, then tested)
       for (int e = 0; e < n_edges; e += 4) {
@@ -131,6 +154,7 @@ __device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* c
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           if (e + u >= n_edges) break;
+          if (!(se[u].x & kLiteral) && !XG_BOUND(se[u].x, g.n_classes, kBoundClass)) continue;
           const bool hit = (se[u].x & kLiteral) ? ((se[u].x & 0x1FFu) == byte) : ((class_bits[se[u].x * 8 + word] & bit) != 0);
           if (hit && !add_item(st, org, start, cnt, cap, se[u].y & ~kSelf, (se[u].y & kSelf) ? self_idx : o)) { *flags |= kWalkOverflow; return k; }
         }
@@ -139,6 +163,7 @@ __device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* c
     if (cnt == start) return k;
     // complete (cascades through the growing set)
     for (int q = start; q < cnt; ++q) {
+      if (!XG_BOUND(st[q], g.n_states, kBoundState)) continue;
       const uint32_t info = g.state[st[q]].info;
       if (!(info >> 31)) continue;
       const int32_t o = org[q];
@@ -235,7 +260,7 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
         int32_t org[kFastCap];
         int16_t lsb[kFastMaxBytes + 2];
         Chart c;
-        c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1;
+        c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1; c.h_items = 0;
         c.i_st = sh_st; c.i_org = sh_org; c.i_cnt = 1; c.i_idx = 0;
         consumed = token_walk<int16_t>(g, class_bits, c, v.bytes + off, len, true, st, org, kFastCap, lsb, &flags, nullptr);
         walked = consumed;
@@ -271,7 +296,7 @@ __global__ void classify_slow_kernel(GrammarDev g, VocabDev v, const int32_t* __
   uint32_t h_st = (uint32_t)positions[pos];
   int32_t h_org = -1;
   Chart c;
-  c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1;
+  c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1; c.h_items = 0;
   c.i_st = &h_st; c.i_org = &h_org; c.i_cnt = 1; c.i_idx = 0;
   const uint32_t off = v.offset[rank];
   const int len = (int)(v.offset[rank + 1] - off);
@@ -435,7 +460,7 @@ exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, con
       int16_t lsb[kFastMaxBytes + 2];
       int flags = 0;
       Chart c;
-      c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1;
+      c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1; c.h_items = 0;
       c.i_st = sh_st; c.i_org = sh_org; c.i_cnt = 1; c.i_idx = 0;
       token_walk<int16_t>(g, class_bits, c, v.bytes + off, len, true, st, org, kFastCap, lsb, &flags, &mask);
       if (flags & kWalkOverflow) mask = 0;
@@ -615,10 +640,13 @@ __device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g,
     p.check_cum[0] = 0;
     for (int i = 0; i < hist.i_cnt && !overflow; ++i) {
       const uint32_t s = hist.i_st[i];
+      if (!XG_BOUND(s, g.n_states, kBoundState)) continue;
       const StateRec rec = g.state[s];
+      if (!XG_BOUND(rec.gather_begin + (int)(rec.n_wait_n_gather >> 16), g.n_gather + 1, kBoundGather)) continue;
       for (int gi = rec.gather_begin; gi < rec.gather_begin + (int)(rec.n_wait_n_gather >> 16); ++gi) {
         const int code = g.gather_state[gi];
         const int q = code & 0x7FFFFFFF;
+        if (!XG_BOUND(q, g.n_states, kBoundEntry)) continue;
         const int origin = code < 0 ? n : hist.i_org[i];          // predicted start states begin here
         bool seen = false;
         if (g.entries[q].kind == kEntryNotBuilt) {                // a just-in-time grammar has not built this entry yet
@@ -703,10 +731,12 @@ __device__ __forceinline__ int accept_one(MatcherDev& m, const GrammarDev& g, co
   // tested, so that they travel together instead of one after the other.
   const bool tok_ok = tok >= 0 && tok < v.vocab_size;
   const int rank = v.id_to_rank[tok_ok ? tok : 0];
+  if (!XG_BOUND(rank, v.vocab_size, kBoundTokenRank)) return -6;
   int n_sets = m.n_sets, n_items = m.n_items;
   const Chart c0 = chart_of_history(m.item_state, m.item_origin, m.set_begin, n_sets - 1);
   const uint32_t off = v.offset[rank];
   const int len = (int)(v.offset[rank + 1] - off);
+  if (!XG_BOUND((long long)off + len, (long long)v.n_bytes + 1, kBoundTokenBytes)) return -6;
   const bool never = v.never[rank] != 0;
   if (c0.i_cnt > 0) asm volatile("prefetch.global.L1 [%0];" ::"l"(&g.state[c0.i_st[0]]));
   if (m.terminated) return -8;
@@ -749,6 +779,7 @@ __device__ __forceinline__ int accept_one(MatcherDev& m, const GrammarDev& g, co
     // append the new sets behind the history (visible to the next piece; committed below)
     const uint32_t* src_st = slow ? m.slow_st : w_st;
     const int32_t* src_org = slow ? m.slow_org : w_org;
+    if (!XG_BOUND(n_items + made, m.cap_items + 1, kBoundChartItem) || !XG_BOUND(n_sets + piece, m.cap_sets + 1, kBoundChartSet)) { st = -6; break; }
     for (int q = lane; q < made; q += 32) { m.item_state[n_items + q] = src_st[q]; m.item_origin[n_items + q] = src_org[q]; }
     for (int j = 1 + lane; j <= piece; j += 32) m.set_begin[n_sets + j] = n_items + (slow ? m.slow_lsb[j + 1] : (int)lsb[j + 1]);
     __syncwarp();
@@ -1336,7 +1367,8 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
         if (walk_one(r, off, 0, 0)) {
           const int id = v.rank_to_id[r];
           const int word = id >> 5, owner = word / chunk;
-          atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
+          if (XG_BOUND(word, v.n_words, kBoundRowWord) && XG_BOUND(owner, n_blocks, kBoundClusterBlock))
+            atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
         }
       }
     }
@@ -1346,8 +1378,10 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
       int e = 0;
       while (j >= ent_cum[e + 1]) ++e;
       const int k = j - ent_cum[e];
+      if (!XG_BOUND(e, n_ent, kBoundPlanEntry) || !XG_BOUND(k, ent_cum[e + 1] - ent_cum[e], kBoundCheckList)) continue;
       uint32_t left = ent_exit[e][k];
       const int trank = (int)ent_rank[e][k];      // read together with the exit mask: one dependent load less for the survivors
+      if (!XG_BOUND(trank, v.vocab_size, kBoundTokenRank)) continue;
       bool pass = false;
       int id = -1;
       if (left == 0) {                // no exit record (very long token, or its build-time walk overflowed): walk in full
@@ -1369,7 +1403,8 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
       }
       if (pass) {
         const int word = id >> 5, owner = word / chunk;
-        atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
+        if (XG_BOUND(word, v.n_words, kBoundRowWord) && XG_BOUND(owner, n_blocks, kBoundClusterBlock))
+          atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
       }
     }
     __threadfence();           // queued tokens are visible to the block that walks them
@@ -1378,7 +1413,8 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
       if (rank == 0 && threadIdx.x == 0) {
         const bool ok = run_slow_walks(mw, g, v, hist, [&](int id) {
           const int word = id >> 5, owner = word / chunk;
-          atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
+          if (XG_BOUND(word, v.n_words, kBoundRowWord) && XG_BOUND(owner, n_blocks, kBoundClusterBlock))
+            atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
         });
         if (!ok) fail_everywhere();
       }

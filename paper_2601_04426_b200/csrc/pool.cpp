@@ -32,7 +32,7 @@ void* DeviceArena::alloc(size_t bytes) {
       if (blk.second >= bytes) { slab = i; offset = blk.first; break; }
   }
   if (slab < 0) {
-    const size_t want = std::max(bytes, std::min<size_t>(size_t(64) << 20, std::max<size_t>(size_t(1) << 20, reserved_)));
+    const size_t want = std::max(bytes, std::min<size_t>(size_t(256) << 20, std::max<size_t>(size_t(1) << 20, reserved_)));
     void* base = nullptr;
     size_t got = want;
     if (cudaMalloc(&base, got) != cudaSuccess) {
@@ -59,6 +59,24 @@ void* DeviceArena::alloc(size_t bytes) {
   return p;
 }
 
+bool DeviceArena::reserve(size_t bytes) {
+  while (bytes > 0) {
+    const size_t want = std::min<size_t>(bytes, size_t(1) << 30);
+    void* base = nullptr;
+    if (cudaMalloc(&base, want) != cudaSuccess) { cudaGetLastError(); return false; }
+    int slab = 0;
+    for (; slab < (int)slabs_.size() && slabs_[slab].base; ++slab) {}
+    if (slab == (int)slabs_.size()) slabs_.emplace_back();
+    Slab& s = slabs_[slab];
+    s.base = (char*)base; s.bytes = want; s.used = 0; s.keep = true;
+    s.free_blocks.clear();
+    s.free_blocks[0] = want;
+    reserved_ += want;
+    bytes -= want;
+  }
+  return true;
+}
+
 void DeviceArena::free(void* p) {
   auto it = live_.find(p);
   if (it == live_.end()) return;
@@ -67,7 +85,7 @@ void DeviceArena::free(void* p) {
   live_.erase(it);
   Slab& s = slabs_[slab];
   s.used -= bytes;
-  if (s.used == 0) {                     // nothing left in it: back to the driver
+  if (s.used == 0 && !s.keep) {          // nothing left in it: back to the driver
     cudaFree(s.base);
     reserved_ -= s.bytes;
     s = Slab();
@@ -85,6 +103,7 @@ void DeviceArena::free(void* p) {
 
 CachePool::~CachePool() {
   for (auto& s : scratch_) cudaFree(s.first);
+  for (auto& s : pinned_) if (s.first) cudaFreeHost(s.first);
   cudaFree(jit_.d_used);
   if (jit_host && jit_host_free) jit_host_free(jit_host);
   for (cudaEvent_t e : timing_) if (e) cudaEventDestroy(e);
@@ -123,6 +142,19 @@ void* CachePool::scratch(int slot, size_t bytes) {
     s = {nullptr, 0};
     size_t want = bytes + bytes / 4;
     if (cudaMalloc(&s.first, want) != cudaSuccess) { s.first = nullptr; return nullptr; }
+    s.second = want;
+  }
+  return s.first;
+}
+
+void* CachePool::pinned(int slot, size_t bytes) {
+  if ((int)pinned_.size() <= slot) pinned_.resize(slot + 1, {nullptr, 0});
+  auto& s = pinned_[slot];
+  if (s.second < bytes) {
+    if (s.first) cudaFreeHost(s.first);
+    s = {nullptr, 0};
+    size_t want = bytes + bytes / 2;
+    if (cudaHostAlloc(&s.first, want, cudaHostAllocDefault) != cudaSuccess) { s.first = nullptr; return nullptr; }
     s.second = want;
   }
   return s.first;

@@ -44,17 +44,18 @@ std::shared_ptr<const void> prepare_interning(const FlatGrammar& g);
 // Device memory in slabs with a first-fit free list.  Compiling a grammar needs a handful of
 // device buffers (its tables, a batch of cache entries, its narrowed check lists); taking each
 // from the driver costs a driver allocation apiece, which on a busy host takes from tens of
-// microseconds to tens of milliseconds.  Slabs grow geometrically up to 64 MiB, so a pool that
+// microseconds to tens of milliseconds.  Slabs grow geometrically up to 256 MiB, so a pool that
 // serves many grammars asks the driver a few dozen times in its life.  Not thread-safe: the
 // owner serialises calls.
 class DeviceArena {
  public:
   ~DeviceArena();
   void* alloc(size_t bytes);            // 256-byte aligned; nullptr when the device is out of memory
-  void free(void* p);                   // p from alloc(); an empty slab goes back to the driver
+  void free(void* p);                   // p from alloc(); an empty slab goes back to the driver (unless it was reserved)
+  bool reserve(size_t bytes);           // take slabs for `bytes` from the driver now; they stay until the arena is destroyed
   size_t reserved() const { return reserved_; }
  private:
-  struct Slab { char* base = nullptr; size_t bytes = 0, used = 0; std::map<size_t, size_t> free_blocks; };   // offset -> length
+  struct Slab { char* base = nullptr; size_t bytes = 0, used = 0; bool keep = false; std::map<size_t, size_t> free_blocks; };   // offset -> length
   std::vector<Slab> slabs_;
   std::unordered_map<void*, std::pair<int, size_t>> live_;      // block -> (slab, bytes)
   size_t reserved_ = 0;
@@ -79,6 +80,7 @@ class CachePool {
   // Plain device memory from the pool's slabs for a grammar's own tables (not subject to the limit).
   void* allocate_plain(size_t bytes) { return arena_.alloc(bytes); }
   void free_plain(void* p) { if (p) arena_.free(p); }
+  bool reserve(size_t bytes) { return arena_.reserve(bytes); }
   void retain(const std::vector<int>& chunk_ids);          // a grammar starts using these chunks
   void release(const std::vector<int>& chunk_ids);         // ... and stops (locks `mu` itself)
   void release_held(const std::vector<int>& chunk_ids);    // the same with `mu` already held
@@ -89,6 +91,10 @@ class CachePool {
   Stats stats() const;
   // reusable build scratch (grow-only, one buffer per slot; call with `mu` held)
   void* scratch(int slot, size_t bytes);
+  // reusable pinned host staging for uploads (grow-only, one buffer per slot; call with `mu` held).  A copy from
+  // pageable memory makes the runtime synchronise the stream first; from here it is only enqueued.  The caller
+  // must have synchronised with the previous copy out of a slot before writing to it again.
+  void* pinned(int slot, size_t bytes);
 
   // Arena of the just-in-time builds (Section 3.5).  A build that runs inside the decode loop
   // cannot stop to learn its size on the host, so it takes its space on the device: a counter of
@@ -113,7 +119,7 @@ class CachePool {
   DeviceArena arena_;
   long long limit_ = 0, bytes_ = 0, evicted_chunks_ = 0, evicted_bytes_ = 0;
   uint64_t clock_ = 0;
-  std::vector<std::pair<void*, size_t>> scratch_;
+  std::vector<std::pair<void*, size_t>> scratch_, pinned_;
   JitArena jit_;
   cudaEvent_t timing_[2] = {nullptr, nullptr};
   int find_or_add(uint64_t hash, std::vector<uint64_t>&& serial);

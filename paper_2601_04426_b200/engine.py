@@ -6,6 +6,7 @@ pointers through `binding`, and moves results to numpy.  It needs a CUDA device.
 from __future__ import annotations
 
 import os
+import time
 from concurrent.futures import ThreadPoolExecutor
 from typing import List, Optional, Sequence
 
@@ -20,7 +21,8 @@ class Session:
     """One tokenizer, its compiled grammars and one matcher per request of a workload."""
 
     def __init__(self, workload: inputs.Workload, share_pool: bool = True, device: str = "cuda:0", state_compression: bool = True,
-                 jit: bool = False, jit_precompute: int = 0, jit_arena_bytes: int = 0, compile_threads: int = 0):
+                 jit: bool = False, jit_precompute: int = 0, jit_arena_bytes: int = 0, compile_threads: int = 0,
+                 reserve_bytes: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         self.device = torch.device(device)
@@ -29,6 +31,8 @@ class Session:
         v = workload.vocab
         self.tokenizer = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
         self.pool = B.CachePool(self.tokenizer) if share_pool else None
+        if self.pool and reserve_bytes > 0:
+            self.pool.reserve(reserve_bytes)       # device memory for the cache taken before the (timed) compiles
         # xg_compile_grammar may be called from several threads: the host front ends run side by side, the
         # cache builds take turns on the pool.  compile_threads: 0 = one per core (at most 16), 1 = in this thread.
         def compile_one(g):
@@ -37,11 +41,15 @@ class Session:
                              jit=jit, jit_precompute=jit_precompute, jit_arena_bytes=jit_arena_bytes)
         n_threads = compile_threads if compile_threads > 0 else min(16, os.cpu_count() or 1)
         n_threads = max(1, min(n_threads, len(workload.grammars)))
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
         if n_threads == 1:
             self.grammars: List[B.Grammar] = [compile_one(g) for g in workload.grammars]
         else:
             with ThreadPoolExecutor(max_workers=n_threads) as ex:
                 self.grammars = list(ex.map(compile_one, workload.grammars))
+        torch.cuda.synchronize()
+        self.compile_wall_s = time.perf_counter() - t0       # the grammar compiles alone (tokenizer and matchers excluded)
         self.matchers = [B.Matcher(self.grammars[gi]) for gi in workload.request_grammar]
         self.batch = B.Batch(self.matchers)
         self.V, self.W, self.n = v.size, self.tokenizer.words, len(self.matchers)

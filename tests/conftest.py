@@ -24,3 +24,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _no_bounds_violation():
+    """With XG_DEBUG_BOUNDS=1 the tests run on the bounds-checking library; none of its checks may fail."""
+    yield
+    if os.environ.get("XG_DEBUG_BOUNDS") == "1":
+        from paper_2601_04426_b200 import binding
+        if binding._lib is not None and binding.lib().xg_debug_bounds_enabled():
+            binding.debug_bounds_check()
