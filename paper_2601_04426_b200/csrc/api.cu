@@ -174,6 +174,7 @@ struct xg_grammar {
   std::vector<int> chunk_refs;          // pool chunks this grammar keeps alive
   xg_grammar_stats_t stats{};
   bool count_visits = false;            // add up the bytes the classification walks consume (statistics only)
+  int max_check = 0;                    // longest check list of this grammar's entries (which fill kernel a batch gets)
   JitState jit;
   // buffers behind xg_grammar_get_cache_entry's view
   mutable std::vector<int32_t> view_list, view_unc;
@@ -679,6 +680,7 @@ static void jit_record(xg_grammar* g, const std::vector<int32_t>& reps, const En
     for (int q = j.member_begin[r]; q < j.member_begin[r + 1]; ++q) {
       const int s = j.members[q];
       g->entries[s] = entries[k]; g->entry_counts[s] = counts[k]; g->entry_chunk[s] = chunk;
+      g->max_check = std::max(g->max_check, (int)entries[k].n_unc);        // (its narrowed list is at most this long)
       const int c = j.canon_of[s];
       if (c >= 0 && !pr.have[c]) { pr.entries[c] = entries[k]; pr.counts[c] = counts[k]; pr.have[c] = 1; }
     }
@@ -1117,6 +1119,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     g->stats.total_accepted += c.x;
     g->stats.total_uncertain += c.y;
     g->stats.total_checked += e.n_chk;
+    g->max_check = std::max(g->max_check, (int)e.n_chk);
     g->stats.total_rejected += tok->vocab_size - c.x - c.y;
     g->stats.kind_count[e.kind]++;
     if (rep[s] == s) g->stats.cache_bytes += 4LL * ((e.kind == 2 ? tok->n_words : e.n_list) + 3LL * e.n_unc + (e.n_unc + 3) / 4);
@@ -1424,23 +1427,26 @@ static xg_status_t accept_and_fill(xg_matcher_t* const* matchers, int32_t batch,
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int per_request = sms * 1024 / batch;
     int blocks = kMaxClusterBlocks, threads = 256;
-    if (per_request < 2048) threads = 128;     // measured: fewer blocks or narrower blocks than this are slower even at batch 256
+    if (per_request < 2048) threads = 128;     // measured: narrower blocks than this are slower even at batch 256
+    // more requests than fit the SMs at eight blocks each (8 blocks of 128 threads per SM): clusters of four, so that
+    // the launch is still one wave (C5, batch 256: fill 74 -> 69 us)
+    if (batch * blocks > sms * 8 && (W + 3) / 4 <= kMergeMaxChunkWords) blocks = 4;
     const size_t smem = 2 * sizeof(uint32_t) * (size_t)((W + blocks - 1) / blocks);
     MatcherDev* const* dm = slot->dev_matchers;
+    // requests with hundreds of uncertain candidates are possible only where some entry has a long check list
+    bool heavy = false;
+    for (int i = 0; i < batch && !heavy; ++i) heavy = matchers[i]->grammar->max_check >= 1024;
     const dim3 grid(blocks, batch), block(threads);
     cudaStream_t cs = (cudaStream_t)stream;
-    if (token_ids_dev)
-      XG_CUDA(launch_step_kernel(fill_cluster_kernel<true, 0>, grid, block, smem, cs, blocks, dm, tok->dev, bitmask_dev, (long long)row_stride_words,
-                                 status_dev, token_ids_dev, accept_status_dev, restart_on_eos, (void*)nullptr, 0LL));
-    else if (!logits_dev)
-      XG_CUDA(launch_step_kernel(fill_cluster_kernel<false, 0>, grid, block, smem, cs, blocks, dm, tok->dev, bitmask_dev, (long long)row_stride_words,
-                                 status_dev, (const int32_t*)nullptr, (int32_t*)nullptr, 0, (void*)nullptr, 0LL));
-    else if (dtype == XG_BF16)
-      XG_CUDA(launch_step_kernel(fill_cluster_kernel<false, 8>, grid, block, smem, cs, blocks, dm, tok->dev, bitmask_dev, (long long)row_stride_words,
-                                 status_dev, (const int32_t*)nullptr, (int32_t*)nullptr, 0, logits_dev, (long long)logits_row_stride_elems));
-    else
-      XG_CUDA(launch_step_kernel(fill_cluster_kernel<false, 4>, grid, block, smem, cs, blocks, dm, tok->dev, bitmask_dev, (long long)row_stride_words,
-                                 status_dev, (const int32_t*)nullptr, (int32_t*)nullptr, 0, logits_dev, (long long)logits_row_stride_elems));
+    const long long stride_w = (long long)row_stride_words, stride_l = (long long)logits_row_stride_elems;
+#define XG_FILL(ACCEPT, ELEMS, HEAVY, TOK, AST, RST, LOGITS)                                                                              \
+    XG_CUDA(launch_step_kernel(fill_cluster_kernel<ACCEPT, ELEMS, HEAVY>, grid, block, smem, cs, blocks, dm, tok->dev, bitmask_dev, stride_w, \
+                               status_dev, (const int32_t*)(TOK), (int32_t*)(AST), (int)(RST), (void*)(LOGITS), stride_l))
+    if (token_ids_dev) { if (heavy) XG_FILL(true, 0, true, token_ids_dev, accept_status_dev, restart_on_eos, nullptr); else XG_FILL(true, 0, false, token_ids_dev, accept_status_dev, restart_on_eos, nullptr); }
+    else if (!logits_dev) { if (heavy) XG_FILL(false, 0, true, nullptr, nullptr, 0, nullptr); else XG_FILL(false, 0, false, nullptr, nullptr, 0, nullptr); }
+    else if (dtype == XG_BF16) { if (heavy) XG_FILL(false, 8, true, nullptr, nullptr, 0, logits_dev); else XG_FILL(false, 8, false, nullptr, nullptr, 0, logits_dev); }
+    else { if (heavy) XG_FILL(false, 4, true, nullptr, nullptr, 0, logits_dev); else XG_FILL(false, 4, false, nullptr, nullptr, 0, logits_dev); }
+#undef XG_FILL
     return XG_OK;
   }
   if (token_ids_dev) {

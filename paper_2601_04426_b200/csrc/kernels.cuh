@@ -180,7 +180,7 @@ __device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* c
 }
 
 // byte-class bitsets staged in shared memory when they fit (the hottest table of a walk)
-constexpr int kSharedClasses = 256;
+constexpr int kSharedClasses = 128;     // (the grammars of all workloads here have at most 124 classes)
 __device__ __forceinline__ const uint32_t* stage_class_bits(const GrammarDev& g, uint32_t* sh) {
   if (g.n_classes > kSharedClasses) return g.class_bits;
   for (int i = threadIdx.x; i < g.n_classes * 8; i += blockDim.x) sh[i] = g.class_bits[i];
@@ -1230,7 +1230,9 @@ apply_kernel(void* __restrict__ logits, int vocab_size, long long row_stride_ele
 constexpr int kMaxClusterBlocks = 8;      // the portable cluster size limit
 
 // launched with a cluster of gridDim.x blocks (2, 4 or 8) along x
-template <bool kAccept, int kApplyElems>
+// kHeavy: the launch may hold requests with hundreds of uncertain candidates (a grammar of the batch has an entry with
+// a long check list); only then does the kernel carry the second-byte sets and the walk queues described below.
+template <bool kAccept, int kApplyElems, bool kHeavy>
 __global__ void __launch_bounds__(256, 4)
 fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __restrict__ bitmask, long long row_stride,
                     int32_t* __restrict__ status_user, const int32_t* __restrict__ token_ids, int32_t* __restrict__ accept_status,
@@ -1253,6 +1255,24 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   __shared__ int16_t acc_lsb[kAccept ? kFastMaxBytes + 2 : 1];
   __shared__ int sh_fail;          // set in every block of the cluster when any of them fails
   __shared__ int sh_slow;          // set in every block of the cluster when a token was queued for the exact slow walk
+  // Second-byte sets.  What a token has left after its exit starts with byte b1, which the entry's continuation set
+  // must be able to scan; the set that scan leads to -- and so the bytes b2 it can scan in turn -- depends only
+  // on (entry, b1), not on the token.  For requests with many candidates every block works these sets out once,
+  // one thread per (entry, b1) pair: a token is then decided by two bit tests when it has at most two bytes left,
+  // and most of the others die on their second byte without a walk.
+  constexpr int kPairs = kHeavy ? 96 : 1, kPairsMinCandidates = 1024;
+  __shared__ __align__(16) uint32_t pair_second[kPairs][8];      // written as two 16-byte vectors per pair
+  __shared__ int pair_base[kHeavy ? kPlanCheckMax + 1 : 1];
+  __shared__ uint8_t pair_unknown[kPairs];      // the pair's walk did not fit the fast arrays: its tokens are walked
+  __shared__ int pair_n;           // pairs built (0: no second-byte sets for this request)
+  // Walks that survive both byte tests cluster in a few warps (tokens with a common prefix are neighbours in the
+  // candidate lists), and the lanes of a warp walk one after the other wherever their paths differ.  For requests with
+  // many candidates the surviving (token, exit) pairs therefore go through queues, one per block of the cluster,
+  // filled round robin so that every block gets an equal share of every run, and each block deals its queue out over
+  // its warps first and over the lanes of a warp last.
+  constexpr int kWalkQueue = kHeavy ? 192 : 1;
+  __shared__ uint2 walk_q[kWalkQueue];          // (token rank, entry | exit offset << 8)
+  __shared__ int walk_q_n;
 
   step_kernel_prologue();
   const int b = blockIdx.y;
@@ -1330,6 +1350,54 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
       if (rank == 0 && threadIdx.x == 0 && plan.n_missing > 0) report_missing(g, plan);
     }
     if (rank == 0 && threadIdx.x == 0) mw->slow_n = 0;
+    if (threadIdx.x == 0) { pair_n = 0; walk_q_n = 0; }
+    uint32_t w_st[kFastCap];                       // this thread's walk arrays
+    int32_t w_org[kFastCap];
+    int16_t w_lsb[kFastMaxBytes + 2];
+    if (kHeavy && total >= kPairsMinCandidates) {  // (uniform over the cluster)
+      __syncthreads();                             // the staged continuation sets are visible
+      if (threadIdx.x == 0) {
+        int run = 0;
+        for (int e = 0; e < n_ent; ++e) {
+          pair_base[e] = run;
+          for (int w = 0; w < 8; ++w) run += __popc(cont_first[e][w]);
+        }
+        pair_base[n_ent] = run;
+        pair_n = run <= kPairs ? run : 0;          // too many pairs for the table: no second-byte sets
+      }
+      __syncthreads();
+      for (int p = threadIdx.x; p < pair_n; p += blockDim.x) {
+        int e = 0;
+        while (p >= pair_base[e + 1]) ++e;
+        int skip = p - pair_base[e], b1 = 0;       // b1 = the (skip)-th byte of the entry's first-byte set
+        for (int w = 0; w < 8; ++w) {
+          uint32_t bits = cont_first[e][w];
+          const int c = __popc(bits);
+          if (skip >= c) { skip -= c; continue; }
+          while (skip--) bits &= bits - 1;
+          b1 = 32 * w + __ffs(bits) - 1;
+          break;
+        }
+        int flags = 0;
+        const uint8_t one_byte = (uint8_t)b1;
+        Chart c = hist;
+        c.i_st = cont_st[e]; c.i_org = cont_org[e]; c.i_cnt = cont_cnt[e]; c.i_idx = n + 1;
+        const int consumed = token_walk<int16_t>(g, class_bits, c, &one_byte, 1, false, w_st, w_org, kFastCap, w_lsb, &flags, nullptr);
+        uint4 fa = make_uint4(0, 0, 0, 0), fb = make_uint4(0, 0, 0, 0);
+        const bool unknown = (flags & kWalkOverflow) || consumed != 1;
+        pair_unknown[p] = unknown ? 1 : 0;
+        if (unknown) fa = fb = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);    // every token goes on to its walk
+        else
+          for (int q = 0; q < w_lsb[2]; ++q) {
+            const uint4* sf = reinterpret_cast<const uint4*>(g.state_first + (size_t)w_st[q] * 8);
+            const uint4 a = sf[0], d = sf[1];
+            fa.x |= a.x; fa.y |= a.y; fa.z |= a.z; fa.w |= a.w;
+            fb.x |= d.x; fb.y |= d.y; fb.z |= d.z; fb.w |= d.w;
+          }
+        uint4* out = reinterpret_cast<uint4*>(pair_second[p]);
+        out[0] = fa; out[1] = fb;
+      }
+    }
     cluster.sync();            // every slice is merged (and this block's staging, and the emptied slow queue, are visible)
     const int stride = n_blocks * blockDim.x;
     // a failure (rare) is recorded in every block's flag, so that each block reads its own at the end and no block has to
@@ -1344,13 +1412,10 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
       const int len = (int)(v.offset[trank + 1] - off);
       bool pass = false, overflow = len - at > kFastMaxBytes;
       if (!overflow) {
-        uint32_t st[kFastCap];
-        int32_t org[kFastCap];
-        int16_t lsb[kFastMaxBytes + 2];
         int flags = 0;
         Chart c = hist;
         if (at > 0) { c.i_st = cont_st[e]; c.i_org = cont_org[e]; c.i_cnt = cont_cnt[e]; c.i_idx = n + at; }
-        pass = token_walk<int16_t>(g, class_bits, c, v.bytes + off + at, len - at, false, st, org, kFastCap, lsb, &flags, nullptr) == len - at;
+        pass = token_walk<int16_t>(g, class_bits, c, v.bytes + off + at, len - at, false, w_st, w_org, kFastCap, w_lsb, &flags, nullptr) == len - at;
         overflow = (flags & kWalkOverflow) != 0;
       }
       if (overflow) walk_slowly(trank);
@@ -1372,6 +1437,39 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
         }
       }
     }
+    const bool queued = kHeavy && total >= kPairsMinCandidates;       // (uniform over the cluster)
+    // one candidate whose exit mask, token rank and (for the survivors of the first test) offsets are already here
+    auto check_candidate = [&](int j, int e, int trank, uint32_t left, uint32_t off, int len) {
+      bool pass = false;
+      while (left && !pass) {
+        const int at = __ffs(left) - 1;
+        left &= left - 1;
+        const uint32_t byte = v.bytes[off + at];
+        if (!((cont_first[e][byte >> 5] >> (byte & 31)) & 1u)) continue;
+        // a single byte left that the continuation set can scan: the set after it is not empty, nothing to walk
+        if (at + 1 == len) { pass = true; break; }
+        if (kHeavy && pair_n > 0) {
+          int p = pair_base[e];
+          for (uint32_t w = 0; w < (byte >> 5); ++w) p += __popc(cont_first[e][w]);
+          p += __popc(cont_first[e][byte >> 5] & ((1u << (byte & 31)) - 1u));
+          const uint32_t b2 = v.bytes[off + at + 1];
+          if (!((pair_second[p][b2 >> 5] >> (b2 & 31)) & 1u)) continue;          // dies on its second byte
+          if (at + 2 == len && !pair_unknown[p]) { pass = true; break; }
+        }
+        if (queued) {             // the walk goes to the queue of block (j mod blocks); a full queue: walk here after all
+          const int target = j % n_blocks;
+          const int slot = atomicAdd(cluster.map_shared_rank(&walk_q_n, target), 1);
+          if (slot < kWalkQueue) { *cluster.map_shared_rank(&walk_q[slot], target) = make_uint2((uint32_t)trank, (uint32_t)e | ((uint32_t)at << 8)); continue; }
+        }
+        pass = walk_one(trank, off, e, at);
+      }
+      if (pass) {
+        const int id = v.rank_to_id[trank];
+        const int word = id >> 5, owner = word / chunk;
+        if (XG_BOUND(word, v.n_words, kBoundRowWord) && XG_BOUND(owner, n_blocks, kBoundClusterBlock))
+          atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
+      }
+    };
     for (int j = rank * blockDim.x + threadIdx.x; j < total; j += stride) {
       // per candidate: its exit mask and the byte at its first exit, both streamed in list order;
       // the token's rank and bytes are only touched by the few that survive the bit test
@@ -1382,29 +1480,36 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
       uint32_t left = ent_exit[e][k];
       const int trank = (int)ent_rank[e][k];      // read together with the exit mask: one dependent load less for the survivors
       if (!XG_BOUND(trank, v.vocab_size, kBoundTokenRank)) continue;
-      bool pass = false;
-      int id = -1;
       if (left == 0) {                // no exit record (very long token, or its build-time walk overflowed): walk in full
         if ((int)(v.offset[trank + 1] - v.offset[trank]) > kFastMaxBytes) { walk_slowly(trank); continue; }
-        id = v.rank_to_id[trank];
-        pass = walk_one(trank, v.offset[trank], e, 0);
-      } else {
-        uint32_t byte = ent_byte[e][k];
-        if (!((cont_first[e][byte >> 5] >> (byte & 31)) & 1u)) left &= left - 1;
-        if (left == 0) continue;                        // the usual end of a candidate
-        const uint32_t off = v.offset[trank];
-        id = v.rank_to_id[trank];                       // requested before the walk, needed after it
-        while (left && !pass) {
-          const int at = __ffs(left) - 1;
-          left &= left - 1;
-          byte = v.bytes[off + at];
-          if ((cont_first[e][byte >> 5] >> (byte & 31)) & 1u) pass = walk_one(trank, off, e, at);
+        if (walk_one(trank, v.offset[trank], e, 0)) {
+          const int id = v.rank_to_id[trank];
+          const int word = id >> 5, owner = word / chunk;
+          if (XG_BOUND(word, v.n_words, kBoundRowWord) && XG_BOUND(owner, n_blocks, kBoundClusterBlock))
+            atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
         }
+        continue;
       }
-      if (pass) {
-        const int word = id >> 5, owner = word / chunk;
-        if (XG_BOUND(word, v.n_words, kBoundRowWord) && XG_BOUND(owner, n_blocks, kBoundClusterBlock))
-          atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
+      const uint32_t byte = ent_byte[e][k];
+      if (!((cont_first[e][byte >> 5] >> (byte & 31)) & 1u)) left &= left - 1;
+      if (left == 0) continue;                        // the usual end of a candidate
+      const uint32_t off = v.offset[trank];
+      check_candidate(j, e, trank, left, off, (int)(v.offset[trank + 1] - off));
+    }
+    if (queued) {
+      cluster.sync();          // every queue is complete
+      const int n_q = min(walk_q_n, kWalkQueue), n_warps = (int)(blockDim.x >> 5);
+      // entry i goes to warp i mod warps, lane i / warps: a short queue puts one walk into every warp before a second
+      const int mine = (int)(threadIdx.x >> 5) + (int)(threadIdx.x & 31) * n_warps;
+      for (int i = mine; i < n_q; i += (int)blockDim.x) {
+        const uint2 entry = walk_q[i];
+        const int trank = (int)entry.x;
+        if (walk_one(trank, v.offset[trank], (int)(entry.y & 0xFFu), (int)(entry.y >> 8))) {
+          const int id = v.rank_to_id[trank];
+          const int word = id >> 5, owner = word / chunk;
+          if (XG_BOUND(word, v.n_words, kBoundRowWord) && XG_BOUND(owner, n_blocks, kBoundClusterBlock))
+            atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
+        }
       }
     }
     __threadfence();           // queued tokens are visible to the block that walks them
