@@ -273,7 +273,7 @@ xg_status_t xg_matcher_is_terminated(const xg_matcher_t* m, void* stream, int32_
 /* What the next xg_fill_next_token_bitmask has to stream for this matcher (for measurements): the
  * bytes of the cache entries it merges (bitsets in full, lists in full -- a block reads only its
  * slice of a list, but all blocks together read all of it), the uncertain candidates it tests
- * (5 bytes each: exit mask and first-exit byte) and the row it writes.  List lengths and check
+ * (12 bytes each: token rank, exit mask, and what is left at the first exit) and the row it writes.  List lengths and check
  * counts are the compile-time ones (entries that arrived just in time count with their whole
  * uncertain list).  Synchronises `stream`. */
 typedef struct {

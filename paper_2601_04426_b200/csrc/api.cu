@@ -557,7 +557,7 @@ static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>&
   XG_CUDA(cudaStreamSynchronize(stream));
   std::vector<long long> offsets(n);
   long long total = 0;
-  for (int k = 0; k < n; ++k) { offsets[k] = total; total += 2LL * counts[k] + (counts[k] + 3) / 4; }
+  for (int k = 0; k < n; ++k) { offsets[k] = total; total += 3LL * counts[k]; }
   g->lookahead_arena = pool.allocate_plain((size_t)std::max<long long>(total, 1) * 4);
   if (!g->lookahead_arena) return set_error(XG_ERR_OOM, "check list allocation failed");
   std::memcpy(h_offsets, offsets.data(), (size_t)n * 8);
@@ -569,14 +569,14 @@ static xg_status_t narrow_check_lists(xg_grammar* g, const std::vector<int32_t>&
     EntryDev& e = g->entries[states[k]];
     e.chk_rank = arena + offsets[k];
     e.chk_exit = e.chk_rank + counts[k];
-    e.chk_byte = reinterpret_cast<const uint8_t*>(e.chk_exit + counts[k]);
+    e.chk_info = e.chk_exit + counts[k];
     e.n_chk = counts[k];
   }
   for (int s : scannable) {
     if (rep[s] == s) continue;
     const EntryDev& r = g->entries[rep[s]];
     EntryDev& e = g->entries[s];
-    e.chk_rank = r.chk_rank; e.chk_exit = r.chk_exit; e.chk_byte = r.chk_byte; e.n_chk = r.n_chk;
+    e.chk_rank = r.chk_rank; e.chk_exit = r.chk_exit; e.chk_info = r.chk_info; e.n_chk = r.n_chk;
   }
   *narrowed = true;
   return XG_OK;
@@ -1122,7 +1122,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     g->max_check = std::max(g->max_check, (int)e.n_chk);
     g->stats.total_rejected += tok->vocab_size - c.x - c.y;
     g->stats.kind_count[e.kind]++;
-    if (rep[s] == s) g->stats.cache_bytes += 4LL * ((e.kind == 2 ? tok->n_words : e.n_list) + 3LL * e.n_unc + (e.n_unc + 3) / 4);
+    if (rep[s] == s) g->stats.cache_bytes += 4LL * ((e.kind == 2 ? tok->n_words : e.n_list) + 4LL * e.n_unc);
   }
   *out = g.release();
   return XG_OK;
@@ -1334,7 +1334,7 @@ xg_status_t xg_matcher_next_fill_work(const xg_matcher_t* m, void* stream, xg_fi
       else if (e.kind == XG_STORE_REJECT_LIST) w.merge_bytes += 4LL * e.n_list + 4LL * e.n_unc;
     }
     w.check_tokens = plan->n_check ? plan->check_cum[plan->n_check] : 0;
-    w.check_bytes = 5 * w.check_tokens;
+    w.check_bytes = 12 * w.check_tokens;
   }
   *out = w;
   return XG_OK;

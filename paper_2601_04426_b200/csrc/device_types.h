@@ -46,13 +46,14 @@ struct EntryDev {
   const uint32_t* unc_id;    // [n_unc] ascending token ids
   const uint32_t* unc_rank;  // [n_unc] ascending ranks
   const uint32_t* unc_exit;  // [n_unc] parallel to unc_rank: bit j = the token leaves the entry's rule after j bytes
-  const uint8_t* unc_byte;   // [n_unc] parallel to unc_rank: the token's byte at its first exit (what the context must scan)
+  const uint32_t* unc_info;  // [n_unc] parallel to unc_rank: what the token has left at its first exit -- its byte there (what the
+                             // context must scan) | the next byte << 8 | the number of bytes left (at most 255) << 16
   // The list the run-time check walks.  In the pool it is the uncertain list itself; a grammar
   // narrows it with its own lookahead (Section 3.3): exits whose next byte can never follow the
   // rule anywhere in that grammar are dropped, and tokens left without an exit with them.
   const uint32_t* chk_rank;
   const uint32_t* chk_exit;
-  const uint8_t* chk_byte;
+  const uint32_t* chk_info;
   int32_t n_chk;
   int32_t pad2;
   int32_t kind;              // xg_store_kind_t; kEntryNotBuilt while a just-in-time grammar has not built it yet

@@ -357,7 +357,7 @@ plan_kernel(const int2* __restrict__ counts, int n_pos, int vocab_size, int n_wo
     if (nr < n_list) { kind = 1; n_list = nr; }
     if (n_words < n_list) { kind = 2; n_list = 0; }
     plan[p].kind = kind; plan[p].n_list = n_list; plan[p].n_acc = na; plan[p].n_unc = nu;
-    local += (kind == 2 ? n_words : n_list) + 3LL * nu + (nu + 3) / 4;
+    local += (kind == 2 ? n_words : n_list) + 4LL * nu;
   }
   sums[threadIdx.x] = local;
   __syncthreads();
@@ -370,7 +370,7 @@ plan_kernel(const int2* __restrict__ counts, int n_pos, int vocab_size, int n_wo
   long long run = sums[threadIdx.x] - local;
   for (int p = lo; p < hi; ++p) {
     plan[p].offset_words = run;
-    run += (plan[p].kind == 2 ? n_words : plan[p].n_list) + 3LL * plan[p].n_unc + (plan[p].n_unc + 3) / 4;
+    run += (plan[p].kind == 2 ? n_words : plan[p].n_list) + 4LL * plan[p].n_unc;
   }
   if (threadIdx.x == blockDim.x - 1) *total_words = sums[threadIdx.x];
 }
@@ -426,11 +426,19 @@ pack_kernel(const uint32_t* __restrict__ acc_id, const uint32_t* __restrict__ un
   if (threadIdx.x == 0) {
     EntryDev e;
     e.data = data; e.unc_id = out_uid; e.unc_rank = out_urank; e.unc_exit = out_urank + pl.n_unc;
-    e.unc_byte = reinterpret_cast<const uint8_t*>(out_urank + 2 * (size_t)pl.n_unc);
+    e.unc_info = out_urank + 2 * (size_t)pl.n_unc;
     e.kind = pl.kind; e.n_list = pl.n_list; e.n_unc = pl.n_unc; e.n_acc = pl.n_acc;
-    e.chk_rank = e.unc_rank; e.chk_exit = e.unc_exit; e.chk_byte = e.unc_byte; e.n_chk = pl.n_unc; e.pad2 = 0;
+    e.chk_rank = e.unc_rank; e.chk_exit = e.unc_exit; e.chk_info = e.unc_info; e.n_chk = pl.n_unc; e.pad2 = 0;
     entries[p] = e;
   }
+}
+
+// what a token (bytes at `off`, `len` of them) has left at the first exit of `exits`: see EntryDev::unc_info
+__device__ __forceinline__ uint32_t first_exit_info(const VocabDev& v, uint32_t off, int len, uint32_t exits) {
+  if (!exits) return 0;
+  const int at = __ffs(exits) - 1;
+  const uint32_t b1 = v.bytes[off + at], b2 = at + 1 < len ? v.bytes[off + at + 1] : 0u;
+  return b1 | (b2 << 8) | ((uint32_t)min(len - at, 255) << 16);
 }
 
 // For every uncertain token of every packed entry: the byte offsets at which the token leaves
@@ -448,7 +456,7 @@ exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, con
   const uint32_t* class_bits = stage_class_bits(g, sh_class);
   __syncthreads();
   uint32_t* out = const_cast<uint32_t*>(e.unc_exit);
-  uint8_t* out_byte = const_cast<uint8_t*>(e.unc_byte);
+  uint32_t* out_info = const_cast<uint32_t*>(e.unc_info);
   for (int k = threadIdx.x; k < e.n_unc; k += blockDim.x) {
     const int rank = (int)e.unc_rank[k];
     const uint32_t off = v.offset[rank];
@@ -466,7 +474,7 @@ exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, con
       if (flags & kWalkOverflow) mask = 0;
     }
     out[k] = mask;
-    out_byte[k] = mask ? v.bytes[off + __ffs(mask) - 1] : 0;
+    out_info[k] = first_exit_info(v, off, len, mask);
   }
 }
 
@@ -513,7 +521,7 @@ lookahead_compact_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ s
   const int n_out = counts[blockIdx.x];
   uint32_t* out_rank = arena + offsets[blockIdx.x];
   uint32_t* out_exit = out_rank + n_out;
-  uint8_t* out_byte = reinterpret_cast<uint8_t*>(out_exit + n_out);
+  uint32_t* out_info = out_exit + n_out;
   const int per = (e.n_unc + blockDim.x - 1) / blockDim.x;
   const int lo = min(e.n_unc, (int)threadIdx.x * per), hi = min(e.n_unc, lo + per);
   int mine = 0;
@@ -537,7 +545,7 @@ lookahead_compact_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ s
     if (exits != 0 && keep == 0) continue;
     out_rank[at] = (uint32_t)rank;
     out_exit[at] = keep;
-    out_byte[at] = keep ? v.bytes[v.offset[rank] + __ffs(keep) - 1] : 0;
+    out_info[at] = first_exit_info(v, v.offset[rank], (int)(v.offset[rank + 1] - v.offset[rank]), keep);
     ++at;
   }
 }
@@ -586,11 +594,11 @@ __global__ void jit_reserve_lists_kernel(const int32_t* __restrict__ counts, int
   *go_lists = 0;
   if (!*go) return;
   unsigned long long need = 1;
-  for (int k = 0; k < n; ++k) need += 2ull * counts[k] + (counts[k] + 3) / 4;
+  for (int k = 0; k < n; ++k) need += 3ull * counts[k];
   const unsigned long long base = atomicAdd(arena_used, need);
   if (base + need > (unsigned long long)arena_cap) return;
   long long run = (long long)base;
-  for (int k = 0; k < n; ++k) { offsets[k] = run; run += 2LL * counts[k] + (counts[k] + 3) / 4; }
+  for (int k = 0; k < n; ++k) { offsets[k] = run; run += 3LL * counts[k]; }
   *go_lists = 1;
 }
 
@@ -607,7 +615,7 @@ jit_patch_lists_kernel(EntryDev* __restrict__ entries, const int32_t* __restrict
       EntryDev& e = entries[s];
       e.chk_rank = arena + offsets[k];
       e.chk_exit = e.chk_rank + counts[k];
-      e.chk_byte = reinterpret_cast<const uint8_t*>(e.chk_exit + counts[k]);
+      e.chk_info = e.chk_exit + counts[k];
       e.n_chk = counts[k];
       return;
     }
@@ -1242,7 +1250,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   extern __shared__ uint32_t dyn_smem[];          // this block's row slice and a scratch slice: 2 x ceil(W / blocks) words
   __shared__ const uint32_t* ent_rank[kPlanCheckMax];
   __shared__ const uint32_t* ent_exit[kPlanCheckMax];
-  __shared__ const uint8_t* ent_byte[kPlanCheckMax];
+  __shared__ const uint32_t* ent_info[kPlanCheckMax];
   __shared__ int ent_cum[kPlanCheckMax + 1];
   __shared__ uint32_t cont_st[kPlanCheckMax][kContCap];
   __shared__ int32_t cont_org[kPlanCheckMax][kContCap];
@@ -1336,7 +1344,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
     const uint32_t* class_bits = stage_class_bits(g, sh_class);
     for (int i = threadIdx.x; i < n_ent; i += blockDim.x) {
       const EntryDev& e = g.entries[plan.check_state[i]];
-      ent_rank[i] = e.chk_rank; ent_exit[i] = e.chk_exit; ent_byte[i] = e.chk_byte;
+      ent_rank[i] = e.chk_rank; ent_exit[i] = e.chk_exit; ent_info[i] = e.chk_info;
       cont_cnt[i] = plan.cont_cnt[i];
     }
     for (int i = threadIdx.x; i <= n_ent; i += blockDim.x) ent_cum[i] = plan.check_cum[i];
@@ -1490,8 +1498,36 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
         }
         continue;
       }
-      const uint32_t byte = ent_byte[e][k];
-      if (!((cont_first[e][byte >> 5] >> (byte & 31)) & 1u)) left &= left - 1;
+      // The first exit (for most tokens the only one) is decided from the list alone: its byte against the bytes the
+      // continuation set can scan, the next byte against the second-byte set of that pair, and with at most two bytes
+      // left the token is allowed without a walk.  Only what is still open after that touches the vocabulary tables.
+      const uint32_t info = ent_info[e][k];
+      const uint32_t b1 = info & 0xFFu, b2 = (info >> 8) & 0xFFu, rem = info >> 16;
+      const int at1 = __ffs(left) - 1;
+      int first = 0;                                  // the first exit: 0 dead, 1 allowed, 2 has to be walked
+      if ((cont_first[e][b1 >> 5] >> (b1 & 31)) & 1u) {
+        first = rem == 1 ? 1 : 2;
+        if (kHeavy && rem > 1 && pair_n > 0) {
+          int p = pair_base[e];
+          for (uint32_t w = 0; w < (b1 >> 5); ++w) p += __popc(cont_first[e][w]);
+          p += __popc(cont_first[e][b1 >> 5] & ((1u << (b1 & 31)) - 1u));
+          if (!((pair_second[p][b2 >> 5] >> (b2 & 31)) & 1u)) first = 0;              // dies on its second byte
+          else if (rem == 2 && !pair_unknown[p]) first = 1;
+        }
+      }
+      if (first == 1) {
+        const int id = v.rank_to_id[trank];
+        const int word = id >> 5, owner = word / chunk;
+        if (XG_BOUND(word, v.n_words, kBoundRowWord) && XG_BOUND(owner, n_blocks, kBoundClusterBlock))
+          atomicOr(cluster.map_shared_rank(&row[word - owner * chunk], owner), 1u << (id & 31));
+        continue;
+      }
+      if (first == 2 && queued) {                     // its walk goes to the queue of block (j mod blocks)
+        const int target = j % n_blocks;
+        const int slot = atomicAdd(cluster.map_shared_rank(&walk_q_n, target), 1);
+        if (slot < kWalkQueue) { *cluster.map_shared_rank(&walk_q[slot], target) = make_uint2((uint32_t)trank, (uint32_t)e | ((uint32_t)at1 << 8)); first = 0; }
+      }
+      if (first == 0) left &= left - 1;               // the first exit is settled (dead, or queued); any others go the general way
       if (left == 0) continue;                        // the usual end of a candidate
       const uint32_t off = v.offset[trank];
       check_candidate(j, e, trank, left, off, (int)(v.offset[trank + 1] - off));

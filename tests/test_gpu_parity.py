@@ -639,7 +639,7 @@ def test_next_fill_work_counts_the_plan():
         fw = s.matchers[0].next_fill_work(s.stream())
         assert fw["row_bytes"] == 4 * s.W and fw["n_missing"] == 0
         assert fw["n_merge"] >= 1 and fw["merge_bytes"] > 0
-        assert fw["check_bytes"] == 5 * fw["check_tokens"] and fw["n_check"] <= fw["n_merge"] * 2 + 2
+        assert fw["check_bytes"] == 12 * fw["check_tokens"] and fw["n_check"] <= fw["n_merge"] * 2 + 2
         s.fill()
         s.accept([w.trajectories[b][step] for b in range(s.n)])
         for b in range(s.n):
