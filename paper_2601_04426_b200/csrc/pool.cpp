@@ -267,15 +267,33 @@ RuleShape shape_of(const FlatGrammar& g, int r, int first, int n) {
   return sh;
 }
 
-// Phase 1 of Algorithm 1: sort the out-edges (ranges by (min, max), references by the hash of
-// the referenced rule), breadth-first search from the start state, canonical ids in discovery
-// order.  Returns canonical index -> state offset.
-std::vector<int> canonical_states(RuleShape& sh, const std::vector<uint64_t>& ref_hash) {
+// A key of a rule's automaton that does not depend on any numbering (of its states, of its edges or of the rules
+// it refers to): sizes and a commutative sum over its byte ranges.  It orders references whose hashes are still
+// equal -- the members of a cycle all carry the placeholder while the cycle is being hashed -- so that the same
+// structure gets the same canonical order in every grammar, whatever indices its rules have there.
+uint64_t shape_key(const RuleShape& sh) {
+  uint64_t ranges = 0, refs = 0, finals = 0;
+  for (int k = 0; k < sh.n; ++k) {
+    finals += sh.fin[k] ? 1 : 0;
+    for (const OutEdge& e : sh.out[k]) {
+      if (e.is_ref) ++refs;
+      else ranges += hash_fold(kRangeTag, ((uint64_t)e.lo << 8) | (uint64_t)e.hi);
+    }
+  }
+  return hash_fold(hash_fold(hash_fold(hash_fold(0, (uint64_t)sh.n), finals), refs), ranges);
+}
+
+// The canonical order of a rule's states (Section 3.3: two automata of the same structure must be numbered alike
+// before they can be hashed): out-edges sorted -- byte ranges by their bounds, references by the hash of the rule
+// they name, then by that rule's shape key --, then a breadth-first search from the start state; a state's
+// canonical id is its place in the order of discovery.  Returns canonical index -> state offset.
+std::vector<int> canonical_states(RuleShape& sh, const std::vector<uint64_t>& ref_hash, const std::vector<uint64_t>& ref_key) {
   for (auto& es : sh.out)
     std::stable_sort(es.begin(), es.end(), [&](const OutEdge& a, const OutEdge& b) {
       if (a.is_ref != b.is_ref) return !a.is_ref;
       if (!a.is_ref) return a.lo != b.lo ? a.lo < b.lo : a.hi < b.hi;
       if (ref_hash[a.rule] != ref_hash[b.rule]) return ref_hash[a.rule] < ref_hash[b.rule];
+      if (ref_key[a.rule] != ref_key[b.rule]) return ref_key[a.rule] < ref_key[b.rule];
       return a.rule < b.rule;
     });
   std::vector<int> order{sh.start}, id(sh.n, -1);
@@ -285,18 +303,25 @@ std::vector<int> canonical_states(RuleShape& sh, const std::vector<uint64_t>& re
   return order;
 }
 
-// Phase 2 of Algorithm 1
+// The hash of a rule: its automaton written out in canonical order as a flat sequence of words -- per state a
+// marker with the accepting flag, per edge its kind, its label (a byte range, or the hash of the referenced rule) and
+// the canonical id of its target -- folded in one pass.  (The pool's exact identity check serialises the same way,
+// with pool ids in place of hashes.)
 uint64_t hash_rule(const RuleShape& sh, const std::vector<int>& order, const std::vector<uint64_t>& ref_hash) {
   std::vector<int> id(sh.n, -1);
   for (size_t k = 0; k < order.size(); ++k) id[order[k]] = (int)k;
-  uint64_t h = 0;
+  std::vector<uint64_t> words;
   for (int s : order) {
-    h = hash_fold(hash_fold(h, kNodeTag), sh.fin[s] ? 1 : 0);
+    words.push_back(kNodeTag);
+    words.push_back(sh.fin[s] ? 1 : 0);
     for (const OutEdge& e : sh.out[s]) {
-      if (!e.is_ref) h = hash_fold(hash_fold(hash_fold(hash_fold(h, kRangeTag), (uint64_t)e.lo), (uint64_t)e.hi), (uint64_t)id[e.target]);
-      else h = hash_fold(hash_fold(hash_fold(h, kRefTag), ref_hash[e.rule]), (uint64_t)id[e.target]);
+      words.push_back(e.is_ref ? kRefTag : kRangeTag);
+      words.push_back(e.is_ref ? ref_hash[e.rule] : (((uint64_t)e.lo << 8) | (uint64_t)e.hi));
+      words.push_back((uint64_t)id[e.target]);
     }
   }
+  uint64_t h = 0;
+  for (uint64_t w : words) h = hash_fold(h, w);
   return h;
 }
 
@@ -347,10 +372,12 @@ Analysis analyse(const FlatGrammar& g) {
   for (int r = 0; r < R; ++r) if (index[r] < 0) dfs(r);
 
   std::vector<uint64_t> ref_hash(R, kPlaceholder);     // unresolved references hash as the placeholder
+  std::vector<uint64_t> ref_key(R);
+  for (int r = 0; r < R; ++r) ref_key[r] = shape_key(a.shapes[r]);
   for (auto& members : a.comps) {
     if (!a.cyclic(members)) {
       const int r = members[0];
-      out.canon[r] = canonical_states(a.shapes[r], ref_hash);
+      out.canon[r] = canonical_states(a.shapes[r], ref_hash, ref_key);
       out.hash[r] = hash_rule(a.shapes[r], out.canon[r], ref_hash);
       ref_hash[r] = out.hash[r];
       continue;
@@ -361,7 +388,7 @@ Analysis analyse(const FlatGrammar& g) {
     // in breadth-first order of the reference edges.
     std::vector<uint64_t> local(R, 0);
     for (int r : members) {
-      out.canon[r] = canonical_states(a.shapes[r], ref_hash);
+      out.canon[r] = canonical_states(a.shapes[r], ref_hash, ref_key);
       local[r] = hash_rule(a.shapes[r], out.canon[r], ref_hash);
     }
     for (int r : members) {
@@ -379,7 +406,7 @@ Analysis analyse(const FlatGrammar& g) {
     }
     for (int r : members) ref_hash[r] = out.hash[r];
     // the hashes of in-cycle references changed the sort keys: fix the canonical orders again
-    for (int r : members) out.canon[r] = canonical_states(a.shapes[r], ref_hash);
+    for (int r : members) out.canon[r] = canonical_states(a.shapes[r], ref_hash, ref_key);
   }
   return a;
 }

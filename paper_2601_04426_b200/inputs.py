@@ -539,17 +539,6 @@ def make_function_tags(rng: Rng, n_tags: int, tag_len: int = 20) -> List[dict]:
     return tools
 
 
-def function_tags_ebnf(tools: List[dict], stop_strs: Sequence[str] = ()) -> Tuple[str, List[str]]:
-    """Grammar text: one tag per tool, `<function=NAME>` -> arguments object then `</function>`.
-    The argument grammars are given as one JSON-schema-shaped EBNF rule each by the caller's own
-    lowering; here only the dispatching skeleton is spelled, with rule names args_<i>."""
-    pairs = ", ".join('("<function=%s>", call_%d)' % (t["name"], i) for i, t in enumerate(tools))
-    stops = ", ".join(json.dumps(s) for s in stop_strs)
-    head = "root ::= TagDispatch(%s, stop_strs=(%s))\n" % (pairs, stops)
-    calls = "".join('call_%d ::= args_%d "</function>"\n' % (i, i) for i in range(len(tools)))
-    return head + calls, ["args_%d" % i for i in range(len(tools))]
-
-
 def sample_function_text(rng: Rng, tools: List[dict], n_calls: int, n_words: int) -> str:
     def free(k: int) -> str:
         return " ".join(_word(rng, 2, 8) for _ in range(k)) + rng.choice([" ", ". ", "\n"])
