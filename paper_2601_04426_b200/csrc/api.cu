@@ -110,6 +110,7 @@ struct xg_tokenizer {
   VocabDev dev{};
   std::vector<void*> allocations;
   std::vector<int32_t> rank_to_id, id_to_rank;
+  std::vector<uint32_t> first_rank;       // [257] host copy of VocabDev::first_rank
   int32_t vocab_size = 0, n_words = 0;
   int64_t first_byte_count[256] = {};     // tokens (other than EOS / special / empty) by first byte
   mutable std::mutex mu;
@@ -260,13 +261,12 @@ xg_status_t xg_tokenizer_create(const uint8_t* bytes, const int64_t* offsets, in
   if (err == cudaSuccess) t->dev.rank_to_id = keep(device_copy(t->rank_to_id, &err));
   if (err == cudaSuccess) t->dev.id_to_rank = keep(device_copy(t->id_to_rank, &err));
   if (err == cudaSuccess) t->dev.never = keep(device_copy(never_rank, &err));
-  std::vector<uint16_t> block_first((vocab_size + 255) / 256);
-  for (size_t vb = 0; vb < block_first.size(); ++vb) {          // empty tokens sort first: they count as byte 0
-    const int r0 = (int)vb * 256, r1 = std::min(vocab_size, r0 + 256) - 1;
-    const unsigned lo = off[r0 + 1] > off[r0] ? arena[off[r0]] : 0u, hi = off[r1 + 1] > off[r1] ? arena[off[r1]] : 0u;
-    block_first[vb] = (uint16_t)(lo | (hi << 8));
-  }
-  if (err == cudaSuccess) t->dev.block_first = keep(device_copy(block_first, &err));
+  // in trie order the tokens that start with byte b are one run of ranks
+  t->first_rank.assign(257, (uint32_t)vocab_size);
+  for (int r = vocab_size - 1; r >= 0; --r)
+    if (off[r + 1] > off[r]) t->first_rank[arena[off[r]]] = (uint32_t)r;
+  for (int b2 = 255; b2 >= 0; --b2) t->first_rank[b2] = std::min(t->first_rank[b2], t->first_rank[b2 + 1]);
+  if (err == cudaSuccess) t->dev.first_rank = keep(device_copy(t->first_rank, &err));
   if (err != cudaSuccess) {
     for (void* p : t->allocations) cudaFree(p);
     return set_error(XG_ERR_CUDA, std::string("vocabulary upload: ") + cudaGetErrorString(err));
@@ -429,6 +429,24 @@ static xg_status_t upload_grammar(xg_grammar* g, cudaStream_t stream) {
   return XG_OK;
 }
 
+// The classification's work list for positions states[0 .. n): per position one block for every kClassifyChunk of
+// the tokens whose first byte one of the state's own edges can take (see classify_kernel).
+static void classify_work_list(const xg_grammar* g, const int32_t* states, int n, std::vector<int2>* work) {
+  const FlatGrammar& f = g->flat;
+  const std::vector<uint32_t>& first_rank = g->tok->first_rank;
+  work->clear();
+  for (int k = 0; k < n; ++k) {
+    const int s = states[k];
+    uint32_t own[8] = {};
+    for (int e = f.cedge_begin[s]; e < f.cedge_begin[s + 1]; ++e)
+      for (int w = 0; w < 8; ++w) own[w] |= f.class_bits[(size_t)f.cedge_class[e] * 8 + w];
+    long long total = 0;
+    for (int w = 0; w < 8; ++w)
+      for (uint32_t bits = own[w]; bits; bits &= bits - 1) { const int b = 32 * w + __builtin_ctz(bits); total += first_rank[b + 1] - first_rank[b]; }
+    for (long long c = 0; c * kClassifyChunk < total; ++c) work->push_back(make_int2(k, (int)c));
+  }
+}
+
 // classify + pack the given states (device work of the compile stage); fills entries / counts
 static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& states, cudaStream_t stream) {
   if (states.empty()) return XG_OK;
@@ -464,20 +482,29 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
     XG_CUDA_C(cudaMemsetAsync(unc, 0, row_bytes * n, stream));
     XG_CUDA_C(cudaMemsetAsync(unr, 0, row_bytes * n, stream));
     XG_CUDA_C(cudaMemsetAsync(d_over_count, 0, 2 * sizeof(int), stream));
-    dim3 grid(((V + 255) / 256 + kClassifySpan - 1) / kClassifySpan, n);
+    std::vector<int2> work;
+    classify_work_list(g, states.data() + begin, n, &work);
+    const int grid = (int)work.size();
+    int2* h_work = (int2*)pool.pinned(5, std::max<size_t>(work.size(), 1) * sizeof(int2));
+    int2* d_work = (int2*)pool.scratch(16, std::max<size_t>(work.size(), 1) * sizeof(int2));
+    if (!h_work || !d_work) return set_error(XG_ERR_OOM, "cache build scratch allocation failed");
+    if (grid > 0) {
+      std::memcpy(h_work, work.data(), work.size() * sizeof(int2));
+      XG_CUDA_C(cudaMemcpyAsync(d_work, h_work, work.size() * sizeof(int2), cudaMemcpyHostToDevice, stream));
+    }
     cudaEvent_t* ev = pool.timing_events();            // device time of the classification itself, for the statistics
     if (ev) cudaEventRecord(ev[0], stream);
     if (g->count_visits) {
       unsigned long long* d_visits = (unsigned long long*)pool.scratch(8, sizeof(unsigned long long));
       if (!d_visits) return set_error(XG_ERR_OOM, "cache build scratch allocation failed");
       XG_CUDA_C(cudaMemsetAsync(d_visits, 0, sizeof(unsigned long long), stream));
-      classify_kernel<true><<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, acc, unc, unr, d_over, d_over_count, over_cap, d_visits);
+      if (grid > 0) classify_kernel<true><<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, d_work, acc, unc, unr, d_over, d_over_count, over_cap, d_visits);
       unsigned long long visits = 0;
       XG_CUDA_C(cudaMemcpyAsync(&visits, d_visits, sizeof visits, cudaMemcpyDeviceToHost, stream));
       XG_CUDA_C(cudaStreamSynchronize(stream));
       g->stats.node_visits += (int64_t)visits;
     } else
-    classify_kernel<false><<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, acc, unc, unr, d_over, d_over_count, over_cap, nullptr);
+    if (grid > 0) classify_kernel<false><<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, d_work, acc, unc, unr, d_over, d_over_count, over_cap, nullptr);
     XG_CUDA_C(cudaGetLastError());
     if (ev) cudaEventRecord(ev[1], stream);
     // count and plan are enqueued behind the classification at once; walks that left the fast path are rare, and when
@@ -755,7 +782,15 @@ static xg_status_t jit_enqueue_build(JitPool* jp, xg_grammar* g, const std::vect
   XG_CUDA(cudaMemsetAsync(unc, 0, row_bytes * n, stream));
   XG_CUDA(cudaMemsetAsync(unr, 0, row_bytes * n, stream));
   XG_CUDA(cudaMemsetAsync(sc.over_count, 0, 2 * sizeof(int), stream));
-  classify_kernel<false><<<dim3(((V + 255) / 256 + kClassifySpan - 1) / kClassifySpan, n), 256, 0, stream>>>(g->host_view, v, sc.pos, acc, unc, unr, sc.over, sc.over_count, 64, nullptr);
+  std::vector<int2> work;
+  classify_work_list(g, reps.data(), n, &work);
+  if (!work.empty()) {
+    // (a pageable source: the runtime stages it before the call returns; a few hundred bytes)
+    int2* d_work = (int2*)pool.scratch(33, work.size() * sizeof(int2));
+    if (!d_work) return set_error(XG_ERR_OOM, "just-in-time scratch allocation failed");
+    XG_CUDA(cudaMemcpyAsync(d_work, work.data(), work.size() * sizeof(int2), cudaMemcpyHostToDevice, stream));
+    classify_kernel<false><<<(int)work.size(), 256, 0, stream>>>(g->host_view, v, sc.pos, d_work, acc, unc, unr, sc.over, sc.over_count, 64, nullptr);
+  }
   count_kernel<<<n, 256, 0, stream>>>(acc, unc, W, sc.counts);
   plan_kernel<<<1, 1024, 0, stream>>>(sc.counts, n, V, W, sc.plan, sc.total);
   jit_reserve_kernel<<<1, 32, 0, stream>>>(sc.plan, n, sc.total, arena->d_used, arena->cap_words, sc.over_count, sc.result);

@@ -33,9 +33,10 @@ struct VocabDev {
   const int32_t* rank_to_id; // [V]
   const int32_t* id_to_rank; // [V]
   const uint8_t* never;      // [V] by rank: 1 = EOS, special or zero-length (never classified)
-  const uint16_t* block_first; // [ceil(V / 256)]: first byte of the first token of a block of 256 ranks | first byte of its last << 8
   uint32_t n_bytes;            // size of the arena (for the bounds-checking build)
   uint32_t pad;
+  const uint32_t* first_rank;  // [257]: the tokens whose first byte is b are the ranks [first_rank[b], first_rank[b + 1])
+                               // (zero-length tokens sort in front of first_rank[0])
 };
 
 // One adaptive cache entry (Section 3.4): the accepted/rejected split in its smallest form plus

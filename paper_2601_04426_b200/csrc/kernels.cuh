@@ -193,23 +193,27 @@ __device__ __forceinline__ const uint32_t* stage_class_bits(const GrammarDev& g,
 // Accepted and uncertain bits are scattered into id-ordered rows; the uncertain bits are also
 // ballot-packed in rank order (the order later walks use).
 // ------------------------------------------------------------------------------------------
-constexpr int kClassifySpan = 8;      // vocabulary blocks of 256 ranks per thread block
+// A block classifies one chunk of kClassifyChunk tokens of one position.  Only tokens whose first byte the position's
+// own edges can take are ever looked at: in trie order the tokens that start with byte b are the ranks
+// [first_rank[b], first_rank[b + 1]), so the position's viable tokens are a union of at most 256 rank ranges, and the
+// host lists, per position, as many chunks as those ranges hold tokens (work[i] = (position, chunk)).  Everything
+// else is rejected without being touched: the rows are zeroed beforehand.
+constexpr int kClassifyChunk = 2048;
 
 // kCount: also add up the bytes the walks consume (viable trie nodes visited, without any sharing between tokens)
 // into *visits -- the work the classification actually does, as opposed to the (position, token) pairs it decides.
 template <bool kCount>
 __global__ void __launch_bounds__(256)
-classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
+classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, const int2* __restrict__ work,
                 uint32_t* __restrict__ acc_id, uint32_t* __restrict__ unc_id, uint32_t* __restrict__ unc_rank,
                 int2* __restrict__ overflow, int* __restrict__ overflow_count, int overflow_cap, unsigned long long* __restrict__ visits) {
   __shared__ uint32_t sh_st[1];
   __shared__ int32_t sh_org[1];
   __shared__ uint32_t sh_class[kSharedClasses * 8];
   __shared__ uint32_t sh_first[8];          // bytes the position's own edges can take
-  __shared__ uint32_t sh_live;              // which of this block's vocabulary blocks hold a token that survives its first byte
-  const int pos = blockIdx.y;
+  __shared__ int sh_cum[257];               // sh_cum[b]: viable tokens whose first byte is below b
+  const int pos = work[blockIdx.x].x, chunk = work[blockIdx.x].y;
   const int state = positions[pos];
-  const int n_vblocks = (v.vocab_size + 255) >> 8;
   if (threadIdx.x < 8) {
     const StateRec rec = g.state[state];
     uint32_t w = 0;
@@ -220,37 +224,34 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
     }
     sh_first[threadIdx.x] = w;
   }
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    // The tokens of a vocabulary block are a contiguous run of the trie order, so their first bytes span
-    // [first of the first token, first of the last] (a table of the tokenizer); most (position, block) pairs
-    // have nothing in common with the position's own first-byte set and are rejected here as a whole.
-    bool any = false;
-    const int vb = blockIdx.x * kClassifySpan + (int)threadIdx.x;
-    if (threadIdx.x < kClassifySpan && vb < n_vblocks) {
-      const uint32_t span = v.block_first[vb];
-      for (int b = (int)(span & 0xFFu); b <= (int)(span >> 8) && !any; ++b) any = (sh_first[b >> 5] >> (b & 31)) & 1u;
-    }
-    const uint32_t live = __ballot_sync(0xFFFFFFFFu, any);
-    if (threadIdx.x == 0) { sh_live = live; sh_st[0] = (uint32_t)state; sh_org[0] = -1; }
-  }
-  __syncthreads();
-  const uint32_t live_blocks = sh_live;
-  if (live_blocks == 0) return;              // every token here is rejected on its first byte (the rows are pre-zeroed)
+  if (threadIdx.x == 0) { sh_st[0] = (uint32_t)state; sh_org[0] = -1; }
   const uint32_t* class_bits = stage_class_bits(g, sh_class);
   __syncthreads();
-  for (int i = 0; i < kClassifySpan; ++i) {
-    if (!((live_blocks >> i) & 1u)) continue;
-    const int rank = ((blockIdx.x * kClassifySpan + i) << 8) + (int)threadIdx.x;
-    int cls = 0, walked = 0;
-    bool live = rank < v.vocab_size && !v.never[rank];
-    uint32_t off = 0;
-    if (live) {
-      off = v.offset[rank];
-      const uint32_t first_byte = v.bytes[off];
-      live = (sh_first[first_byte >> 5] >> (first_byte & 31)) & 1u;             // else rejected on the first byte
+  {   // inclusive scan of the 256 range lengths (thread b holds byte b), shifted into sh_cum[b + 1]
+    const int b = (int)threadIdx.x;
+    int x = ((sh_first[b >> 5] >> (b & 31)) & 1u) ? (int)(v.first_rank[b + 1] - v.first_rank[b]) : 0;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xFFFFFFFFu, x, o); if ((b & 31) >= o) x += y; }
+    __shared__ int warp_sum[8];
+    if ((b & 31) == 31) warp_sum[b >> 5] = x;
+    __syncthreads();
+    int base = 0;
+    for (int w = 0; w < (b >> 5); ++w) base += warp_sum[w];
+    sh_cum[b + 1] = base + x;
+    if (b == 0) sh_cum[0] = 0;
+  }
+  __syncthreads();
+  const int total = sh_cum[256];
+  for (int i = 0; i < kClassifyChunk / 256; ++i) {
+    const int idx = chunk * kClassifyChunk + i * 256 + (int)threadIdx.x;        // the idx-th viable token of this position
+    int cls = 0, walked = 0, rank = -1;
+    if (idx < total) {
+      int lo = 0, hi = 256;                   // the first byte whose range holds idx: sh_cum[lo] <= idx < sh_cum[lo + 1]
+      while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (sh_cum[mid] <= idx) lo = mid; else hi = mid; }
+      rank = (int)v.first_rank[lo] + (idx - sh_cum[lo]);
     }
-    if (live) {
+    if (rank >= 0 && XG_BOUND(rank, v.vocab_size, kBoundTokenRank) && !v.never[rank]) {
+      const uint32_t off = v.offset[rank];
       const int len = (int)(v.offset[rank + 1] - off);
       int flags = 0;
       int consumed = 0;
@@ -274,10 +275,9 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
         const int id = v.rank_to_id[rank];
         uint32_t* row = (cls == 1 ? acc_id : unc_id) + (size_t)pos * v.n_words;
         atomicOr(&row[id >> 5], 1u << (id & 31));
+        if (cls == 2) atomicOr(&unc_rank[(size_t)pos * v.n_words + (rank >> 5)], 1u << (rank & 31));
       }
     }
-    const uint32_t ballot = __ballot_sync(0xFFFFFFFFu, cls == 2);
-    if ((threadIdx.x & 31) == 0 && rank < v.vocab_size) unc_rank[(size_t)pos * v.n_words + (rank >> 5)] = ballot;
     if (kCount) {
       const int sum = __reduce_add_sync(0xFFFFFFFFu, walked);
       if ((threadIdx.x & 31) == 0 && sum) atomicAdd(visits, (unsigned long long)sum);
