@@ -725,8 +725,169 @@ __global__ void matcher_reset_kernel(MatcherDev* m) {      // one warp
   prepare_plan(*m, *m->grammar, threadIdx.x);
 }
 
-// Accept one sampled token of one request (Section 2.2 "trace the output"), by one warp.  Lane 0
-// walks the token's bytes into the warp's scratch (w_st, w_org: kFastCap items, lsb: kFastMaxBytes
+// ------------------------------------------------------------------------------------------
+// The token walk by a whole warp (the sampled token of one request: nothing else to do at that moment, and its
+// latency is the step's).  The same scan / complete as token_walk, but the lanes share every round of loads: in the
+// scan each lane takes one (item, scan edge) pair of the current set -- the records of all items, then all edges,
+// then the class words they need are each one round trip, however many edges a state has (a string-body state has
+// about ten) --, a ballot collects the hits, and in a completion each lane takes one (waiting item, wait edge)
+// pair of the origin set.  Sets live in the warp's shared-memory scratch (st, org: `cap` items; lsb as in
+// token_walk).  All 32 lanes must call; the result is the same in every lane.
+// ------------------------------------------------------------------------------------------
+constexpr uint32_t kFullWarp = 0xFFFFFFFFu;
+
+// append (ns, no) to the set [start, cnt) unless present (same arguments in every lane); false on overflow
+__device__ __forceinline__ bool warp_add_item(uint32_t* st, int32_t* org, int start, int& cnt, int cap, uint32_t ns, int32_t no, int lane) {
+  bool dup = false;
+  for (int q = start + lane; q < cnt; q += 32) dup = dup || (st[q] == ns && org[q] == no);
+  if (__any_sync(kFullWarp, dup)) return true;
+  if (cnt >= cap) return false;
+  if (lane == 0) { st[cnt] = ns; org[cnt] = no; }
+  ++cnt;
+  __syncwarp();
+  return true;
+}
+
+// lane -> the index of the first lane whose inclusive prefix exceeds p (the owner of flattened pair p); `n` lanes hold items
+__device__ __forceinline__ int owner_of_pair(int incl, int p, int n) {
+  int own = 0;
+  for (int l = 0; l < n; ++l) own += p >= __shfl_sync(kFullWarp, incl, l) ? 1 : 0;
+  return own;
+}
+
+__device__ __forceinline__ int warp_inclusive_scan(int x, int lane) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(kFullWarp, x, o); if (lane >= o) x += y; }
+  return x;
+}
+
+// advance every item of chart set `o` that waits for `rule` into the set [start, cnt)
+template <typename LsbT>
+__device__ __forceinline__ bool warp_advance_waiters(const GrammarDev& g, const Chart& c, uint32_t rule, int32_t o, uint32_t* st, int32_t* org,
+                                                     const LsbT* lsb, int start, int& cnt, int cap, int lane) {
+  const uint32_t* src_st;
+  const int32_t* src_org;
+  int b, e;
+  if (o < c.i_idx) {
+    if (!XG_BOUND(o, c.n + 1, kBoundChartSet)) return true;
+    src_st = c.h_st; src_org = c.h_org; b = c.h_sb[o]; e = c.h_sb[o + 1];
+    if (!XG_BOUND(e, c.h_items + 1, kBoundChartItem) || !XG_BOUND(b, e + 1, kBoundChartItem)) return true;
+  }
+  else if (o == c.i_idx) { src_st = c.i_st; src_org = c.i_org; b = 0; e = c.i_cnt; }
+  else {
+    src_st = st; src_org = org; b = lsb[o - c.i_idx]; e = lsb[o - c.i_idx + 1];
+    if (!XG_BOUND(e, cnt + 1, kBoundWalkItem) || !XG_BOUND(b, e + 1, kBoundWalkItem)) return true;
+  }
+  for (int base = b; base < e; base += 32) {
+    const int n_here = min(32, e - base);
+    const bool have = lane < n_here;
+    const uint32_t s2 = have ? src_st[base + lane] : 0u;
+    const int32_t o2 = have ? src_org[base + lane] : 0;
+    uint4 rec = make_uint4(0, 0, 0, 0);
+    if (have && XG_BOUND(s2, g.n_states, kBoundState)) rec = *reinterpret_cast<const uint4*>(&g.state[s2]);
+    int n_wait = (int)(rec.w & 0xFFFFu);
+    if (!XG_BOUND((int)rec.z + n_wait, g.n_wait_edges + 1, kBoundWaitEdge)) n_wait = 0;
+    const int incl = warp_inclusive_scan(n_wait, lane);
+    const int total = __shfl_sync(kFullWarp, incl, 31);
+    for (int p0 = 0; p0 < total; p0 += 32) {
+      const int p = p0 + lane;
+      const int own = min(owner_of_pair(incl, p, n_here), 31);
+      const int first = __shfl_sync(kFullWarp, incl - n_wait, own), wb = __shfl_sync(kFullWarp, (int)rec.z, own);
+      const int32_t o2_own = __shfl_sync(kFullWarp, o2, own);
+      uint2 we = make_uint2(0xFFFFFFFFu, 0u);
+      if (p < total) we = g.wait_edge[wb + (p - first)];
+      uint32_t hits = __ballot_sync(kFullWarp, p < total && we.x == rule);
+      while (hits) {
+        const int h = __ffs(hits) - 1;
+        hits &= hits - 1;
+        const uint32_t ns = __shfl_sync(kFullWarp, we.y & ~kSelf, h);
+        const int32_t no = __shfl_sync(kFullWarp, (we.y & kSelf) ? o : o2_own, h);
+        if (!warp_add_item(st, org, start, cnt, cap, ns, no, lane)) return false;
+      }
+    }
+  }
+  return true;
+}
+
+template <typename LsbT>
+__device__ __forceinline__ int warp_token_walk(const GrammarDev& g, const Chart& c, const uint8_t* __restrict__ bytes, int len,
+                                               uint32_t* st, int32_t* org, int cap, LsbT* lsb, int* flags, int lane) {
+  int cnt = 0;
+  const uint32_t* cur_st = c.i_st;
+  const int32_t* cur_org = c.i_org;
+  int cur_b = 0, cur_e = c.i_cnt;
+  if (lane == 0) { lsb[0] = 0; lsb[1] = 0; }
+  for (int k = 0; k < len; ++k) {
+    const uint32_t byte = bytes[k];
+    const uint32_t word = byte >> 5, bit = 1u << (byte & 31);
+    const int start = cnt;
+    const int self_idx = c.i_idx + k;
+    // scan: one (item, edge) pair per lane
+    for (int base = cur_b; base < cur_e; base += 32) {
+      const int n_here = min(32, cur_e - base);
+      const bool have = lane < n_here;
+      const uint32_t s = have ? cur_st[base + lane] : 0u;
+      const int32_t o = have ? cur_org[base + lane] : 0;
+      uint4 ra = make_uint4(0, 0, 0, 0), rb = ra;
+      if (have && XG_BOUND(s, g.n_states, kBoundState)) {
+        ra = *reinterpret_cast<const uint4*>(&g.state[s]);
+        rb = *(reinterpret_cast<const uint4*>(&g.state[s]) + 1);
+      }
+      int n_edges = (int)(ra.y >> 16);
+      if (!XG_BOUND((int)ra.x + n_edges, g.n_scan_edges + 1, kBoundScanEdge)) n_edges = 0;
+      const int incl = warp_inclusive_scan(n_edges, lane);
+      const int total = __shfl_sync(kFullWarp, incl, 31);
+      for (int p0 = 0; p0 < total; p0 += 32) {
+        const int p = p0 + lane;
+        const int own = min(owner_of_pair(incl, p, n_here), 31);
+        const int first = __shfl_sync(kFullWarp, incl - n_edges, own), sb = __shfl_sync(kFullWarp, (int)ra.x, own);
+        const int32_t o_own = __shfl_sync(kFullWarp, o, own);
+        const uint32_t e0c = __shfl_sync(kFullWarp, rb.z, own), e0t = __shfl_sync(kFullWarp, rb.w, own);
+        uint2 se = make_uint2(kLiteral | 0x100u, 0u);
+        if (p < total) se = p == first ? make_uint2(e0c, e0t) : g.scan_edge[sb + (p - first)];      // the first edge is inline in the record
+        // the record of the edge's target is requested before the byte is tested against the edge's class: if the edge
+        // is taken, the new item's `info` word (and the scan of the next byte) find it on its way
+        if (p < total && XG_BOUND(se.y & ~kSelf, g.n_states, kBoundState)) asm volatile("prefetch.global.L1 [%0];" ::"l"(&g.state[se.y & ~kSelf]));
+        bool hit = false;
+        if (se.x & kLiteral) hit = (se.x & 0x1FFu) == byte;
+        else if (XG_BOUND(se.x, g.n_classes, kBoundClass)) hit = (g.class_bits[se.x * 8 + word] & bit) != 0;
+        uint32_t hits = __ballot_sync(kFullWarp, hit);
+        while (hits) {
+          const int h = __ffs(hits) - 1;
+          hits &= hits - 1;
+          const uint32_t ns = __shfl_sync(kFullWarp, se.y & ~kSelf, h);
+          const int32_t no = __shfl_sync(kFullWarp, (se.y & kSelf) ? self_idx : o_own, h);
+          if (!warp_add_item(st, org, start, cnt, cap, ns, no, lane)) { *flags |= kWalkOverflow; return k; }
+        }
+      }
+    }
+    if (cnt == start) return k;
+    // complete (cascades through the growing set): the `info` words of the new items one per lane, then one completion at a time
+    for (int q = start; q < cnt;) {
+      const int n_here = min(32, cnt - q);
+      uint32_t info = 0;
+      int32_t o = 0;
+      if (lane < n_here && XG_BOUND(st[q + lane], g.n_states, kBoundState)) { info = g.state[st[q + lane]].info; o = org[q + lane]; }
+      uint32_t done = __ballot_sync(kFullWarp, (info >> 31) != 0);
+      q += n_here;
+      while (done) {
+        const int h = __ffs(done) - 1;
+        done &= done - 1;
+        const uint32_t rule = __shfl_sync(kFullWarp, info, h) & 0x7FFFFFFFu;
+        const int32_t oo = __shfl_sync(kFullWarp, o, h);
+        if (oo < 0) continue;             // (an item of unknown context: cache build only, never in a request's chart)
+        if (!warp_advance_waiters(g, c, rule, oo, st, org, lsb, start, cnt, cap, lane)) { *flags |= kWalkOverflow; return k; }
+      }
+    }
+    cur_st = st; cur_org = org; cur_b = start; cur_e = cnt;
+    if (lane == 0) lsb[k + 2] = (LsbT)cnt;
+    __syncwarp();
+  }
+  return len;
+}
+
+// Accept one sampled token of one request (Section 2.2 "trace the output"), by one warp.  The warp
+// walks the token's bytes into its scratch (w_st, w_org: kFastCap items, lsb: kFastMaxBytes
 // + 2); if every byte survived, the warp appends the new sets behind the request's history, lane
 // 0 commits the counters and the warp builds the plan of the next mask.  A rejected token leaves
 // the matcher as it was.  With restart_on_eos an accepted end-of-sequence token puts the matcher
@@ -765,22 +926,20 @@ __device__ __forceinline__ int accept_one(MatcherDev& m, const GrammarDev& g, co
     const int piece = min(len - done, kFastMaxBytes);
     int made = 0, slow = 0;
     if (n_sets + piece > m.cap_sets) st = -6;
-    else if (lane == 0) {
+    else {
       int flags = 0;
       const Chart c = done == 0 ? c0 : chart_of_history(m.item_state, m.item_origin, m.set_begin, n_sets - 1);
-      int consumed = token_walk<int16_t>(g, g.class_bits, c, v.bytes + off + done, piece, false, w_st, w_org, kFastCap, lsb, &flags, nullptr);
+      int consumed = warp_token_walk<int16_t>(g, c, v.bytes + off + done, piece, w_st, w_org, kFastCap, lsb, &flags, lane);
       if (flags & kWalkOverflow) {       // the sets do not fit the warp's scratch: the same walk again, exactly, in the matcher's large one
         flags = 0;
         slow = 1;
-        consumed = token_walk<int32_t>(g, g.class_bits, c, v.bytes + off + done, piece, false, m.slow_st, m.slow_org, kSlowCap, m.slow_lsb, &flags, nullptr);
+        consumed = warp_token_walk<int32_t>(g, c, v.bytes + off + done, piece, m.slow_st, m.slow_org, kSlowCap, m.slow_lsb, &flags, lane);
       }
+      __syncwarp();
       if (flags & kWalkOverflow) st = -6;
       else if (consumed < piece) st = -7;
       else { made = slow ? m.slow_lsb[piece + 1] : lsb[piece + 1]; if (n_items + made > m.cap_items) st = -6; }
     }
-    st = __shfl_sync(0xFFFFFFFFu, st, 0);
-    made = __shfl_sync(0xFFFFFFFFu, made, 0);
-    slow = __shfl_sync(0xFFFFFFFFu, slow, 0);
     if (st != 0) break;
     __syncwarp();
     // origins written by the walk are already chart indices (its base is set n_sets - 1);
