@@ -72,6 +72,21 @@ __device__ __forceinline__ Chart chart_of_history(const uint32_t* h_st, const in
   return c;
 }
 
+constexpr uint32_t kFullWarp = 0xFFFFFFFFu;
+
+// lane -> the index of the first lane whose inclusive prefix exceeds p (the owner of flattened pair p); `n` lanes hold items
+__device__ __forceinline__ int owner_of_pair(int incl, int p, int n) {
+  int own = 0;
+  for (int l = 0; l < n; ++l) own += p >= __shfl_sync(kFullWarp, incl, l) ? 1 : 0;
+  return own;
+}
+
+__device__ __forceinline__ int warp_inclusive_scan(int x, int lane) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(kFullWarp, x, o); if (lane >= o) x += y; }
+  return x;
+}
+
 // append (ns, no) to the set [start, cnt) unless present; false on overflow
 __device__ __forceinline__ bool add_item(uint32_t* st, int32_t* org, int start, int& cnt, int cap, uint32_t ns, int32_t no) {
   for (int q = start; q < cnt; ++q) if (st[q] == ns && org[q] == no) return true;
@@ -636,49 +651,85 @@ __device__ __forceinline__ bool root_complete(const MatcherDev& m, const Grammar
   return false;
 }
 
-// Build the step plan of the request's current set.  One warp: lane 0 lists the entries, then
-// one lane per entry completes that entry's rule into its continuation set.
+// Build the step plan of the request's current set, by one warp.  The entries are listed with one lane per (item of
+// the set, entry of its gather list) pair, so that the table lookups behind every pair -- the item's record, the gather
+// entry, the cache entry's header -- are three rounds of loads for the whole set; the lists themselves are kept in
+// registers, one slot per lane, and a pair is added to them by a compare in every lane and a vote.  Then one lane per
+// entry completes that entry's rule into its continuation set.
 __device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g, int lane) {
   StepPlan& p = *m.plan;
   const int n = m.n_sets - 1;
   const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
-  int n_check = 0;
-  if (lane == 0) {
-    int n_merge = 0, overflow = 0, n_missing = 0;
-    p.check_cum[0] = 0;
-    for (int i = 0; i < hist.i_cnt && !overflow; ++i) {
-      const uint32_t s = hist.i_st[i];
-      if (!XG_BOUND(s, g.n_states, kBoundState)) continue;
-      const StateRec rec = g.state[s];
-      if (!XG_BOUND(rec.gather_begin + (int)(rec.n_wait_n_gather >> 16), g.n_gather + 1, kBoundGather)) continue;
-      for (int gi = rec.gather_begin; gi < rec.gather_begin + (int)(rec.n_wait_n_gather >> 16); ++gi) {
-        const int code = g.gather_state[gi];
-        const int q = code & 0x7FFFFFFF;
-        if (!XG_BOUND(q, g.n_states, kBoundEntry)) continue;
-        const int origin = code < 0 ? n : hist.i_org[i];          // predicted start states begin here
-        bool seen = false;
-        if (g.entries[q].kind == kEntryNotBuilt) {                // a just-in-time grammar has not built this entry yet
-          for (int z = 0; z < min(n_missing, kPlanMissingMax); ++z) seen = seen || p.missing_state[z] == q;
-          if (!seen) { if (n_missing < kPlanMissingMax) p.missing_state[n_missing] = q; ++n_missing; }
+  int n_merge = 0, n_check = 0, n_missing = 0, overflow = 0;       // (the same in every lane)
+  int merge_lo = -1, merge_hi = -1;           // slots lane and lane + 32 of the merge list
+  int check_q = -1, check_o = 0, check_n = 0; // slot lane of the check list: state, origin, candidates
+  int missing_q = -1;                         // slot lane of the missing list (lanes below kPlanMissingMax)
+  bool root_done = m.n_sets == 1 && g.root_nullable;
+  static_assert(kPlanMergeMax == 64 && kPlanCheckMax == 32 && kPlanMissingMax <= 32, "one or two list slots per lane");
+  for (int base = 0; base < hist.i_cnt && !overflow; base += 32) {
+    const int n_here = min(32, hist.i_cnt - base);
+    const bool have = lane < n_here;
+    const uint32_t s = have ? hist.i_st[base + lane] : 0u;
+    const int32_t o = have ? hist.i_org[base + lane] : 0;
+    int gather_begin = 0, n_gather = 0;
+    if (have && XG_BOUND(s, g.n_states, kBoundState)) {
+      const uint4 ra = *reinterpret_cast<const uint4*>(&g.state[s]), rb = *(reinterpret_cast<const uint4*>(&g.state[s]) + 1);
+      gather_begin = (int)rb.x; n_gather = (int)(ra.w >> 16);
+      if (!XG_BOUND(gather_begin + n_gather, g.n_gather + 1, kBoundGather)) n_gather = 0;
+      // EOS is allowed iff the root rule is complete with origin 0
+      root_done = root_done || (o == 0 && (rb.y >> 31) && (rb.y & 0x7FFFFFFFu) == (uint32_t)g.root_rule);
+    }
+    const int incl = warp_inclusive_scan(n_gather, lane);
+    const int total = __shfl_sync(kFullWarp, incl, 31);
+    for (int p0 = 0; p0 < total && !overflow; p0 += 32) {
+      const int pi = p0 + lane;
+      const int own = min(owner_of_pair(incl, pi, n_here), 31);
+      const int first = __shfl_sync(kFullWarp, incl - n_gather, own), gb = __shfl_sync(kFullWarp, gather_begin, own);
+      const int32_t o_own = __shfl_sync(kFullWarp, o, own);
+      int q = -1, origin = 0, kind = 0, n_chk = 0;
+      if (pi < total) {
+        const int code = g.gather_state[gb + (pi - first)];
+        q = code & 0x7FFFFFFF;
+        origin = code < 0 ? n : o_own;                       // predicted start states begin here
+        if (XG_BOUND(q, g.n_states, kBoundEntry)) { kind = g.entries[q].kind; n_chk = g.entries[q].n_chk; } else q = -1;
+      }
+      uint32_t todo = __ballot_sync(kFullWarp, q >= 0);
+      while (todo && !overflow) {                            // the pairs in order, each decided by all lanes at once
+        const int h = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const int qh = __shfl_sync(kFullWarp, q, h), oh = __shfl_sync(kFullWarp, origin, h);
+        const int kh = __shfl_sync(kFullWarp, kind, h), nh = __shfl_sync(kFullWarp, n_chk, h);
+        if (kh == kEntryNotBuilt) {                          // a just-in-time grammar has not built this entry yet
+          if (!__any_sync(kFullWarp, lane < min(n_missing, kPlanMissingMax) && missing_q == qh)) {
+            if (lane == n_missing) missing_q = qh;           // (beyond kPlanMissingMax only counted)
+            ++n_missing;
+          }
           continue;
         }
-        for (int z = 0; z < n_merge; ++z) seen = seen || p.merge_state[z] == q;
-        if (!seen) { if (n_merge == kPlanMergeMax) { overflow = 1; break; } p.merge_state[n_merge++] = q; }
-        const int n_unc = g.entries[q].n_chk;
-        if (n_unc == 0) continue;
-        seen = false;
-        for (int z = 0; z < n_check; ++z) seen = seen || (p.check_state[z] == q && p.check_origin[z] == origin);
-        if (seen) continue;
+        if (!__any_sync(kFullWarp, (lane < n_merge && merge_lo == qh) || (lane + 32 < n_merge && merge_hi == qh))) {
+          if (n_merge == kPlanMergeMax) { overflow = 1; break; }
+          if (lane == (n_merge & 31)) { if (n_merge < 32) merge_lo = qh; else merge_hi = qh; }
+          ++n_merge;
+        }
+        if (nh == 0) continue;
+        if (__any_sync(kFullWarp, lane < n_check && check_q == qh && check_o == oh)) continue;
         if (n_check == kPlanCheckMax) { overflow = 1; break; }
-        p.check_state[n_check] = q; p.check_origin[n_check] = origin;
-        p.check_cum[n_check + 1] = p.check_cum[n_check] + n_unc;
+        if (lane == n_check) { check_q = qh; check_o = oh; check_n = nh; }
         ++n_check;
       }
     }
-    p.n_merge = n_merge; p.n_check = n_check; p.overflow = overflow; p.n_missing = n_missing;
-    p.eos_ok = root_complete(m, g) ? 1 : 0;
   }
-  n_check = __shfl_sync(0xFFFFFFFFu, n_check, 0);
+  if (lane < n_merge) p.merge_state[lane] = merge_lo;
+  if (lane + 32 < n_merge) p.merge_state[lane + 32] = merge_hi;
+  if (lane < min(n_missing, kPlanMissingMax)) p.missing_state[lane] = missing_q;
+  const int cum = warp_inclusive_scan(lane < n_check ? check_n : 0, lane);
+  if (lane < n_check) { p.check_state[lane] = check_q; p.check_origin[lane] = check_o; p.check_cum[lane + 1] = cum; }
+  root_done = __any_sync(kFullWarp, root_done);
+  if (lane == 0) {
+    p.check_cum[0] = 0;
+    p.n_merge = n_merge; p.n_check = n_check; p.overflow = overflow; p.n_missing = n_missing;
+    p.eos_ok = root_done ? 1 : 0;
+  }
   __syncwarp();
   // continuation set of every entry: complete rule(q) started at its origin, with cascades
   bool bad = false;
@@ -734,7 +785,6 @@ __global__ void matcher_reset_kernel(MatcherDev* m) {      // one warp
 // pair of the origin set.  Sets live in the warp's shared-memory scratch (st, org: `cap` items; lsb as in
 // token_walk).  All 32 lanes must call; the result is the same in every lane.
 // ------------------------------------------------------------------------------------------
-constexpr uint32_t kFullWarp = 0xFFFFFFFFu;
 
 // append (ns, no) to the set [start, cnt) unless present (same arguments in every lane); false on overflow
 __device__ __forceinline__ bool warp_add_item(uint32_t* st, int32_t* org, int start, int& cnt, int cap, uint32_t ns, int32_t no, int lane) {
@@ -746,19 +796,6 @@ __device__ __forceinline__ bool warp_add_item(uint32_t* st, int32_t* org, int st
   ++cnt;
   __syncwarp();
   return true;
-}
-
-// lane -> the index of the first lane whose inclusive prefix exceeds p (the owner of flattened pair p); `n` lanes hold items
-__device__ __forceinline__ int owner_of_pair(int incl, int p, int n) {
-  int own = 0;
-  for (int l = 0; l < n; ++l) own += p >= __shfl_sync(kFullWarp, incl, l) ? 1 : 0;
-  return own;
-}
-
-__device__ __forceinline__ int warp_inclusive_scan(int x, int lane) {
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(kFullWarp, x, o); if (lane >= o) x += y; }
-  return x;
 }
 
 // advance every item of chart set `o` that waits for `rule` into the set [start, cnt)
