@@ -766,15 +766,28 @@ struct Tables {
   std::vector<uint8_t> state_final;
   std::vector<int32_t> cb, cc, ct, rb, rr, rt;
   std::vector<uint32_t> class_bits;
-  std::map<int, std::vector<uint8_t>> cls_cache;     // state -> per-token class (filled lazily)
+  // counted repetitions (Section 3.6, "the parser state for R{l,r} is (R{l,r}, k)"): rule r with rep_hi[r] != 0 is
+  // X{rep_lo[r], rep_hi[r]} on the automaton of X; ci / ri mark the edges that start the next iteration
+  std::vector<int32_t> rep_lo, rep_hi;
+  std::vector<uint8_t> ci, ri;
+  std::map<std::pair<int, int>, std::vector<uint8_t>> cls_cache;     // (state, count) -> per-token class (filled lazily)
   bool class_has(int c, uint8_t b) const { return (class_bits[(size_t)c * 8 + (b >> 5)] >> (b & 31)) & 1u; }
   bool scannable(int s) const { return cb[s + 1] > cb[s]; }
+  bool counted(int s) const { return !rep_hi.empty() && rep_hi[state_rule[s]] != 0; }
+  // may an item at state s that has finished k iterations start another one?
+  bool may_iterate(int s, int k) const { return k + 1 < rep_hi[state_rule[s]]; }
+  // is an item at state s with count k a finished instance of its rule?
+  bool complete(int s, int k) const { return state_final[s] && (!counted(s) || k + 1 >= rep_lo[state_rule[s]]); }
+  bool citer(int e) const { return !ci.empty() && ci[e]; }
+  bool riter(int e) const { return !ri.empty() && ri[e]; }
 };
 
-struct TItem { int state, origin; };      // origin -1: the unknown context that referenced the rule
+// origin -1: the unknown context that referenced the rule.  k: inside a counted repetition, the iterations finished
+// before the current one (0 elsewhere).
+struct TItem { int state, origin, k; };
 typedef std::vector<TItem> TSet;
 inline bool tadd(TSet& s, TItem it) {
-  for (const TItem& x : s) if (x.state == it.state && x.origin == it.origin) return false;
+  for (const TItem& x : s) if (x.state == it.state && x.origin == it.origin && x.k == it.k) return false;
   s.push_back(it);
   return true;
 }
@@ -787,21 +800,28 @@ struct TView {
 
 // predict + complete to a fixpoint.  Completing an item whose origin is the unknown context
 // cannot advance anything here; it is reported through *left_rule.
+// An edge that starts the next iteration of a counted repetition exists only while k + 1 < hi and leads to k + 1.
 void tclosure(const Tables& t, const TView& v, TSet& cur, int i, bool* left_rule) {
   bool changed = true;
   while (changed) {
     changed = false;
     for (size_t k = 0; k < cur.size(); ++k) {
       TItem it = cur[k];
-      for (int e = t.rb[it.state]; e < t.rb[it.state + 1]; ++e) changed |= tadd(cur, {t.rule_start[t.rr[e]], i});
-      if (t.state_final[it.state]) {
+      for (int e = t.rb[it.state]; e < t.rb[it.state + 1]; ++e) {
+        if (t.riter(e) && !t.may_iterate(it.state, it.k)) continue;
+        changed |= tadd(cur, {t.rule_start[t.rr[e]], i, 0});
+      }
+      if (t.complete(it.state, it.k)) {
         if (it.origin < 0) { if (left_rule) *left_rule = true; continue; }
         int rule = t.state_rule[it.state];
         const TSet& os = it.origin == i ? cur : v.get(it.origin);
         for (size_t q = 0; q < os.size(); ++q) {
           TItem p = os[q];
-          for (int e = t.rb[p.state]; e < t.rb[p.state + 1]; ++e)
-            if (t.rr[e] == rule) changed |= tadd(cur, {t.rt[e], p.origin});
+          for (int e = t.rb[p.state]; e < t.rb[p.state + 1]; ++e) {
+            if (t.rr[e] != rule) continue;
+            if (t.riter(e)) { if (t.may_iterate(p.state, p.k)) changed |= tadd(cur, {t.rt[e], p.origin, p.k + 1}); }
+            else changed |= tadd(cur, {t.rt[e], p.origin, p.k});
+          }
         }
       }
     }
@@ -809,8 +829,11 @@ void tclosure(const Tables& t, const TView& v, TSet& cur, int i, bool* left_rule
 }
 void tscan(const Tables& t, const TSet& cur, TSet& next, uint8_t b) {
   for (const TItem& it : cur)
-    for (int e = t.cb[it.state]; e < t.cb[it.state + 1]; ++e)
-      if (t.class_has(t.cc[e], b)) tadd(next, {t.ct[e], it.origin});
+    for (int e = t.cb[it.state]; e < t.cb[it.state + 1]; ++e) {
+      if (!t.class_has(t.cc[e], b)) continue;
+      if (t.citer(e)) { if (t.may_iterate(it.state, it.k)) tadd(next, {t.ct[e], it.origin, it.k + 1}); }
+      else tadd(next, {t.ct[e], it.origin, it.k});
+    }
 }
 bool tfeed(const Tables& t, const std::vector<TSet>& base, std::vector<TSet>& extra, const uint8_t* bytes, int n) {
   TView v{&base, &extra};
@@ -825,14 +848,14 @@ bool tfeed(const Tables& t, const std::vector<TSet>& base, std::vector<TSet>& ex
 }
 
 // class of one token at one scannable state: 1 accepted, 2 uncertain, 0 rejected.
-// The parse starts from the single item (state, unknown context); its first byte must be taken
+// The parse starts from the single item (state, unknown context, count); its first byte must be taken
 // by one of the state's own byte-class edges.  Accepted: every byte is consumed and the set
 // stays non-empty.  Uncertain: not accepted, but the state's rule finished (the parse would
 // continue in the unknown context) with bytes left.  Otherwise rejected.
-int classify_one(const Tables& t, int state, const uint8_t* bytes, int n) {
+int classify_one(const Tables& t, int state, int count, const uint8_t* bytes, int n) {
   if (n == 0) return 0;
   std::vector<TSet> base(1), extra;
-  base[0].push_back({state, -1});
+  base[0].push_back({state, -1, count});
   TView v{&base, &extra};
   bool uncertain = false;
   for (int k = 0; k < n; ++k) {
@@ -854,7 +877,7 @@ struct TMatcher {
   void reset() {
     chart.clear();
     TSet s;
-    tadd(s, {t->rule_start[t->root_rule], 0});
+    tadd(s, {t->rule_start[t->root_rule], 0, 0});
     std::vector<TSet> none, none2;
     TView v{&none, &none2};
     tclosure(*t, v, s, 0, nullptr);
@@ -863,7 +886,7 @@ struct TMatcher {
   bool can_terminate() const {
     if (chart.size() == 1 && t->root_nullable) return true;
     for (const TItem& it : chart.back())
-      if (it.origin == 0 && t->state_final[it.state] && t->state_rule[it.state] == t->root_rule) return true;
+      if (it.origin == 0 && t->complete(it.state, it.k) && t->state_rule[it.state] == t->root_rule) return true;
     return false;
   }
 };
@@ -985,7 +1008,8 @@ void* orc_tables_create(int32_t n_rules, int32_t n_states, int32_t n_classes, in
                         const int32_t* rule_start, const int32_t* state_rule, const uint8_t* state_final,
                         const int32_t* cedge_begin, const int32_t* cedge_class, const int32_t* cedge_target,
                         const int32_t* redge_begin, const int32_t* redge_rule, const int32_t* redge_target,
-                        const uint32_t* class_bits) {
+                        const uint32_t* class_bits, const int32_t* rule_rep_lo, const int32_t* rule_rep_hi,
+                        const uint8_t* cedge_iter, const uint8_t* redge_iter) {
   Tables* t = new Tables();
   t->n_rules = n_rules; t->n_states = n_states; t->root_rule = root_rule; t->root_nullable = root_nullable;
   t->rule_start.assign(rule_start, rule_start + n_rules);
@@ -998,19 +1022,26 @@ void* orc_tables_create(int32_t n_rules, int32_t n_states, int32_t n_classes, in
   t->rr.assign(redge_rule, redge_rule + t->rb[n_states]);
   t->rt.assign(redge_target, redge_target + t->rb[n_states]);
   t->class_bits.assign(class_bits, class_bits + (size_t)n_classes * 8);
+  if (rule_rep_hi) {        // (all four or none)
+    t->rep_lo.assign(rule_rep_lo, rule_rep_lo + n_rules);
+    t->rep_hi.assign(rule_rep_hi, rule_rep_hi + n_rules);
+    t->ci.assign(cedge_iter, cedge_iter + t->cb[n_states]);
+    t->ri.assign(redge_iter, redge_iter + t->rb[n_states]);
+  }
   return t;
 }
 void orc_tables_destroy(void* t) { delete (Tables*)t; }
 
 // out[token] = 1 accepted / 2 uncertain / 0 rejected for every token (EOS, specials, empty: 0)
-void orc_tables_classify(void* tp, void* vp, int32_t state, uint8_t* out, int nthreads) {
+// `count`: inside a counted repetition, the iterations finished before the current one (0 elsewhere)
+void orc_tables_classify(void* tp, void* vp, int32_t state, int32_t count, uint8_t* out, int nthreads) {
   Tables* t = (Tables*)tp;
   VocabO* v = (VocabO*)vp;
   parallel_for(v->size, nthreads, [&](int lo, int hi) {
     for (int tok = lo; tok < hi; ++tok) {
       int n = (int)(v->offsets[tok + 1] - v->offsets[tok]);
       if (tok == v->eos || v->special[tok] || n == 0) { out[tok] = 0; continue; }
-      out[tok] = (uint8_t)classify_one(*t, state, v->bytes.data() + v->offsets[tok], n);
+      out[tok] = (uint8_t)classify_one(*t, state, count, v->bytes.data() + v->offsets[tok], n);
     }
   });
 }
@@ -1032,6 +1063,13 @@ int orc_tmatcher_get_set(void* mp, int i, int32_t* out, int cap) {
   TMatcher* m = (TMatcher*)mp;
   const TSet& s = m->chart[i];
   for (size_t k = 0; k < s.size() && (int)k < cap; ++k) { out[2 * k] = s[k].state; out[2 * k + 1] = s[k].origin; }
+  return (int)s.size();
+}
+// the iteration counts of the items of set i, in the same order
+int orc_tmatcher_get_set_counts(void* mp, int i, int32_t* out, int cap) {
+  TMatcher* m = (TMatcher*)mp;
+  const TSet& s = m->chart[i];
+  for (size_t k = 0; k < s.size() && (int)k < cap; ++k) out[k] = s[k].k;
   return (int)s.size();
 }
 // plain definition on the tables: allowed iff every byte leaves a non-empty set
@@ -1064,13 +1102,13 @@ void orc_tmatcher_mask_merged(void* mp, void* vp, uint32_t* words, int64_t* n_ch
   VocabO* v = (VocabO*)vp;
   int nwords = (v->size + 31) / 32;
   std::memset(words, 0, sizeof(uint32_t) * nwords);
-  std::vector<int> states;
+  std::vector<std::pair<int, int>> states;          // (state, count)
   for (const TItem& it : m->chart.back())
-    if (t->scannable(it.state) && std::find(states.begin(), states.end(), it.state) == states.end()) states.push_back(it.state);
-  for (int s : states)
+    if (t->scannable(it.state) && std::find(states.begin(), states.end(), std::make_pair(it.state, it.k)) == states.end()) states.push_back({it.state, it.k});
+  for (auto s : states)
     if (!t->cls_cache.count(s)) {
       std::vector<uint8_t> cls(v->size);
-      orc_tables_classify(t, v, s, cls.data(), 1);
+      orc_tables_classify(t, v, s.first, s.second, cls.data(), 1);
       t->cls_cache[s] = cls;
     }
   int64_t checked = 0;
@@ -1080,7 +1118,7 @@ void orc_tmatcher_mask_merged(void* mp, void* vp, uint32_t* words, int64_t* n_ch
     if (tok == v->eos) { if (m->can_terminate()) set_bit(words, tok); continue; }
     if (v->special[tok] || n == 0) continue;
     bool acc = false, unc = false;
-    for (int s : states) { uint8_t c = t->cls_cache[s][tok]; acc |= c == 1; unc |= c == 2; }
+    for (auto s : states) { uint8_t c = t->cls_cache[s][tok]; acc |= c == 1; unc |= c == 2; }
     if (!acc && unc) { ++checked; extra.clear(); acc = tfeed(*t, m->chart, extra, v->bytes.data() + v->offsets[tok], n); }
     if (acc) set_bit(words, tok);
   }

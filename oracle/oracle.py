@@ -49,15 +49,16 @@ def lib():
         L.orc_apply_f32.argtypes = [vp, i32, i32, i64, vp, i64]
         L.orc_apply_bf16.argtypes = [vp, i32, i32, i64, vp, i64]
         L.orc_tables_create.restype = vp
-        L.orc_tables_create.argtypes = [i32, i32, i32, i32, i32] + [vp] * 10
+        L.orc_tables_create.argtypes = [i32, i32, i32, i32, i32] + [vp] * 14
         L.orc_tables_destroy.argtypes = [vp]
-        L.orc_tables_classify.argtypes = [vp, vp, i32, vp, C.c_int]
+        L.orc_tables_classify.argtypes = [vp, vp, i32, i32, vp, C.c_int]
         L.orc_tmatcher_create.restype = vp
         L.orc_tmatcher_create.argtypes = [vp]
         for name in ("orc_tmatcher_destroy", "orc_tmatcher_reset", "orc_tmatcher_can_terminate", "orc_tmatcher_num_sets"):
             getattr(L, name).argtypes = [vp]
         L.orc_tmatcher_accept_bytes.argtypes = [vp, C.c_char_p, C.c_int]
         L.orc_tmatcher_get_set.argtypes = [vp, C.c_int, vp, C.c_int]
+        L.orc_tmatcher_get_set_counts.argtypes = [vp, C.c_int, vp, C.c_int]
         L.orc_tmatcher_mask_plain.argtypes = [vp, vp, vp, C.c_int]
         L.orc_tmatcher_mask_merged.argtypes = [vp, vp, vp, vp]
         _lib = L
@@ -184,9 +185,19 @@ class Tables:
         for f in self.FIELDS:
             dt = np.uint8 if f == "state_final" else (np.uint32 if f == "class_bits" else np.int32)
             self.a[f] = np.ascontiguousarray(arrays[f], dtype=dt)
+        # counted repetitions (Section 3.6): bounds per rule and the edges that start the next iteration; absent or
+        # empty when the grammar has none
+        self.counted = "rule_rep_hi" in arrays and np.asarray(arrays["rule_rep_hi"]).size > 0
+        for f, dt in (("rule_rep_lo", np.int32), ("rule_rep_hi", np.int32), ("cedge_iter", np.uint8), ("redge_iter", np.uint8)):
+            self.a[f] = np.ascontiguousarray(arrays[f], dtype=dt) if self.counted else np.zeros(0, dtype=dt)
+        if self.counted:       # (an edge array may be empty: pass a valid pointer anyway)
+            for f in ("cedge_iter", "redge_iter"):
+                if self.a[f].size == 0:
+                    self.a[f] = np.zeros(1, dtype=np.uint8)
         ptr = lambda f: self.a[f].ctypes.data if self.a[f].size else None
         self.h = lib().orc_tables_create(n_rules, n_states, n_classes, root_rule, root_nullable,
-                                         *[ptr(f) for f in self.FIELDS])
+                                         *[ptr(f) for f in self.FIELDS],
+                                         *[ptr(f) for f in ("rule_rep_lo", "rule_rep_hi", "cedge_iter", "redge_iter")])
 
     def __del__(self):
         if getattr(self, "h", None):
@@ -197,10 +208,11 @@ class Tables:
         cb = self.a["cedge_begin"]
         return [s for s in range(self.n_states) if cb[s + 1] > cb[s]]
 
-    def classify(self, vocab: Vocab, state: int, threads: Optional[int] = None) -> np.ndarray:
-        """uint8[V]: 1 accepted, 2 uncertain, 0 rejected."""
+    def classify(self, vocab: Vocab, state: int, threads: Optional[int] = None, count: int = 0) -> np.ndarray:
+        """uint8[V]: 1 accepted, 2 uncertain, 0 rejected.  count: iterations finished before the current one, for a
+        state of a counted repetition (Section 3.6)."""
         out = np.zeros(vocab.size, dtype=np.uint8)
-        lib().orc_tables_classify(self.h, vocab.h, int(state), out.ctypes.data, threads or default_threads())
+        lib().orc_tables_classify(self.h, vocab.h, int(state), int(count), out.ctypes.data, threads or default_threads())
         return out
 
 
@@ -230,6 +242,12 @@ class TableMatcher:
         buf = np.zeros(2 * 4096, dtype=np.int32)
         n = lib().orc_tmatcher_get_set(self.h, i, buf.ctypes.data, 4096)
         return [(int(buf[2 * k]), int(buf[2 * k + 1])) for k in range(min(n, 4096))]
+
+    def get_set_counts(self, i: int) -> List[int]:
+        """Iteration counts of the items of set i, in get_set's order."""
+        buf = np.zeros(4096, dtype=np.int32)
+        n = lib().orc_tmatcher_get_set_counts(self.h, i, buf.ctypes.data, 4096)
+        return [int(buf[k]) for k in range(min(n, 4096))]
 
     def mask_plain(self, vocab: Vocab, threads: Optional[int] = None) -> np.ndarray:
         out = np.zeros(vocab.words, dtype=np.uint32)
