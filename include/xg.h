@@ -135,6 +135,12 @@ typedef struct {
                                  <= 0 = default (32 MiB).  Only the pool's first just-in-time compile sets it. */
   int32_t count_node_visits;  /* non-zero: the classification also counts the token bytes its walks consume
                                  (xg_grammar_stats_t.node_visits); statistics only, costs an atomic per warp. */
+  int32_t repeat_threshold;   /* counted repetitions (Section 3.6): a bounded repetition X{l,r} with r >= this many iterations
+                                 is kept as one copy of X whose Earley items carry the count k of finished iterations (the
+                                 paper's parser state (R{l,r}, k)), so states and front-end time do not grow with r.
+                                 0 = default (64); negative = never (every repetition is expanded into explicit states). */
+  int32_t repeat_depth;       /* the longest token in bytes, for front-end-only compiles (tok == NULL); ignored when a
+                                 tokenizer is given (its own longest token is used).  Without either, nothing is counted. */
   int32_t reserved;
 } xg_compile_options_t;
 
@@ -177,8 +183,25 @@ typedef struct {
   const int32_t* redge_rule;
   const int32_t* redge_target;
   const uint32_t* class_bits;
+  /* Counted repetitions (Section 3.6), NULL when the grammar has none.  rule_rep_lo/hi[r] != 0: rule r is X{lo,hi}
+   * (1 <= lo <= hi) on the automaton of X, whose accepting states also carry copies of the start state's edges with
+   * cedge_iter / redge_iter set ("the next iteration starts here").  An item of such a rule is (state, origin, k),
+   * k = iterations finished before the current one: an iteration edge needs k + 1 < hi and leads to k + 1, the other
+   * edges keep k, and the item is complete iff its state is accepting and k + 1 >= lo. */
+  const int32_t* rule_rep_lo;
+  const int32_t* rule_rep_hi;
+  const uint8_t* cedge_iter;
+  const uint8_t* redge_iter;
+  int32_t n_records;          /* what the cache is indexed by: n_states, plus one record per class of counts for the states
+                                 of counted rules (xg_grammar_record_of) */
 } xg_grammar_tables_t;
 xg_status_t xg_grammar_get_tables(const xg_grammar_t* g, xg_grammar_tables_t* host_view);
+
+/* The cache record of (state, count): `state` itself for ordinary states; for a state of a counted rule the record of
+ * the class its count falls into -- counts that no token of this vocabulary can tell apart, i.e. equally far (up to the
+ * longest token's length) from both bounds, share one record and one cache entry (Section 3.6).
+ * xg_grammar_get_cache_entry takes records.  XG_ERR_INVALID_ARG if the count is not below the rule's upper bound. */
+xg_status_t xg_grammar_record_of(const xg_grammar_t* g, int32_t state, int32_t count, int32_t* record);
 
 /* Structural hash of every rule (Section 3.3: Algorithm 1 bottom-up over the reference graph,
  * cycles refined as in Algorithm 2), the keys of the cross-grammar cache.  out: host, [n_rules].

@@ -26,7 +26,7 @@ DTYPE_BY_NAME = {"f32": XG_F32, "bf16": XG_BF16}
 
 EXPORTS = [
     "xg_last_error", "xg_debug_bounds_enabled", "xg_debug_bounds_check", "xg_tokenizer_create", "xg_tokenizer_destroy", "xg_cache_pool_create", "xg_cache_pool_destroy", "xg_cache_pool_set_limit", "xg_cache_pool_reserve", "xg_cache_pool_stats",
-    "xg_compile_grammar", "xg_grammar_destroy", "xg_grammar_get_tables", "xg_grammar_get_rule_hashes", "xg_grammar_get_cache_entry", "xg_grammar_get_state_classes", "xg_grammar_stats", "xg_jit_service",
+    "xg_compile_grammar", "xg_grammar_destroy", "xg_grammar_get_tables", "xg_grammar_get_rule_hashes", "xg_grammar_get_cache_entry", "xg_grammar_record_of", "xg_grammar_get_state_classes", "xg_grammar_stats", "xg_jit_service",
     "xg_matcher_create", "xg_matcher_reset", "xg_matcher_destroy", "xg_matcher_is_terminated", "xg_matcher_next_fill_work",
     "xg_fill_next_token_bitmask", "xg_fill_next_token_bitmask_static", "xg_apply_token_bitmask", "xg_accept_token",
     "xg_accept_token_ex", "xg_accept_token_and_fill_next_bitmask", "xg_fill_and_apply_token_bitmask",
@@ -43,7 +43,7 @@ class XgError(RuntimeError):
 class CompileOptions(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("inline_max_states", C.c_int32), ("max_rule_states", C.c_int32), ("build_cache", C.c_int32),
                 ("no_state_compression", C.c_int32), ("jit", C.c_int32), ("jit_precompute", C.c_int32), ("jit_arena_bytes", C.c_int64),
-                ("count_node_visits", C.c_int32), ("reserved", C.c_int32)]
+                ("count_node_visits", C.c_int32), ("repeat_threshold", C.c_int32), ("repeat_depth", C.c_int32), ("reserved", C.c_int32)]
 
 
 class FillWork(C.Structure):
@@ -66,7 +66,8 @@ class PoolStats(C.Structure):
 class GrammarTables(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_rules", "n_states", "n_classes", "n_class_edges", "n_ref_edges", "root_rule", "root_nullable")] + \
                [(n, C.c_void_p) for n in ("rule_start", "state_rule", "state_final", "cedge_begin", "cedge_class", "cedge_target",
-                                          "redge_begin", "redge_rule", "redge_target", "class_bits")]
+                                          "redge_begin", "redge_rule", "redge_target", "class_bits",
+                                          "rule_rep_lo", "rule_rep_hi", "cedge_iter", "redge_iter")] + [("n_records", C.c_int32)]
 
 
 class CacheEntryView(C.Structure):
@@ -120,6 +121,7 @@ def lib():
         L.xg_grammar_get_rule_hashes.argtypes = [vp, vp]
         L.xg_grammar_get_cache_entry.argtypes = [vp, i32, C.POINTER(CacheEntryView)]
         L.xg_grammar_get_state_classes.argtypes = [vp, i32, vp]
+        L.xg_grammar_record_of.argtypes = [vp, i32, i32, C.POINTER(C.c_int32)]
         L.xg_jit_service.argtypes = [vp, i32, vp, i32, C.POINTER(JitStats)]
         L.xg_grammar_stats.argtypes = [vp, C.POINTER(GrammarStats)]
         L.xg_matcher_create.argtypes = [vp, C.POINTER(MatcherOptions), vp, C.POINTER(vp)]
@@ -190,11 +192,12 @@ class CachePool:
 class Grammar:
     def __init__(self, tokenizer: Optional[Tokenizer], kind, text: str, pool: Optional[CachePool] = None, root: Optional[str] = None,
                  inline_max_states: int = -1, build_cache: bool = True, stream: int = 0, state_compression: bool = True,
-                 jit: bool = False, jit_precompute: int = 0, jit_arena_bytes: int = 0, count_node_visits: bool = False):
+                 jit: bool = False, jit_precompute: int = 0, jit_arena_bytes: int = 0, count_node_visits: bool = False,
+                 repeat_threshold: int = 0, repeat_depth: int = 0):
         kind = KIND_BY_NAME.get(kind, kind)
         raw = text.encode("utf-8") if isinstance(text, str) else text
         opt = CompileOptions(C.sizeof(CompileOptions), inline_max_states, 0, 1 if build_cache else 0, 0 if state_compression else 1,
-                             1 if jit else 0, int(jit_precompute), int(jit_arena_bytes), 1 if count_node_visits else 0, 0)
+                             1 if jit else 0, int(jit_precompute), int(jit_arena_bytes), 1 if count_node_visits else 0, int(repeat_threshold), int(repeat_depth), 0)
         h = C.c_void_p()
         _check(lib().xg_compile_grammar(tokenizer.h if tokenizer else None, pool.h if pool else None, kind, raw, len(raw),
                                         root.encode() if root else None, C.byref(opt), stream, C.byref(h)))
@@ -222,7 +225,17 @@ class Grammar:
             cedge_begin=arr(t.cedge_begin, t.n_states + 1, np.int32), cedge_class=arr(t.cedge_class, t.n_class_edges, np.int32),
             cedge_target=arr(t.cedge_target, t.n_class_edges, np.int32),
             redge_begin=arr(t.redge_begin, t.n_states + 1, np.int32), redge_rule=arr(t.redge_rule, t.n_ref_edges, np.int32),
-            redge_target=arr(t.redge_target, t.n_ref_edges, np.int32), class_bits=arr(t.class_bits, t.n_classes * 8, np.uint32))
+            redge_target=arr(t.redge_target, t.n_ref_edges, np.int32), class_bits=arr(t.class_bits, t.n_classes * 8, np.uint32),
+            # counted repetitions (empty arrays when the grammar has none)
+            rule_rep_lo=arr(t.rule_rep_lo, t.n_rules, np.int32), rule_rep_hi=arr(t.rule_rep_hi, t.n_rules, np.int32),
+            cedge_iter=arr(t.cedge_iter, t.n_class_edges, np.uint8), redge_iter=arr(t.redge_iter, t.n_ref_edges, np.uint8),
+            n_records=t.n_records)
+
+    def record_of(self, state: int, count: int = 0) -> int:
+        """The cache record of (state, count of finished iterations); the state itself outside counted repetitions."""
+        out = C.c_int32()
+        _check(lib().xg_grammar_record_of(self.h, int(state), int(count), C.byref(out)))
+        return out.value
 
     def rule_hashes(self) -> np.ndarray:
         s = GrammarStats()

@@ -86,6 +86,7 @@ double now_ms() {
 // asynchronous copy from the entry's own pinned staging buffer on the caller's stream.  After the tables have grown
 // to the largest batch in use there is no allocation, no device-wide synchronisation and no blocking copy.
 constexpr int kBatchEntries = 64;
+constexpr int kDefaultRepeatThreshold = 64;   // bounded repetitions of at least this many iterations are counted, not expanded
 struct BatchSlot {
   std::vector<xg_matcher_t*> key;
   MatcherDev** dev_matchers = nullptr;   // [cap], inside the tokenizer's slab
@@ -163,7 +164,10 @@ struct JitState {                         // per grammar
 struct xg_grammar {
   const xg_tokenizer* tok = nullptr;
   std::shared_ptr<CachePool> pool;
-  FlatGrammar flat;
+  FlatGrammar flat;                     // what the device runs on: with counted repetitions, one state record per class of counts
+  FlatGrammar base;                     // the automata as the front end made them (only kept when they differ from `flat`)
+  bool counted = false;                 // the grammar has counted repetitions (Section 3.6): `base` is set
+  const FlatGrammar& tables() const { return counted ? base : flat; }
   std::vector<EntryDev> entries;        // [n_states], host copy of the device headers
   std::vector<int2> entry_counts;       // [n_states] (accepted, uncertain)
   GrammarDev host_view{};               // device pointers
@@ -387,6 +391,9 @@ static xg_status_t upload_grammar(xg_grammar* g, cudaStream_t stream) {
     r.edge0_class = n_scan ? scan[f.scan_begin[s]].x : 0; r.edge0_target = n_scan ? scan[f.scan_begin[s]].y : 0;
   }
   const std::vector<uint32_t>& state_first = f.state_first;
+  std::vector<int4> rep_state(f.rep_rec_base.size());
+  for (size_t i = 0; i < rep_state.size(); ++i) rep_state[i] = make_int4(f.rep_rec_base[i], f.rep_lo[i], f.rep_hi[i], 0);
+  size_t o_rep = reserve(rep_state.size() * sizeof(int4)), o_word = reserve(f.rec_word.size() * 4);
   size_t o_first = reserve(state_first.size() * 4), o_follow = reserve(f.rule_follow.size() * 4);
   size_t o_rec = reserve(recs.size() * sizeof(StateRec)), o_scan = reserve(scan.size() * sizeof(uint2)), o_wait = reserve(wait.size() * sizeof(uint2)),
          o_gs = reserve(f.gather_state.size() * 4), o_cb = reserve(f.class_bits.size() * 4),
@@ -395,6 +402,8 @@ static xg_status_t upload_grammar(xg_grammar* g, cudaStream_t stream) {
   if (!host) return set_error(XG_ERR_OOM, "pinned staging allocation failed");
   std::memset(host, 0, total);
   auto put = [&](size_t at, const void* src, size_t bytes) { if (bytes) std::memcpy(host + at, src, bytes); };
+  put(o_rep, rep_state.data(), rep_state.size() * sizeof(int4));
+  put(o_word, f.rec_word.data(), f.rec_word.size() * 4);
   put(o_first, state_first.data(), state_first.size() * 4);
   put(o_follow, f.rule_follow.data(), f.rule_follow.size() * 4);
   put(o_rec, recs.data(), recs.size() * sizeof(StateRec));
@@ -422,6 +431,10 @@ static xg_status_t upload_grammar(xg_grammar* g, cudaStream_t stream) {
   g->entries_offset = o_en;
   v.miss_ring = g->jit.slot >= 0 ? ((JitPool*)g->pool->jit_host)->d_ring : nullptr;
   v.jit_slot = g->jit.slot;
+  v.rep_first = f.rep_first; v.rep_shift = f.rep_shift; v.rep_depth = f.rep_depth;
+  v.n_words_states = f.rep_rec_base.empty() ? f.n_states : f.n_base_states;
+  v.rep_state = rep_state.empty() ? nullptr : (const int4*)(d + o_rep);
+  v.rec_word = f.rec_word.empty() ? nullptr : (const uint32_t*)(d + o_word);
   v.n_scan_edges = (int32_t)scan.size(); v.n_wait_edges = (int32_t)wait.size(); v.n_gather = (int32_t)f.gather_state.size();
   put(o_self, &v, sizeof(GrammarDev));
   g->dev = (GrammarDev*)(d + o_self);
@@ -954,7 +967,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   if (!text) return set_error(XG_ERR_INVALID_ARG, "text is NULL");
   FrontendOptions fo;
   bool build_cache = tok != nullptr, compress = true, jit = false, count_visits = false;
-  int jit_precompute = 0;
+  int jit_precompute = 0, repeat_threshold = 0, repeat_depth = 0;
   long long jit_arena_words = 0;
   if (opt) {
     if (opt->struct_size < 8) return set_error(XG_ERR_INVALID_ARG, "bad options struct_size");
@@ -965,13 +978,21 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
     if (opt->struct_size >= 28 && opt->jit != 0) { jit = true; jit_precompute = std::max(0, opt->jit_precompute); }
     if (opt->struct_size >= 40 && opt->jit_arena_bytes > 0) jit_arena_words = std::max<long long>(1024, opt->jit_arena_bytes / 4);
     if (opt->struct_size >= 44 && opt->count_node_visits != 0) count_visits = true;
+    if (opt->struct_size >= 48) repeat_threshold = opt->repeat_threshold;
+    if (opt->struct_size >= 52 && opt->repeat_depth > 0) repeat_depth = opt->repeat_depth;
   }
+  // counted repetitions (Section 3.6): on by default wherever the longest token is known
+  if (tok && tok->dev.max_len > 0) repeat_depth = tok->dev.max_len;
+  if (repeat_threshold == 0) repeat_threshold = kDefaultRepeatThreshold;
+  if (repeat_threshold > 0 && repeat_depth > 0) { fo.repeat_threshold = repeat_threshold; fo.repeat_depth = repeat_depth; }
   if (pool && pool->impl->owner() != (const void*)tok) return set_error(XG_ERR_INVALID_ARG, "the pool belongs to another tokenizer");
   std::unique_ptr<xg_grammar> g(new xg_grammar());
   g->count_visits = count_visits;
   const double t0 = now_ms();
   try {
-    g->flat = compile_frontend((int)kind, std::string(text, len), root_rule ? root_rule : "root", fo);
+    FlatGrammar made = compile_frontend((int)kind, std::string(text, len), root_rule ? root_rule : "root", fo);
+    if (made.rule_rep_lo.empty()) g->flat = std::move(made);
+    else { g->flat = expand_counted_rules(made); g->base = std::move(made); g->counted = true; }
   } catch (const FrontendError& e) {
     return set_error(e.status, e.message);
   } catch (const std::bad_alloc&) {
@@ -981,7 +1002,7 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   }
   const FlatGrammar& f = g->flat;
   g->stats.frontend_ms = now_ms() - t0;
-  g->stats.n_rules = f.n_rules; g->stats.n_states = f.n_states; g->stats.n_classes = f.n_classes;
+  g->stats.n_rules = f.n_rules; g->stats.n_states = g->tables().n_states; g->stats.n_classes = f.n_classes;
   std::vector<int32_t> scannable;
   for (int s = 0; s < f.n_states; ++s) if (f.cedge_begin[s + 1] > f.cedge_begin[s]) scannable.push_back(s);
   g->stats.n_scannable = (int)scannable.size();
@@ -1209,7 +1230,12 @@ void xg_grammar_destroy(xg_grammar_t* g) {
 
 xg_status_t xg_grammar_get_tables(const xg_grammar_t* g, xg_grammar_tables_t* t) {
   if (!g || !t) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
-  const FlatGrammar& f = g->flat;
+  const FlatGrammar& f = g->tables();
+  t->rule_rep_lo = f.rule_rep_lo.empty() ? nullptr : f.rule_rep_lo.data();
+  t->rule_rep_hi = f.rule_rep_hi.empty() ? nullptr : f.rule_rep_hi.data();
+  t->cedge_iter = f.cedge_iter.empty() ? nullptr : f.cedge_iter.data();
+  t->redge_iter = f.redge_iter.empty() ? nullptr : f.redge_iter.data();
+  t->n_records = g->flat.n_states;
   t->n_rules = f.n_rules; t->n_states = f.n_states; t->n_classes = f.n_classes;
   t->n_class_edges = (int32_t)f.cedge_class.size(); t->n_ref_edges = (int32_t)f.redge_rule.size();
   t->root_rule = f.root_rule; t->root_nullable = f.root_nullable;
@@ -1217,6 +1243,16 @@ xg_status_t xg_grammar_get_tables(const xg_grammar_t* g, xg_grammar_tables_t* t)
   t->cedge_begin = f.cedge_begin.data(); t->cedge_class = f.cedge_class.data(); t->cedge_target = f.cedge_target.data();
   t->redge_begin = f.redge_begin.data(); t->redge_rule = f.redge_rule.data(); t->redge_target = f.redge_target.data();
   t->class_bits = f.class_bits.data();
+  return XG_OK;
+}
+
+xg_status_t xg_grammar_record_of(const xg_grammar_t* g, int32_t state, int32_t count, int32_t* record) {
+  if (!g || !record) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
+  const FlatGrammar& f = g->tables();
+  if (state < 0 || state >= f.n_states || count < 0) return set_error(XG_ERR_INVALID_ARG, "state or count out of range");
+  if (!g->counted || state < g->flat.rep_first) { *record = state; return XG_OK; }
+  if (count >= f.rule_rep_hi[f.state_rule[state]]) return set_error(XG_ERR_INVALID_ARG, "count beyond the repetition's upper bound");
+  *record = record_of(g->flat, state, count);
   return XG_OK;
 }
 
@@ -1233,6 +1269,7 @@ xg_status_t xg_grammar_get_rule_hashes(const xg_grammar_t* g, uint64_t* out) {
 
 xg_status_t xg_grammar_get_state_classes(const xg_grammar_t* g, int32_t depth, int32_t* out) {
   if (!g || !out) return set_error(XG_ERR_INVALID_ARG, "NULL argument");
+  if (g->counted) return set_error(XG_ERR_UNSUPPORTED, "the grammar has counted repetitions: its records are the classes");
   if (depth < 0) {
     if (!g->tok) return set_error(XG_ERR_INVALID_ARG, "depth < 0 needs a grammar compiled with a tokenizer");
     depth = g->tok->dev.max_len;

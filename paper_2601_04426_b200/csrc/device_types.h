@@ -104,6 +104,16 @@ struct GrammarDev {
   JitRing* miss_ring;             // just-in-time grammars only (else nullptr)
   int32_t jit_slot;               // this grammar's number in the ring's reports
   int32_t n_scan_edges, n_wait_edges, n_gather;      // table sizes (for the bounds-checking build)
+  // Counted repetitions (Section 3.6: the parser state (R{l,r}, k)).  An item's state word is state | k << rep_shift;
+  // words below rep_first are ordinary states (k = 0) and index the tables directly.  A state q >= rep_first belongs
+  // to a counted rule and has one record (tables, cache entry) per class of counts:
+  //   rep_state[q - rep_first] = (first record, lo, hi, -),  record = first + dl * (rep_depth + 1) + dr,
+  //   dl = min(max(lo - k - 1, 0), rep_depth), dr = min(hi - k - 1, rep_depth).
+  // Edge targets inside such a rule carry kRel (keep the count) and kIter (one more).  rec_word[record] is a state
+  // word of the record's class (the item a cache entry is classified from).  No counted rule: rep_first = INT32_MAX.
+  int32_t rep_first, rep_shift, rep_depth, n_words_states;     // n_words_states: states before the records were written out
+  const int4* rep_state;
+  const uint32_t* rec_word;
 };
 
 // What the next mask needs from the current Earley set, worked out once when the set is made
@@ -156,5 +166,6 @@ struct MatcherDev {
 constexpr int kSlowQueue = 1024;
 
 constexpr uint32_t kSelf = 0x80000000u;
+constexpr uint32_t kRel = 0x40000000u, kIter = 0x20000000u, kTarget = 0x1FFFFFFFu;
 
 }  // namespace xg

@@ -334,6 +334,7 @@ struct Edge {
   int rule;        // kRef
   int to;
   ByteSet set;     // kBytes
+  bool iter = false;   // inside a counted repetition: the edge starts the next iteration
 };
 struct Fsm {
   std::vector<std::vector<Edge>> out;
@@ -412,11 +413,28 @@ struct AhoCorasick {
 
 constexpr int kKeepDispatchedRules = 8;
 
+// A counted repetition (Section 3.6): rule `rep` stands for body{lo,hi}.  Until the tables are written its automaton
+// is a single reference to `body`, so that nullability, trimming and the reference graph see it as an ordinary rule.
+struct CountedRule {
+  int body = -1, lo = 0, hi = 0;
+};
+
 struct Builder {
   std::set<int> keep_as_rule;             // rules that inlining leaves alone
   std::vector<std::string> names;
   std::map<std::string, int> ids;
   std::vector<Fsm> rules;
+  int repeat_threshold = 0;               // bounded repetitions with at least this many iterations become counted rules (0: never)
+  std::map<int, CountedRule> counted;     // rule id -> what it repeats
+  std::map<int, Fsm> pending;             // automata of the rules made while another rule is being built (appended afterwards)
+
+  int new_rule(const std::string& name) {
+    const int id = (int)names.size();
+    names.push_back(name);
+    ids[name] = id;
+    keep_as_rule.insert(id);
+    return id;
+  }
 
   int lookup(const std::string& n) const {
     auto it = ids.find(n);
@@ -460,6 +478,27 @@ struct Builder {
         return {s, t};
       }
       case Expr::kRepeat: {
+        if (repeat_threshold > 0 && e.hi >= repeat_threshold) {
+          // X{lo,hi} as a rule of its own with a counter in its items: one copy of X whatever the bounds
+          const std::string tag = "%rep" + std::to_string(names.size());
+          const int body = new_rule(tag + ".body"), rep = new_rule(tag);
+          {
+            Fsm bf;
+            auto p = frag(bf, *e.kids[0]);
+            bf.start = p.first; bf.fin[p.second] = 1;
+            pending[body] = std::move(bf);
+          }
+          Fsm rf;
+          const int a = rf.add(), z = rf.add();
+          rf.ref(a, body, z);
+          rf.start = a; rf.fin[z] = 1;
+          if (e.lo == 0) rf.fin[a] = 1;
+          pending[rep] = std::move(rf);
+          counted[rep] = {body, e.lo, e.hi};
+          int s = f.add(), t = f.add();
+          f.ref(s, rep, t);
+          return {s, t};
+        }
         int s = f.add(), cur = s;
         for (int i = 0; i < e.lo; ++i) { auto p = frag(f, *e.kids[0]); f.eps(cur, p.first); cur = p.second; }
         int t = f.add();
@@ -856,6 +895,9 @@ struct Compiler {
   void remove_nullability() {
     std::vector<char> nullable = nullable_rules();
     root_nullable = nullable[root];
+    // a counted rule loses the empty string like every other rule (its users get the bypass below); with a body
+    // that derives the empty string, body{lo,hi} is (body minus empty){0,hi}
+    for (auto& kv : b.counted) kv.second.lo = nullable[kv.second.body] ? 1 : std::max(kv.second.lo, 1);
     for (Fsm& f : b.rules)
       for (int s = 0; s < f.size(); ++s) {
         size_t n = f.out[s].size();
@@ -954,7 +996,7 @@ struct Compiler {
         std::vector<Edge> keep;
         const std::vector<Edge> edges = g.out[s];     // g.out may reallocate while copies are appended
         for (const Edge& e : edges) {
-          bool take = e.kind == Edge::kRef && e.rule != r && candidate[e.rule] &&
+          bool take = e.kind == Edge::kRef && e.rule != r && candidate[e.rule] && !b.counted.count(r) &&
                       (b.rules[e.rule].size() <= opt.inline_max_states || uses[e.rule] == 1 ||
                        b.rules[e.rule].size() * uses[e.rule] <= 16 * opt.inline_max_states) &&
                       g.size() + b.rules[e.rule].size() <= opt.max_rule_states;
@@ -988,27 +1030,57 @@ struct Compiler {
     for (int r = 0; r < R; ++r) process(r);
   }
 
+  // the automaton a counted rule runs on: its body's, and at every accepting state copies of the start state's
+  // edges that begin the next iteration
+  Fsm counted_automaton(const CountedRule& c) const {
+    Fsm f = b.rules[c.body];
+    const std::vector<Edge> first = f.out[f.start];
+    for (int s = 0; s < f.size(); ++s)
+      if (f.fin[s]) for (Edge e : first) { e.iter = true; f.out[s].push_back(e); }
+    return f;
+  }
+
   FlatGrammar flatten() {
     int R = n_rules();
-    // keep only rules reachable from the root
+    std::map<int, Fsm> counted_fsm;
+    auto fsm_of = [&](int r) -> const Fsm& {
+      auto c = b.counted.find(r);
+      if (c == b.counted.end()) return b.rules[r];
+      auto it = counted_fsm.find(r);
+      if (it == counted_fsm.end()) it = counted_fsm.emplace(r, counted_automaton(c->second)).first;
+      return it->second;
+    };
+    // keep only rules reachable from the root; counted rules go last, so that their states are the top of the
+    // state numbering (an item's state word below FlatGrammar::rep_first needs no decoding)
     std::vector<int> new_id(R, -1), order;
     order.push_back(root); new_id[root] = 0;
     for (size_t q = 0; q < order.size(); ++q)
-      for (auto& es : b.rules[order[q]].out)
+      for (auto& es : fsm_of(order[q]).out)
         for (const Edge& e : es) if (e.kind == Edge::kRef && new_id[e.rule] < 0) { new_id[e.rule] = (int)order.size(); order.push_back(e.rule); }
+    std::stable_partition(order.begin() + 1, order.end(), [&](int r) { return !b.counted.count(r); });
+    for (size_t k = 0; k < order.size(); ++k) new_id[order[k]] = (int)k;
+    bool any_counted = false;
+    for (int r : order) any_counted = any_counted || b.counted.count(r);
     FlatGrammar g;
     g.n_rules = (int)order.size();
     g.root_rule = 0;
     g.root_nullable = root_nullable ? 1 : 0;
     std::map<ByteSet, int> class_id;
     std::vector<int> base(g.n_rules);
-    for (int k = 0; k < g.n_rules; ++k) { base[k] = g.n_states; g.n_states += b.rules[order[k]].size(); }
+    for (int k = 0; k < g.n_rules; ++k) { base[k] = g.n_states; g.n_states += fsm_of(order[k]).size(); }
+    g.n_base_states = g.n_states;
     g.cedge_begin.push_back(0); g.redge_begin.push_back(0);
+    if (any_counted) { g.rule_rep_lo.assign(g.n_rules, 0); g.rule_rep_hi.assign(g.n_rules, 0); g.rep_depth = opt.repeat_depth; }
     for (int k = 0; k < g.n_rules; ++k) {
-      const Fsm& f = b.rules[order[k]];
+      const Fsm& f = fsm_of(order[k]);
       g.rule_names.push_back(b.names[order[k]]);
       g.rule_start.push_back(base[k] + f.start);
       g.rule_kind.push_back(f.has_tag_dispatch ? 1 : 0);
+      auto c = b.counted.find(order[k]);
+      if (c != b.counted.end()) {
+        g.rule_rep_lo[k] = c->second.lo; g.rule_rep_hi[k] = c->second.hi;
+        if (g.rep_first == 0x7FFFFFFF) g.rep_first = base[k];
+      }
       for (int s = 0; s < f.size(); ++s) {
         g.state_rule.push_back(k);
         g.state_final.push_back(f.fin[s] ? 1 : 0);
@@ -1021,9 +1093,11 @@ struct Compiler {
             }
             g.cedge_class.push_back(it->second);
             g.cedge_target.push_back(base[k] + e.to);
+            if (any_counted) g.cedge_iter.push_back(e.iter ? 1 : 0);
           } else if (e.kind == Edge::kRef) {
             g.redge_rule.push_back(new_id[e.rule]);
             g.redge_target.push_back(base[k] + e.to);
+            if (any_counted) g.redge_iter.push_back(e.iter ? 1 : 0);
           }
         }
         g.cedge_begin.push_back((int)g.cedge_class.size());
@@ -1052,6 +1126,11 @@ struct Compiler {
     }
     g.scan_begin.assign(1, 0); g.wait_begin.assign(1, 0); g.gather_begin.assign(1, 0);
     g.scan_own_end.clear();
+    g.scan_class.clear(); g.scan_target.clear(); g.wait_rule.clear(); g.wait_target.clear(); g.gather_state.clear();
+    // what the device follows along an edge: the target state, or in the device view of a grammar with counted
+    // repetitions the packed word (an edge copied from a predicted start state begins at count 0: no count flags)
+    auto cword = [&](int e) { return g.cedge_word.empty() ? (uint32_t)g.cedge_target[e] : g.cedge_word[e]; };
+    auto rword = [&](int e) { return g.redge_word.empty() ? (uint32_t)g.redge_target[e] : g.redge_word[e]; };
     std::vector<int> predicted;
     std::vector<char> mark(R, 0);
     for (int s = 0; s < S; ++s) {
@@ -1060,14 +1139,14 @@ struct Compiler {
         for (int r : closure[g.redge_rule[e]]) if (!mark[r]) { mark[r] = 1; predicted.push_back(r); }
       std::sort(predicted.begin(), predicted.end());
       for (int r : predicted) mark[r] = 0;
-      for (int e = g.cedge_begin[s]; e < g.cedge_begin[s + 1]; ++e) { g.scan_class.push_back(g.cedge_class[e]); g.scan_target.push_back(g.cedge_target[e]); }
+      for (int e = g.cedge_begin[s]; e < g.cedge_begin[s + 1]; ++e) { g.scan_class.push_back(g.cedge_class[e]); g.scan_target.push_back(cword(e)); }
       g.scan_own_end.push_back((int)g.scan_class.size());
-      for (int e = g.redge_begin[s]; e < g.redge_begin[s + 1]; ++e) { g.wait_rule.push_back(g.redge_rule[e]); g.wait_target.push_back(g.redge_target[e]); }
+      for (int e = g.redge_begin[s]; e < g.redge_begin[s + 1]; ++e) { g.wait_rule.push_back(g.redge_rule[e]); g.wait_target.push_back(rword(e)); }
       if (g.cedge_begin[s + 1] > g.cedge_begin[s]) g.gather_state.push_back(s);
       for (int r : predicted) {
         int s0 = g.rule_start[r];
-        for (int e = g.cedge_begin[s0]; e < g.cedge_begin[s0 + 1]; ++e) { g.scan_class.push_back(g.cedge_class[e]); g.scan_target.push_back((uint32_t)g.cedge_target[e] | kSelfBit); }
-        for (int e = g.redge_begin[s0]; e < g.redge_begin[s0 + 1]; ++e) { g.wait_rule.push_back(g.redge_rule[e]); g.wait_target.push_back((uint32_t)g.redge_target[e] | kSelfBit); }
+        for (int e = g.cedge_begin[s0]; e < g.cedge_begin[s0 + 1]; ++e) { g.scan_class.push_back(g.cedge_class[e]); g.scan_target.push_back((cword(e) & kTargetMask) | kSelfBit); }
+        for (int e = g.redge_begin[s0]; e < g.redge_begin[s0 + 1]; ++e) { g.wait_rule.push_back(g.redge_rule[e]); g.wait_target.push_back((rword(e) & kTargetMask) | kSelfBit); }
         if (g.cedge_begin[s0 + 1] > g.cedge_begin[s0]) g.gather_state.push_back((int32_t)((uint32_t)s0 | kSelfBit));
       }
       g.scan_begin.push_back((int)g.scan_class.size());
@@ -1414,6 +1493,8 @@ FlatGrammar compile_frontend(int kind, const std::string& text, const std::strin
   std::string root_name = (kind == kEbnf && !root.empty()) ? root : "root";
   c.root = c.b.lookup(root_name);
   c.b.max_states = opt.max_rule_states;
+  if (opt.repeat_threshold > 0 && opt.repeat_depth <= 0) fail(XG_ERR_INVALID_ARG, "counted repetitions need the longest token's length");
+  c.b.repeat_threshold = opt.repeat_threshold;
   for (auto& r : parsed) {
     Fsm f;
     auto p = c.b.frag(f, *r.second);
@@ -1422,6 +1503,11 @@ FlatGrammar compile_frontend(int kind, const std::string& text, const std::strin
     if (f.size() > opt.max_rule_states) fail(XG_ERR_CAPACITY, "rule " + r.first + " exceeds max_rule_states");
     c.b.rules.push_back(std::move(f));
   }
+  for (auto& kv : c.b.pending) {              // the rules behind counted repetitions, in the order of their ids
+    if (kv.first != c.n_rules()) fail(XG_ERR_INVALID_ARG, "internal: rule numbering");
+    c.b.rules.push_back(std::move(kv.second));
+  }
+  c.b.pending.clear();
   c.remove_nullability();
   for (Fsm& f : c.b.rules) f = normalize(f, opt.max_rule_states);
   std::vector<char> stale = c.trim(), renormalized;           // stale: trimmed since it was last minimised
@@ -1430,6 +1516,103 @@ FlatGrammar compile_frontend(int kind, const std::string& text, const std::strin
   for (int r = 0; r < c.n_rules(); ++r)
     if (trimmed_again[r] || (stale[r] && !renormalized[r])) c.b.rules[r] = canonical_order(minimize(c.b.rules[r]));
   return c.flatten();
+}
+
+// ------------------------------------------------------------------------------------------
+// Counted repetitions on the device (Section 3.6).  An item of X{lo,hi} is (state of X, origin, k).  How a token of
+// at most L bytes behaves from it depends on k only through how far k + 1 is from the two bounds, and only up to L
+// iterations away (every iteration consumes a byte), so the states are written out once per class
+//   (dl, dr) = (min(max(lo - k - 1, 0), D), min(hi - k - 1, D)),   D = L + 1:
+// the record is accepting iff X's state is and dl = 0, it has the iteration edges iff dr > 0, and its cache entry
+// is exact for every count of the class.  The number of records depends on D, not on the bounds.
+// ------------------------------------------------------------------------------------------
+namespace {
+struct CountClass { int dl, dr; };
+CountClass count_class(int lo, int hi, int D, int k) {
+  const int done = k + 1;
+  return {std::min(std::max(lo - done, 0), D), std::min(hi - done, D)};
+}
+// the largest count of class (dl, dr), or -1 when no count in [0, hi) falls into it
+int class_largest_count(int lo, int hi, int D, int dl, int dr) {
+  int done_min = 1, done_max = hi;
+  if (dl == D) done_max = std::min(done_max, lo - D);
+  else if (dl == 0) done_min = std::max(done_min, lo);
+  else { done_min = std::max(done_min, lo - dl); done_max = std::min(done_max, lo - dl); }
+  if (dr == D) done_max = std::min(done_max, hi - D);
+  else { done_min = std::max(done_min, hi - dr); done_max = std::min(done_max, hi - dr); }
+  return done_min <= done_max ? done_max - 1 : -1;
+}
+}  // namespace
+
+int32_t record_of(const FlatGrammar& r, int32_t q, int32_t k) {
+  if (q < r.rep_first) return q;
+  const int i = q - r.rep_first, D = r.rep_depth;
+  const CountClass c = count_class(r.rep_lo[i], r.rep_hi[i], D, k);
+  return r.rep_rec_base[i] + c.dl * (D + 1) + c.dr;
+}
+
+FlatGrammar expand_counted_rules(const FlatGrammar& g) {
+  if (g.rule_rep_lo.empty()) return g;
+  const int D = g.rep_depth, per = (D + 1) * (D + 1);
+  const int n_rep = g.n_base_states - g.rep_first;
+  FlatGrammar r;
+  r.n_rules = g.n_rules; r.n_classes = g.n_classes; r.root_rule = g.root_rule; r.root_nullable = g.root_nullable;
+  r.rule_names = g.rule_names; r.rule_kind = g.rule_kind; r.class_bits = g.class_bits;
+  r.rule_rep_lo = g.rule_rep_lo; r.rule_rep_hi = g.rule_rep_hi;
+  r.rep_first = g.rep_first; r.rep_depth = D; r.n_base_states = g.n_base_states;
+  r.rep_shift = 1;
+  while ((1ll << r.rep_shift) < g.n_base_states) ++r.rep_shift;
+  int hi_max = 0;
+  for (int x : g.rule_rep_hi) hi_max = std::max(hi_max, x);
+  if (r.rep_shift > 28 || (long long)hi_max >= (1ll << (32 - r.rep_shift))) fail(XG_ERR_CAPACITY, "a repetition bound does not fit the item's count field");
+  const long long n_states = (long long)g.rep_first + (long long)n_rep * per;
+  if (n_states > (long long)kTargetMask) fail(XG_ERR_CAPACITY, "too many state records");
+  r.n_states = (int)n_states;
+  r.rep_rec_base.resize(n_rep); r.rep_lo.resize(n_rep); r.rep_hi.resize(n_rep);
+  for (int i = 0; i < n_rep; ++i) {
+    const int rule = g.state_rule[g.rep_first + i];
+    r.rep_rec_base[i] = g.rep_first + i * per; r.rep_lo[i] = g.rule_rep_lo[rule]; r.rep_hi[i] = g.rule_rep_hi[rule];
+  }
+  r.cedge_begin.push_back(0); r.redge_begin.push_back(0);
+  r.rec_word.reserve(r.n_states);
+  for (int s = 0; s < g.rep_first; ++s) {           // ordinary states: as they are
+    r.state_rule.push_back(g.state_rule[s]); r.state_final.push_back(g.state_final[s]); r.rec_word.push_back((uint32_t)s);
+    for (int e = g.cedge_begin[s]; e < g.cedge_begin[s + 1]; ++e) { r.cedge_class.push_back(g.cedge_class[e]); r.cedge_target.push_back(record_of(r, g.cedge_target[e], 0)); r.cedge_word.push_back((uint32_t)g.cedge_target[e]); }
+    for (int e = g.redge_begin[s]; e < g.redge_begin[s + 1]; ++e) { r.redge_rule.push_back(g.redge_rule[e]); r.redge_target.push_back(record_of(r, g.redge_target[e], 0)); r.redge_word.push_back((uint32_t)g.redge_target[e]); }
+    r.cedge_begin.push_back((int)r.cedge_class.size()); r.redge_begin.push_back((int)r.redge_rule.size());
+  }
+  for (int i = 0; i < n_rep; ++i) {
+    const int q = g.rep_first + i, lo = r.rep_lo[i], hi = r.rep_hi[i];
+    for (int dl = 0; dl <= D; ++dl)
+      for (int dr = 0; dr <= D; ++dr) {
+        const int k = class_largest_count(lo, hi, D, dl, dr);
+        r.state_rule.push_back(g.state_rule[q]);
+        r.state_final.push_back(k >= 0 && g.state_final[q] && dl == 0 ? 1 : 0);
+        r.rec_word.push_back((uint32_t)q | (k >= 0 ? (uint32_t)k << r.rep_shift : 0u));
+        if (k >= 0) {
+          for (int e = g.cedge_begin[q]; e < g.cedge_begin[q + 1]; ++e) {
+            const bool iter = g.cedge_iter[e] != 0;
+            if (iter && dr == 0) continue;
+            r.cedge_class.push_back(g.cedge_class[e]);
+            r.cedge_target.push_back(record_of(r, g.cedge_target[e], iter ? k + 1 : k));
+            r.cedge_word.push_back((uint32_t)g.cedge_target[e] | kRelBit | (iter ? kIterBit : 0u));
+          }
+          for (int e = g.redge_begin[q]; e < g.redge_begin[q + 1]; ++e) {
+            const bool iter = g.redge_iter[e] != 0;
+            if (iter && dr == 0) continue;
+            r.redge_rule.push_back(g.redge_rule[e]);
+            r.redge_target.push_back(record_of(r, g.redge_target[e], iter ? k + 1 : k));
+            r.redge_word.push_back((uint32_t)g.redge_target[e] | kRelBit | (iter ? kIterBit : 0u));
+          }
+        }
+        r.cedge_begin.push_back((int)r.cedge_class.size()); r.redge_begin.push_back((int)r.redge_rule.size());
+      }
+  }
+  for (int rule = 0; rule < g.n_rules; ++rule) r.rule_start.push_back(record_of(r, g.rule_start[rule], 0));
+  Compiler::build_closure_lists(r);
+  // follow sets from the plain automata (every edge enabled, acceptance as in X): a superset for every count
+  r.rule_follow = g.rule_follow;
+  return r;
 }
 
 
@@ -1463,9 +1646,10 @@ std::vector<int32_t> bounded_equivalence(const FlatGrammar& g, int depth) {
   std::vector<int> block(S), count;
   {
     SignatureTable table;
-    std::vector<uint32_t> sig(2);
+    std::vector<uint32_t> sig(3);
     for (int s = 0; s < S; ++s) {
       sig[0] = (uint32_t)g.state_rule[s]; sig[1] = g.state_final[s];
+      sig[2] = s >= g.rep_first ? (uint32_t)s + 1 : 0u;        // the records of a counted rule are classes already
       block[s] = table.intern(sig);
       if (block[s] == (int)count.size()) count.push_back(0);
       ++count[block[s]];

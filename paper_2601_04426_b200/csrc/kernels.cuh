@@ -74,6 +74,27 @@ __device__ __forceinline__ Chart chart_of_history(const uint32_t* h_st, const in
 
 constexpr uint32_t kFullWarp = 0xFFFFFFFFu;
 
+// Counted repetitions (Section 3.6).  rec_of: the record (index into state[], state_first[], entries[]) of an item's
+// state word; ordinary states are their own record.
+__device__ __forceinline__ uint32_t rec_of(const GrammarDev& g, uint32_t w) {
+  if (w < (uint32_t)g.rep_first) return w;
+  const uint32_t q = w & ((1u << g.rep_shift) - 1u);
+  const int done = (int)(w >> g.rep_shift) + 1;
+  if (!XG_BOUND((int)q - g.rep_first, g.n_words_states - g.rep_first, kBoundState)) return 0;
+  const int4 rs = g.rep_state[q - (uint32_t)g.rep_first];
+  const int dl = min(max(rs.y - done, 0), g.rep_depth), dr = max(min(rs.z - done, g.rep_depth), 0);
+  return (uint32_t)(rs.x + dl * (g.rep_depth + 1) + dr);
+}
+// a state word that belongs to record `rec` (the record itself for ordinary states)
+__device__ __forceinline__ uint32_t word_of_record(const GrammarDev& g, int rec) { return g.rec_word ? g.rec_word[rec] : (uint32_t)rec; }
+// the state word an edge leads to from the item whose state word is `from`: the packed target, with the count of
+// `from` when the edge stays inside a counted rule (kRel), one more when it starts the next iteration (kIter)
+__device__ __forceinline__ uint32_t next_word(const GrammarDev& g, uint32_t from, uint32_t packed) {
+  uint32_t w = packed & kTarget;
+  if (packed & kRel) w += (from >> g.rep_shift << g.rep_shift) + ((packed & kIter) ? (1u << g.rep_shift) : 0u);
+  return w;
+}
+
 // lane -> the index of the first lane whose inclusive prefix exceeds p (the owner of flattened pair p); `n` lanes hold items
 __device__ __forceinline__ int owner_of_pair(int incl, int p, int n) {
   int own = 0;
@@ -115,8 +136,9 @@ __device__ __forceinline__ bool advance_waiters(const GrammarDev& g, const Chart
   for (int i = b; i < e; ++i) {
     const uint32_t s2 = src_st[i];
     const int32_t o2 = src_org[i];
-    if (!XG_BOUND(s2, g.n_states, kBoundState)) continue;
-    const uint4 rec = *reinterpret_cast<const uint4*>(&g.state[s2]);
+    const uint32_t r2 = rec_of(g, s2);
+    if (!XG_BOUND(r2, g.n_states, kBoundState)) continue;
+    const uint4 rec = *reinterpret_cast<const uint4*>(&g.state[r2]);
     const int wait_end = (int)rec.z + (int)(rec.w & 0xFFFFu);
     if (!XG_BOUND(wait_end, g.n_wait_edges + 1, kBoundWaitEdge)) continue;
     // four edges at a time: their loads are issued together, then compared (one at a time, each load would be
@@ -128,7 +150,7 @@ __device__ __forceinline__ bool advance_waiters(const GrammarDev& g, const Chart
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         if (we[u].x != rule) continue;
-        if (!add_item(st, org, start, cnt, cap, we[u].y & ~kSelf, (we[u].y & kSelf) ? o : o2)) return false;
+        if (!add_item(st, org, start, cnt, cap, next_word(g, s2, we[u].y), (we[u].y & kSelf) ? o : o2)) return false;
       }
     }
   }
@@ -154,12 +176,13 @@ __device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* c
     for (int i = cur_b; i < cur_e; ++i) {
       const uint32_t s = cur_st[i];
       const int32_t o = cur_org[i];
-      if (!XG_BOUND(s, g.n_states, kBoundState)) continue;
-      const uint4 ra = *reinterpret_cast<const uint4*>(&g.state[s]);
+      const uint32_t sr = rec_of(g, s);
+      if (!XG_BOUND(sr, g.n_states, kBoundState)) continue;
+      const uint4 ra = *reinterpret_cast<const uint4*>(&g.state[sr]);
       const int n_edges = (k == 0 && own_edges_first) ? (int)(ra.y & 0xFFFFu) : (int)(ra.y >> 16);
       if (n_edges == 0) continue;
       if (!XG_BOUND((int)ra.x + n_edges, g.n_scan_edges + 1, kBoundScanEdge)) continue;
-      const uint4 rb = *(reinterpret_cast<const uint4*>(&g.state[s]) + 1);
+      const uint4 rb = *(reinterpret_cast<const uint4*>(&g.state[sr]) + 1);
       // the first edge is inline in the record; the others are fetched four at a time (loads issued together, then tested)
       for (int e = 0; e < n_edges; e += 4) {
         uint2 se[4];
@@ -171,15 +194,16 @@ __device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* c
           if (e + u >= n_edges) break;
           if (!(se[u].x & kLiteral) && !XG_BOUND(se[u].x, g.n_classes, kBoundClass)) continue;
           const bool hit = (se[u].x & kLiteral) ? ((se[u].x & 0x1FFu) == byte) : ((class_bits[se[u].x * 8 + word] & bit) != 0);
-          if (hit && !add_item(st, org, start, cnt, cap, se[u].y & ~kSelf, (se[u].y & kSelf) ? self_idx : o)) { *flags |= kWalkOverflow; return k; }
+          if (hit && !add_item(st, org, start, cnt, cap, next_word(g, s, se[u].y), (se[u].y & kSelf) ? self_idx : o)) { *flags |= kWalkOverflow; return k; }
         }
       }
     }
     if (cnt == start) return k;
     // complete (cascades through the growing set)
     for (int q = start; q < cnt; ++q) {
-      if (!XG_BOUND(st[q], g.n_states, kBoundState)) continue;
-      const uint32_t info = g.state[st[q]].info;
+      const uint32_t qr = rec_of(g, st[q]);
+      if (!XG_BOUND(qr, g.n_states, kBoundState)) continue;
+      const uint32_t info = g.state[qr].info;
       if (!(info >> 31)) continue;
       const int32_t o = org[q];
       if (o < 0) {
@@ -239,7 +263,7 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
     }
     sh_first[threadIdx.x] = w;
   }
-  if (threadIdx.x == 0) { sh_st[0] = (uint32_t)state; sh_org[0] = -1; }
+  if (threadIdx.x == 0) { sh_st[0] = word_of_record(g, state); sh_org[0] = -1; }
   const uint32_t* class_bits = stage_class_bits(g, sh_class);
   __syncthreads();
   {   // inclusive scan of the 256 range lengths (thread b holds byte b), shifted into sh_cum[b + 1]
@@ -308,7 +332,7 @@ __global__ void classify_slow_kernel(GrammarDev g, VocabDev v, const int32_t* __
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_pairs) return;
   const int pos = pairs[i].x, rank = pairs[i].y;
-  uint32_t h_st = (uint32_t)positions[pos];
+  uint32_t h_st = word_of_record(g, positions[pos]);
   int32_t h_org = -1;
   Chart c;
   c.h_st = nullptr; c.h_org = nullptr; c.h_sb = nullptr; c.n = -1; c.h_items = 0;
@@ -467,7 +491,7 @@ exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, con
   __shared__ uint32_t sh_class[kSharedClasses * 8];
   const int p = blockIdx.x;
   const EntryDev e = entries[p];
-  if (threadIdx.x == 0) { sh_st[0] = (uint32_t)positions[p]; sh_org[0] = -1; }
+  if (threadIdx.x == 0) { sh_st[0] = word_of_record(g, positions[p]); sh_org[0] = -1; }
   const uint32_t* class_bits = stage_class_bits(g, sh_class);
   __syncthreads();
   uint32_t* out = const_cast<uint32_t*>(e.unc_exit);
@@ -645,7 +669,7 @@ __device__ __forceinline__ bool root_complete(const MatcherDev& m, const Grammar
   const int n = m.n_sets - 1;
   for (int i = m.set_begin[n]; i < m.set_begin[n + 1]; ++i) {
     if (m.item_origin[i] != 0) continue;
-    const uint32_t info = g.state[m.item_state[i]].info;
+    const uint32_t info = g.state[rec_of(g, m.item_state[i])].info;
     if ((info >> 31) && (info & 0x7FFFFFFFu) == (uint32_t)g.root_rule) return true;
   }
   return false;
@@ -669,7 +693,7 @@ __device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g,
   for (int base = 0; base < hist.i_cnt && !overflow; base += 32) {
     const int n_here = min(32, hist.i_cnt - base);
     const bool have = lane < n_here;
-    const uint32_t s = have ? hist.i_st[base + lane] : 0u;
+    const uint32_t s = have ? rec_of(g, hist.i_st[base + lane]) : 0u;
     const int32_t o = have ? hist.i_org[base + lane] : 0;
     int gather_begin = 0, n_gather = 0;
     if (have && XG_BOUND(s, g.n_states, kBoundState)) {
@@ -740,14 +764,14 @@ __device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g,
     int16_t no_local[2] = {0, 0};
     bool ok = advance_waiters(g, hist, g.state[p.check_state[e]].info & 0x7FFFFFFFu, p.check_origin[e], st, org, no_local, 0, cnt, kContCap);
     for (int q = 0; ok && q < cnt; ++q) {
-      const uint32_t info = g.state[st[q]].info;
+      const uint32_t info = g.state[rec_of(g, st[q])].info;
       if (info >> 31) ok = advance_waiters(g, hist, info & 0x7FFFFFFFu, org[q], st, org, no_local, 0, cnt, kContCap);
     }
     if (!ok) { bad = true; cnt = 0; }
     p.cont_cnt[e] = cnt;
     uint4 fa = make_uint4(0, 0, 0, 0), fb = make_uint4(0, 0, 0, 0);
     for (int q = 0; q < cnt; ++q) {
-      const uint4* sf = reinterpret_cast<const uint4*>(g.state_first + (size_t)st[q] * 8);
+      const uint4* sf = reinterpret_cast<const uint4*>(g.state_first + (size_t)rec_of(g, st[q]) * 8);
       const uint4 a = sf[0], c = sf[1];
       fa.x |= a.x; fa.y |= a.y; fa.z |= a.z; fa.w |= a.w;
       fb.x |= c.x; fb.y |= c.y; fb.z |= c.z; fb.w |= c.w;
@@ -821,7 +845,8 @@ __device__ __forceinline__ bool warp_advance_waiters(const GrammarDev& g, const 
     const uint32_t s2 = have ? src_st[base + lane] : 0u;
     const int32_t o2 = have ? src_org[base + lane] : 0;
     uint4 rec = make_uint4(0, 0, 0, 0);
-    if (have && XG_BOUND(s2, g.n_states, kBoundState)) rec = *reinterpret_cast<const uint4*>(&g.state[s2]);
+    const uint32_t r2 = have ? rec_of(g, s2) : 0u;
+    if (have && XG_BOUND(r2, g.n_states, kBoundState)) rec = *reinterpret_cast<const uint4*>(&g.state[r2]);
     int n_wait = (int)(rec.w & 0xFFFFu);
     if (!XG_BOUND((int)rec.z + n_wait, g.n_wait_edges + 1, kBoundWaitEdge)) n_wait = 0;
     const int incl = warp_inclusive_scan(n_wait, lane);
@@ -831,13 +856,14 @@ __device__ __forceinline__ bool warp_advance_waiters(const GrammarDev& g, const 
       const int own = min(owner_of_pair(incl, p, n_here), 31);
       const int first = __shfl_sync(kFullWarp, incl - n_wait, own), wb = __shfl_sync(kFullWarp, (int)rec.z, own);
       const int32_t o2_own = __shfl_sync(kFullWarp, o2, own);
+      const uint32_t s2_own = __shfl_sync(kFullWarp, s2, own);
       uint2 we = make_uint2(0xFFFFFFFFu, 0u);
       if (p < total) we = g.wait_edge[wb + (p - first)];
       uint32_t hits = __ballot_sync(kFullWarp, p < total && we.x == rule);
       while (hits) {
         const int h = __ffs(hits) - 1;
         hits &= hits - 1;
-        const uint32_t ns = __shfl_sync(kFullWarp, we.y & ~kSelf, h);
+        const uint32_t ns = __shfl_sync(kFullWarp, next_word(g, s2_own, we.y), h);
         const int32_t no = __shfl_sync(kFullWarp, (we.y & kSelf) ? o : o2_own, h);
         if (!warp_add_item(st, org, start, cnt, cap, ns, no, lane)) return false;
       }
@@ -866,9 +892,10 @@ __device__ __forceinline__ int warp_token_walk(const GrammarDev& g, const Chart&
       const uint32_t s = have ? cur_st[base + lane] : 0u;
       const int32_t o = have ? cur_org[base + lane] : 0;
       uint4 ra = make_uint4(0, 0, 0, 0), rb = ra;
-      if (have && XG_BOUND(s, g.n_states, kBoundState)) {
-        ra = *reinterpret_cast<const uint4*>(&g.state[s]);
-        rb = *(reinterpret_cast<const uint4*>(&g.state[s]) + 1);
+      const uint32_t sr = have ? rec_of(g, s) : 0u;
+      if (have && XG_BOUND(sr, g.n_states, kBoundState)) {
+        ra = *reinterpret_cast<const uint4*>(&g.state[sr]);
+        rb = *(reinterpret_cast<const uint4*>(&g.state[sr]) + 1);
       }
       int n_edges = (int)(ra.y >> 16);
       if (!XG_BOUND((int)ra.x + n_edges, g.n_scan_edges + 1, kBoundScanEdge)) n_edges = 0;
@@ -879,12 +906,13 @@ __device__ __forceinline__ int warp_token_walk(const GrammarDev& g, const Chart&
         const int own = min(owner_of_pair(incl, p, n_here), 31);
         const int first = __shfl_sync(kFullWarp, incl - n_edges, own), sb = __shfl_sync(kFullWarp, (int)ra.x, own);
         const int32_t o_own = __shfl_sync(kFullWarp, o, own);
+        const uint32_t s_own = __shfl_sync(kFullWarp, s, own);
         const uint32_t e0c = __shfl_sync(kFullWarp, rb.z, own), e0t = __shfl_sync(kFullWarp, rb.w, own);
         uint2 se = make_uint2(kLiteral | 0x100u, 0u);
         if (p < total) se = p == first ? make_uint2(e0c, e0t) : g.scan_edge[sb + (p - first)];      // the first edge is inline in the record
         // the record of the edge's target is requested before the byte is tested against the edge's class: if the edge
         // is taken, the new item's `info` word (and the scan of the next byte) find it on its way
-        if (p < total && XG_BOUND(se.y & ~kSelf, g.n_states, kBoundState)) asm volatile("prefetch.global.L1 [%0];" ::"l"(&g.state[se.y & ~kSelf]));
+        if (p < total && (se.y & kTarget) < (uint32_t)g.rep_first && XG_BOUND(se.y & kTarget, g.n_states, kBoundState)) asm volatile("prefetch.global.L1 [%0];" ::"l"(&g.state[se.y & kTarget]));
         bool hit = false;
         if (se.x & kLiteral) hit = (se.x & 0x1FFu) == byte;
         else if (XG_BOUND(se.x, g.n_classes, kBoundClass)) hit = (g.class_bits[se.x * 8 + word] & bit) != 0;
@@ -892,7 +920,7 @@ __device__ __forceinline__ int warp_token_walk(const GrammarDev& g, const Chart&
         while (hits) {
           const int h = __ffs(hits) - 1;
           hits &= hits - 1;
-          const uint32_t ns = __shfl_sync(kFullWarp, se.y & ~kSelf, h);
+          const uint32_t ns = __shfl_sync(kFullWarp, next_word(g, s_own, se.y), h);
           const int32_t no = __shfl_sync(kFullWarp, (se.y & kSelf) ? self_idx : o_own, h);
           if (!warp_add_item(st, org, start, cnt, cap, ns, no, lane)) { *flags |= kWalkOverflow; return k; }
         }
@@ -904,7 +932,7 @@ __device__ __forceinline__ int warp_token_walk(const GrammarDev& g, const Chart&
       const int n_here = min(32, cnt - q);
       uint32_t info = 0;
       int32_t o = 0;
-      if (lane < n_here && XG_BOUND(st[q + lane], g.n_states, kBoundState)) { info = g.state[st[q + lane]].info; o = org[q + lane]; }
+      if (lane < n_here) { const uint32_t qr = rec_of(g, st[q + lane]); if (XG_BOUND(qr, g.n_states, kBoundState)) { info = g.state[qr].info; o = org[q + lane]; } }
       uint32_t done = __ballot_sync(kFullWarp, (info >> 31) != 0);
       q += n_here;
       while (done) {
@@ -944,7 +972,7 @@ __device__ __forceinline__ int accept_one(MatcherDev& m, const GrammarDev& g, co
   const int len = (int)(v.offset[rank + 1] - off);
   if (!XG_BOUND((long long)off + len, (long long)v.n_bytes + 1, kBoundTokenBytes)) return -6;
   const bool never = v.never[rank] != 0;
-  if (c0.i_cnt > 0) asm volatile("prefetch.global.L1 [%0];" ::"l"(&g.state[c0.i_st[0]]));
+  if (c0.i_cnt > 0 && c0.i_st[0] < (uint32_t)g.rep_first) asm volatile("prefetch.global.L1 [%0];" ::"l"(&g.state[c0.i_st[0]]));
   if (m.terminated) return -8;
   if (!tok_ok) return -7;
   if (tok == v.eos_id) {
@@ -1062,7 +1090,7 @@ __device__ __forceinline__ void for_ids_in_slice(const uint32_t* __restrict__ li
 __device__ __forceinline__ void current_first_bytes(const GrammarDev& g, const Chart& hist, uint32_t* out8, int lane) {
   if (lane < 8) {
     uint32_t w = 0;
-    for (int i = 0; i < hist.i_cnt; ++i) w |= g.state_first[(size_t)hist.i_st[i] * 8 + lane];
+    for (int i = 0; i < hist.i_cnt; ++i) w |= g.state_first[(size_t)rec_of(g, hist.i_st[i]) * 8 + lane];
     out8[lane] = w;
   }
 }
@@ -1593,7 +1621,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
         if (unknown) fa = fb = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);    // every token goes on to its walk
         else
           for (int q = 0; q < w_lsb[2]; ++q) {
-            const uint4* sf = reinterpret_cast<const uint4*>(g.state_first + (size_t)w_st[q] * 8);
+            const uint4* sf = reinterpret_cast<const uint4*>(g.state_first + (size_t)rec_of(g, w_st[q]) * 8);
             const uint4 a = sf[0], d = sf[1];
             fa.x |= a.x; fa.y |= a.y; fa.z |= a.z; fa.w |= a.w;
             fb.x |= d.x; fb.y |= d.y; fb.z |= d.z; fb.w |= d.w;

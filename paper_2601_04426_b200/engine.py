@@ -22,7 +22,7 @@ class Session:
 
     def __init__(self, workload: inputs.Workload, share_pool: bool = True, device: str = "cuda:0", state_compression: bool = True,
                  jit: bool = False, jit_precompute: int = 0, jit_arena_bytes: int = 0, compile_threads: int = 0,
-                 reserve_bytes: int = 0):
+                 reserve_bytes: int = 0, repeat_threshold: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         self.device = torch.device(device)
@@ -38,7 +38,7 @@ class Session:
         def compile_one(g):
             torch.cuda.set_device(self.device)
             return B.Grammar(self.tokenizer, g.kind, g.text, pool=self.pool, state_compression=state_compression,
-                             jit=jit, jit_precompute=jit_precompute, jit_arena_bytes=jit_arena_bytes)
+                             jit=jit, jit_precompute=jit_precompute, jit_arena_bytes=jit_arena_bytes, repeat_threshold=repeat_threshold)
         n_threads = compile_threads if compile_threads > 0 else min(16, os.cpu_count() or 1)
         n_threads = max(1, min(n_threads, len(workload.grammars)))
         torch.cuda.synchronize()
