@@ -139,3 +139,78 @@ def test_classification_is_the_same_for_every_count_of_a_record():
         rows[rec] = cls[0]
     assert not np.array_equal(rows[g.record_of(s, 199)], rows[g.record_of(s, 100)])      # at the upper bound nothing may follow
     assert not np.array_equal(rows[g.record_of(s, 30)], rows[g.record_of(s, 100)])       # below the lower bound the quote may not close
+
+
+# ---- GPU ------------------------------------------------------------------------------------------------------------
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name,vsize,steps", [("R256", 16384, 200), ("R1024", 8192, 160), ("R4096", 8192, 160)])
+def test_gpu_masks_with_counted_repetitions_bit_exact(name, vsize, steps):
+    """The default compile counts these workloads' repetitions; every compared mask equals the grammar-text oracle's."""
+    from test_gpu_parity import _run_trajectories
+    w = inputs.make_workload(name, batch=8, steps=steps, vocab_size=vsize)
+    compared = _run_trajectories(w, set(range(0, steps, 9)), check_requests={1, 2})
+    assert compared > steps
+
+
+@pytest.mark.gpu
+def test_gpu_counted_repetitions_fused_steps_and_restart():
+    from test_gpu_parity import _run_trajectories
+    w = inputs.make_workload("R256", batch=4, steps=150, vocab_size=8192)
+    assert _run_trajectories(w, set(range(0, 150, 7)), fused=True) > 40
+    assert _run_trajectories(w, set(range(0, 150, 11)), restart=True) > 20
+
+
+@pytest.mark.gpu
+def test_gpu_counted_grammar_is_small_and_fast_to_compile():
+    """States and records do not depend on the bound (the section's claim); the expanded compile of the same grammar
+    has hundreds of times more states."""
+    w = inputs.make_workload("R4096", batch=1, steps=2, vocab_size=8192)
+    v = w.vocab
+    tok = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
+    spec = w.grammars[0]
+    counted = B.Grammar(tok, spec.kind, spec.text)
+    w2 = inputs.make_workload("R1024", batch=1, steps=2, vocab_size=8192)      # (every bound of it is counted too)
+    small = B.Grammar(tok, w2.grammars[0].kind, w2.grammars[0].text)
+    expanded = B.Grammar(tok, spec.kind, spec.text, repeat_threshold=-1)
+    a, b, c = counted.stats(), small.stats(), expanded.stats()
+    # (the two schemas differ in a few literal bytes, nothing else: four times the bounds, about the same states)
+    assert abs(a["n_states"] - b["n_states"]) < 20 and a["n_states"] * 100 < c["n_states"]
+    assert abs(counted.tables()["n_records"] - small.tables()["n_records"]) < 20
+    assert a["frontend_ms"] * 10 < c["frontend_ms"]
+    counted.close(); small.close(); expanded.close(); tok.close()
+
+
+@pytest.mark.gpu
+def test_gpu_cache_entries_of_counted_records_match_the_oracle():
+    """Per (state, count): the entry of its record equals the oracle's classification from that very count --
+    in the middle of the repetition, near both bounds, and at them."""
+    from test_gpu_parity import _entry_classes
+    w = inputs.make_workload("R256", batch=1, steps=2, vocab_size=8192)
+    v = w.vocab
+    ov = O.Vocab(v.tokens, v.eos_id, v.special_ids)
+    tok = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
+    text = 'root ::= "[" ("\\"" [a-z0-9 ]{40,300} "\\"" ", "){2,80} "]"'
+    g = B.Grammar(tok, "ebnf", text)
+    t = g.tables()
+    scal = {k: t.pop(k) for k in ("n_rules", "n_states", "n_classes", "root_rule", "root_nullable")}
+    tb = O.Tables(scal["n_rules"], scal["n_states"], scal["n_classes"], scal["root_rule"], scal["root_nullable"], **t)
+    assert tb.counted and (t["rule_rep_hi"] > 0).sum() == 2
+    checked = 0
+    for s in tb.scannable_states():
+        hi = int(t["rule_rep_hi"][t["state_rule"][s]])
+        lo = int(t["rule_rep_lo"][t["state_rule"][s]])
+        counts = [0] if hi == 0 else sorted({0, 1, lo - 2, lo - 1, lo, (lo + hi) // 2, hi - 13, hi - 2, hi - 1} & set(range(hi)))
+        for k in counts:
+            ref = tb.classify(ov, s, count=k)
+            try:
+                cls = _entry_classes(g.cache_entry(g.record_of(s, k)), v.size)
+            except B.XgError:
+                # a state whose only byte edges start the next iteration has none at the last count: no entry, and
+                # the oracle rejects every token there
+                assert k == hi - 1 and not ref.any(), (s, k)
+                continue
+            assert np.array_equal(cls, ref), (s, k, np.nonzero(cls != ref)[0][:5])
+            checked += 1
+    assert checked > 20
+    g.close(); tok.close()

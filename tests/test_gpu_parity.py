@@ -28,14 +28,14 @@ def _oracle_side(w):
     return ov, grammars, matchers
 
 
-def _run_trajectories(w, check_steps, check_requests=None, fused=False, restart=False):
+def _run_trajectories(w, check_steps, check_requests=None, fused=False, restart=False, **session_kw):
     """Drive GPU and oracle along the seeded trajectories; compare masks where asked, and the
     cheap invariants everywhere (sampled token allowed, statuses, termination).  fused: after the
     first fill every step is one accept-and-fill launch that restarts a request at end of
     sequence, instead of accept, reset and fill.  restart: the accept call restarts a request at
     end of sequence (no reset call)."""
     torch, engine = _engine()
-    s = engine.Session(w)
+    s = engine.Session(w, **session_kw)
     ov, _, oms = _oracle_side(w)
     n = s.n
     compared = 0

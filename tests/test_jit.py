@@ -271,7 +271,7 @@ def test_just_in_time_entries_serve_whole_classes_of_states():
     """Long repetitions: one entry built just in time is published to every state of its class
     (repetition state compression), so a string of hundreds of characters costs a handful of builds."""
     w = inputs.make_workload("R256", batch=4, steps=150, vocab_size=8192)
-    s, final, _, stats = _drive(w, 6, "each")
+    s, final, _, stats = _drive(w, 6, "each", repeat_threshold=-1)
     assert 0 < final["n_built"] < 400
     assert sum(x["n_states"] for x in stats) > 20 * final["n_built"]
     s.close()

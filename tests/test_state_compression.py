@@ -136,8 +136,9 @@ def test_gpu_shared_entries_match_oracle_rows_and_the_uncompressed_build():
     ov = O.Vocab(v.tokens, v.eos_id, v.special_ids)
     tok = B.Tokenizer(v.tokens, v.eos_id, v.special_ids)
     spec = w.grammars[0]
-    g = B.Grammar(tok, spec.kind, spec.text)
-    plain = B.Grammar(tok, spec.kind, spec.text, state_compression=False)
+    # (repeat_threshold=-1: the repetitions expanded into explicit states, which is what this sharing is about)
+    g = B.Grammar(tok, spec.kind, spec.text, repeat_threshold=-1)
+    plain = B.Grammar(tok, spec.kind, spec.text, state_compression=False, repeat_threshold=-1)
     tb, _ = tables_of(spec.kind, spec.text)
     rep = g.state_classes()
     st, st_plain = g.stats(), plain.stats()
@@ -158,7 +159,8 @@ def test_gpu_shared_entries_match_oracle_rows_and_the_uncompressed_build():
 @pytest.mark.gpu
 @pytest.mark.parametrize("name,vsize,steps", [("R256", 16384, 200), ("R1024", 8192, 120)])
 def test_gpu_masks_through_long_repetitions_bit_exact(name, vsize, steps):
+    """With the repetitions expanded into explicit states whose cache entries are shared."""
     from test_gpu_parity import _run_trajectories
     w = inputs.make_workload(name, batch=8, steps=steps, vocab_size=vsize)
-    compared = _run_trajectories(w, set(range(0, steps, 9)), check_requests={1, 2})
+    compared = _run_trajectories(w, set(range(0, steps, 9)), check_requests={1, 2}, repeat_threshold=-1)
     assert compared > steps
