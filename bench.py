@@ -210,6 +210,9 @@ def main():
                     help="comma-separated K values (or 'full'): compile just in time with K entries precomputed and report "
                          "compile time and per-step time avg / P99 / max over the trajectory (the shape of the paper's K sweep)")
     ap.add_argument("--compile-threads", type=int, default=0, help="host threads compiling the grammars (0 = one per core, at most 16)")
+    ap.add_argument("--repeat-threshold", type=int, default=0,
+                    help="bounded repetitions of at least this many iterations keep a count in the Earley item (Section 3.6); "
+                         "0 = the library's default (64), -1 = expand every repetition into explicit states")
     ap.add_argument("--no-state-compression", action="store_true",
                     help="build one cache entry per scannable state (ablation of the repetition state compression)")
     args = ap.parse_args()
@@ -255,7 +258,8 @@ def main():
     wt.close()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
-    s = engine.Session(w, device="cuda:%d" % local_rank, state_compression=not args.no_state_compression, compile_threads=args.compile_threads)
+    s = engine.Session(w, device="cuda:%d" % local_rank, state_compression=not args.no_state_compression, compile_threads=args.compile_threads,
+                       repeat_threshold=args.repeat_threshold)
     torch.cuda.synchronize()
     session_s = time.perf_counter() - t0
     compile_s = s.compile_wall_s
@@ -654,7 +658,7 @@ def main():
     # the same compile into a pool whose device memory was taken from the driver beforehand (a server that reserves its
     # cache budget at start-up): what is left is the build itself
     s2 = engine.Session(w, device="cuda:%d" % local_rank, state_compression=not args.no_state_compression, compile_threads=args.compile_threads,
-                        reserve_bytes=int(pool_reserved * 1.25) + (64 << 20))
+                        reserve_bytes=int(pool_reserved * 1.25) + (64 << 20), repeat_threshold=args.repeat_threshold)
     st2 = [g.stats() for g in s2.grammars]
     line["cache_build"]["with_reserved_pool"] = {"seconds": sum(x["cache_build_ms"] for x in st2) / 1e3, "compile_wall_s": s2.compile_wall_s,
                                                  "pairs_per_s": pairs / max(sum(x["cache_build_ms"] for x in st2) / 1e3, 1e-9),

@@ -214,3 +214,15 @@ def test_gpu_cache_entries_of_counted_records_match_the_oracle():
             checked += 1
     assert checked > 20
     g.close(); tok.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("static_fill", [False, True])
+def test_gpu_counted_repetitions_with_a_just_in_time_cache(static_fill):
+    """Entries of counted records are built on first visit like any other; until then the mask comes from the walk of
+    the whole vocabulary against the chart, counts included.  Also through the allocation-free fill."""
+    from test_jit import _drive
+    w = inputs.make_workload("R1024", batch=4, steps=150, vocab_size=8192)
+    s, final, _, stats = _drive(w, 6, "each", static_fill=static_fill)
+    assert final["n_built"] > 0 and sum(x["n_states"] for x in stats) < 4 * 1200
+    s.close()

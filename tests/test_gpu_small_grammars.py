@@ -20,14 +20,30 @@ CASES = [(c[0], c[1], c[3]) for c in CFG_CASES] + [("regex_%d" % i, c[0], c[2]) 
 @pytest.mark.parametrize("inline", [-1, 0], ids=["inlined", "rules_kept"])
 @pytest.mark.parametrize("name,ebnf,alphabet", CASES, ids=[c[0] for c in CASES])
 def test_every_prefix_every_token(name, ebnf, alphabet, inline):
+    _every_prefix_every_token(name, ebnf, alphabet, 4, inline_max_states=inline)
+
+
+def _counted_cases():
+    from test_counted_repetition import COUNTED_CASES
+    return [("counted_%d" % i, c[0], c[1], min(c[2], 6)) for i, c in enumerate(COUNTED_CASES)]
+
+
+@pytest.mark.parametrize("name,ebnf,alphabet,max_len", _counted_cases(), ids=[c[0] for c in _counted_cases()])
+def test_every_prefix_every_token_with_counted_repetitions(name, ebnf, alphabet, max_len):
+    """Repetitions of two or more iterations kept as counters (Section 3.6): tokens of up to three bytes cross
+    iteration boundaries, both bounds and the end of the rule from every count."""
+    _every_prefix_every_token(name, ebnf, alphabet, max_len, repeat_threshold=2)
+
+
+def _every_prefix_every_token(name, ebnf, alphabet, max_prefix, **compile_kw):
     import torch
     tokens = [s.encode() for n in (1, 2, 3) for s in map("".join, itertools.product(alphabet, repeat=n))]
     tokens.append(b"")
     eos = len(tokens) - 1
     tokens += [b"\xf0\x9f" + bytes([65 + i]) for i in range(-len(tokens) % 32)]       # padding that no grammar here accepts
     tok = B.Tokenizer(tokens, eos)
-    g = B.Grammar(tok, "ebnf", ebnf, inline_max_states=inline)
-    jit = B.Grammar(tok, "ebnf", ebnf, inline_max_states=inline, jit=True)           # nothing built: whole-vocabulary walks
+    g = B.Grammar(tok, "ebnf", ebnf, **compile_kw)
+    jit = B.Grammar(tok, "ebnf", ebnf, jit=True, **compile_kw)                       # nothing built: whole-vocabulary walks
     ov = O.Vocab(tokens, eos)
     og = O.Grammar(ebnf)
     matchers = [B.Matcher(g), B.Matcher(jit)]
@@ -37,7 +53,7 @@ def test_every_prefix_every_token(name, ebnf, alphabet, inline):
     ids = torch.zeros(2, dtype=torch.int32, device="cuda")
     single = {bytes([ord(c)]): tokens.index(bytes([ord(c)])) for c in alphabet}
     checked = 0
-    for prefix in all_strings(alphabet, 4):
+    for prefix in all_strings(alphabet, max_prefix):
         data = prefix.encode()
         om = O.Matcher(og)
         if not om.accept_bytes(data):
