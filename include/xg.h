@@ -209,14 +209,15 @@ xg_status_t xg_grammar_record_of(const xg_grammar_t* g, int32_t state, int32_t c
  * compares canonical serialisations, so a collision can never share an entry. */
 xg_status_t xg_grammar_get_rule_hashes(const xg_grammar_t* g, uint64_t* out);
 
-/* Repetition state compression (Section 3.6).  A bounded repetition R{l,r} is kept as explicit
- * automaton states (the count k of the paper's state (R{l,r}, k) is the state itself), but cache
- * entries are built once per class of states that no token can tell apart: states of one rule
- * whose automata agree when unrolled `depth` edges deep.  With depth = the longest token in bytes
- * their accepted / rejected / uncertain sets are identical, so inside a long repetition only the
- * copies within `depth` of the bounds get entries of their own.  out (host, [n_states]): for each
- * state the smallest state of its class.  depth < 0: the tokenizer's longest token (grammars
- * compiled without a tokenizer: XG_ERR_INVALID_ARG).  Host work only. */
+/* Repetition state compression (Section 3.6), for repetitions below xg_compile_options_t.repeat_threshold.  Such an
+ * R{l,r} is kept as explicit automaton states (the count k of the paper's state (R{l,r}, k) is the state itself), but
+ * cache entries are built once per class of states that no token can tell apart: states of one rule whose automata
+ * agree when unrolled `depth` edges deep.  With depth = the longest token in bytes their accepted / rejected /
+ * uncertain sets are identical, so inside a repetition only the copies within `depth` of the bounds get entries of
+ * their own.  out (host, [n_states]): for each state the smallest state of its class.  depth < 0: the tokenizer's
+ * longest token (grammars compiled without a tokenizer: XG_ERR_INVALID_ARG).  A grammar with counted repetitions
+ * (rule_rep_hi != NULL in its tables) answers XG_ERR_UNSUPPORTED: its records are the classes (xg_grammar_record_of).
+ * Host work only. */
 xg_status_t xg_grammar_get_state_classes(const xg_grammar_t* g, int32_t depth, int32_t* out);
 
 /* One cache entry, copied to the host (valid until the next call on this grammar or its
