@@ -474,6 +474,22 @@ def main():
     torch.cuda.synchronize()
     t_apply_alone = a0.elapsed_time(a1) * 1e3 / reps
     alone_zero_bits = n * s.V - int(np.unpackbits(s.mask_numpy().view(np.uint8)).sum())
+    # the same launches with a mask that allows nothing: every vector is overwritten and none is read, i.e. what the
+    # memory system takes from this kernel as a pure store stream of the same size (the mask is still read first)
+    saved_mask = s.bitmask.clone()
+    s.bitmask.zero_()
+    for k in range(ring_n):
+        s.apply(ring[k])
+    torch.cuda.synchronize()
+    torch.cuda._sleep(int(4.0e6))
+    a0.record()
+    for k in range(reps):
+        s.apply(ring[k % ring_n])
+    a1.record()
+    torch.cuda.synchronize()
+    t_apply_all_masked = a0.elapsed_time(a1) * 1e3 / reps
+    s.bitmask.copy_(saved_mask)
+    del saved_mask
     clocks = sampler.finish()          # sampled over the timed pass and the per-kernel passes (same steps, same kernels)
     t_fill, t_apply, t_accept = eager_us["fill"], eager_us["apply"], eager_us["accept"]
     zero_bits = zero_bits_sum / max(mask_samples, 1)
@@ -508,7 +524,9 @@ def main():
                 "in_step": apply_at(t_apply_in_step), "dominant_by_time": dominant,
                 "eager_event_interval": apply_at(t_apply),
                 "alone": dict(apply_at(t_apply_alone, alone_zero_bits),
-                              how="%d launches back to back over the logits ring (queued behind a primer kernel), last step's mask" % reps)}
+                              how="%d launches back to back over the logits ring (queued behind a primer kernel), last step's mask" % reps),
+                "alone_all_masked": dict({k_: v_ for k_, v_ in apply_at(t_apply_all_masked, n * s.V).items() if k_ in ("us_per_launch", "achieved", "frac")},
+                                         how="the same launches with an all-zero mask: stores only, no logit is read (the store ceiling of this kernel and size)")}
 
     # The fill and accept kernels are bound by latency, not by a memory or arithmetic pipe.  What can be said against a
     # peak is their issue rate: warp instructions per launch (ncu) over the launch time, against 148 SMs x 4 schedulers
