@@ -1478,6 +1478,13 @@ static xg_status_t batch_slot(xg_matcher_t* const* matchers, int32_t batch, cuda
   return XG_OK;
 }
 
+// Does a grammar of the batch have counted repetitions (Section 3.6)?  Then the step kernels decode the count out of
+// every state word; otherwise the variants without that decode run.
+static bool batch_has_counted_rules(xg_matcher_t* const* matchers, int32_t batch) {
+  for (int i = 0; i < batch; ++i) if (matchers[i]->grammar->counted) return true;
+  return false;
+}
+
 static xg_status_t apply_rows(void* logits_dev, xg_dtype_t dtype, int32_t rows, int32_t vocab_size, int64_t logits_row_stride_elems,
                               const int32_t* bitmask_dev, int64_t mask_row_stride_words, const int32_t* row_indices_dev, void* stream);
 
@@ -1511,19 +1518,23 @@ static xg_status_t accept_and_fill(xg_matcher_t* const* matchers, int32_t batch,
     const dim3 grid(blocks, batch), block(threads);
     cudaStream_t cs = (cudaStream_t)stream;
     const long long stride_w = (long long)row_stride_words, stride_l = (long long)logits_row_stride_elems;
-#define XG_FILL(ACCEPT, ELEMS, HEAVY, TOK, AST, RST, LOGITS)                                                                              \
-    XG_CUDA(launch_step_kernel(fill_cluster_kernel<ACCEPT, ELEMS, HEAVY>, grid, block, smem, cs, blocks, dm, tok->dev, bitmask_dev, stride_w, \
+    const bool counts = batch_has_counted_rules(matchers, batch);
+#define XG_FILL_C(ACCEPT, ELEMS, HEAVY, COUNTS, TOK, AST, RST, LOGITS)                                                                              \
+    XG_CUDA(launch_step_kernel(fill_cluster_kernel<ACCEPT, ELEMS, HEAVY, COUNTS>, grid, block, smem, cs, blocks, dm, tok->dev, bitmask_dev, stride_w, \
                                status_dev, (const int32_t*)(TOK), (int32_t*)(AST), (int)(RST), (void*)(LOGITS), stride_l))
+#define XG_FILL(ACCEPT, ELEMS, HEAVY, TOK, AST, RST, LOGITS) \
+    do { if (counts) XG_FILL_C(ACCEPT, ELEMS, HEAVY, true, TOK, AST, RST, LOGITS); else XG_FILL_C(ACCEPT, ELEMS, HEAVY, false, TOK, AST, RST, LOGITS); } while (0)
     if (token_ids_dev) { if (heavy) XG_FILL(true, 0, true, token_ids_dev, accept_status_dev, restart_on_eos, nullptr); else XG_FILL(true, 0, false, token_ids_dev, accept_status_dev, restart_on_eos, nullptr); }
     else if (!logits_dev) { if (heavy) XG_FILL(false, 0, true, nullptr, nullptr, 0, nullptr); else XG_FILL(false, 0, false, nullptr, nullptr, 0, nullptr); }
     else if (dtype == XG_BF16) { if (heavy) XG_FILL(false, 8, true, nullptr, nullptr, 0, logits_dev); else XG_FILL(false, 8, false, nullptr, nullptr, 0, logits_dev); }
     else { if (heavy) XG_FILL(false, 4, true, nullptr, nullptr, 0, logits_dev); else XG_FILL(false, 4, false, nullptr, nullptr, 0, logits_dev); }
 #undef XG_FILL
+#undef XG_FILL_C
     return XG_OK;
   }
   if (token_ids_dev) {
-    XG_CUDA(launch_step_kernel(accept_kernel, dim3((batch + 3) / 4), dim3(128), 0, (cudaStream_t)stream, 1, (MatcherDev* const*)slot->dev_matchers,
-                               (int)batch, tok->dev, token_ids_dev, accept_status_dev, restart_on_eos));
+    XG_CUDA(launch_step_kernel(batch_has_counted_rules(matchers, batch) ? accept_kernel<true> : accept_kernel<false>, dim3((batch + 3) / 4), dim3(128), 0,
+                               (cudaStream_t)stream, 1, (MatcherDev* const*)slot->dev_matchers, (int)batch, tok->dev, token_ids_dev, accept_status_dev, restart_on_eos));
   }
   int chunks = std::max((W + kMergeMaxChunkWords - 1) / kMergeMaxChunkWords, std::min(8, (W + 127) / 128));
   dim3 grid_merge(chunks, batch);
@@ -1649,8 +1660,8 @@ xg_status_t xg_accept_token_ex(xg_matcher_t* const* matchers, int32_t batch, con
   xg_status_t st = batch_slot(matchers, batch, (cudaStream_t)stream, &tok, &slot);
   if (st != XG_OK) return st;
   if (!token_ids_dev) return set_error(XG_ERR_INVALID_ARG, "token_ids_dev is NULL");
-  XG_CUDA(launch_step_kernel(accept_kernel, dim3((batch + 3) / 4), dim3(128), 0, (cudaStream_t)stream, 1, (MatcherDev* const*)slot->dev_matchers,
-                             (int)batch, tok->dev, token_ids_dev, status_dev, restart_on_eos ? 1 : 0));
+  XG_CUDA(launch_step_kernel(batch_has_counted_rules(matchers, batch) ? accept_kernel<true> : accept_kernel<false>, dim3((batch + 3) / 4), dim3(128), 0,
+                             (cudaStream_t)stream, 1, (MatcherDev* const*)slot->dev_matchers, (int)batch, tok->dev, token_ids_dev, status_dev, restart_on_eos ? 1 : 0));
   return XG_OK;
 }
 

@@ -74,10 +74,25 @@ __device__ __forceinline__ Chart chart_of_history(const uint32_t* h_st, const in
 
 constexpr uint32_t kFullWarp = 0xFFFFFFFFu;
 
+// A grammar that is known to have no counted repetition: the same tables seen through a type for which the decoding
+// of state words below compiles away.  The step kernels exist in both forms and the host picks per batch (C3: the
+// decode costs 1.2 us of a 38 us step, although it never finds a count there).
+struct PlainGrammarDev : GrammarDev {};
+template <typename G> struct HasCounts { static constexpr bool value = true; };
+template <> struct HasCounts<PlainGrammarDev> { static constexpr bool value = false; };
+template <bool kCounts> struct GrammarAs { typedef GrammarDev type; };
+template <> struct GrammarAs<false> { typedef PlainGrammarDev type; };
+template <bool kCounts>
+__device__ __forceinline__ const typename GrammarAs<kCounts>::type& grammar_as(const GrammarDev& g) { return static_cast<const typename GrammarAs<kCounts>::type&>(g); }
+
 // Counted repetitions (Section 3.6).  rec_of: the record (index into state[], state_first[], entries[]) of an item's
 // state word; ordinary states are their own record.
-__device__ __forceinline__ uint32_t rec_of(const GrammarDev& g, uint32_t w) {
-  if (w < (uint32_t)g.rep_first) return w;
+// (`rep_first`: g.rep_first, read once by the caller -- the walks are chains of dependent loads, and the test that almost
+// always ends here must not wait for a load of its own)
+template <typename G>
+__device__ __forceinline__ uint32_t rec_of(const G& g, uint32_t w, uint32_t rep_first) {
+  if (!HasCounts<G>::value) return w;
+  if (w < rep_first) return w;
   const uint32_t q = w & ((1u << g.rep_shift) - 1u);
   const int done = (int)(w >> g.rep_shift) + 1;
   if (!XG_BOUND((int)q - g.rep_first, g.n_words_states - g.rep_first, kBoundState)) return 0;
@@ -85,11 +100,15 @@ __device__ __forceinline__ uint32_t rec_of(const GrammarDev& g, uint32_t w) {
   const int dl = min(max(rs.y - done, 0), g.rep_depth), dr = max(min(rs.z - done, g.rep_depth), 0);
   return (uint32_t)(rs.x + dl * (g.rep_depth + 1) + dr);
 }
+template <typename G>
+__device__ __forceinline__ uint32_t rec_of(const G& g, uint32_t w) { return rec_of(g, w, (uint32_t)g.rep_first); }
 // a state word that belongs to record `rec` (the record itself for ordinary states)
 __device__ __forceinline__ uint32_t word_of_record(const GrammarDev& g, int rec) { return g.rec_word ? g.rec_word[rec] : (uint32_t)rec; }
 // the state word an edge leads to from the item whose state word is `from`: the packed target, with the count of
 // `from` when the edge stays inside a counted rule (kRel), one more when it starts the next iteration (kIter)
-__device__ __forceinline__ uint32_t next_word(const GrammarDev& g, uint32_t from, uint32_t packed) {
+template <typename G>
+__device__ __forceinline__ uint32_t next_word(const G& g, uint32_t from, uint32_t packed) {
+  if (!HasCounts<G>::value) return packed & ~kSelf;
   uint32_t w = packed & kTarget;
   if (packed & kRel) w += (from >> g.rep_shift << g.rep_shift) + ((packed & kIter) ? (1u << g.rep_shift) : 0u);
   return w;
@@ -117,8 +136,8 @@ __device__ __forceinline__ bool add_item(uint32_t* st, int32_t* org, int start, 
 }
 
 // advance every item of chart set `o` that waits for `rule` into the set [start, cnt)
-template <typename LsbT>
-__device__ __forceinline__ bool advance_waiters(const GrammarDev& g, const Chart& c, uint32_t rule, int32_t o, uint32_t* st, int32_t* org,
+template <typename LsbT, typename G>
+__device__ __forceinline__ bool advance_waiters(const G& g, const Chart& c, uint32_t rule, int32_t o, uint32_t* st, int32_t* org,
                                                 const LsbT* lsb, int start, int& cnt, int cap) {
   const uint32_t* src_st;
   const int32_t* src_org;
@@ -133,10 +152,11 @@ __device__ __forceinline__ bool advance_waiters(const GrammarDev& g, const Chart
     src_st = st; src_org = org; b = lsb[o - c.i_idx]; e = lsb[o - c.i_idx + 1];
     if (!XG_BOUND(e, cnt + 1, kBoundWalkItem) || !XG_BOUND(b, e + 1, kBoundWalkItem)) return true;
   }
+  const uint32_t rep_first = (uint32_t)g.rep_first;
   for (int i = b; i < e; ++i) {
     const uint32_t s2 = src_st[i];
     const int32_t o2 = src_org[i];
-    const uint32_t r2 = rec_of(g, s2);
+    const uint32_t r2 = rec_of(g, s2, rep_first);
     if (!XG_BOUND(r2, g.n_states, kBoundState)) continue;
     const uint4 rec = *reinterpret_cast<const uint4*>(&g.state[r2]);
     const int wait_end = (int)rec.z + (int)(rec.w & 0xFFFFu);
@@ -158,10 +178,11 @@ __device__ __forceinline__ bool advance_waiters(const GrammarDev& g, const Chart
 }
 
 // class_bits may point to a shared-memory copy of g.class_bits
-template <typename LsbT>
-__device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* class_bits, const Chart& c, const uint8_t* __restrict__ bytes, int len,
+template <typename LsbT, typename G>
+__device__ __forceinline__ int token_walk(const G& g, const uint32_t* class_bits, const Chart& c, const uint8_t* __restrict__ bytes, int len,
                                           bool own_edges_first, uint32_t* st, int32_t* org, int cap, LsbT* lsb, int* flags, uint32_t* exit_mask) {
   int cnt = 0;
+  const uint32_t rep_first = (uint32_t)g.rep_first;
   const uint32_t* cur_st = c.i_st;
   const int32_t* cur_org = c.i_org;
   int cur_b = 0, cur_e = c.i_cnt;
@@ -176,7 +197,7 @@ __device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* c
     for (int i = cur_b; i < cur_e; ++i) {
       const uint32_t s = cur_st[i];
       const int32_t o = cur_org[i];
-      const uint32_t sr = rec_of(g, s);
+      const uint32_t sr = rec_of(g, s, rep_first);
       if (!XG_BOUND(sr, g.n_states, kBoundState)) continue;
       const uint4 ra = *reinterpret_cast<const uint4*>(&g.state[sr]);
       const int n_edges = (k == 0 && own_edges_first) ? (int)(ra.y & 0xFFFFu) : (int)(ra.y >> 16);
@@ -201,7 +222,7 @@ __device__ __forceinline__ int token_walk(const GrammarDev& g, const uint32_t* c
     if (cnt == start) return k;
     // complete (cascades through the growing set)
     for (int q = start; q < cnt; ++q) {
-      const uint32_t qr = rec_of(g, st[q]);
+      const uint32_t qr = rec_of(g, st[q], rep_first);
       if (!XG_BOUND(qr, g.n_states, kBoundState)) continue;
       const uint32_t info = g.state[qr].info;
       if (!(info >> 31)) continue;
@@ -664,7 +685,8 @@ jit_patch_lists_kernel(EntryDev* __restrict__ entries, const int32_t* __restrict
 // matcher state
 // ------------------------------------------------------------------------------------------
 // is the root rule complete in the current set (EOS allowed)?
-__device__ __forceinline__ bool root_complete(const MatcherDev& m, const GrammarDev& g) {
+template <typename G>
+__device__ __forceinline__ bool root_complete(const MatcherDev& m, const G& g) {
   if (m.n_sets == 1 && g.root_nullable) return true;
   const int n = m.n_sets - 1;
   for (int i = m.set_begin[n]; i < m.set_begin[n + 1]; ++i) {
@@ -680,9 +702,11 @@ __device__ __forceinline__ bool root_complete(const MatcherDev& m, const Grammar
 // entry, the cache entry's header -- are three rounds of loads for the whole set; the lists themselves are kept in
 // registers, one slot per lane, and a pair is added to them by a compare in every lane and a vote.  Then one lane per
 // entry completes that entry's rule into its continuation set.
-__device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g, int lane) {
+template <typename G>
+__device__ __forceinline__ void prepare_plan(MatcherDev& m, const G& g, int lane) {
   StepPlan& p = *m.plan;
   const int n = m.n_sets - 1;
+  const uint32_t rep_first = (uint32_t)g.rep_first;
   const Chart hist = chart_of_history(m.item_state, m.item_origin, m.set_begin, n);
   int n_merge = 0, n_check = 0, n_missing = 0, overflow = 0;       // (the same in every lane)
   int merge_lo = -1, merge_hi = -1;           // slots lane and lane + 32 of the merge list
@@ -693,7 +717,7 @@ __device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g,
   for (int base = 0; base < hist.i_cnt && !overflow; base += 32) {
     const int n_here = min(32, hist.i_cnt - base);
     const bool have = lane < n_here;
-    const uint32_t s = have ? rec_of(g, hist.i_st[base + lane]) : 0u;
+    const uint32_t s = have ? rec_of(g, hist.i_st[base + lane], rep_first) : 0u;
     const int32_t o = have ? hist.i_org[base + lane] : 0;
     int gather_begin = 0, n_gather = 0;
     if (have && XG_BOUND(s, g.n_states, kBoundState)) {
@@ -764,14 +788,14 @@ __device__ __forceinline__ void prepare_plan(MatcherDev& m, const GrammarDev& g,
     int16_t no_local[2] = {0, 0};
     bool ok = advance_waiters(g, hist, g.state[p.check_state[e]].info & 0x7FFFFFFFu, p.check_origin[e], st, org, no_local, 0, cnt, kContCap);
     for (int q = 0; ok && q < cnt; ++q) {
-      const uint32_t info = g.state[rec_of(g, st[q])].info;
+      const uint32_t info = g.state[rec_of(g, st[q], rep_first)].info;
       if (info >> 31) ok = advance_waiters(g, hist, info & 0x7FFFFFFFu, org[q], st, org, no_local, 0, cnt, kContCap);
     }
     if (!ok) { bad = true; cnt = 0; }
     p.cont_cnt[e] = cnt;
     uint4 fa = make_uint4(0, 0, 0, 0), fb = make_uint4(0, 0, 0, 0);
     for (int q = 0; q < cnt; ++q) {
-      const uint4* sf = reinterpret_cast<const uint4*>(g.state_first + (size_t)rec_of(g, st[q]) * 8);
+      const uint4* sf = reinterpret_cast<const uint4*>(g.state_first + (size_t)rec_of(g, st[q], rep_first) * 8);
       const uint4 a = sf[0], c = sf[1];
       fa.x |= a.x; fa.y |= a.y; fa.z |= a.z; fa.w |= a.w;
       fb.x |= c.x; fb.y |= c.y; fb.z |= c.z; fb.w |= c.w;
@@ -823,8 +847,8 @@ __device__ __forceinline__ bool warp_add_item(uint32_t* st, int32_t* org, int st
 }
 
 // advance every item of chart set `o` that waits for `rule` into the set [start, cnt)
-template <typename LsbT>
-__device__ __forceinline__ bool warp_advance_waiters(const GrammarDev& g, const Chart& c, uint32_t rule, int32_t o, uint32_t* st, int32_t* org,
+template <typename LsbT, typename G>
+__device__ __forceinline__ bool warp_advance_waiters(const G& g, const Chart& c, uint32_t rule, int32_t o, uint32_t* st, int32_t* org,
                                                      const LsbT* lsb, int start, int& cnt, int cap, int lane) {
   const uint32_t* src_st;
   const int32_t* src_org;
@@ -839,13 +863,14 @@ __device__ __forceinline__ bool warp_advance_waiters(const GrammarDev& g, const 
     src_st = st; src_org = org; b = lsb[o - c.i_idx]; e = lsb[o - c.i_idx + 1];
     if (!XG_BOUND(e, cnt + 1, kBoundWalkItem) || !XG_BOUND(b, e + 1, kBoundWalkItem)) return true;
   }
+  const uint32_t rep_first = (uint32_t)g.rep_first;
   for (int base = b; base < e; base += 32) {
     const int n_here = min(32, e - base);
     const bool have = lane < n_here;
     const uint32_t s2 = have ? src_st[base + lane] : 0u;
     const int32_t o2 = have ? src_org[base + lane] : 0;
     uint4 rec = make_uint4(0, 0, 0, 0);
-    const uint32_t r2 = have ? rec_of(g, s2) : 0u;
+    const uint32_t r2 = have ? rec_of(g, s2, rep_first) : 0u;
     if (have && XG_BOUND(r2, g.n_states, kBoundState)) rec = *reinterpret_cast<const uint4*>(&g.state[r2]);
     int n_wait = (int)(rec.w & 0xFFFFu);
     if (!XG_BOUND((int)rec.z + n_wait, g.n_wait_edges + 1, kBoundWaitEdge)) n_wait = 0;
@@ -872,10 +897,11 @@ __device__ __forceinline__ bool warp_advance_waiters(const GrammarDev& g, const 
   return true;
 }
 
-template <typename LsbT>
-__device__ __forceinline__ int warp_token_walk(const GrammarDev& g, const Chart& c, const uint8_t* __restrict__ bytes, int len,
+template <typename LsbT, typename G>
+__device__ __forceinline__ int warp_token_walk(const G& g, const Chart& c, const uint8_t* __restrict__ bytes, int len,
                                                uint32_t* st, int32_t* org, int cap, LsbT* lsb, int* flags, int lane) {
   int cnt = 0;
+  const uint32_t rep_first = (uint32_t)g.rep_first;
   const uint32_t* cur_st = c.i_st;
   const int32_t* cur_org = c.i_org;
   int cur_b = 0, cur_e = c.i_cnt;
@@ -892,7 +918,7 @@ __device__ __forceinline__ int warp_token_walk(const GrammarDev& g, const Chart&
       const uint32_t s = have ? cur_st[base + lane] : 0u;
       const int32_t o = have ? cur_org[base + lane] : 0;
       uint4 ra = make_uint4(0, 0, 0, 0), rb = ra;
-      const uint32_t sr = have ? rec_of(g, s) : 0u;
+      const uint32_t sr = have ? rec_of(g, s, rep_first) : 0u;
       if (have && XG_BOUND(sr, g.n_states, kBoundState)) {
         ra = *reinterpret_cast<const uint4*>(&g.state[sr]);
         rb = *(reinterpret_cast<const uint4*>(&g.state[sr]) + 1);
@@ -912,7 +938,7 @@ __device__ __forceinline__ int warp_token_walk(const GrammarDev& g, const Chart&
         if (p < total) se = p == first ? make_uint2(e0c, e0t) : g.scan_edge[sb + (p - first)];      // the first edge is inline in the record
         // the record of the edge's target is requested before the byte is tested against the edge's class: if the edge
         // is taken, the new item's `info` word (and the scan of the next byte) find it on its way
-        if (p < total && (se.y & kTarget) < (uint32_t)g.rep_first && XG_BOUND(se.y & kTarget, g.n_states, kBoundState)) asm volatile("prefetch.global.L1 [%0];" ::"l"(&g.state[se.y & kTarget]));
+        if (p < total && (se.y & kTarget) < rep_first && XG_BOUND(se.y & kTarget, g.n_states, kBoundState)) asm volatile("prefetch.global.L1 [%0];" ::"l"(&g.state[se.y & kTarget]));
         bool hit = false;
         if (se.x & kLiteral) hit = (se.x & 0x1FFu) == byte;
         else if (XG_BOUND(se.x, g.n_classes, kBoundClass)) hit = (g.class_bits[se.x * 8 + word] & bit) != 0;
@@ -932,7 +958,7 @@ __device__ __forceinline__ int warp_token_walk(const GrammarDev& g, const Chart&
       const int n_here = min(32, cnt - q);
       uint32_t info = 0;
       int32_t o = 0;
-      if (lane < n_here) { const uint32_t qr = rec_of(g, st[q + lane]); if (XG_BOUND(qr, g.n_states, kBoundState)) { info = g.state[qr].info; o = org[q + lane]; } }
+      if (lane < n_here) { const uint32_t qr = rec_of(g, st[q + lane], rep_first); if (XG_BOUND(qr, g.n_states, kBoundState)) { info = g.state[qr].info; o = org[q + lane]; } }
       uint32_t done = __ballot_sync(kFullWarp, (info >> 31) != 0);
       q += n_here;
       while (done) {
@@ -957,7 +983,8 @@ __device__ __forceinline__ int warp_token_walk(const GrammarDev& g, const Chart&
 // 0 commits the counters and the warp builds the plan of the next mask.  A rejected token leaves
 // the matcher as it was.  With restart_on_eos an accepted end-of-sequence token puts the matcher
 // back into its initial state instead of terminating it.  Returns the status, the same in every lane.
-__device__ __forceinline__ int accept_one(MatcherDev& m, const GrammarDev& g, const VocabDev& v, int tok, bool restart_on_eos, int lane,
+template <typename G>
+__device__ __forceinline__ int accept_one(MatcherDev& m, const G& g, const VocabDev& v, int tok, bool restart_on_eos, int lane,
                                           uint32_t* w_st, int32_t* w_org, int16_t* lsb) {
   int st = 0;   // XG_OK
   // The token's bytes and the request's current set are each a few dependent loads away (id -> rank -> offset ->
@@ -1029,6 +1056,8 @@ __device__ __forceinline__ int accept_one(MatcherDev& m, const GrammarDev& g, co
 
 // One warp per request: requests follow unrelated paths, so sharing a warp between them would
 // serialise their walks.
+// kCounts: some grammar of the batch has counted repetitions (otherwise the decoding of state words compiles away)
+template <bool kCounts>
 __global__ void __launch_bounds__(128)
 accept_kernel(MatcherDev* const* __restrict__ matchers, int batch, VocabDev v,
               const int32_t* __restrict__ token_ids, int32_t* __restrict__ status, int restart_on_eos) {
@@ -1040,7 +1069,7 @@ accept_kernel(MatcherDev* const* __restrict__ matchers, int batch, VocabDev v,
   __shared__ uint32_t sh_st[4][kFastCap];
   __shared__ int32_t sh_org[4][kFastCap];
   __shared__ int16_t sh_lsb[4][kFastMaxBytes + 2];
-  const int st = accept_one(m, *m.grammar, v, token_ids[b], restart_on_eos != 0, lane, sh_st[threadIdx.x >> 5], sh_org[threadIdx.x >> 5], sh_lsb[threadIdx.x >> 5]);
+  const int st = accept_one(m, grammar_as<kCounts>(*m.grammar), v, token_ids[b], restart_on_eos != 0, lane, sh_st[threadIdx.x >> 5], sh_org[threadIdx.x >> 5], sh_lsb[threadIdx.x >> 5]);
   if (status && lane == 0) status[b] = st;
 }
 
@@ -1087,7 +1116,8 @@ __device__ __forceinline__ void for_ids_in_slice(const uint32_t* __restrict__ li
 // is the plain definition -- every token walked against the full Earley state.  The bytes the
 // current set can scan at all (OR of the per-state first-byte sets) reject most tokens before a
 // walk starts.  One warp computes it.
-__device__ __forceinline__ void current_first_bytes(const GrammarDev& g, const Chart& hist, uint32_t* out8, int lane) {
+template <typename G>
+__device__ __forceinline__ void current_first_bytes(const G& g, const Chart& hist, uint32_t* out8, int lane) {
   if (lane < 8) {
     uint32_t w = 0;
     for (int i = 0; i < hist.i_cnt; ++i) w |= g.state_first[(size_t)rec_of(g, hist.i_st[i]) * 8 + lane];
@@ -1120,8 +1150,8 @@ __device__ __forceinline__ bool queue_slow_walk(MatcherDev* m, int token_rank) {
 // The queued tokens, one after the other, by one thread: each walked in full from the request's current set (the
 // plain definition) in the matcher's large scratch; allow(id) records a token that passes.  false: a walk exceeded
 // even that scratch, or the queue had overflowed.
-template <typename F>
-__device__ __forceinline__ bool run_slow_walks(MatcherDev* m, const GrammarDev& g, const VocabDev& v, const Chart& hist, F allow) {
+template <typename F, typename G>
+__device__ __forceinline__ bool run_slow_walks(MatcherDev* m, const G& g, const VocabDev& v, const Chart& hist, F allow) {
   const int n = m->slow_n;
   if (n > kSlowQueue) return false;
   for (int i = 0; i < n; ++i) {
@@ -1464,7 +1494,8 @@ constexpr int kMaxClusterBlocks = 8;      // the portable cluster size limit
 // launched with a cluster of gridDim.x blocks (2, 4 or 8) along x
 // kHeavy: the launch may hold requests with hundreds of uncertain candidates (a grammar of the batch has an entry with
 // a long check list); only then does the kernel carry the second-byte sets and the walk queues described below.
-template <bool kAccept, int kApplyElems, bool kHeavy>
+// kCounts: some grammar of the batch has counted repetitions (Section 3.6); without, state words need no decoding.
+template <bool kAccept, int kApplyElems, bool kHeavy, bool kCounts>
 __global__ void __launch_bounds__(256, 4)
 fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_t* __restrict__ bitmask, long long row_stride,
                     int32_t* __restrict__ status_user, const int32_t* __restrict__ token_ids, int32_t* __restrict__ accept_status,
@@ -1511,7 +1542,7 @@ fill_cluster_kernel(MatcherDev* const* __restrict__ matchers, VocabDev v, int32_
   const int rank = (int)cluster.block_rank();
   MatcherDev* mw = matchers[b];
   const MatcherDev& m = *matchers[b];
-  const GrammarDev& g = *m.grammar;
+  const typename GrammarAs<kCounts>::type& g = grammar_as<kCounts>(*m.grammar);
   const StepPlan& plan = *m.plan;
   const int n_blocks = (int)gridDim.x;
   const int chunk = (v.n_words + n_blocks - 1) / n_blocks;
