@@ -226,3 +226,14 @@ def test_gpu_counted_repetitions_with_a_just_in_time_cache(static_fill):
     s, final, _, stats = _drive(w, 6, "each", static_fill=static_fill)
     assert final["n_built"] > 0 and sum(x["n_states"] for x in stats) < 4 * 1200
     s.close()
+
+
+@pytest.mark.gpu
+def test_gpu_counted_repetitions_at_the_full_vocabulary():
+    """R1024 as bench.py runs it (16 requests, 128 256 tokens, 256 steps): every step of one request and every
+    thirty-second step of all of them against the grammar-text oracle."""
+    from test_gpu_parity import _run_trajectories
+    w = inputs.make_workload("R1024")
+    assert w.vocab.size == 128256 and w.batch == 16
+    compared = _run_trajectories(w, set(range(0, w.steps, 32)), check_requests={11})
+    assert compared >= w.steps
