@@ -28,6 +28,7 @@ COUNTED_CASES = [
     ('root ::= ("a" "b"{2,3}){2,3}', "ab", 9),                        # a counted repetition inside another
     ('root ::= "a"{3,3} | "a"{5,5} "b"', "ab", 7),                    # two of them side by side from one state
     ('root ::= ("a" | "aa"){2,3} "a"', "a", 8),                       # ambiguous: several counts alive at once
+    ('root ::= TagDispatch(("<a", g), stop_strs=("!"))\ng ::= "x"{2,4} ">"', "<ax>!", 6),      # inside a dispatched grammar
 ]
 
 
@@ -75,6 +76,20 @@ def test_state_count_does_not_grow_with_the_bound():
     assert sizes[0] == sizes[1] == sizes[2], sizes
     expanded = B.Grammar(None, "ebnf", 'root ::= "\\"" [a-z0-9 ]{0,1024} "\\""', build_cache=False, repeat_threshold=-1).tables()
     assert expanded["n_states"] > 1024 > sizes[0][0]
+
+
+def test_largest_bounds():
+    """Bounds up to the grammar text's largest number (10^6) are counted with the same handful of states; beyond that
+    the text is refused.  (The count shares the item's 32-bit state word with the state number; a bound that would not
+    fit beside a very large grammar's state numbers is XG_ERR_CAPACITY, never a wrong parse.)"""
+    ok = B.Grammar(None, "ebnf", 'root ::= "a"{0,1000000}', build_cache=False, repeat_threshold=64, repeat_depth=8)
+    assert ok.tables()["rule_rep_hi"].max() == 1000000 and ok.tables()["n_states"] < 10
+    with pytest.raises(B.XgError) as e:
+        B.Grammar(None, "ebnf", 'root ::= "a"{0,2000000000}', build_cache=False, repeat_threshold=64, repeat_depth=8)
+    assert e.value.status == B.XG_ERR_PARSE
+    # without the longest token's length nothing is counted
+    plain = B.Grammar(None, "ebnf", 'root ::= "a"{0,100}', build_cache=False, repeat_threshold=64)
+    assert plain.tables()["rule_rep_hi"].size == 0 and plain.tables()["n_states"] > 100
 
 
 def test_items_carry_the_count():
