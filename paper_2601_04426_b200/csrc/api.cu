@@ -86,7 +86,8 @@ double now_ms() {
 // asynchronous copy from the entry's own pinned staging buffer on the caller's stream.  After the tables have grown
 // to the largest batch in use there is no allocation, no device-wide synchronisation and no blocking copy.
 constexpr int kBatchEntries = 64;
-constexpr int kDefaultRepeatThreshold = 64;   // bounded repetitions of at least this many iterations are counted, not expanded
+constexpr int kDefaultRepeatThreshold = 64;
+constexpr int kShareEntriesFromRepeat = 24;   // explicit states share cache entries (state classes) in grammars with an expanded repetition this long   // bounded repetitions of at least this many iterations are counted, not expanded
 struct BatchSlot {
   std::vector<xg_matcher_t*> key;
   MatcherDev** dev_matchers = nullptr;   // [cap], inside the tokenizer's slab
@@ -486,14 +487,12 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
 #define XG_CUDA_C(expr) do { cudaError_t e__ = (expr); if (e__ != cudaSuccess) { cleanup(); return set_error(XG_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)); } } while (0)
   for (size_t begin = 0; begin < states.size(); begin += per_batch) {
     const int n = (int)std::min<size_t>(per_batch, states.size() - begin);
-    uint32_t* acc = d_rows;
-    uint32_t* unc = d_rows + (size_t)per_batch * W;
-    uint32_t* unr = d_rows + 2 * (size_t)per_batch * W;
+    uint32_t* acc = d_rows;                                      // the three row sets back to back: one clearing call
+    uint32_t* unc = d_rows + (size_t)n * W;
+    uint32_t* unr = d_rows + 2 * (size_t)n * W;
     std::memcpy(h_pos, states.data() + begin, n * sizeof(int32_t));       // (the previous batch ended with a synchronisation)
     XG_CUDA_C(cudaMemcpyAsync(d_pos, h_pos, n * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
-    XG_CUDA_C(cudaMemsetAsync(acc, 0, row_bytes * n, stream));      // blocks with nothing to scan leave their part of the rows untouched
-    XG_CUDA_C(cudaMemsetAsync(unc, 0, row_bytes * n, stream));
-    XG_CUDA_C(cudaMemsetAsync(unr, 0, row_bytes * n, stream));
+    XG_CUDA_C(cudaMemsetAsync(acc, 0, 3 * row_bytes * n, stream));  // blocks with nothing to scan leave their part of the rows untouched
     XG_CUDA_C(cudaMemsetAsync(d_over_count, 0, 2 * sizeof(int), stream));
     std::vector<int2> work;
     classify_work_list(g, states.data() + begin, n, &work);
@@ -1022,7 +1021,9 @@ xg_status_t xg_compile_grammar(const xg_tokenizer_t* tok, xg_cache_pool_t* pool,
   const double t_pre = now_ms();
   try {
     prepared = prepare_interning(f);
-    if (compress && tok->dev.max_len > 0) rep = bounded_equivalence(f, tok->dev.max_len);
+    // (the classes only pay where a repetition of some length was expanded: inside a{0,16} they save a dozen entries
+    // and cost as much host time as hashing the grammar)
+    if (compress && tok->dev.max_len > 0 && f.max_expanded_repeat >= kShareEntriesFromRepeat) rep = bounded_equivalence(f, tok->dev.max_len);
     else for (int s = 0; s < f.n_states; ++s) rep[s] = s;
   } catch (const std::exception& e) {
     return set_error(XG_ERR_OOM, e.what());

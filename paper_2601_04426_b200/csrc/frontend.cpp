@@ -425,6 +425,7 @@ struct Builder {
   std::map<std::string, int> ids;
   std::vector<Fsm> rules;
   int repeat_threshold = 0;               // bounded repetitions with at least this many iterations become counted rules (0: never)
+  int max_expanded = 0;                   // the largest bound among the repetitions expanded into explicit states
   std::map<int, CountedRule> counted;     // rule id -> what it repeats
   std::map<int, Fsm> pending;             // automata of the rules made while another rule is being built (appended afterwards)
 
@@ -499,6 +500,7 @@ struct Builder {
           f.ref(s, rep, t);
           return {s, t};
         }
+        max_expanded = std::max(max_expanded, e.hi < 0 ? e.lo : e.hi);
         int s = f.add(), cur = s;
         for (int i = 0; i < e.lo; ++i) { auto p = frag(f, *e.kids[0]); f.eps(cur, p.first); cur = p.second; }
         int t = f.add();
@@ -1065,6 +1067,7 @@ struct Compiler {
     g.n_rules = (int)order.size();
     g.root_rule = 0;
     g.root_nullable = root_nullable ? 1 : 0;
+    g.max_expanded_repeat = b.max_expanded;
     std::map<ByteSet, int> class_id;
     std::vector<int> base(g.n_rules);
     for (int k = 0; k < g.n_rules; ++k) { base[k] = g.n_states; g.n_states += fsm_of(order[k]).size(); }
@@ -1559,7 +1562,7 @@ FlatGrammar expand_counted_rules(const FlatGrammar& g) {
   r.n_rules = g.n_rules; r.n_classes = g.n_classes; r.root_rule = g.root_rule; r.root_nullable = g.root_nullable;
   r.rule_names = g.rule_names; r.rule_kind = g.rule_kind; r.class_bits = g.class_bits;
   r.rule_rep_lo = g.rule_rep_lo; r.rule_rep_hi = g.rule_rep_hi;
-  r.rep_first = g.rep_first; r.rep_depth = D; r.n_base_states = g.n_base_states;
+  r.rep_first = g.rep_first; r.rep_depth = D; r.n_base_states = g.n_base_states; r.max_expanded_repeat = g.max_expanded_repeat;
   r.rep_shift = 1;
   while ((1ll << r.rep_shift) < g.n_base_states) ++r.rep_shift;
   int hi_max = 0;

@@ -49,6 +49,7 @@ constexpr uint32_t kTargetMask = 0x1FFFFFFFu;
 struct FlatGrammar {
   int32_t n_rules = 0, n_states = 0, n_classes = 0;
   int32_t root_rule = 0, root_nullable = 0;
+  int32_t max_expanded_repeat = 0;                 // the largest bound of a repetition that was expanded into explicit states
   std::vector<std::string> rule_names;
   std::vector<int32_t> rule_start, rule_kind;      // kind 1 = holds a TagDispatch automaton
   std::vector<int32_t> state_rule;

@@ -63,10 +63,10 @@ def test_masks_exact_with_nothing_built():
 def test_masks_exact_while_entries_arrive_between_steps():
     w = inputs.make_workload("C2", steps=120, vocab_size=16384)
     s, final, history, stats = _drive(w, 5, "each")
-    classes = len(np.unique(s.grammars[0].state_classes()[[st for st in range(stats[0]["n_states"])]]))
     assert final["n_built"] > 10 and final["n_in_flight"] == 0
     assert final["n_missing"] > 0, "states the trajectory never visited must stay unbuilt"
-    assert final["n_built"] + final["n_missing"] <= classes
+    # (C2's repetitions are short: its states do not share entries, every scannable state has its own)
+    assert final["n_built"] + final["n_missing"] <= stats[0]["n_scannable"]
     built_so_far = [h["n_built"] for h in history]
     assert built_so_far == sorted(built_so_far) and built_so_far[-1] > built_so_far[2]
     s.close()
