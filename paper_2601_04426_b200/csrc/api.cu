@@ -510,13 +510,13 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
       unsigned long long* d_visits = (unsigned long long*)pool.scratch(8, sizeof(unsigned long long));
       if (!d_visits) return set_error(XG_ERR_OOM, "cache build scratch allocation failed");
       XG_CUDA_C(cudaMemsetAsync(d_visits, 0, sizeof(unsigned long long), stream));
-      if (grid > 0) classify_kernel<true><<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, d_work, acc, unc, unr, d_over, d_over_count, over_cap, d_visits);
+      if (grid > 0) (g->counted ? classify_kernel<true, true> : classify_kernel<true, false>)<<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, d_work, acc, unc, unr, d_over, d_over_count, over_cap, d_visits);
       unsigned long long visits = 0;
       XG_CUDA_C(cudaMemcpyAsync(&visits, d_visits, sizeof visits, cudaMemcpyDeviceToHost, stream));
       XG_CUDA_C(cudaStreamSynchronize(stream));
       g->stats.node_visits += (int64_t)visits;
     } else
-    if (grid > 0) classify_kernel<false><<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, d_work, acc, unc, unr, d_over, d_over_count, over_cap, nullptr);
+    if (grid > 0) (g->counted ? classify_kernel<false, true> : classify_kernel<false, false>)<<<grid, 256, 0, stream>>>(g->host_view, v, d_pos, d_work, acc, unc, unr, d_over, d_over_count, over_cap, nullptr);
     XG_CUDA_C(cudaGetLastError());
     if (ev) cudaEventRecord(ev[1], stream);
     // count and plan are enqueued behind the classification at once; walks that left the fast path are rare, and when
@@ -555,7 +555,7 @@ static xg_status_t build_entries(xg_grammar* g, const std::vector<int32_t>& stat
     uint32_t* arena = (uint32_t*)g->pool->allocate_device((size_t)std::max<long long>(total_words, 1) * 4, &chunk_id);
     if (!arena) { cleanup(); return set_error(XG_ERR_OOM, "cache arena allocation failed"); }
     pack_kernel<<<n, 256, 0, stream>>>(acc, unc, unr, d_plan, V, W, arena, d_entries, nullptr);
-    exit_kernel<<<n, 256, 0, stream>>>(g->host_view, v, d_pos, d_entries, nullptr);
+    (g->counted ? exit_kernel<true> : exit_kernel<false>)<<<n, 256, 0, stream>>>(g->host_view, v, d_pos, d_entries, nullptr);
     XG_CUDA_C(cudaGetLastError());
     std::vector<EntryDev> built(n);
     std::vector<int2> counts(n);
@@ -801,13 +801,13 @@ static xg_status_t jit_enqueue_build(JitPool* jp, xg_grammar* g, const std::vect
     int2* d_work = (int2*)pool.scratch(33, work.size() * sizeof(int2));
     if (!d_work) return set_error(XG_ERR_OOM, "just-in-time scratch allocation failed");
     XG_CUDA(cudaMemcpyAsync(d_work, work.data(), work.size() * sizeof(int2), cudaMemcpyHostToDevice, stream));
-    classify_kernel<false><<<(int)work.size(), 256, 0, stream>>>(g->host_view, v, sc.pos, d_work, acc, unc, unr, sc.over, sc.over_count, 64, nullptr);
+    (g->counted ? classify_kernel<false, true> : classify_kernel<false, false>)<<<(int)work.size(), 256, 0, stream>>>(g->host_view, v, sc.pos, d_work, acc, unc, unr, sc.over, sc.over_count, 64, nullptr);
   }
   count_kernel<<<n, 256, 0, stream>>>(acc, unc, W, sc.counts);
   plan_kernel<<<1, 1024, 0, stream>>>(sc.counts, n, V, W, sc.plan, sc.total);
   jit_reserve_kernel<<<1, 32, 0, stream>>>(sc.plan, n, sc.total, arena->d_used, arena->cap_words, sc.over_count, sc.result);
   pack_kernel<<<n, 256, 0, stream>>>(acc, unc, unr, sc.plan, V, W, arena->base, sc.entries, sc.result);
-  exit_kernel<<<n, 256, 0, stream>>>(g->host_view, v, sc.pos, sc.entries, sc.result);
+  (g->counted ? exit_kernel<true> : exit_kernel<false>)<<<n, 256, 0, stream>>>(g->host_view, v, sc.pos, sc.entries, sc.result);
   jit_publish_kernel<<<(g->flat.n_states + 255) / 256, 256, 0, stream>>>(const_cast<EntryDev*>(g->host_view.entries), j.d_rep, g->flat.n_states,
                                                                          sc.pos, sc.entries, n, sc.result);
   jit_enqueue_narrowing(g, sc, arena, sc.pos, n, sc.result, stream);

@@ -262,9 +262,10 @@ constexpr int kClassifyChunk = 2048;
 
 // kCount: also add up the bytes the walks consume (viable trie nodes visited, without any sharing between tokens)
 // into *visits -- the work the classification actually does, as opposed to the (position, token) pairs it decides.
-template <bool kCount>
+// kCounts: the grammar has counted repetitions (otherwise the decoding of state words compiles away)
+template <bool kCount, bool kCounts>
 __global__ void __launch_bounds__(256)
-classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, const int2* __restrict__ work,
+classify_kernel(GrammarDev g_, VocabDev v, const int32_t* __restrict__ positions, const int2* __restrict__ work,
                 uint32_t* __restrict__ acc_id, uint32_t* __restrict__ unc_id, uint32_t* __restrict__ unc_rank,
                 int2* __restrict__ overflow, int* __restrict__ overflow_count, int overflow_cap, unsigned long long* __restrict__ visits) {
   __shared__ uint32_t sh_st[1];
@@ -272,6 +273,7 @@ classify_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions,
   __shared__ uint32_t sh_class[kSharedClasses * 8];
   __shared__ uint32_t sh_first[8];          // bytes the position's own edges can take
   __shared__ int sh_cum[257];               // sh_cum[b]: viable tokens whose first byte is below b
+  const typename GrammarAs<kCounts>::type& g = grammar_as<kCounts>(g_);
   const int pos = work[blockIdx.x].x, chunk = work[blockIdx.x].y;
   const int state = positions[pos];
   if (threadIdx.x < 8) {
@@ -504,9 +506,11 @@ __device__ __forceinline__ uint32_t first_exit_info(const VocabDev& v, uint32_t 
 // For every uncertain token of every packed entry: the byte offsets at which the token leaves
 // the entry's rule (bit j = after j bytes).  The run-time check restarts there instead of
 // re-walking the part of the token that the cache already decided.  0 = unknown (walk in full).
+template <bool kCounts>
 __global__ void __launch_bounds__(256)
-exit_kernel(GrammarDev g, VocabDev v, const int32_t* __restrict__ positions, const EntryDev* __restrict__ entries, const int* __restrict__ go) {
+exit_kernel(GrammarDev g_, VocabDev v, const int32_t* __restrict__ positions, const EntryDev* __restrict__ entries, const int* __restrict__ go) {
   if (go && !*go) return;
+  const typename GrammarAs<kCounts>::type& g = grammar_as<kCounts>(g_);
   __shared__ uint32_t sh_st[1];
   __shared__ int32_t sh_org[1];
   __shared__ uint32_t sh_class[kSharedClasses * 8];
